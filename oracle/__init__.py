@@ -1,0 +1,24 @@
+"""CPU oracle for Approximate Random Dropout (ARD): TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, fp64 statement of what the hot path computes: the dropout
+pattern (Sec. 3.1 Eq. 1, Sec. 3.2, Sec. 3.4) expanded to a dense 0/1 mask and
+applied to full-size matrix products.  It shares no code with the CUDA path and
+must never be imported by the product package; only the tests, the smoke check
+and the CPU-baseline leg of the benchmark may call it.
+
+Pins (each lives in tests/test_oracle_*.py):
+  pattern.philox4x32_10    known-answer vectors of the published generator
+  pattern.quantise_K       exact integer sum 2^32; zero-probability entries never drawn
+  pattern.draw             Monte-Carlo per-neuron drop rate vs Eq. 2-3; chi^2 of dp; b uniform
+  pattern.row_keep         worked example of Sec. 3.1 (dp=3, b=1); kept fraction 1/dp
+  pattern.tile_keep        worked example of Sec. 3.2 (dp=4, b=1); kept fraction 1/dp
+  gemm.*                   scalar triple loops on tiny shapes; dp=1 == numpy matmul; adjoint identity
+  lstm.*                   dp=1 == torch.nn.LSTM (fp64, forward and autograd gradients);
+                           kept sub-network == torch.nn.LSTM of hidden size n_k; finite differences
+  mlp_chain.*              finite differences of the scalar <dZ3, Z3>
+
+Parity unpinned (the paper fixes no value to compare with): the choice of the
+distribution K itself (the body of Algorithm 1 is not printed), the tile
+linearisation order beyond the first tile of the worked example, the LSTM
+reading (which units are dropped, gate order) and the rescale convention.
+"""
