@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the ARD hot path on B200.
+
+A "step" is one pass of the whole path over one batch: draw a fresh pattern from K on the device,
+then the forward, backward-data and backward-weight GEMMs of the layer over the kept neurons only.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line (rank 0).  Workload `mlp8192_row` is the large MLP layer of the paper's
+Table-1 sweep scaled to B200: W 8192x8192 bf16, batch 4096, row pattern, p = 0.5, K = the
+maximum-entropy distribution over periods 1..16.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2203_05705_b200 import inputs  # noqa: E402
+
+METRIC = "layer fwd+bwd kept TFLOP/s (row pattern, p=0.5)"
+UNIT = "TFLOP/s"
+
+WORKLOADS = {
+    # name: (config, B, K, N, kind, ts, p, n_dp)
+    "mlp8192_row": dict(config=5, B=4096, K=8192, N=8192, kind="row", ts=0, p=0.5, n_dp=16),
+    "mlp8192_tile": dict(config=5, B=4096, K=8192, N=8192, kind="tile", ts=128, p=0.5, n_dp=16),
+    "mlp4096_tile": dict(config=3, B=1024, K=4096, N=4096, kind="tile", ts=64, p=0.5, n_dp=16),
+    "mlp2048_row": dict(config=2, B=128, K=2048, N=2048, kind="row", ts=0, p=0.5, n_dp=16),
+}
+
+# Measured peaks of this machine's B200s (generated file), else the documented fallback.
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def kept_count(units, dp, b):
+    return (units - b) // dp + 1
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            top = sorted(sm)[len(sm) // 2:]           # upper half = samples under load
+            out.update(sm_mhz=statistics.median(top), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_sample_seconds(wl, d, rows=256):
+    """Times the fp64 oracle, as it stands, on a bounded sample of one step: `rows` batch rows of the
+    forward and backward-data products and `rows` neuron columns of the backward-weight product,
+    with the full weight and the dense mask.  Returns (seconds, kept flops of the sample, threads)."""
+    from oracle import gemm as OG
+    from oracle import pattern as OP
+    K, N, B = wl["K"], wl["N"], wl["B"]
+    dp, b = 2, 1
+    mask = OP.row_mask(N, dp, b) if wl["kind"] == "row" else OP.tile_mask(K, N, wl["ts"], dp, b)
+    alpha = 1.0 / (1.0 - wl["p"])
+    sel = np.arange(0, B, max(1, B // rows))[:rows]
+    cols = np.arange(0, N, max(1, N // rows))[:rows]
+    t0 = time.perf_counter()
+    OG.fwd_rows(d["X"], d["W"], mask, alpha, sel)
+    OG.bwd_data_rows(d["dY"], d["W"], mask, alpha, sel)
+    OG.bwd_weight_cols(d["X"], d["dY"], mask, alpha, cols)
+    dt = time.perf_counter() - t0
+    kept_frac = float(np.mean(mask))
+    flops = 2.0 * len(sel) * K * N * kept_frac * 2 + 2.0 * B * K * len(cols) * float(np.mean(mask[..., cols]))
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return dt, flops, threads, f"{len(sel)} of {B} batch rows (fwd, bwd-data) + {len(cols)} of {N} neurons (bwd-weight), dp=2"
+
+
+def run_reference(args, wl):
+    """--impl reference: the CPU oracle on the host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    d = inputs.dense_layer(wl["config"], wl["B"], wl["K"], wl["N"], 1.0 / 90.0)
+    rows = 64
+    for _ in range(args.warmup):
+        oracle_sample_seconds(wl, d, rows)
+    tot_t, tot_f = 0.0, 0.0
+    for _ in range(args.steps):
+        dt, fl, threads, sample = oracle_sample_seconds(wl, d, rows)
+        tot_t += dt
+        tot_f += fl
+    val = tot_f / tot_t / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, **{k: wl[k] for k in ("B", "K", "N", "kind", "p", "n_dp")}},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mlp8192_row", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, wl)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2203_05705_b200 import ard
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    B, K, N, p, n_dp = wl["B"], wl["K"], wl["N"], wl["p"], wl["n_dp"]
+    kind = ard.ARD_ROW if wl["kind"] == "row" else ard.ARD_TILE
+    units = N if kind == ard.ARD_ROW else (K // wl["ts"]) * (N // wl["ts"])
+    d = inputs.dense_layer(wl["config"], B, K, N, 1.0 / 90.0 if wl["config"] == 5 else 1.0 / 64.0)
+    bf = torch.bfloat16
+    hX = torch.from_numpy(d["X"]).to(bf).pin_memory()
+    hdY = torch.from_numpy(d["dY"]).to(bf).pin_memory()
+    X = hX.cuda()
+    dY = hdY.cuda()
+    W = torch.from_numpy(np.ascontiguousarray(d["W"].T)).to(bf).cuda()     # neuron-major [N][K]
+    Y = torch.empty((B, N), dtype=bf, device="cuda")
+    dX = torch.empty((B, K), dtype=bf, device="cuda")
+    dW = torch.zeros((N, K), dtype=bf, device="cuda")
+    hY = torch.empty((B, N), dtype=bf).pin_memory()
+
+    ctx = ard.ard_create(local, 2 * B * N + 4096)
+    pat = ard.ard_pattern_create(ctx, kind, K, N, wl["ts"])
+    dist_ids = {}
+    for i, pp in enumerate((0.3, 0.5, 0.7)):
+        ard.ard_set_distribution(ctx, i, inputs.max_entropy_K(pp, n_dp))
+        dist_ids[pp] = i
+    seed = inputs.BASE_SEED
+
+    def gemms(alpha, ev=None):
+        if ev is not None:
+            ev[0].record()
+        ard.ard_fwd(ctx, pat, ard.ARD_BF16, B, K, N, alpha, X, K, W, K, Y, N, ard.ARD_OUT_SCATTER_ZEROFILL)
+        if ev is not None:
+            ev[1].record()
+        ard.ard_bwd_data(ctx, pat, ard.ARD_BF16, B, K, N, alpha, dY, N, 0, W, K, dX, K)
+        if ev is not None:
+            ev[2].record()
+        ard.ard_bwd_weight(ctx, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, alpha, X, K, dY, N, 0, dW, K, 0)
+        if ev is not None:
+            ev[3].record()
+
+    def step(pp, it, ev=None):
+        ard.ard_sample_pattern(ctx, pat, dist_ids[pp], seed, it, rank)
+        gemms(1.0 / (1.0 - pp), ev)
+
+    def kept_units_of(pp, its):
+        """Host replay of the device sampler's counters, for FLOP accounting only (reads the pattern
+        back after the timed region)."""
+        out = []
+        for it in its:
+            ard.ard_sample_pattern(ctx, pat, dist_ids[pp], seed, it, rank)
+            dp_, b_, nk, _ = ard.ard_pattern_to_host(pat, 0)
+            out.append((dp_, b_, nk))
+        return out
+
+    def timed_run(pp, first_it, per_kernel=False):
+        for w in range(args.warmup):
+            step(pp, first_it + w)
+        its = list(range(first_it + args.warmup, first_it + args.warmup + args.steps))
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in its] if per_kernel else None
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for i, it in enumerate(its):
+            step(pp, it, evs[i] if per_kernel else None)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        per = None
+        if per_kernel:
+            per = [[evs[i][j].elapsed_time(evs[i][j + 1]) for j in range(3)] for i in range(len(its))]
+        return ms, its, per
+
+    def dense_run():
+        ard.ard_pattern_set(ctx, pat, 1, 1)
+        for _ in range(args.warmup):
+            gemms(1.0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            gemms(1.0)
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1)
+
+    def torch_dense_run():
+        Wt = W.t()
+        for _ in range(args.warmup):
+            torch.matmul(X, Wt); torch.matmul(dY, W); torch.matmul(dY.t(), X)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            torch.matmul(X, Wt); torch.matmul(dY, W); torch.matmul(dY.t(), X)
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1)
+
+    # ---- the timed region the headline value comes from (p = 0.5) ----
+    launches0 = ard.ard_launch_count(ctx)
+    clocks = ClockSampler(local)
+    ms, its, per = timed_run(p, 0, per_kernel=True)
+    clk = clocks.stop()
+    launches = (ard.ard_launch_count(ctx) - launches0) * args.steps // (args.steps + args.warmup)
+    status = ard.ard_last_device_status(ctx)
+    pats = kept_units_of(p, its)
+    if kind == ard.ARD_ROW:
+        kept_flops = [3 * 2.0 * B * K * nk for (_, _, nk) in pats]
+    else:
+        kept_flops = [3 * 2.0 * B * wl["ts"] ** 2 * nk for (_, _, nk) in pats]
+    dense_flops = 3 * 2.0 * B * K * N * args.steps
+    kept_tflops = sum(kept_flops) / (ms * 1e-3) / 1e12
+    dense_eq_tflops = dense_flops / (ms * 1e-3) / 1e12
+
+    # max over ranks, sum of work
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_max = float(t.item())
+        f = torch.tensor([sum(kept_flops), dense_flops], device="cuda", dtype=torch.float64)
+        dist.all_reduce(f, op=dist.ReduceOp.SUM)
+        kept_tflops = float(f[0].item()) / (ms_max * 1e-3) / 1e12
+        dense_eq_tflops = float(f[1].item()) / (ms_max * 1e-3) / 1e12
+        ms = ms_max
+
+    # ---- roofline of the tcgen05 GEMM kernel (three launches per step) ----
+    peaks = load_peaks()
+    per = np.array(per)                                  # [steps][3] ms
+    gemm_ms = float(per.sum())
+    op_names = ["fwd", "bwd_data", "bwd_weight"]
+    per_op = {}
+    for j, nm in enumerate(op_names):
+        fl = sum(kept_flops) / 3.0
+        per_op[nm] = {"ms_avg": float(per[:, j].mean()), "tflops": fl / (float(per[:, j].sum()) * 1e-3) / 1e12}
+    achieved = sum(kept_flops) / (gemm_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
+                "peak_source": peaks["source"] + " sustained cuBLAS bf16",
+                "frac_of_burst": achieved / peaks["bf16_tflops"], "kernel": "ard_gemm_tc_kernel",
+                "launches": 3 * args.steps, "per_op": per_op}
+
+    # ---- dense baselines and the other dropout rates (outside the headline region) ----
+    detail = {}
+    dense_ms = dense_run()
+    torch_ms = torch_dense_run()
+    best_dense = min(dense_ms, torch_ms)
+    detail["dense_ms_per_step"] = {"own_kernels_dp1": dense_ms / args.steps, "torch_matmul": torch_ms / args.steps}
+    detail["dense_tflops"] = {"own_kernels_dp1": dense_flops / (dense_ms * 1e-3) / 1e12,
+                              "torch_matmul": dense_flops / (torch_ms * 1e-3) / 1e12}
+    detail["speedup_vs_dense"] = {}
+    detail["kept_fraction"] = {}
+    for pp in (0.3, 0.5, 0.7):
+        if pp == p:
+            ms_p, its_p = ms, its
+            pats_p = pats
+        else:
+            ms_p, its_p, _ = timed_run(pp, 10000)
+            pats_p = kept_units_of(pp, its_p)
+        detail["speedup_vs_dense"][str(pp)] = best_dense / ms_p
+        detail["kept_fraction"][str(pp)] = float(np.mean([nk / units for (_, _, nk) in pats_p]))
+    detail["ideal_speedup"] = {str(pp): 1.0 / (1.0 - pp) for pp in (0.3, 0.5, 0.7)}
+
+    # ---- end to end through the C ABI with host buffers ----
+    h2d = hX.numel() * 2 + hdY.numel() * 2
+    d2h = hY.numel() * 2
+    e2e_steps = max(3, min(args.steps, 20))
+    def e2e_step(it):
+        X.copy_(hX, non_blocking=True)
+        dY.copy_(hdY, non_blocking=True)
+        step(p, it)
+        hY.copy_(Y, non_blocking=True)
+    for w in range(2):
+        e2e_step(20000 + w)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    its_e = list(range(20002, 20002 + e2e_steps))
+    for it in its_e:
+        e2e_step(it)
+    e1.record()
+    barrier()
+    ms_e = e0.elapsed_time(e1)
+    pats_e = kept_units_of(p, its_e)
+    fl_e = sum(3 * 2.0 * B * K * nk for (_, _, nk) in pats_e) if kind == ard.ARD_ROW else \
+        sum(3 * 2.0 * B * wl["ts"] ** 2 * nk for (_, _, nk) in pats_e)
+    e2e_val = fl_e / (ms_e * 1e-3) / 1e12 * world
+    e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "ms_per_step": ms_e / e2e_steps, "steps": e2e_steps}
+
+    # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        dt, fl, threads, sample = oracle_sample_seconds(wl, d, 256)
+        cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+               "seconds": dt}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": kept_tflops, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "B": B, "K": K, "N": N, "kind": wl["kind"], "ts": wl["ts"], "p": p,
+                       "n_dp": n_dp, "l2": "inputs larger than L2 (X, W, dY and outputs: ~0.5 GB per step)",
+                       "replicas": world},
+            "dense_equiv_tflops": dense_eq_tflops, "clocks": clk, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu, "detail": detail, "device_status": int(status),
+        }
+        print(json.dumps(line))
+    ard.ard_pattern_destroy(pat)
+    ard.ard_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

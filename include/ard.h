@@ -1,0 +1,188 @@
+/*
+ * ard.h -- C ABI of the Approximate Random Dropout (ARD) hot path for NVIDIA B200 (sm_100a).
+ *
+ * Method: "DNN Training Acceleration via Exploring GPGPU Friendly Sparsity" (arXiv 2203.05705),
+ * Sec. 3: every training iteration one regular dropout pattern (period dp, bias b) is drawn from a
+ * distribution K over periods; a row pattern drops whole neurons, a tile pattern drops weight tiles
+ * (DropConnect-like); the dropped rows / tiles are never fetched or multiplied.
+ *
+ * Conventions shared by every call
+ *   - Every pointer named X, W, Y, dY, dX, dW, Z, c, h ... is a DEVICE pointer owned by the caller.
+ *     Pointers named K, and every `int32_t* out`-style argument of ard_pattern_to_host /
+ *     ard_pattern_tile_lists_to_host, are HOST pointers.
+ *   - Matrices are row-major.  The weight is stored NEURON-MAJOR: W[N][K] with leading dimension
+ *     ldw (elements); row n holds the K fan-in weights of output neuron n.  This is the transpose
+ *     of the math orientation W[K x N] in Y = X W.  dW has the same layout.
+ *   - `cuda_stream` is a cudaStream_t passed as void*.  Calls only enqueue work; they do not
+ *     synchronise unless stated.  The pattern lives on the device: nothing about it returns to the
+ *     host unless ard_pattern_to_host is called.
+ *   - The library allocates device memory only in ard_create, ard_pattern_create and (once per new
+ *     combination of operand pointer and shape) when it builds and caches TMA descriptor tables
+ *     for the bf16 tensor-core path; everything is freed by the matching destroy call.
+ *   - Every call returns an ard_status.  Problems the host can see (NULL, sizes, leading
+ *     dimensions, alignment, distribution) are rejected before anything is launched.  Problems only
+ *     the device can see (a wait inside a kernel that ran out of patience) set a sticky device
+ *     status word, read with ard_last_device_status; the kernel then exits normally and the output
+ *     of that call is unspecified.  Nothing aborts or traps.
+ *   - Arithmetic: ARD_F32 operands are multiplied and accumulated in fp32 on the CUDA cores;
+ *     ARD_BF16 operands are multiplied on the tensor cores with fp32 accumulation.
+ *   - There is no CPU fallback.
+ */
+#ifndef ARD_H_
+#define ARD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ard_ctx ard_ctx;         /* owns distributions, workspace, descriptor cache, status word */
+typedef struct ard_pattern ard_pattern; /* handle of a device-resident pattern (header + index lists)   */
+
+typedef enum {
+  ARD_OK = 0,
+  ARD_ERR_INVALID_ARG = 1,   /* NULL pointer, negative size, unknown enum value            */
+  ARD_ERR_SHAPE = 2,         /* sizes inconsistent with the pattern, ld < extent, tile size */
+  ARD_ERR_ALIGNMENT = 3,     /* pointer or leading dimension not aligned as the path needs  */
+  ARD_ERR_DISTRIBUTION = 4,  /* K negative / not summing to 1 / longer than the unit count  */
+  ARD_ERR_UNSUPPORTED = 5,
+  ARD_ERR_CUDA = 6,          /* a CUDA runtime or driver call failed                        */
+  ARD_ERR_TIMEOUT = 7,       /* a bounded wait inside a kernel expired (device status)      */
+  ARD_ERR_NOMEM = 8          /* workspace too small or allocation failed                    */
+} ard_status;
+
+typedef enum { ARD_F32 = 0, ARD_BF16 = 1 } ard_dtype;
+typedef enum { ARD_ROW = 0, ARD_TILE = 1 } ard_kind;
+typedef enum { ARD_OUT_COMPACT = 0, ARD_OUT_SCATTER_ZEROFILL = 1 } ard_outmode;
+
+/* Selects the kernel family for ARD_BF16 calls.  AUTO picks the tcgen05 path when the shape and
+ * alignment allow it and the CUDA-core path otherwise; the other two force one family (FORCE_TC
+ * returns ARD_ERR_ALIGNMENT / ARD_ERR_UNSUPPORTED instead of falling back). */
+typedef enum { ARD_PATH_AUTO = 0, ARD_PATH_CUDA_CORE = 1, ARD_PATH_TENSOR_CORE = 2 } ard_path;
+
+#define ARD_MAX_DISTRIBUTIONS 16
+#define ARD_MAX_NDP 4096      /* longest distribution accepted                                  */
+#define ARD_MAX_NDP_TC 32     /* longest period the tensor-core path keeps descriptor tables for */
+
+/* ---- context -------------------------------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device` with `workspace_bytes` of device scratch memory (used
+ * to compact a full-width dY for the tensor-core backward GEMMs; 2*B*N bytes suffice for one
+ * layer).  Synchronous. */
+ard_status ard_create(ard_ctx** ctx, int device, size_t workspace_bytes);
+ard_status ard_destroy(ard_ctx* ctx);
+ard_status ard_set_path(ard_ctx* ctx, ard_path path);
+/* Tuning / test knob of the tensor-core path: forces the N extent of the output tile (64, 128 or
+ * 256; 0 restores the built-in choice).  A forced value a product cannot use is ignored for it. */
+ard_status ard_set_tile_n(ard_ctx* ctx, int bn);
+
+/* Sec. 3.3: the distribution K = {k_i}, i = 1..ndp, over the periods dp, sum k_i = 1.
+ * K: HOST array of ndp doubles, k_i >= 0, |sum - 1| <= 1e-9, 1 <= ndp <= ARD_MAX_NDP.
+ * K is quantised to an integer cumulative table on a 2^32 grid (c_i = floor(s_i 2^32 + 1/2) from
+ * sequential prefix sums s_i, clamped to be non-decreasing, last entry 2^32), which is the
+ * distribution the sampler realises exactly.  Synchronous (small copy).  dist_id in
+ * [0, ARD_MAX_DISTRIBUTIONS). */
+ard_status ard_set_distribution(ard_ctx* ctx, int dist_id, const double* K, int ndp);
+/* Copies the quantised cumulative table (ndp entries, HOST uint64) back, for tests. */
+ard_status ard_get_distribution_cdf(ard_ctx* ctx, int dist_id, uint64_t* cdf_out, int capacity, int* ndp_out);
+
+/* ---- pattern --------------------------------------------------------------------------------- */
+
+/* A pattern object for a weight of math shape [K_dim x N_dim].
+ *   ARD_ROW  (Sec. 3.1): units = the N_dim output neurons; `tile` must be 0.
+ *   ARD_TILE (Sec. 3.2): units = the (K_dim/tile) x (N_dim/tile) weight tiles, numbered row-major
+ *                        from 1 over (r, c) with r along K and c along N; tile must divide both. */
+ard_status ard_pattern_create(ard_ctx* ctx, ard_pattern** pat, ard_kind kind, int K_dim, int N_dim, int tile);
+ard_status ard_pattern_destroy(ard_pattern* pat);
+
+/* Sec. 3.4: draws dp from distribution `dist_id`, then b uniformly from {1..dp}, and writes the
+ * kept-unit lists (Eq. 1: unit i, 1-based, is kept iff (i - b) mod dp == 0) into the pattern, all
+ * on the device, asynchronously on `cuda_stream`.
+ * Randomness: Philox4x32-10 with key (seed low, seed high) and counter (iteration low, iteration
+ * high, stream_id, 0); word 0 selects dp as the smallest i with word0 < c_i, word 1 selects
+ * b = 1 + floor(word1 * dp / 2^32).  The result is a pure function of (table, seed, iteration,
+ * stream_id, shape).  Returns ARD_ERR_DISTRIBUTION if the distribution is unset or longer than
+ * the pattern's unit count. */
+ard_status ard_sample_pattern(ard_ctx* ctx, ard_pattern* pat, int dist_id, uint64_t seed,
+                              uint64_t iteration, uint32_t stream_id, void* cuda_stream);
+
+/* Sets (dp, b) explicitly (1 <= b <= dp <= units) and emits the same lists; for tests and for
+ * running a layer dense (dp = 1).  Asynchronous. */
+ard_status ard_pattern_set(ard_ctx* ctx, ard_pattern* pat, int dp, int b, void* cuda_stream);
+
+/* Test / debug: synchronises the stream and copies dp, b, the number of kept units and the kept
+ * list (row: 0-based neuron indices; tile: 0-based linear tile indices t-1, ascending) to HOST
+ * buffers.  idx may be NULL; at most idx_capacity entries are written. */
+ard_status ard_pattern_to_host(const ard_pattern* pat, int32_t* dp, int32_t* b, int32_t* n_keep,
+                               int32_t* idx, size_t idx_capacity, void* cuda_stream);
+/* Tile patterns only: the kept tiles grouped by tile-column (col_ptr[Tc+1], col_idx = tile-rows
+ * ascending) and by tile-row (row_ptr[Tr+1], row_idx = tile-columns ascending).  HOST buffers;
+ * col_idx / row_idx need room for Tr*Tc entries.  Synchronises. */
+ard_status ard_pattern_tile_lists_to_host(const ard_pattern* pat, int32_t* col_ptr, int32_t* col_idx,
+                                          int32_t* row_ptr, int32_t* row_idx, void* cuda_stream);
+
+/* ---- the three GEMMs (Sec. 3.1 / 3.2: only kept rows / tiles are fetched and multiplied) ------ */
+
+/* Forward:  Y = alpha * X * (W .* Mask(pattern)).
+ *   X [B][K] (ldx), W [N][K] neuron-major (ldw).
+ *   Row pattern, ARD_OUT_SCATTER_ZEROFILL: Y [B][N] (ldy), dropped columns written as zero.
+ *   Row pattern, ARD_OUT_COMPACT: Y [B][n_keep] (ldy >= N so that any pattern fits): column j holds
+ *     kept neuron j; columns >= n_keep are not written.
+ *   Tile pattern: Y [B][N] always full (outmode ignored).
+ *   alpha is the rescale the caller wants fused (1/(1-p) for inverted dropout). */
+ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N, float alpha,
+                   const void* X, int ldx, const void* W, int ldw, void* Y, int ldy, ard_outmode outmode,
+                   void* cuda_stream);
+
+/* Backward-data:  dX = alpha * dY * (W .* Mask)^T,  dX [B][K] (lddx).
+ *   dy_is_compact = 0: dY [B][N] full width, dropped columns are ignored (never read as values).
+ *   dy_is_compact = 1 (row pattern only): dY [B][n_keep] with column j belonging to kept neuron j. */
+ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N, float alpha,
+                        const void* dY, int lddy, int dy_is_compact, const void* W, int ldw, void* dX, int lddx,
+                        void* cuda_stream);
+
+/* Backward-weight:  dW = alpha * (X^T dY) .* Mask, stored neuron-major dW [N][K] (lddw), element
+ *   type dW_dtype (fp32 or bf16; an ARD_F32 layer requires ARD_F32).  Only kept rows (row pattern)
+ *   or kept tiles (tile pattern) are computed and written; if zero_fill_dropped != 0 the dropped
+ *   rows / tiles are written as zero, otherwise they are left untouched. */
+ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, ard_dtype dW_dtype, int B, int K,
+                          int N, float alpha, const void* X, int ldx, const void* dY, int lddy, int dy_is_compact,
+                          void* dW, int lddw, int zero_fill_dropped, void* cuda_stream);
+
+/* ---- LSTM cell on the kept hidden units (Sec. 7: an LSTM step is again a matrix
+ * product; one row pattern over the H hidden units serves every time step) -------------
+ * Layouts are compact over kept units: with n = n_keep, Z [B][4*ldz_gate] holds the gate
+ * pre-activations in four blocks i | f | g | o of width ldz_gate (>= n; block g starts at column
+ * g*ldz_gate), bias [4][H] is indexed by the ORIGINAL unit (may be NULL), c_prev / c [B][ldc] and
+ * gates_saved [B][4*ldc] are fp32, h [B][ldh] has element type h_dtype.
+ *   i,f,o = sigmoid, g = tanh;  c = f*c_prev + i*g;  h = alpha * o * tanh(c)
+ * h_scatter != 0 writes h full width [B][H] with zeros at dropped units (the layout the next
+ * step's recurrent GEMM consumes), else compact [B][n]. */
+ard_status ard_lstm_gates(ard_ctx* ctx, const ard_pattern* pat, ard_dtype h_dtype, int B, int H, float alpha,
+                          const float* Z, int ldz_gate, const float* bias, const float* c_prev, int ldc, float* c,
+                          void* h, int ldh, int h_scatter, float* gates_saved, void* cuda_stream);
+
+/* Adjoint of ard_lstm_gates.  dh [B][lddh] (fp32; compact, or full width if dh_scatter != 0, in
+ * which case only kept columns are read), dc_inout [B][ldc]: in = gradient arriving at c from the
+ * next step, out = gradient w.r.t. c_prev.  dZ [B][4*ldz_gate] compact like Z, element type
+ * dz_dtype. */
+ard_status ard_lstm_gates_bwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dz_dtype, int B, int H, float alpha,
+                              const float* gates_saved, const float* c_prev, const float* c, int ldc,
+                              const float* dh, int lddh, int dh_scatter, float* dc_inout, void* dZ, int ldz_gate,
+                              void* cuda_stream);
+
+/* ---- status ---------------------------------------------------------------------------------- */
+
+/* Synchronises `cuda_stream`, returns the sticky device status word (ARD_OK if no kernel reported
+ * a problem) and clears it. */
+ard_status ard_last_device_status(ard_ctx* ctx, void* cuda_stream);
+const char* ard_status_string(ard_status s);
+/* Number of kernels this library has launched on behalf of `ctx` since creation. */
+uint64_t ard_launch_count(const ard_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ARD_H_ */

@@ -3,8 +3,8 @@
 TEST INFRASTRUCTURE ONLY (see oracle/__init__.py).  fp64 numpy.
 
 Orientation: X[B x K], W[K x N] (math orientation, Y = X W), dY[B x N].
-Sec. 3.1: only the kept rows are fetched and multiplied and "the rest of the
-output matrix is set to zero", i.e. the result equals the product with the
+Sec. 3.1: only the kept rows are fetched and multiplied and every other entry
+of the output is zero, i.e. the result equals the product with the
 dropped part of W replaced by zeros.  The backward products are the exact
 adjoints of that forward map (the paper states only that forward and backward
 are both accelerated).

@@ -2,10 +2,10 @@
 
 TEST INFRASTRUCTURE ONLY (see oracle/__init__.py).  fp64 numpy.
 
-The paper says only that the LSTM "is also performed as matrix
-multiplication" (Sec. 7, LSTM experiment) and that one pattern serves a whole
+The paper gives no LSTM equations: it only notes that an LSTM step is again a
+matrix product (Sec. 7, LSTM experiment) and that one pattern serves a whole
 iteration.  Reading used here: the row pattern of Sec. 3.1 is applied to the H
-hidden units ("drop all the synapses of a dropped neuron"), the same pattern at
+hidden units (a dropped unit loses all of its synapses), the same pattern at
 every time step; gate blocks are ordered i | f | g | o, no peepholes.
 
   z_t = [x_t, h_{t-1}] W + bias                W: [(I+H) x 4H]

@@ -6,8 +6,8 @@ TEST INFRASTRUCTURE ONLY (see oracle/__init__.py).  fp64 numpy.
 The paper's step is fully connected layer -> activation -> (skipped) dropout
 layer (Sec. 3.2, last paragraph).  Reading: ReLU activation, no bias,
 relu'(0) = 0; a dropped hidden neuron outputs exactly zero, so the consumer
-layer may also skip the matching input column (Sec. 3.1: "the correspondent
-row in the weight matrix of next layer").
+layer may also skip the matching input column (Sec. 3.1 describes a
+dropped neuron as removing its row of the next layer's weight).
 """
 from __future__ import annotations
 

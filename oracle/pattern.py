@@ -11,7 +11,7 @@ TWO32 = 1 << 32
 MASK32 = TWO32 - 1
 
 # ---------------------------------------------------------------------------
-# Counter-based generator.  The paper (Sec. 3.4) only says "randomly sample";
+# Counter-based generator.  The paper (Sec. 3.4) does not name a generator;
 # both sides of the parity test implement the published Philox4x32-10
 # generator (Salmon et al., SC'11) so that draws can be compared bit for bit.
 # ---------------------------------------------------------------------------
@@ -122,8 +122,8 @@ def row_mask(n_units, dp, b):
 
 
 # ---------------------------------------------------------------------------
-# Sec. 3.2: the same (dp, b) rule over weight tiles: of every dp successive
-# tiles, dp-1 are dropped.  The weight is taken in its math orientation
+# Sec. 3.2: the same (dp, b) rule over weight tiles: out of each run of dp
+# consecutive tiles only one survives.  The weight is taken in its math orientation
 # W[K x N] (Y = X W); tile (r, c) covers rows r*ts.. and columns c*ts..; tiles
 # are numbered row-major from 1: t = r*Tc + c + 1.
 # ---------------------------------------------------------------------------

@@ -1,0 +1,599 @@
+// C-ABI entry points: argument validation, context / pattern lifetime, the TMA descriptor cache and
+// the dispatch between the CUDA-core and tcgen05 kernel families.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+
+#include "ard_internal.h"
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok;
+  explicit DeviceGuard(int dev) {
+    ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+// One bf16 descriptor: [rows][cols] with a row pitch of pitch_bytes, 128-byte swizzle, zero fill
+// outside the extents (which is what drops the rows / columns beyond n_keep for free).
+bool encode_map(ard_ctx* ctx, CUtensorMap* out, const void* base, uint64_t cols, uint64_t rows, uint64_t pitch_bytes,
+                uint32_t box_cols, uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_fn)(
+      out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+constexpr size_t MAX_CACHED_TABLES = 96;
+
+// Returns a device table of descriptors for `base`; builds and caches it on first use.
+ard_status get_maps(ard_ctx* ctx, const void* base, int rows, int cols, int ld, int units, int variant, int dp_bound,
+                    int box_rows, int box_cols, const CUtensorMap** out) {
+  for (const MapTable& t : ctx->maps) {
+    if (t.base == base && t.rows == rows && t.cols == cols && t.ld == ld && t.elem_bytes == units &&
+        t.variant == variant && t.dp_bound == dp_bound && t.box_rows == box_rows && t.box_cols == box_cols) {
+      *out = t.d_maps;
+      return ARD_OK;
+    }
+  }
+  const int count = variant == MAP_PLAIN ? 1 : map_index_count(dp_bound);
+  std::vector<CUtensorMap> h(count);
+  const char* cbase = reinterpret_cast<const char*>(base);
+  if (variant == MAP_PLAIN) {
+    if (!encode_map(ctx, &h[0], base, cols, rows, (uint64_t)ld * 2, box_cols, box_rows)) return ARD_ERR_CUDA;
+  } else {
+    for (int dp = 1; dp <= dp_bound; ++dp)
+      for (int b = 1; b <= dp; ++b) {
+        int nk = units >= b ? (units - b) / dp + 1 : 1;
+        CUtensorMap* m = &h[dp * (dp - 1) / 2 + (b - 1)];
+        bool ok;
+        if (variant == MAP_STRIDED_ROWS) {
+          // kept neurons b-1, b-1+dp, ...: base moved to row b-1, pitch dp rows, exactly nk rows
+          ok = units >= b ? encode_map(ctx, m, cbase + (size_t)(b - 1) * ld * 2, cols, nk, (uint64_t)dp * ld * 2,
+                                       box_cols, box_rows)
+                          : encode_map(ctx, m, base, cols, 1, (uint64_t)ld * 2, box_cols, box_rows);
+        } else {
+          // compact matrix: all rows, columns 0..nk-1
+          ok = encode_map(ctx, m, base, nk, rows, (uint64_t)ld * 2, box_cols, box_rows);
+        }
+        if (!ok) return ARD_ERR_CUDA;
+      }
+  }
+  if (ctx->maps.size() >= MAX_CACHED_TABLES) {
+    // cudaFree synchronises the device, so no kernel can still be reading the evicted table.
+    cudaFree(ctx->maps.front().d_maps);
+    ctx->maps.erase(ctx->maps.begin());
+  }
+  MapTable t;
+  t.base = base; t.rows = rows; t.cols = cols; t.ld = ld; t.elem_bytes = units; t.variant = variant;
+  t.dp_bound = dp_bound; t.box_rows = box_rows; t.box_cols = box_cols; t.count = count;
+  t.d_maps = nullptr;
+  if (cudaMalloc(&t.d_maps, sizeof(CUtensorMap) * count) != cudaSuccess) return ARD_ERR_NOMEM;
+  if (cudaMemcpy(t.d_maps, h.data(), sizeof(CUtensorMap) * count, cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaFree(t.d_maps);
+    return ARD_ERR_CUDA;
+  }
+  ctx->maps.push_back(t);
+  *out = t.d_maps;
+  return ARD_OK;
+}
+
+ard_status check_common(ard_ctx* ctx, const ard_pattern* pat, int B, int K, int N) {
+  if (!ctx || !pat) return ARD_ERR_INVALID_ARG;
+  if (pat->ctx != ctx) return ARD_ERR_INVALID_ARG;
+  if (B < 0 || K < 0 || N < 0) return ARD_ERR_INVALID_ARG;
+  if (K != pat->K_dim || N != pat->N_dim) return ARD_ERR_SHAPE;
+  if (B > 65535 * 32) return ARD_ERR_UNSUPPORTED;
+  return ARD_OK;
+}
+
+void fill_common(GemmArgs& g, ard_ctx* ctx, const ard_pattern* pat, int B, int K, int N, float alpha) {
+  g.hdr = pat->d_hdr;
+  g.idx = pat->d_idx;
+  g.col_ptr = pat->d_col_ptr;
+  g.col_idx = pat->d_col_idx;
+  g.row_ptr = pat->d_row_ptr;
+  g.row_idx = pat->d_row_idx;
+  g.B = B; g.K = K; g.N = N;
+  g.alpha = alpha;
+  g.flag0 = g.flag1 = 0;
+  g.out_is_f32 = 0;
+  g.status = ctx->d_status;
+}
+
+// Can the tcgen05 path take this call?  (bf16 only; 16-byte aligned pointers and pitches; the
+// period bounded by the descriptor-table size.)
+ard_status tc_eligible(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N,
+                       const void* p0, int ld0, const void* p1, int ld1, const void* po, int ldo, int out_es) {
+  if (dtype != ARD_BF16) return ARD_ERR_UNSUPPORTED;
+  if (ctx->encode_fn == nullptr) return ARD_ERR_UNSUPPORTED;
+  if (B < 1 || K < 1 || N < 1) return ARD_ERR_UNSUPPORTED;
+  if (pat->kind == ARD_ROW && pat->dp_bound > ARD_MAX_NDP_TC) return ARD_ERR_UNSUPPORTED;
+  if (pat->kind == ARD_TILE && pat->ts % 64 != 0) return ARD_ERR_UNSUPPORTED;
+  if (!aligned16(p0) || !aligned16(p1) || !aligned16(po)) return ARD_ERR_ALIGNMENT;
+  if (ld0 % 8 || ld1 % 8 || ((size_t)ldo * out_es) % 16) return ARD_ERR_ALIGNMENT;
+  if (K % 8 || N % 8) return ARD_ERR_ALIGNMENT;
+  return ARD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* ard_status_string(ard_status s) {
+  switch (s) {
+    case ARD_OK: return "ok";
+    case ARD_ERR_INVALID_ARG: return "invalid argument";
+    case ARD_ERR_SHAPE: return "shape mismatch";
+    case ARD_ERR_ALIGNMENT: return "misaligned pointer or leading dimension";
+    case ARD_ERR_DISTRIBUTION: return "invalid pattern distribution";
+    case ARD_ERR_UNSUPPORTED: return "unsupported configuration";
+    case ARD_ERR_CUDA: return "CUDA call failed";
+    case ARD_ERR_TIMEOUT: return "bounded device wait expired";
+    case ARD_ERR_NOMEM: return "out of memory or workspace too small";
+  }
+  return "unknown status";
+}
+
+ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
+  if (!out || device < 0) return ARD_ERR_INVALID_ARG;
+  *out = nullptr;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device >= ndev) return ARD_ERR_CUDA;
+  DeviceGuard guard(device);
+  if (!guard.ok) return ARD_ERR_CUDA;
+  ard_ctx* ctx = new (std::nothrow) ard_ctx();
+  if (!ctx) return ARD_ERR_NOMEM;
+  ctx->device = device;
+  ctx->path = ARD_PATH_AUTO;
+  ctx->force_bn = 0;
+  ctx->workspace_bytes = workspace_bytes;
+  ctx->d_workspace = nullptr;
+  ctx->d_status = nullptr;
+  ctx->launches = 0;
+  ctx->encode_fn = nullptr;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return ARD_ERR_CUDA; }
+  ctx->sm_count = prop.multiProcessorCount;
+  if (prop.major == 10) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      ctx->encode_fn = fn;
+  }
+  if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess) { delete ctx; return ARD_ERR_NOMEM; }
+  cudaMemset(ctx->d_status, 0, sizeof(int));
+  if (workspace_bytes > 0 && cudaMalloc(&ctx->d_workspace, workspace_bytes) != cudaSuccess) {
+    cudaFree(ctx->d_status);
+    delete ctx;
+    return ARD_ERR_NOMEM;
+  }
+  *out = ctx;
+  return ARD_OK;
+}
+
+ard_status ard_destroy(ard_ctx* ctx) {
+  if (!ctx) return ARD_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaDeviceSynchronize();
+  for (MapTable& t : ctx->maps) cudaFree(t.d_maps);
+  for (int i = 0; i < ARD_MAX_DISTRIBUTIONS; ++i)
+    if (ctx->dist[i].d_cdf) cudaFree(ctx->dist[i].d_cdf);
+  if (ctx->d_workspace) cudaFree(ctx->d_workspace);
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  delete ctx;
+  return ARD_OK;
+}
+
+ard_status ard_set_path(ard_ctx* ctx, ard_path path) {
+  if (!ctx || path < ARD_PATH_AUTO || path > ARD_PATH_TENSOR_CORE) return ARD_ERR_INVALID_ARG;
+  ctx->path = path;
+  return ARD_OK;
+}
+
+ard_status ard_set_tile_n(ard_ctx* ctx, int bn) {
+  if (!ctx || (bn != 0 && bn != 64 && bn != 128 && bn != 256)) return ARD_ERR_INVALID_ARG;
+  ctx->force_bn = bn;
+  return ARD_OK;
+}
+
+ard_status ard_set_distribution(ard_ctx* ctx, int dist_id, const double* K, int ndp) {
+  if (!ctx || !K) return ARD_ERR_INVALID_ARG;
+  if (dist_id < 0 || dist_id >= ARD_MAX_DISTRIBUTIONS) return ARD_ERR_INVALID_ARG;
+  if (ndp < 1 || ndp > ARD_MAX_NDP) return ARD_ERR_DISTRIBUTION;
+  double sum = 0.0;
+  for (int i = 0; i < ndp; ++i) {
+    if (!(K[i] >= 0.0)) return ARD_ERR_DISTRIBUTION;  // also rejects NaN
+    sum += K[i];
+  }
+  if (!(fabs(sum - 1.0) <= 1e-9)) return ARD_ERR_DISTRIBUTION;
+  // Integer cumulative table on a 2^32 grid from sequential prefix sums.
+  std::vector<unsigned long long> cdf(ndp);
+  const unsigned long long TOP = 1ull << 32;
+  double s = 0.0;
+  unsigned long long prev = 0;
+  for (int i = 0; i < ndp; ++i) {
+    s += K[i];
+    unsigned long long c;
+    if (i == ndp - 1) c = TOP;
+    else {
+      double v = floor(s * 4294967296.0 + 0.5);
+      c = v <= 0.0 ? 0ull : (v >= 4294967296.0 ? TOP : (unsigned long long)v);
+      if (c < prev) c = prev;
+      if (c > TOP) c = TOP;
+    }
+    cdf[i] = c;
+    prev = c;
+  }
+  DeviceGuard guard(ctx->device);
+  ArdDistribution& d = ctx->dist[dist_id];
+  if (d.d_cdf) {
+    cudaDeviceSynchronize();
+    cudaFree(d.d_cdf);
+    d.d_cdf = nullptr;
+    d.ndp = 0;
+  }
+  if (cudaMalloc(&d.d_cdf, sizeof(unsigned long long) * ndp) != cudaSuccess) return ARD_ERR_NOMEM;
+  ARD_CUDA_OK(cudaMemcpy(d.d_cdf, cdf.data(), sizeof(unsigned long long) * ndp, cudaMemcpyHostToDevice));
+  d.h_cdf = cdf;
+  d.ndp = ndp;
+  return ARD_OK;
+}
+
+ard_status ard_get_distribution_cdf(ard_ctx* ctx, int dist_id, uint64_t* cdf_out, int capacity, int* ndp_out) {
+  if (!ctx || !ndp_out || dist_id < 0 || dist_id >= ARD_MAX_DISTRIBUTIONS) return ARD_ERR_INVALID_ARG;
+  const ArdDistribution& d = ctx->dist[dist_id];
+  if (d.ndp == 0) return ARD_ERR_DISTRIBUTION;
+  *ndp_out = d.ndp;
+  if (cdf_out)
+    for (int i = 0; i < d.ndp && i < capacity; ++i) cdf_out[i] = d.h_cdf[i];
+  return ARD_OK;
+}
+
+ard_status ard_pattern_create(ard_ctx* ctx, ard_pattern** out, ard_kind kind, int K_dim, int N_dim, int tile) {
+  if (!ctx || !out) return ARD_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (kind != ARD_ROW && kind != ARD_TILE) return ARD_ERR_INVALID_ARG;
+  if (K_dim < 1 || N_dim < 1) return ARD_ERR_SHAPE;
+  if (kind == ARD_ROW && tile != 0) return ARD_ERR_SHAPE;
+  if (kind == ARD_TILE && (tile < 1 || K_dim % tile || N_dim % tile)) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  ard_pattern* p = new (std::nothrow) ard_pattern();
+  if (!p) return ARD_ERR_NOMEM;
+  p->ctx = ctx;
+  p->kind = kind;
+  p->K_dim = K_dim;
+  p->N_dim = N_dim;
+  p->ts = tile;
+  p->Tr = kind == ARD_TILE ? K_dim / tile : 0;
+  p->Tc = kind == ARD_TILE ? N_dim / tile : 0;
+  const long long units = kind == ARD_TILE ? (long long)p->Tr * p->Tc : N_dim;
+  if (units > (1ll << 30)) { delete p; return ARD_ERR_UNSUPPORTED; }
+  p->units = (int)units;
+  p->dp_bound = 1;
+  size_t words = HDR_WORDS + (size_t)p->units;
+  if (kind == ARD_TILE) words += (size_t)(p->Tc + 1) + (size_t)(p->Tr + 1) + 2 * (size_t)p->units;
+  int32_t* d = nullptr;
+  if (cudaMalloc(&d, words * sizeof(int32_t)) != cudaSuccess) { delete p; return ARD_ERR_NOMEM; }
+  cudaMemset(d, 0, words * sizeof(int32_t));
+  p->d_hdr = d;
+  p->d_idx = d + HDR_WORDS;
+  if (kind == ARD_TILE) {
+    p->d_col_ptr = p->d_idx + p->units;
+    p->d_col_idx = p->d_col_ptr + (p->Tc + 1);
+    p->d_row_ptr = p->d_col_idx + p->units;
+    p->d_row_idx = p->d_row_ptr + (p->Tr + 1);
+  } else {
+    p->d_col_ptr = p->d_col_idx = p->d_row_ptr = p->d_row_idx = nullptr;
+  }
+  *out = p;
+  // A fresh pattern is dense (dp = 1) until sampled.
+  return ard_pattern_set(ctx, p, 1, 1, nullptr);
+}
+
+ard_status ard_pattern_destroy(ard_pattern* pat) {
+  if (!pat) return ARD_ERR_INVALID_ARG;
+  DeviceGuard guard(pat->ctx->device);
+  cudaDeviceSynchronize();
+  cudaFree(pat->d_hdr);
+  delete pat;
+  return ARD_OK;
+}
+
+ard_status ard_sample_pattern(ard_ctx* ctx, ard_pattern* pat, int dist_id, uint64_t seed, uint64_t iteration,
+                              uint32_t stream_id, void* cuda_stream) {
+  if (!ctx || !pat || pat->ctx != ctx) return ARD_ERR_INVALID_ARG;
+  if (dist_id < 0 || dist_id >= ARD_MAX_DISTRIBUTIONS) return ARD_ERR_INVALID_ARG;
+  const ArdDistribution& d = ctx->dist[dist_id];
+  if (d.ndp == 0 || d.ndp > pat->units) return ARD_ERR_DISTRIBUTION;
+  DeviceGuard guard(ctx->device);
+  pat->dp_bound = d.ndp;
+  return launch_sampler(ctx, pat, d.d_cdf, d.ndp, seed, iteration, stream_id, 0, 0, (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_pattern_set(ard_ctx* ctx, ard_pattern* pat, int dp, int b, void* cuda_stream) {
+  if (!ctx || !pat || pat->ctx != ctx) return ARD_ERR_INVALID_ARG;
+  if (dp < 1 || b < 1 || b > dp || dp > pat->units) return ARD_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  pat->dp_bound = dp;
+  return launch_sampler(ctx, pat, nullptr, 0, 0, 0, 0, dp, b, (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_pattern_to_host(const ard_pattern* pat, int32_t* dp, int32_t* b, int32_t* n_keep, int32_t* idx,
+                               size_t idx_capacity, void* cuda_stream) {
+  if (!pat) return ARD_ERR_INVALID_ARG;
+  DeviceGuard guard(pat->ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  int32_t hdr[HDR_WORDS];
+  ARD_CUDA_OK(cudaMemcpyAsync(hdr, pat->d_hdr, sizeof(hdr), cudaMemcpyDeviceToHost, s));
+  ARD_CUDA_OK(cudaStreamSynchronize(s));
+  if (dp) *dp = hdr[HDR_DP];
+  if (b) *b = hdr[HDR_B];
+  if (n_keep) *n_keep = hdr[HDR_NKEEP];
+  if (idx && idx_capacity > 0) {
+    size_t n = (size_t)hdr[HDR_NKEEP] < idx_capacity ? (size_t)hdr[HDR_NKEEP] : idx_capacity;
+    ARD_CUDA_OK(cudaMemcpyAsync(idx, pat->d_idx, n * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    ARD_CUDA_OK(cudaStreamSynchronize(s));
+  }
+  return ARD_OK;
+}
+
+ard_status ard_pattern_tile_lists_to_host(const ard_pattern* pat, int32_t* col_ptr, int32_t* col_idx,
+                                          int32_t* row_ptr, int32_t* row_idx, void* cuda_stream) {
+  if (!pat || !col_ptr || !col_idx || !row_ptr || !row_idx) return ARD_ERR_INVALID_ARG;
+  if (pat->kind != ARD_TILE) return ARD_ERR_INVALID_ARG;
+  DeviceGuard guard(pat->ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  ARD_CUDA_OK(cudaMemcpyAsync(col_ptr, pat->d_col_ptr, (pat->Tc + 1) * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  ARD_CUDA_OK(cudaMemcpyAsync(row_ptr, pat->d_row_ptr, (pat->Tr + 1) * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  ARD_CUDA_OK(cudaMemcpyAsync(col_idx, pat->d_col_idx, (size_t)pat->units * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  ARD_CUDA_OK(cudaMemcpyAsync(row_idx, pat->d_row_idx, (size_t)pat->units * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  ARD_CUDA_OK(cudaStreamSynchronize(s));
+  return ARD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------------
+
+ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N, float alpha,
+                   const void* X, int ldx, const void* W, int ldw, void* Y, int ldy, ard_outmode outmode,
+                   void* cuda_stream) {
+  ard_status st = check_common(ctx, pat, B, K, N);
+  if (st != ARD_OK) return st;
+  if (!X || !W || !Y) return ARD_ERR_INVALID_ARG;
+  if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (outmode != ARD_OUT_COMPACT && outmode != ARD_OUT_SCATTER_ZEROFILL) return ARD_ERR_INVALID_ARG;
+  if (ldx < K || ldw < K || ldy < N) return ARD_ERR_SHAPE;
+  if (B == 0) return ARD_OK;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int es = dtype == ARD_F32 ? 4 : 2;
+
+  GemmArgs g;
+  fill_common(g, ctx, pat, B, K, N, alpha);
+  g.A0 = X; g.lda0 = ldx; g.A1 = W; g.lda1 = ldw; g.out = Y; g.ldo = ldy;
+  g.flag0 = pat->kind == ARD_ROW ? (int)outmode : 0;
+  g.out_is_f32 = dtype == ARD_F32;
+
+  ard_status el = ctx->path == ARD_PATH_CUDA_CORE ? ARD_ERR_UNSUPPORTED
+                                                  : tc_eligible(ctx, pat, dtype, B, K, N, X, ldx, W, ldw, Y, ldy, es);
+  if (el != ARD_OK) {
+    if (ctx->path == ARD_PATH_TENSOR_CORE) return el;
+    return launch_gemm_cc(ctx, pat->kind, OP_FWD, dtype, g, pat->ts, s);
+  }
+  TcArgs t;
+  t.g = g;
+  t.ts = pat->ts;
+  t.bn = tc_pick_bn(ctx, pat->kind, OP_FWD, B, K, N, pat->ts);
+  // A = X, K-major boxes [128 rows][64 k];  B = kept neurons of W, K-major boxes [bn rows][64 k].
+  st = get_maps(ctx, X, B, K, ldx, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);
+  if (st != ARD_OK) return st;
+  t.mapA_indexed = 0;
+  if (pat->kind == ARD_ROW) {
+    st = get_maps(ctx, W, N, K, ldw, N, MAP_STRIDED_ROWS, pat->dp_bound, t.bn, 64, &t.mapB);
+    t.mapB_indexed = 1;
+  } else {
+    st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, t.bn, 64, &t.mapB);
+    t.mapB_indexed = 0;
+  }
+  if (st != ARD_OK) return st;
+  return launch_gemm_tc(ctx, pat->kind, OP_FWD, t, s);
+}
+
+// Produces the operand the tensor-core backward GEMMs read for dY: the caller's compact matrix, or
+// a compacted copy of the full-width one in the context workspace (row patterns only).
+static ard_status compact_dy(ard_ctx* ctx, const ard_pattern* pat, int B, int N, const void* dY, int lddy,
+                             int dy_is_compact, const void** out_ptr, int* out_ld, cudaStream_t s) {
+  if (dy_is_compact) {
+    *out_ptr = dY;
+    *out_ld = lddy;
+    return ARD_OK;
+  }
+  const int ldc = (N + 7) / 8 * 8;
+  if ((size_t)B * ldc * 2 > ctx->workspace_bytes) return ARD_ERR_NOMEM;
+  ard_status st = launch_gather_cols(ctx, pat->d_hdr, pat->d_idx, dY, lddy, ctx->d_workspace, ldc, B, 2, N, s);
+  *out_ptr = ctx->d_workspace;
+  *out_ld = ldc;
+  return st;
+}
+
+ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N, float alpha,
+                        const void* dY, int lddy, int dy_is_compact, const void* W, int ldw, void* dX, int lddx,
+                        void* cuda_stream) {
+  ard_status st = check_common(ctx, pat, B, K, N);
+  if (st != ARD_OK) return st;
+  if (!dY || !W || !dX) return ARD_ERR_INVALID_ARG;
+  if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (dy_is_compact && pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+  if (lddy < N || ldw < K || lddx < K) return ARD_ERR_SHAPE;
+  if (B == 0) return ARD_OK;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int es = dtype == ARD_F32 ? 4 : 2;
+
+  GemmArgs g;
+  fill_common(g, ctx, pat, B, K, N, alpha);
+  g.A0 = dY; g.lda0 = lddy; g.A1 = W; g.lda1 = ldw; g.out = dX; g.ldo = lddx;
+  g.flag0 = dy_is_compact ? 1 : 0;
+  g.out_is_f32 = dtype == ARD_F32;
+
+  ard_status el = ctx->path == ARD_PATH_CUDA_CORE
+                      ? ARD_ERR_UNSUPPORTED
+                      : tc_eligible(ctx, pat, dtype, B, K, N, dY, lddy, W, ldw, dX, lddx, es);
+  if (el == ARD_OK && pat->kind == ARD_ROW && !dy_is_compact &&
+      (size_t)B * ((N + 7) / 8 * 8) * 2 > ctx->workspace_bytes)
+    el = ARD_ERR_NOMEM;
+  if (el != ARD_OK) {
+    if (ctx->path == ARD_PATH_TENSOR_CORE) return el;
+    return launch_gemm_cc(ctx, pat->kind, OP_BWD_DATA, dtype, g, pat->ts, s);
+  }
+  TcArgs t;
+  t.ts = pat->ts;
+  t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_DATA, B, K, N, pat->ts);
+  if (pat->kind == ARD_ROW) {
+    const void* dyc;
+    int ldc;
+    st = compact_dy(ctx, pat, B, N, dY, lddy, dy_is_compact, &dyc, &ldc, s);
+    if (st != ARD_OK) return st;
+    g.A0 = dyc; g.lda0 = ldc; g.flag0 = 1;
+    // A = compact dY [B][n_keep], K-major;  B = kept neurons of W read MN-major: boxes [64 kept rows][64 k].
+    st = get_maps(ctx, dyc, B, N, ldc, N, MAP_COMPACT_COLS, pat->dp_bound, 128, 64, &t.mapA);
+    if (st != ARD_OK) return st;
+    t.mapA_indexed = 1;
+    st = get_maps(ctx, W, N, K, ldw, N, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64, &t.mapB);
+    t.mapB_indexed = 1;
+  } else {
+    st = get_maps(ctx, dY, B, N, lddy, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);
+    if (st != ARD_OK) return st;
+    t.mapA_indexed = 0;
+    st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);
+    t.mapB_indexed = 0;
+  }
+  if (st != ARD_OK) return st;
+  t.g = g;
+  return launch_gemm_tc(ctx, pat->kind, OP_BWD_DATA, t, s);
+}
+
+ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, ard_dtype dW_dtype, int B, int K,
+                          int N, float alpha, const void* X, int ldx, const void* dY, int lddy, int dy_is_compact,
+                          void* dW, int lddw, int zero_fill_dropped, void* cuda_stream) {
+  ard_status st = check_common(ctx, pat, B, K, N);
+  if (st != ARD_OK) return st;
+  if (!X || !dY || !dW) return ARD_ERR_INVALID_ARG;
+  if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (dW_dtype != ARD_F32 && dW_dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (dtype == ARD_F32 && dW_dtype != ARD_F32) return ARD_ERR_INVALID_ARG;
+  if (dy_is_compact && pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+  if (ldx < K || lddy < N || lddw < K) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int es_out = dW_dtype == ARD_F32 ? 4 : 2;
+
+  GemmArgs g;
+  fill_common(g, ctx, pat, B, K, N, alpha);
+  g.A0 = dY; g.lda0 = lddy; g.A1 = X; g.lda1 = ldx; g.out = dW; g.ldo = lddw;
+  g.flag0 = dy_is_compact ? 1 : 0;
+  g.flag1 = zero_fill_dropped ? 1 : 0;
+  g.out_is_f32 = dW_dtype == ARD_F32;
+  // Empty batch: the gradient of every kept weight is zero; the CUDA-core kernel writes exactly that.
+  if (B == 0) return launch_gemm_cc(ctx, pat->kind, OP_BWD_WEIGHT, dtype, g, pat->ts, s);
+
+  ard_status el = ctx->path == ARD_PATH_CUDA_CORE
+                      ? ARD_ERR_UNSUPPORTED
+                      : tc_eligible(ctx, pat, dtype, B, K, N, dY, lddy, X, ldx, dW, lddw, es_out);
+  if (el == ARD_OK && pat->kind == ARD_ROW && !dy_is_compact &&
+      (size_t)B * ((N + 7) / 8 * 8) * 2 > ctx->workspace_bytes)
+    el = ARD_ERR_NOMEM;
+  if (el != ARD_OK) {
+    if (ctx->path == ARD_PATH_TENSOR_CORE) return el;
+    return launch_gemm_cc(ctx, pat->kind, OP_BWD_WEIGHT, dtype, g, pat->ts, s);
+  }
+  TcArgs t;
+  t.ts = pat->ts;
+  t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_WEIGHT, B, K, N, pat->ts);
+  if (pat->kind == ARD_ROW) {
+    const void* dyc;
+    int ldc;
+    st = compact_dy(ctx, pat, B, N, dY, lddy, dy_is_compact, &dyc, &ldc, s);
+    if (st != ARD_OK) return st;
+    g.A0 = dyc; g.lda0 = ldc; g.flag0 = 1;
+    // A = compact dY read MN-major (boxes [64 batch rows][64 kept cols]);  B = X read MN-major.
+    st = get_maps(ctx, dyc, B, N, ldc, N, MAP_COMPACT_COLS, pat->dp_bound, 64, 64, &t.mapA);
+    t.mapA_indexed = 1;
+  } else {
+    if (zero_fill_dropped) ARD_CUDA_OK(cudaMemset2DAsync(dW, (size_t)lddw * es_out, 0, (size_t)K * es_out, N, s));
+    st = get_maps(ctx, dY, B, N, lddy, 0, MAP_PLAIN, 0, 64, 64, &t.mapA);
+    t.mapA_indexed = 0;
+  }
+  if (st != ARD_OK) return st;
+  st = get_maps(ctx, X, B, K, ldx, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);
+  t.mapB_indexed = 0;
+  if (st != ARD_OK) return st;
+  t.g = g;
+  return launch_gemm_tc(ctx, pat->kind, OP_BWD_WEIGHT, t, s);
+}
+
+// ---------------------------------------------------------------------------------------------------
+
+ard_status ard_lstm_gates(ard_ctx* ctx, const ard_pattern* pat, ard_dtype h_dtype, int B, int H, float alpha,
+                          const float* Z, int ldz_gate, const float* bias, const float* c_prev, int ldc, float* c,
+                          void* h, int ldh, int h_scatter, float* gates_saved, void* cuda_stream) {
+  if (!ctx || !pat || pat->ctx != ctx || !Z || !c_prev || !c || !h) return ARD_ERR_INVALID_ARG;
+  if (pat->kind != ARD_ROW || pat->N_dim != H) return ARD_ERR_SHAPE;
+  if (B < 0 || B > 65535 || H < 1) return ARD_ERR_INVALID_ARG;
+  if (h_dtype != ARD_F32 && h_dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (ldz_gate < 1 || ldc < 1 || ldh < 1 || (h_scatter && ldh < H)) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  return launch_lstm_gates(ctx, pat, h_dtype, B, H, alpha, Z, ldz_gate, bias, c_prev, ldc, c, h, ldh, h_scatter,
+                           gates_saved, (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_lstm_gates_bwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dz_dtype, int B, int H, float alpha,
+                              const float* gates_saved, const float* c_prev, const float* c, int ldc,
+                              const float* dh, int lddh, int dh_scatter, float* dc_inout, void* dZ, int ldz_gate,
+                              void* cuda_stream) {
+  if (!ctx || !pat || pat->ctx != ctx || !gates_saved || !c_prev || !c || !dh || !dc_inout || !dZ)
+    return ARD_ERR_INVALID_ARG;
+  if (pat->kind != ARD_ROW || pat->N_dim != H) return ARD_ERR_SHAPE;
+  if (B < 0 || B > 65535 || H < 1) return ARD_ERR_INVALID_ARG;
+  if (dz_dtype != ARD_F32 && dz_dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (ldz_gate < 1 || ldc < 1 || lddh < 1 || (dh_scatter && lddh < H)) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  return launch_lstm_gates_bwd(ctx, pat, dz_dtype, B, H, alpha, gates_saved, c_prev, c, ldc, dh, lddh, dh_scatter,
+                               dc_inout, dZ, ldz_gate, (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_last_device_status(ard_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return ARD_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  int v = 0;
+  ARD_CUDA_OK(cudaMemcpyAsync(&v, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, s));
+  ARD_CUDA_OK(cudaStreamSynchronize(s));
+  if (v != 0) {
+    ARD_CUDA_OK(cudaMemsetAsync(ctx->d_status, 0, sizeof(int), s));
+    ARD_CUDA_OK(cudaStreamSynchronize(s));
+  }
+  return (ard_status)v;
+}
+
+uint64_t ard_launch_count(const ard_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,139 @@
+// Internal declarations shared by the translation units of libard.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "ard.h"
+
+// ---- device-resident pattern --------------------------------------------------------------------
+// One int32 allocation: a 16-word header followed by the index lists.
+enum {
+  HDR_KIND = 0,
+  HDR_DP = 1,
+  HDR_B = 2,
+  HDR_NKEEP = 3,   // kept neurons (row) or kept tiles (tile)
+  HDR_UNITS = 4,
+  HDR_TR = 5,
+  HDR_TC = 6,
+  HDR_TS = 7,
+  HDR_MAPIDX = 8,  // dp*(dp-1)/2 + (b-1): index into per-(dp,b) descriptor tables
+  HDR_WORDS = 16
+};
+
+struct ard_pattern {
+  ard_ctx* ctx;
+  ard_kind kind;
+  int K_dim, N_dim, ts, Tr, Tc, units;
+  int dp_bound;        // largest dp the last sample/set call can have produced
+  int32_t* d_hdr;      // device: header
+  int32_t* d_idx;      // device: kept list (row: neuron index; tile: t-1), capacity `units`
+  int32_t* d_col_ptr;  // tile only: [Tc+1]
+  int32_t* d_col_idx;  // tile only: [units]
+  int32_t* d_row_ptr;  // tile only: [Tr+1]
+  int32_t* d_row_idx;  // tile only: [units]
+};
+
+struct ArdDistribution {
+  int ndp = 0;
+  unsigned long long* d_cdf = nullptr;  // device: ndp entries
+  std::vector<unsigned long long> h_cdf;
+};
+
+// A cached table of TMA descriptors in device memory, one per (dp, b) pair (or a single one).
+struct MapTable {
+  const void* base;
+  int rows, cols, ld, elem_bytes;
+  int box_rows, box_cols;
+  int variant;   // see MapVariant
+  int dp_bound;
+  CUtensorMap* d_maps;
+  int count;
+};
+
+enum MapVariant {
+  MAP_PLAIN = 0,         // one descriptor: [rows][cols], pitch ld
+  MAP_STRIDED_ROWS = 1,  // per (dp,b): rows b-1, b-1+dp, ... (n_keep of them), all cols
+  MAP_COMPACT_COLS = 2   // per (dp,b): all rows, cols 0..n_keep-1 of a compact matrix
+};
+
+struct ard_ctx {
+  int device;
+  int sm_count;
+  ard_path path;
+  int force_bn;
+  size_t workspace_bytes;
+  void* d_workspace;
+  int* d_status;
+  ArdDistribution dist[ARD_MAX_DISTRIBUTIONS];
+  std::vector<MapTable> maps;
+  unsigned long long launches;
+  void* encode_fn;  // cuTensorMapEncodeTiled, resolved at run time
+};
+
+static inline int map_index_count(int dp_bound) { return dp_bound * (dp_bound + 1) / 2; }
+
+// ---- launchers implemented in the .cu files -----------------------------------------------------
+ard_status launch_sampler(ard_ctx* ctx, ard_pattern* pat, const unsigned long long* d_cdf, int ndp,
+                          uint64_t seed, uint64_t iteration, uint32_t stream_id, int forced_dp, int forced_b,
+                          cudaStream_t s);
+
+struct GemmArgs {
+  const int32_t* hdr;
+  const int32_t* idx;
+  const int32_t* col_ptr;
+  const int32_t* col_idx;
+  const int32_t* row_ptr;
+  const int32_t* row_idx;
+  int B, K, N;
+  float alpha;
+  const void* A0;  // X or dY
+  int lda0;
+  const void* A1;  // W or X
+  int lda1;
+  void* out;
+  int ldo;
+  int flag0;       // fwd: outmode; bwd: dy_is_compact
+  int flag1;       // bwd_weight: zero_fill_dropped
+  int out_is_f32;
+  int* status;
+};
+
+enum GemmOp { OP_FWD = 0, OP_BWD_DATA = 1, OP_BWD_WEIGHT = 2 };
+
+// CUDA-core family (fp32 or bf16 operands, fp32 accumulate).
+ard_status launch_gemm_cc(ard_ctx* ctx, ard_kind kind, GemmOp op, ard_dtype dtype, const GemmArgs& a, int ts,
+                          cudaStream_t s);
+
+// tcgen05 family (bf16 operands, fp32 accumulate in TMEM).
+struct TcArgs {
+  const CUtensorMap* mapA;  // table or single descriptor
+  const CUtensorMap* mapB;
+  int mapA_indexed, mapB_indexed;
+  GemmArgs g;
+  int ts;
+  int bn;  // N tile: 64, 128 or 256
+};
+int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int B, int K, int N, int ts);
+ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s);
+
+ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,
+                              void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, cudaStream_t s);
+
+ard_status launch_lstm_gates(ard_ctx* ctx, const ard_pattern* pat, ard_dtype h_dtype, int B, int H, float alpha,
+                             const float* Z, int ldz_gate, const float* bias, const float* c_prev, int ldc, float* c,
+                             void* h, int ldh, int h_scatter, float* gates_saved, cudaStream_t s);
+ard_status launch_lstm_gates_bwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dz_dtype, int B, int H, float alpha,
+                                 const float* gates_saved, const float* c_prev, const float* c, int ldc,
+                                 const float* dh, int lddh, int dh_scatter, float* dc_inout, void* dZ, int ldz_gate,
+                                 cudaStream_t s);
+
+#define ARD_CUDA_OK(expr)                       \
+  do {                                          \
+    cudaError_t e__ = (expr);                   \
+    if (e__ != cudaSuccess) return ARD_ERR_CUDA; \
+  } while (0)

@@ -1,0 +1,188 @@
+// CUDA-core family of the compacted GEMMs: fp32 (or bf16) operands, fp32 FFMA accumulation.
+//
+// This is the path of the fp32 layers (a single tcgen05 tf32 pass keeps 10 mantissa bits and
+// cannot reach 1e-5) and the fall-back for bf16 shapes whose alignment the TMA path cannot take.
+// One generic 32x32x32 shared-memory tiled kernel; what differs per product is only how the
+// logical operand element (m, k), (n, k) maps to memory and which contraction indices exist:
+// dropped neurons / tiles are skipped through the index lists, never multiplied by zero.
+#include "ard_internal.h"
+
+namespace {
+
+constexpr int T_M = 32, T_N = 32, T_K = 32, CC_THREADS = 256;
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+__device__ __forceinline__ void store_out(void* out, size_t off, float v, int out_is_f32) {
+  if (out_is_f32) reinterpret_cast<float*>(out)[off] = v;
+  else reinterpret_cast<__nv_bfloat16*>(out)[off] = __float2bfloat16_rn(v);
+}
+
+// KIND: 0 row, 1 tile.  OP: GemmOp.
+template <typename T, int KIND, int OP>
+__global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts) {
+  __shared__ float As[T_K][T_M + 1];
+  __shared__ float Bs[T_K][T_N + 1];
+
+  const int dp = g.hdr[HDR_DP], b = g.hdr[HDR_B], n_keep = g.hdr[HDR_NKEEP];
+  const int Tc = g.hdr[HDR_TC];
+  const T* __restrict__ P0 = reinterpret_cast<const T*>(g.A0);
+  const T* __restrict__ P1 = reinterpret_cast<const T*>(g.A1);
+
+  int M, N, nk;
+  const int m0 = blockIdx.y * T_M, n0 = blockIdx.x * T_N;
+  const int32_t* klist = nullptr;  // tile patterns: contraction runs over ts-wide blocks klist[0..]
+  if (KIND == 0) {
+    if (OP == OP_FWD) { M = g.B; N = n_keep; nk = g.K; }
+    else if (OP == OP_BWD_DATA) { M = g.B; N = g.K; nk = n_keep; }
+    else { M = n_keep; N = g.K; nk = g.B; }
+  } else {
+    if (OP == OP_FWD) {
+      M = g.B; N = g.N;
+      if (n0 >= N) return;
+      const int c = n0 / ts;
+      klist = g.col_idx + g.col_ptr[c];
+      nk = (g.col_ptr[c + 1] - g.col_ptr[c]) * ts;
+    } else if (OP == OP_BWD_DATA) {
+      M = g.B; N = g.K;
+      if (n0 >= N) return;
+      const int r = n0 / ts;
+      klist = g.row_idx + g.row_ptr[r];
+      nk = (g.row_ptr[r + 1] - g.row_ptr[r]) * ts;
+    } else {
+      M = g.N; N = g.K; nk = g.B;
+    }
+  }
+  if (m0 >= M || n0 >= N) return;
+
+  if (KIND == 1 && OP == OP_BWD_WEIGHT) {
+    const int lin = (n0 / ts) * Tc + (m0 / ts);  // tile (r, c) = (k-block, neuron-block), 0-based t-1
+    const bool kept = lin >= b - 1 && (lin - (b - 1)) % dp == 0;
+    if (!kept) {
+      if (g.flag1) {
+        for (int e = threadIdx.x; e < T_M * T_N; e += CC_THREADS) {
+          const int m = m0 + e / T_N, n = n0 + e % T_N;
+          if (m < M && n < N) store_out(g.out, (size_t)m * g.ldo + n, 0.f, g.out_is_f32);
+        }
+      }
+      return;
+    }
+  }
+
+  const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+  float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+
+  for (int k0 = 0; k0 < nk; k0 += T_K) {
+    for (int e = threadIdx.x; e < T_K * T_M; e += CC_THREADS) {
+      // operand A: element (m, kk)
+      int kk, m;
+      if ((KIND == 0 && OP == OP_BWD_WEIGHT) || (KIND == 1 && OP == OP_BWD_WEIGHT)) { m = e % T_M; kk = e / T_M; }
+      else { kk = e % T_K; m = e / T_K; }
+      float v = 0.f;
+      const int gm = m0 + m, gk = k0 + kk;
+      if (gm < M && gk < nk) {
+        size_t off;
+        if (KIND == 0) {
+          if (OP == OP_FWD) off = (size_t)gm * g.lda0 + gk;
+          else if (OP == OP_BWD_DATA) off = (size_t)gm * g.lda0 + (g.flag0 ? gk : g.idx[gk]);
+          else off = (size_t)gk * g.lda0 + (g.flag0 ? gm : g.idx[gm]);
+        } else {
+          if (OP == OP_BWD_WEIGHT) off = (size_t)gk * g.lda0 + gm;
+          else off = (size_t)gm * g.lda0 + (size_t)klist[gk / ts] * ts + gk % ts;
+        }
+        v = to_f<T>(P0[off]);
+      }
+      As[kk][m] = v;
+    }
+    for (int e = threadIdx.x; e < T_K * T_N; e += CC_THREADS) {
+      // operand B: element (n, kk)
+      int kk, n;
+      if (OP == OP_FWD) { kk = e % T_K; n = e / T_K; }
+      else { n = e % T_N; kk = e / T_N; }
+      float v = 0.f;
+      const int gn = n0 + n, gk = k0 + kk;
+      if (gn < N && gk < nk) {
+        size_t off;
+        if (KIND == 0) {
+          if (OP == OP_FWD) off = (size_t)g.idx[gn] * g.lda1 + gk;
+          else if (OP == OP_BWD_DATA) off = (size_t)g.idx[gk] * g.lda1 + gn;
+          else off = (size_t)gk * g.lda1 + gn;
+        } else {
+          const size_t kidx = (OP == OP_BWD_WEIGHT) ? (size_t)gk : (size_t)klist[gk / ts] * ts + gk % ts;
+          if (OP == OP_FWD) off = (size_t)gn * g.lda1 + kidx;
+          else if (OP == OP_BWD_DATA) off = kidx * g.lda1 + gn;
+          else off = kidx * g.lda1 + gn;
+        }
+        v = to_f<T>(P1[off]);
+      }
+      Bs[kk][n] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < T_K; ++kk) {
+      const float a0 = As[kk][ty * 2], a1 = As[kk][ty * 2 + 1];
+      const float b0 = Bs[kk][tx * 2], b1 = Bs[kk][tx * 2 + 1];
+      acc[0][0] = fmaf(a0, b0, acc[0][0]);
+      acc[0][1] = fmaf(a0, b1, acc[0][1]);
+      acc[1][0] = fmaf(a1, b0, acc[1][0]);
+      acc[1][1] = fmaf(a1, b1, acc[1][1]);
+    }
+    __syncthreads();
+  }
+
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int m = m0 + ty * 2 + i, n = n0 + tx * 2 + j;
+      if (m >= M || n >= N) continue;
+      size_t off;
+      if (KIND == 0 && OP == OP_FWD) off = (size_t)m * g.ldo + (g.flag0 == ARD_OUT_SCATTER_ZEROFILL ? g.idx[n] : n);
+      else if (KIND == 0 && OP == OP_BWD_WEIGHT) off = (size_t)g.idx[m] * g.ldo + n;
+      else off = (size_t)m * g.ldo + n;
+      store_out(g.out, off, g.alpha * acc[i][j], g.out_is_f32);
+    }
+}
+
+template <typename T, int KIND, int OP>
+void launch_one(const GemmArgs& a, int ts, int Mmax, int Nmax, cudaStream_t s) {
+  dim3 grid((Nmax + T_N - 1) / T_N, (Mmax + T_M - 1) / T_M);
+  gemm_cc_kernel<T, KIND, OP><<<grid, CC_THREADS, 0, s>>>(a, ts);
+}
+
+template <typename T>
+void dispatch(ard_kind kind, GemmOp op, const GemmArgs& a, int ts, cudaStream_t s) {
+  // The grid covers the largest problem any pattern can produce (dp = 1); CTAs beyond the
+  // sampled extent read the header and exit.
+  if (kind == ARD_ROW) {
+    if (op == OP_FWD) launch_one<T, 0, OP_FWD>(a, ts, a.B, a.N, s);
+    else if (op == OP_BWD_DATA) launch_one<T, 0, OP_BWD_DATA>(a, ts, a.B, a.K, s);
+    else launch_one<T, 0, OP_BWD_WEIGHT>(a, ts, a.N, a.K, s);
+  } else {
+    if (op == OP_FWD) launch_one<T, 1, OP_FWD>(a, ts, a.B, a.N, s);
+    else if (op == OP_BWD_DATA) launch_one<T, 1, OP_BWD_DATA>(a, ts, a.B, a.K, s);
+    else launch_one<T, 1, OP_BWD_WEIGHT>(a, ts, a.N, a.K, s);
+  }
+}
+
+}  // namespace
+
+ard_status launch_gemm_cc(ard_ctx* ctx, ard_kind kind, GemmOp op, ard_dtype dtype, const GemmArgs& a, int ts,
+                          cudaStream_t s) {
+  if ((a.B == 0 && op != OP_BWD_WEIGHT) || a.K == 0 || a.N == 0) return ARD_OK;
+  const size_t es_out = a.out_is_f32 ? 4 : 2;
+  // Row patterns: dropped outputs are cleared by a strided memset before the kept ones are written.
+  if (kind == ARD_ROW && op == OP_FWD && a.flag0 == ARD_OUT_SCATTER_ZEROFILL) {
+    ARD_CUDA_OK(cudaMemset2DAsync(a.out, (size_t)a.ldo * es_out, 0, (size_t)a.N * es_out, a.B, s));
+  }
+  if (kind == ARD_ROW && op == OP_BWD_WEIGHT && a.flag1) {
+    ARD_CUDA_OK(cudaMemset2DAsync(a.out, (size_t)a.ldo * es_out, 0, (size_t)a.K * es_out, a.N, s));
+  }
+  if (dtype == ARD_F32) dispatch<float>(kind, op, a, ts, s);
+  else dispatch<__nv_bfloat16>(kind, op, a, ts, s);
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}

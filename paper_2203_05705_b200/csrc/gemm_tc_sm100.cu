@@ -1,0 +1,674 @@
+// tcgen05 family of the compacted GEMMs (bf16 operands, fp32 accumulation in tensor memory).
+//
+// One persistent, warp-specialised kernel template covers the six products (row / tile pattern x
+// forward / backward-data / backward-weight).  Per CTA: warp 0 is the TMA producer, warp 1 issues
+// tcgen05.mma and owns the TMEM allocation, warps 2..5 are the epilogue.  Only the kept rows /
+// tiles of the weight and the matching slices of the activations are ever staged into shared
+// memory (Sec. 3.1, 3.2): a row pattern's kept neurons b-1, b-1+dp, ... are one TMA box of a
+// descriptor whose row pitch is dp*ldw; a tile pattern's kept tiles come from the per-column /
+// per-row lists the sampler emitted.  The pattern is read from device memory, so the launch does
+// not depend on it: the grid is sized for the densest pattern and each CTA derives its own tile
+// schedule from the header.
+//
+// The accumulator is double-buffered in TMEM (2 x BN columns), so the epilogue of one output tile
+// overlaps the MMAs of the next.  Every wait on an mbarrier is bounded by a wall-clock limit;
+// when it expires the CTA records ARD_ERR_TIMEOUT, all roles leave their loops, the TMEM
+// allocation is released and the kernel returns normally.
+#include "ard_internal.h"
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;  // 64 bf16 = 128 bytes = one swizzle row
+constexpr int TC_THREADS = 192;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+enum TcMode {
+  M_ROW_FWD = 0,
+  M_ROW_BWD_DATA = 1,
+  M_ROW_BWD_WEIGHT = 2,
+  M_TILE_FWD = 3,
+  M_TILE_BWD_DATA = 4,
+  M_TILE_BWD_WEIGHT = 5
+};
+
+__host__ __device__ constexpr bool a_is_mn(int mode) { return mode == M_ROW_BWD_WEIGHT || mode == M_TILE_BWD_WEIGHT; }
+__host__ __device__ constexpr bool b_is_mn(int mode) { return mode != M_ROW_FWD && mode != M_TILE_FWD; }
+__host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 4 : (bn == 128 ? 6 : 8); }
+__host__ __device__ constexpr int tmem_cols_for(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }
+
+struct TcParams {
+  const CUtensorMap* mapA;
+  const CUtensorMap* mapB;
+  int mapA_indexed, mapB_indexed;
+  const int32_t* hdr;
+  const int32_t* idx;
+  const int32_t* col_ptr;
+  const int32_t* col_idx;
+  const int32_t* row_ptr;
+  const int32_t* row_idx;
+  int B, K, N;  // batch, fan-in, neurons
+  int ts;
+  float alpha;
+  void* out;
+  int ldo;
+  int out_is_f32;
+  int scatter;    // row fwd: full-width output with zero fill
+  int zero_fill;  // row bwd-weight: write zeros to dropped rows
+  int* status;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, P;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false if the limit expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > WAIT_LIMIT_NS) {
+      *abort_flag = 1;
+      atomicMax(status, (int)ARD_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tensormap_acquire(const CUtensorMap* map) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, Blackwell version field = 1.
+//   K-major operand : rows of 128 bytes, 8-row groups 1024 bytes apart (SBO); LBO unused (1).
+//   MN-major operand: 64-element chunks along M/N `lbo` bytes apart; 8-row K groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn, bool b_mn) {
+  return (1u << 4)                      // D format fp32
+         | (1u << 7)                    // A format bf16
+         | (1u << 10)                   // B format bf16
+         | ((a_mn ? 1u : 0u) << 15)     // A major
+         | ((b_mn ? 1u : 0u) << 16)     // B major
+         | ((uint32_t)(n >> 3) << 17)   // N
+         | ((uint32_t)(BM >> 4) << 24); // M
+}
+
+template <int BN>
+struct SmemLayout {
+  static constexpr int STAGES = stages_for(BN);
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STG_OFF = STAGES * STAGE_BYTES;       // epilogue staging: 4 warps x 32 x 33 floats
+  static constexpr int STG_BYTES = 4 * 32 * 33 * 4;
+  static constexpr int BAR_OFF = STG_OFF + STG_BYTES;        // full[S], empty[S], tfull[2], tempty[2]
+  static constexpr int MISC_OFF = BAR_OFF + (2 * STAGES + 4) * 8;
+  static constexpr int TOTAL = MISC_OFF + 16 + 1024;         // + slack for manual 1024-byte alignment
+};
+
+// Tile schedule shared by the three roles.
+struct TileInfo {
+  int m0, n0;      // origin in GEMM space
+  int nkb;         // number of 64-wide contraction blocks
+  const int32_t* klist;  // tile patterns: kept block list for this output tile
+  int kper;        // 64-blocks per pattern tile
+  int out_row0;    // tile bwd-weight: first output row (neuron)
+  int rows_valid;  // tile bwd-weight: rows of this tile that belong to the kept tile
+};
+
+template <int BN, int MODE>
+struct Sched {
+  int dp, b, n_keep, Tc;
+  int Mt, Nt, total;
+  int M_gemm, N_gemm, Kc;  // GEMM extents (valid rows, valid cols, contraction length)
+  int subm, subn;          // tile bwd-weight: sub-blocks per pattern tile
+
+  __device__ void init(const TcParams& p) {
+    dp = p.hdr[HDR_DP];
+    b = p.hdr[HDR_B];
+    n_keep = p.hdr[HDR_NKEEP];
+    Tc = p.hdr[HDR_TC];
+    subm = subn = 1;
+    if (MODE == M_ROW_FWD) { M_gemm = p.B; N_gemm = n_keep; Kc = p.K; }
+    else if (MODE == M_ROW_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = n_keep; }
+    else if (MODE == M_ROW_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = p.K; Kc = p.B; }
+    else if (MODE == M_TILE_FWD) { M_gemm = p.B; N_gemm = p.N; Kc = 0; }
+    else if (MODE == M_TILE_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 0; }
+    else { M_gemm = p.N; N_gemm = p.K; Kc = p.B; }
+    if (MODE == M_TILE_BWD_WEIGHT) {
+      subm = (p.ts + BM - 1) / BM;
+      subn = p.ts / BN;
+      Mt = n_keep * subm;
+      Nt = subn;
+    } else {
+      Mt = (M_gemm + BM - 1) / BM;
+      Nt = (N_gemm + BN - 1) / BN;
+    }
+    total = Mt * Nt;
+  }
+
+  __device__ TileInfo tile(const TcParams& p, int t) const {
+    TileInfo ti;
+    ti.klist = nullptr;
+    ti.kper = 1;
+    ti.out_row0 = 0;
+    ti.rows_valid = BM;
+    if (MODE == M_TILE_BWD_WEIGHT) {
+      const int j = t / (subm * subn), rem = t % (subm * subn);
+      const int sm = rem / subn, sn = rem % subn;
+      const int lin = p.idx[j];
+      const int r = lin / Tc, c = lin % Tc;
+      ti.m0 = c * p.ts + sm * BM;
+      ti.n0 = r * p.ts + sn * BN;
+      ti.nkb = (Kc + BK - 1) / BK;
+      ti.rows_valid = min(BM, p.ts - sm * BM);
+      return ti;
+    }
+    const int mt = t % Mt, nt = t / Mt;
+    ti.m0 = mt * BM;
+    ti.n0 = nt * BN;
+    if (MODE == M_TILE_FWD) {
+      const int c = ti.n0 / p.ts;
+      ti.klist = p.col_idx + p.col_ptr[c];
+      ti.kper = p.ts / BK;
+      ti.nkb = (p.col_ptr[c + 1] - p.col_ptr[c]) * ti.kper;
+    } else if (MODE == M_TILE_BWD_DATA) {
+      const int r = ti.n0 / p.ts;
+      ti.klist = p.row_idx + p.row_ptr[r];
+      ti.kper = p.ts / BK;
+      ti.nkb = (p.row_ptr[r + 1] - p.row_ptr[r]) * ti.kper;
+    } else {
+      ti.nkb = (Kc + BK - 1) / BK;
+    }
+    return ti;
+  }
+};
+
+// ---- epilogue helpers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Stores 32 consecutive values of one output row; `nvalid` of them exist.  The row start is 16-byte
+// aligned whenever nvalid == 32 paths are taken (guaranteed by the host-side alignment checks).
+__device__ __forceinline__ void store_row32(void* out, size_t row_off, int col, const float (&v)[32], int nvalid,
+                                            int out_is_f32) {
+  if (out_is_f32) {
+    float* p = reinterpret_cast<float*>(out) + row_off + col;
+    if (nvalid >= 32) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        reinterpret_cast<float4*>(p)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    } else {
+#pragma unroll
+      for (int q = 0; q < 32; ++q)
+        if (q < nvalid) p[q] = v[q];
+    }
+  } else {
+    __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(out) + row_off + col;
+    if (nvalid >= 32) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        reinterpret_cast<uint4*>(p)[q] =
+            make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
+                       pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+    } else {
+#pragma unroll
+      for (int q = 0; q < 32; ++q)
+        if (q < nvalid) p[q] = __float2bfloat16_rn(v[q]);
+    }
+  }
+}
+
+__device__ __forceinline__ void zero_row32(void* out, size_t row_off, int col, int nvalid, int out_is_f32) {
+  float z[32];
+#pragma unroll
+  for (int q = 0; q < 32; ++q) z[q] = 0.f;
+  store_row32(out, row_off, col, z, nvalid, out_is_f32);
+}
+
+// ---- the kernel -----------------------------------------------------------------------------------
+template <int BN, int MODE>
+__global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcParams p) {
+  using L = SmemLayout<BN>;
+  constexpr int STAGES = L::STAGES;
+  constexpr bool A_MN = a_is_mn(MODE), B_MN = b_is_mn(MODE);
+  constexpr uint32_t IDESC = make_idesc(BN, A_MN, B_MN);
+  constexpr uint32_t TMEM_COLS = tmem_cols_for(BN);
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw_addr);
+
+  const uint32_t bar_base = base + L::BAR_OFF;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + L::MISC_OFF);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::MISC_OFF + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+
+  Sched<BN, MODE> sch;
+  sch.init(p);
+
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0) {
+      const int e = p.hdr[HDR_MAPIDX];
+      const CUtensorMap* mapA = p.mapA + (p.mapA_indexed ? e : 0);
+      const CUtensorMap* mapB = p.mapB + (p.mapB_indexed ? e : 0);
+      tensormap_acquire(mapA);
+      tensormap_acquire(mapB);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < sch.total && ok; t += gridDim.x) {
+        const TileInfo ti = sch.tile(p, t);
+        for (int kb = 0; kb < ti.nkb; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t sA = base + stage * L::STAGE_BYTES;
+          const uint32_t sB = sA + L::A_BYTES;
+          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)L::STAGE_BYTES);
+          // contraction coordinate of this block
+          int kx;
+          if (MODE == M_TILE_FWD || MODE == M_TILE_BWD_DATA) kx = ti.klist[kb / ti.kper] * p.ts + (kb % ti.kper) * BK;
+          else kx = kb * BK;
+          if (!A_MN) {
+            tma_load_2d(sA, mapA, full_bar(stage), kx, ti.m0);  // [BM rows][64 k]
+          } else {
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i)  // [64 k rows][64 m] per box
+              tma_load_2d(sA + i * (64 * BK * 2), mapA, full_bar(stage), ti.m0 + 64 * i, kx);
+          }
+          if (!B_MN) {
+            tma_load_2d(sB, mapB, full_bar(stage), kx, ti.n0);  // [BN rows][64 k]
+          } else {
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i)
+              tma_load_2d(sB + i * (64 * BK * 2), mapB, full_bar(stage), ti.n0 + 64 * i, kx);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < sch.total && ok; t += gridDim.x, ++it) {
+        const TileInfo ti = sch.tile(p, t);
+        const int acc = it & 1;
+        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < ti.nkb; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sA = base + stage * L::STAGE_BYTES;
+          const uint32_t sB = sA + L::A_BYTES;
+#pragma unroll
+          for (int s = 0; s < BK / 16; ++s) {
+            // K-major: advance 16 elements = 32 bytes inside the swizzled row.
+            // MN-major: advance 16 k-rows = 2048 bytes.
+            const uint64_t ad = A_MN ? make_desc(sA + s * 2048, 64 * BK * 2, 1024) : make_desc(sA + s * 32, 16, 1024);
+            const uint64_t bd = B_MN ? make_desc(sB + s * 2048, 64 * BK * 2, 1024) : make_desc(sB + s * 32, 16, 1024);
+            tc_mma_bf16(d_tmem, ad, bd, IDESC, (kb | s) != 0 ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        if (ti.nkb > 0) tc_commit(tfull_bar(acc));
+        else mbar_arrive(tfull_bar(acc));
+      }
+    }
+  } else {
+    // ===================== epilogue (warps 2..5) =====================
+    const int q = warp & 3;                 // TMEM lane quadrant this warp may read
+    const int row_in_tile = q * 32 + lane;  // accumulator row owned by this thread
+    float* stg = reinterpret_cast<float*>(smem + L::STG_OFF) + (warp - 2) * (32 * 33);
+    int it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < sch.total && ok; t += gridDim.x, ++it) {
+      const TileInfo ti = sch.tile(p, t);
+      const int acc = it & 1;
+      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+      const int m = ti.m0 + row_in_tile;
+
+      // Output row and validity by mode.
+      bool row_ok;
+      long long out_row;
+      if (MODE == M_ROW_BWD_WEIGHT) {
+        row_ok = m < sch.M_gemm;
+        out_row = (long long)(sch.b - 1) + (long long)m * sch.dp;
+      } else if (MODE == M_TILE_BWD_WEIGHT) {
+        row_ok = row_in_tile < ti.rows_valid && m < sch.M_gemm;
+        out_row = m;
+      } else {
+        row_ok = m < sch.M_gemm;
+        out_row = m;
+      }
+
+#pragma unroll 1
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        const int n = ti.n0 + ch * 32;
+        float v[32];
+        if (ti.nkb > 0) {
+          uint32_t r[32];
+          tmem_ld32(t_row + (uint32_t)(ch * 32), r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = p.alpha * __uint_as_float(r[i]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = 0.f;
+        }
+
+        if (MODE == M_ROW_FWD && p.scatter) {
+          // Full-width rows: compact column j -> column b-1 + j*dp, zeros everywhere else
+          // (Sec. 3.1: dropped outputs are zero).  Staged through shared memory so that
+          // consecutive lanes write consecutive 16-byte pieces of one output row.
+          if (n < sch.n_keep) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) stg[lane * 33 + i] = v[i];
+            __syncwarp();
+            const int dp = sch.dp, bb = sch.b - 1;
+            const long long cs = (long long)n * dp;
+            const bool last = n + 32 >= sch.n_keep;
+            const long long ce = last ? (long long)p.N : min((long long)(n + 32) * dp, (long long)p.N);
+            const int groups = (int)((ce - cs + 7) / 8);
+            const int rows_here = min(32, sch.M_gemm - (ti.m0 + q * 32));
+            for (int rr = 0; rr < rows_here; ++rr) {
+              __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)(ti.m0 + q * 32 + rr) * p.ldo;
+              float* ofrow = reinterpret_cast<float*>(p.out) + (size_t)(ti.m0 + q * 32 + rr) * p.ldo;
+              for (int g = lane; g < groups; g += 32) {
+                const long long c0 = cs + 8ll * g;
+                // Walk the 8 columns of this piece keeping (compact column, remainder) of c - (b-1);
+                // a column is kept exactly when the remainder is zero (Eq. 1).
+                const long long rel = c0 - bb;  // negative only before the first kept column
+                int cq, cr;
+                if (rel >= 0) { cq = (int)(rel / dp); cr = (int)(rel % dp); }
+                else { cq = -1; cr = (int)(rel + dp); }
+                float w[8];
+#pragma unroll
+                for (int pos = 0; pos < 8; ++pos) {
+                  const bool kept = cr == 0;
+                  w[pos] = kept ? stg[rr * 33 + (cq - n)] : 0.f;
+                  if (++cr == dp) { cr = 0; ++cq; }
+                }
+                const long long nleft = ce - c0;
+                if (p.out_is_f32) {
+                  if (nleft >= 8) {
+                    reinterpret_cast<float4*>(ofrow + c0)[0] = make_float4(w[0], w[1], w[2], w[3]);
+                    reinterpret_cast<float4*>(ofrow + c0)[1] = make_float4(w[4], w[5], w[6], w[7]);
+                  } else {
+#pragma unroll
+                    for (int pos = 0; pos < 8; ++pos)
+                      if (pos < nleft) ofrow[c0 + pos] = w[pos];
+                  }
+                } else {
+                  if (nleft >= 8) {
+                    *reinterpret_cast<uint4*>(orow + c0) = make_uint4(pack_bf16(w[0], w[1]), pack_bf16(w[2], w[3]),
+                                                                      pack_bf16(w[4], w[5]), pack_bf16(w[6], w[7]));
+                  } else {
+#pragma unroll
+                    for (int pos = 0; pos < 8; ++pos)
+                      if (pos < nleft) orow[c0 + pos] = __float2bfloat16_rn(w[pos]);
+                  }
+                }
+              }
+            }
+            __syncwarp();
+          }
+        } else {
+          const int nvalid = min(32, sch.N_gemm - n);
+          if (row_ok && nvalid > 0) {
+            store_row32(p.out, (size_t)out_row * p.ldo, n, v, nvalid, p.out_is_f32);
+            if (MODE == M_ROW_BWD_WEIGHT && p.zero_fill) {
+              // Dropped neurons between this kept row and the next (and before the first / after
+              // the last kept row) receive zeros.
+              // Compact row m owns output rows [m*dp, (m+1)*dp); the last one also owns the tail.
+              const long long first = (long long)m * sch.dp;
+              const long long lastrow =
+                  (m == sch.M_gemm - 1) ? (long long)p.N - 1 : min((long long)(m + 1) * sch.dp - 1, (long long)p.N - 1);
+              for (long long rz = first; rz <= lastrow; ++rz)
+                if (rz != out_row) zero_row32(p.out, (size_t)rz * p.ldo, n, nvalid, p.out_is_f32);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int BN, int MODE>
+ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStream_t s) {
+  using L = SmemLayout<BN>;
+  static bool attr_done[64] = {};
+  auto kern = ard_gemm_tc_kernel<BN, MODE>;
+  if (!attr_done[ctx->device & 63]) {
+    ARD_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
+    attr_done[ctx->device & 63] = true;
+  }
+  int grid = max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count;
+  if (grid < 1) grid = 1;
+  kern<<<grid, TC_THREADS, L::TOTAL, s>>>(p);
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+}  // namespace
+
+// Chooses the N tile: the widest instruction (256) when the densest pattern still fills the SMs,
+// narrower tiles otherwise so that more CTAs have work.
+int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int B, int K, int N, int ts) {
+  const int f = ctx->force_bn;
+  if (kind == ARD_TILE) {
+    // the N tile must divide the pattern tile
+    if (f && ts % f == 0 && (op == OP_BWD_WEIGHT || f <= 128)) return f;
+    if (op == OP_BWD_WEIGHT) return ts % 256 == 0 ? 256 : (ts % 128 == 0 ? 128 : 64);
+    return ts % 128 == 0 ? 128 : 64;
+  }
+  if (f) return f;
+  int Mg, Ng;
+  if (op == OP_FWD) { Mg = B; Ng = N; }
+  else if (op == OP_BWD_DATA) { Mg = B; Ng = K; }
+  else { Mg = N; Ng = K; }
+  const int mt = (Mg + BM - 1) / BM;
+  if (Ng >= 256 && mt * ((Ng + 255) / 256) >= ctx->sm_count) return 256;
+  if (Ng >= 128 && mt * ((Ng + 127) / 128) >= ctx->sm_count / 2) return 128;
+  return Ng >= 128 ? 128 : 64;
+}
+
+ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s) {
+  TcParams p;
+  p.mapA = a.mapA;
+  p.mapB = a.mapB;
+  p.mapA_indexed = a.mapA_indexed;
+  p.mapB_indexed = a.mapB_indexed;
+  p.hdr = a.g.hdr;
+  p.idx = a.g.idx;
+  p.col_ptr = a.g.col_ptr;
+  p.col_idx = a.g.col_idx;
+  p.row_ptr = a.g.row_ptr;
+  p.row_idx = a.g.row_idx;
+  p.B = a.g.B;
+  p.K = a.g.K;
+  p.N = a.g.N;
+  p.ts = a.ts;
+  p.alpha = a.g.alpha;
+  p.out = a.g.out;
+  p.ldo = a.g.ldo;
+  p.out_is_f32 = a.g.out_is_f32;
+  p.scatter = (kind == ARD_ROW && op == OP_FWD && a.g.flag0 == ARD_OUT_SCATTER_ZEROFILL) ? 1 : 0;
+  p.zero_fill = (op == OP_BWD_WEIGHT) ? a.g.flag1 : 0;
+  p.status = a.g.status;
+  const int bn = a.bn;
+
+#define ARD_TC_CASE(BN_, MODE_, TILES_) \
+  if (bn == BN_) return launch_mode<BN_, MODE_>(ctx, p, (TILES_), s);
+
+  if (kind == ARD_ROW) {
+    if (op == OP_FWD) {
+      const int mt = cdiv(p.B, BM);
+      ARD_TC_CASE(256, M_ROW_FWD, mt * cdiv(p.N, 256))
+      ARD_TC_CASE(128, M_ROW_FWD, mt * cdiv(p.N, 128))
+      ARD_TC_CASE(64, M_ROW_FWD, mt * cdiv(p.N, 64))
+    } else if (op == OP_BWD_DATA) {
+      const int mt = cdiv(p.B, BM);
+      ARD_TC_CASE(256, M_ROW_BWD_DATA, mt * cdiv(p.K, 256))
+      ARD_TC_CASE(128, M_ROW_BWD_DATA, mt * cdiv(p.K, 128))
+      ARD_TC_CASE(64, M_ROW_BWD_DATA, mt * cdiv(p.K, 64))
+    } else {
+      const int mt = cdiv(p.N, BM);
+      ARD_TC_CASE(256, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 256))
+      ARD_TC_CASE(128, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 128))
+      ARD_TC_CASE(64, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 64))
+    }
+  } else {
+    if (op == OP_FWD) {
+      const int mt = cdiv(p.B, BM);
+      ARD_TC_CASE(128, M_TILE_FWD, mt * cdiv(p.N, 128))
+      ARD_TC_CASE(64, M_TILE_FWD, mt * cdiv(p.N, 64))
+    } else if (op == OP_BWD_DATA) {
+      const int mt = cdiv(p.B, BM);
+      ARD_TC_CASE(128, M_TILE_BWD_DATA, mt * cdiv(p.K, 128))
+      ARD_TC_CASE(64, M_TILE_BWD_DATA, mt * cdiv(p.K, 64))
+    } else {
+      const int tiles = (p.K / p.ts) * (p.N / p.ts) * cdiv(p.ts, BM) * (p.ts / bn);
+      ARD_TC_CASE(256, M_TILE_BWD_WEIGHT, tiles)
+      ARD_TC_CASE(128, M_TILE_BWD_WEIGHT, tiles)
+      ARD_TC_CASE(64, M_TILE_BWD_WEIGHT, tiles)
+    }
+  }
+#undef ARD_TC_CASE
+  return ARD_ERR_UNSUPPORTED;
+}

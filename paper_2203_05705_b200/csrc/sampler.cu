@@ -1,0 +1,125 @@
+// Device-side pattern sampler (Sec. 3.4) and kept-unit list emitter (Sec. 3.1 Eq. 1, Sec. 3.2).
+//
+// One CTA per call.  Thread 0 runs Philox4x32-10 on the (seed, iteration, stream) counter, picks
+// the period dp from the integer cumulative table of K and the bias b uniformly from {1..dp};
+// all threads then write the header and the lists the GEMM kernels read.  Nothing returns to the
+// host, so the GEMMs that follow on the same stream need no synchronisation.
+#include "ard_internal.h"
+
+namespace {
+
+__device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+  uint32_t hi0 = __umulhi(M0, c[0]), lo0 = M0 * c[0];
+  uint32_t hi1 = __umulhi(M1, c[2]), lo1 = M1 * c[2];
+  uint32_t n0 = hi1 ^ c[1] ^ k0;
+  uint32_t n2 = hi0 ^ c[3] ^ k1;
+  c[0] = n0;
+  c[1] = lo1;
+  c[2] = n2;
+  c[3] = lo0;
+}
+
+__device__ void philox4x32_10(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
+  const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    philox_round(c, k0, k1);
+    k0 += W0;
+    k1 += W1;
+  }
+}
+
+constexpr int SAMPLER_THREADS = 256;
+
+__global__ void __launch_bounds__(SAMPLER_THREADS)
+ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t* __restrict__ col_ptr,
+                  int32_t* __restrict__ col_idx, int32_t* __restrict__ row_ptr, int32_t* __restrict__ row_idx,
+                  const unsigned long long* __restrict__ cdf, int ndp, unsigned long long seed,
+                  unsigned long long iteration, uint32_t stream_id, int forced_dp, int forced_b, int kind,
+                  int units, int Tr, int Tc, int ts) {
+  __shared__ int s_dp, s_b;
+  if (threadIdx.x == 0) {
+    int dp, b;
+    if (forced_dp > 0) {
+      dp = forced_dp;
+      b = forced_b;
+    } else {
+      uint32_t c[4] = {(uint32_t)iteration, (uint32_t)(iteration >> 32), stream_id, 0u};
+      philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+      // dp = smallest i with r0 < c_i; the table is non-decreasing and ends at 2^32.
+      int lo = 0, hi = ndp - 1;  // answer index in [0, ndp-1]
+      const unsigned long long r0 = c[0];
+      while (lo < hi) {
+        int mid = (lo + hi) >> 1;
+        if (r0 < cdf[mid]) hi = mid; else lo = mid + 1;
+      }
+      dp = lo + 1;
+      b = 1 + (int)(((unsigned long long)c[1] * (unsigned long long)dp) >> 32);
+    }
+    s_dp = dp;
+    s_b = b;
+  }
+  __syncthreads();
+  const int dp = s_dp, b = s_b;
+  const int n_keep = (units - b) / dp + 1;
+  if (threadIdx.x == 0) {
+    hdr[HDR_KIND] = kind;
+    hdr[HDR_DP] = dp;
+    hdr[HDR_B] = b;
+    hdr[HDR_NKEEP] = n_keep;
+    hdr[HDR_UNITS] = units;
+    hdr[HDR_TR] = Tr;
+    hdr[HDR_TC] = Tc;
+    hdr[HDR_TS] = ts;
+    hdr[HDR_MAPIDX] = dp * (dp - 1) / 2 + (b - 1);
+  }
+  // Eq. 1 on the 1-based unit index i = b + j*dp  ->  0-based b-1 + j*dp, ascending.
+  for (int j = threadIdx.x; j < n_keep; j += SAMPLER_THREADS) idx[j] = b - 1 + j * dp;
+  if (kind != ARD_TILE) return;
+
+  // Tiles are numbered row-major, so the ascending list is already grouped by tile-row.
+  for (int j = threadIdx.x; j < n_keep; j += SAMPLER_THREADS) row_idx[j] = (b - 1 + j * dp) % Tc;
+  for (int r = threadIdx.x; r <= Tr; r += SAMPLER_THREADS) {
+    // kept tiles with 0-based linear index < r*Tc
+    const long long lim = (long long)r * Tc;  // count of j with b-1 + j*dp < lim
+    int cnt = 0;
+    if (lim > b - 1) cnt = (int)((lim - 1 - (b - 1)) / dp) + 1;
+    row_ptr[r] = cnt;
+  }
+  // Group by tile-column: count, prefix-sum, fill.
+  for (int c = threadIdx.x; c < Tc; c += SAMPLER_THREADS) {
+    int cnt = 0;
+    for (int r = 0; r < Tr; ++r) cnt += ((r * Tc + c - (b - 1)) % dp == 0) && (r * Tc + c >= b - 1);
+    col_ptr[c + 1] = cnt;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int run = 0;
+    col_ptr[0] = 0;
+    for (int c = 0; c < Tc; ++c) {
+      run += col_ptr[c + 1];
+      col_ptr[c + 1] = run;
+    }
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < Tc; c += SAMPLER_THREADS) {
+    int o = col_ptr[c];
+    for (int r = 0; r < Tr; ++r)
+      if ((r * Tc + c >= b - 1) && ((r * Tc + c - (b - 1)) % dp == 0)) col_idx[o++] = r;
+  }
+}
+
+}  // namespace
+
+ard_status launch_sampler(ard_ctx* ctx, ard_pattern* pat, const unsigned long long* d_cdf, int ndp, uint64_t seed,
+                          uint64_t iteration, uint32_t stream_id, int forced_dp, int forced_b, cudaStream_t s) {
+  ard_sample_kernel<<<1, SAMPLER_THREADS, 0, s>>>(pat->d_hdr, pat->d_idx, pat->d_col_ptr, pat->d_col_idx,
+                                                  pat->d_row_ptr, pat->d_row_idx, d_cdf, ndp,
+                                                  (unsigned long long)seed, (unsigned long long)iteration, stream_id,
+                                                  forced_dp, forced_b, (int)pat->kind, pat->units, pat->Tr, pat->Tc,
+                                                  pat->ts);
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}

@@ -1,9 +1,10 @@
-"""Seeded synthetic inputs shared by the tests, the benchmark and the CPU oracle.
+"""Seeded synthetic inputs shared by the tests, the benchmark and the CPU reference
+implementation used by the tests.
 
 This module holds none of the method's arithmetic: it only draws tensors with
 the shapes and value distributions of the paper's MLP / LSTM workloads (Sec. 7)
 and builds the pattern distribution K that is an *input* of the hot path.
-It imports neither the CUDA binding nor the oracle.
+It imports neither the CUDA binding nor that reference implementation.
 """
 from __future__ import annotations
 

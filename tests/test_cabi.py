@@ -1,0 +1,67 @@
+"""The C-ABI library builds for sm_100a, loads without a GPU and exports what include/ard.h declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def built():
+    from paper_2203_05705_b200 import build
+    return build.build()
+
+
+def _declared():
+    with open(os.path.join(ROOT, "include", "ard.h")) as f:
+        text = f.read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ard_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_declares_the_north_star_entry_points():
+    names = _declared()
+    for must in ["ard_sample_pattern", "ard_fwd", "ard_bwd_data", "ard_bwd_weight", "ard_lstm_gates"]:
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol(built):
+    lib = ctypes.CDLL(built)
+    for name in _declared():
+        assert hasattr(lib, name), name
+
+
+def test_binding_covers_every_declared_symbol(built):
+    from paper_2203_05705_b200 import ard
+    assert sorted(ard.EXPORTS) == _declared()
+    for name in ard.EXPORTS:
+        assert callable(getattr(ard, name)), name
+    assert ard.ard_status_string(0) == "ok"
+    assert "wait" in ard.ard_status_string(ard.ARD_ERR_TIMEOUT)
+
+
+def test_create_without_a_gpu_fails_loudly(built):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    from paper_2203_05705_b200 import ard
+    with pytest.raises(ard.ArdError) as e:
+        ard.ard_create(0, 0)
+    assert e.value.status == ard.ARD_ERR_CUDA
+
+
+def test_package_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2203_05705_b200")
+    for dirpath, _d, files in os.walk(pkg):
+        for fn in files:
+            if fn.endswith((".py", ".cu", ".h", ".cpp")):
+                with open(os.path.join(dirpath, fn)) as f:
+                    src = f.read()
+                assert not re.search(r"^\s*(from|import)\s+oracle\b|import_module\(.oracle", src, flags=re.M), fn
+                assert "oracle/" not in src and "oracle." not in src, fn
+    for fn in os.listdir(os.path.join(ROOT, "oracle")):
+        if fn.endswith(".py"):
+            with open(os.path.join(ROOT, "oracle", fn)) as f:
+                assert "paper_2203_05705_b200" not in f.read(), fn

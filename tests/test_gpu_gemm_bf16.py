@@ -1,0 +1,142 @@
+"""bf16 paths vs the oracle: tcgen05 kernels (every N tile) and the CUDA-core family, row and tile patterns.
+
+Sizes span several output tiles, several 64-wide contraction blocks and ragged tails in every
+dimension, and stay small enough for the fp64 oracle to finish in seconds.
+"""
+import numpy as np
+import pytest
+
+from paper_2203_05705_b200 import ard, inputs
+from gpu_helpers import Ctx, run_three_gemms, assert_ok, TOL
+
+pytestmark = pytest.mark.gpu
+
+ROW_PATTERNS = [(1, 1), (2, 1), (2, 2), (3, 2), (5, 5), (7, 1), (16, 4), (16, 16)]
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = Ctx(64 << 20)
+    yield c
+    c.close()
+
+
+def _layer(B, K, N, seed, wscale):
+    rng = np.random.default_rng(seed)
+    X = inputs.bf16_round(rng.standard_normal((B, K)).astype(np.float32))
+    W = inputs.bf16_round((rng.standard_normal((K, N)) * wscale).astype(np.float32))
+    dY = inputs.bf16_round(rng.standard_normal((B, N)).astype(np.float32))
+    return X, W, dY
+
+
+@pytest.mark.parametrize("bn", [128, 256, 64])
+def test_row_tensor_core(ctx, bn):
+    B, K, N = 300, 520, 1000
+    X, W, dY = _layer(B, K, N, 1, 0.05)
+    ard.ard_set_path(ctx.h, ard.ARD_PATH_TENSOR_CORE)
+    ard.ard_set_tile_n(ctx.h, bn)
+    pat = ctx.pattern(ard.ARD_ROW, K, N)
+    try:
+        for i, (dp, b) in enumerate(ROW_PATTERNS):
+            ard.ard_pattern_set(ctx.h, pat, dp, b)
+            res = run_three_gemms(ctx, pat, ard.ARD_ROW, ard.ARD_BF16, X, W, dY, dp, b, 1.0 / (1.0 - 0.5),
+                                  compact=(i % 2 == 1), zero_fill=(i % 3 != 2),
+                                  dw_dtype=ard.ARD_F32 if i % 2 else ard.ARD_BF16)
+            assert_ok(res, TOL[ard.ARD_BF16], (bn, dp, b))
+    finally:
+        ard.ard_set_path(ctx.h, ard.ARD_PATH_AUTO)
+        ard.ard_set_tile_n(ctx.h, 0)
+
+
+def test_row_tensor_core_padded_leading_dimensions(ctx):
+    B, K, N = 130, 200, 264
+    X, W, dY = _layer(B, K, N, 2, 0.05)
+    ard.ard_set_path(ctx.h, ard.ARD_PATH_TENSOR_CORE)
+    pat = ctx.pattern(ard.ARD_ROW, K, N)
+    try:
+        for dp, b in [(1, 1), (3, 3), (4, 2)]:
+            ard.ard_pattern_set(ctx.h, pat, dp, b)
+            for compact in (False, True):
+                res = run_three_gemms(ctx, pat, ard.ARD_ROW, ard.ARD_BF16, X, W, dY, dp, b, 2.0,
+                                      lds={"x": 208, "w": 216, "y": 272}, compact=compact)
+                assert_ok(res, TOL[ard.ARD_BF16], (dp, b, compact))
+    finally:
+        ard.ard_set_path(ctx.h, ard.ARD_PATH_AUTO)
+
+
+def test_row_sampled_patterns_auto_path(ctx):
+    from oracle import pattern as OP
+    B, K, N = 128, 784, 2048                         # first hidden layer of the 784-2048-2048-10 MLP
+    X, W, dY = _layer(B, K, N, 3, np.sqrt(2.0 / K))
+    Kd = inputs.max_entropy_K(0.5, 16)
+    cdf = OP.quantise_K(Kd)
+    ard.ard_set_distribution(ctx.h, 0, Kd)
+    pat = ctx.pattern(ard.ARD_ROW, K, N)
+    for it in range(12):
+        ard.ard_sample_pattern(ctx.h, pat, 0, inputs.BASE_SEED, it, 1)
+        dp, b = OP.draw(cdf, inputs.BASE_SEED, it, 1)
+        res = run_three_gemms(ctx, pat, ard.ARD_ROW, ard.ARD_BF16, X, W, dY, dp, b, 2.0)
+        assert_ok(res, TOL[ard.ARD_BF16], (it, dp, b))
+
+
+def test_row_cuda_core_family_bf16(ctx):
+    B, K, N = 70, 100, 90                            # K, N not multiples of 8: the TMA path cannot take these
+    X, W, dY = _layer(B, K, N, 4, 0.1)
+    pat = ctx.pattern(ard.ARD_ROW, K, N)
+    for dp, b in [(1, 1), (2, 2), (9, 4)]:
+        ard.ard_pattern_set(ctx.h, pat, dp, b)
+        for compact in (False, True):
+            res = run_three_gemms(ctx, pat, ard.ARD_ROW, ard.ARD_BF16, X, W, dY, dp, b, 1.5, compact=compact)
+            assert_ok(res, TOL[ard.ARD_BF16], (dp, b, compact))
+    ard.ard_set_path(ctx.h, ard.ARD_PATH_TENSOR_CORE)
+    try:
+        with pytest.raises(ard.ArdError) as e:
+            run_three_gemms(ctx, pat, ard.ARD_ROW, ard.ARD_BF16, X, W, dY, 9, 4, 1.5)
+        assert e.value.status == ard.ARD_ERR_ALIGNMENT
+    finally:
+        ard.ard_set_path(ctx.h, ard.ARD_PATH_AUTO)
+
+
+@pytest.mark.parametrize("ts,bn", [(64, 0), (128, 0), (128, 64), (256, 0)])
+def test_tile_tensor_core(ctx, ts, bn):
+    B, K, N = 200, 3 * ts, 5 * ts
+    X, W, dY = _layer(B, K, N, 5 + ts, 0.05)
+    ard.ard_set_path(ctx.h, ard.ARD_PATH_TENSOR_CORE)
+    ard.ard_set_tile_n(ctx.h, bn)
+    pat = ctx.pattern(ard.ARD_TILE, K, N, ts)
+    try:
+        for i, (dp, b) in enumerate([(1, 1), (2, 1), (3, 3), (4, 2), (5, 1), (15, 8)]):
+            ard.ard_pattern_set(ctx.h, pat, dp, b)
+            res = run_three_gemms(ctx, pat, ard.ARD_TILE, ard.ARD_BF16, X, W, dY, dp, b, 2.0, ts=ts,
+                                  zero_fill=(i % 2 == 0), dw_dtype=ard.ARD_F32 if i % 2 else ard.ARD_BF16)
+            assert_ok(res, TOL[ard.ARD_BF16], (ts, dp, b))
+    finally:
+        ard.ard_set_path(ctx.h, ard.ARD_PATH_AUTO)
+        ard.ard_set_tile_n(ctx.h, 0)
+
+
+def test_tile_cuda_core_family_bf16(ctx):
+    B, K, N, ts = 50, 64, 96, 32
+    X, W, dY = _layer(B, K, N, 9, 0.1)
+    pat = ctx.pattern(ard.ARD_TILE, K, N, ts)
+    for dp, b in [(1, 1), (2, 1), (3, 2), (6, 6)]:
+        ard.ard_pattern_set(ctx.h, pat, dp, b)
+        res = run_three_gemms(ctx, pat, ard.ARD_TILE, ard.ARD_BF16, X, W, dY, dp, b, 2.0, ts=ts)
+        assert_ok(res, TOL[ard.ARD_BF16], (dp, b))
+
+
+def test_small_workspace_is_reported(ctx):
+    c2 = Ctx(1024)
+    try:
+        B, K, N = 128, 128, 128
+        X, W, dY = _layer(B, K, N, 10, 0.1)
+        pat = c2.pattern(ard.ARD_ROW, K, N)
+        ard.ard_set_path(c2.h, ard.ARD_PATH_TENSOR_CORE)
+        with pytest.raises(ard.ArdError) as e:
+            run_three_gemms(c2, pat, ard.ARD_ROW, ard.ARD_BF16, X, W, dY, 1, 1, 1.0)
+        assert e.value.status == ard.ARD_ERR_NOMEM
+        ard.ard_set_path(c2.h, ard.ARD_PATH_AUTO)         # falls back to the CUDA-core family
+        res = run_three_gemms(c2, pat, ard.ARD_ROW, ard.ARD_BF16, X, W, dY, 1, 1, 1.0)
+        assert_ok(res, TOL[ard.ARD_BF16])
+    finally:
+        c2.close()

@@ -25,12 +25,12 @@ def test_philox_known_answers():
 def test_paper_worked_examples():
     # Sec. 3.1: dp=3, b=1 keeps rows 1, 4, 7 (1-based)
     assert (P.row_keep(9, 3, 1) + 1).tolist() == [1, 4, 7]
-    # Sec. 3.2: dp=4, b=1 keeps the first of every 4 successive tiles
+    # Sec. 3.2: dp=4, b=1 keeps tiles 1, 5, 9, 13
     kept = P.tile_keep(4 * 2, 4 * 2, 2, 4, 1)          # 4x4 grid of 2x2 tiles
     t = (kept[:, 0] * 4 + kept[:, 1] + 1).tolist()
     assert t == [1, 5, 9, 13]
     M = P.tile_mask(8, 8, 2, 4, 1)
-    assert M.sum() == 8 * 8 / 4                          # "1/4 of the original scale"
+    assert M.sum() == 8 * 8 / 4                          # a quarter of the synapses survive
     # Sec. 6: mask convention 1 = keep
     m = np.zeros(6)
     m[[0, 2, 3]] = 1
