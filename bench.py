@@ -56,7 +56,7 @@ def kept_count(units, dp, b):
 
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
@@ -65,12 +65,22 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                       "--format=csv,noheader,nounits", "-lms", "50"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
 
-    def stop(self):
+    @staticmethod
+    def _ts(s):
+        import datetime
+        try:
+            return datetime.datetime.strptime(s, "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except ValueError:
+            return None
+
+    def stop(self, t_begin=None, t_end=None):
+        """Median SM clock over the samples taken inside [t_begin, t_end] (wall clock), else over the
+        busier half of all samples."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
             return out
@@ -81,25 +91,32 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, reasons, inside = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.f.read().splitlines():
             parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 7:
+            if len(parts) < 8:
                 continue
             try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
+                clk = float(parts[1])
+                mx.append(float(parts[2]))
             except ValueError:
                 continue
-            for nm, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
+            sm.append(clk)
+            ts = self._ts(parts[0])
+            hit = ts is not None and t_begin is not None and t_begin - 0.05 <= ts <= t_end + 0.05
+            if hit:
+                inside.append(clk)
+            if hit or t_begin is None:
+                for nm, val in zip(names, parts[4:8]):
+                    if val.lower().startswith("active"):
+                        reasons.add(nm)
         self.f.close()
         os.unlink(self.f.name)
         if sm:
-            top = sorted(sm)[len(sm) // 2:]           # upper half = samples under load
-            out.update(sm_mhz=statistics.median(top), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+            use = inside if inside else sorted(sm)[len(sm) // 2:]
+            out.update(sm_mhz=statistics.median(use), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(use), window="timed region" if inside else "busier half of the run")
         return out
 
 
@@ -160,11 +177,12 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mlp8192_row", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true", help="headline region only (for profiler captures)")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -236,6 +254,8 @@ def main():
             out.append((dp_, b_, nk))
         return out
 
+    wall = [0.0, 0.0]
+
     def timed_run(pp, first_it, per_kernel=False):
         for w in range(args.warmup):
             step(pp, first_it + w)
@@ -243,11 +263,13 @@ def main():
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in its] if per_kernel else None
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
+        wall[0] = time.time()
         e0.record()
         for i, it in enumerate(its):
             step(pp, it, evs[i] if per_kernel else None)
         e1.record()
         barrier()
+        wall[1] = time.time()
         ms = e0.elapsed_time(e1)
         per = None
         if per_kernel:
@@ -281,10 +303,11 @@ def main():
         return e0.elapsed_time(e1)
 
     # ---- the timed region the headline value comes from (p = 0.5) ----
-    launches0 = ard.ard_launch_count(ctx)
     clocks = ClockSampler(local)
+    launches0 = ard.ard_launch_count(ctx)
     ms, its, per = timed_run(p, 0, per_kernel=True)
-    clk = clocks.stop()
+    t_begin, t_end = wall
+    clk = clocks.stop(t_begin, t_end)
     launches = (ard.ard_launch_count(ctx) - launches0) * args.steps // (args.steps + args.warmup)
     status = ard.ard_last_device_status(ctx)
     pats = kept_units_of(p, its)
@@ -325,6 +348,13 @@ def main():
 
     # ---- dense baselines and the other dropout rates (outside the headline region) ----
     detail = {}
+    if args.quick:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": kept_tflops, "unit": UNIT, "quick": True,
+                              "ms_per_step": ms / args.steps, "roofline": roofline, "clocks": clk}))
+        ard.ard_pattern_destroy(pat)
+        ard.ard_destroy(ctx)
+        return
     dense_ms = dense_run()
     torch_ms = torch_dense_run()
     best_dense = min(dense_ms, torch_ms)
