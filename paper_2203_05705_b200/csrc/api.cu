@@ -45,9 +45,10 @@ constexpr size_t MAX_CACHED_TABLES = 96;
 
 // Returns a device table of descriptors for `base`; builds and caches it on first use.
 ard_status get_maps(ard_ctx* ctx, const void* base, int rows, int cols, int ld, int units, int variant, int dp_bound,
-                    int box_rows, int box_cols, const CUtensorMap** out) {
+                    int box_rows, int box_cols, const CUtensorMap** out, const void* dense_base = nullptr,
+                    int dense_ld = 0) {
   for (const MapTable& t : ctx->maps) {
-    if (t.base == base && t.rows == rows && t.cols == cols && t.ld == ld && t.elem_bytes == units &&
+    if (t.base == base && t.dense_base == dense_base && t.dense_ld == dense_ld && t.rows == rows && t.cols == cols && t.ld == ld && t.elem_bytes == units &&
         t.variant == variant && t.dp_bound == dp_bound && t.box_rows == box_rows && t.box_cols == box_cols) {
       *out = t.d_maps;
       return ARD_OK;
@@ -70,8 +71,12 @@ ard_status get_maps(ard_ctx* ctx, const void* base, int rows, int cols, int ld, 
                                        box_cols, box_rows)
                           : encode_map(ctx, m, base, cols, 1, (uint64_t)ld * 2, box_cols, box_rows);
         } else {
-          // compact matrix: all rows, columns 0..nk-1
-          ok = encode_map(ctx, m, base, nk, rows, (uint64_t)ld * 2, box_cols, box_rows);
+          // compact matrix: all rows, columns 0..nk-1.  A dense pattern needs no compaction: its
+          // entry may point straight at the full-width matrix.
+          if (dp == 1 && dense_base != nullptr)
+            ok = encode_map(ctx, m, dense_base, nk, rows, (uint64_t)dense_ld * 2, box_cols, box_rows);
+          else
+            ok = encode_map(ctx, m, base, nk, rows, (uint64_t)ld * 2, box_cols, box_rows);
         }
         if (!ok) return ARD_ERR_CUDA;
       }
@@ -82,7 +87,7 @@ ard_status get_maps(ard_ctx* ctx, const void* base, int rows, int cols, int ld, 
     ctx->maps.erase(ctx->maps.begin());
   }
   MapTable t;
-  t.base = base; t.rows = rows; t.cols = cols; t.ld = ld; t.elem_bytes = units; t.variant = variant;
+  t.base = base; t.dense_base = dense_base; t.dense_ld = dense_ld; t.rows = rows; t.cols = cols; t.ld = ld; t.elem_bytes = units; t.variant = variant;
   t.dp_bound = dp_bound; t.box_rows = box_rows; t.box_cols = box_cols; t.count = count;
   t.d_maps = nullptr;
   if (cudaMalloc(&t.d_maps, sizeof(CUtensorMap) * count) != cudaSuccess) return ARD_ERR_NOMEM;
@@ -420,15 +425,21 @@ ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B,
 // Produces the operand the tensor-core backward GEMMs read for dY: the caller's compact matrix, or
 // a compacted copy of the full-width one in the context workspace (row patterns only).
 static ard_status compact_dy(ard_ctx* ctx, const ard_pattern* pat, int B, int N, const void* dY, int lddy,
-                             int dy_is_compact, const void** out_ptr, int* out_ld, cudaStream_t s) {
+                             int dy_is_compact, const void** out_ptr, int* out_ld, const void** dense_ptr,
+                             int* dense_ld, cudaStream_t s) {
+  *dense_ptr = nullptr;
+  *dense_ld = 0;
   if (dy_is_compact) {
     *out_ptr = dY;
     *out_ld = lddy;
     return ARD_OK;
   }
+  // A dense pattern (dp = 1) is not copied: the descriptor of that case reads dY itself.
+  *dense_ptr = dY;
+  *dense_ld = lddy;
   const int ldc = (N + 7) / 8 * 8;
   if ((size_t)B * ldc * 2 > ctx->workspace_bytes) return ARD_ERR_NOMEM;
-  ard_status st = launch_gather_cols(ctx, pat->d_hdr, pat->d_idx, dY, lddy, ctx->d_workspace, ldc, B, 2, N, s);
+  ard_status st = launch_gather_cols(ctx, pat->d_hdr, pat->d_idx, dY, lddy, ctx->d_workspace, ldc, B, 2, N, 1, s);
   *out_ptr = ctx->d_workspace;
   *out_ld = ldc;
   return st;
@@ -468,13 +479,13 @@ ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, i
   t.ts = pat->ts;
   t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_DATA, B, K, N, pat->ts);
   if (pat->kind == ARD_ROW) {
-    const void* dyc;
-    int ldc;
-    st = compact_dy(ctx, pat, B, N, dY, lddy, dy_is_compact, &dyc, &ldc, s);
+    const void *dyc, *dense;
+    int ldc, dense_ld;
+    st = compact_dy(ctx, pat, B, N, dY, lddy, dy_is_compact, &dyc, &ldc, &dense, &dense_ld, s);
     if (st != ARD_OK) return st;
     g.A0 = dyc; g.lda0 = ldc; g.flag0 = 1;
     // A = compact dY [B][n_keep], K-major;  B = kept neurons of W read MN-major: boxes [64 kept rows][64 k].
-    st = get_maps(ctx, dyc, B, N, ldc, N, MAP_COMPACT_COLS, pat->dp_bound, 128, 64, &t.mapA);
+    st = get_maps(ctx, dyc, B, N, ldc, N, MAP_COMPACT_COLS, pat->dp_bound, 128, 64, &t.mapA, dense, dense_ld);
     if (st != ARD_OK) return st;
     t.mapA_indexed = 1;
     st = get_maps(ctx, W, N, K, ldw, N, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64, &t.mapB);
@@ -529,13 +540,13 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
   t.ts = pat->ts;
   t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_WEIGHT, B, K, N, pat->ts);
   if (pat->kind == ARD_ROW) {
-    const void* dyc;
-    int ldc;
-    st = compact_dy(ctx, pat, B, N, dY, lddy, dy_is_compact, &dyc, &ldc, s);
+    const void *dyc, *dense;
+    int ldc, dense_ld;
+    st = compact_dy(ctx, pat, B, N, dY, lddy, dy_is_compact, &dyc, &ldc, &dense, &dense_ld, s);
     if (st != ARD_OK) return st;
     g.A0 = dyc; g.lda0 = ldc; g.flag0 = 1;
     // A = compact dY read MN-major (boxes [64 batch rows][64 kept cols]);  B = X read MN-major.
-    st = get_maps(ctx, dyc, B, N, ldc, N, MAP_COMPACT_COLS, pat->dp_bound, 64, 64, &t.mapA);
+    st = get_maps(ctx, dyc, B, N, ldc, N, MAP_COMPACT_COLS, pat->dp_bound, 64, 64, &t.mapA, dense, dense_ld);
     t.mapA_indexed = 1;
   } else {
     if (zero_fill_dropped) ARD_CUDA_OK(cudaMemset2DAsync(dW, (size_t)lddw * es_out, 0, (size_t)K * es_out, N, s));

@@ -47,6 +47,8 @@ struct ArdDistribution {
 // A cached table of TMA descriptors in device memory, one per (dp, b) pair (or a single one).
 struct MapTable {
   const void* base;
+  const void* dense_base;  // MAP_COMPACT_COLS: matrix the dp = 1 entry points at (nullptr: same as base)
+  int dense_ld;
   int rows, cols, ld, elem_bytes;
   int box_rows, box_cols;
   int variant;   // see MapVariant
@@ -122,7 +124,8 @@ int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int B, int K, int N, int 
 ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s);
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,
-                              void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, cudaStream_t s);
+                              void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, int skip_dense,
+                              cudaStream_t s);
 
 ard_status launch_lstm_gates(ard_ctx* ctx, const ard_pattern* pat, ard_dtype h_dtype, int B, int H, float alpha,
                              const float* Z, int ldz_gate, const float* bias, const float* c_prev, int ldc, float* c,

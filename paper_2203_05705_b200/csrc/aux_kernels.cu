@@ -16,6 +16,66 @@ __global__ void __launch_bounds__(256) gather_cols_kernel(const int32_t* __restr
   for (int r = blockIdx.y; r < rows; r += gridDim.y) dst[(size_t)r * ld_dst + j] = src[(size_t)r * ld_src + col];
 }
 
+// Faster form for 2-byte elements with 16-byte aligned rows: a block stages the source span of up to
+// 1024 outputs in shared memory with coalesced 16-byte loads, then every thread assembles 8 kept
+// values into one 16-byte store.  With skip_dense != 0 a dense pattern (dp = 1) is left alone: the
+// GEMM then reads the original matrix directly.
+constexpr int GATHER_SPAN = 16384;  // staged source elements
+
+__global__ void __launch_bounds__(256)
+gather_cols_staged_kernel(const int32_t* __restrict__ hdr, const uint16_t* __restrict__ src, int ld_src,
+                          uint16_t* __restrict__ dst, int ld_dst, int rows, int n_cols, int skip_dense) {
+  __shared__ __align__(16) uint16_t buf[GATHER_SPAN + 16];
+  const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
+  if (skip_dense && dp == 1) return;
+  int outs = (GATHER_SPAN / dp) & ~7;
+  if (outs > 1024) outs = 1024;
+  if (outs < 8) {
+    // period too long for the staging buffer: element-wise copy
+    for (long long e = (long long)blockIdx.x * 256 + threadIdx.x; e < (long long)rows * n_keep;
+         e += (long long)gridDim.x * 256) {
+      const int r = (int)(e / n_keep), j = (int)(e % n_keep);
+      dst[(size_t)r * ld_dst + j] = src[(size_t)r * ld_src + bb + (long long)j * dp];
+    }
+    return;
+  }
+  const int chunks = (n_keep + outs - 1) / outs;
+  for (long long item = blockIdx.x; item < (long long)rows * chunks; item += gridDim.x) {
+    const int r = (int)(item / chunks), ch = (int)(item % chunks);
+    const int j0 = ch * outs;
+    const int nout = min(outs, n_keep - j0);
+    const int s0 = bb + j0 * dp;                 // first source column
+    const int a0 = s0 & ~7;                      // 16-byte aligned start
+    const int count = bb + (j0 + nout - 1) * dp - a0 + 1;
+    const uint16_t* srow = src + (size_t)r * ld_src;
+    for (int v = threadIdx.x; v * 8 < count; v += 256) {
+      const int col = a0 + 8 * v;
+      if (col + 8 <= ld_src) {
+        *reinterpret_cast<uint4*>(buf + 8 * v) = *reinterpret_cast<const uint4*>(srow + col);
+      } else {
+        for (int i = 0; i < 8; ++i) buf[8 * v + i] = (col + i < n_cols) ? srow[col + i] : (uint16_t)0;
+      }
+    }
+    __syncthreads();
+    const int off = s0 - a0;
+    uint16_t* drow = dst + (size_t)r * ld_dst + j0;
+    for (int t = threadIdx.x; t * 8 < nout; t += 256) {
+      if (t * 8 + 8 <= nout) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t lo = buf[off + (t * 8 + 2 * i) * dp], hi = buf[off + (t * 8 + 2 * i + 1) * dp];
+          w[i] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4*>(drow + t * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+      } else {
+        for (int i = t * 8; i < nout; ++i) drow[i] = buf[off + i * dp];
+      }
+    }
+    __syncthreads();
+  }
+}
+
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + __expf(-x)); }
 
 template <typename HT>
@@ -94,14 +154,22 @@ lstm_gates_bwd_kernel(const int32_t* __restrict__ hdr, int B, int H, float alpha
 }  // namespace
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,
-                              void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, cudaStream_t s) {
+                              void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, int skip_dense,
+                              cudaStream_t s) {
   (void)idx;
   if (rows == 0 || max_cols == 0) return ARD_OK;
-  dim3 grid((max_cols + 255) / 256, rows < 1024 ? rows : 1024);
-  if (elem_bytes == 2)
-    gather_cols_kernel<uint16_t><<<grid, 256, 0, s>>>(hdr, (const uint16_t*)src, ld_src, (uint16_t*)dst, ld_dst, rows);
-  else
-    gather_cols_kernel<uint32_t><<<grid, 256, 0, s>>>(hdr, (const uint32_t*)src, ld_src, (uint32_t*)dst, ld_dst, rows);
+  const bool vec_ok = elem_bytes == 2 && ld_src % 8 == 0 && ld_dst % 8 == 0 &&
+                      (reinterpret_cast<uintptr_t>(src) & 15) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0;
+  if (vec_ok) {
+    gather_cols_staged_kernel<<<ctx->sm_count * 8, 256, 0, s>>>(hdr, (const uint16_t*)src, ld_src, (uint16_t*)dst,
+                                                                 ld_dst, rows, max_cols, skip_dense);
+  } else {
+    dim3 grid((max_cols + 255) / 256, rows < 1024 ? rows : 1024);
+    if (elem_bytes == 2)
+      gather_cols_kernel<uint16_t><<<grid, 256, 0, s>>>(hdr, (const uint16_t*)src, ld_src, (uint16_t*)dst, ld_dst, rows);
+    else
+      gather_cols_kernel<uint32_t><<<grid, 256, 0, s>>>(hdr, (const uint32_t*)src, ld_src, (uint32_t*)dst, ld_dst, rows);
+  }
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;

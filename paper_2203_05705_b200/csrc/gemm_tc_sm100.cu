@@ -477,58 +477,52 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
           for (int i = 0; i < 32; ++i) v[i] = 0.f;
         }
 
-        if (MODE == M_ROW_FWD && p.scatter) {
+        if (MODE == M_ROW_FWD && p.scatter && sch.dp > 1) {
           // Full-width rows: compact column j -> column b-1 + j*dp, zeros everywhere else
-          // (Sec. 3.1: dropped outputs are zero).  Staged through shared memory so that
-          // consecutive lanes write consecutive 16-byte pieces of one output row.
+          // (Sec. 3.1: dropped outputs are zero).  The 32x32 block is staged through shared memory
+          // and the (row, 16-byte piece) pairs of the 32 x 32*dp output block are dealt to the lanes
+          // round-robin, so consecutive lanes write consecutive pieces of one output row.
           if (n < sch.n_keep) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) stg[lane * 33 + i] = v[i];
             __syncwarp();
             const int dp = sch.dp, bb = sch.b - 1;
-            const long long cs = (long long)n * dp;
+            const int cs = n * dp;
             const bool last = n + 32 >= sch.n_keep;
-            const long long ce = last ? (long long)p.N : min((long long)(n + 32) * dp, (long long)p.N);
-            const int groups = (int)((ce - cs + 7) / 8);
+            const int ce = last ? p.N : min((n + 32) * dp, p.N);
+            const int groups = (ce - cs + 7) >> 3;  // 16-byte pieces per output row
             const int rows_here = min(32, sch.M_gemm - (ti.m0 + q * 32));
-            for (int rr = 0; rr < rows_here; ++rr) {
-              __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)(ti.m0 + q * 32 + rr) * p.ldo;
-              float* ofrow = reinterpret_cast<float*>(p.out) + (size_t)(ti.m0 + q * 32 + rr) * p.ldo;
-              for (int g = lane; g < groups; g += 32) {
-                const long long c0 = cs + 8ll * g;
-                // Walk the 8 columns of this piece keeping (compact column, remainder) of c - (b-1);
-                // a column is kept exactly when the remainder is zero (Eq. 1).
-                const long long rel = c0 - bb;  // negative only before the first kept column
-                int cq, cr;
-                if (rel >= 0) { cq = (int)(rel / dp); cr = (int)(rel % dp); }
-                else { cq = -1; cr = (int)(rel + dp); }
-                float w[8];
+            const int items = rows_here * groups;
+            __nv_bfloat16* obase = reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)(ti.m0 + q * 32) * p.ldo;
+            for (int w = lane; w < items; w += 32) {
+              const int rr = w / groups, g = w - rr * groups;
+              const int c0 = cs + 8 * g;
+              __nv_bfloat16* dst = obase + (size_t)rr * p.ldo + c0;
+              // (compact column, remainder) of c0 - (b-1); a column is kept when the remainder is 0 (Eq. 1).
+              const int rel = c0 - bb;  // negative only before the first kept column
+              int cq, cr;
+              if (rel >= 0) { cq = rel / dp; cr = rel - cq * dp; }
+              else { cq = -1; cr = rel + dp; }
+              const int first_kept = cr == 0 ? 0 : dp - cr;  // position of the first kept column
+              const int nleft = ce - c0;
+              if (first_kept >= 8 && nleft >= 8) {
+                *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+                continue;
+              }
+              float x[8];
+              const float* srow = stg + rr * 33 - n;
 #pragma unroll
-                for (int pos = 0; pos < 8; ++pos) {
-                  const bool kept = cr == 0;
-                  w[pos] = kept ? stg[rr * 33 + (cq - n)] : 0.f;
-                  if (++cr == dp) { cr = 0; ++cq; }
-                }
-                const long long nleft = ce - c0;
-                if (p.out_is_f32) {
-                  if (nleft >= 8) {
-                    reinterpret_cast<float4*>(ofrow + c0)[0] = make_float4(w[0], w[1], w[2], w[3]);
-                    reinterpret_cast<float4*>(ofrow + c0)[1] = make_float4(w[4], w[5], w[6], w[7]);
-                  } else {
+              for (int pos = 0; pos < 8; ++pos) {
+                x[pos] = (cr == 0) ? srow[cq] : 0.f;
+                if (++cr == dp) { cr = 0; ++cq; }
+              }
+              if (nleft >= 8) {
+                *reinterpret_cast<uint4*>(dst) = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]),
+                                                            pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+              } else {
 #pragma unroll
-                    for (int pos = 0; pos < 8; ++pos)
-                      if (pos < nleft) ofrow[c0 + pos] = w[pos];
-                  }
-                } else {
-                  if (nleft >= 8) {
-                    *reinterpret_cast<uint4*>(orow + c0) = make_uint4(pack_bf16(w[0], w[1]), pack_bf16(w[2], w[3]),
-                                                                      pack_bf16(w[4], w[5]), pack_bf16(w[6], w[7]));
-                  } else {
-#pragma unroll
-                    for (int pos = 0; pos < 8; ++pos)
-                      if (pos < nleft) orow[c0 + pos] = __float2bfloat16_rn(w[pos]);
-                  }
-                }
+                for (int pos = 0; pos < 8; ++pos)
+                  if (pos < nleft) dst[pos] = __float2bfloat16_rn(x[pos]);
               }
             }
             __syncwarp();
