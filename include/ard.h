@@ -143,6 +143,28 @@ ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, i
                         const void* dY, int lddy, int dy_is_compact, const void* W, int ldw, void* dX, int lddx,
                         void* cuda_stream);
 
+/* Backward-data without any allocation (the paper has no counterpart: this is a deployment
+ * variant of ard_bwd_data, same result).  For callers that are not allowed to allocate device
+ * memory when they run the layer: a process whose memory plan was frozen after start-up, a plug-in
+ * inside an application that owns the allocator, or anyone who must avoid the device-wide
+ * synchronisation of cudaMalloc / cudaFree.  ard_bwd_data can allocate (descriptor tables on first
+ * use of new buffers); this call never does, and neither calls cudaMalloc / cudaFree nor any
+ * allocating library routine.
+ *   Row patterns only, full-width dY [B][N] (lddy), W [N][K] (ldw), dX [B][K] (lddx); runs on the
+ *   CUDA cores (fp32 accumulate) for both dtypes.  The compacted copy of dY is kept in a fixed
+ *   array inside the library image: ARD_STATIC_SCRATCH_BYTES per GPU that loads the library, held
+ *   until the process exits.  B*N*sizeof(element) must not exceed that size, otherwise the call
+ *   returns ARD_ERR_NOMEM and launches nothing.
+ *   The first call on each device looks up the array's device address; make that first call before
+ *   starting any stream capture.  Every call on a device shares the one array, which keeps the
+ *   previous call's contents (all entries that are read are rewritten first; nothing needs
+ *   clearing).  Calls that overlap on the GPU (other streams, other host threads) race on it:
+ *   serialise them. */
+#define ARD_STATIC_SCRATCH_BYTES (8u << 20)
+ard_status ard_bwd_data_static_scratch(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N,
+                                       float alpha, const void* dY, int lddy, const void* W, int ldw, void* dX,
+                                       int lddx, void* cuda_stream);
+
 /* Backward-weight:  dW = alpha * (X^T dY) .* Mask, stored neuron-major dW [N][K] (lddw), element
  *   type dW_dtype (fp32 or bf16; an ARD_F32 layer requires ARD_F32).  Only kept rows (row pattern)
  *   or kept tiles (tile pattern) are computed and written; if zero_fill_dropped != 0 the dropped

@@ -23,12 +23,13 @@ ARD_F32, ARD_BF16 = 0, 1
 ARD_ROW, ARD_TILE = 0, 1
 ARD_OUT_COMPACT, ARD_OUT_SCATTER_ZEROFILL = 0, 1
 ARD_PATH_AUTO, ARD_PATH_CUDA_CORE, ARD_PATH_TENSOR_CORE = 0, 1, 2
+ARD_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = [
     "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_distribution", "ard_get_distribution_cdf",
     "ard_pattern_create", "ard_pattern_destroy", "ard_sample_pattern", "ard_pattern_set",
     "ard_pattern_to_host", "ard_pattern_tile_lists_to_host", "ard_fwd", "ard_bwd_data", "ard_bwd_weight",
-    "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_last_device_status", "ard_status_string", "ard_launch_count",
+    "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_last_device_status", "ard_status_string", "ard_launch_count",
 ]
 
 _lib = None
@@ -66,6 +67,7 @@ def lib():
         "ard_pattern_tile_lists_to_host": [vp, P(C.c_int32), P(C.c_int32), P(C.c_int32), P(C.c_int32), vp],
         "ard_fwd": [vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, i32, vp],
         "ard_bwd_data": [vp, vp, i32, i32, i32, i32, f32, vp, i32, i32, vp, i32, vp, i32, vp],
+        "ard_bwd_data_static_scratch": [vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_bwd_weight": [vp, vp, i32, i32, i32, i32, i32, f32, vp, i32, vp, i32, i32, vp, i32, i32, vp],
         "ard_lstm_gates": [vp, vp, i32, i32, i32, f32, vp, i32, vp, vp, i32, vp, vp, i32, i32, vp, vp],
         "ard_lstm_gates_bwd": [vp, vp, i32, i32, i32, f32, vp, vp, vp, i32, vp, i32, i32, vp, vp, i32, vp],
@@ -187,6 +189,13 @@ def ard_fwd(ctx, pat, dtype, B, K, N, alpha, X, ldx, W, ldw, Y, ldy, outmode, st
 def ard_bwd_data(ctx, pat, dtype, B, K, N, alpha, dY, lddy, dy_is_compact, W, ldw, dX, lddx, stream=None):
     _check(lib().ard_bwd_data(ctx, pat, dtype, B, K, N, alpha, _ptr(dY), lddy, dy_is_compact, _ptr(W), ldw,
                               _ptr(dX), lddx, _stream(stream)), "ard_bwd_data")
+
+
+def ard_bwd_data_static_scratch(ctx, pat, dtype, B, K, N, alpha, dY, lddy, W, ldw, dX, lddx, stream=None):
+    """Backward-data for callers that must not allocate: same result as ard_bwd_data (row pattern,
+    full-width dY), with the compacted dY kept in the library's fixed device array."""
+    _check(lib().ard_bwd_data_static_scratch(ctx, pat, dtype, B, K, N, alpha, _ptr(dY), lddy, _ptr(W), ldw,
+                                             _ptr(dX), lddx, _stream(stream)), "ard_bwd_data_static_scratch")
 
 
 def ard_bwd_weight(ctx, pat, dtype, dW_dtype, B, K, N, alpha, X, ldx, dY, lddy, dy_is_compact, dW, lddw,
