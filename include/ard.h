@@ -74,6 +74,13 @@ typedef enum { ARD_PATH_AUTO = 0, ARD_PATH_CUDA_CORE = 1, ARD_PATH_TENSOR_CORE =
 ard_status ard_create(ard_ctx** ctx, int device, size_t workspace_bytes);
 ard_status ard_destroy(ard_ctx* ctx);
 ard_status ard_set_path(ard_ctx* ctx, ard_path path);
+/* Opt-in for training loops.  The tensor-core backward GEMMs of a row pattern read a compacted copy
+ * of a full-width dY (kept columns only) that the library makes in the context workspace.  With
+ * enable != 0, a backward call whose dY pointer, leading dimension, batch size, pattern sample and
+ * stream equal those of the previous backward call on this context reuses that copy instead of
+ * gathering again (ard_bwd_data followed by ard_bwd_weight of the same layer then gather once).
+ * Enable only if dY is not written between such calls.  Default: off. */
+ard_status ard_set_compact_reuse(ard_ctx* ctx, int enable);
 /* Tuning / test knob of the tensor-core path: forces the N extent of the output tile (64, 128 or
  * 256; 0 restores the built-in choice).  A forced value a product cannot use is ignored for it. */
 ard_status ard_set_tile_n(ard_ctx* ctx, int bn);

@@ -26,7 +26,7 @@ ARD_PATH_AUTO, ARD_PATH_CUDA_CORE, ARD_PATH_TENSOR_CORE = 0, 1, 2
 ARD_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = [
-    "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_distribution", "ard_get_distribution_cdf",
+    "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_compact_reuse", "ard_set_distribution", "ard_get_distribution_cdf",
     "ard_pattern_create", "ard_pattern_destroy", "ard_sample_pattern", "ard_pattern_set",
     "ard_pattern_to_host", "ard_pattern_tile_lists_to_host", "ard_fwd", "ard_bwd_data", "ard_bwd_weight",
     "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_last_device_status", "ard_status_string", "ard_launch_count",
@@ -57,6 +57,7 @@ def lib():
         "ard_destroy": [vp],
         "ard_set_path": [vp, i32],
         "ard_set_tile_n": [vp, i32],
+        "ard_set_compact_reuse": [vp, i32],
         "ard_set_distribution": [vp, i32, P(C.c_double), i32],
         "ard_get_distribution_cdf": [vp, i32, P(u64), i32, P(i32)],
         "ard_pattern_create": [vp, P(vp), i32, i32, i32, i32],
@@ -119,6 +120,10 @@ def ard_destroy(ctx):
 
 def ard_set_path(ctx, path):
     _check(lib().ard_set_path(ctx, path), "ard_set_path")
+
+
+def ard_set_compact_reuse(ctx, enable):
+    _check(lib().ard_set_compact_reuse(ctx, 1 if enable else 0), "ard_set_compact_reuse")
 
 
 def ard_set_tile_n(ctx, bn):

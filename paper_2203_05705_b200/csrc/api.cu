@@ -169,6 +169,8 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->device = device;
   ctx->path = ARD_PATH_AUTO;
   ctx->force_bn = 0;
+  ctx->reuse_compact = 0;
+  ctx->last_gather = {nullptr, 0, 0, 0, nullptr, 0ull, nullptr};
   ctx->workspace_bytes = workspace_bytes;
   ctx->d_workspace = nullptr;
   ctx->d_status = nullptr;
@@ -211,6 +213,13 @@ ard_status ard_destroy(ard_ctx* ctx) {
 ard_status ard_set_path(ard_ctx* ctx, ard_path path) {
   if (!ctx || path < ARD_PATH_AUTO || path > ARD_PATH_TENSOR_CORE) return ARD_ERR_INVALID_ARG;
   ctx->path = path;
+  return ARD_OK;
+}
+
+ard_status ard_set_compact_reuse(ard_ctx* ctx, int enable) {
+  if (!ctx) return ARD_ERR_INVALID_ARG;
+  ctx->reuse_compact = enable ? 1 : 0;
+  ctx->last_gather.src = nullptr;
   return ARD_OK;
 }
 
@@ -294,6 +303,7 @@ ard_status ard_pattern_create(ard_ctx* ctx, ard_pattern** out, ard_kind kind, in
   if (units > (1ll << 30)) { delete p; return ARD_ERR_UNSUPPORTED; }
   p->units = (int)units;
   p->dp_bound = 1;
+  p->generation = 0;
   size_t words = HDR_WORDS + (size_t)p->units;
   if (kind == ARD_TILE) words += (size_t)(p->Tc + 1) + (size_t)(p->Tr + 1) + 2 * (size_t)p->units;
   int32_t* d = nullptr;
@@ -331,6 +341,7 @@ ard_status ard_sample_pattern(ard_ctx* ctx, ard_pattern* pat, int dist_id, uint6
   if (d.ndp == 0 || d.ndp > pat->units) return ARD_ERR_DISTRIBUTION;
   DeviceGuard guard(ctx->device);
   pat->dp_bound = d.ndp;
+  pat->generation++;
   return launch_sampler(ctx, pat, d.d_cdf, d.ndp, seed, iteration, stream_id, 0, 0, (cudaStream_t)cuda_stream);
 }
 
@@ -339,6 +350,7 @@ ard_status ard_pattern_set(ard_ctx* ctx, ard_pattern* pat, int dp, int b, void* 
   if (dp < 1 || b < 1 || b > dp || dp > pat->units) return ARD_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   pat->dp_bound = dp;
+  pat->generation++;
   return launch_sampler(ctx, pat, nullptr, 0, 0, 0, 0, dp, b, (cudaStream_t)cuda_stream);
 }
 
@@ -407,15 +419,15 @@ ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B,
   t.g = g;
   t.ts = pat->ts;
   t.bn = tc_pick_bn(ctx, pat->kind, OP_FWD, B, K, N, pat->ts);
-  // A = X, K-major boxes [128 rows][64 k];  B = kept neurons of W, K-major boxes [bn rows][64 k].
+  // A = X, K-major boxes [128 rows][64 k];  B = kept neurons of W, K-major boxes [64 rows][64 k].
   st = get_maps(ctx, X, B, K, ldx, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);
   if (st != ARD_OK) return st;
   t.mapA_indexed = 0;
   if (pat->kind == ARD_ROW) {
-    st = get_maps(ctx, W, N, K, ldw, N, MAP_STRIDED_ROWS, pat->dp_bound, t.bn, 64, &t.mapB);
+    st = get_maps(ctx, W, N, K, ldw, N, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64, &t.mapB);
     t.mapB_indexed = 1;
   } else {
-    st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, t.bn, 64, &t.mapB);
+    st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);
     t.mapB_indexed = 0;
   }
   if (st != ARD_OK) return st;
@@ -439,6 +451,13 @@ static ard_status compact_dy(ard_ctx* ctx, const ard_pattern* pat, int B, int N,
   *dense_ld = lddy;
   const int ldc = (N + 7) / 8 * 8;
   if ((size_t)B * ldc * 2 > ctx->workspace_bytes) return ARD_ERR_NOMEM;
+  *out_ptr = ctx->d_workspace;
+  *out_ld = ldc;
+  auto& lg = ctx->last_gather;
+  if (ctx->reuse_compact && lg.src == dY && lg.ld == lddy && lg.B == B && lg.N == N && lg.pat == pat &&
+      lg.gen == pat->generation && lg.stream == s)
+    return ARD_OK;  // the previous backward call on this stream already compacted this dY for this pattern
+  lg = {dY, lddy, B, N, pat, pat->generation, s};
   ard_status st = launch_gather_cols(ctx, pat->d_hdr, pat->d_idx, dY, lddy, ctx->d_workspace, ldc, B, 2, N, 1, s);
   *out_ptr = ctx->d_workspace;
   *out_ld = ldc;

@@ -30,6 +30,7 @@ struct ard_pattern {
   ard_kind kind;
   int K_dim, N_dim, ts, Tr, Tc, units;
   int dp_bound;        // largest dp the last sample/set call can have produced
+  unsigned long long generation;  // bumped by every sample / set call
   int32_t* d_hdr;      // device: header
   int32_t* d_idx;      // device: kept list (row: neuron index; tile: t-1), capacity `units`
   int32_t* d_col_ptr;  // tile only: [Tc+1]
@@ -68,6 +69,8 @@ struct ard_ctx {
   int sm_count;
   ard_path path;
   int force_bn;
+  int reuse_compact;  // opt-in: consecutive backward calls share one compacted dY
+  struct { const void* src; int ld, B, N; const ard_pattern* pat; unsigned long long gen; cudaStream_t stream; } last_gather;
   size_t workspace_bytes;
   void* d_workspace;
   int* d_status;

@@ -16,63 +16,70 @@ __global__ void __launch_bounds__(256) gather_cols_kernel(const int32_t* __restr
   for (int r = blockIdx.y; r < rows; r += gridDim.y) dst[(size_t)r * ld_dst + j] = src[(size_t)r * ld_src + col];
 }
 
-// Faster form for 2-byte elements with 16-byte aligned rows: a block stages the source span of up to
-// 1024 outputs in shared memory with coalesced 16-byte loads, then every thread assembles 8 kept
-// values into one 16-byte store.  With skip_dense != 0 a dense pattern (dp = 1) is left alone: the
-// GEMM then reads the original matrix directly.
-constexpr int GATHER_SPAN = 16384;  // staged source elements
+// Faster form for 2-byte elements with 16-byte aligned rows.  Each warp owns a private slice of
+// shared memory: it pulls the source span of up to 256 outputs with coalesced 16-byte loads (all of
+// a lane's loads are issued before any is consumed), then every lane assembles 8 kept values into one
+// 16-byte store.  No block-wide barrier, so the warps of a block overlap each other's latency.
+// With skip_dense != 0 a dense pattern (dp = 1) is left alone: the GEMM then reads the original matrix.
+constexpr int GATHER_WARPS = 4;
+constexpr int GATHER_SPAN = 4096;  // staged source elements per warp (8 KiB)
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(GATHER_WARPS * 32)
 gather_cols_staged_kernel(const int32_t* __restrict__ hdr, const uint16_t* __restrict__ src, int ld_src,
                           uint16_t* __restrict__ dst, int ld_dst, int rows, int n_cols, int skip_dense) {
-  __shared__ __align__(16) uint16_t buf[GATHER_SPAN + 16];
+  __shared__ __align__(16) uint16_t smem[GATHER_WARPS][GATHER_SPAN + 8];
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
   if (skip_dense && dp == 1) return;
-  int outs = (GATHER_SPAN / dp) & ~7;
-  if (outs > 1024) outs = 1024;
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const long long warp_id = (long long)blockIdx.x * GATHER_WARPS + wib;
+  const long long n_warps = (long long)gridDim.x * GATHER_WARPS;
+  int outs = ((GATHER_SPAN - 8) / dp) & ~7;  // outputs per warp pass (multiple of 8)
+  if (outs > 256) outs = 256;
   if (outs < 8) {
-    // period too long for the staging buffer: element-wise copy
-    for (long long e = (long long)blockIdx.x * 256 + threadIdx.x; e < (long long)rows * n_keep;
-         e += (long long)gridDim.x * 256) {
+    // period too long for the staging slice: element-wise copy
+    for (long long e = warp_id * 32 + lane; e < (long long)rows * n_keep; e += n_warps * 32) {
       const int r = (int)(e / n_keep), j = (int)(e % n_keep);
       dst[(size_t)r * ld_dst + j] = src[(size_t)r * ld_src + bb + (long long)j * dp];
     }
     return;
   }
+  uint16_t* buf = smem[wib];
   const int chunks = (n_keep + outs - 1) / outs;
-  for (long long item = blockIdx.x; item < (long long)rows * chunks; item += gridDim.x) {
-    const int r = (int)(item / chunks), ch = (int)(item % chunks);
+  for (long long item = warp_id; item < (long long)rows * chunks; item += n_warps) {
+    const int r = (int)(item / chunks), ch = (int)(item - (long long)r * chunks);
     const int j0 = ch * outs;
     const int nout = min(outs, n_keep - j0);
-    const int s0 = bb + j0 * dp;                 // first source column
-    const int a0 = s0 & ~7;                      // 16-byte aligned start
+    const int s0 = bb + j0 * dp;  // first source column
+    const int a0 = s0 & ~7;       // 16-byte aligned start
     const int count = bb + (j0 + nout - 1) * dp - a0 + 1;
     const uint16_t* srow = src + (size_t)r * ld_src;
-    for (int v = threadIdx.x; v * 8 < count; v += 256) {
+    for (int v = lane; v * 8 < count; v += 32) {
       const int col = a0 + 8 * v;
       if (col + 8 <= ld_src) {
-        *reinterpret_cast<uint4*>(buf + 8 * v) = *reinterpret_cast<const uint4*>(srow + col);
+        // asynchronous 16-byte copy: every piece of the span is in flight at once
+        const uint32_t saddr = (uint32_t)__cvta_generic_to_shared(buf + 8 * v);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(saddr), "l"(srow + col) : "memory");
       } else {
         for (int i = 0; i < 8; ++i) buf[8 * v + i] = (col + i < n_cols) ? srow[col + i] : (uint16_t)0;
       }
     }
-    __syncthreads();
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncwarp();
     const int off = s0 - a0;
     uint16_t* drow = dst + (size_t)r * ld_dst + j0;
-    for (int t = threadIdx.x; t * 8 < nout; t += 256) {
-      if (t * 8 + 8 <= nout) {
-        uint32_t w[4];
+    const int t = lane;
+    if (t * 8 + 8 <= nout) {
+      uint32_t w[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint32_t lo = buf[off + (t * 8 + 2 * i) * dp], hi = buf[off + (t * 8 + 2 * i + 1) * dp];
-          w[i] = lo | (hi << 16);
-        }
-        *reinterpret_cast<uint4*>(drow + t * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-      } else {
-        for (int i = t * 8; i < nout; ++i) drow[i] = buf[off + i * dp];
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t lo = buf[off + (t * 8 + 2 * i) * dp], hi = buf[off + (t * 8 + 2 * i + 1) * dp];
+        w[i] = lo | (hi << 16);
       }
+      *reinterpret_cast<uint4*>(drow + t * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+    } else {
+      for (int i = t * 8; i < nout && i < t * 8 + 8; ++i) drow[i] = buf[off + i * dp];
     }
-    __syncthreads();
+    __syncwarp();
   }
 }
 
@@ -161,7 +168,7 @@ ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* i
   const bool vec_ok = elem_bytes == 2 && ld_src % 8 == 0 && ld_dst % 8 == 0 &&
                       (reinterpret_cast<uintptr_t>(src) & 15) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0;
   if (vec_ok) {
-    gather_cols_staged_kernel<<<ctx->sm_count * 8, 256, 0, s>>>(hdr, (const uint16_t*)src, ld_src, (uint16_t*)dst,
+    gather_cols_staged_kernel<<<ctx->sm_count * 6, GATHER_WARPS * 32, 0, s>>>(hdr, (const uint16_t*)src, ld_src, (uint16_t*)dst,
                                                                  ld_dst, rows, max_cols, skip_dense);
   } else {
     dim3 grid((max_cols + 255) / 256, rows < 1024 ? rows : 1024);

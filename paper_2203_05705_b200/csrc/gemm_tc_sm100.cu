@@ -2,13 +2,18 @@
 //
 // One persistent, warp-specialised kernel template covers the six products (row / tile pattern x
 // forward / backward-data / backward-weight).  Per CTA: warp 0 is the TMA producer, warp 1 issues
-// tcgen05.mma and owns the TMEM allocation, warps 2..5 are the epilogue.  Only the kept rows /
+// tcgen05.mma and owns the TMEM allocation, warps 2..9 are the epilogue (two warps per TMEM lane
+// quadrant, each taking half of the tile's columns).  Only the kept rows /
 // tiles of the weight and the matching slices of the activations are ever staged into shared
 // memory (Sec. 3.1, 3.2): a row pattern's kept neurons b-1, b-1+dp, ... are one TMA box of a
 // descriptor whose row pitch is dp*ldw; a tile pattern's kept tiles come from the per-column /
 // per-row lists the sampler emitted.  The pattern is read from device memory, so the launch does
 // not depend on it: the grid is sized for the densest pattern and each CTA derives its own tile
 // schedule from the header.
+//
+// Row patterns pick the N extent of the output tile (64, 128 or 256) on the device from the sampled
+// n_keep, so that a sparse pattern still spreads over all SMs; the instruction descriptor, the
+// number of TMA boxes per stage and the tile schedule follow that choice.
 //
 // The accumulator is double-buffered in TMEM (2 x BN columns), so the epilogue of one output tile
 // overlaps the MMAs of the next.  Every wait on an mbarrier is bounded by a wall-clock limit;
@@ -20,7 +25,8 @@ namespace {
 
 constexpr int BM = 128;
 constexpr int BK = 64;  // 64 bf16 = 128 bytes = one swizzle row
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;  // warp 0 producer, warp 1 MMA, warps 2..9 epilogue
+constexpr int EPI_WARPS = 8;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum TcMode {
@@ -55,6 +61,7 @@ struct TcParams {
   int out_is_f32;
   int scatter;    // row fwd: full-width output with zero fill
   int zero_fill;  // row bwd-weight: write zeros to dropped rows
+  int force_bn;   // row modes: 0 = choose the N tile on the device, else 64 / 128 / 256
   int* status;
 };
 
@@ -180,8 +187,8 @@ struct SmemLayout {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STG_OFF = STAGES * STAGE_BYTES;       // epilogue staging: 4 warps x 32 x 33 floats
-  static constexpr int STG_BYTES = 4 * 32 * 33 * 4;
+  static constexpr int STG_OFF = STAGES * STAGE_BYTES;       // epilogue staging: 8 warps x 32 x 33 floats
+  static constexpr int STG_BYTES = EPI_WARPS * 32 * 33 * 4;
   static constexpr int BAR_OFF = STG_OFF + STG_BYTES;        // full[S], empty[S], tfull[2], tempty[2]
   static constexpr int MISC_OFF = BAR_OFF + (2 * STAGES + 4) * 8;
   static constexpr int TOTAL = MISC_OFF + 16 + 1024;         // + slack for manual 1024-byte alignment
@@ -203,6 +210,7 @@ struct Sched {
   int Mt, Nt, total;
   int M_gemm, N_gemm, Kc;  // GEMM extents (valid rows, valid cols, contraction length)
   int subm, subn;          // tile bwd-weight: sub-blocks per pattern tile
+  int bn;                  // N extent of the output tile actually used (<= BN)
 
   __device__ void init(const TcParams& p) {
     dp = p.hdr[HDR_DP];
@@ -216,6 +224,7 @@ struct Sched {
     else if (MODE == M_TILE_FWD) { M_gemm = p.B; N_gemm = p.N; Kc = 0; }
     else if (MODE == M_TILE_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 0; }
     else { M_gemm = p.N; N_gemm = p.K; Kc = p.B; }
+    bn = BN;
     if (MODE == M_TILE_BWD_WEIGHT) {
       subm = (p.ts + BM - 1) / BM;
       subn = p.ts / BN;
@@ -223,7 +232,23 @@ struct Sched {
       Nt = subn;
     } else {
       Mt = (M_gemm + BM - 1) / BM;
-      Nt = (N_gemm + BN - 1) / BN;
+      if (MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA || MODE == M_ROW_BWD_WEIGHT) {
+        if (p.force_bn) {
+          bn = p.force_bn;
+        } else {
+          // Fewest (waves x time per tile).  Narrow tiles re-read the A operand more often and use
+          // narrower instructions: a 128-wide tile is charged 0.7 and a 64-wide one 0.55 of the time of
+          // a 256-wide tile (measured on dense problems).  Ties go to the wider tile.
+          int best_cost = 0x7fffffff;
+          for (int cand = BN; cand >= 64; cand >>= 1) {
+            const int tiles = Mt * ((N_gemm + cand - 1) / cand);
+            const int waves = (tiles + (int)gridDim.x - 1) / (int)gridDim.x;
+            const int cost = waves * (cand == 256 ? 100 : (cand == 128 ? 70 : 55));
+            if (cost < best_cost) { best_cost = cost; bn = cand; }
+          }
+        }
+      }
+      Nt = (N_gemm + bn - 1) / bn;
     }
     total = Mt * Nt;
   }
@@ -247,7 +272,7 @@ struct Sched {
     }
     const int mt = t % Mt, nt = t / Mt;
     ti.m0 = mt * BM;
-    ti.n0 = nt * BN;
+    ti.n0 = nt * bn;
     if (MODE == M_TILE_FWD) {
       const int c = ti.n0 / p.ts;
       ti.klist = p.col_idx + p.col_ptr[c];
@@ -315,7 +340,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   using L = SmemLayout<BN>;
   constexpr int STAGES = L::STAGES;
   constexpr bool A_MN = a_is_mn(MODE), B_MN = b_is_mn(MODE);
-  constexpr uint32_t IDESC = make_idesc(BN, A_MN, B_MN);
   constexpr uint32_t TMEM_COLS = tmem_cols_for(BN);
 
   extern __shared__ uint8_t smem_raw[];
@@ -340,7 +364,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4);
+      mbar_init(tempty_bar(a), EPI_WARPS);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -356,6 +380,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
 
   Sched<BN, MODE> sch;
   sch.init(p);
+  const int bn = sch.bn;  // N extent of this launch's output tiles (runtime for row patterns)
 
   if (warp == 0) {
     // ===================== TMA producer =====================
@@ -365,6 +390,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       const CUtensorMap* mapB = p.mapB + (p.mapB_indexed ? e : 0);
       tensormap_acquire(mapA);
       tensormap_acquire(mapB);
+      const uint32_t stage_tx = (uint32_t)(L::A_BYTES + bn * BK * 2);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -374,7 +400,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sA = base + stage * L::STAGE_BYTES;
           const uint32_t sB = sA + L::A_BYTES;
-          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)L::STAGE_BYTES);
+          mbar_arrive_expect_tx(full_bar(stage), stage_tx);
           // contraction coordinate of this block
           int kx;
           if (MODE == M_TILE_FWD || MODE == M_TILE_BWD_DATA) kx = ti.klist[kb / ti.kper] * p.ts + (kb % ti.kper) * BK;
@@ -386,12 +412,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
             for (int i = 0; i < BM / 64; ++i)  // [64 k rows][64 m] per box
               tma_load_2d(sA + i * (64 * BK * 2), mapA, full_bar(stage), ti.m0 + 64 * i, kx);
           }
-          if (!B_MN) {
-            tma_load_2d(sB, mapB, full_bar(stage), kx, ti.n0);  // [BN rows][64 k]
-          } else {
-#pragma unroll
-            for (int i = 0; i < BN / 64; ++i)
-              tma_load_2d(sB + i * (64 * BK * 2), mapB, full_bar(stage), ti.n0 + 64 * i, kx);
+          // B always moves in 64-wide boxes: K-major [64 rows][64 k] stacked, MN-major [64 k][64 n].
+          for (int i = 0; i < bn / 64; ++i) {
+            if (!B_MN) tma_load_2d(sB + i * (64 * BK * 2), mapB, full_bar(stage), kx, ti.n0 + 64 * i);
+            else tma_load_2d(sB + i * (64 * BK * 2), mapB, full_bar(stage), ti.n0 + 64 * i, kx);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -400,6 +424,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
     if (lane == 0) {
+      const uint32_t idesc = make_idesc(bn, A_MN, B_MN);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -422,7 +447,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
             // MN-major: advance 16 k-rows = 2048 bytes.
             const uint64_t ad = A_MN ? make_desc(sA + s * 2048, 64 * BK * 2, 1024) : make_desc(sA + s * 32, 16, 1024);
             const uint64_t bd = B_MN ? make_desc(sB + s * 2048, 64 * BK * 2, 1024) : make_desc(sB + s * 32, 16, 1024);
-            tc_mma_bf16(d_tmem, ad, bd, IDESC, (kb | s) != 0 ? 1u : 0u);
+            tc_mma_bf16(d_tmem, ad, bd, idesc, (kb | s) != 0 ? 1u : 0u);
           }
           tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -433,10 +458,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       }
     }
   } else {
-    // ===================== epilogue (warps 2..5) =====================
+    // ===================== epilogue (warps 2..9) =====================
     const int q = warp & 3;                 // TMEM lane quadrant this warp may read
+    const int half = (warp - 2) >> 2;       // which half of the tile's columns
     const int row_in_tile = q * 32 + lane;  // accumulator row owned by this thread
     float* stg = reinterpret_cast<float*>(smem + L::STG_OFF) + (warp - 2) * (32 * 33);
+    const int nch = bn / 32;                // 32-column chunks in a tile
+    const int ch_lo = half * (nch / 2), ch_hi = (half == 0) ? nch / 2 : nch;
+    const int dp = sch.dp, bb = sch.b - 1;
+    const uint32_t magic_dp = (uint32_t)(0x100000000ull / (unsigned)dp) + 1u;  // exact x/dp for x < 2^16
     int it = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < sch.total && ok; t += gridDim.x, ++it) {
@@ -453,7 +483,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       long long out_row;
       if (MODE == M_ROW_BWD_WEIGHT) {
         row_ok = m < sch.M_gemm;
-        out_row = (long long)(sch.b - 1) + (long long)m * sch.dp;
+        out_row = (long long)bb + (long long)m * dp;
       } else if (MODE == M_TILE_BWD_WEIGHT) {
         row_ok = row_in_tile < ti.rows_valid && m < sch.M_gemm;
         out_row = m;
@@ -462,22 +492,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         out_row = m;
       }
 
-#pragma unroll 1
-      for (int ch = 0; ch < BN / 32; ++ch) {
+      // One 32-column chunk of this thread's accumulator row, already loaded into r[].
+      auto emit = [&](const uint32_t (&r)[32], int ch) {
         const int n = ti.n0 + ch * 32;
         float v[32];
-        if (ti.nkb > 0) {
-          uint32_t r[32];
-          tmem_ld32(t_row + (uint32_t)(ch * 32), r);
-          tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = p.alpha * __uint_as_float(r[i]);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = 0.f;
-        }
+        for (int i = 0; i < 32; ++i) v[i] = (ti.nkb > 0) ? p.alpha * __uint_as_float(r[i]) : 0.f;
 
-        if (MODE == M_ROW_FWD && p.scatter && sch.dp > 1) {
+        if (MODE == M_ROW_FWD && p.scatter && dp > 1) {
           // Full-width rows: compact column j -> column b-1 + j*dp, zeros everywhere else
           // (Sec. 3.1: dropped outputs are zero).  The 32x32 block is staged through shared memory
           // and the (row, 16-byte piece) pairs of the 32 x 32*dp output block are dealt to the lanes
@@ -486,43 +508,58 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
 #pragma unroll
             for (int i = 0; i < 32; ++i) stg[lane * 33 + i] = v[i];
             __syncwarp();
-            const int dp = sch.dp, bb = sch.b - 1;
             const int cs = n * dp;
             const bool last = n + 32 >= sch.n_keep;
             const int ce = last ? p.N : min((n + 32) * dp, p.N);
             const int groups = (ce - cs + 7) >> 3;  // 16-byte pieces per output row
+            const uint32_t magic_g = (uint32_t)(0x100000000ull / (unsigned)groups) + 1u;
             const int rows_here = min(32, sch.M_gemm - (ti.m0 + q * 32));
             const int items = rows_here * groups;
-            __nv_bfloat16* obase = reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)(ti.m0 + q * 32) * p.ldo;
+            __nv_bfloat16* obase = reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)(ti.m0 + q * 32) * p.ldo + cs;
             for (int w = lane; w < items; w += 32) {
-              const int rr = w / groups, g = w - rr * groups;
-              const int c0 = cs + 8 * g;
-              __nv_bfloat16* dst = obase + (size_t)rr * p.ldo + c0;
-              // (compact column, remainder) of c0 - (b-1); a column is kept when the remainder is 0 (Eq. 1).
-              const int rel = c0 - bb;  // negative only before the first kept column
+              const int rr = groups == 1 ? w : (int)__umulhi((uint32_t)w, magic_g);  // w / groups
+              const int g = w - rr * groups;
+              __nv_bfloat16* dst = obase + (size_t)rr * p.ldo + 8 * g;
+              // (compact column, remainder) of the piece's first column relative to column n*dp + b-1;
+              // a column is kept when the remainder is 0 (Eq. 1).
+              const int rel = 8 * g - bb;  // negative only before the first kept column
               int cq, cr;
-              if (rel >= 0) { cq = rel / dp; cr = rel - cq * dp; }
+              if (rel >= 0) { cq = (int)__umulhi((uint32_t)rel, magic_dp); cr = rel - cq * dp; }
               else { cq = -1; cr = rel + dp; }
               const int first_kept = cr == 0 ? 0 : dp - cr;  // position of the first kept column
-              const int nleft = ce - c0;
-              if (first_kept >= 8 && nleft >= 8) {
-                *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
-                continue;
-              }
-              float x[8];
-              const float* srow = stg + rr * 33 - n;
-#pragma unroll
-              for (int pos = 0; pos < 8; ++pos) {
-                x[pos] = (cr == 0) ? srow[cq] : 0.f;
-                if (++cr == dp) { cr = 0; ++cq; }
-              }
+              const int nleft = ce - cs - 8 * g;
+              const float* srow = stg + rr * 33;
               if (nleft >= 8) {
-                *reinterpret_cast<uint4*>(dst) = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]),
-                                                            pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+                uint4 o = make_uint4(0u, 0u, 0u, 0u);
+                if (dp >= 8) {
+                  // at most one kept column per piece
+                  if (first_kept < 8) {
+                    const uint32_t hbits = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(srow[cq + (cr != 0)]));
+                    const uint32_t u = hbits << ((first_kept & 1) * 16);
+                    const int wd = first_kept >> 1;
+                    o.x = wd == 0 ? u : 0u;
+                    o.y = wd == 1 ? u : 0u;
+                    o.z = wd == 2 ? u : 0u;
+                    o.w = wd == 3 ? u : 0u;
+                  }
+                } else if (first_kept < 8) {
+                  float x[8];
+#pragma unroll
+                  for (int pos = 0; pos < 8; ++pos) {
+                    x[pos] = (cr == 0) ? srow[cq] : 0.f;
+                    if (++cr == dp) { cr = 0; ++cq; }
+                  }
+                  o = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]),
+                                 pack_bf16(x[6], x[7]));
+                }
+                *reinterpret_cast<uint4*>(dst) = o;
               } else {
 #pragma unroll
-                for (int pos = 0; pos < 8; ++pos)
-                  if (pos < nleft) dst[pos] = __float2bfloat16_rn(x[pos]);
+                for (int pos = 0; pos < 8; ++pos) {
+                  const float xv = (cr == 0) ? srow[cq] : 0.f;
+                  if (pos < nleft) dst[pos] = __float2bfloat16_rn(xv);
+                  if (++cr == dp) { cr = 0; ++cq; }
+                }
               }
             }
             __syncwarp();
@@ -532,16 +569,34 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
           if (row_ok && nvalid > 0) {
             store_row32(p.out, (size_t)out_row * p.ldo, n, v, nvalid, p.out_is_f32);
             if (MODE == M_ROW_BWD_WEIGHT && p.zero_fill) {
-              // Dropped neurons between this kept row and the next (and before the first / after
-              // the last kept row) receive zeros.
               // Compact row m owns output rows [m*dp, (m+1)*dp); the last one also owns the tail.
-              const long long first = (long long)m * sch.dp;
+              const long long first = (long long)m * dp;
               const long long lastrow =
-                  (m == sch.M_gemm - 1) ? (long long)p.N - 1 : min((long long)(m + 1) * sch.dp - 1, (long long)p.N - 1);
+                  (m == sch.M_gemm - 1) ? (long long)p.N - 1 : min((long long)(m + 1) * dp - 1, (long long)p.N - 1);
               for (long long rz = first; rz <= lastrow; ++rz)
                 if (rz != out_row) zero_row32(p.out, (size_t)rz * p.ldo, n, nvalid, p.out_is_f32);
             }
           }
+        }
+      };
+
+      // Software pipeline over this warp's chunks: the TMEM load of chunk i+1 is in flight while
+      // chunk i is converted and stored.
+      uint32_t ra[32], rb[32];
+      if (ti.nkb > 0 && ch_lo < ch_hi) tmem_ld32(t_row + (uint32_t)(ch_lo * 32), ra);
+#pragma unroll 1
+      for (int ch = ch_lo; ch < ch_hi; ch += 2) {
+        if (ti.nkb > 0) {
+          tmem_ld_wait();
+          if (ch + 1 < ch_hi) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), rb);
+        }
+        emit(ra, ch);
+        if (ch + 1 < ch_hi) {
+          if (ti.nkb > 0) {
+            tmem_ld_wait();
+            if (ch + 2 < ch_hi) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), ra);
+          }
+          emit(rb, ch + 1);
         }
       }
       tc_fence_before();
@@ -569,7 +624,7 @@ ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStrea
     ARD_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
     attr_done[ctx->device & 63] = true;
   }
-  int grid = max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count;
+  int grid = max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count;  // max_tiles: tile count of the densest pattern
   if (grid < 1) grid = 1;
   kern<<<grid, TC_THREADS, L::TOTAL, s>>>(p);
   ctx->launches++;
@@ -581,25 +636,17 @@ inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 
 }  // namespace
 
-// Chooses the N tile: the widest instruction (256) when the densest pattern still fills the SMs,
-// narrower tiles otherwise so that more CTAs have work.
+// N extent of the output tile.  Tile patterns: fixed per launch (it must divide the pattern tile).
+// Row patterns: 0 = chosen on the device from the sampled n_keep, or the value forced by ard_set_tile_n.
 int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int B, int K, int N, int ts) {
+  (void)B; (void)K; (void)N;
   const int f = ctx->force_bn;
   if (kind == ARD_TILE) {
-    // the N tile must divide the pattern tile
     if (f && ts % f == 0 && (op == OP_BWD_WEIGHT || f <= 128)) return f;
     if (op == OP_BWD_WEIGHT) return ts % 256 == 0 ? 256 : (ts % 128 == 0 ? 128 : 64);
     return ts % 128 == 0 ? 128 : 64;
   }
-  if (f) return f;
-  int Mg, Ng;
-  if (op == OP_FWD) { Mg = B; Ng = N; }
-  else if (op == OP_BWD_DATA) { Mg = B; Ng = K; }
-  else { Mg = N; Ng = K; }
-  const int mt = (Mg + BM - 1) / BM;
-  if (Ng >= 256 && mt * ((Ng + 255) / 256) >= ctx->sm_count) return 256;
-  if (Ng >= 128 && mt * ((Ng + 127) / 128) >= ctx->sm_count / 2) return 128;
-  return Ng >= 128 ? 128 : 64;
+  return f;
 }
 
 ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s) {
@@ -625,7 +672,8 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
   p.scatter = (kind == ARD_ROW && op == OP_FWD && a.g.flag0 == ARD_OUT_SCATTER_ZEROFILL) ? 1 : 0;
   p.zero_fill = (op == OP_BWD_WEIGHT) ? a.g.flag1 : 0;
   p.status = a.g.status;
-  const int bn = a.bn;
+  p.force_bn = (kind == ARD_ROW) ? a.bn : 0;
+  const int bn = (kind == ARD_ROW) ? 256 : a.bn;
 
 #define ARD_TC_CASE(BN_, MODE_, TILES_) \
   if (bn == BN_) return launch_mode<BN_, MODE_>(ctx, p, (TILES_), s);
@@ -633,19 +681,13 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
   if (kind == ARD_ROW) {
     if (op == OP_FWD) {
       const int mt = cdiv(p.B, BM);
-      ARD_TC_CASE(256, M_ROW_FWD, mt * cdiv(p.N, 256))
-      ARD_TC_CASE(128, M_ROW_FWD, mt * cdiv(p.N, 128))
-      ARD_TC_CASE(64, M_ROW_FWD, mt * cdiv(p.N, 64))
+      ARD_TC_CASE(256, M_ROW_FWD, mt * cdiv(p.N, 64))
     } else if (op == OP_BWD_DATA) {
       const int mt = cdiv(p.B, BM);
-      ARD_TC_CASE(256, M_ROW_BWD_DATA, mt * cdiv(p.K, 256))
-      ARD_TC_CASE(128, M_ROW_BWD_DATA, mt * cdiv(p.K, 128))
-      ARD_TC_CASE(64, M_ROW_BWD_DATA, mt * cdiv(p.K, 64))
+      ARD_TC_CASE(256, M_ROW_BWD_DATA, mt * cdiv(p.K, 64))
     } else {
       const int mt = cdiv(p.N, BM);
-      ARD_TC_CASE(256, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 256))
-      ARD_TC_CASE(128, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 128))
-      ARD_TC_CASE(64, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 64))
+      ARD_TC_CASE(256, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 64))
     }
   } else {
     if (op == OP_FWD) {

@@ -140,3 +140,23 @@ def test_small_workspace_is_reported(ctx):
         assert_ok(res, TOL[ard.ARD_BF16])
     finally:
         c2.close()
+
+
+def test_compact_reuse_option(ctx):
+    """With reuse enabled bwd-weight consumes the copy bwd-data compacted; results stay within tolerance
+    across pattern changes (every new sample invalidates the copy)."""
+    B, K, N = 256, 256, 1024
+    ard.ard_set_path(ctx.h, ard.ARD_PATH_TENSOR_CORE)
+    ard.ard_set_compact_reuse(ctx.h, 1)
+    pat = ctx.pattern(ard.ARD_ROW, K, N)
+    try:
+        for i, (dp, b) in enumerate([(2, 1), (2, 2), (1, 1), (7, 3), (7, 3)]):
+            X, W, dY = _layer(B, K, N, 100 + i, 0.05)
+            ard.ard_pattern_set(ctx.h, pat, dp, b)
+            n0 = ard.ard_launch_count(ctx.h)
+            res = run_three_gemms(ctx, pat, ard.ARD_ROW, ard.ARD_BF16, X, W, dY, dp, b, 2.0)
+            assert_ok(res, TOL[ard.ARD_BF16], (dp, b))
+            assert ard.ard_launch_count(ctx.h) - n0 == 4          # fwd, gather, bwd-data, bwd-weight
+    finally:
+        ard.ard_set_compact_reuse(ctx.h, 0)
+        ard.ard_set_path(ctx.h, ard.ARD_PATH_AUTO)
