@@ -56,6 +56,10 @@ typedef enum {
 typedef enum { ARD_F32 = 0, ARD_BF16 = 1 } ard_dtype;
 typedef enum { ARD_ROW = 0, ARD_TILE = 1 } ard_kind;
 typedef enum { ARD_OUT_COMPACT = 0, ARD_OUT_SCATTER_ZEROFILL = 1 } ard_outmode;
+/* Flags that may be OR-ed into the `outmode` argument of ard_fwd and into the `dy_is_compact`
+ * argument of ard_bwd_data (whose bit 0 keeps its meaning): */
+#define ARD_FLAG_OUT_F32 0x10    /* bf16 operands: write the result as fp32 (leading dimension in fp32 elements) */
+#define ARD_FLAG_ACCUMULATE 0x20 /* add the product to the existing output; not with ARD_OUT_SCATTER_ZEROFILL   */
 
 /* Selects the kernel family for ARD_BF16 calls.  AUTO picks the tcgen05 path when the shape and
  * alignment allow it and the CUDA-core path otherwise; the other two force one family (FORCE_TC

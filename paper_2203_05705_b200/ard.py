@@ -22,6 +22,7 @@ ARD_ERR_UNSUPPORTED, ARD_ERR_CUDA, ARD_ERR_TIMEOUT, ARD_ERR_NOMEM = 5, 6, 7, 8
 ARD_F32, ARD_BF16 = 0, 1
 ARD_ROW, ARD_TILE = 0, 1
 ARD_OUT_COMPACT, ARD_OUT_SCATTER_ZEROFILL = 0, 1
+ARD_FLAG_OUT_F32, ARD_FLAG_ACCUMULATE = 0x10, 0x20
 ARD_PATH_AUTO, ARD_PATH_CUDA_CORE, ARD_PATH_TENSOR_CORE = 0, 1, 2
 ARD_STATIC_SCRATCH_BYTES = 8 << 20
 

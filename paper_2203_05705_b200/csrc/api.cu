@@ -120,6 +120,7 @@ void fill_common(GemmArgs& g, ard_ctx* ctx, const ard_pattern* pat, int B, int K
   g.alpha = alpha;
   g.flag0 = g.flag1 = 0;
   g.out_is_f32 = 0;
+  g.accumulate = 0;
   g.status = ctx->d_status;
 }
 
@@ -396,21 +397,29 @@ ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B,
   if (st != ARD_OK) return st;
   if (!X || !W || !Y) return ARD_ERR_INVALID_ARG;
   if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
-  if (outmode != ARD_OUT_COMPACT && outmode != ARD_OUT_SCATTER_ZEROFILL) return ARD_ERR_INVALID_ARG;
+  const int mode = (int)outmode & 0xF;
+  const bool out_f32 = dtype == ARD_F32 || ((int)outmode & ARD_FLAG_OUT_F32);
+  const bool accumulate = ((int)outmode & ARD_FLAG_ACCUMULATE) != 0;
+  if (((int)outmode & ~(0xF | ARD_FLAG_OUT_F32 | ARD_FLAG_ACCUMULATE)) != 0) return ARD_ERR_INVALID_ARG;
+  if (mode != ARD_OUT_COMPACT && mode != ARD_OUT_SCATTER_ZEROFILL) return ARD_ERR_INVALID_ARG;
+  if (accumulate && mode == ARD_OUT_SCATTER_ZEROFILL && pat->kind == ARD_ROW) return ARD_ERR_INVALID_ARG;
   if (ldx < K || ldw < K || ldy < N) return ARD_ERR_SHAPE;
   if (B == 0) return ARD_OK;
   DeviceGuard guard(ctx->device);
   cudaStream_t s = (cudaStream_t)cuda_stream;
-  const int es = dtype == ARD_F32 ? 4 : 2;
+  const int es = out_f32 ? 4 : 2;
 
   GemmArgs g;
   fill_common(g, ctx, pat, B, K, N, alpha);
   g.A0 = X; g.lda0 = ldx; g.A1 = W; g.lda1 = ldw; g.out = Y; g.ldo = ldy;
-  g.flag0 = pat->kind == ARD_ROW ? (int)outmode : 0;
-  g.out_is_f32 = dtype == ARD_F32;
+  g.flag0 = pat->kind == ARD_ROW ? mode : 0;
+  g.out_is_f32 = out_f32;
+  g.accumulate = accumulate;
 
   ard_status el = ctx->path == ARD_PATH_CUDA_CORE ? ARD_ERR_UNSUPPORTED
                                                   : tc_eligible(ctx, pat, dtype, B, K, N, X, ldx, W, ldw, Y, ldy, es);
+  // the tensor-core scatter epilogue writes bf16 only
+  if (el == ARD_OK && out_f32 && pat->kind == ARD_ROW && mode == ARD_OUT_SCATTER_ZEROFILL) el = ARD_ERR_UNSUPPORTED;
   if (el != ARD_OK) {
     if (ctx->path == ARD_PATH_TENSOR_CORE) return el;
     return launch_gemm_cc(ctx, pat->kind, OP_FWD, dtype, g, pat->ts, s);
@@ -471,18 +480,23 @@ ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, i
   if (st != ARD_OK) return st;
   if (!dY || !W || !dX) return ARD_ERR_INVALID_ARG;
   if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  const int flags = dy_is_compact;
+  if ((flags & ~(1 | ARD_FLAG_OUT_F32 | ARD_FLAG_ACCUMULATE)) != 0) return ARD_ERR_INVALID_ARG;
+  dy_is_compact = flags & 1;
+  const bool out_f32 = dtype == ARD_F32 || (flags & ARD_FLAG_OUT_F32);
   if (dy_is_compact && pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
-  if (lddy < N || ldw < K || lddx < K) return ARD_ERR_SHAPE;
+  if (lddy < (dy_is_compact ? 1 : N) || ldw < K || lddx < K) return ARD_ERR_SHAPE;
   if (B == 0) return ARD_OK;
   DeviceGuard guard(ctx->device);
   cudaStream_t s = (cudaStream_t)cuda_stream;
-  const int es = dtype == ARD_F32 ? 4 : 2;
+  const int es = out_f32 ? 4 : 2;
 
   GemmArgs g;
   fill_common(g, ctx, pat, B, K, N, alpha);
   g.A0 = dY; g.lda0 = lddy; g.A1 = W; g.lda1 = ldw; g.out = dX; g.ldo = lddx;
   g.flag0 = dy_is_compact ? 1 : 0;
-  g.out_is_f32 = dtype == ARD_F32;
+  g.out_is_f32 = out_f32;
+  g.accumulate = (flags & ARD_FLAG_ACCUMULATE) != 0;
 
   ard_status el = ctx->path == ARD_PATH_CUDA_CORE
                       ? ARD_ERR_UNSUPPORTED

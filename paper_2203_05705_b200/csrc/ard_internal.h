@@ -105,6 +105,7 @@ struct GemmArgs {
   int flag0;       // fwd: outmode; bwd: dy_is_compact
   int flag1;       // bwd_weight: zero_fill_dropped
   int out_is_f32;
+  int accumulate;  // add to the existing output instead of overwriting it
   int* status;
 };
 

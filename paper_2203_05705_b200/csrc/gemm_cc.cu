@@ -15,9 +15,14 @@ template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-__device__ __forceinline__ void store_out(void* out, size_t off, float v, int out_is_f32) {
-  if (out_is_f32) reinterpret_cast<float*>(out)[off] = v;
-  else reinterpret_cast<__nv_bfloat16*>(out)[off] = __float2bfloat16_rn(v);
+__device__ __forceinline__ void store_out(void* out, size_t off, float v, int out_is_f32, int accumulate = 0) {
+  if (out_is_f32) {
+    float* p = reinterpret_cast<float*>(out) + off;
+    *p = accumulate ? *p + v : v;
+  } else {
+    __nv_bfloat16* p = reinterpret_cast<__nv_bfloat16*>(out) + off;
+    *p = __float2bfloat16_rn(accumulate ? __bfloat162float(*p) + v : v);
+  }
 }
 
 // KIND: 0 row, 1 tile.  OP: GemmOp.
@@ -142,7 +147,7 @@ __global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts)
       if (KIND == 0 && OP == OP_FWD) off = (size_t)m * g.ldo + (g.flag0 == ARD_OUT_SCATTER_ZEROFILL ? g.idx[n] : n);
       else if (KIND == 0 && OP == OP_BWD_WEIGHT) off = (size_t)g.idx[m] * g.ldo + n;
       else off = (size_t)m * g.ldo + n;
-      store_out(g.out, off, g.alpha * acc[i][j], g.out_is_f32);
+      store_out(g.out, off, g.alpha * acc[i][j], g.out_is_f32, g.accumulate);
     }
 }
 

@@ -62,6 +62,7 @@ struct TcParams {
   int scatter;    // row fwd: full-width output with zero fill
   int zero_fill;  // row bwd-weight: write zeros to dropped rows
   int force_bn;   // row modes: 0 = choose the N tile on the device, else 64 / 128 / 256
+  int accumulate; // plain stores add to the existing output
   int* status;
 };
 
@@ -298,8 +299,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // Stores 32 consecutive values of one output row; `nvalid` of them exist.  The row start is 16-byte
 // aligned whenever nvalid == 32 paths are taken (guaranteed by the host-side alignment checks).
-__device__ __forceinline__ void store_row32(void* out, size_t row_off, int col, const float (&v)[32], int nvalid,
-                                            int out_is_f32) {
+__device__ __forceinline__ void store_row32(void* out, size_t row_off, int col, float (&v)[32], int nvalid,
+                                            int out_is_f32, int accumulate = 0) {
+  if (accumulate) {
+    // read-modify-write of this thread's own 32 outputs
+    if (out_is_f32) {
+      const float* p = reinterpret_cast<const float*>(out) + row_off + col;
+#pragma unroll
+      for (int q = 0; q < 32; ++q)
+        if (q < nvalid) v[q] += p[q];
+    } else {
+      const __nv_bfloat16* p = reinterpret_cast<const __nv_bfloat16*>(out) + row_off + col;
+#pragma unroll
+      for (int q = 0; q < 32; ++q)
+        if (q < nvalid) v[q] += __bfloat162float(p[q]);
+    }
+  }
   if (out_is_f32) {
     float* p = reinterpret_cast<float*>(out) + row_off + col;
     if (nvalid >= 32) {
@@ -567,7 +582,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         } else {
           const int nvalid = min(32, sch.N_gemm - n);
           if (row_ok && nvalid > 0) {
-            store_row32(p.out, (size_t)out_row * p.ldo, n, v, nvalid, p.out_is_f32);
+            store_row32(p.out, (size_t)out_row * p.ldo, n, v, nvalid, p.out_is_f32, p.accumulate);
             if (MODE == M_ROW_BWD_WEIGHT && p.zero_fill) {
               // Compact row m owns output rows [m*dp, (m+1)*dp); the last one also owns the tail.
               const long long first = (long long)m * dp;
@@ -673,6 +688,7 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
   p.zero_fill = (op == OP_BWD_WEIGHT) ? a.g.flag1 : 0;
   p.status = a.g.status;
   p.force_bn = (kind == ARD_ROW) ? a.bn : 0;
+  p.accumulate = a.g.accumulate;
   const int bn = (kind == ARD_ROW) ? 256 : a.bn;
 
 #define ARD_TC_CASE(BN_, MODE_, TILES_) \

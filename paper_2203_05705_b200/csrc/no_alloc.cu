@@ -95,6 +95,7 @@ extern "C" ard_status ard_bwd_data_static_scratch(ard_ctx* ctx, const ard_patter
       g.flag0 = 1;                    // columns are already compact
       g.flag1 = 0;
       g.out_is_f32 = dtype == ARD_F32;
+      g.accumulate = 0;
       g.status = ctx->d_status;
       st = launch_gemm_cc(ctx, ARD_ROW, OP_BWD_DATA, dtype, g, 0, s);
     }
