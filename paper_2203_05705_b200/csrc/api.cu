@@ -1,6 +1,7 @@
 // C-ABI entry points: argument validation, context / pattern lifetime, the TMA descriptor cache and
 // the dispatch between the CUDA-core and tcgen05 kernel families.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -170,6 +171,10 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->device = device;
   ctx->path = ARD_PATH_AUTO;
   ctx->force_bn = 0;
+  ctx->band_m = 16;
+  ctx->use_pairs = 1;
+  if (const char* e = getenv("ARD_USE_PAIRS")) ctx->use_pairs = atoi(e);
+  if (const char* e = getenv("ARD_BAND_M")) ctx->band_m = atoi(e);
   ctx->reuse_compact = 0;
   ctx->last_gather = {nullptr, 0, 0, 0, nullptr, 0ull, nullptr};
   ctx->workspace_bytes = workspace_bytes;

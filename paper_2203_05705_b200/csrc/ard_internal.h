@@ -69,6 +69,8 @@ struct ard_ctx {
   int sm_count;
   ard_path path;
   int force_bn;
+  int use_pairs;      // tensor-core row kernels: CTA pairs (cta_group::2) when the output has >= 2 row tiles
+  int band_m;         // raster band height of the tensor-core kernels, in 128-row tiles
   int reuse_compact;  // opt-in: consecutive backward calls share one compacted dY
   struct { const void* src; int ld, B, N; const ard_pattern* pat; unsigned long long gen; cudaStream_t stream; } last_gather;
   size_t workspace_bytes;

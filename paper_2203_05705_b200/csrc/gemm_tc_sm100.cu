@@ -63,6 +63,7 @@ struct TcParams {
   int zero_fill;  // row bwd-weight: write zeros to dropped rows
   int force_bn;   // row modes: 0 = choose the N tile on the device, else 64 / 128 / 256
   int accumulate; // plain stores add to the existing output
+  int band_m;     // M-tiles per raster band (0: one band)
   int* status;
 };
 
@@ -159,6 +160,61 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- CTA-pair (cluster of 2, cta_group::2) forms ---------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load issued inside a CTA pair: the data lands in this CTA, the byte count is reported to the
+// mbarrier at `bar_cluster`, which may live in the peer CTA.  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int x,
+                                                 int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// Arrives on the mbarrier at the same shared-memory offset in every CTA of `mask` once the MMAs issued
+// so far by this thread have completed.
+__device__ __forceinline__ void tc_commit2(uint32_t bar, uint16_t mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, Blackwell version field = 1.
 //   K-major operand : rows of 128 bytes, 8-row groups 1024 bytes apart (SBO); LBO unused (1).
 //   MN-major operand: 64-element chunks along M/N `lbo` bytes apart; 8-row K groups 1024 bytes apart.
@@ -172,21 +228,23 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
   return d;
 }
 
-__host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn, bool b_mn) {
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn, bool b_mn, int m = BM) {
   return (1u << 4)                      // D format fp32
          | (1u << 7)                    // A format bf16
          | (1u << 10)                   // B format bf16
          | ((a_mn ? 1u : 0u) << 15)     // A major
          | ((b_mn ? 1u : 0u) << 16)     // B major
          | ((uint32_t)(n >> 3) << 17)   // N
-         | ((uint32_t)(BM >> 4) << 24); // M
+         | ((uint32_t)(m >> 4) << 24);  // M (256 for a CTA pair)
 }
 
-template <int BN>
+// CTAS = 2: a cluster of two CTAs shares one 256 x BN output tile; each CTA stages its own 128 rows
+// of A and half of the B rows, so a stage is smaller and the pipeline deeper.
+template <int BN, int CTAS = 1>
 struct SmemLayout {
-  static constexpr int STAGES = stages_for(BN);
+  static constexpr int STAGES = stages_for(BN / CTAS);
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int B_BYTES = (BN / CTAS) * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STG_OFF = STAGES * STAGE_BYTES;       // epilogue staging: 8 warps x 32 x 33 floats
   static constexpr int STG_BYTES = EPI_WARPS * 32 * 33 * 4;
@@ -205,15 +263,19 @@ struct TileInfo {
   int rows_valid;  // tile bwd-weight: rows of this tile that belong to the kept tile
 };
 
-template <int BN, int MODE>
+template <int BN, int MODE, int CTAS = 1>
 struct Sched {
   int dp, b, n_keep, Tc;
   int Mt, Nt, total;
   int M_gemm, N_gemm, Kc;  // GEMM extents (valid rows, valid cols, contraction length)
   int subm, subn;          // tile bwd-weight: sub-blocks per pattern tile
   int bn;                  // N extent of the output tile actually used (<= BN)
+  int rank;                // CTA rank inside the pair (0 for single-CTA tiles)
+  int workers;             // CTAs (or CTA pairs) sharing the tile loop
 
-  __device__ void init(const TcParams& p) {
+  __device__ void init(const TcParams& p, int rank_) {
+    rank = rank_;
+    workers = (int)gridDim.x / CTAS;
     dp = p.hdr[HDR_DP];
     b = p.hdr[HDR_B];
     n_keep = p.hdr[HDR_NKEEP];
@@ -232,7 +294,7 @@ struct Sched {
       Mt = n_keep * subm;
       Nt = subn;
     } else {
-      Mt = (M_gemm + BM - 1) / BM;
+      Mt = (M_gemm + BM * CTAS - 1) / (BM * CTAS);
       if (MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA || MODE == M_ROW_BWD_WEIGHT) {
         if (p.force_bn) {
           bn = p.force_bn;
@@ -241,9 +303,9 @@ struct Sched {
           // narrower instructions: a 128-wide tile is charged 0.7 and a 64-wide one 0.55 of the time of
           // a 256-wide tile (measured on dense problems).  Ties go to the wider tile.
           int best_cost = 0x7fffffff;
-          for (int cand = BN; cand >= 64; cand >>= 1) {
+          for (int cand = BN; cand >= 64 * CTAS; cand >>= 1) {
             const int tiles = Mt * ((N_gemm + cand - 1) / cand);
-            const int waves = (tiles + (int)gridDim.x - 1) / (int)gridDim.x;
+            const int waves = (tiles + workers - 1) / workers;
             const int cost = waves * (cand == 256 ? 100 : (cand == 128 ? 70 : 55));
             if (cost < best_cost) { best_cost = cost; bn = cand; }
           }
@@ -271,8 +333,18 @@ struct Sched {
       ti.rows_valid = min(BM, p.ts - sm * BM);
       return ti;
     }
-    const int mt = t % Mt, nt = t / Mt;
-    ti.m0 = mt * BM;
+    // Raster order: bands of band_m M-tiles; inside a band the M index runs fastest, so the CTAs that
+    // run together share a few B tiles and one band of A, and consecutive waves reuse that band from L2.
+    int mt, nt;
+    {
+      const int bm = (p.band_m > 0 && p.band_m < Mt) ? p.band_m : Mt;
+      const int per_band = bm * Nt;
+      const int band = t / per_band, r = t - band * per_band;
+      const int rows_in_band = min(bm, Mt - band * bm);
+      nt = r / rows_in_band;
+      mt = band * bm + (r - nt * rows_in_band);
+    }
+    ti.m0 = mt * BM * CTAS + rank * BM;  // this CTA's 128 rows of the tile
     ti.n0 = nt * bn;
     if (MODE == M_TILE_FWD) {
       const int c = ti.n0 / p.ts;
@@ -350,9 +422,10 @@ __device__ __forceinline__ void zero_row32(void* out, size_t row_off, int col, i
 }
 
 // ---- the kernel -----------------------------------------------------------------------------------
-template <int BN, int MODE>
+template <int BN, int MODE, int CTAS>
 __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcParams p) {
-  using L = SmemLayout<BN>;
+  using L = SmemLayout<BN, CTAS>;
+  const uint32_t rank = (CTAS == 2) ? cluster_ctarank() : 0u;  // rank 0 leads the pair and issues its MMAs
   constexpr int STAGES = L::STAGES;
   constexpr bool A_MN = a_is_mn(MODE), B_MN = b_is_mn(MODE);
   constexpr uint32_t TMEM_COLS = tmem_cols_for(BN);
@@ -379,22 +452,29 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), EPI_WARPS);
+      mbar_init(tempty_bar(a), EPI_WARPS * CTAS);  // the pair's epilogue warps all report to the leader
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), TMEM_COLS);
-    tmem_relinquish();
+    if (CTAS == 2) {
+      tmem_alloc2(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), TMEM_COLS);
+      tmem_relinquish2();
+    } else {
+      tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), TMEM_COLS);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync_all();  // both CTAs' barriers exist before anyone signals across the pair
+  else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_smem;
 
-  Sched<BN, MODE> sch;
-  sch.init(p);
+  Sched<BN, MODE, CTAS> sch;
+  sch.init(p, (int)rank);
+  const int w0 = (int)blockIdx.x / CTAS;  // first tile of this CTA (pair)
   const int bn = sch.bn;  // N extent of this launch's output tiles (runtime for row patterns)
 
   if (warp == 0) {
@@ -405,32 +485,41 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       const CUtensorMap* mapB = p.mapB + (p.mapB_indexed ? e : 0);
       tensormap_acquire(mapA);
       tensormap_acquire(mapB);
-      const uint32_t stage_tx = (uint32_t)(L::A_BYTES + bn * BK * 2);
+      const int bn_cta = bn / CTAS;  // B rows staged by this CTA
+      const uint32_t stage_tx = (uint32_t)(L::A_BYTES + bn_cta * BK * 2) * CTAS;  // bytes of the whole pair
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < sch.total && ok; t += gridDim.x) {
+      for (int t = w0; t < sch.total && ok; t += sch.workers) {
         const TileInfo ti = sch.tile(p, t);
         for (int kb = 0; kb < ti.nkb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sA = base + stage * L::STAGE_BYTES;
           const uint32_t sB = sA + L::A_BYTES;
-          mbar_arrive_expect_tx(full_bar(stage), stage_tx);
+          // In a pair every load reports to the leader's barrier, which expects the bytes of both CTAs.
+          const uint32_t fbar = (CTAS == 2) ? mapa_u32(full_bar(stage), 0u) : full_bar(stage);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), stage_tx);
+          auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+            if (CTAS == 2) tma_load_2d_pair(dst, map, fbar, x, y);
+            else tma_load_2d(dst, map, fbar, x, y);
+          };
           // contraction coordinate of this block
           int kx;
           if (MODE == M_TILE_FWD || MODE == M_TILE_BWD_DATA) kx = ti.klist[kb / ti.kper] * p.ts + (kb % ti.kper) * BK;
           else kx = kb * BK;
           if (!A_MN) {
-            tma_load_2d(sA, mapA, full_bar(stage), kx, ti.m0);  // [BM rows][64 k]
+            load(sA, mapA, kx, ti.m0);  // [BM rows][64 k]
           } else {
 #pragma unroll
             for (int i = 0; i < BM / 64; ++i)  // [64 k rows][64 m] per box
-              tma_load_2d(sA + i * (64 * BK * 2), mapA, full_bar(stage), ti.m0 + 64 * i, kx);
+              load(sA + i * (64 * BK * 2), mapA, ti.m0 + 64 * i, kx);
           }
           // B always moves in 64-wide boxes: K-major [64 rows][64 k] stacked, MN-major [64 k][64 n].
-          for (int i = 0; i < bn / 64; ++i) {
-            if (!B_MN) tma_load_2d(sB + i * (64 * BK * 2), mapB, full_bar(stage), kx, ti.n0 + 64 * i);
-            else tma_load_2d(sB + i * (64 * BK * 2), mapB, full_bar(stage), ti.n0 + 64 * i, kx);
+          // In a pair this CTA stages the B rows [rank*bn/2, (rank+1)*bn/2) of the tile.
+          const int nb0 = ti.n0 + (int)rank * bn_cta;
+          for (int i = 0; i < bn_cta / 64; ++i) {
+            if (!B_MN) load(sB + i * (64 * BK * 2), mapB, kx, nb0 + 64 * i);
+            else load(sB + i * (64 * BK * 2), mapB, nb0 + 64 * i, kx);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -438,13 +527,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc(bn, A_MN, B_MN);
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = make_idesc(bn, A_MN, B_MN, BM * CTAS);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < sch.total && ok; t += gridDim.x, ++it) {
+      for (int t = w0; t < sch.total && ok; t += sch.workers, ++it) {
         const TileInfo ti = sch.tile(p, t);
         const int acc = it & 1;
         const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
@@ -462,14 +551,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
             // MN-major: advance 16 k-rows = 2048 bytes.
             const uint64_t ad = A_MN ? make_desc(sA + s * 2048, 64 * BK * 2, 1024) : make_desc(sA + s * 32, 16, 1024);
             const uint64_t bd = B_MN ? make_desc(sB + s * 2048, 64 * BK * 2, 1024) : make_desc(sB + s * 32, 16, 1024);
-            tc_mma_bf16(d_tmem, ad, bd, idesc, (kb | s) != 0 ? 1u : 0u);
+            if (CTAS == 2) tc_mma_bf16_pair(d_tmem, ad, bd, idesc, (kb | s) != 0 ? 1u : 0u);
+            else tc_mma_bf16(d_tmem, ad, bd, idesc, (kb | s) != 0 ? 1u : 0u);
           }
-          tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if (CTAS == 2) tc_commit2(empty_bar(stage), (uint16_t)3);
+          else tc_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        if (ti.nkb > 0) tc_commit(tfull_bar(acc));
-        else mbar_arrive(tfull_bar(acc));
+        if (CTAS == 2) {
+          if (ti.nkb > 0) tc_commit2(tfull_bar(acc), (uint16_t)3);
+          else { mbar_arrive(tfull_bar(acc)); mbar_arrive_cluster(mapa_u32(tfull_bar(acc), 1u)); }
+        } else {
+          if (ti.nkb > 0) tc_commit(tfull_bar(acc));
+          else mbar_arrive(tfull_bar(acc));
+        }
       }
     }
   } else {
@@ -484,7 +581,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
     const uint32_t magic_dp = (uint32_t)(0x100000000ull / (unsigned)dp) + 1u;  // exact x/dp for x < 2^16
     int it = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < sch.total && ok; t += gridDim.x, ++it) {
+    for (int t = w0; t < sch.total && ok; t += sch.workers, ++it) {
       const TileInfo ti = sch.tile(p, t);
       const int acc = it & 1;
       const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
@@ -616,32 +713,63 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) {
+        if (CTAS == 2) mbar_arrive_cluster(mapa_u32(tempty_bar(acc), 0u));  // the leader's barrier
+        else mbar_arrive(tempty_bar(acc));
+      }
     }
   }
 
   // ---- teardown ----
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync_all();  // neither CTA may leave while its peer can still touch its memory
+  else __syncthreads();
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    if (CTAS == 2) tmem_dealloc2(tmem_base, TMEM_COLS);
+    else tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
 
-template <int BN, int MODE>
+template <int BN, int MODE, int CTAS>
 ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStream_t s) {
-  using L = SmemLayout<BN>;
+  using L = SmemLayout<BN, CTAS>;
   static bool attr_done[64] = {};
-  auto kern = ard_gemm_tc_kernel<BN, MODE>;
-  if (!attr_done[ctx->device & 63]) {
+  static int max_clusters[64] = {};
+  auto kern = ard_gemm_tc_kernel<BN, MODE, CTAS>;
+  const int dev = ctx->device & 63;
+  if (!attr_done[dev]) {
     ARD_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
-    attr_done[ctx->device & 63] = true;
+    attr_done[dev] = true;
   }
-  int grid = max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count;  // max_tiles: tile count of the densest pattern
-  if (grid < 1) grid = 1;
-  kern<<<grid, TC_THREADS, L::TOTAL, s>>>(p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = L::TOTAL;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  int workers = ctx->sm_count / CTAS;
+  if (CTAS == 2) {
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (max_clusters[dev] == 0) {
+      // how many CTA pairs the device can hold at once (SM pairs must share a TPC)
+      cfg.gridDim = dim3(ctx->sm_count / 2 * 2);
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) n = ctx->sm_count / 2;
+      max_clusters[dev] = n;
+    }
+    workers = max_clusters[dev];
+  }
+  if (max_tiles < workers) workers = max_tiles;  // max_tiles: tile count of the densest pattern
+  if (workers < 1) workers = 1;
+  cfg.gridDim = dim3(workers * CTAS);
+  TcParams pc = p;
+  ARD_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, pc));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;
@@ -689,20 +817,28 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
   p.status = a.g.status;
   p.force_bn = (kind == ARD_ROW) ? a.bn : 0;
   p.accumulate = a.g.accumulate;
+  p.band_m = ctx->band_m;
   const int bn = (kind == ARD_ROW) ? 256 : a.bn;
 
 #define ARD_TC_CASE(BN_, MODE_, TILES_) \
-  if (bn == BN_) return launch_mode<BN_, MODE_>(ctx, p, (TILES_), s);
+  if (bn == BN_) return launch_mode<BN_, MODE_, 1>(ctx, p, (TILES_), s);
+  // Row patterns with at least two 128-row tiles of output use CTA pairs (256-row tiles).
+#define ARD_TC_PAIR(MODE_, MROWS_, NCOLS_)                                                      \
+  if (ctx->use_pairs && (MROWS_) > BM && (p.force_bn == 0 || p.force_bn >= 128))                \
+    return launch_mode<256, MODE_, 2>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s);
 
   if (kind == ARD_ROW) {
     if (op == OP_FWD) {
       const int mt = cdiv(p.B, BM);
+      ARD_TC_PAIR(M_ROW_FWD, p.B, p.N)
       ARD_TC_CASE(256, M_ROW_FWD, mt * cdiv(p.N, 64))
     } else if (op == OP_BWD_DATA) {
       const int mt = cdiv(p.B, BM);
+      ARD_TC_PAIR(M_ROW_BWD_DATA, p.B, p.K)
       ARD_TC_CASE(256, M_ROW_BWD_DATA, mt * cdiv(p.K, 64))
     } else {
       const int mt = cdiv(p.N, BM);
+      ARD_TC_PAIR(M_ROW_BWD_WEIGHT, p.N, p.K)
       ARD_TC_CASE(256, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 64))
     }
   } else {
@@ -722,5 +858,6 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
     }
   }
 #undef ARD_TC_CASE
+#undef ARD_TC_PAIR
   return ARD_ERR_UNSUPPORTED;
 }
