@@ -30,7 +30,7 @@ from paper_2203_05705_b200 import inputs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of ard_gemm_tc_kernel, averaged over the three
 # GEMMs of one dense (dp = 1) step of this workload, from the ncu capture summarised under profiles/.
-DRAM_TRAFFIC_PER_LAUNCH = None
+DRAM_TRAFFIC_PER_LAUNCH = 569.0e6   # bytes (fwd 661.7 MB, bwd-data 658.0 MB, bwd-weight 387.8 MB)
 
 METRIC = "layer fwd+bwd kept TFLOP/s (row pattern, p=0.5)"
 UNIT = "TFLOP/s"
@@ -359,7 +359,7 @@ def main():
     burst = clk["sm_mhz"] is None or clk["sm_max_mhz"] is None or clk["sm_mhz"] >= 0.9 * clk["sm_max_mhz"]
     peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
     roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": DRAM_TRAFFIC_PER_LAUNCH,
+                "frac": achieved / peak, "traffic": DRAM_TRAFFIC_PER_LAUNCH, "traffic_unit": "bytes per launch (dense step)",
                 "peak_source": peaks["source"] + (" burst" if burst else " sustained") + " cuBLAS bf16 8192^3",
                 "frac_of_burst": achieved / peaks["bf16_tflops"],
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
