@@ -432,7 +432,7 @@ ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B,
   TcArgs t;
   t.g = g;
   t.ts = pat->ts;
-  t.bn = tc_pick_bn(ctx, pat->kind, OP_FWD, B, K, N, pat->ts);
+  t.bn = tc_pick_bn(ctx, pat->kind, OP_FWD, pat->dp_bound, pat->ts);
   // A = X, K-major boxes [128 rows][64 k];  B = kept neurons of W, K-major boxes [64 rows][64 k].
   st = get_maps(ctx, X, B, K, ldx, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);
   if (st != ARD_OK) return st;
@@ -515,7 +515,7 @@ ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, i
   }
   TcArgs t;
   t.ts = pat->ts;
-  t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_DATA, B, K, N, pat->ts);
+  t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_DATA, pat->dp_bound, pat->ts);
   if (pat->kind == ARD_ROW) {
     const void *dyc, *dense;
     int ldc, dense_ld;
@@ -576,7 +576,7 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
   }
   TcArgs t;
   t.ts = pat->ts;
-  t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_WEIGHT, B, K, N, pat->ts);
+  t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_WEIGHT, pat->dp_bound, pat->ts);
   if (pat->kind == ARD_ROW) {
     const void *dyc, *dense;
     int ldc, dense_ld;

@@ -126,7 +126,7 @@ struct TcArgs {
   int ts;
   int bn;  // N tile: 64, 128 or 256
 };
-int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int B, int K, int N, int ts);
+int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int dp_bound, int ts);
 ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s);
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,

@@ -35,11 +35,22 @@ enum TcMode {
   M_ROW_BWD_WEIGHT = 2,
   M_TILE_FWD = 3,
   M_TILE_BWD_DATA = 4,
-  M_TILE_BWD_WEIGHT = 5
+  M_TILE_BWD_WEIGHT = 5,
+  // Tile patterns, "class" form: tile-columns with equal (c mod dp) share one kept-row set and tile-rows
+  // with equal (r mod s) share one kept-column set, so a tile pattern is a handful of dense products
+  // over gathered 64-wide blocks; these modes build 256-wide output tiles from such blocks.
+  M_TILEC_FWD = 6,
+  M_TILEC_BWD_DATA = 7,
+  M_TILEC_BWD_WEIGHT = 8
 };
 
-__host__ __device__ constexpr bool a_is_mn(int mode) { return mode == M_ROW_BWD_WEIGHT || mode == M_TILE_BWD_WEIGHT; }
-__host__ __device__ constexpr bool b_is_mn(int mode) { return mode != M_ROW_FWD && mode != M_TILE_FWD; }
+__host__ __device__ constexpr bool a_is_mn(int mode) {
+  return mode == M_ROW_BWD_WEIGHT || mode == M_TILE_BWD_WEIGHT || mode == M_TILEC_BWD_WEIGHT;
+}
+__host__ __device__ constexpr bool b_is_mn(int mode) {
+  return mode != M_ROW_FWD && mode != M_TILE_FWD && mode != M_TILEC_FWD;
+}
+__host__ __device__ constexpr bool is_class_mode(int mode) { return mode >= M_TILEC_FWD; }
 __host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 4 : (bn == 128 ? 6 : 8); }
 __host__ __device__ constexpr int tmem_cols_for(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }
 
@@ -253,6 +264,11 @@ struct SmemLayout {
   static constexpr int TOTAL = MISC_OFF + 16 + 1024;         // + slack for manual 1024-byte alignment
 };
 
+// Element i of a 4-entry array without dynamic indexing (keeps the array in registers).
+__device__ __forceinline__ int sel4(const int (&a)[4], int i) {
+  return i == 0 ? a[0] : (i == 1 ? a[1] : (i == 2 ? a[2] : a[3]));
+}
+
 // Tile schedule shared by the three roles.
 struct TileInfo {
   int m0, n0;      // origin in GEMM space
@@ -261,6 +277,12 @@ struct TileInfo {
   int kper;        // 64-blocks per pattern tile
   int out_row0;    // tile bwd-weight: first output row (neuron)
   int rows_valid;  // tile bwd-weight: rows of this tile that belong to the kept tile
+  int bn;          // N extent of this tile (whole pair)
+  int nbox;        // 64-wide B boxes this CTA stages
+  int bx[4];       // their coordinates along the B operand's N axis (out of range: a box of zeros)
+  int ax[2];       // MN-major A: coordinates of this CTA's two 64-row boxes
+  int ocol[4];     // output column of each 64-column group of the tile (-1: nothing to write)
+  int orow[2];     // class bwd-weight: output row of each 64-row group of this CTA (-1: nothing to write)
 };
 
 template <int BN, int MODE, int CTAS = 1>
@@ -272,6 +294,11 @@ struct Sched {
   int bn;                  // N extent of the output tile actually used (<= BN)
   int rank;                // CTA rank inside the pair (0 for single-CTA tiles)
   int workers;             // CTAs (or CTA pairs) sharing the tile loop
+  // class modes
+  int Tr, nclass, cstep;   // tile-rows; number of classes; distance between members of a class
+  const int32_t* list;     // kept-tile list the class modes walk (a shared-memory copy when it fits)
+  const int4* ctab;        // per class {first item, list offset, list length, members} (shared memory)
+  int qn, qm;              // pattern tiles per output tile along N and along M
 
   __device__ void init(const TcParams& p, int rank_) {
     rank = rank_;
@@ -284,10 +311,31 @@ struct Sched {
     if (MODE == M_ROW_FWD) { M_gemm = p.B; N_gemm = n_keep; Kc = p.K; }
     else if (MODE == M_ROW_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = n_keep; }
     else if (MODE == M_ROW_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = p.K; Kc = p.B; }
-    else if (MODE == M_TILE_FWD) { M_gemm = p.B; N_gemm = p.N; Kc = 0; }
-    else if (MODE == M_TILE_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 0; }
+    else if (MODE == M_TILE_FWD || MODE == M_TILEC_FWD) { M_gemm = p.B; N_gemm = p.N; Kc = 0; }
+    else if (MODE == M_TILE_BWD_DATA || MODE == M_TILEC_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 0; }
     else { M_gemm = p.N; N_gemm = p.K; Kc = p.B; }
     bn = BN;
+    Tr = p.hdr[HDR_TR];
+    nclass = cstep = qn = qm = 1;
+    list = (MODE == M_TILEC_BWD_DATA) ? p.row_idx : p.col_idx;
+    ctab = nullptr;
+    if (is_class_mode(MODE)) {
+      qn = BN / p.ts;
+      qm = (BM * CTAS) / p.ts;
+      Mt = (M_gemm + BM * CTAS - 1) / (BM * CTAS);
+      if (MODE == M_TILEC_BWD_DATA) {
+        // tile-rows r and r' keep the same tile-columns when (r - r') * (Tc mod dp) = 0 (mod dp)
+        int g = Tc % dp, a = dp;
+        while (g) { const int tmp = a % g; a = g; g = tmp; }  // a = gcd(Tc mod dp, dp)
+        cstep = dp / a;
+        nclass = min(cstep, Tr);
+      } else {
+        cstep = dp;
+        nclass = min(dp, Tc);
+      }
+      total = 0;  // filled in by build_class_table()
+      return;
+    }
     if (MODE == M_TILE_BWD_WEIGHT) {
       subm = (p.ts + BM - 1) / BM;
       subn = p.ts / BN;
@@ -316,7 +364,110 @@ struct Sched {
     total = Mt * Nt;
   }
 
+  // ---- class modes ----
+  __device__ int class_members(int c) const {  // pattern tiles in class c along the gathered axis
+    const int extent = (MODE == M_TILEC_BWD_DATA) ? Tr : Tc;
+    return (extent - 1 - c) / cstep + 1;
+  }
+  __device__ int class_items(int cnt, int len) const {  // output tiles of a class with cnt members
+    if (MODE == M_TILEC_BWD_WEIGHT) return ((cnt + qm - 1) / qm) * ((len + qn - 1) / qn);
+    return Mt * ((cnt + qn - 1) / qn);
+  }
+  // One thread fills the per-class table in shared memory (at most 64 classes); callers synchronise.
+  __device__ void build_class_table(const TcParams& p, int4* tab, int* total_out) const {
+    const int32_t* ptr = (MODE == M_TILEC_BWD_DATA) ? p.row_ptr : p.col_ptr;
+    int run = 0;
+    for (int c = 0; c < nclass; ++c) {
+      const int off = ptr[c], len = ptr[c + 1] - off;
+      const int cnt = class_members(c);
+      tab[c] = make_int4(run, off, len, cnt);
+      run += class_items(cnt, len);
+    }
+    *total_out = run;
+  }
+  __device__ TileInfo class_tile(const TcParams& p, int t) const {
+    TileInfo ti;
+    ti.klist = nullptr;
+    ti.kper = p.ts / BK;
+    ti.out_row0 = 0;
+    ti.rows_valid = BM;
+    ti.n0 = 0;
+    int c = nclass - 1;
+    while (c > 0 && ctab[c].x > t) --c;  // class whose item range holds t
+    const int4 ce = ctab[c];
+    t -= ce.x;
+    const int cnt = ce.w;
+    const int sub64 = p.ts / 64;  // 64-wide boxes per pattern tile
+    int nm;                       // pattern tiles along N in this output tile
+    if (MODE == M_TILEC_BWD_WEIGHT) {
+      const int32_t* rlist = list + ce.y;
+      const int rn = ce.z;
+      const int mtiles = (cnt + qm - 1) / qm;
+      const int mi = t % mtiles, ni = t / mtiles;
+      ti.m0 = 0;
+      ti.nkb = (Kc + BK - 1) / BK;
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {  // this CTA's two 64-row boxes of gathered neurons
+        const int row = rank * BM + 64 * k;
+        const int mem = mi * qm + row / p.ts;
+        const int coord = (mem < cnt) ? (c + mem * cstep) * p.ts + (row % p.ts) : -1;
+        ti.orow[k] = coord;
+        ti.ax[k] = coord >= 0 ? coord : p.N;  // beyond the matrix: TMA fills zeros
+      }
+      const int j0 = ni * qn;
+      nm = min(qn, rn - j0);
+      ti.bn = (nm * p.ts + 64 * CTAS - 1) / (64 * CTAS) * (64 * CTAS);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int mem = j / sub64;
+        ti.ocol[j] = (mem < nm) ? rlist[j0 + mem] * p.ts + (j % sub64) * 64 : -1;
+      }
+    } else {
+      const int ntiles = (cnt + qn - 1) / qn;
+      (void)ntiles;
+      const int mt = t % Mt, v = t / Mt;
+      ti.m0 = mt * BM * CTAS + rank * BM;
+      ti.ax[0] = ti.m0; ti.ax[1] = ti.m0 + 64;
+      ti.orow[0] = ti.orow[1] = 0;
+      const int i0 = v * qn;
+      nm = min(qn, cnt - i0);
+      ti.bn = (nm * p.ts + 64 * CTAS - 1) / (64 * CTAS) * (64 * CTAS);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int mem = j / sub64;
+        ti.ocol[j] = (mem < nm) ? (c + (i0 + mem) * cstep) * p.ts + (j % sub64) * 64 : -1;
+      }
+      ti.klist = list + ce.y;
+      ti.nkb = ce.z * ti.kper;
+    }
+    // this CTA's share of the B boxes
+    const int oob = (MODE == M_TILEC_FWD) ? p.N : p.K;
+    ti.nbox = ti.bn / 64 / CTAS;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int oc = sel4(ti.ocol, rank * ti.nbox + i);
+      ti.bx[i] = (i < ti.nbox && oc >= 0) ? oc : oob;
+    }
+    return ti;
+  }
+
   __device__ TileInfo tile(const TcParams& p, int t) const {
+    if (is_class_mode(MODE)) return class_tile(p, t);
+    TileInfo ti = plain_tile(p, t);
+    // affine block coordinates
+    ti.bn = bn;
+    ti.nbox = bn / CTAS / 64;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      ti.bx[i] = ti.n0 + rank * (bn / CTAS) + 64 * i;
+      ti.ocol[i] = ti.n0 + 64 * i;
+    }
+    ti.ax[0] = ti.m0; ti.ax[1] = ti.m0 + 64;
+    ti.orow[0] = ti.orow[1] = 0;
+    return ti;
+  }
+
+  __device__ TileInfo plain_tile(const TcParams& p, int t) const {
     TileInfo ti;
     ti.klist = nullptr;
     ti.kper = 1;
@@ -474,8 +625,25 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
 
   Sched<BN, MODE, CTAS> sch;
   sch.init(p, (int)rank);
+  if (is_class_mode(MODE)) {
+    // The producer reads one list entry per contraction block: keep the list in shared memory (the
+    // staging area of the forward scatter epilogue is free in these modes) instead of paying a
+    // global-memory round trip on its critical path.
+    // The last KiB of that area holds the per-class table (first item, list offset, length, members).
+    const int n_list = p.hdr[HDR_NKEEP];
+    int4* tab = reinterpret_cast<int4*>(smem + L::STG_OFF + L::STG_BYTES - 1024);
+    int* total_smem = reinterpret_cast<int*>(smem + L::MISC_OFF + 8);
+    int32_t* slist = reinterpret_cast<int32_t*>(smem + L::STG_OFF);
+    const bool fits = n_list * 4 <= L::STG_BYTES - 1024;
+    if (threadIdx.x == 0) sch.build_class_table(p, tab, total_smem);
+    if (fits)
+      for (int i = threadIdx.x; i < n_list; i += TC_THREADS) slist[i] = sch.list[i];
+    __syncthreads();
+    sch.ctab = tab;
+    sch.total = *total_smem;
+    if (fits) sch.list = slist;
+  }
   const int w0 = (int)blockIdx.x / CTAS;  // first tile of this CTA (pair)
-  const int bn = sch.bn;  // N extent of this launch's output tiles (runtime for row patterns)
 
   if (warp == 0) {
     // ===================== TMA producer =====================
@@ -485,13 +653,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       const CUtensorMap* mapB = p.mapB + (p.mapB_indexed ? e : 0);
       tensormap_acquire(mapA);
       tensormap_acquire(mapB);
-      const int bn_cta = bn / CTAS;  // B rows staged by this CTA
-      const uint32_t stage_tx = (uint32_t)(L::A_BYTES + bn_cta * BK * 2) * CTAS;  // bytes of the whole pair
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int t = w0; t < sch.total && ok; t += sch.workers) {
         const TileInfo ti = sch.tile(p, t);
+        const uint32_t stage_tx = (uint32_t)(L::A_BYTES + ti.nbox * 64 * BK * 2) * CTAS;  // bytes of the whole pair
+        // walk of the kept-block list: entry li, 64-wide piece `sub` of that pattern tile
+        int li = 0, sub = 0;
+        int kbase = (ti.klist != nullptr && ti.nkb > 0) ? ti.klist[0] * p.ts : 0;
         for (int kb = 0; kb < ti.nkb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sA = base + stage * L::STAGE_BYTES;
@@ -505,21 +675,31 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
           };
           // contraction coordinate of this block
           int kx;
-          if (MODE == M_TILE_FWD || MODE == M_TILE_BWD_DATA) kx = ti.klist[kb / ti.kper] * p.ts + (kb % ti.kper) * BK;
-          else kx = kb * BK;
+          if (ti.klist != nullptr) {
+            kx = kbase + sub * BK;
+            if (++sub == ti.kper) {
+              sub = 0;
+              ++li;
+              if (kb + 1 < ti.nkb) kbase = ti.klist[li] * p.ts;  // used by the next block, not this one
+            }
+          } else {
+            kx = kb * BK;
+          }
           if (!A_MN) {
             load(sA, mapA, kx, ti.m0);  // [BM rows][64 k]
           } else {
 #pragma unroll
             for (int i = 0; i < BM / 64; ++i)  // [64 k rows][64 m] per box
-              load(sA + i * (64 * BK * 2), mapA, ti.m0 + 64 * i, kx);
+              load(sA + i * (64 * BK * 2), mapA, ti.ax[i], kx);
           }
           // B always moves in 64-wide boxes: K-major [64 rows][64 k] stacked, MN-major [64 k][64 n].
-          // In a pair this CTA stages the B rows [rank*bn/2, (rank+1)*bn/2) of the tile.
-          const int nb0 = ti.n0 + (int)rank * bn_cta;
-          for (int i = 0; i < bn_cta / 64; ++i) {
-            if (!B_MN) load(sB + i * (64 * BK * 2), mapB, kx, nb0 + 64 * i);
-            else load(sB + i * (64 * BK * 2), mapB, nb0 + 64 * i, kx);
+          // In a pair this CTA stages the second half of the tile's B boxes if its rank is 1.
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (i < ti.nbox) {
+              if (!B_MN) load(sB + i * (64 * BK * 2), mapB, kx, ti.bx[i]);
+              else load(sB + i * (64 * BK * 2), mapB, ti.bx[i], kx);
+            }
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -528,13 +708,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
     if (lane == 0 && rank == 0) {
-      const uint32_t idesc = make_idesc(bn, A_MN, B_MN, BM * CTAS);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
       for (int t = w0; t < sch.total && ok; t += sch.workers, ++it) {
         const TileInfo ti = sch.tile(p, t);
+        const uint32_t idesc = make_idesc(ti.bn, A_MN, B_MN, BM * CTAS);
         const int acc = it & 1;
         const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
@@ -575,8 +755,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
     const int half = (warp - 2) >> 2;       // which half of the tile's columns
     const int row_in_tile = q * 32 + lane;  // accumulator row owned by this thread
     float* stg = reinterpret_cast<float*>(smem + L::STG_OFF) + (warp - 2) * (32 * 33);
-    const int nch = bn / 32;                // 32-column chunks in a tile
-    const int ch_lo = half * (nch / 2), ch_hi = (half == 0) ? nch / 2 : nch;
     const int dp = sch.dp, bb = sch.b - 1;
     const uint32_t magic_dp = (uint32_t)(0x100000000ull / (unsigned)dp) + 1u;  // exact x/dp for x < 2^16
     int it = 0;
@@ -589,6 +767,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
       const int m = ti.m0 + row_in_tile;
+      const int nch = ti.bn / 32;  // 32-column chunks in this tile, split between the two warps of a quadrant
+      const int ch_lo = half * (nch / 2), ch_hi = (half == 0) ? nch / 2 : nch;
 
       // Output row and validity by mode.
       bool row_ok;
@@ -599,6 +779,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       } else if (MODE == M_TILE_BWD_WEIGHT) {
         row_ok = row_in_tile < ti.rows_valid && m < sch.M_gemm;
         out_row = m;
+      } else if (MODE == M_TILEC_BWD_WEIGHT) {
+        const int orow = (row_in_tile >> 6) ? ti.orow[1] : ti.orow[0];
+        row_ok = orow >= 0;
+        out_row = orow + (row_in_tile & 63);
       } else {
         row_ok = m < sch.M_gemm;
         out_row = m;
@@ -606,7 +790,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
 
       // One 32-column chunk of this thread's accumulator row, already loaded into r[].
       auto emit = [&](const uint32_t (&r)[32], int ch) {
-        const int n = ti.n0 + ch * 32;
+        const int oc = sel4(ti.ocol, ch >> 1);
+        if (oc < 0) return;                    // padding of a class tile
+        const int n = oc + (ch & 1) * 32;      // output column of this chunk
         float v[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = (ti.nkb > 0) ? p.alpha * __uint_as_float(r[i]) : 0.f;
@@ -677,7 +863,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
             __syncwarp();
           }
         } else {
-          const int nvalid = min(32, sch.N_gemm - n);
+          const int nvalid = is_class_mode(MODE) ? 32 : min(32, sch.N_gemm - n);
           if (row_ok && nvalid > 0) {
             store_row32(p.out, (size_t)out_row * p.ldo, n, v, nvalid, p.out_is_f32, p.accumulate);
             if (MODE == M_ROW_BWD_WEIGHT && p.zero_fill) {
@@ -779,12 +965,16 @@ inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 
 }  // namespace
 
-// N extent of the output tile.  Tile patterns: fixed per launch (it must divide the pattern tile).
-// Row patterns: 0 = chosen on the device from the sampled n_keep, or the value forced by ard_set_tile_n.
-int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int B, int K, int N, int ts) {
-  (void)B; (void)K; (void)N;
+// N extent of the output tile.
+//   Row patterns: 0 = chosen on the device from the sampled n_keep, or the value forced by ard_set_tile_n.
+//   Tile patterns: 0 = class form (256-wide tiles gathered from pattern tiles of one class), available for
+//   pattern tiles of 64 / 128 (forward and backward-data also 256) and periods up to 64; otherwise a fixed
+//   width that divides the pattern tile.
+int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int dp_bound, int ts) {
   const int f = ctx->force_bn;
   if (kind == ARD_TILE) {
+    const bool class_ok = dp_bound <= 64 && (ts == 64 || ts == 128 || (ts == 256 && op != OP_BWD_WEIGHT));
+    if (f == 0 && class_ok) return 0;
     if (f && ts % f == 0 && (op == OP_BWD_WEIGHT || f <= 128)) return f;
     if (op == OP_BWD_WEIGHT) return ts % 256 == 0 ? 256 : (ts % 128 == 0 ? 128 : 64);
     return ts % 128 == 0 ? 128 : 64;
@@ -841,6 +1031,18 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
       ARD_TC_PAIR(M_ROW_BWD_WEIGHT, p.N, p.K)
       ARD_TC_CASE(256, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 64))
     }
+  } else if (bn == 0) {
+    // class form of the tile pattern; the grid covers all SMs, CTAs without tiles leave at once
+    const int many = 1 << 30;
+    const int rows = (op == OP_BWD_WEIGHT) ? p.N : p.B;
+    const bool pairs = ctx->use_pairs && rows > BM;
+    if (op == OP_FWD)
+      return pairs ? launch_mode<256, M_TILEC_FWD, 2>(ctx, p, many, s) : launch_mode<256, M_TILEC_FWD, 1>(ctx, p, many, s);
+    if (op == OP_BWD_DATA)
+      return pairs ? launch_mode<256, M_TILEC_BWD_DATA, 2>(ctx, p, many, s)
+                   : launch_mode<256, M_TILEC_BWD_DATA, 1>(ctx, p, many, s);
+    return pairs ? launch_mode<256, M_TILEC_BWD_WEIGHT, 2>(ctx, p, many, s)
+                 : launch_mode<256, M_TILEC_BWD_WEIGHT, 1>(ctx, p, many, s);
   } else {
     if (op == OP_FWD) {
       const int mt = cdiv(p.B, BM);
