@@ -424,7 +424,7 @@ def main():
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only) ----
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        dt, fl, threads, sample = oracle_sample_seconds(wl, d, 4096)
+        dt, fl, threads, sample = oracle_sample_seconds(wl, d, max(wl["B"], wl["N"]))   # one full step
         cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
                "seconds": dt}
 
