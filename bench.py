@@ -41,6 +41,8 @@ WORKLOADS = {
     "mlp8192_tile": dict(config=5, B=4096, K=8192, N=8192, kind="tile", ts=128, p=0.5, n_dp=16),
     "mlp4096_tile": dict(config=3, B=1024, K=4096, N=4096, kind="tile", ts=64, p=0.5, n_dp=16),
     "mlp2048_row": dict(config=2, B=128, K=2048, N=2048, kind="row", ts=0, p=0.5, n_dp=16),
+    # LSTM layer (config 4): a step is one sequence, forward + BPTT, one fresh pattern per sequence
+    "lstm1024": dict(config=4, T=35, B=64, I=1024, H=1024, kind="lstm", p=0.5, n_dp=16),
 }
 
 # Measured peaks of this machine's B200s (generated file), else the documented fallback.
@@ -201,6 +203,116 @@ def run_reference(args, wl):
     print(json.dumps(line))
 
 
+def run_lstm(args, wl):
+    """LSTM workload: every step is one sequence (T time steps forward, then BPTT and the weight gradient)."""
+    import torch
+    from paper_2203_05705_b200 import ard
+    from paper_2203_05705_b200.lstm import LstmLayer
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    clocks = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    T, B, I, H, p, n_dp = wl["T"], wl["B"], wl["I"], wl["H"], wl["p"], wl["n_dp"]
+    c4 = inputs.config4(T, B, I, H, 0)
+    bf = torch.bfloat16
+    W = torch.from_numpy(np.ascontiguousarray(c4["W"].T)).to(bf).cuda()
+    hX = torch.from_numpy(c4["X"]).to(bf).pin_memory()
+    hdH = torch.from_numpy(c4["dH"]).pin_memory()
+    X, dH = hX.cuda(), hdH.cuda()
+    hH = torch.empty((T, B, H), dtype=bf).pin_memory()
+    ctx = ard.ard_create(0, 2 * T * B * 4 * H + 4096)
+    ard.ard_set_distribution(ctx, 0, inputs.max_entropy_K(p, n_dp))
+    pat = ard.ard_pattern_create(ctx, ard.ARD_ROW, I + H, H, 0)
+    layer = LstmLayer(ctx, pat, T, B, I, H, W)
+    alpha = 1.0 / (1.0 - p)
+
+    def seq(it, dense=False, host=False):
+        if dense:
+            ard.ard_pattern_set(ctx, pat, 1, 1)
+        else:
+            ard.ard_sample_pattern(ctx, pat, 0, inputs.BASE_SEED, it, 4)
+        if host:
+            X.copy_(hX, non_blocking=True)
+            dH.copy_(hdH, non_blocking=True)
+        layer.load_inputs(X)
+        Hs = layer.forward(alpha)
+        layer.backward(alpha, dH)
+        if host:
+            hH.copy_(Hs, non_blocking=True)
+
+    def timed(n, first, **kw):
+        for w in range(args.warmup):
+            seq(first + w, **kw)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record()
+        for i in range(n):
+            seq(first + args.warmup + i, **kw)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1), t0, time.time()
+
+    steps = args.steps
+    l0 = ard.ard_launch_count(ctx)
+    ms, t0, t1 = timed(steps, 0)
+    launches = (ard.ard_launch_count(ctx) - l0) * steps // (steps + args.warmup)
+    clk = clocks.stop(t0, t1)
+    status = ard.ard_last_device_status(ctx)
+    nks = []
+    for i in range(steps):
+        ard.ard_sample_pattern(ctx, pat, 0, inputs.BASE_SEED, args.warmup + i, 4)
+        nks.append(ard.ard_pattern_to_host(pat, 0)[2])
+    per_unit = 3 * 2.0 * T * B * (I + H) * 4            # FLOPs per kept hidden unit and sequence
+    kept = sum(per_unit * nk for nk in nks)
+    value = kept / (ms * 1e-3) / 1e12
+    ms_dense, _, _ = timed(max(5, steps // 4), 100000, dense=True)
+    ms_e, _, _ = timed(max(5, steps // 4), 200000, host=True)
+    ne = max(5, steps // 4)
+    nks_e = []
+    for i in range(ne):
+        ard.ard_sample_pattern(ctx, pat, 0, inputs.BASE_SEED, 200000 + args.warmup + i, 4)
+        nks_e.append(ard.ard_pattern_to_host(pat, 0)[2])
+    peaks = load_peaks()
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import lstm as OL
+        from oracle import pattern as OP
+        m = OP.row_mask(H, 2, 1)
+        tc0 = time.perf_counter()
+        fw = OL.fwd(c4["X"], c4["W"], None, m, alpha)
+        OL.bwd(fw, c4["W"], m, alpha, c4["dH"])
+        dt = time.perf_counter() - tc0
+        try:
+            from threadpoolctl import threadpool_info
+            threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        except Exception:
+            threads = os.cpu_count() or 1
+        cpu = {"value": per_unit * (H // 2) / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": "one full sequence, dp=2", "seconds": dt}
+    line = {
+        "metric": "LSTM layer fwd+BPTT kept TFLOP/s (row pattern on hidden units, p=0.5)", "value": value,
+        "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": args.warmup, "ms_per_step": ms / steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "T": T, "B": B, "I": I, "H": H, "p": p, "n_dp": n_dp,
+                   "l2": "weights (16 MB) stay in L2 by design; a step is a whole sequence"},
+        "dense_equiv_tflops": per_unit * H * steps / (ms * 1e-3) / 1e12, "clocks": clk,
+        "e2e": {"value": sum(per_unit * nk for nk in nks_e) / (ms_e * 1e-3) / 1e12, "unit": UNIT,
+                "h2d_bytes_per_step": hX.numel() * 2 + hdH.numel() * 4, "d2h_bytes_per_step": hH.numel() * 2,
+                "ms_per_step": ms_e / ne},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "achieved": value, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": value / peaks["bf16_tflops"], "traffic": None,
+                     "note": "35 dependent steps of a 64-row product: bound by per-step latency, not by the tensor pipe"},
+        "cpu_baseline": cpu,
+        "detail": {"dense_ms_per_step": {"own_kernels_dp1": ms_dense / max(5, steps // 4)},
+                   "speedup_vs_dense": {str(p): (ms_dense / max(5, steps // 4)) / (ms / steps)},
+                   "kept_fraction": {str(p): float(np.mean(nks)) / H}},
+        "device_status": int(status),
+    }
+    print(json.dumps(line))
+    ard.ard_pattern_destroy(pat)
+    ard.ard_destroy(ctx)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -214,6 +326,8 @@ def main():
     wl = WORKLOADS[args.workload]
     if args.impl == "reference":
         return run_reference(args, wl)
+    if wl["kind"] == "lstm":
+        return run_lstm(args, wl)
 
     import torch
     import torch.distributed as dist

@@ -197,6 +197,36 @@ ard_status ard_lstm_gates(ard_ctx* ctx, const ard_pattern* pat, ard_dtype h_dtyp
                           const float* Z, int ldz_gate, const float* bias, const float* c_prev, int ldc, float* c,
                           void* h, int ldh, int h_scatter, float* gates_saved, void* cuda_stream);
 
+/* Gate pre-activations of the kept hidden units for one time step, all four gate blocks in one call:
+ *   Z[:, g*ldz_gate + j] = sum_k XH[:, k] * W[g*H + keep[j]][k],   g = 0..3 (i|f|g|o), j < n_keep.
+ * XH [B][KH] bf16 (ldxh) is [x_t, h_{t-1}] side by side (KH = I + H; h full width, zeros at dropped
+ * units), W [4H][KH] bf16 neuron-major (ldw), Z fp32 [B][4*ldz_gate] with ldz_gate >= H.  `pat` is a row
+ * pattern created with K_dim = KH and N_dim = H (Sec. 3.1 applied to the hidden units, Sec. 7). */
+ard_status ard_lstm_gate_gemm(ard_ctx* ctx, const ard_pattern* pat, int B, int KH, int H, const void* XH, int ldxh,
+                              const void* W, int ldw, float* Z, int ldz_gate, void* cuda_stream);
+/* Its adjoint with respect to XH:  dXH[:, k] (+)= sum_g sum_j dZ[:, g*ldz_gate + j] * W[g*H + keep[j]][k].
+ * dZ bf16 compact [B][4*ldz_gate], dXH fp32 [B][KH] (lddxh); accumulate != 0 adds to dXH. */
+ard_status ard_lstm_gate_gemm_bwd(ard_ctx* ctx, const ard_pattern* pat, int B, int KH, int H, const void* dZ,
+                                  int ldz_gate, const void* W, int ldw, float* dXH, int lddxh, int accumulate,
+                                  void* cuda_stream);
+
+/* Whole-sequence forward: for t = 0..T-1, ard_lstm_gate_gemm on XH[t] followed by ard_lstm_gates, which writes
+ * h_t into the h half of XH[t+1].  The loop runs in native code and only enqueues kernels.
+ *   XH [T+1][B][I+H] bf16: the caller fills the x halves of XH[0..T-1] and the h half of XH[0] (h_0, zeros at
+ *   dropped units); C [T+1][B][H] fp32 compact cell states, C[0] = c_0; G [T][B][4H] fp32 saved gates;
+ *   Z [B][4H] fp32 scratch; W [4H][I+H] bf16 (ldw); bias [4][H] or NULL. */
+ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha, void* XH,
+                            const void* W, int ldw, const float* bias, float* C, float* G, float* Z,
+                            void* cuda_stream);
+/* Whole-sequence BPTT of ard_lstm_forward.  D [T][B][I+H] fp32 must hold, on entry, zeros in the x halves and
+ * the upstream gradient of h_{t-1} in the h half of D[t] (t >= 1); on return its x halves hold dx_t and the h
+ * half of D[0] the gradient of h_0.  dH_last [B][H] fp32 is the gradient of h_{T-1}; dc [B][H] fp32 must be
+ * zero on entry (or hold the gradient of c_T) and returns the gradient of c_0; DZ [T][B][4H] bf16 scratch;
+ * dW [4H][I+H] fp32 receives the weight gradient (dropped units' rows zero). */
+ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                             const void* XH, const void* W, int ldw, const float* C, const float* G,
+                             const float* dH_last, float* D, float* dc, void* DZ, float* dW, void* cuda_stream);
+
 /* Adjoint of ard_lstm_gates.  dh [B][lddh] (fp32; compact, or full width if dh_scatter != 0, in
  * which case only kept columns are read), dc_inout [B][ldc]: in = gradient arriving at c from the
  * next step, out = gradient w.r.t. c_prev.  dZ [B][4*ldz_gate] compact like Z, element type

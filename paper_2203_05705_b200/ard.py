@@ -30,7 +30,7 @@ EXPORTS = [
     "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_compact_reuse", "ard_set_distribution", "ard_get_distribution_cdf",
     "ard_pattern_create", "ard_pattern_destroy", "ard_sample_pattern", "ard_pattern_set",
     "ard_pattern_to_host", "ard_pattern_tile_lists_to_host", "ard_fwd", "ard_bwd_data", "ard_bwd_weight",
-    "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_last_device_status", "ard_status_string", "ard_launch_count",
+    "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_lstm_forward", "ard_lstm_backward", "ard_last_device_status", "ard_status_string", "ard_launch_count",
 ]
 
 _lib = None
@@ -71,6 +71,10 @@ def lib():
         "ard_bwd_data": [vp, vp, i32, i32, i32, i32, f32, vp, i32, i32, vp, i32, vp, i32, vp],
         "ard_bwd_data_static_scratch": [vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_bwd_weight": [vp, vp, i32, i32, i32, i32, i32, f32, vp, i32, vp, i32, i32, vp, i32, i32, vp],
+        "ard_lstm_gate_gemm": [vp, vp, i32, i32, i32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_lstm_gate_gemm_bwd": [vp, vp, i32, i32, i32, vp, i32, vp, i32, vp, i32, i32, vp],
+        "ard_lstm_forward": [vp, vp, i32, i32, i32, i32, f32, vp, vp, i32, vp, vp, vp, vp, vp],
+        "ard_lstm_backward": [vp, vp, i32, i32, i32, i32, f32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp],
         "ard_lstm_gates": [vp, vp, i32, i32, i32, f32, vp, i32, vp, vp, i32, vp, vp, i32, i32, vp, vp],
         "ard_lstm_gates_bwd": [vp, vp, i32, i32, i32, f32, vp, vp, vp, i32, vp, i32, i32, vp, vp, i32, vp],
         "ard_last_device_status": [vp, vp],
@@ -209,6 +213,27 @@ def ard_bwd_weight(ctx, pat, dtype, dW_dtype, B, K, N, alpha, X, ldx, dY, lddy, 
     _check(lib().ard_bwd_weight(ctx, pat, dtype, dW_dtype, B, K, N, alpha, _ptr(X), ldx, _ptr(dY), lddy,
                                 dy_is_compact, _ptr(dW), lddw, zero_fill_dropped, _stream(stream)),
            "ard_bwd_weight")
+
+
+def ard_lstm_gate_gemm(ctx, pat, B, KH, H, XH, ldxh, W, ldw, Z, ldz_gate, stream=None):
+    _check(lib().ard_lstm_gate_gemm(ctx, pat, B, KH, H, _ptr(XH), ldxh, _ptr(W), ldw, _ptr(Z), ldz_gate,
+                                    _stream(stream)), "ard_lstm_gate_gemm")
+
+
+def ard_lstm_gate_gemm_bwd(ctx, pat, B, KH, H, dZ, ldz_gate, W, ldw, dXH, lddxh, accumulate, stream=None):
+    _check(lib().ard_lstm_gate_gemm_bwd(ctx, pat, B, KH, H, _ptr(dZ), ldz_gate, _ptr(W), ldw, _ptr(dXH), lddxh,
+                                        accumulate, _stream(stream)), "ard_lstm_gate_gemm_bwd")
+
+
+def ard_lstm_forward(ctx, pat, T, B, I, H, alpha, XH, W, ldw, bias, C, G, Z, stream=None):
+    _check(lib().ard_lstm_forward(ctx, pat, T, B, I, H, alpha, _ptr(XH), _ptr(W), ldw, _ptr(bias), _ptr(C), _ptr(G),
+                                  _ptr(Z), _stream(stream)), "ard_lstm_forward")
+
+
+def ard_lstm_backward(ctx, pat, T, B, I, H, alpha, XH, W, ldw, C, G, dH_last, D, dc, DZ, dW, stream=None):
+    _check(lib().ard_lstm_backward(ctx, pat, T, B, I, H, alpha, _ptr(XH), _ptr(W), ldw, _ptr(C), _ptr(G),
+                                   _ptr(dH_last), _ptr(D), _ptr(dc), _ptr(DZ), _ptr(dW), _stream(stream)),
+           "ard_lstm_backward")
 
 
 def ard_lstm_gates(ctx, pat, h_dtype, B, H, alpha, Z, ldz_gate, bias, c_prev, ldc, c, h, ldh, h_scatter,

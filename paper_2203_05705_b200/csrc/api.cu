@@ -42,15 +42,16 @@ bool encode_map(ard_ctx* ctx, CUtensorMap* out, const void* base, uint64_t cols,
   return r == CUDA_SUCCESS;
 }
 
-constexpr size_t MAX_CACHED_TABLES = 96;
+constexpr size_t MAX_CACHED_TABLES = 1024;
 
 // Returns a device table of descriptors for `base`; builds and caches it on first use.
 ard_status get_maps(ard_ctx* ctx, const void* base, int rows, int cols, int ld, int units, int variant, int dp_bound,
                     int box_rows, int box_cols, const CUtensorMap** out, const void* dense_base = nullptr,
                     int dense_ld = 0) {
-  for (const MapTable& t : ctx->maps) {
+  for (MapTable& t : ctx->maps) {
     if (t.base == base && t.dense_base == dense_base && t.dense_ld == dense_ld && t.rows == rows && t.cols == cols && t.ld == ld && t.elem_bytes == units &&
         t.variant == variant && t.dp_bound == dp_bound && t.box_rows == box_rows && t.box_cols == box_cols) {
+      t.epoch = ctx->epoch;
       *out = t.d_maps;
       return ARD_OK;
     }
@@ -83,13 +84,20 @@ ard_status get_maps(ard_ctx* ctx, const void* base, int rows, int cols, int ld, 
       }
   }
   if (ctx->maps.size() >= MAX_CACHED_TABLES) {
-    // cudaFree synchronises the device, so no kernel can still be reading the evicted table.
-    cudaFree(ctx->maps.front().d_maps);
-    ctx->maps.erase(ctx->maps.begin());
+    // Evict the table that has gone unused for the longest time, never one the running call already
+    // handed out.  cudaFree synchronises the device, so no kernel can still be reading it.
+    size_t victim = ctx->maps.size();
+    for (size_t i = 0; i < ctx->maps.size(); ++i)
+      if (ctx->maps[i].epoch != ctx->epoch && (victim == ctx->maps.size() || ctx->maps[i].epoch < ctx->maps[victim].epoch))
+        victim = i;
+    if (victim == ctx->maps.size()) return ARD_ERR_NOMEM;
+    cudaFree(ctx->maps[victim].d_maps);
+    ctx->maps.erase(ctx->maps.begin() + victim);
   }
   MapTable t;
   t.base = base; t.dense_base = dense_base; t.dense_ld = dense_ld; t.rows = rows; t.cols = cols; t.ld = ld; t.elem_bytes = units; t.variant = variant;
   t.dp_bound = dp_bound; t.box_rows = box_rows; t.box_cols = box_cols; t.count = count;
+  t.epoch = ctx->epoch;
   t.d_maps = nullptr;
   if (cudaMalloc(&t.d_maps, sizeof(CUtensorMap) * count) != cudaSuccess) return ARD_ERR_NOMEM;
   if (cudaMemcpy(t.d_maps, h.data(), sizeof(CUtensorMap) * count, cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -103,6 +111,7 @@ ard_status get_maps(ard_ctx* ctx, const void* base, int rows, int cols, int ld, 
 
 ard_status check_common(ard_ctx* ctx, const ard_pattern* pat, int B, int K, int N) {
   if (!ctx || !pat) return ARD_ERR_INVALID_ARG;
+  ctx->epoch++;  // a new public call: descriptor tables it obtains stay pinned until it returns
   if (pat->ctx != ctx) return ARD_ERR_INVALID_ARG;
   if (B < 0 || K < 0 || N < 0) return ARD_ERR_INVALID_ARG;
   if (K != pat->K_dim || N != pat->N_dim) return ARD_ERR_SHAPE;
@@ -181,6 +190,7 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->d_workspace = nullptr;
   ctx->d_status = nullptr;
   ctx->launches = 0;
+  ctx->epoch = 1;
   ctx->encode_fn = nullptr;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return ARD_ERR_CUDA; }
@@ -601,6 +611,105 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
 
 // ---------------------------------------------------------------------------------------------------
 
+// One launch for the four gate blocks when the tensor-core path can take the operands; otherwise four
+// calls of the single-gate products.
+ard_status ard_lstm_gate_gemm(ard_ctx* ctx, const ard_pattern* pat, int B, int KH, int H, const void* XH, int ldxh,
+                              const void* W, int ldw, float* Z, int ldz_gate, void* cuda_stream) {
+  ard_status st = check_common(ctx, pat, B, KH, H);
+  if (st != ARD_OK) return st;
+  if (!XH || !W || !Z) return ARD_ERR_INVALID_ARG;
+  if (pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+  if (ldxh < KH || ldw < KH || ldz_gate < H) return ARD_ERR_SHAPE;
+  if (B == 0) return ARD_OK;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const char* Wc = reinterpret_cast<const char*>(W);
+  ard_status el = ctx->path == ARD_PATH_CUDA_CORE
+                      ? ARD_ERR_UNSUPPORTED
+                      : tc_eligible(ctx, pat, ARD_BF16, B, KH, H, XH, ldxh, W, ldw, Z, 4 * ldz_gate, 4);
+  if (el == ARD_OK && (ldz_gate % 8 != 0 || ((size_t)H * ldw * 2) % 16 != 0)) el = ARD_ERR_ALIGNMENT;
+  if (el != ARD_OK) {
+    if (ctx->path == ARD_PATH_TENSOR_CORE) return el;
+    for (int g = 0; g < 4; ++g) {
+      st = ard_fwd(ctx, pat, ARD_BF16, B, KH, H, 1.0f, XH, ldxh, Wc + (size_t)g * H * ldw * 2, ldw, Z + (size_t)g * ldz_gate,
+                   4 * ldz_gate, (ard_outmode)(ARD_OUT_COMPACT | ARD_FLAG_OUT_F32), cuda_stream);
+      if (st != ARD_OK) return st;
+    }
+    return ARD_OK;
+  }
+  TcArgs t;
+  GemmArgs g;
+  fill_common(g, ctx, pat, B, KH, H, 1.0f);
+  g.A0 = XH; g.lda0 = ldxh; g.A1 = W; g.lda1 = ldw; g.out = Z; g.ldo = 4 * ldz_gate;
+  g.out_is_f32 = 1;
+  t.g = g;
+  t.ts = ldz_gate;
+  t.bn = 0;
+  st = get_maps(ctx, XH, B, KH, ldxh, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);
+  if (st != ARD_OK) return st;
+  t.mapA_indexed = 0;
+  for (int gate = 0; gate < 4; ++gate) {
+    st = get_maps(ctx, Wc + (size_t)gate * H * ldw * 2, H, KH, ldw, H, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64,
+                  &t.mapB4[gate]);
+    if (st != ARD_OK) return st;
+    t.mapA4[gate] = t.mapA;
+  }
+  t.mapB = t.mapB4[0];
+  t.mapB_indexed = 1;
+  return launch_lstm_tc(ctx, 0, t, s);
+}
+
+ard_status ard_lstm_gate_gemm_bwd(ard_ctx* ctx, const ard_pattern* pat, int B, int KH, int H, const void* dZ,
+                                  int ldz_gate, const void* W, int ldw, float* dXH, int lddxh, int accumulate,
+                                  void* cuda_stream) {
+  ard_status st = check_common(ctx, pat, B, KH, H);
+  if (st != ARD_OK) return st;
+  if (!dZ || !W || !dXH) return ARD_ERR_INVALID_ARG;
+  if (pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+  if (ldz_gate < 1 || ldw < KH || lddxh < KH) return ARD_ERR_SHAPE;
+  if (B == 0) return ARD_OK;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const char* Wc = reinterpret_cast<const char*>(W);
+  const char* dZc = reinterpret_cast<const char*>(dZ);
+  ard_status el = ctx->path == ARD_PATH_CUDA_CORE
+                      ? ARD_ERR_UNSUPPORTED
+                      : tc_eligible(ctx, pat, ARD_BF16, B, KH, H, dZ, 4 * ldz_gate, W, ldw, dXH, lddxh, 4);
+  if (el == ARD_OK && (ldz_gate % 8 != 0 || ((size_t)H * ldw * 2) % 16 != 0)) el = ARD_ERR_ALIGNMENT;
+  if (el != ARD_OK) {
+    if (ctx->path == ARD_PATH_TENSOR_CORE) return el;
+    for (int g = 0; g < 4; ++g) {
+      const int flags = 1 | ARD_FLAG_OUT_F32 | ((accumulate || g > 0) ? ARD_FLAG_ACCUMULATE : 0);
+      st = ard_bwd_data(ctx, pat, ARD_BF16, B, KH, H, 1.0f, dZc + (size_t)g * ldz_gate * 2, 4 * ldz_gate, flags,
+                        Wc + (size_t)g * H * ldw * 2, ldw, dXH, lddxh, cuda_stream);
+      if (st != ARD_OK) return st;
+    }
+    return ARD_OK;
+  }
+  TcArgs t;
+  GemmArgs g;
+  fill_common(g, ctx, pat, B, KH, H, 1.0f);
+  g.A0 = dZ; g.lda0 = 4 * ldz_gate; g.A1 = W; g.lda1 = ldw; g.out = dXH; g.ldo = lddxh;
+  g.flag0 = 1;
+  g.out_is_f32 = 1;
+  g.accumulate = accumulate ? 1 : 0;
+  t.g = g;
+  t.ts = ldz_gate;
+  t.bn = ctx->force_bn;
+  for (int gate = 0; gate < 4; ++gate) {
+    st = get_maps(ctx, dZc + (size_t)gate * ldz_gate * 2, B, H, 4 * ldz_gate, H, MAP_COMPACT_COLS, pat->dp_bound, 128, 64,
+                  &t.mapA4[gate]);
+    if (st != ARD_OK) return st;
+    st = get_maps(ctx, Wc + (size_t)gate * H * ldw * 2, H, KH, ldw, H, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64,
+                  &t.mapB4[gate]);
+    if (st != ARD_OK) return st;
+  }
+  t.mapA = t.mapA4[0];
+  t.mapB = t.mapB4[0];
+  t.mapA_indexed = t.mapB_indexed = 1;
+  return launch_lstm_tc(ctx, 1, t, s);
+}
+
 ard_status ard_lstm_gates(ard_ctx* ctx, const ard_pattern* pat, ard_dtype h_dtype, int B, int H, float alpha,
                           const float* Z, int ldz_gate, const float* bias, const float* c_prev, int ldc, float* c,
                           void* h, int ldh, int h_scatter, float* gates_saved, void* cuda_stream) {
@@ -627,6 +736,52 @@ ard_status ard_lstm_gates_bwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dz
   DeviceGuard guard(ctx->device);
   return launch_lstm_gates_bwd(ctx, pat, dz_dtype, B, H, alpha, gates_saved, c_prev, c, ldc, dh, lddh, dh_scatter,
                                dc_inout, dZ, ldz_gate, (cudaStream_t)cuda_stream);
+}
+
+// Whole-sequence drivers: the time loop runs here, in native code, and only enqueues kernels.
+ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha, void* XH,
+                            const void* W, int ldw, const float* bias, float* C, float* G, float* Z,
+                            void* cuda_stream) {
+  if (!ctx || !pat || !XH || !W || !C || !G || !Z) return ARD_ERR_INVALID_ARG;
+  if (T < 0 || B < 0 || I < 0 || H < 1) return ARD_ERR_INVALID_ARG;
+  const int KH = I + H;
+  __nv_bfloat16* xh = reinterpret_cast<__nv_bfloat16*>(XH);
+  for (int t = 0; t < T; ++t) {
+    __nv_bfloat16* xh_t = xh + (size_t)t * B * KH;
+    __nv_bfloat16* h_out = xh + (size_t)(t + 1) * B * KH + I;  // h_t lands in the operand of step t+1
+    ard_status st = ard_lstm_gate_gemm(ctx, pat, B, KH, H, xh_t, KH, W, ldw, Z, H, cuda_stream);
+    if (st != ARD_OK) return st;
+    st = ard_lstm_gates(ctx, pat, ARD_BF16, B, H, alpha, Z, H, bias, C + (size_t)t * B * H, H,
+                        C + (size_t)(t + 1) * B * H, h_out, KH, 1, G + (size_t)t * B * 4 * H, cuda_stream);
+    if (st != ARD_OK) return st;
+  }
+  return ARD_OK;
+}
+
+ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                             const void* XH, const void* W, int ldw, const float* C, const float* G,
+                             const float* dH_last, float* D, float* dc, void* DZ, float* dW, void* cuda_stream) {
+  if (!ctx || !pat || !XH || !W || !C || !G || !dH_last || !D || !dc || !DZ || !dW) return ARD_ERR_INVALID_ARG;
+  if (T < 1 || B < 0 || I < 0 || H < 1) return ARD_ERR_INVALID_ARG;
+  const int KH = I + H;
+  __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(DZ);
+  for (int t = T - 1; t >= 0; --t) {
+    const float* dh = (t == T - 1) ? dH_last : D + (size_t)(t + 1) * B * KH + I;
+    const int lddh = (t == T - 1) ? H : KH;
+    ard_status st = ard_lstm_gates_bwd(ctx, pat, ARD_BF16, B, H, alpha, G + (size_t)t * B * 4 * H,
+                                       C + (size_t)t * B * H, C + (size_t)(t + 1) * B * H, H, dh, lddh, 1, dc,
+                                       dz + (size_t)t * B * 4 * H, H, cuda_stream);
+    if (st != ARD_OK) return st;
+    st = ard_lstm_gate_gemm_bwd(ctx, pat, B, KH, H, dz + (size_t)t * B * 4 * H, H, W, ldw, D + (size_t)t * B * KH, KH,
+                                1, cuda_stream);
+    if (st != ARD_OK) return st;
+  }
+  for (int g = 0; g < 4; ++g) {  // weight gradient: one product over all T*B rows per gate
+    ard_status st = ard_bwd_weight(ctx, pat, ARD_BF16, ARD_F32, T * B, KH, H, 1.0f, XH, KH, dz + (size_t)g * H, 4 * H,
+                                   1, dW + (size_t)g * H * KH, KH, 1, cuda_stream);
+    if (st != ARD_OK) return st;
+  }
+  return ARD_OK;
 }
 
 ard_status ard_last_device_status(ard_ctx* ctx, void* cuda_stream) {

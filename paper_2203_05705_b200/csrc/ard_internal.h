@@ -56,6 +56,7 @@ struct MapTable {
   int dp_bound;
   CUtensorMap* d_maps;
   int count;
+  unsigned long long epoch;  // public call that last used the table (tables of the running call are never evicted)
 };
 
 enum MapVariant {
@@ -79,6 +80,7 @@ struct ard_ctx {
   ArdDistribution dist[ARD_MAX_DISTRIBUTIONS];
   std::vector<MapTable> maps;
   unsigned long long launches;
+  unsigned long long epoch;   // bumped by every public GEMM call
   void* encode_fn;  // cuTensorMapEncodeTiled, resolved at run time
 };
 
@@ -121,6 +123,8 @@ ard_status launch_gemm_cc(ard_ctx* ctx, ard_kind kind, GemmOp op, ard_dtype dtyp
 struct TcArgs {
   const CUtensorMap* mapA;  // table or single descriptor
   const CUtensorMap* mapB;
+  const CUtensorMap* mapA4[4];  // LSTM gate products: one table per gate
+  const CUtensorMap* mapB4[4];
   int mapA_indexed, mapB_indexed;
   GemmArgs g;
   int ts;
@@ -128,6 +132,7 @@ struct TcArgs {
 };
 int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int dp_bound, int ts);
 ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s);
+ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStream_t s);
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,
                               void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, int skip_dense,

@@ -41,22 +41,28 @@ enum TcMode {
   // over gathered 64-wide blocks; these modes build 256-wide output tiles from such blocks.
   M_TILEC_FWD = 6,
   M_TILEC_BWD_DATA = 7,
-  M_TILEC_BWD_WEIGHT = 8
+  M_TILEC_BWD_WEIGHT = 8,
+  // LSTM gate products over the four gate blocks i|f|g|o of one weight in a single launch: the kept
+  // units of gate g are the rows g*H + keep[j] of W, reached through one descriptor table per gate.
+  M_LSTM_FWD = 9,       // Z[:, g*ldz + j] = [x,h] . W[g*H + keep[j], :]
+  M_LSTM_BWD_DATA = 10  // d[x,h] = sum_g dZ[:, g*ldz + j] . W[g*H + keep[j], :]
 };
 
 __host__ __device__ constexpr bool a_is_mn(int mode) {
   return mode == M_ROW_BWD_WEIGHT || mode == M_TILE_BWD_WEIGHT || mode == M_TILEC_BWD_WEIGHT;
 }
 __host__ __device__ constexpr bool b_is_mn(int mode) {
-  return mode != M_ROW_FWD && mode != M_TILE_FWD && mode != M_TILEC_FWD;
+  return mode != M_ROW_FWD && mode != M_TILE_FWD && mode != M_TILEC_FWD && mode != M_LSTM_FWD;
 }
-__host__ __device__ constexpr bool is_class_mode(int mode) { return mode >= M_TILEC_FWD; }
+__host__ __device__ constexpr bool is_class_mode(int mode) { return mode >= M_TILEC_FWD && mode <= M_TILEC_BWD_WEIGHT; }
 __host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 4 : (bn == 128 ? 6 : 8); }
 __host__ __device__ constexpr int tmem_cols_for(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }
 
 struct TcParams {
   const CUtensorMap* mapA;
   const CUtensorMap* mapB;
+  const CUtensorMap* mapA4[4];  // LSTM modes: one table per gate
+  const CUtensorMap* mapB4[4];
   int mapA_indexed, mapB_indexed;
   const int32_t* hdr;
   const int32_t* idx;
@@ -310,6 +316,8 @@ struct Sched {
     subm = subn = 1;
     if (MODE == M_ROW_FWD) { M_gemm = p.B; N_gemm = n_keep; Kc = p.K; }
     else if (MODE == M_ROW_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = n_keep; }
+    else if (MODE == M_LSTM_FWD) { M_gemm = p.B; N_gemm = ((n_keep + 63) / 64) * 256; Kc = p.K; }
+    else if (MODE == M_LSTM_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 4 * (((n_keep + 63) / 64) * 64); }
     else if (MODE == M_ROW_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = p.K; Kc = p.B; }
     else if (MODE == M_TILE_FWD || MODE == M_TILEC_FWD) { M_gemm = p.B; N_gemm = p.N; Kc = 0; }
     else if (MODE == M_TILE_BWD_DATA || MODE == M_TILEC_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 0; }
@@ -343,7 +351,7 @@ struct Sched {
       Nt = subn;
     } else {
       Mt = (M_gemm + BM * CTAS - 1) / (BM * CTAS);
-      if (MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA || MODE == M_ROW_BWD_WEIGHT) {
+      if (MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA || MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_DATA) {
         if (p.force_bn) {
           bn = p.force_bn;
         } else {
@@ -464,6 +472,16 @@ struct Sched {
     }
     ti.ax[0] = ti.m0; ti.ax[1] = ti.m0 + 64;
     ti.orow[0] = ti.orow[1] = 0;
+    if (MODE == M_LSTM_FWD) {
+      // N tile = the same 64 kept units of all four gates; p.ts carries the gate block width of Z
+      const int j0 = ti.n0 / 4;
+      ti.n0 = j0;
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        ti.bx[g] = j0;
+        ti.ocol[g] = g * p.ts + j0;
+      }
+    }
     return ti;
   }
 
@@ -653,6 +671,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       const CUtensorMap* mapB = p.mapB + (p.mapB_indexed ? e : 0);
       tensormap_acquire(mapA);
       tensormap_acquire(mapB);
+      if (MODE == M_LSTM_FWD || MODE == M_LSTM_BWD_DATA) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          tensormap_acquire(p.mapB4[g] + e);
+          if (MODE == M_LSTM_BWD_DATA) tensormap_acquire(p.mapA4[g] + e);
+        }
+      }
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -685,7 +710,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
           } else {
             kx = kb * BK;
           }
-          if (!A_MN) {
+          const CUtensorMap* mapBk = mapB;
+          if (MODE == M_LSTM_BWD_DATA) {
+            // contraction runs gate by gate over the kept units: block kb = (gate, 64 kept units)
+            const int nkg = ti.nkb >> 2;
+            const int g = kb / nkg;
+            kx = (kb - g * nkg) * BK;
+            mapBk = p.mapB4[g] + e;
+            load(sA, p.mapA4[g] + e, kx, ti.m0);
+          } else if (!A_MN) {
             load(sA, mapA, kx, ti.m0);  // [BM rows][64 k]
           } else {
 #pragma unroll
@@ -697,8 +730,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             if (i < ti.nbox) {
-              if (!B_MN) load(sB + i * (64 * BK * 2), mapB, kx, ti.bx[i]);
-              else load(sB + i * (64 * BK * 2), mapB, ti.bx[i], kx);
+              if (MODE == M_LSTM_FWD) load(sB + i * (64 * BK * 2), p.mapB4[i] + e, kx, ti.bx[i]);
+              else if (!B_MN) load(sB + i * (64 * BK * 2), mapBk, kx, ti.bx[i]);
+              else load(sB + i * (64 * BK * 2), mapBk, ti.bx[i], kx);
             }
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -863,7 +897,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
             __syncwarp();
           }
         } else {
-          const int nvalid = is_class_mode(MODE) ? 32 : min(32, sch.N_gemm - n);
+          const int nvalid = is_class_mode(MODE) ? 32
+                             : (MODE == M_LSTM_FWD ? min(32, sch.n_keep - (ti.n0 + (ch & 1) * 32))
+                                                   : min(32, sch.N_gemm - n));
           if (row_ok && nvalid > 0) {
             store_row32(p.out, (size_t)out_row * p.ldo, n, v, nvalid, p.out_is_f32, p.accumulate);
             if (MODE == M_ROW_BWD_WEIGHT && p.zero_fill) {
@@ -1062,4 +1098,34 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
 #undef ARD_TC_CASE
 #undef ARD_TC_PAIR
   return ARD_ERR_UNSUPPORTED;
+}
+
+// LSTM gate products (single CTA per tile; the batch of a recurrent step is small).
+ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStream_t s) {
+  TcParams p;
+  p.mapA = a.mapA;
+  p.mapB = a.mapB;
+  for (int g = 0; g < 4; ++g) { p.mapA4[g] = a.mapA4[g]; p.mapB4[g] = a.mapB4[g]; }
+  p.mapA_indexed = a.mapA_indexed;
+  p.mapB_indexed = a.mapB_indexed;
+  p.hdr = a.g.hdr;
+  p.idx = a.g.idx;
+  p.col_ptr = p.col_idx = p.row_ptr = p.row_idx = nullptr;
+  p.B = a.g.B;
+  p.K = a.g.K;
+  p.N = a.g.N;
+  p.ts = a.ts;  // forward: gate block width of Z
+  p.alpha = a.g.alpha;
+  p.out = a.g.out;
+  p.ldo = a.g.ldo;
+  p.out_is_f32 = a.g.out_is_f32;
+  p.scatter = 0;
+  p.zero_fill = 0;
+  p.status = a.g.status;
+  p.force_bn = a.bn;
+  p.accumulate = a.g.accumulate;
+  p.band_m = 0;
+  const int mt = cdiv(p.B, BM);
+  if (!backward) return launch_mode<256, M_LSTM_FWD, 1>(ctx, p, mt * cdiv(p.N, 64), s);
+  return launch_mode<256, M_LSTM_BWD_DATA, 1>(ctx, p, mt * cdiv(p.K, 64), s);
 }

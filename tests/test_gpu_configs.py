@@ -148,46 +148,15 @@ def test_config5_sampled_outputs(kind, ts):
 
 # --------------------------------------------------------------------------------------------------
 def _lstm_gpu(ctx, pat, Wnm, X, dH, I, H, alpha):
-    """LSTM layer forward + BPTT composed from C-ABI calls only (torch: buffers, copies of inputs)."""
+    """LSTM layer forward + BPTT through the C ABI (buffers and call order: paper_2203_05705_b200/lstm.py)."""
+    from paper_2203_05705_b200.lstm import LstmLayer
     T, B, _ = X.shape
-    KH = I + H
-    XH = torch.zeros((T + 1, B, KH), dtype=BF, device="cuda")
-    XH[:T, :, :I] = X
-    C = torch.zeros((T + 1, B, H), dtype=torch.float32, device="cuda")
-    G = torch.zeros((T, B, 4 * H), dtype=torch.float32, device="cuda")
-    Z = torch.zeros((B, 4 * H), dtype=torch.float32, device="cuda")
-    zp, wp = Z.data_ptr(), Wnm.data_ptr()
-    f32c = ard.ARD_OUT_COMPACT | ard.ARD_FLAG_OUT_F32
-    for t in range(T):
-        for g in range(4):       # gate pre-activations of the kept units: [x_t, h_{t-1}] . W[:, gate g, keep]
-            ard.ard_fwd(ctx.h, pat, ard.ARD_BF16, B, KH, H, 1.0, XH[t], KH, wp + g * H * KH * 2, KH,
-                        zp + g * H * 4, 4 * H, f32c)
-        ard.ard_lstm_gates(ctx.h, pat, ard.ARD_BF16, B, H, alpha, Z, H, None, C[t], H, C[t + 1],
-                           XH[t + 1].data_ptr() + I * 2, KH, 1, G[t])
-    Hs = XH[1:, :, I:].float()
-    # ---- BPTT ----
-    DZ = torch.zeros((T, B, 4 * H), dtype=BF, device="cuda")
-    D = torch.zeros((T, B, KH), dtype=torch.float32, device="cuda")     # [dx_t | total dh_{t-1}]
-    D[1:, :, I:] = dH[:-1]                                              # upstream dH_{t-1}, bwd-data adds to it
-    dc = torch.zeros((B, H), dtype=torch.float32, device="cuda")
-    dh_last = dH[T - 1].contiguous()
-    accf = 1 | ard.ARD_FLAG_OUT_F32 | ard.ARD_FLAG_ACCUMULATE
-    for t in reversed(range(T)):
-        if t == T - 1:
-            dh_ptr, lddh = dh_last.data_ptr(), H
-        else:
-            dh_ptr, lddh = D[t + 1].data_ptr() + I * 4, KH
-        ard.ard_lstm_gates_bwd(ctx.h, pat, ard.ARD_BF16, B, H, alpha, G[t], C[t], C[t + 1], H, dh_ptr, lddh, 1,
-                               dc, DZ[t], H)
-        for g in range(4):
-            ard.ard_bwd_data(ctx.h, pat, ard.ARD_BF16, B, KH, H, 1.0, DZ[t].data_ptr() + g * H * 2, 4 * H, accf,
-                             wp + g * H * KH * 2, KH, D[t], KH)
-    dW = torch.full((4 * H, KH), float("nan"), dtype=torch.float32, device="cuda")
-    for g in range(4):           # one product over all T*B rows per gate
-        ard.ard_bwd_weight(ctx.h, pat, ard.ARD_BF16, ard.ARD_F32, T * B, KH, H, 1.0, XH[:T], KH,
-                           DZ.data_ptr() + g * H * 2, 4 * H, 1, dW.data_ptr() + g * H * KH * 4, KH, 1)
+    layer = LstmLayer(ctx.h, pat, T, B, I, H, Wnm)
+    layer.load_inputs(X)
+    Hs = layer.forward(alpha).float()
+    dX, dW = layer.backward(alpha, dH)
     torch.cuda.synchronize()
-    return Hs, C[T], D[:, :, :I], dW
+    return Hs, layer.C[T], dX, dW
 
 
 @pytest.mark.parametrize("p,seq", [(0.5, 0), (0.7, 1)])

@@ -160,3 +160,89 @@ def test_compact_reuse_option(ctx):
     finally:
         ard.ard_set_compact_reuse(ctx.h, 0)
         ard.ard_set_path(ctx.h, ard.ARD_PATH_AUTO)
+
+
+def test_output_flags_fp32_and_accumulate(ctx):
+    """ARD_FLAG_OUT_F32 / ARD_FLAG_ACCUMULATE on the tensor-core path (CTA pairs: more than 128 rows) and on the
+    CUDA-core family."""
+    import torch
+    from oracle import gemm as OG
+    from oracle import pattern as OP
+    B, K, N, dp, b = 300, 264, 520, 3, 2
+    X, W, dY = _layer(B, K, N, 21, 0.05)
+    keep = OP.row_keep(N, dp, b)
+    m = OP.row_mask(N, dp, b)
+    pat = ctx.pattern(ard.ARD_ROW, K, N)
+    ard.ard_pattern_set(ctx.h, pat, dp, b)
+    bf = torch.bfloat16
+    Xd = torch.from_numpy(X).to(bf).cuda()
+    Wd = torch.from_numpy(np.ascontiguousarray(W.T)).to(bf).cuda()
+    ldc = (len(keep) + 7) // 8 * 8                                        # 16-byte aligned rows for the TMA path
+    dYc = torch.full((B, ldc), float("nan"), dtype=bf, device="cuda")
+    dYc[:, :len(keep)] = torch.from_numpy(np.ascontiguousarray(dY[:, keep])).to(bf)
+    Yref = OG.fwd(X, W, m, 2.0)[:, keep]
+    dXref = OG.bwd_data(dY, W, m, 2.0)
+    for path in (ard.ARD_PATH_TENSOR_CORE, ard.ARD_PATH_CUDA_CORE):
+        ard.ard_set_path(ctx.h, path)
+        try:
+            Y = torch.full((B, N), 1.0, dtype=torch.float32, device="cuda")
+            ard.ard_fwd(ctx.h, pat, ard.ARD_BF16, B, K, N, 2.0, Xd, K, Wd, K, Y, N,
+                        ard.ARD_OUT_COMPACT | ard.ARD_FLAG_OUT_F32 | ard.ARD_FLAG_ACCUMULATE)
+            got = Y.double().cpu().numpy()
+            assert OG.rel_fro(got[:, :len(keep)] - 1.0, Yref) <= TOL[ard.ARD_BF16]
+            assert np.all(got[:, len(keep):] == 1.0)                       # columns beyond n_keep untouched
+            dX = torch.full((B, K), 0.5, dtype=torch.float32, device="cuda")
+            ard.ard_bwd_data(ctx.h, pat, ard.ARD_BF16, B, K, N, 2.0, dYc, ldc, 1 | ard.ARD_FLAG_OUT_F32, Wd, K,
+                             dX, K)
+            assert OG.rel_fro(dX.double().cpu().numpy(), dXref) <= TOL[ard.ARD_BF16]
+            ard.ard_bwd_data(ctx.h, pat, ard.ARD_BF16, B, K, N, 2.0, dYc, ldc,
+                             1 | ard.ARD_FLAG_OUT_F32 | ard.ARD_FLAG_ACCUMULATE, Wd, K, dX, K)
+            assert OG.rel_fro(dX.double().cpu().numpy(), 2.0 * dXref) <= TOL[ard.ARD_BF16]
+            with pytest.raises(ard.ArdError):                              # accumulate cannot be combined with zero fill
+                ard.ard_fwd(ctx.h, pat, ard.ARD_BF16, B, K, N, 2.0, Xd, K, Wd, K, Y, N,
+                            ard.ARD_OUT_SCATTER_ZEROFILL | ard.ARD_FLAG_ACCUMULATE)
+        finally:
+            ard.ard_set_path(ctx.h, ard.ARD_PATH_AUTO)
+    assert ard.ard_last_device_status(ctx.h) == 0
+
+
+def test_lstm_gate_products_against_per_gate_calls(ctx):
+    """ard_lstm_gate_gemm(_bwd): tensor-core single launch and the four-call fall-back agree with the oracle."""
+    import torch
+    from oracle import gemm as OG
+    from oracle import pattern as OP
+    B, I, H, dp, b = 40, 64, 136, 3, 1
+    KH = I + H
+    rng = np.random.default_rng(5)
+    XH = inputs.bf16_round(rng.standard_normal((B, KH)).astype(np.float32))
+    W = inputs.bf16_round((rng.standard_normal((KH, 4 * H)) * 0.1).astype(np.float32))     # math orientation
+    keep = OP.row_keep(H, dp, b)
+    n = len(keep)
+    dZ = inputs.bf16_round(rng.standard_normal((B, 4 * n)).astype(np.float32))
+    pat = ctx.pattern(ard.ARD_ROW, KH, H)
+    ard.ard_pattern_set(ctx.h, pat, dp, b)
+    bf = torch.bfloat16
+    XHd = torch.from_numpy(XH).to(bf).cuda()
+    Wd = torch.from_numpy(np.ascontiguousarray(W.T)).to(bf).cuda()
+    gcols = np.concatenate([g * H + keep for g in range(4)])
+    Zref = XH.astype(np.float64) @ W.astype(np.float64)[:, gcols]
+    dref = dZ.astype(np.float64) @ W.astype(np.float64)[:, gcols].T
+    for path in (ard.ARD_PATH_AUTO, ard.ARD_PATH_CUDA_CORE):
+        ard.ard_set_path(ctx.h, path)
+        try:
+            Z = torch.full((B, 4 * H), float("nan"), dtype=torch.float32, device="cuda")
+            ard.ard_lstm_gate_gemm(ctx.h, pat, B, KH, H, XHd, KH, Wd, KH, Z, H)
+            Zh = Z.double().cpu().numpy()
+            got = np.concatenate([Zh[:, g * H:g * H + n] for g in range(4)], axis=1)
+            assert OG.rel_fro(got, Zref) <= TOL[ard.ARD_BF16]
+            assert all(np.all(np.isnan(Zh[:, g * H + n:(g + 1) * H])) for g in range(4))
+            dZd = torch.zeros((B, 4 * H), dtype=bf, device="cuda")
+            for g in range(4):
+                dZd[:, g * H:g * H + n] = torch.from_numpy(dZ[:, g * n:(g + 1) * n]).to(bf)
+                dZd[:, g * H + n:(g + 1) * H] = float("nan")               # beyond n_keep: must not be read
+            D = torch.full((B, KH), 0.25, dtype=torch.float32, device="cuda")
+            ard.ard_lstm_gate_gemm_bwd(ctx.h, pat, B, KH, H, dZd, H, Wd, KH, D, KH, 1)
+            assert OG.rel_fro(D.double().cpu().numpy() - 0.25, dref) <= TOL[ard.ARD_BF16]
+        finally:
+            ard.ard_set_path(ctx.h, ard.ARD_PATH_AUTO)
+    assert ard.ard_last_device_status(ctx.h) == 0
