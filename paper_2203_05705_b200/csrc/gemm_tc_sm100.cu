@@ -305,6 +305,7 @@ struct Sched {
   const int32_t* list;     // kept-tile list the class modes walk (a shared-memory copy when it fits)
   const int4* ctab;        // per class {first item, list offset, list length, members} (shared memory)
   int qn, qm;              // pattern tiles per output tile along N and along M
+  int lts;                 // log2 of the pattern tile size (64, 128 or 256 in the class modes)
 
   __device__ void init(const TcParams& p, int rank_) {
     rank = rank_;
@@ -327,6 +328,7 @@ struct Sched {
     nclass = cstep = qn = qm = 1;
     list = (MODE == M_TILEC_BWD_DATA) ? p.row_idx : p.col_idx;
     ctab = nullptr;
+    lts = 31 - __clz(p.ts > 0 ? p.ts : 1);
     if (is_class_mode(MODE)) {
       qn = BN / p.ts;
       qm = (BM * CTAS) / p.ts;
@@ -396,16 +398,17 @@ struct Sched {
   __device__ TileInfo class_tile(const TcParams& p, int t) const {
     TileInfo ti;
     ti.klist = nullptr;
-    ti.kper = p.ts / BK;
+    ti.kper = p.ts >> 6;
     ti.out_row0 = 0;
     ti.rows_valid = BM;
     ti.n0 = 0;
+    const int tmask = p.ts - 1;   // the pattern tile size is a power of two here
     int c = nclass - 1;
     while (c > 0 && ctab[c].x > t) --c;  // class whose item range holds t
     const int4 ce = ctab[c];
     t -= ce.x;
     const int cnt = ce.w;
-    const int sub64 = p.ts / 64;  // 64-wide boxes per pattern tile
+    const int lsub = lts - 6;     // log2 of the 64-wide boxes per pattern tile
     int nm;                       // pattern tiles along N in this output tile
     if (MODE == M_TILEC_BWD_WEIGHT) {
       const int32_t* rlist = list + ce.y;
@@ -417,18 +420,18 @@ struct Sched {
 #pragma unroll
       for (int k = 0; k < 2; ++k) {  // this CTA's two 64-row boxes of gathered neurons
         const int row = rank * BM + 64 * k;
-        const int mem = mi * qm + row / p.ts;
-        const int coord = (mem < cnt) ? (c + mem * cstep) * p.ts + (row % p.ts) : -1;
+        const int mem = mi * qm + (row >> lts);
+        const int coord = (mem < cnt) ? (((c + mem * cstep) << lts) + (row & tmask)) : -1;
         ti.orow[k] = coord;
         ti.ax[k] = coord >= 0 ? coord : p.N;  // beyond the matrix: TMA fills zeros
       }
       const int j0 = ni * qn;
       nm = min(qn, rn - j0);
-      ti.bn = (nm * p.ts + 64 * CTAS - 1) / (64 * CTAS) * (64 * CTAS);
+      ti.bn = ((nm << lts) + 64 * CTAS - 1) / (64 * CTAS) * (64 * CTAS);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const int mem = j / sub64;
-        ti.ocol[j] = (mem < nm) ? rlist[j0 + mem] * p.ts + (j % sub64) * 64 : -1;
+        const int mem = j >> lsub;
+        ti.ocol[j] = (mem < nm) ? ((rlist[j0 + mem] << lts) + ((j & ((1 << lsub) - 1)) << 6)) : -1;
       }
     } else {
       const int ntiles = (cnt + qn - 1) / qn;
@@ -439,11 +442,11 @@ struct Sched {
       ti.orow[0] = ti.orow[1] = 0;
       const int i0 = v * qn;
       nm = min(qn, cnt - i0);
-      ti.bn = (nm * p.ts + 64 * CTAS - 1) / (64 * CTAS) * (64 * CTAS);
+      ti.bn = ((nm << lts) + 64 * CTAS - 1) / (64 * CTAS) * (64 * CTAS);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const int mem = j / sub64;
-        ti.ocol[j] = (mem < nm) ? (c + (i0 + mem) * cstep) * p.ts + (j % sub64) * 64 : -1;
+        const int mem = j >> lsub;
+        ti.ocol[j] = (mem < nm) ? (((c + (i0 + mem) * cstep) << lts) + ((j & ((1 << lsub) - 1)) << 6)) : -1;
       }
       ti.klist = list + ce.y;
       ti.nkb = ce.z * ti.kper;
