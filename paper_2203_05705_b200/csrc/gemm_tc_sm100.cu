@@ -306,6 +306,7 @@ struct Sched {
   const int4* ctab;        // per class {first item, list offset, list length, members} (shared memory)
   int qn, qm;              // pattern tiles per output tile along N and along M
   int lts;                 // log2 of the pattern tile size (64, 128 or 256 in the class modes)
+  bool dense;              // class modes with dp = 1: nothing is dropped, plain dense tiling
 
   __device__ void init(const TcParams& p, int rank_) {
     rank = rank_;
@@ -329,6 +330,15 @@ struct Sched {
     list = (MODE == M_TILEC_BWD_DATA) ? p.row_idx : p.col_idx;
     ctab = nullptr;
     lts = 31 - __clz(p.ts > 0 ? p.ts : 1);
+    dense = is_class_mode(MODE) && dp == 1;
+    if (dense) {
+      // every tile is kept: the contraction runs over the whole operand
+      Kc = (MODE == M_TILEC_FWD) ? p.K : (MODE == M_TILEC_BWD_DATA ? p.N : p.B);
+      Mt = (M_gemm + BM * CTAS - 1) / (BM * CTAS);
+      Nt = (N_gemm + bn - 1) / bn;
+      total = Mt * Nt;
+      return;
+    }
     if (is_class_mode(MODE)) {
       qn = BN / p.ts;
       qm = (BM * CTAS) / p.ts;
@@ -463,7 +473,7 @@ struct Sched {
   }
 
   __device__ TileInfo tile(const TcParams& p, int t) const {
-    if (is_class_mode(MODE)) return class_tile(p, t);
+    if (is_class_mode(MODE) && !dense) return class_tile(p, t);
     TileInfo ti = plain_tile(p, t);
     // affine block coordinates
     ti.bn = bn;
@@ -474,7 +484,7 @@ struct Sched {
       ti.ocol[i] = ti.n0 + 64 * i;
     }
     ti.ax[0] = ti.m0; ti.ax[1] = ti.m0 + 64;
-    ti.orow[0] = ti.orow[1] = 0;
+    ti.orow[0] = ti.m0; ti.orow[1] = ti.m0 + 64;
     if (MODE == M_LSTM_FWD) {
       // N tile = the same 64 kept units of all four gates; p.ts carries the gate block width of Z
       const int j0 = ti.n0 / 4;
@@ -646,7 +656,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
 
   Sched<BN, MODE, CTAS> sch;
   sch.init(p, (int)rank);
-  if (is_class_mode(MODE)) {
+  if (is_class_mode(MODE) && !sch.dense) {
     // The producer reads one list entry per contraction block: keep the list in shared memory (the
     // staging area of the forward scatter epilogue is free in these modes) instead of paying a
     // global-memory round trip on its critical path.
@@ -818,8 +828,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         out_row = m;
       } else if (MODE == M_TILEC_BWD_WEIGHT) {
         const int orow = (row_in_tile >> 6) ? ti.orow[1] : ti.orow[0];
-        row_ok = orow >= 0;
         out_row = orow + (row_in_tile & 63);
+        row_ok = orow >= 0 && out_row < sch.M_gemm;
       } else {
         row_ok = m < sch.M_gemm;
         out_row = m;
@@ -900,7 +910,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
             __syncwarp();
           }
         } else {
-          const int nvalid = is_class_mode(MODE) ? 32
+          const int nvalid = (is_class_mode(MODE) && !sch.dense) ? 32
                              : (MODE == M_LSTM_FWD ? min(32, sch.n_keep - (ti.n0 + (ch & 1) * 32))
                                                    : min(32, sch.N_gemm - n));
           if (row_ok && nvalid > 0) {
