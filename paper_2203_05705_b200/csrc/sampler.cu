@@ -31,6 +31,7 @@ __device__ void philox4x32_10(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
 }
 
 constexpr int SAMPLER_THREADS = 256;
+constexpr int SCAN_CAP = 2048;  // tile-columns whose running count fits in shared memory
 
 __global__ void __launch_bounds__(SAMPLER_THREADS)
 ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t* __restrict__ col_ptr,
@@ -87,24 +88,33 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
     if (lim > b - 1) cnt = (int)((lim - 1 - (b - 1)) / dp) + 1;
     row_ptr[r] = cnt;
   }
-  // Group by tile-column: count, prefix-sum, fill.
+  // Group by tile-column: count, prefix-sum, fill.  The running sum lives in shared memory when the
+  // grid is narrow enough (one thread scans it; a dependent chain through global memory would cost
+  // a round trip per column).
+  __shared__ int s_cnt[SCAN_CAP];
+  const bool in_smem = Tc <= SCAN_CAP;
   for (int c = threadIdx.x; c < Tc; c += SAMPLER_THREADS) {
     int cnt = 0;
     for (int r = 0; r < Tr; ++r) cnt += ((r * Tc + c - (b - 1)) % dp == 0) && (r * Tc + c >= b - 1);
-    col_ptr[c + 1] = cnt;
+    if (in_smem) s_cnt[c] = cnt; else col_ptr[c + 1] = cnt;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
     int run = 0;
-    col_ptr[0] = 0;
-    for (int c = 0; c < Tc; ++c) {
-      run += col_ptr[c + 1];
-      col_ptr[c + 1] = run;
+    if (in_smem) {
+      for (int c = 0; c < Tc; ++c) { const int n = s_cnt[c]; s_cnt[c] = run; run += n; }
+    } else {
+      col_ptr[0] = 0;
+      for (int c = 0; c < Tc; ++c) { run += col_ptr[c + 1]; col_ptr[c + 1] = run; }
     }
   }
   __syncthreads();
+  if (in_smem) {
+    for (int c = threadIdx.x; c < Tc; c += SAMPLER_THREADS) col_ptr[c] = s_cnt[c];
+    if (threadIdx.x == 0) col_ptr[Tc] = n_keep;
+  }
   for (int c = threadIdx.x; c < Tc; c += SAMPLER_THREADS) {
-    int o = col_ptr[c];
+    int o = in_smem ? s_cnt[c] : col_ptr[c];
     for (int r = 0; r < Tr; ++r)
       if ((r * Tc + c >= b - 1) && ((r * Tc + c - (b - 1)) % dp == 0)) col_idx[o++] = r;
   }
