@@ -370,21 +370,25 @@ def main():
         dist_ids[pp] = i
     seed = inputs.BASE_SEED
 
+    # raw handles, looked up once: the per-call cost of the binding matters for the small workloads
+    cs = torch.cuda.current_stream().cuda_stream
+    pX, pW, pY, pdY, pdX, pdW = (t.data_ptr() for t in (X, W, Y, dY, dX, dW))
+
     def gemms(alpha, ev=None):
         if ev is not None:
             ev[0].record()
-        ard.ard_fwd(ctx, pat, ard.ARD_BF16, B, K, N, alpha, X, K, W, K, Y, N, ard.ARD_OUT_SCATTER_ZEROFILL)
+        ard.ard_fwd(ctx, pat, ard.ARD_BF16, B, K, N, alpha, pX, K, pW, K, pY, N, ard.ARD_OUT_SCATTER_ZEROFILL, cs)
         if ev is not None:
             ev[1].record()
-        ard.ard_bwd_data(ctx, pat, ard.ARD_BF16, B, K, N, alpha, dY, N, 0, W, K, dX, K)
+        ard.ard_bwd_data(ctx, pat, ard.ARD_BF16, B, K, N, alpha, pdY, N, 0, pW, K, pdX, K, cs)
         if ev is not None:
             ev[2].record()
-        ard.ard_bwd_weight(ctx, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, alpha, X, K, dY, N, 0, dW, K, 0)
+        ard.ard_bwd_weight(ctx, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, alpha, pX, K, pdY, N, 0, pdW, K, 0, cs)
         if ev is not None:
             ev[3].record()
 
     def step(pp, it, ev=None):
-        ard.ard_sample_pattern(ctx, pat, dist_ids[pp], seed, it, rank)
+        ard.ard_sample_pattern(ctx, pat, dist_ids[pp], seed, it, rank, cs)
         gemms(1.0 / (1.0 - pp), ev)
 
     def kept_units_of(pp, its):

@@ -19,11 +19,16 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 struct DeviceGuard {
   int prev = -1;
   bool ok;
+  bool switched = false;
   explicit DeviceGuard(int dev) {
-    ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess;
+    ok = cudaGetDevice(&prev) == cudaSuccess;
+    if (ok && prev != dev) {  // the usual case needs no switch at all
+      ok = cudaSetDevice(dev) == cudaSuccess;
+      switched = ok;
+    }
   }
   ~DeviceGuard() {
-    if (prev >= 0) cudaSetDevice(prev);
+    if (switched) cudaSetDevice(prev);
   }
 };
 
