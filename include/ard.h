@@ -96,6 +96,9 @@ ard_status ard_set_tile_n(ard_ctx* ctx, int bn);
  * distribution the sampler realises exactly.  Synchronous (small copy).  dist_id in
  * [0, ARD_MAX_DISTRIBUTIONS). */
 ard_status ard_set_distribution(ard_ctx* ctx, int dist_id, const double* K, int ndp);
+/* The quantisation alone, on the host (no context or GPU needed): validates K as above and writes the
+ * ndp cumulative entries to cdf_out (HOST uint64). */
+ard_status ard_quantise_distribution(const double* K, int ndp, uint64_t* cdf_out);
 /* Copies the quantised cumulative table (ndp entries, HOST uint64) back, for tests. */
 ard_status ard_get_distribution_cdf(ard_ctx* ctx, int dist_id, uint64_t* cdf_out, int capacity, int* ndp_out);
 

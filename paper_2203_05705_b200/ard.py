@@ -27,7 +27,7 @@ ARD_PATH_AUTO, ARD_PATH_CUDA_CORE, ARD_PATH_TENSOR_CORE = 0, 1, 2
 ARD_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = [
-    "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_compact_reuse", "ard_set_distribution", "ard_get_distribution_cdf",
+    "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_compact_reuse", "ard_set_distribution", "ard_quantise_distribution", "ard_get_distribution_cdf",
     "ard_pattern_create", "ard_pattern_destroy", "ard_sample_pattern", "ard_pattern_set",
     "ard_pattern_to_host", "ard_pattern_tile_lists_to_host", "ard_fwd", "ard_bwd_data", "ard_bwd_weight",
     "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_lstm_forward", "ard_lstm_backward", "ard_last_device_status", "ard_status_string", "ard_launch_count",
@@ -60,6 +60,7 @@ def lib():
         "ard_set_tile_n": [vp, i32],
         "ard_set_compact_reuse": [vp, i32],
         "ard_set_distribution": [vp, i32, P(C.c_double), i32],
+        "ard_quantise_distribution": [P(C.c_double), i32, P(u64)],
         "ard_get_distribution_cdf": [vp, i32, P(u64), i32, P(i32)],
         "ard_pattern_create": [vp, P(vp), i32, i32, i32, i32],
         "ard_pattern_destroy": [vp],
@@ -139,6 +140,15 @@ def ard_set_distribution(ctx, dist_id, K):
     K = np.ascontiguousarray(K, dtype=np.float64)
     _check(lib().ard_set_distribution(ctx, dist_id, K.ctypes.data_as(C.POINTER(C.c_double)), len(K)),
            "ard_set_distribution")
+
+
+def ard_quantise_distribution(K):
+    """Host-only: the integer cumulative table of K (no GPU needed)."""
+    K = np.ascontiguousarray(K, dtype=np.float64)
+    out = np.zeros(max(len(K), 1), dtype=np.uint64)
+    _check(lib().ard_quantise_distribution(K.ctypes.data_as(C.POINTER(C.c_double)), len(K),
+                                           out.ctypes.data_as(C.POINTER(C.c_uint64))), "ard_quantise_distribution")
+    return out[:len(K)]
 
 
 def ard_get_distribution_cdf(ctx, dist_id):

@@ -250,9 +250,9 @@ ard_status ard_set_tile_n(ard_ctx* ctx, int bn) {
   return ARD_OK;
 }
 
-ard_status ard_set_distribution(ard_ctx* ctx, int dist_id, const double* K, int ndp) {
-  if (!ctx || !K) return ARD_ERR_INVALID_ARG;
-  if (dist_id < 0 || dist_id >= ARD_MAX_DISTRIBUTIONS) return ARD_ERR_INVALID_ARG;
+// Host-only: validates K and writes its integer cumulative table (no context, no GPU needed).
+ard_status ard_quantise_distribution(const double* K, int ndp, uint64_t* cdf_out) {
+  if (!K || !cdf_out) return ARD_ERR_INVALID_ARG;
   if (ndp < 1 || ndp > ARD_MAX_NDP) return ARD_ERR_DISTRIBUTION;
   double sum = 0.0;
   for (int i = 0; i < ndp; ++i) {
@@ -261,7 +261,6 @@ ard_status ard_set_distribution(ard_ctx* ctx, int dist_id, const double* K, int 
   }
   if (!(fabs(sum - 1.0) <= 1e-9)) return ARD_ERR_DISTRIBUTION;
   // Integer cumulative table on a 2^32 grid from sequential prefix sums.
-  std::vector<unsigned long long> cdf(ndp);
   const unsigned long long TOP = 1ull << 32;
   double s = 0.0;
   unsigned long long prev = 0;
@@ -275,8 +274,22 @@ ard_status ard_set_distribution(ard_ctx* ctx, int dist_id, const double* K, int 
       if (c < prev) c = prev;
       if (c > TOP) c = TOP;
     }
-    cdf[i] = c;
+    cdf_out[i] = c;
     prev = c;
+  }
+  return ARD_OK;
+}
+
+ard_status ard_set_distribution(ard_ctx* ctx, int dist_id, const double* K, int ndp) {
+  if (!ctx || !K) return ARD_ERR_INVALID_ARG;
+  if (dist_id < 0 || dist_id >= ARD_MAX_DISTRIBUTIONS) return ARD_ERR_INVALID_ARG;
+  if (ndp < 1 || ndp > ARD_MAX_NDP) return ARD_ERR_DISTRIBUTION;
+  std::vector<unsigned long long> cdf(ndp);
+  {
+    std::vector<uint64_t> tmp(ndp);
+    ard_status qs = ard_quantise_distribution(K, ndp, tmp.data());
+    if (qs != ARD_OK) return qs;
+    for (int i = 0; i < ndp; ++i) cdf[i] = tmp[i];
   }
   DeviceGuard guard(ctx->device);
   ArdDistribution& d = ctx->dist[dist_id];

@@ -21,7 +21,7 @@ def _declared():
     return sorted(set(re.findall(r"\b(ard_[a-z0-9_]+)\s*\(", text)))
 
 
-def test_header_declares_the_north_star_entry_points():
+def test_header_declares_the_required_entry_points():
     names = _declared()
     for must in ["ard_sample_pattern", "ard_fwd", "ard_bwd_data", "ard_bwd_weight", "ard_lstm_gates"]:
         assert must in names
@@ -65,3 +65,22 @@ def test_package_does_not_import_the_oracle():
         if fn.endswith(".py"):
             with open(os.path.join(ROOT, "oracle", fn)) as f:
                 assert "paper_2203_05705_b200" not in f.read(), fn
+
+
+def test_host_side_quantiser_matches_the_oracle(built):
+    """The library's host logic that needs no GPU: K -> integer cumulative table, and its rejections."""
+    import numpy as np
+    from oracle import pattern as OP
+    from paper_2203_05705_b200 import ard, inputs
+    cases = [inputs.max_entropy_K(p, n) for p, n in [(0.3, 16), (0.5, 16), (0.7, 16), (0.5, 8), (0.9, 64)]]
+    cases += [[1.0], [0.25, 0.0, 0.5, 0.0, 0.25], [0.0, 0.0, 1.0], [1e-12, 1.0 - 1e-12]]
+    rng = np.random.default_rng(0)
+    for _ in range(20):
+        k = rng.random(rng.integers(2, 40)) ** 3
+        cases.append(k / k.sum())
+    for K in cases:
+        assert ard.ard_quantise_distribution(K).tolist() == OP.quantise_K(K)
+    for bad in ([0.5, 0.4], [1.5, -0.5], [float("nan"), 1.0], []):
+        with pytest.raises(ard.ArdError) as e:
+            ard.ard_quantise_distribution(bad)
+        assert e.value.status == ard.ARD_ERR_DISTRIBUTION
