@@ -19,6 +19,9 @@
  *   - The library allocates device memory only in ard_create, ard_pattern_create and (once per new
  *     combination of operand pointer and shape) when it builds and caches TMA descriptor tables
  *     for the bf16 tensor-core path; everything is freed by the matching destroy call.
+ *   - A context's scratch memory and status word are shared by its calls: work enqueued through one
+ *     context must be ordered (one stream, or streams ordered by events).  Use one context per
+ *     concurrently running stream.
  *   - Every call returns an ard_status.  Problems the host can see (NULL, sizes, leading
  *     dimensions, alignment, distribution) are rejected before anything is launched.  Problems only
  *     the device can see (a wait inside a kernel that ran out of patience) set a sticky device
@@ -88,6 +91,19 @@ ard_status ard_set_compact_reuse(ard_ctx* ctx, int enable);
 /* Tuning / test knob of the tensor-core path: forces the N extent of the output tile (64, 128 or
  * 256; 0 restores the built-in choice).  A forced value a product cannot use is ignored for it. */
 ard_status ard_set_tile_n(ard_ctx* ctx, int bn);
+/* Optional schedule of the tensor-core path for row patterns.  The output tiles of a product are
+ * dealt to the SMs (or SM pairs) in waves.  With enable != 0, when the tile count leaves a partial
+ * wave after at least one complete wave, the left-over tiles are computed first, cut along the
+ * contraction dimension and shared by all workers, which park fp32 partial sums in context
+ * scratch; the share that arrives last adds them in contraction order (so the result does not
+ * depend on the arrival order and is the same from launch to launch) and writes the tile.
+ * min_blocks: fewest 64-wide contraction blocks worth a separate share (default 16).
+ * min_gain_blocks: used only if it shortens the work of every worker by at least this many blocks
+ * (default 24).  0 keeps the current value of either.
+ * Default: disabled.  On a B200 the parked partial sums and the later start of the shared tiles'
+ * epilogues cost about what the better balance saves (a few percent either way, depending on the
+ * period), and the forward product with zero fill gets slower. */
+ard_status ard_set_shared_tail(ard_ctx* ctx, int enable, int min_blocks, int min_gain_blocks);
 
 /* Sec. 3.3: the distribution K = {k_i}, i = 1..ndp, over the periods dp, sum k_i = 1.
  * K: HOST array of ndp doubles, k_i >= 0, |sum - 1| <= 1e-9, 1 <= ndp <= ARD_MAX_NDP.

@@ -190,6 +190,14 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   if (const char* e = getenv("ARD_USE_PAIRS")) ctx->use_pairs = atoi(e);
   if (const char* e = getenv("ARD_BAND_M")) ctx->band_m = atoi(e);
   ctx->reuse_compact = 0;
+  ctx->stream_k = 0;
+  ctx->sk_min_blocks = 16;
+  if (const char* e = getenv("ARD_STREAM_K")) ctx->stream_k = atoi(e);
+  ctx->sk_min_gain = 24;
+  if (const char* e = getenv("ARD_SK_MIN_BLOCKS")) ctx->sk_min_blocks = atoi(e) > 0 ? atoi(e) : 16;
+  if (const char* e = getenv("ARD_SK_MIN_GAIN")) ctx->sk_min_gain = atoi(e) > 0 ? atoi(e) : 24;
+  ctx->d_sk_ws = nullptr;
+  ctx->d_sk_cnt = nullptr;
   ctx->last_gather = {nullptr, 0, 0, 0, nullptr, 0ull, nullptr};
   ctx->workspace_bytes = workspace_bytes;
   ctx->d_workspace = nullptr;
@@ -214,6 +222,21 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
     delete ctx;
     return ARD_ERR_NOMEM;
   }
+  if (ctx->encode_fn != nullptr) {
+    // scratch of the tensor-core row kernels' shared tail
+    const size_t ws_bytes = sk_ws_bytes(ctx->sm_count);
+    const size_t cnt_bytes = sk_cnt_bytes(ctx->sm_count);
+    if (cudaMalloc(&ctx->d_sk_ws, ws_bytes) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&ctx->d_sk_cnt), cnt_bytes) != cudaSuccess ||
+        cudaMemset(ctx->d_sk_cnt, 0, cnt_bytes) != cudaSuccess) {
+      if (ctx->d_sk_ws) cudaFree(ctx->d_sk_ws);
+      if (ctx->d_sk_cnt) cudaFree(ctx->d_sk_cnt);
+      if (ctx->d_workspace) cudaFree(ctx->d_workspace);
+      cudaFree(ctx->d_status);
+      delete ctx;
+      return ARD_ERR_NOMEM;
+    }
+  }
   *out = ctx;
   return ARD_OK;
 }
@@ -226,6 +249,8 @@ ard_status ard_destroy(ard_ctx* ctx) {
   for (int i = 0; i < ARD_MAX_DISTRIBUTIONS; ++i)
     if (ctx->dist[i].d_cdf) cudaFree(ctx->dist[i].d_cdf);
   if (ctx->d_workspace) cudaFree(ctx->d_workspace);
+  if (ctx->d_sk_ws) cudaFree(ctx->d_sk_ws);
+  if (ctx->d_sk_cnt) cudaFree(ctx->d_sk_cnt);
   if (ctx->d_status) cudaFree(ctx->d_status);
   delete ctx;
   return ARD_OK;
@@ -241,6 +266,14 @@ ard_status ard_set_compact_reuse(ard_ctx* ctx, int enable) {
   if (!ctx) return ARD_ERR_INVALID_ARG;
   ctx->reuse_compact = enable ? 1 : 0;
   ctx->last_gather.src = nullptr;
+  return ARD_OK;
+}
+
+ard_status ard_set_shared_tail(ard_ctx* ctx, int enable, int min_blocks, int min_gain_blocks) {
+  if (!ctx || min_blocks < 0 || min_gain_blocks < 0) return ARD_ERR_INVALID_ARG;
+  ctx->stream_k = enable ? 1 : 0;
+  if (min_blocks > 0) ctx->sk_min_blocks = min_blocks;
+  if (min_gain_blocks > 0) ctx->sk_min_gain = min_gain_blocks;
   return ARD_OK;
 }
 

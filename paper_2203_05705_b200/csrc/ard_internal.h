@@ -73,6 +73,11 @@ struct ard_ctx {
   int use_pairs;      // tensor-core row kernels: CTA pairs (cta_group::2) when the output has >= 2 row tiles
   int band_m;         // raster band height of the tensor-core kernels, in 128-row tiles
   int reuse_compact;  // opt-in: consecutive backward calls share one compacted dY
+  int stream_k;       // tensor-core row kernels: share the last, partial wave of tiles along the contraction
+  int sk_min_blocks;  // fewest 64-wide contraction blocks worth a separate share
+  int sk_min_gain;    // fewest blocks the sharing must save per worker to be used
+  void* d_sk_ws;      // partial accumulators of the shared tail, sk_ws_bytes(sm_count)
+  int* d_sk_cnt;      // arrival counters, zero between launches
   struct { const void* src; int ld, B, N; const ard_pattern* pat; unsigned long long gen; cudaStream_t stream; } last_gather;
   size_t workspace_bytes;
   void* d_workspace;
@@ -83,6 +88,12 @@ struct ard_ctx {
   unsigned long long epoch;   // bumped by every public GEMM call
   void* encode_fn;  // cuTensorMapEncodeTiled, resolved at run time
 };
+
+// Shared tail of the tensor-core row kernels: every CTA owns two slots, each holding the fp32 partial
+// sums of its 128 rows x 256 columns of a tile; one arrival counter per (tail tile, epilogue warp),
+// fewer tail tiles than CTAs, 8 epilogue warps per CTA.
+static inline size_t sk_ws_bytes(int sm_count) { return (size_t)sm_count * 2 * 128 * 256 * sizeof(float); }
+static inline size_t sk_cnt_bytes(int sm_count) { return (size_t)sm_count * 8 * sizeof(int); }
 
 static inline int map_index_count(int dp_bound) { return dp_bound * (dp_bound + 1) / 2; }
 

@@ -81,6 +81,14 @@ struct TcParams {
   int force_bn;   // row modes: 0 = choose the N tile on the device, else 64 / 128 / 256
   int accumulate; // plain stores add to the existing output
   int band_m;     // M-tiles per raster band (0: one band)
+  // Shared tiles (row modes): when the tile count is not a multiple of the worker count, the tiles
+  // that do not fill a wave are cut along the contraction and shared by all workers.  sk_ws holds the
+  // fp32 partial accumulators (two slots per worker), sk_cnt one arrival counter per (shared tile,
+  // epilogue warp).
+  float4* sk_ws;      // nullptr: every tile is computed by one worker
+  int* sk_cnt;
+  int sk_min_blocks;  // fewest contraction blocks worth a separate share
+  int sk_min_gain;    // fewest contraction blocks sharing must take off the last wave to be used
   int* status;
 };
 
@@ -275,6 +283,18 @@ __device__ __forceinline__ int sel4(const int (&a)[4], int i) {
   return i == 0 ? a[0] : (i == 1 ? a[1] : (i == 2 ? a[2] : a[3]));
 }
 
+// One piece of work of a CTA (pair): contraction blocks [kb0, kb1) of output tile t.
+struct Unit {
+  int t;
+  int kb0, kb1;    // kb1 < 0: the whole tile
+  int sk_tile;     // index of t among the shared tiles, -1 if this worker computes t alone
+  int slot;        // which of the worker's two partial slots this piece uses
+  int jfirst;      // first worker contributing to t
+  int nsplit;      // number of contributing workers
+};
+
+constexpr int SK_SLOT_F4 = 1024;  // float4 per (epilogue warp, partial): 32 rows x 128 columns of fp32
+
 // Tile schedule shared by the three roles.
 struct TileInfo {
   int m0, n0;      // origin in GEMM space
@@ -291,7 +311,7 @@ struct TileInfo {
   int orow[2];     // class bwd-weight: output row of each 64-row group of this CTA (-1: nothing to write)
 };
 
-template <int BN, int MODE, int CTAS = 1>
+template <int BN, int MODE, int CTAS = 1, bool SHARE = false>
 struct Sched {
   int dp, b, n_keep, Tc;
   int Mt, Nt, total;
@@ -307,6 +327,24 @@ struct Sched {
   int qn, qm;              // pattern tiles per output tile along N and along M
   int lts;                 // log2 of the pattern tile size (64, 128 or 256 in the class modes)
   bool dense;              // class modes with dp = 1: nothing is dropped, plain dense tiling
+  // shared tiles of the row modes
+  int KT;                  // contraction blocks per tile
+  int sk_tiles;            // tiles 0 .. sk_tiles-1 are shared along the contraction (0: none)
+  int sk_S;                // workers sharing them
+  int sk_blocks;           // their contraction blocks
+
+  // compiled in only for the row products launched with the sharing enabled
+  static constexpr bool SK_MODE = SHARE && (MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA || MODE == M_ROW_BWD_WEIGHT);
+
+  // Workers that would share the `rem` tiles left over by `full` complete waves (0: not worth it).
+  // The shared tiles are computed first, so that parking and adding their partial sums overlaps the
+  // contraction of the tiles that follow; without a complete wave there is nothing to hide behind.
+  __device__ static int sharing_workers(int full, int rem, int kt, int nworkers, int min_blocks, int min_gain) {
+    if (rem == 0 || full == 0) return 0;
+    const int S = min(nworkers, rem * kt / min_blocks);
+    if (S <= rem) return 0;
+    return kt - (rem * kt + S - 1) / S >= min_gain ? S : 0;
+  }
 
   __device__ void init(const TcParams& p, int rank_) {
     rank = rank_;
@@ -316,6 +354,7 @@ struct Sched {
     n_keep = p.hdr[HDR_NKEEP];
     Tc = p.hdr[HDR_TC];
     subm = subn = 1;
+    KT = sk_tiles = sk_S = sk_blocks = 0;
     if (MODE == M_ROW_FWD) { M_gemm = p.B; N_gemm = n_keep; Kc = p.K; }
     else if (MODE == M_ROW_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = n_keep; }
     else if (MODE == M_LSTM_FWD) { M_gemm = p.B; N_gemm = ((n_keep + 63) / 64) * 256; Kc = p.K; }
@@ -370,11 +409,18 @@ struct Sched {
           // Fewest (waves x time per tile).  Narrow tiles re-read the A operand more often and use
           // narrower instructions: a 128-wide tile is charged 0.7 and a 64-wide one 0.55 of the time of
           // a 256-wide tile (measured on dense problems).  Ties go to the wider tile.
+          // Shared tiles cost each worker its share of their contraction plus some of the reduction.
+          const int kt = (Kc + BK - 1) / BK;
           int best_cost = 0x7fffffff;
           for (int cand = BN; cand >= 64 * CTAS; cand >>= 1) {
             const int tiles = Mt * ((N_gemm + cand - 1) / cand);
-            const int waves = (tiles + workers - 1) / workers;
-            const int cost = waves * (cand == 256 ? 100 : (cand == 128 ? 70 : 55));
+            const int w16 = 16 * (cand == 256 ? 100 : (cand == 128 ? 70 : 55));
+            const int full = tiles / workers, rem = tiles % workers;
+            const int S = (SK_MODE && p.sk_ws != nullptr && kt > 0)
+                              ? sharing_workers(full, rem, kt, workers, p.sk_min_blocks, p.sk_min_gain) : 0;
+            int cost = full * w16;
+            if (S > 0) cost += (((rem * kt + S - 1) / S) + p.sk_min_gain / 2) * w16 / kt;
+            else if (rem > 0) cost += w16;
             if (cost < best_cost) { best_cost = cost; bn = cand; }
           }
         }
@@ -382,6 +428,50 @@ struct Sched {
       Nt = (N_gemm + bn - 1) / bn;
     }
     total = Mt * Nt;
+    KT = (Kc + BK - 1) / BK;
+    sk_tiles = sk_S = sk_blocks = 0;
+    if (SK_MODE && p.sk_ws != nullptr && KT > 0) {
+      const int rem = total % workers;
+      const int S = sharing_workers(total / workers, rem, KT, workers, p.sk_min_blocks, p.sk_min_gain);
+      if (S > 0) { sk_tiles = rem; sk_S = S; sk_blocks = rem * KT; }
+    }
+  }
+
+  // Worker whose share holds contraction block x of the shared tiles (shares start at
+  // floor(j * sk_blocks / sk_S)).
+  __device__ int share_worker_of(int x) const { return (int)((((long long)x + 1) * sk_S - 1) / sk_blocks); }
+  __device__ int share_start(int j) const { return (int)((long long)j * sk_blocks / sk_S); }
+
+  // i-th piece of work of worker w: first the one or two pieces of its share of the shared tiles
+  // 0 .. sk_tiles-1, then its own tiles sk_tiles + w, sk_tiles + w + workers, ...  Returns false when
+  // there is none.
+  __device__ bool unit(int w, int i, Unit& u) const {
+    u.sk_tile = -1;
+    u.slot = 0;
+    u.jfirst = w;
+    u.nsplit = 1;
+    int n_shared = 0;
+    if (SK_MODE && w < sk_S) {
+      const int r0 = share_start(w), r1 = share_start(w + 1);
+      const int tile0 = r0 / KT;
+      n_shared = (r1 > (tile0 + 1) * KT) ? 2 : 1;
+      if (i < n_shared) {
+        const int tile = tile0 + i;
+        const int lo = max(r0, tile * KT), hi = min(r1, (tile + 1) * KT);
+        u.t = tile;
+        u.kb0 = lo - tile * KT;
+        u.kb1 = hi - tile * KT;
+        u.jfirst = share_worker_of(tile * KT);
+        u.nsplit = share_worker_of((tile + 1) * KT - 1) - u.jfirst + 1;
+        if (u.nsplit > 1) { u.sk_tile = tile; u.slot = i; }
+        return true;
+      }
+    }
+    const int first = SK_MODE ? sk_tiles : 0;
+    u.t = first + w + (i - n_shared) * workers;
+    u.kb0 = 0;
+    u.kb1 = -1;
+    return u.t < total;
   }
 
   // ---- class modes ----
@@ -604,7 +694,7 @@ __device__ __forceinline__ void zero_row32(void* out, size_t row_off, int col, i
 }
 
 // ---- the kernel -----------------------------------------------------------------------------------
-template <int BN, int MODE, int CTAS>
+template <int BN, int MODE, int CTAS, bool SHARE>
 __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcParams p) {
   using L = SmemLayout<BN, CTAS>;
   const uint32_t rank = (CTAS == 2) ? cluster_ctarank() : 0u;  // rank 0 leads the pair and issues its MMAs
@@ -654,7 +744,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_smem;
 
-  Sched<BN, MODE, CTAS> sch;
+  Sched<BN, MODE, CTAS, SHARE> sch;
   sch.init(p, (int)rank);
   if (is_class_mode(MODE) && !sch.dense) {
     // The producer reads one list entry per contraction block: keep the list in shared memory (the
@@ -694,13 +784,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int t = w0; t < sch.total && ok; t += sch.workers) {
-        const TileInfo ti = sch.tile(p, t);
+      Unit un;
+      for (int i = 0; ok && sch.unit(w0, i, un); ++i) {
+        const TileInfo ti = sch.tile(p, un.t);
+        const int kb_begin = un.kb0, kb_end = un.kb1 < 0 ? ti.nkb : un.kb1;
         const uint32_t stage_tx = (uint32_t)(L::A_BYTES + ti.nbox * 64 * BK * 2) * CTAS;  // bytes of the whole pair
         // walk of the kept-block list: entry li, 64-wide piece `sub` of that pattern tile
         int li = 0, sub = 0;
         int kbase = (ti.klist != nullptr && ti.nkb > 0) ? ti.klist[0] * p.ts : 0;
-        for (int kb = 0; kb < ti.nkb; ++kb) {
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sA = base + stage * L::STAGE_BYTES;
           const uint32_t sB = sA + L::A_BYTES;
@@ -759,15 +851,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int t = w0; t < sch.total && ok; t += sch.workers, ++it) {
-        const TileInfo ti = sch.tile(p, t);
+      Unit un;
+      for (; ok && sch.unit(w0, it, un); ++it) {
+        const TileInfo ti = sch.tile(p, un.t);
+        const int kb_begin = un.kb0, kb_end = un.kb1 < 0 ? ti.nkb : un.kb1;
         const uint32_t idesc = make_idesc(ti.bn, A_MN, B_MN, BM * CTAS);
         const int acc = it & 1;
         const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < ti.nkb; ++kb) {
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sA = base + stage * L::STAGE_BYTES;
@@ -778,8 +872,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
             // MN-major: advance 16 k-rows = 2048 bytes.
             const uint64_t ad = A_MN ? make_desc(sA + s * 2048, 64 * BK * 2, 1024) : make_desc(sA + s * 32, 16, 1024);
             const uint64_t bd = B_MN ? make_desc(sB + s * 2048, 64 * BK * 2, 1024) : make_desc(sB + s * 32, 16, 1024);
-            if (CTAS == 2) tc_mma_bf16_pair(d_tmem, ad, bd, idesc, (kb | s) != 0 ? 1u : 0u);
-            else tc_mma_bf16(d_tmem, ad, bd, idesc, (kb | s) != 0 ? 1u : 0u);
+            const uint32_t accum = (kb != kb_begin || s != 0) ? 1u : 0u;
+            if (CTAS == 2) tc_mma_bf16_pair(d_tmem, ad, bd, idesc, accum);
+            else tc_mma_bf16(d_tmem, ad, bd, idesc, accum);
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if (CTAS == 2) tc_commit2(empty_bar(stage), (uint16_t)3);
@@ -788,10 +883,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         }
         if (!ok) break;
         if (CTAS == 2) {
-          if (ti.nkb > 0) tc_commit2(tfull_bar(acc), (uint16_t)3);
+          if (kb_end > kb_begin) tc_commit2(tfull_bar(acc), (uint16_t)3);
           else { mbar_arrive(tfull_bar(acc)); mbar_arrive_cluster(mapa_u32(tfull_bar(acc), 1u)); }
         } else {
-          if (ti.nkb > 0) tc_commit(tfull_bar(acc));
+          if (kb_end > kb_begin) tc_commit(tfull_bar(acc));
           else mbar_arrive(tfull_bar(acc));
         }
       }
@@ -806,8 +901,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
     const uint32_t magic_dp = (uint32_t)(0x100000000ull / (unsigned)dp) + 1u;  // exact x/dp for x < 2^16
     int it = 0;
     bool ok = true;
-    for (int t = w0; t < sch.total && ok; t += sch.workers, ++it) {
-      const TileInfo ti = sch.tile(p, t);
+    Unit un;
+    for (; ok && sch.unit(w0, it, un); ++it) {
+      const TileInfo ti = sch.tile(p, un.t);
+      const bool has_acc = (un.kb1 < 0 ? ti.nkb : un.kb1) > un.kb0;  // an empty contraction leaves zeros
       const int acc = it & 1;
       const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
@@ -842,68 +939,80 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         const int n = oc + (ch & 1) * 32;      // output column of this chunk
         float v[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = (ti.nkb > 0) ? p.alpha * __uint_as_float(r[i]) : 0.f;
+        for (int i = 0; i < 32; ++i) v[i] = has_acc ? p.alpha * __uint_as_float(r[i]) : 0.f;
 
         if (MODE == M_ROW_FWD && p.scatter && dp > 1) {
           // Full-width rows: compact column j -> column b-1 + j*dp, zeros everywhere else
-          // (Sec. 3.1: dropped outputs are zero).  The 32x32 block is staged through shared memory
-          // and the (row, 16-byte piece) pairs of the 32 x 32*dp output block are dealt to the lanes
-          // round-robin, so consecutive lanes write consecutive pieces of one output row.
+          // (Sec. 3.1: dropped outputs are zero).  The 32x32 block is staged through shared memory.
+          // The 32 x (32*dp) output block is written in 16-byte pieces; a lane keeps the same piece of
+          // the row (or, for narrow blocks, the same piece of a few rows) for the whole block, so where
+          // the kept columns fall inside its piece (Eq. 1) is worked out once and each row then costs
+          // a shared-memory read, a shift and one store.  Consecutive lanes write consecutive pieces.
           if (n < sch.n_keep) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) stg[lane * 33 + i] = v[i];
             __syncwarp();
+            const int nv = min(32, sch.n_keep - n);  // kept columns in this chunk
             const int cs = n * dp;
             const bool last = n + 32 >= sch.n_keep;
-            const int ce = last ? p.N : min((n + 32) * dp, p.N);
-            const int groups = (ce - cs + 7) >> 3;  // 16-byte pieces per output row
-            const uint32_t magic_g = (uint32_t)(0x100000000ull / (unsigned)groups) + 1u;
+            const int width = (last ? p.N : (n + 32) * dp) - cs;  // the last chunk also owns the dropped tail
+            const int G = (width + 7) >> 3;                        // 16-byte pieces per output row
             const int rows_here = min(32, sch.M_gemm - (ti.m0 + q * 32));
-            const int items = rows_here * groups;
             __nv_bfloat16* obase = reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)(ti.m0 + q * 32) * p.ldo + cs;
-            for (int w = lane; w < items; w += 32) {
-              const int rr = groups == 1 ? w : (int)__umulhi((uint32_t)w, magic_g);  // w / groups
-              const int g = w - rr * groups;
-              __nv_bfloat16* dst = obase + (size_t)rr * p.ldo + 8 * g;
-              // (compact column, remainder) of the piece's first column relative to column n*dp + b-1;
-              // a column is kept when the remainder is 0 (Eq. 1).
-              const int rel = 8 * g - bb;  // negative only before the first kept column
-              int cq, cr;
-              if (rel >= 0) { cq = (int)__umulhi((uint32_t)rel, magic_dp); cr = rel - cq * dp; }
-              else { cq = -1; cr = rel + dp; }
-              const int first_kept = cr == 0 ? 0 : dp - cr;  // position of the first kept column
-              const int nleft = ce - cs - 8 * g;
-              const float* srow = stg + rr * 33;
-              if (nleft >= 8) {
-                uint4 o = make_uint4(0u, 0u, 0u, 0u);
+            int rpp = 1, rsub = 0, g = lane, gstep = 32;  // rows per pass, this lane's row in a pass, its piece
+            if (G < 32) {
+              rpp = 32 / G;
+              rsub = lane / G;
+              g = lane - rsub * G;
+              gstep = G;
+              if (rsub >= rpp) g = G;  // no work for this lane
+            }
+            for (; g < G; g += gstep) {
+              // first kept column j0 (relative to n) at or after the piece's first column, and its
+              // position inside the piece; further kept columns follow dp positions apart
+              const int rel = 8 * g - bb;
+              int j0 = 0, pos0 = -rel;
+              if (rel > 0) {
+                j0 = (int)__umulhi((uint32_t)(rel + dp - 1), magic_dp);
+                pos0 = j0 * dp - rel;
+              }
+              const int nleft = width - 8 * g;  // < 8 only for the last piece of a ragged row
+              const float* src = stg + rsub * 33 + j0;
+              __nv_bfloat16* dst = obase + (size_t)rsub * p.ldo + 8 * g;
+              const size_t dstep = (size_t)rpp * p.ldo;
+              for (int rr = rsub; rr < rows_here; rr += rpp, src += rpp * 33, dst += dstep) {
+                uint32_t w0 = 0u, w1 = 0u, w2 = 0u, w3 = 0u;
                 if (dp >= 8) {
-                  // at most one kept column per piece
-                  if (first_kept < 8) {
-                    const uint32_t hbits = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(srow[cq + (cr != 0)]));
-                    const uint32_t u = hbits << ((first_kept & 1) * 16);
-                    const int wd = first_kept >> 1;
-                    o.x = wd == 0 ? u : 0u;
-                    o.y = wd == 1 ? u : 0u;
-                    o.z = wd == 2 ? u : 0u;
-                    o.w = wd == 3 ? u : 0u;
+                  if (pos0 < 8 && j0 < nv) {  // at most one kept column per piece
+                    const uint32_t u = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(src[0])) << ((pos0 & 1) * 16);
+                    const int wd = pos0 >> 1;
+                    w0 = wd == 0 ? u : 0u;
+                    w1 = wd == 1 ? u : 0u;
+                    w2 = wd == 2 ? u : 0u;
+                    w3 = wd == 3 ? u : 0u;
                   }
-                } else if (first_kept < 8) {
-                  float x[8];
+                } else {
 #pragma unroll
-                  for (int pos = 0; pos < 8; ++pos) {
-                    x[pos] = (cr == 0) ? srow[cq] : 0.f;
-                    if (++cr == dp) { cr = 0; ++cq; }
+                  for (int m = 0; m < 4; ++m) {
+                    const int pos = pos0 + m * dp;
+                    if (pos < 8 && j0 + m < nv) {
+                      const uint32_t u = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(src[m])) << ((pos & 1) * 16);
+                      const int wd = pos >> 1;
+                      w0 |= wd == 0 ? u : 0u;
+                      w1 |= wd == 1 ? u : 0u;
+                      w2 |= wd == 2 ? u : 0u;
+                      w3 |= wd == 3 ? u : 0u;
+                    }
                   }
-                  o = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]),
-                                 pack_bf16(x[6], x[7]));
                 }
-                *reinterpret_cast<uint4*>(dst) = o;
-              } else {
+                if (nleft >= 8) {
+                  *reinterpret_cast<uint4*>(dst) = make_uint4(w0, w1, w2, w3);
+                } else {
+                  const uint32_t w[4] = {w0, w1, w2, w3};
 #pragma unroll
-                for (int pos = 0; pos < 8; ++pos) {
-                  const float xv = (cr == 0) ? srow[cq] : 0.f;
-                  if (pos < nleft) dst[pos] = __float2bfloat16_rn(xv);
-                  if (++cr == dp) { cr = 0; ++cq; }
+                  for (int pos = 0; pos < 8; ++pos)
+                    if (pos < nleft)
+                      dst[pos] = __ushort_as_bfloat16((unsigned short)(w[pos >> 1] >> ((pos & 1) * 16)));
                 }
               }
             }
@@ -927,23 +1036,107 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         }
       };
 
-      // Software pipeline over this warp's chunks: the TMEM load of chunk i+1 is in flight while
-      // chunk i is converted and stored.
-      uint32_t ra[32], rb[32];
-      if (ti.nkb > 0 && ch_lo < ch_hi) tmem_ld32(t_row + (uint32_t)(ch_lo * 32), ra);
+      if (Sched<BN, MODE, CTAS, SHARE>::SK_MODE && un.sk_tile >= 0) {
+        // A share of a shared tile.  The raw fp32 partial sums are parked in global memory; the warp that
+        // arrives last for this 32-row block of the tile adds the shares in contraction order (so the
+        // result does not depend on who is last) and runs the normal epilogue.  Nobody waits.
+        constexpr int WSLOTS = EPI_WARPS * CTAS;
+        const int wslot = (int)rank * EPI_WARPS + (warp - 2);
+        float4* mine = p.sk_ws + (size_t)((w0 * 2 + un.slot) * WSLOTS + wslot) * SK_SLOT_F4 + lane;
+        uint32_t r[32];
 #pragma unroll 1
-      for (int ch = ch_lo; ch < ch_hi; ch += 2) {
-        if (ti.nkb > 0) {
+        for (int ch = ch_lo; ch < ch_hi; ++ch) {
+          tmem_ld32(t_row + (uint32_t)(ch * 32), r);
           tmem_ld_wait();
-          if (ch + 1 < ch_hi) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), rb);
+          float4* dst = mine + (ch - ch_lo) * 256;
+#pragma unroll
+          for (int q8 = 0; q8 < 8; ++q8)
+            __stcg(dst + q8 * 32, make_float4(__uint_as_float(r[4 * q8]), __uint_as_float(r[4 * q8 + 1]),
+                                              __uint_as_float(r[4 * q8 + 2]), __uint_as_float(r[4 * q8 + 3])));
         }
-        emit(ra, ch);
-        if (ch + 1 < ch_hi) {
-          if (ti.nkb > 0) {
-            tmem_ld_wait();
-            if (ch + 2 < ch_hi) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), ra);
+        __threadfence();
+        __syncwarp();
+        int* cnt = p.sk_cnt + un.sk_tile * WSLOTS + wslot;
+        int arrived = 0;
+        if (lane == 0) arrived = atomicAdd(cnt, 1);
+        arrived = __shfl_sync(0xffffffffu, arrived, 0);
+        if (arrived == un.nsplit - 1) {
+          if (lane == 0) *cnt = 0;  // armed again for the next launch
+          __threadfence();
+          // Two 32-column chunks per round, so that 16 loads per thread are in flight for each share.
+#pragma unroll 1
+          for (int ch = ch_lo; ch < ch_hi; ch += 2) {
+            const bool two = ch + 1 < ch_hi;
+            float sum0[32], sum1[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sum0[i] = sum1[i] = 0.f;
+#pragma unroll 1
+            for (int j = un.jfirst; j < un.jfirst + un.nsplit; ++j) {
+              if (j == w0) {
+                tmem_ld32(t_row + (uint32_t)(ch * 32), r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) sum0[i] += __uint_as_float(r[i]);
+                if (two) {
+                  tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), r);
+                  tmem_ld_wait();
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) sum1[i] += __uint_as_float(r[i]);
+                }
+              } else {
+                const int slot_j = un.sk_tile - sch.share_start(j) / sch.KT;
+                const float4* src =
+                    p.sk_ws + (size_t)((j * 2 + slot_j) * WSLOTS + wslot) * SK_SLOT_F4 + lane + (ch - ch_lo) * 256;
+                float4 x0[8], x1[8];
+#pragma unroll
+                for (int q8 = 0; q8 < 8; ++q8) x0[q8] = __ldcg(src + q8 * 32);
+#pragma unroll
+                for (int q8 = 0; q8 < 8; ++q8) x1[q8] = two ? __ldcg(src + 256 + q8 * 32) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int q8 = 0; q8 < 8; ++q8) {
+                  sum0[4 * q8] += x0[q8].x;
+                  sum0[4 * q8 + 1] += x0[q8].y;
+                  sum0[4 * q8 + 2] += x0[q8].z;
+                  sum0[4 * q8 + 3] += x0[q8].w;
+                }
+#pragma unroll
+                for (int q8 = 0; q8 < 8; ++q8) {
+                  sum1[4 * q8] += x1[q8].x;
+                  sum1[4 * q8 + 1] += x1[q8].y;
+                  sum1[4 * q8 + 2] += x1[q8].z;
+                  sum1[4 * q8 + 3] += x1[q8].w;
+                }
+              }
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum0[i]);
+            emit(r, ch);
+            if (two) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(sum1[i]);
+              emit(r, ch + 1);
+            }
           }
-          emit(rb, ch + 1);
+        }
+      } else {
+        // Software pipeline over this warp's chunks: the TMEM load of chunk i+1 is in flight while
+        // chunk i is converted and stored.
+        uint32_t ra[32], rb[32];
+        if (has_acc && ch_lo < ch_hi) tmem_ld32(t_row + (uint32_t)(ch_lo * 32), ra);
+#pragma unroll 1
+        for (int ch = ch_lo; ch < ch_hi; ch += 2) {
+          if (has_acc) {
+            tmem_ld_wait();
+            if (ch + 1 < ch_hi) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), rb);
+          }
+          emit(ra, ch);
+          if (ch + 1 < ch_hi) {
+            if (has_acc) {
+              tmem_ld_wait();
+              if (ch + 2 < ch_hi) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), ra);
+            }
+            emit(rb, ch + 1);
+          }
         }
       }
       tc_fence_before();
@@ -967,12 +1160,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   }
 }
 
-template <int BN, int MODE, int CTAS>
+// max_tiles: tile count of the densest pattern
+template <int BN, int MODE, int CTAS, bool SHARE = false>
 ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStream_t s) {
   using L = SmemLayout<BN, CTAS>;
   static bool attr_done[64] = {};
   static int max_clusters[64] = {};
-  auto kern = ard_gemm_tc_kernel<BN, MODE, CTAS>;
+  auto kern = ard_gemm_tc_kernel<BN, MODE, CTAS, SHARE>;
   const int dev = ctx->device & 63;
   if (!attr_done[dev]) {
     ARD_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
@@ -1000,8 +1194,9 @@ ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStrea
     }
     workers = max_clusters[dev];
   }
-  if (max_tiles < workers) workers = max_tiles;  // max_tiles: tile count of the densest pattern
+  if (max_tiles < workers) workers = max_tiles;
   if (workers < 1) workers = 1;
+  if (workers * CTAS > ctx->sm_count) return ARD_ERR_UNSUPPORTED;  // the partial-sum scratch is sized per SM
   cfg.gridDim = dim3(workers * CTAS);
   TcParams pc = p;
   ARD_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, pc));
@@ -1057,28 +1252,36 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
   p.force_bn = (kind == ARD_ROW) ? a.bn : 0;
   p.accumulate = a.g.accumulate;
   p.band_m = ctx->band_m;
+  const bool share = kind == ARD_ROW && ctx->stream_k && ctx->d_sk_ws != nullptr;
+  p.sk_ws = share ? reinterpret_cast<float4*>(ctx->d_sk_ws) : nullptr;
+  p.sk_cnt = ctx->d_sk_cnt;
+  p.sk_min_blocks = ctx->sk_min_blocks;
+  p.sk_min_gain = ctx->sk_min_gain;
   const int bn = (kind == ARD_ROW) ? 256 : a.bn;
 
 #define ARD_TC_CASE(BN_, MODE_, TILES_) \
   if (bn == BN_) return launch_mode<BN_, MODE_, 1>(ctx, p, (TILES_), s);
+#define ARD_TC_ROW(MODE_, TILES_)                                                      \
+  return share ? launch_mode<256, MODE_, 1, true>(ctx, p, (TILES_), s) : launch_mode<256, MODE_, 1, false>(ctx, p, (TILES_), s);
   // Row patterns with at least two 128-row tiles of output use CTA pairs (256-row tiles).
 #define ARD_TC_PAIR(MODE_, MROWS_, NCOLS_)                                                      \
   if (ctx->use_pairs && (MROWS_) > BM && (p.force_bn == 0 || p.force_bn >= 128))                \
-    return launch_mode<256, MODE_, 2>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s);
+    return share ? launch_mode<256, MODE_, 2, true>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s)         \
+                 : launch_mode<256, MODE_, 2, false>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s);
 
   if (kind == ARD_ROW) {
     if (op == OP_FWD) {
       const int mt = cdiv(p.B, BM);
       ARD_TC_PAIR(M_ROW_FWD, p.B, p.N)
-      ARD_TC_CASE(256, M_ROW_FWD, mt * cdiv(p.N, 64))
+      ARD_TC_ROW(M_ROW_FWD, mt * cdiv(p.N, 64))
     } else if (op == OP_BWD_DATA) {
       const int mt = cdiv(p.B, BM);
       ARD_TC_PAIR(M_ROW_BWD_DATA, p.B, p.K)
-      ARD_TC_CASE(256, M_ROW_BWD_DATA, mt * cdiv(p.K, 64))
+      ARD_TC_ROW(M_ROW_BWD_DATA, mt * cdiv(p.K, 64))
     } else {
       const int mt = cdiv(p.N, BM);
       ARD_TC_PAIR(M_ROW_BWD_WEIGHT, p.N, p.K)
-      ARD_TC_CASE(256, M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 64))
+      ARD_TC_ROW(M_ROW_BWD_WEIGHT, mt * cdiv(p.K, 64))
     }
   } else if (bn == 0) {
     // class form of the tile pattern; the grid covers all SMs, CTAs without tiles leave at once
@@ -1109,6 +1312,7 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
     }
   }
 #undef ARD_TC_CASE
+#undef ARD_TC_ROW
 #undef ARD_TC_PAIR
   return ARD_ERR_UNSUPPORTED;
 }
@@ -1138,6 +1342,10 @@ ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStrea
   p.force_bn = a.bn;
   p.accumulate = a.g.accumulate;
   p.band_m = 0;
+  p.sk_ws = nullptr;
+  p.sk_cnt = nullptr;
+  p.sk_min_blocks = 16;
+  p.sk_min_gain = 1;
   const int mt = cdiv(p.B, BM);
   if (!backward) return launch_mode<256, M_LSTM_FWD, 1>(ctx, p, mt * cdiv(p.N, 64), s);
   return launch_mode<256, M_LSTM_BWD_DATA, 1>(ctx, p, mt * cdiv(p.K, 64), s);
