@@ -191,6 +191,8 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   if (const char* e = getenv("ARD_BAND_M")) ctx->band_m = atoi(e);
   ctx->reuse_compact = 0;
   ctx->stream_k = 0;
+  ctx->use_pdl = 1;
+  if (const char* e = getenv("ARD_PDL")) ctx->use_pdl = atoi(e) ? 1 : 0;
   ctx->sk_min_blocks = 16;
   if (const char* e = getenv("ARD_STREAM_K")) ctx->stream_k = atoi(e);
   ctx->sk_min_gain = 24;

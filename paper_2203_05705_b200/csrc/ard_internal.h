@@ -73,6 +73,7 @@ struct ard_ctx {
   int use_pairs;      // tensor-core row kernels: CTA pairs (cta_group::2) when the output has >= 2 row tiles
   int band_m;         // raster band height of the tensor-core kernels, in 128-row tiles
   int reuse_compact;  // opt-in: consecutive backward calls share one compacted dY
+  int use_pdl;        // launch kernels with programmatic stream serialization (see ard_launch)
   int stream_k;       // tensor-core row kernels: share the last, partial wave of tiles along the contraction
   int sk_min_blocks;  // fewest 64-wide contraction blocks worth a separate share
   int sk_min_gain;    // fewest blocks the sharing must save per worker to be used
@@ -156,6 +157,36 @@ ard_status launch_lstm_gates_bwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype
                                  const float* gates_saved, const float* c_prev, const float* c, int ldc,
                                  const float* dh, int lddh, int dh_scatter, float* dc_inout, void* dZ, int ldz_gate,
                                  cudaStream_t s);
+
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// Every kernel of the library is launched so that its blocks may become resident while the previous
+// kernel of the stream is still draining: the block set-up (barriers, tensor memory, index arithmetic)
+// and the launch latency then overlap the tail of that kernel.  In return every kernel (1) lets its own
+// successor start early with pdl_launch_dependents() and (2) calls pdl_wait_prior_grids() before its
+// first access to global memory; that call returns once all earlier kernels of the stream have
+// completed and their writes are visible.  Both are no-ops for a kernel launched the ordinary way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
+template <typename... P, typename... A>
+inline cudaError_t ard_launch(const ard_ctx* ctx, void (*kern)(P...), dim3 grid, dim3 block, size_t smem,
+                              cudaStream_t s, A... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  if (ctx->use_pdl) {
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, kern, P(args)...);
+}
 
 #define ARD_CUDA_OK(expr)                       \
   do {                                          \

@@ -9,6 +9,8 @@ namespace {
 template <typename T>
 __global__ void __launch_bounds__(256) gather_cols_kernel(const int32_t* __restrict__ hdr, const T* __restrict__ src,
                                                           int ld_src, T* __restrict__ dst, int ld_dst, int rows) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], b = hdr[HDR_B];
   const int j = blockIdx.x * 256 + threadIdx.x;
   if (j >= n_keep) return;
@@ -28,6 +30,8 @@ __global__ void __launch_bounds__(GATHER_WARPS * 32)
 gather_cols_staged_kernel(const int32_t* __restrict__ hdr, const uint16_t* __restrict__ src, int ld_src,
                           uint16_t* __restrict__ dst, int ld_dst, int rows, int n_cols, int skip_dense) {
   __shared__ __align__(16) uint16_t smem[GATHER_WARPS][GATHER_SPAN + 8];
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
   if (skip_dense && dp == 1) return;
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -91,6 +95,8 @@ lstm_gates_kernel(const int32_t* __restrict__ hdr, int B, int H, float alpha, co
                   int ldz, const float* __restrict__ bias, const float* __restrict__ c_prev, int ldc,
                   float* __restrict__ c, HT* __restrict__ h, int ldh, int h_scatter,
                   float* __restrict__ gates_saved) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], b = hdr[HDR_B];
   const int i = blockIdx.y;
   const int x = blockIdx.x * 256 + threadIdx.x;  // unit (scatter) or kept index (compact)
@@ -137,6 +143,8 @@ lstm_gates_bwd_kernel(const int32_t* __restrict__ hdr, int B, int H, float alpha
                       const float* __restrict__ gates_saved, const float* __restrict__ c_prev,
                       const float* __restrict__ c, int ldc, const float* __restrict__ dh, int lddh, int dh_scatter,
                       float* __restrict__ dc_inout, ZT* __restrict__ dZ, int ldz) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], b = hdr[HDR_B];
   const int i = blockIdx.y;
   const int j = blockIdx.x * 256 + threadIdx.x;
@@ -168,14 +176,16 @@ ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* i
   const bool vec_ok = elem_bytes == 2 && ld_src % 8 == 0 && ld_dst % 8 == 0 &&
                       (reinterpret_cast<uintptr_t>(src) & 15) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0;
   if (vec_ok) {
-    gather_cols_staged_kernel<<<ctx->sm_count * 6, GATHER_WARPS * 32, 0, s>>>(hdr, (const uint16_t*)src, ld_src, (uint16_t*)dst,
-                                                                 ld_dst, rows, max_cols, skip_dense);
+    ARD_CUDA_OK(ard_launch(ctx, gather_cols_staged_kernel, dim3(ctx->sm_count * 6), dim3(GATHER_WARPS * 32), 0, s, hdr,
+                           (const uint16_t*)src, ld_src, (uint16_t*)dst, ld_dst, rows, max_cols, skip_dense));
   } else {
     dim3 grid((max_cols + 255) / 256, rows < 1024 ? rows : 1024);
     if (elem_bytes == 2)
-      gather_cols_kernel<uint16_t><<<grid, 256, 0, s>>>(hdr, (const uint16_t*)src, ld_src, (uint16_t*)dst, ld_dst, rows);
+      ARD_CUDA_OK(ard_launch(ctx, gather_cols_kernel<uint16_t>, grid, dim3(256), 0, s, hdr, (const uint16_t*)src, ld_src,
+                             (uint16_t*)dst, ld_dst, rows));
     else
-      gather_cols_kernel<uint32_t><<<grid, 256, 0, s>>>(hdr, (const uint32_t*)src, ld_src, (uint32_t*)dst, ld_dst, rows);
+      ARD_CUDA_OK(ard_launch(ctx, gather_cols_kernel<uint32_t>, grid, dim3(256), 0, s, hdr, (const uint32_t*)src, ld_src,
+                             (uint32_t*)dst, ld_dst, rows));
   }
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
@@ -188,11 +198,11 @@ ard_status launch_lstm_gates(ard_ctx* ctx, const ard_pattern* pat, ard_dtype h_d
   if (B == 0 || H == 0) return ARD_OK;
   dim3 grid((H + 255) / 256, B);
   if (h_dtype == ARD_F32)
-    lstm_gates_kernel<float><<<grid, 256, 0, s>>>(pat->d_hdr, B, H, alpha, Z, ldz_gate, bias, c_prev, ldc, c,
-                                                  (float*)h, ldh, h_scatter, gates_saved);
+    ARD_CUDA_OK(ard_launch(ctx, lstm_gates_kernel<float>, grid, dim3(256), 0, s, (const int32_t*)pat->d_hdr, B, H, alpha, Z,
+                           ldz_gate, bias, c_prev, ldc, c, (float*)h, ldh, h_scatter, gates_saved));
   else
-    lstm_gates_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(pat->d_hdr, B, H, alpha, Z, ldz_gate, bias, c_prev, ldc, c,
-                                                          (__nv_bfloat16*)h, ldh, h_scatter, gates_saved);
+    ARD_CUDA_OK(ard_launch(ctx, lstm_gates_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, (const int32_t*)pat->d_hdr, B, H,
+                           alpha, Z, ldz_gate, bias, c_prev, ldc, c, (__nv_bfloat16*)h, ldh, h_scatter, gates_saved));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;
@@ -205,12 +215,12 @@ ard_status launch_lstm_gates_bwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype
   if (B == 0 || H == 0) return ARD_OK;
   dim3 grid((H + 255) / 256, B);
   if (dz_dtype == ARD_F32)
-    lstm_gates_bwd_kernel<float><<<grid, 256, 0, s>>>(pat->d_hdr, B, H, alpha, gates_saved, c_prev, c, ldc, dh, lddh,
-                                                      dh_scatter, dc_inout, (float*)dZ, ldz_gate);
+    ARD_CUDA_OK(ard_launch(ctx, lstm_gates_bwd_kernel<float>, grid, dim3(256), 0, s, (const int32_t*)pat->d_hdr, B, H, alpha,
+                           gates_saved, c_prev, c, ldc, dh, lddh, dh_scatter, dc_inout, (float*)dZ, ldz_gate));
   else
-    lstm_gates_bwd_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(pat->d_hdr, B, H, alpha, gates_saved, c_prev, c, ldc,
-                                                              dh, lddh, dh_scatter, dc_inout, (__nv_bfloat16*)dZ,
-                                                              ldz_gate);
+    ARD_CUDA_OK(ard_launch(ctx, lstm_gates_bwd_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, (const int32_t*)pat->d_hdr, B,
+                           H, alpha, gates_saved, c_prev, c, ldc, dh, lddh, dh_scatter, dc_inout, (__nv_bfloat16*)dZ,
+                           ldz_gate));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;

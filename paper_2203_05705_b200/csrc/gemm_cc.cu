@@ -31,6 +31,8 @@ __global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts)
   __shared__ float As[T_K][T_M + 1];
   __shared__ float Bs[T_K][T_N + 1];
 
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
   const int dp = g.hdr[HDR_DP], b = g.hdr[HDR_B], n_keep = g.hdr[HDR_NKEEP];
   const int Tc = g.hdr[HDR_TC];
   const T* __restrict__ P0 = reinterpret_cast<const T*>(g.A0);
@@ -152,23 +154,23 @@ __global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts)
 }
 
 template <typename T, int KIND, int OP>
-void launch_one(const GemmArgs& a, int ts, int Mmax, int Nmax, cudaStream_t s) {
+void launch_one(const ard_ctx* ctx, const GemmArgs& a, int ts, int Mmax, int Nmax, cudaStream_t s) {
   dim3 grid((Nmax + T_N - 1) / T_N, (Mmax + T_M - 1) / T_M);
-  gemm_cc_kernel<T, KIND, OP><<<grid, CC_THREADS, 0, s>>>(a, ts);
+  (void)ard_launch(ctx, gemm_cc_kernel<T, KIND, OP>, grid, dim3(CC_THREADS), 0, s, a, ts);  // errors: cudaGetLastError
 }
 
 template <typename T>
-void dispatch(ard_kind kind, GemmOp op, const GemmArgs& a, int ts, cudaStream_t s) {
+void dispatch(const ard_ctx* ctx, ard_kind kind, GemmOp op, const GemmArgs& a, int ts, cudaStream_t s) {
   // The grid covers the largest problem any pattern can produce (dp = 1); CTAs beyond the
   // sampled extent read the header and exit.
   if (kind == ARD_ROW) {
-    if (op == OP_FWD) launch_one<T, 0, OP_FWD>(a, ts, a.B, a.N, s);
-    else if (op == OP_BWD_DATA) launch_one<T, 0, OP_BWD_DATA>(a, ts, a.B, a.K, s);
-    else launch_one<T, 0, OP_BWD_WEIGHT>(a, ts, a.N, a.K, s);
+    if (op == OP_FWD) launch_one<T, 0, OP_FWD>(ctx, a, ts, a.B, a.N, s);
+    else if (op == OP_BWD_DATA) launch_one<T, 0, OP_BWD_DATA>(ctx, a, ts, a.B, a.K, s);
+    else launch_one<T, 0, OP_BWD_WEIGHT>(ctx, a, ts, a.N, a.K, s);
   } else {
-    if (op == OP_FWD) launch_one<T, 1, OP_FWD>(a, ts, a.B, a.N, s);
-    else if (op == OP_BWD_DATA) launch_one<T, 1, OP_BWD_DATA>(a, ts, a.B, a.K, s);
-    else launch_one<T, 1, OP_BWD_WEIGHT>(a, ts, a.N, a.K, s);
+    if (op == OP_FWD) launch_one<T, 1, OP_FWD>(ctx, a, ts, a.B, a.N, s);
+    else if (op == OP_BWD_DATA) launch_one<T, 1, OP_BWD_DATA>(ctx, a, ts, a.B, a.K, s);
+    else launch_one<T, 1, OP_BWD_WEIGHT>(ctx, a, ts, a.N, a.K, s);
   }
 }
 
@@ -185,8 +187,8 @@ ard_status launch_gemm_cc(ard_ctx* ctx, ard_kind kind, GemmOp op, ard_dtype dtyp
   if (kind == ARD_ROW && op == OP_BWD_WEIGHT && a.flag1) {
     ARD_CUDA_OK(cudaMemset2DAsync(a.out, (size_t)a.ldo * es_out, 0, (size_t)a.K * es_out, a.N, s));
   }
-  if (dtype == ARD_F32) dispatch<float>(kind, op, a, ts, s);
-  else dispatch<__nv_bfloat16>(kind, op, a, ts, s);
+  if (dtype == ARD_F32) dispatch<float>(ctx, kind, op, a, ts, s);
+  else dispatch<__nv_bfloat16>(ctx, kind, op, a, ts, s);
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;

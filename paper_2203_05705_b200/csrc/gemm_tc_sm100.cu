@@ -716,6 +716,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::MISC_OFF + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_launch_dependents();  // the next kernel of the stream may set up while this one runs
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -743,6 +744,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_ptr_smem;
+  // Everything above touched only this CTA's shared and tensor memory; from here on the kernel reads
+  // what earlier kernels of the stream wrote (the pattern, the operands) and overwrites what they read.
+  pdl_wait_prior_grids();
 
   Sched<BN, MODE, CTAS, SHARE> sch;
   sch.init(p, (int)rank);
@@ -1176,14 +1180,15 @@ ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStrea
   cfg.blockDim = dim3(TC_THREADS);
   cfg.dynamicSmemBytes = L::TOTAL;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   int workers = ctx->sm_count / CTAS;
+  cfg.attrs = attr;
+  cfg.numAttrs = 0;
   if (CTAS == 2) {
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (max_clusters[dev] == 0) {
       // how many CTA pairs the device can hold at once (SM pairs must share a TPC)
@@ -1198,6 +1203,11 @@ ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStrea
   if (workers < 1) workers = 1;
   if (workers * CTAS > ctx->sm_count) return ARD_ERR_UNSUPPORTED;  // the partial-sum scratch is sized per SM
   cfg.gridDim = dim3(workers * CTAS);
+  if (ctx->use_pdl) {
+    attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs++;
+  }
   TcParams pc = p;
   ARD_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, pc));
   ctx->launches++;

@@ -40,6 +40,8 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
                   unsigned long long iteration, uint32_t stream_id, int forced_dp, int forced_b, int kind,
                   int units, int Tr, int Tc, int ts) {
   __shared__ int s_dp, s_b;
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();  // earlier kernels may still be reading the lists this kernel rewrites
   if (threadIdx.x == 0) {
     int dp, b;
     if (forced_dp > 0) {
@@ -124,11 +126,10 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
 
 ard_status launch_sampler(ard_ctx* ctx, ard_pattern* pat, const unsigned long long* d_cdf, int ndp, uint64_t seed,
                           uint64_t iteration, uint32_t stream_id, int forced_dp, int forced_b, cudaStream_t s) {
-  ard_sample_kernel<<<1, SAMPLER_THREADS, 0, s>>>(pat->d_hdr, pat->d_idx, pat->d_col_ptr, pat->d_col_idx,
-                                                  pat->d_row_ptr, pat->d_row_idx, d_cdf, ndp,
-                                                  (unsigned long long)seed, (unsigned long long)iteration, stream_id,
-                                                  forced_dp, forced_b, (int)pat->kind, pat->units, pat->Tr, pat->Tc,
-                                                  pat->ts);
+  ARD_CUDA_OK(ard_launch(ctx, ard_sample_kernel, dim3(1), dim3(SAMPLER_THREADS), 0, s, pat->d_hdr, pat->d_idx,
+                         pat->d_col_ptr, pat->d_col_idx, pat->d_row_ptr, pat->d_row_idx, d_cdf, ndp,
+                         (unsigned long long)seed, (unsigned long long)iteration, stream_id, forced_dp, forced_b,
+                         (int)pat->kind, pat->units, pat->Tr, pat->Tc, pat->ts));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;
