@@ -16,9 +16,13 @@ Pins (each lives in tests/test_oracle_*.py):
   lstm.*                   dp=1 == torch.nn.LSTM (fp64, forward and autograd gradients);
                            kept sub-network == torch.nn.LSTM of hidden size n_k; finite differences
   mlp_chain.*              finite differences of the scalar <dZ3, Z3>
+  search.*                 gradient vs central differences; stationary points lie in the Gibbs family
+                           ln k_i = beta (i-1)/i + c with beta = -2 (k.p_u - p)/lambda; small-lambda limit ==
+                           the maximum-entropy distribution at rate p; Eq. 2-3 in exact rationals
 
-Parity unpinned (the paper fixes no value to compare with): the choice of the
-distribution K itself (the body of Algorithm 1 is not printed), the tile
+Parity unpinned (the paper fixes no value to compare with): the constants of the
+distribution search (the body of Algorithm 1 is not printed: loss form, lambda, step size, start and
+stopping rule are a reading, see search.py) and therefore the authors' own K, the tile
 linearisation order beyond the first tile of the worked example, the LSTM
 reading (which units are dropped, gate order) and the rescale convention.
 """
