@@ -115,6 +115,20 @@ ard_status ard_set_distribution(ard_ctx* ctx, int dist_id, const double* K, int 
 /* The quantisation alone, on the host (no context or GPU needed): validates K as above and writes the
  * ndp cumulative entries to cdf_out (HOST uint64). */
 ard_status ard_quantise_distribution(const double* K, int ndp, uint64_t* cdf_out);
+/* Sec. 3.3, Algorithm 1: finds K for a target global dropout rate p by gradient descent, on the host
+ * in fp64 (no context or GPU needed).  v (length ndp) starts at zero, d = softmax(v) is the
+ * distribution, p_u = {(i-1)/i}; the loss (d.p_u - p)^2 + lambda * sum_i d_i ln d_i is reduced by
+ * steps v <- v - step * dloss/dv until it changes by less than tol or max_iter steps were taken.
+ * (The paper's listing is not printed; squared difference, lambda, the start and the stopping rule are
+ * this library's reading of the text.)  At convergence ln k_i is affine in (i-1)/i and
+ * K.p_u - p = -lambda*beta/2 with beta its slope, so a small lambda meets the rate closely:
+ * lambda = 1e-3, step = 10, tol = 1e-16 reaches |K.p_u - p| ~ 1e-3 in ~2e4 steps for ndp = 16.
+ * K_out: HOST array of ndp doubles, summing to 1 within rounding (pass it to ard_set_distribution).
+ * iterations_out (may be NULL): steps taken.  Errors: ARD_ERR_INVALID_ARG (NULL, ndp out of range,
+ * p outside [0,1), non-positive lambda / step, negative tol), ARD_ERR_DISTRIBUTION (p above the
+ * reachable (ndp-1)/ndp, or the iteration diverged because step is too large). */
+ard_status ard_search_distribution(double p, int ndp, double lambda, double step, int max_iter, double tol,
+                                   double* K_out, int* iterations_out);
 /* Copies the quantised cumulative table (ndp entries, HOST uint64) back, for tests. */
 ard_status ard_get_distribution_cdf(ard_ctx* ctx, int dist_id, uint64_t* cdf_out, int capacity, int* ndp_out);
 

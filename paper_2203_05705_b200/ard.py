@@ -27,7 +27,7 @@ ARD_PATH_AUTO, ARD_PATH_CUDA_CORE, ARD_PATH_TENSOR_CORE = 0, 1, 2
 ARD_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = [
-    "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_shared_tail", "ard_set_compact_reuse", "ard_set_distribution", "ard_quantise_distribution", "ard_get_distribution_cdf",
+    "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_shared_tail", "ard_set_compact_reuse", "ard_set_distribution", "ard_quantise_distribution", "ard_search_distribution", "ard_get_distribution_cdf",
     "ard_pattern_create", "ard_pattern_destroy", "ard_sample_pattern", "ard_pattern_set",
     "ard_pattern_to_host", "ard_pattern_tile_lists_to_host", "ard_fwd", "ard_bwd_data", "ard_bwd_weight",
     "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_lstm_forward", "ard_lstm_backward", "ard_last_device_status", "ard_status_string", "ard_launch_count",
@@ -62,6 +62,7 @@ def lib():
         "ard_set_compact_reuse": [vp, i32],
         "ard_set_distribution": [vp, i32, P(C.c_double), i32],
         "ard_quantise_distribution": [P(C.c_double), i32, P(u64)],
+        "ard_search_distribution": [C.c_double, i32, C.c_double, C.c_double, i32, C.c_double, P(C.c_double), P(i32)],
         "ard_get_distribution_cdf": [vp, i32, P(u64), i32, P(i32)],
         "ard_pattern_create": [vp, P(vp), i32, i32, i32, i32],
         "ard_pattern_destroy": [vp],
@@ -145,6 +146,16 @@ def ard_set_distribution(ctx, dist_id, K):
     K = np.ascontiguousarray(K, dtype=np.float64)
     _check(lib().ard_set_distribution(ctx, dist_id, K.ctypes.data_as(C.POINTER(C.c_double)), len(K)),
            "ard_set_distribution")
+
+
+def ard_search_distribution(p, ndp, lam=1e-3, step=10.0, max_iter=200000, tol=1e-16):
+    """Host-only: Algorithm 1.  Returns (K as a float64 array, iterations)."""
+    K = np.zeros(max(int(ndp), 1), dtype=np.float64)
+    it = C.c_int(0)
+    _check(lib().ard_search_distribution(float(p), int(ndp), float(lam), float(step), int(max_iter), float(tol),
+                                         K.ctypes.data_as(C.POINTER(C.c_double)), C.byref(it)),
+           "ard_search_distribution")
+    return K[:ndp], it.value
 
 
 def ard_quantise_distribution(K):

@@ -84,3 +84,29 @@ def test_host_side_quantiser_matches_the_oracle(built):
         with pytest.raises(ard.ArdError) as e:
             ard.ard_quantise_distribution(bad)
         assert e.value.status == ard.ARD_ERR_DISTRIBUTION
+
+
+def test_host_side_distribution_search_matches_the_oracle(built):
+    """Algorithm 1 on the host: same iterates as the oracle's numpy statement, and the rejections."""
+    import numpy as np
+    from oracle import search as OS
+    from paper_2203_05705_b200 import ard
+    for p, ndp, lam in [(0.5, 16, 1e-2), (0.3, 8, 1e-1), (0.7, 16, 1e-2), (0.5, 3, 1e-3)]:
+        # the same number of steps on both sides: the iterates agree to rounding
+        K, it = ard.ard_search_distribution(p, ndp, lam=lam, step=10.0, max_iter=5000, tol=0.0)
+        Ko, ito = OS.search_K(p, ndp, lam=lam, lr=10.0, max_iter=5000, tol=0.0)
+        assert it == ito == 5000
+        assert np.abs(K - Ko).max() <= 1e-12, (p, ndp, lam)
+        # the stopping rule fires where the loss flattens; libm and numpy differ in the last bits of
+        # exp / log, so the step count and the returned point agree only to the flatness of the loss there
+        K, it = ard.ard_search_distribution(p, ndp, lam=lam, step=10.0, max_iter=100000, tol=1e-17)
+        Ko, ito = OS.search_K(p, ndp, lam=lam, lr=10.0, max_iter=100000, tol=1e-17)
+        assert it < 100000 and ito < 100000
+        assert np.abs(K - Ko).max() <= 1e-7, (p, ndp, lam)
+        assert abs(K.sum() - 1.0) <= 1e-12
+        ard.ard_quantise_distribution(K)                     # acceptable to the sampler's quantiser
+    for args in [(1.0, 16), (-0.1, 16), (0.5, 0), (0.9, 4)]:
+        with pytest.raises(ard.ArdError):
+            ard.ard_search_distribution(*args)
+    with pytest.raises(ard.ArdError):
+        ard.ard_search_distribution(0.5, 16, lam=0.0)
