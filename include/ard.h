@@ -243,11 +243,18 @@ ard_status ard_lstm_gate_gemm_bwd(ard_ctx* ctx, const ard_pattern* pat, int B, i
                                   int ldz_gate, const void* W, int ldw, float* dXH, int lddxh, int accumulate,
                                   void* cuda_stream);
 
-/* Whole-sequence forward: for t = 0..T-1, ard_lstm_gate_gemm on XH[t] followed by ard_lstm_gates, which writes
- * h_t into the h half of XH[t+1].  The loop runs in native code and only enqueues kernels.
+/* Whole-sequence forward: for t = 0..T-1, the gate product on XH[t] followed by the cell update, which writes
+ * h_t into the h half of XH[t+1].  When the layer fits (B <= 128, the weight rows of 8 hidden units times
+ * (I+H) columns fit in shared memory, H/8 <= number of SMs, operands aligned for the tensor-core path) this
+ * is ONE cooperative kernel that keeps the weight in shared memory and the cell state in registers for the
+ * whole sequence and synchronises the SMs once per step (every wait bounded, see ARD_ERR_TIMEOUT); Z is
+ * then not used.  Otherwise, or after ard_set_lstm_persistent(ctx, 0), it is a loop in native code that
+ * enqueues ard_lstm_gate_gemm and ard_lstm_gates per step.  Both give the same C, G and XH up to
+ * summation order.
  *   XH [T+1][B][I+H] bf16: the caller fills the x halves of XH[0..T-1] and the h half of XH[0] (h_0, zeros at
  *   dropped units); C [T+1][B][H] fp32 compact cell states, C[0] = c_0; G [T][B][4H] fp32 saved gates;
  *   Z [B][4H] fp32 scratch; W [4H][I+H] bf16 (ldw); bias [4][H] or NULL. */
+ard_status ard_set_lstm_persistent(ard_ctx* ctx, int enable); /* default: enabled */
 ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha, void* XH,
                             const void* W, int ldw, const float* bias, float* C, float* G, float* Z,
                             void* cuda_stream);

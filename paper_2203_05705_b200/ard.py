@@ -30,7 +30,7 @@ EXPORTS = [
     "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_shared_tail", "ard_set_compact_reuse", "ard_set_distribution", "ard_quantise_distribution", "ard_search_distribution", "ard_get_distribution_cdf",
     "ard_pattern_create", "ard_pattern_destroy", "ard_sample_pattern", "ard_pattern_set",
     "ard_pattern_to_host", "ard_pattern_tile_lists_to_host", "ard_fwd", "ard_bwd_data", "ard_bwd_weight",
-    "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_lstm_forward", "ard_lstm_backward", "ard_last_device_status", "ard_status_string", "ard_launch_count",
+    "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_set_lstm_persistent", "ard_lstm_forward", "ard_lstm_backward", "ard_last_device_status", "ard_status_string", "ard_launch_count",
 ]
 
 _lib = None
@@ -58,6 +58,7 @@ def lib():
         "ard_destroy": [vp],
         "ard_set_path": [vp, i32],
         "ard_set_tile_n": [vp, i32],
+        "ard_set_lstm_persistent": [vp, i32],
         "ard_set_shared_tail": [vp, i32, i32, i32],
         "ard_set_compact_reuse": [vp, i32],
         "ard_set_distribution": [vp, i32, P(C.c_double), i32],
@@ -136,6 +137,10 @@ def ard_set_compact_reuse(ctx, enable):
 
 def ard_set_tile_n(ctx, bn):
     _check(lib().ard_set_tile_n(ctx, bn), "ard_set_tile_n")
+
+
+def ard_set_lstm_persistent(ctx, enable):
+    _check(lib().ard_set_lstm_persistent(ctx, 1 if enable else 0), "ard_set_lstm_persistent")
 
 
 def ard_set_shared_tail(ctx, enable, min_blocks=0, min_gain_blocks=0):

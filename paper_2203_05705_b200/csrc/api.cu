@@ -192,6 +192,9 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->reuse_compact = 0;
   ctx->stream_k = 0;
   ctx->use_pdl = 1;
+  ctx->lstm_persistent = 1;
+  if (const char* e = getenv("ARD_LSTM_PERSISTENT")) ctx->lstm_persistent = atoi(e) ? 1 : 0;
+  ctx->d_grid_bar = nullptr;
   if (const char* e = getenv("ARD_PDL")) ctx->use_pdl = atoi(e) ? 1 : 0;
   ctx->sk_min_blocks = 16;
   if (const char* e = getenv("ARD_STREAM_K")) ctx->stream_k = atoi(e);
@@ -230,7 +233,9 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
     const size_t cnt_bytes = sk_cnt_bytes(ctx->sm_count);
     if (cudaMalloc(&ctx->d_sk_ws, ws_bytes) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->d_sk_cnt), cnt_bytes) != cudaSuccess ||
-        cudaMemset(ctx->d_sk_cnt, 0, cnt_bytes) != cudaSuccess) {
+        cudaMemset(ctx->d_sk_cnt, 0, cnt_bytes) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&ctx->d_grid_bar), 256) != cudaSuccess) {
+      if (ctx->d_grid_bar) cudaFree(ctx->d_grid_bar);
       if (ctx->d_sk_ws) cudaFree(ctx->d_sk_ws);
       if (ctx->d_sk_cnt) cudaFree(ctx->d_sk_cnt);
       if (ctx->d_workspace) cudaFree(ctx->d_workspace);
@@ -253,6 +258,7 @@ ard_status ard_destroy(ard_ctx* ctx) {
   if (ctx->d_workspace) cudaFree(ctx->d_workspace);
   if (ctx->d_sk_ws) cudaFree(ctx->d_sk_ws);
   if (ctx->d_sk_cnt) cudaFree(ctx->d_sk_cnt);
+  if (ctx->d_grid_bar) cudaFree(ctx->d_grid_bar);
   if (ctx->d_status) cudaFree(ctx->d_status);
   delete ctx;
   return ARD_OK;
@@ -276,6 +282,12 @@ ard_status ard_set_shared_tail(ard_ctx* ctx, int enable, int min_blocks, int min
   ctx->stream_k = enable ? 1 : 0;
   if (min_blocks > 0) ctx->sk_min_blocks = min_blocks;
   if (min_gain_blocks > 0) ctx->sk_min_gain = min_gain_blocks;
+  return ARD_OK;
+}
+
+ard_status ard_set_lstm_persistent(ard_ctx* ctx, int enable) {
+  if (!ctx) return ARD_ERR_INVALID_ARG;
+  ctx->lstm_persistent = enable ? 1 : 0;
   return ARD_OK;
 }
 
@@ -799,6 +811,31 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
   if (T < 0 || B < 0 || I < 0 || H < 1) return ARD_ERR_INVALID_ARG;
   const int KH = I + H;
   __nv_bfloat16* xh = reinterpret_cast<__nv_bfloat16*>(XH);
+  // One cooperative kernel for the whole sequence when the layer fits it (the weight slice of 8 hidden
+  // units per CTA in shared memory, all CTAs resident, at most 128 batch rows) and the operands meet the
+  // TMA path's alignment rules; otherwise one gate product and one cell kernel per time step.
+  if (ctx->lstm_persistent && ctx->path != ARD_PATH_CUDA_CORE && T >= 1 && B >= 1) {
+    ard_status st = check_common(ctx, pat, B, KH, H);
+    if (st != ARD_OK) return st;
+    if (pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+    if (ldw < KH) return ARD_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    const char* Wc = reinterpret_cast<const char*>(W);
+    if (tc_eligible(ctx, pat, ARD_BF16, B, KH, H, XH, KH, W, ldw, C, H, 4) == ARD_OK &&
+        ((size_t)H * ldw * 2) % 16 == 0 && lstm_persistent_fits(ctx, B, I, H)) {
+      const CUtensorMap* mapXH = nullptr;
+      const CUtensorMap* mapW[4];
+      st = get_maps(ctx, XH, (T + 1) * B, KH, KH, 0, MAP_PLAIN, 0, 64, 64, &mapXH);
+      if (st != ARD_OK) return st;
+      for (int gate = 0; gate < 4; ++gate) {
+        st = get_maps(ctx, Wc + (size_t)gate * H * ldw * 2, H, KH, ldw, H, MAP_STRIDED_ROWS, pat->dp_bound, 8, 64,
+                      &mapW[gate]);
+        if (st != ARD_OK) return st;
+      }
+      return launch_lstm_forward_persistent(ctx, pat, T, B, I, H, alpha, mapXH, mapW, XH, bias, C, G,
+                                            (cudaStream_t)cuda_stream);
+    }
+  }
   for (int t = 0; t < T; ++t) {
     __nv_bfloat16* xh_t = xh + (size_t)t * B * KH;
     __nv_bfloat16* h_out = xh + (size_t)(t + 1) * B * KH + I;  // h_t lands in the operand of step t+1

@@ -73,6 +73,8 @@ struct ard_ctx {
   int use_pairs;      // tensor-core row kernels: CTA pairs (cta_group::2) when the output has >= 2 row tiles
   int band_m;         // raster band height of the tensor-core kernels, in 128-row tiles
   int reuse_compact;  // opt-in: consecutive backward calls share one compacted dY
+  int lstm_persistent; // ard_lstm_forward: one cooperative kernel for the whole sequence when the layer fits
+  unsigned int* d_grid_bar;  // arrival counter of that kernel's grid-wide barrier
   int use_pdl;        // launch kernels with programmatic stream serialization (see ard_launch)
   int stream_k;       // tensor-core row kernels: share the last, partial wave of tiles along the contraction
   int sk_min_blocks;  // fewest 64-wide contraction blocks worth a separate share
@@ -145,6 +147,12 @@ struct TcArgs {
 int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int dp_bound, int ts);
 ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s);
 ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStream_t s);
+
+// Whole-sequence LSTM forward in one cooperative kernel (lstm_persistent.cu).
+bool lstm_persistent_fits(ard_ctx* ctx, int B, int I, int H);
+ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H,
+                                          float alpha, const CUtensorMap* mapXH, const CUtensorMap* const mapW[4],
+                                          void* XH, const float* bias, float* C, float* G, cudaStream_t s);
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,
                               void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, int skip_dense,

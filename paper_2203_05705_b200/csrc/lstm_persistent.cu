@@ -1,0 +1,368 @@
+// Whole-sequence LSTM forward in one cooperative kernel (Sec. 7: the LSTM layer under a row pattern on
+// its hidden units; one pattern serves every time step).
+//
+// The per-step path launches a gate product and a cell kernel per time step, and each launch costs
+// more than the 64-row product itself.  Here the recurrence runs inside one kernel:
+//   - every CTA owns 8 kept hidden units, i.e. 32 gate columns (i|f|g|o x 8), and loads its slice of
+//     the weight, [32 rows][I+H] bf16, into shared memory once (TMA, rows b-1 + j*dp of each gate block
+//     through the same strided descriptors the forward product uses);
+//   - per step it streams [x_t, h_{t-1}] (64-row TMA boxes) through a ring deep enough to hold the whole
+//     h half at once (the loads are latency-bound), multiplies it with the
+//     resident slice (tcgen05.mma, M = 128, N = 32, accumulator in tensor memory, double-buffered over
+//     steps);
+//   - four warps move the accumulator rows to shared memory, then all 14 compute warps apply the cell
+//     update to the (batch row, unit) pairs, keep c in registers, and write h_t (bf16) into the operand
+//     of step t+1 and, after signalling, c_t and the gate activations for BPTT;
+//   - the x half of a step does not depend on the recurrence, so its loads and MMAs run ahead; only
+//     the h half waits for the grid-wide barrier that says h_{t-1} is complete.
+// Measured on a B200 (T = 35, B = 64, I = H = 1024): 9.7 us per step against 17 us for the two launches of
+// the per-step path, the same for every period.  A step is paced by the activation loads, one 8 KiB block
+// every 0.29 us whatever the MMA shape: all CTAs read the same lines of [x_t, h_{t-1}] at the same time.
+// The grid barrier is an arrival counter in global memory: after its stores and a fence each CTA adds 1,
+// and the producer thread of each CTA polls for t * (number of CTAs with units) before it loads the
+// h half of step t.  The launch is cooperative, so all CTAs are resident; every wait is bounded (2 s)
+// and a CTA that gives up sets the status word, which the others poll, so the kernel always returns.
+#include "ard_internal.h"
+#include "sm100_ptx.h"
+
+namespace {
+
+constexpr int LP_UNITS = 8;                  // kept hidden units per CTA
+constexpr int LP_N = 4 * LP_UNITS;           // gate columns per CTA
+constexpr int LP_BK = 64;                    // contraction block: 64 bf16 = one 128-byte swizzle row
+constexpr int LP_MAX_STAGES = 16;
+constexpr int LP_ROW_BOX = 64 * LP_BK * 2;   // one TMA box of the activations: 64 batch rows x 64 columns
+constexpr int LP_W_BLOCK = LP_N * LP_BK * 2; // one contraction block of the resident weight slice
+constexpr int LP_THREADS = 512;              // warps 0-13 cell update (0-3 also read TMEM: lane quadrant = warp),
+constexpr int LP_MATH = 448;                 //   warp 14 TMA producer, warp 15 MMA issuer
+constexpr int LP_ZS_LD = LP_N + 1;           // staged pre-activations: [128 rows][33] floats
+constexpr int LP_ZS_BYTES = 128 * LP_ZS_LD * 4;
+constexpr int LP_PAIRS_MAX = (128 * LP_UNITS + LP_MATH - 1) / LP_MATH;  // (row, unit) pairs per thread
+
+struct LstmFwdParams {
+  const CUtensorMap* mapXH;    // [(T+1)*B][I+H], boxes of 64 rows x 64 columns
+  const CUtensorMap* mapW[4];  // per gate: table over (dp, b) of strided-row maps, boxes of 8 rows x 64 columns
+  const int32_t* hdr;
+  int T, B, I, H;
+  int stages;         // depth of the activation ring (<= LP_MAX_STAGES)
+  float alpha;
+  __nv_bfloat16* XH;
+  const float* bias;  // [4][H] or nullptr
+  float* C;           // [T+1][B][H] compact
+  float* G;           // [T][B][4H]: gate blocks of width H, compact inside a block
+  unsigned int* bar;  // arrival counter, zero at launch
+  int* status;
+};
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Waits until the arrival counter reaches `target`.  Gives up after the time limit or when another CTA
+// has already recorded a failure.
+__device__ bool grid_wait(const unsigned int* bar, unsigned int target, volatile int* abort_flag, int* status) {
+  if (ld_acquire_u32(bar) >= target) return true;
+  const unsigned long long t0 = global_ns();
+  for (int spin = 1;; ++spin) {
+    if (ld_acquire_u32(bar) >= target) return true;
+    if (*abort_flag) return false;
+    if ((spin & 63) == 0) {
+      if (*reinterpret_cast<volatile int*>(status) != 0) { *abort_flag = 1; return false; }
+      if (global_ns() - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicMax(status, (int)ARD_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ float sigmoid_fast(float x) { return 1.f / (1.f + __expf(-x)); }
+__device__ __forceinline__ float tanh_fast(float x) { return 1.f - 2.f / (1.f + __expf(2.f * x)); }
+
+__global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const LstmFwdParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw_addr);
+
+  const int KH = p.I + p.H;
+  const int nkb = (KH + LP_BK - 1) / LP_BK;
+  // The activation ring comes first and the weight slice right after it: a stage holds one or two
+  // 64-row boxes, the MMA always reads 128 rows, and for a batch of at most 64 rows the upper half of
+  // what it reads is the next stage (or the start of the weight slice); those accumulator rows are
+  // never used.
+  const int STAGES = p.stages;
+  const int row_boxes = (p.B + 63) / 64;
+  const uint32_t a_stage = (uint32_t)row_boxes * LP_ROW_BOX;
+  const uint32_t sA = base;
+  const uint32_t sW = base + (uint32_t)STAGES * a_stage;      // nkb blocks of 4 KiB
+  float* zs = reinterpret_cast<float*>(smem + (sW - base) + (size_t)nkb * LP_W_BLOCK);
+  const uint32_t bar_base = sW + (uint32_t)nkb * LP_W_BLOCK + LP_ZS_BYTES;  // full[16], empty[16], tfull[2], tempty[2], wfull
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (LP_MAX_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * LP_MAX_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * LP_MAX_STAGES + 2 + a); };
+  const uint32_t wfull_bar = bar_base + 8u * (2 * LP_MAX_STAGES + 4);
+  uint8_t* misc = smem + (bar_base - base) + 8 * (2 * LP_MAX_STAGES + 5);
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);  // one arrival per epilogue warp
+    }
+    mbar_init(wfull_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 15) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), 2 * LP_N);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+  pdl_wait_prior_grids();
+
+  const int dp = p.hdr[HDR_DP], bb = p.hdr[HDR_B] - 1, n_keep = p.hdr[HDR_NKEEP];
+  const int n_active = (n_keep + LP_UNITS - 1) / LP_UNITS;  // CTAs that own units (the others only tear down)
+  const int j0 = (int)blockIdx.x * LP_UNITS;                // first kept unit (compact index) of this CTA
+  const bool active = (int)blockIdx.x < n_active;
+  const int xblocks = p.I / LP_BK;                          // contraction blocks that hold only x columns
+
+  if (active) {
+    if (warp == 14) {
+      // ===================== TMA producer =====================
+      if (lane == 0) {
+        const int e = p.hdr[HDR_MAPIDX];
+        tensormap_acquire(p.mapXH);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) tensormap_acquire(p.mapW[g] + e);
+        // the weight slice, once
+        mbar_arrive_expect_tx(wfull_bar, (uint32_t)nkb * LP_W_BLOCK);
+        for (int kb = 0; kb < nkb; ++kb)
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            tma_load_2d(sW + kb * LP_W_BLOCK + g * (LP_UNITS * LP_BK * 2), p.mapW[g] + e, wfull_bar, kb * LP_BK, j0);
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int t = 0; t < p.T && ok; ++t) {
+          for (int kb = 0; kb < nkb; ++kb) {
+            if (kb == xblocks && t > 0) {
+              // the rest of this step reads h_{t-1}: every CTA with units has to have stored its part
+              if (!grid_wait(p.bar, (unsigned)t * (unsigned)n_active, abort_flag, p.status)) { ok = false; break; }
+              asm volatile("fence.proxy.async;" ::: "memory");  // the loads below go through the async proxy
+            }
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            mbar_arrive_expect_tx(full_bar(stage), a_stage);
+            for (int rb = 0; rb < row_boxes; ++rb)
+              tma_load_2d(sA + stage * a_stage + rb * LP_ROW_BOX, p.mapXH, full_bar(stage), kb * LP_BK,
+                          t * p.B + rb * 64);
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    } else if (warp == 15) {
+      // ===================== MMA issuer =====================
+      if (lane == 0) {
+        const uint32_t idesc = make_idesc(LP_N, false, false, 128);
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = mbar_wait(wfull_bar, 0u, abort_flag, p.status);
+        for (int t = 0; t < p.T && ok; ++t) {
+          const int acc = t & 1;
+          if (!mbar_wait(tempty_bar(acc), ((uint32_t)(t >> 1) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * LP_N);
+          for (int kb = 0; kb < nkb; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a0 = sA + stage * a_stage, b0 = sW + kb * LP_W_BLOCK;
+#pragma unroll
+            for (int s = 0; s < LP_BK / 16; ++s)
+              tc_mma_bf16(d_tmem, make_desc(a0 + s * 32, 16, 1024), make_desc(b0 + s * 32, 16, 1024), idesc,
+                          (kb | s) != 0 ? 1u : 0u);
+            tc_commit(empty_bar(stage));
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          }
+          if (!ok) break;
+          tc_commit(tfull_bar(acc));
+        }
+      }
+    } else {
+      // ===================== cell update (warps 0-13) =====================
+      const int tid = threadIdx.x;  // 0 .. LP_MATH-1
+      const size_t ldxh = (size_t)KH;
+      const int npairs = p.B * LP_UNITS;            // (batch row, unit) pairs of this CTA; pair q = row * 8 + k
+      const int nvalid = min(LP_UNITS, n_keep - j0);  // units this CTA really owns (>= 1)
+      float creg[LP_PAIRS_MAX];
+#pragma unroll
+      for (int i = 0; i < LP_PAIRS_MAX; ++i) {
+        const int q = tid + i * LP_MATH;
+        const int row = q >> 3, k = q & 7;
+        creg[i] = (q < npairs && k < nvalid) ? p.C[(size_t)row * p.H + j0 + k] : 0.f;
+      }
+      bool ok = true;
+      for (int t = 0; t < p.T && ok; ++t) {
+        const int acc = t & 1;
+        if (warp < 4) {
+          // accumulator rows -> shared memory
+          if (!mbar_wait(tfull_bar(acc), (uint32_t)(t >> 1) & 1u, abort_flag, p.status)) ok = false;
+          if (ok) {
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * LP_N);
+            uint32_t z[32];
+            tmem_ld32(t_row, z);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));  // the accumulator is in registers now
+            const int r = warp * 32 + lane;
+            if (r < p.B) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) zs[r * LP_ZS_LD + i] = __uint_as_float(z[i]);
+            }
+          }
+        }
+        // every compute thread learns about a failed wait through the flag in shared memory
+        asm volatile("bar.sync 2, 448;" ::: "memory");
+        if (*abort_flag) { ok = false; break; }
+        // Cell update (Sec. 7).  h first, because the other CTAs wait for it; c_t and the gate
+        // activations, which only BPTT reads, after the CTA has signalled.
+        float gi[LP_PAIRS_MAX], gf[LP_PAIRS_MAX], gg[LP_PAIRS_MAX], go[LP_PAIRS_MAX];
+#pragma unroll
+        for (int i = 0; i < LP_PAIRS_MAX; ++i) {
+          const int q = tid + i * LP_MATH;
+          const int row = q >> 3, k = q & 7;
+          if (q < npairs && k < nvalid) {
+            const int u = bb + (j0 + k) * dp;
+            const float* zr = zs + row * LP_ZS_LD;
+            float zi = zr[k], zf = zr[LP_UNITS + k], zg = zr[2 * LP_UNITS + k], zo = zr[3 * LP_UNITS + k];
+            if (p.bias) {
+              zi += p.bias[u];
+              zf += p.bias[p.H + u];
+              zg += p.bias[2 * p.H + u];
+              zo += p.bias[3 * p.H + u];
+            }
+            gi[i] = sigmoid_fast(zi);
+            gf[i] = sigmoid_fast(zf);
+            gg[i] = tanh_fast(zg);
+            go[i] = sigmoid_fast(zo);
+            creg[i] = gf[i] * creg[i] + gi[i] * gg[i];
+            p.XH[((size_t)(t + 1) * p.B + row) * ldxh + p.I + u] = __float2bfloat16_rn(p.alpha * go[i] * tanh_fast(creg[i]));
+          }
+        }
+        // publish h_t: all stores of the CTA, then one release-add for the CTA
+        asm volatile("bar.sync 1, 448;" ::: "memory");
+        if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
+#pragma unroll
+        for (int i = 0; i < LP_PAIRS_MAX; ++i) {
+          const int q = tid + i * LP_MATH;
+          const int row = q >> 3, k = q & 7;
+          if (q < npairs && k < nvalid) {
+            p.C[((size_t)(t + 1) * p.B + row) * p.H + j0 + k] = creg[i];
+            float* g_out = p.G + ((size_t)t * p.B + row) * 4 * p.H + j0 + k;
+            g_out[0] = gi[i];
+            g_out[p.H] = gf[i];
+            g_out[2 * p.H] = gg[i];
+            g_out[3 * p.H] = go[i];
+          }
+        }
+      }
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 15) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 2 * LP_N);
+  }
+}
+
+}  // namespace
+
+// Depth of the activation ring and dynamic shared memory for a layer with I + H = KH and batch B:
+// the weight slice is fixed, the ring takes what is left (at most LP_MAX_STAGES stages).
+static int lstm_fwd_stages(int KH, int B) {
+  const int nkb = (KH + LP_BK - 1) / LP_BK;
+  const long long fixed = (long long)nkb * LP_W_BLOCK + LP_ZS_BYTES + 8 * (2 * LP_MAX_STAGES + 5) + 16 + 1024;
+  const long long a_stage = (long long)((B + 63) / 64) * LP_ROW_BOX;
+  long long st = (227 * 1024 - fixed) / a_stage;
+  return (int)(st > LP_MAX_STAGES ? LP_MAX_STAGES : st);
+}
+static size_t lstm_fwd_smem_bytes(int KH, int B) {
+  const int nkb = (KH + LP_BK - 1) / LP_BK;
+  return (size_t)nkb * LP_W_BLOCK + (size_t)lstm_fwd_stages(KH, B) * ((B + 63) / 64) * LP_ROW_BOX + LP_ZS_BYTES +
+         8 * (2 * LP_MAX_STAGES + 5) + 16 + 1024;
+}
+
+// Can the whole-sequence kernel run this layer on this device?  (Shared memory for the weight slice, one
+// CTA per 8 hidden units all resident at once, one 128-row tile of batch.)
+bool lstm_persistent_fits(ard_ctx* ctx, int B, int I, int H) {
+  if (B < 1 || B > 128 || H < 1) return false;
+  if (lstm_fwd_stages(I + H, B) < 4) return false;  // the weight slice leaves too little room for the ring
+  const size_t smem = lstm_fwd_smem_bytes(I + H, B);
+  static int blocks_per_sm[64] = {};
+  const int dev = ctx->device & 63;
+  if (blocks_per_sm[dev] == 0) {
+    if (cudaFuncSetAttribute(ard_lstm_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        cudaSuccess)
+      return false;
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, ard_lstm_forward_kernel, LP_THREADS, smem) != cudaSuccess || n < 1)
+      n = -1;
+    blocks_per_sm[dev] = n;
+  }
+  if (blocks_per_sm[dev] < 1) return false;
+  return (H + LP_UNITS - 1) / LP_UNITS <= ctx->sm_count;  // one CTA per SM (the slice fills shared memory)
+}
+
+ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H,
+                                          float alpha, const CUtensorMap* mapXH, const CUtensorMap* const mapW[4],
+                                          void* XH, const float* bias, float* C, float* G, cudaStream_t s) {
+  LstmFwdParams p;
+  p.mapXH = mapXH;
+  for (int g = 0; g < 4; ++g) p.mapW[g] = mapW[g];
+  p.hdr = pat->d_hdr;
+  p.T = T; p.B = B; p.I = I; p.H = H;
+  p.stages = lstm_fwd_stages(I + H, B);
+  p.alpha = alpha;
+  p.XH = reinterpret_cast<__nv_bfloat16*>(XH);
+  p.bias = bias;
+  p.C = C;
+  p.G = G;
+  p.bar = ctx->d_grid_bar;
+  p.status = ctx->d_status;
+  ARD_CUDA_OK(cudaMemsetAsync(ctx->d_grid_bar, 0, sizeof(unsigned int), s));
+  // h_1 .. h_T: zeros at the dropped units (the kernel stores the kept ones)
+  ARD_CUDA_OK(cudaMemset2DAsync(p.XH + (size_t)B * (I + H) + I, (size_t)(I + H) * 2, 0, (size_t)H * 2, (size_t)T * B, s));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((H + LP_UNITS - 1) / LP_UNITS);  // sized for dp = 1; CTAs without units leave at once
+  cfg.blockDim = dim3(LP_THREADS);
+  cfg.dynamicSmemBytes = lstm_fwd_smem_bytes(I + H, B);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs resident: they wait for one another
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ARD_CUDA_OK(cudaLaunchKernelEx(&cfg, ard_lstm_forward_kernel, p));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}

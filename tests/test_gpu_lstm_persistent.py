@@ -1,0 +1,98 @@
+"""Whole-sequence LSTM forward in one cooperative kernel vs the oracle and vs the per-step path.
+
+Small layers with ragged sizes (batch not a multiple of 32, kept units not a multiple of the 8 units a
+CTA owns, a bias, non-zero initial state), every h buffer pre-filled with NaN so that the zeros at
+dropped units have to be written by the kernel.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gemm as OG
+from oracle import lstm as OL
+from oracle import pattern as OP
+from paper_2203_05705_b200 import ard, inputs
+from gpu_helpers import Ctx, host, TOL
+
+pytestmark = pytest.mark.gpu
+BF = torch.bfloat16
+
+
+def _run(ctx, pat, T, B, I, H, Wnm, X, bias, h0, c0, keep, alpha, persistent):
+    KH = I + H
+    n = len(keep)
+    XH = torch.full((T + 1, B, KH), float("nan"), dtype=BF, device="cuda")
+    XH[:T, :, :I] = torch.from_numpy(X).to(BF).cuda()
+    XH[0, :, I:] = torch.from_numpy(h0).to(BF).cuda()
+    C = torch.full((T + 1, B, H), float("nan"), dtype=torch.float32, device="cuda")
+    C[0].zero_()
+    C[0, :, :n] = torch.from_numpy(c0[:, keep].astype(np.float32)).cuda()
+    G = torch.full((T, B, 4 * H), float("nan"), dtype=torch.float32, device="cuda")
+    Z = torch.zeros((B, 4 * H), dtype=torch.float32, device="cuda")
+    bias_d = None if bias is None else torch.from_numpy(bias.astype(np.float32)).cuda()
+    ard.ard_set_lstm_persistent(ctx.h, persistent)
+    launches = ard.ard_launch_count(ctx.h)
+    ard.ard_lstm_forward(ctx.h, pat, T, B, I, H, alpha, XH, Wnm, KH, bias_d, C, G, Z)
+    torch.cuda.synchronize()
+    launches = ard.ard_launch_count(ctx.h) - launches
+    assert ard.ard_last_device_status(ctx.h) == 0
+    return XH[1:, :, I:].float(), C, G, launches
+
+
+@pytest.mark.parametrize("T,B,I,H", [(6, 33, 128, 264), (4, 128, 192, 64), (3, 1, 64, 1024)])
+def test_persistent_forward_matches_the_oracle_and_the_per_step_path(T, B, I, H):
+    rng = np.random.default_rng(T * 1000 + B)
+    W = inputs.bf16_round(rng.uniform(-0.08, 0.08, size=(I + H, 4 * H)).astype(np.float32))
+    X = inputs.bf16_round(rng.standard_normal((T, B, I)).astype(np.float32))
+    bias = rng.uniform(-0.5, 0.5, size=4 * H).astype(np.float32)
+    Wnm = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+    ctx = Ctx(1 << 20)
+    try:
+        pat = ctx.pattern(ard.ARD_ROW, I + H, H)
+        for dp, b in [(1, 1), (2, 2), (3, 1), (5, 4), (16, 7)]:
+            ard.ard_pattern_set(ctx.h, pat, dp, b)
+            m = OP.row_mask(H, dp, b)
+            keep = OP.row_keep(H, dp, b)
+            h0 = inputs.bf16_round((rng.uniform(-1, 1, size=(B, H)) * m[None, :]).astype(np.float32))
+            c0 = (rng.uniform(-1, 1, size=(B, H)) * m[None, :]).astype(np.float32)
+            alpha = 1.7
+            Hp, Cp, Gp, lp = _run(ctx, pat, T, B, I, H, Wnm, X, bias, h0, c0, keep, alpha, 1)
+            Hs, Cs, Gs, ls = _run(ctx, pat, T, B, I, H, Wnm, X, bias, h0, c0, keep, alpha, 0)
+            assert lp == 1 and ls == 2 * T, (lp, ls)          # one launch against two per step
+            fw = OL.fwd(X, W, bias, m, alpha, h0=h0, c0=c0)
+            n = len(keep)
+            for name, Hg, Cg in (("persistent", Hp, Cp), ("per-step", Hs, Cs)):
+                assert OG.rel_fro(host(Hg), fw["Hs"]) <= TOL[ard.ARD_BF16], (name, dp, b)
+                assert OG.rel_fro(host(Cg[T])[:, :n], fw["cT"][:, keep]) <= TOL[ard.ARD_BF16], (name, dp, b)
+                assert bool(torch.all(Hg[:, :, torch.from_numpy(m == 0).cuda()] == 0)), (name, dp, b)
+            # saved gate activations and cell states feed BPTT: same layout, same values up to rounding
+            for t in range(T):
+                i_, f_, g_, o_ = fw["saved"][t][1:5]
+                ref = np.concatenate([i_[:, keep], f_[:, keep], g_[:, keep], o_[:, keep]], axis=1)
+                got = torch.cat([Gp[t, :, g * H:g * H + n] for g in range(4)], dim=1)
+                assert OG.rel_fro(host(got), ref) <= TOL[ard.ARD_BF16], (dp, b, t)
+            assert float((Hp - Hs).abs().max()) <= 0.05
+            assert float((Cp[1:, :, :n] - Cs[1:, :, :n]).abs().max()) <= 0.05
+    finally:
+        ctx.close()
+
+
+def test_layers_that_do_not_fit_use_the_per_step_path():
+    """Batch above 128 rows: the same call enqueues the per-step kernels."""
+    T, B, I, H = 2, 130, 64, 64
+    rng = np.random.default_rng(1)
+    W = inputs.bf16_round(rng.uniform(-0.08, 0.08, size=(I + H, 4 * H)).astype(np.float32))
+    X = inputs.bf16_round(rng.standard_normal((T, B, I)).astype(np.float32))
+    Wnm = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+    ctx = Ctx(1 << 20)
+    try:
+        pat = ctx.pattern(ard.ARD_ROW, I + H, H)
+        ard.ard_pattern_set(ctx.h, pat, 2, 1)
+        m, keep = OP.row_mask(H, 2, 1), OP.row_keep(H, 2, 1)
+        z = np.zeros((B, H), np.float32)
+        Hg, Cg, _, launches = _run(ctx, pat, T, B, I, H, Wnm, X, None, z, z, keep, 2.0, 1)
+        assert launches == 2 * T
+        fw = OL.fwd(X, W, None, m, 2.0)
+        assert OG.rel_fro(host(Hg), fw["Hs"]) <= TOL[ard.ARD_BF16]
+    finally:
+        ctx.close()
