@@ -822,9 +822,35 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
     DeviceGuard guard(ctx->device);
     const char* Wc = reinterpret_cast<const char*>(W);
     if (tc_eligible(ctx, pat, ARD_BF16, B, KH, H, XH, KH, W, ldw, C, H, 4) == ARD_OK &&
-        ((size_t)H * ldw * 2) % 16 == 0 && lstm_persistent_fits(ctx, B, I, H)) {
+        ((size_t)H * ldw * 2) % 16 == 0 && lstm_persistent_fits(ctx, B, H, H)) {
+      cudaStream_t s = (cudaStream_t)cuda_stream;
       const CUtensorMap* mapXH = nullptr;
       const CUtensorMap* mapW[4];
+      // 1. The input half for all steps at once: G[t][:, g*H + j] = x_t . W[g*H + keep[j]][0:I]  (T*B rows).
+      if (I > 0) {
+        TcArgs t;
+        GemmArgs g;
+        fill_common(g, ctx, pat, T * B, I, H, 1.0f);
+        g.A0 = XH; g.lda0 = KH; g.A1 = W; g.lda1 = ldw; g.out = G; g.ldo = 4 * H;
+        g.out_is_f32 = 1;
+        t.g = g;
+        t.ts = H;
+        t.bn = 0;
+        st = get_maps(ctx, XH, T * B, I, KH, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);
+        if (st != ARD_OK) return st;
+        t.mapA_indexed = 0;
+        for (int gate = 0; gate < 4; ++gate) {
+          st = get_maps(ctx, Wc + (size_t)gate * H * ldw * 2, H, I, ldw, H, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64,
+                        &t.mapB4[gate]);
+          if (st != ARD_OK) return st;
+          t.mapA4[gate] = t.mapA;
+        }
+        t.mapB = t.mapB4[0];
+        t.mapB_indexed = 1;
+        st = launch_lstm_tc(ctx, 0, t, s);
+        if (st != ARD_OK) return st;
+      }
+      // 2. The recurrence: one kernel, recurrent half of the weight resident in shared memory.
       st = get_maps(ctx, XH, (T + 1) * B, KH, KH, 0, MAP_PLAIN, 0, 64, 64, &mapXH);
       if (st != ARD_OK) return st;
       for (int gate = 0; gate < 4; ++gate) {
@@ -832,8 +858,8 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
                       &mapW[gate]);
         if (st != ARD_OK) return st;
       }
-      return launch_lstm_forward_persistent(ctx, pat, T, B, I, H, alpha, mapXH, mapW, XH, bias, C, G,
-                                            (cudaStream_t)cuda_stream);
+      return launch_lstm_forward_persistent(ctx, pat, T, B, I, H, I, H, I > 0 ? 1 : 0, alpha, mapXH, mapW, XH, bias, C,
+                                            G, s);
     }
   }
   for (int t = 0; t < T; ++t) {

@@ -149,9 +149,9 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
 ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStream_t s);
 
 // Whole-sequence LSTM forward in one cooperative kernel (lstm_persistent.cu).
-bool lstm_persistent_fits(ard_ctx* ctx, int B, int I, int H);
+bool lstm_persistent_fits(ard_ctx* ctx, int B, int klen, int H);
 ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H,
-                                          float alpha, const CUtensorMap* mapXH, const CUtensorMap* const mapW[4],
+                                          int kx0, int klen, int add_zx, float alpha, const CUtensorMap* mapXH, const CUtensorMap* const mapW[4],
                                           void* XH, const float* bias, float* C, float* G, cudaStream_t s);
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,

@@ -3,21 +3,26 @@
 //
 // The per-step path launches a gate product and a cell kernel per time step, and each launch costs
 // more than the 64-row product itself.  Here the recurrence runs inside one kernel:
+//   - the input half of the gate pre-activations does not depend on the recurrence: the caller computes
+//     x_t . W_x for all steps with one large product beforehand and leaves it where the gate activations
+//     of step t will be stored; the kernel adds it in its epilogue and handles the recurrent half only
+//     (it can also take the whole [x_t, h_{t-1}] row, at the price of a larger resident slice);
 //   - every CTA owns 8 kept hidden units, i.e. 32 gate columns (i|f|g|o x 8), and loads its slice of
-//     the weight, [32 rows][I+H] bf16, into shared memory once (TMA, rows b-1 + j*dp of each gate block
+//     the weight, [32 rows][H] bf16, into shared memory once (TMA, rows b-1 + j*dp of each gate block
 //     through the same strided descriptors the forward product uses);
-//   - per step it streams [x_t, h_{t-1}] (64-row TMA boxes) through a ring deep enough to hold the whole
-//     h half at once (the loads are latency-bound), multiplies it with the
+//   - per step it loads its contraction columns of [x_t, h_{t-1}] (64-row TMA boxes of 64 columns) into a
+//     buffer that holds all of them at once; the lanes of the producer warp issue one box each, so all
+//     loads of a step are in flight together (one thread issuing box after box, with a barrier hand-off
+//     per box, was measured at ~410 SM cycles per box, which paced the whole step); the boxes arrive on
+//     four barriers, so the MMAs of the first quarter start while the rest is in flight; it multiplies
+//     the row with the
 //     resident slice (tcgen05.mma, M = 128, N = 32, accumulator in tensor memory, double-buffered over
 //     steps);
 //   - four warps move the accumulator rows to shared memory, then all 14 compute warps apply the cell
 //     update to the (batch row, unit) pairs, keep c in registers, and write h_t (bf16) into the operand
 //     of step t+1 and, after signalling, c_t and the gate activations for BPTT;
-//   - the x half of a step does not depend on the recurrence, so its loads and MMAs run ahead; only
-//     the h half waits for the grid-wide barrier that says h_{t-1} is complete.
-// Measured on a B200 (T = 35, B = 64, I = H = 1024): 9.7 us per step against 17 us for the two launches of
-// the per-step path, the same for every period.  A step is paced by the activation loads, one 8 KiB block
-// every 0.29 us whatever the MMA shape: all CTAs read the same lines of [x_t, h_{t-1}] at the same time.
+//   - columns of x, if the kernel is given any, are loaded ahead; the h columns wait for the grid-wide
+//     barrier that says h_{t-1} is complete.
 // The grid barrier is an arrival counter in global memory: after its stores and a fence each CTA adds 1,
 // and the producer thread of each CTA polls for t * (number of CTAs with units) before it loads the
 // h half of step t.  The launch is cooperative, so all CTAs are resident; every wait is bounded (2 s)
@@ -30,11 +35,12 @@ namespace {
 constexpr int LP_UNITS = 8;                  // kept hidden units per CTA
 constexpr int LP_N = 4 * LP_UNITS;           // gate columns per CTA
 constexpr int LP_BK = 64;                    // contraction block: 64 bf16 = one 128-byte swizzle row
-constexpr int LP_MAX_STAGES = 16;
+constexpr int LP_MAX_BLOCKS = 32;            // contraction blocks per step: one lane of the producer warp each
+constexpr int LP_GROUPS = 4;                 // the blocks of a step arrive on this many barriers
 constexpr int LP_ROW_BOX = 64 * LP_BK * 2;   // one TMA box of the activations: 64 batch rows x 64 columns
 constexpr int LP_W_BLOCK = LP_N * LP_BK * 2; // one contraction block of the resident weight slice
-constexpr int LP_THREADS = 512;              // warps 0-13 cell update (0-3 also read TMEM: lane quadrant = warp),
-constexpr int LP_MATH = 448;                 //   warp 14 TMA producer, warp 15 MMA issuer
+constexpr int LP_THREADS = 512;              // warps 0-10 cell update (0-3 also read TMEM: lane quadrant = warp),
+constexpr int LP_MATH = 352;                 //   warp 11 TMA producer, warps 12-15 MMA issuers (one per group)
 constexpr int LP_ZS_LD = LP_N + 1;           // staged pre-activations: [128 rows][33] floats
 constexpr int LP_ZS_BYTES = 128 * LP_ZS_LD * 4;
 constexpr int LP_PAIRS_MAX = (128 * LP_UNITS + LP_MATH - 1) / LP_MATH;  // (row, unit) pairs per thread
@@ -44,7 +50,8 @@ struct LstmFwdParams {
   const CUtensorMap* mapW[4];  // per gate: table over (dp, b) of strided-row maps, boxes of 8 rows x 64 columns
   const int32_t* hdr;
   int T, B, I, H;
-  int stages;         // depth of the activation ring (<= LP_MAX_STAGES)
+  int kx0, klen;      // contraction columns [kx0, kx0 + klen) of [x | h] this kernel multiplies
+  int add_zx;         // the products of the other columns are waiting in G[t] (same layout as the gates)
   float alpha;
   __nv_bfloat16* XH;
   const float* bias;  // [4][H] or nullptr
@@ -89,44 +96,42 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
   uint8_t* smem = smem_raw + (base - raw_addr);
 
   const int KH = p.I + p.H;
-  const int nkb = (KH + LP_BK - 1) / LP_BK;
-  // The activation ring comes first and the weight slice right after it: a stage holds one or two
+  const int nkb = (p.klen + LP_BK - 1) / LP_BK;
+  // The activation row buffer comes first and the weight slice right after it: a block holds one or two
   // 64-row boxes, the MMA always reads 128 rows, and for a batch of at most 64 rows the upper half of
-  // what it reads is the next stage (or the start of the weight slice); those accumulator rows are
+  // what it reads is the next block (or the start of the weight slice); those accumulator rows are
   // never used.
-  const int STAGES = p.stages;
   const int row_boxes = (p.B + 63) / 64;
-  const uint32_t a_stage = (uint32_t)row_boxes * LP_ROW_BOX;
+  const uint32_t a_block = (uint32_t)row_boxes * LP_ROW_BOX;
   const uint32_t sA = base;
-  const uint32_t sW = base + (uint32_t)STAGES * a_stage;      // nkb blocks of 4 KiB
+  const uint32_t sW = base + (uint32_t)nkb * a_block;         // nkb blocks of 4 KiB
   float* zs = reinterpret_cast<float*>(smem + (sW - base) + (size_t)nkb * LP_W_BLOCK);
-  const uint32_t bar_base = sW + (uint32_t)nkb * LP_W_BLOCK + LP_ZS_BYTES;  // full[16], empty[16], tfull[2], tempty[2], wfull
-  auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (LP_MAX_STAGES + s); };
-  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * LP_MAX_STAGES + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * LP_MAX_STAGES + 2 + a); };
-  const uint32_t wfull_bar = bar_base + 8u * (2 * LP_MAX_STAGES + 4);
-  uint8_t* misc = smem + (bar_base - base) + 8 * (2 * LP_MAX_STAGES + 5);
+  const uint32_t bar_base = sW + (uint32_t)nkb * LP_W_BLOCK + LP_ZS_BYTES;  // gfull[4], tfull[2], tempty[2], wfull
+  auto gfull_bar = [&](int g) { return bar_base + 8u * g; };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (LP_GROUPS + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (LP_GROUPS + 2 + a); };
+  const uint32_t wfull_bar = bar_base + 8u * (LP_GROUPS + 4);
+  const uint32_t hready_bar = bar_base + 8u * (LP_GROUPS + 5);  // h_{t-1} is complete (relayed from the grid barrier)
+  uint8_t* misc = smem + (bar_base - base) + 8 * (LP_GROUPS + 6);
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+  const int gsz = (nkb + LP_GROUPS - 1) / LP_GROUPS;          // blocks per arrival group
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
-    }
+    for (int g = 0; g < LP_GROUPS; ++g) mbar_init(gfull_bar(g), 1);
     for (int a = 0; a < 2; ++a) {
-      mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4);  // one arrival per epilogue warp
+      mbar_init(tfull_bar(a), LP_GROUPS);  // one commit per MMA issuer
+      mbar_init(tempty_bar(a), 4);         // one arrival per TMEM-reading warp
     }
     mbar_init(wfull_bar, 1);
+    mbar_init(hready_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 15) {
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), 2 * LP_N);
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), 2 * LP_GROUPS * LP_N);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -139,70 +144,91 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
   const int n_active = (n_keep + LP_UNITS - 1) / LP_UNITS;  // CTAs that own units (the others only tear down)
   const int j0 = (int)blockIdx.x * LP_UNITS;                // first kept unit (compact index) of this CTA
   const bool active = (int)blockIdx.x < n_active;
-  const int xblocks = p.I / LP_BK;                          // contraction blocks that hold only x columns
+  const int xblocks = p.I > p.kx0 ? (p.I - p.kx0) / LP_BK : 0;  // contraction blocks that hold only x columns
 
   if (active) {
-    if (warp == 14) {
-      // ===================== TMA producer =====================
-      if (lane == 0) {
-        const int e = p.hdr[HDR_MAPIDX];
-        tensormap_acquire(p.mapXH);
+    if (warp == 11) {
+      // ===================== weight loader and barrier relay =====================
+      // Loads the weight slice (lane = contraction block), then relays the grid barrier of every step to
+      // the warps of this CTA through a shared-memory barrier.
+      const int e = p.hdr[HDR_MAPIDX];
+      const int kb = lane;
+      if (kb < nkb) {
 #pragma unroll
         for (int g = 0; g < 4; ++g) tensormap_acquire(p.mapW[g] + e);
-        // the weight slice, once
-        mbar_arrive_expect_tx(wfull_bar, (uint32_t)nkb * LP_W_BLOCK);
-        for (int kb = 0; kb < nkb; ++kb)
+      }
+      if (lane == 0) mbar_arrive_expect_tx(wfull_bar, (uint32_t)nkb * LP_W_BLOCK);
+      __syncwarp();
+      if (kb < nkb) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g)
-            tma_load_2d(sW + kb * LP_W_BLOCK + g * (LP_UNITS * LP_BK * 2), p.mapW[g] + e, wfull_bar, kb * LP_BK, j0);
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        for (int t = 0; t < p.T && ok; ++t) {
-          for (int kb = 0; kb < nkb; ++kb) {
-            if (kb == xblocks && t > 0) {
-              // the rest of this step reads h_{t-1}: every CTA with units has to have stored its part
-              if (!grid_wait(p.bar, (unsigned)t * (unsigned)n_active, abort_flag, p.status)) { ok = false; break; }
-              asm volatile("fence.proxy.async;" ::: "memory");  // the loads below go through the async proxy
-            }
-            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
-            mbar_arrive_expect_tx(full_bar(stage), a_stage);
-            for (int rb = 0; rb < row_boxes; ++rb)
-              tma_load_2d(sA + stage * a_stage + rb * LP_ROW_BOX, p.mapXH, full_bar(stage), kb * LP_BK,
-                          t * p.B + rb * 64);
-            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-          }
+        for (int g = 0; g < 4; ++g)
+          tma_load_2d(sW + kb * LP_W_BLOCK + g * (LP_UNITS * LP_BK * 2), p.mapW[g] + e, wfull_bar, p.kx0 + kb * LP_BK,
+                      j0);
+      }
+      if (lane == 0) {
+        for (int t = 1; t < p.T; ++t) {
+          // h_{t-1} is complete when every CTA with units has arrived t times
+          if (!grid_wait(p.bar, (unsigned)t * (unsigned)n_active, abort_flag, p.status)) break;
+          mbar_arrive(hready_bar);
         }
       }
-    } else if (warp == 15) {
-      // ===================== MMA issuer =====================
-      if (lane == 0) {
-        const uint32_t idesc = make_idesc(LP_N, false, false, 128);
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = mbar_wait(wfull_bar, 0u, abort_flag, p.status);
-        for (int t = 0; t < p.T && ok; ++t) {
-          const int acc = t & 1;
-          if (!mbar_wait(tempty_bar(acc), ((uint32_t)(t >> 1) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * LP_N);
-          for (int kb = 0; kb < nkb; ++kb) {
-            if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t a0 = sA + stage * a_stage, b0 = sW + kb * LP_W_BLOCK;
-#pragma unroll
-            for (int s = 0; s < LP_BK / 16; ++s)
-              tc_mma_bf16(d_tmem, make_desc(a0 + s * 32, 16, 1024), make_desc(b0 + s * 32, 16, 1024), idesc,
-                          (kb | s) != 0 ? 1u : 0u);
-            tc_commit(empty_bar(stage));
-            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-          }
-          if (!ok) break;
-          tc_commit(tfull_bar(acc));
+    } else if (warp >= 12) {
+      // ===================== loaders and MMA issuers: warp 12 + g owns the contraction blocks of group g =====================
+      // Lanes 0 .. gsz-1 issue one TMA box each (a single thread issuing box after box was measured at
+      // ~410 cycles per box, and the lanes of ONE warp still issue one after the other, ~70 cycles each,
+      // so the four groups are issued by four warps side by side).  Lane 0 then issues the MMAs of the
+      // group: a tcgen05.mma this narrow (N = 32) costs ~110 cycles to issue whatever its shape, so one
+      // thread issuing all 4 * nkb of a step would pace the step; the four warps issue their quarters side
+      // by side into four accumulators, which the epilogue adds.
+      const int g = warp - 12;
+      const int kb0 = g * gsz, kb1 = min(nkb, kb0 + gsz);
+      const int kb = kb0 + lane;
+      const bool mine = kb < kb1;
+      if (mine) tensormap_acquire(p.mapXH);
+      const uint32_t idesc = make_idesc(LP_N, false, false, 128);
+      bool ok = (lane != 0) || mbar_wait(wfull_bar, 0u, abort_flag, p.status);
+      for (int t = 0; t < p.T; ++t) {
+        const int acc = t & 1;
+        // this group's part of the row buffer is free once the MMAs of the previous step have completed
+        if (ok && t > 0 && !mbar_wait(tfull_bar((t - 1) & 1), (uint32_t)((t - 1) >> 1) & 1u, abort_flag, p.status)) ok = false;
+        if (!__all_sync(0xffffffffu, ok)) break;
+        if (lane == 0 && kb0 < kb1) mbar_arrive_expect_tx(gfull_bar(g), (uint32_t)(kb1 - kb0) * a_block);
+        __syncwarp();
+        auto issue = [&]() {
+          for (int rb = 0; rb < row_boxes; ++rb)
+            tma_load_2d(sA + kb * a_block + rb * LP_ROW_BOX, p.mapXH, gfull_bar(g), p.kx0 + kb * LP_BK,
+                        t * p.B + rb * 64);
+        };
+        if (mine && kb < xblocks) issue();  // columns of x do not depend on the recurrence
+        if (t > 0 && kb1 > xblocks) {
+          // the other columns are h_{t-1}
+          if (!mbar_wait(hready_bar, (uint32_t)(t - 1) & 1u, abort_flag, p.status)) ok = false;
+          if (!__all_sync(0xffffffffu, ok)) break;
+          asm volatile("fence.proxy.async.global;" ::: "memory");  // generic-proxy stores of other CTAs -> TMA reads
         }
+        if (mine && kb >= xblocks) issue();
+        if (lane == 0) {
+          if (!mbar_wait(tempty_bar(acc), ((uint32_t)(t >> 1) & 1u) ^ 1u, abort_flag, p.status)) ok = false;
+          if (ok && kb0 < kb1) {
+            if (!mbar_wait(gfull_bar(g), (uint32_t)t & 1u, abort_flag, p.status)) ok = false;
+            if (ok) {
+              tc_fence_after();
+              const uint32_t d_tmem = tmem_base + (uint32_t)((acc * LP_GROUPS + g) * LP_N);
+              for (int k2 = kb0; k2 < kb1; ++k2) {
+                const uint32_t a0 = sA + k2 * a_block, b0 = sW + k2 * LP_W_BLOCK;
+#pragma unroll
+                for (int s = 0; s < LP_BK / 16; ++s)
+                  tc_mma_bf16(d_tmem, make_desc(a0 + s * 32, 16, 1024), make_desc(b0 + s * 32, 16, 1024), idesc,
+                              (k2 != kb0 || s != 0) ? 1u : 0u);
+              }
+            }
+          }
+          if (ok) tc_commit(tfull_bar(acc));  // this quarter is complete; with all four, the row buffer may be overwritten
+        }
+        __syncwarp();
       }
     } else {
-      // ===================== cell update (warps 0-13) =====================
+      // ===================== cell update (warps 0-10) =====================
       const int tid = threadIdx.x;  // 0 .. LP_MATH-1
       const size_t ldxh = (size_t)KH;
       const int npairs = p.B * LP_UNITS;            // (batch row, unit) pairs of this CTA; pair q = row * 8 + k
@@ -217,15 +243,42 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
       bool ok = true;
       for (int t = 0; t < p.T && ok; ++t) {
         const int acc = t & 1;
+        // what does not depend on the recurrence is fetched before the wait: x_t . W_x and the bias
+        float zadd[LP_PAIRS_MAX][4];
+#pragma unroll
+        for (int i = 0; i < LP_PAIRS_MAX; ++i) {
+          const int q = tid + i * LP_MATH;
+          const int row = q >> 3, k = q & 7;
+          zadd[i][0] = zadd[i][1] = zadd[i][2] = zadd[i][3] = 0.f;
+          if (q < npairs && k < nvalid) {
+            if (p.add_zx) {  // left in the slot of this step's gate activations
+              const float* zx = p.G + ((size_t)t * p.B + row) * 4 * p.H + j0 + k;
+#pragma unroll
+              for (int g = 0; g < 4; ++g) zadd[i][g] = __ldcg(zx + (size_t)g * p.H);
+            }
+            if (p.bias) {
+              const int u = bb + (j0 + k) * dp;
+#pragma unroll
+              for (int g = 0; g < 4; ++g) zadd[i][g] += p.bias[g * p.H + u];
+            }
+          }
+        }
         if (warp < 4) {
           // accumulator rows -> shared memory
           if (!mbar_wait(tfull_bar(acc), (uint32_t)(t >> 1) & 1u, abort_flag, p.status)) ok = false;
           if (ok) {
             tc_fence_after();
-            const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * LP_N);
-            uint32_t z[32];
+            const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(acc * LP_GROUPS * LP_N);
+            const int ngroups = (nkb + gsz - 1) / gsz;  // accumulators that received MMAs
+            uint32_t z[32], y[32];
             tmem_ld32(t_row, z);
             tmem_ld_wait();
+            for (int c = 1; c < ngroups; ++c) {
+              tmem_ld32(t_row + (uint32_t)(c * LP_N), y);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) z[i] = __float_as_uint(__uint_as_float(z[i]) + __uint_as_float(y[i]));
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));  // the accumulator is in registers now
@@ -237,7 +290,7 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
           }
         }
         // every compute thread learns about a failed wait through the flag in shared memory
-        asm volatile("bar.sync 2, 448;" ::: "memory");
+        asm volatile("bar.sync 2, 352;" ::: "memory");
         if (*abort_flag) { ok = false; break; }
         // Cell update (Sec. 7).  h first, because the other CTAs wait for it; c_t and the gate
         // activations, which only BPTT reads, after the CTA has signalled.
@@ -249,13 +302,8 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
           if (q < npairs && k < nvalid) {
             const int u = bb + (j0 + k) * dp;
             const float* zr = zs + row * LP_ZS_LD;
-            float zi = zr[k], zf = zr[LP_UNITS + k], zg = zr[2 * LP_UNITS + k], zo = zr[3 * LP_UNITS + k];
-            if (p.bias) {
-              zi += p.bias[u];
-              zf += p.bias[p.H + u];
-              zg += p.bias[2 * p.H + u];
-              zo += p.bias[3 * p.H + u];
-            }
+            const float zi = zr[k] + zadd[i][0], zf = zr[LP_UNITS + k] + zadd[i][1];
+            const float zg = zr[2 * LP_UNITS + k] + zadd[i][2], zo = zr[3 * LP_UNITS + k] + zadd[i][3];
             gi[i] = sigmoid_fast(zi);
             gf[i] = sigmoid_fast(zf);
             gg[i] = tanh_fast(zg);
@@ -265,7 +313,7 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
           }
         }
         // publish h_t: all stores of the CTA, then one release-add for the CTA
-        asm volatile("bar.sync 1, 448;" ::: "memory");
+        asm volatile("bar.sync 1, 352;" ::: "memory");
         if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
 #pragma unroll
         for (int i = 0; i < LP_PAIRS_MAX; ++i) {
@@ -290,57 +338,51 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
   if (warp == 15) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, 2 * LP_N);
+    tmem_dealloc(tmem_base, 2 * LP_GROUPS * LP_N);
   }
 }
 
 }  // namespace
 
-// Depth of the activation ring and dynamic shared memory for a layer with I + H = KH and batch B:
-// the weight slice is fixed, the ring takes what is left (at most LP_MAX_STAGES stages).
-static int lstm_fwd_stages(int KH, int B) {
-  const int nkb = (KH + LP_BK - 1) / LP_BK;
-  const long long fixed = (long long)nkb * LP_W_BLOCK + LP_ZS_BYTES + 8 * (2 * LP_MAX_STAGES + 5) + 16 + 1024;
-  const long long a_stage = (long long)((B + 63) / 64) * LP_ROW_BOX;
-  long long st = (227 * 1024 - fixed) / a_stage;
-  return (int)(st > LP_MAX_STAGES ? LP_MAX_STAGES : st);
-}
-static size_t lstm_fwd_smem_bytes(int KH, int B) {
-  const int nkb = (KH + LP_BK - 1) / LP_BK;
-  return (size_t)nkb * LP_W_BLOCK + (size_t)lstm_fwd_stages(KH, B) * ((B + 63) / 64) * LP_ROW_BOX + LP_ZS_BYTES +
-         8 * (2 * LP_MAX_STAGES + 5) + 16 + 1024;
+// Dynamic shared memory for klen contraction columns and batch B: the row buffer, the weight slice, the
+// staged pre-activations, barriers, and slack for the 1024-byte alignment.
+static size_t lstm_fwd_smem_bytes(int klen, int B) {
+  const size_t nkb = (size_t)(klen + LP_BK - 1) / LP_BK;
+  return nkb * ((B + 63) / 64) * LP_ROW_BOX + nkb * LP_W_BLOCK + LP_ZS_BYTES + 8 * (LP_GROUPS + 6) + 16 + 1024;
 }
 
 // Can the whole-sequence kernel run this layer on this device?  (Shared memory for the weight slice, one
 // CTA per 8 hidden units all resident at once, one 128-row tile of batch.)
-bool lstm_persistent_fits(ard_ctx* ctx, int B, int I, int H) {
-  if (B < 1 || B > 128 || H < 1) return false;
-  if (lstm_fwd_stages(I + H, B) < 4) return false;  // the weight slice leaves too little room for the ring
-  const size_t smem = lstm_fwd_smem_bytes(I + H, B);
-  static int blocks_per_sm[64] = {};
+bool lstm_persistent_fits(ard_ctx* ctx, int B, int klen, int H) {
+  if (B < 1 || B > 128 || H < 1 || klen < 1) return false;
+  if ((klen + LP_BK - 1) / LP_BK > LP_MAX_BLOCKS) return false;
+  const size_t smem = lstm_fwd_smem_bytes(klen, B);
+  if (smem > 227 * 1024) return false;  // the row of activations and the weight slice must both be resident
+  static int probed[64] = {};
   const int dev = ctx->device & 63;
-  if (blocks_per_sm[dev] == 0) {
-    if (cudaFuncSetAttribute(ard_lstm_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-        cudaSuccess)
-      return false;
+  if (probed[dev] == 0) {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, ard_lstm_forward_kernel, LP_THREADS, smem) != cudaSuccess || n < 1)
-      n = -1;
-    blocks_per_sm[dev] = n;
+    if (cudaFuncSetAttribute(ard_lstm_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, ard_lstm_forward_kernel, LP_THREADS, smem) != cudaSuccess ||
+        n < 1)
+      probed[dev] = -1;
+    else
+      probed[dev] = 1;
   }
-  if (blocks_per_sm[dev] < 1) return false;
-  return (H + LP_UNITS - 1) / LP_UNITS <= ctx->sm_count;  // one CTA per SM (the slice fills shared memory)
+  if (probed[dev] < 1) return false;
+  return (H + LP_UNITS - 1) / LP_UNITS <= ctx->sm_count;  // one CTA per SM, all resident at once
 }
 
 ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H,
-                                          float alpha, const CUtensorMap* mapXH, const CUtensorMap* const mapW[4],
+                                          int kx0, int klen, int add_zx, float alpha, const CUtensorMap* mapXH, const CUtensorMap* const mapW[4],
                                           void* XH, const float* bias, float* C, float* G, cudaStream_t s) {
   LstmFwdParams p;
   p.mapXH = mapXH;
   for (int g = 0; g < 4; ++g) p.mapW[g] = mapW[g];
   p.hdr = pat->d_hdr;
   p.T = T; p.B = B; p.I = I; p.H = H;
-  p.stages = lstm_fwd_stages(I + H, B);
+  p.kx0 = kx0; p.klen = klen; p.add_zx = add_zx;
   p.alpha = alpha;
   p.XH = reinterpret_cast<__nv_bfloat16*>(XH);
   p.bias = bias;
@@ -354,7 +396,7 @@ ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((H + LP_UNITS - 1) / LP_UNITS);  // sized for dp = 1; CTAs without units leave at once
   cfg.blockDim = dim3(LP_THREADS);
-  cfg.dynamicSmemBytes = lstm_fwd_smem_bytes(I + H, B);
+  cfg.dynamicSmemBytes = lstm_fwd_smem_bytes(klen, B);
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs resident: they wait for one another

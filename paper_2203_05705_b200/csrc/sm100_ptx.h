@@ -39,14 +39,31 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 
+// One poll of the barrier.  With a suspend-time hint the hardware parks the thread until the phase
+// completes or about `hint_ns` have passed, so a waiting thread neither spins on the barrier nor
+// competes for issue slots.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n\t"
+      "selp.b32 %0, 1, 0, P;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait.  Returns false if the limit expired or another role already gave up.
+// Reading %globaltimer costs a few hundred nanoseconds, so the clock is consulted only after a first
+// long poll has failed; a wait that is merely a pipeline hand-off never touches it.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  constexpr uint32_t HINT_NS = 1000000u;  // 1 ms per poll; the abort flag is looked at between polls
   if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait_hint(bar, parity, HINT_NS)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 32; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait_hint(bar, parity, HINT_NS)) return true;
     if (*abort_flag) return false;
     if (global_ns() - t0 > WAIT_LIMIT_NS) {
       *abort_flag = 1;

@@ -58,7 +58,7 @@ def test_persistent_forward_matches_the_oracle_and_the_per_step_path(T, B, I, H)
             alpha = 1.7
             Hp, Cp, Gp, lp = _run(ctx, pat, T, B, I, H, Wnm, X, bias, h0, c0, keep, alpha, 1)
             Hs, Cs, Gs, ls = _run(ctx, pat, T, B, I, H, Wnm, X, bias, h0, c0, keep, alpha, 0)
-            assert lp == 1 and ls == 2 * T, (lp, ls)          # one launch against two per step
+            assert lp == 2 and ls == 2 * T, (lp, ls)          # input-half product + recurrence against two per step
             fw = OL.fwd(X, W, bias, m, alpha, h0=h0, c0=c0)
             n = len(keep)
             for name, Hg, Cg in (("persistent", Hp, Cp), ("per-step", Hs, Cs)):
