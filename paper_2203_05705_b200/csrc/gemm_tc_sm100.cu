@@ -680,6 +680,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
     if (lane == 0 && rank == 0) {
+      // descriptors without the start address: K-major (LBO unused, SBO 1024) or MN-major (LBO 8 KiB, SBO 1024)
+      const uint64_t desc_a_hi = A_MN ? make_desc(0, 64 * BK * 2, 1024) : make_desc(0, 16, 1024);
+      const uint64_t desc_b_hi = B_MN ? make_desc(0, 64 * BK * 2, 1024) : make_desc(0, 16, 1024);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -696,15 +699,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
-          tc_fence_after();
+          // This thread's instruction stream is what feeds the tensor pipe: the descriptors of a block are
+          // the stage's descriptor plus a constant per 16-deep step (the start-address field counts 16-byte
+          // units: K-major 32 bytes = 2 per step, MN-major 16 k-rows = 2048 bytes = 128 per step).
           const uint32_t sA = base + stage * L::STAGE_BYTES;
-          const uint32_t sB = sA + L::A_BYTES;
+          const uint64_t ad0 = desc_a_hi | (uint64_t)((sA & 0x3FFFFu) >> 4);
+          const uint64_t bd0 = desc_b_hi | (uint64_t)(((sA + L::A_BYTES) & 0x3FFFFu) >> 4);
 #pragma unroll
           for (int s = 0; s < BK / 16; ++s) {
-            // K-major: advance 16 elements = 32 bytes inside the swizzled row.
-            // MN-major: advance 16 k-rows = 2048 bytes.
-            const uint64_t ad = A_MN ? make_desc(sA + s * 2048, 64 * BK * 2, 1024) : make_desc(sA + s * 32, 16, 1024);
-            const uint64_t bd = B_MN ? make_desc(sB + s * 2048, 64 * BK * 2, 1024) : make_desc(sB + s * 32, 16, 1024);
+            const uint64_t ad = ad0 + (uint64_t)(s * (A_MN ? 128 : 2));
+            const uint64_t bd = bd0 + (uint64_t)(s * (B_MN ? 128 : 2));
             const uint32_t accum = (kb != kb_begin || s != 0) ? 1u : 0u;
             if (CTAS == 2) tc_mma_bf16_pair(d_tmem, ad, bd, idesc, accum);
             else tc_mma_bf16(d_tmem, ad, bd, idesc, accum);
