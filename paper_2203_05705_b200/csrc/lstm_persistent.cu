@@ -214,12 +214,12 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
             if (ok) {
               tc_fence_after();
               const uint32_t d_tmem = tmem_base + (uint32_t)((acc * LP_GROUPS + g) * LP_N);
-              for (int k2 = kb0; k2 < kb1; ++k2) {
-                const uint32_t a0 = sA + k2 * a_block, b0 = sW + k2 * LP_W_BLOCK;
+              // descriptors by addition: the start-address field counts 16-byte units
+              uint64_t ad = make_desc(sA + kb0 * a_block, 16, 1024), bd = make_desc(sW + kb0 * LP_W_BLOCK, 16, 1024);
+              for (int k2 = kb0; k2 < kb1; ++k2, ad += a_block >> 4, bd += LP_W_BLOCK >> 4) {
 #pragma unroll
                 for (int s = 0; s < LP_BK / 16; ++s)
-                  tc_mma_bf16(d_tmem, make_desc(a0 + s * 32, 16, 1024), make_desc(b0 + s * 32, 16, 1024), idesc,
-                              (k2 != kb0 || s != 0) ? 1u : 0u);
+                  tc_mma_bf16(d_tmem, ad + 2 * s, bd + 2 * s, idesc, (k2 != kb0 || s != 0) ? 1u : 0u);
               }
             }
           }
