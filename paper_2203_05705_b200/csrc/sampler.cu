@@ -40,8 +40,14 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
                   unsigned long long iteration, uint32_t stream_id, int forced_dp, int forced_b, int kind,
                   int units, int Tr, int Tc, int ts) {
   __shared__ int s_dp, s_b;
+  __shared__ unsigned long long s_cdf[64];
   pdl_launch_dependents();
   pdl_wait_prior_grids();  // earlier kernels may still be reading the lists this kernel rewrites
+  // The cumulative table is searched by one thread; short tables are fetched by all threads at once first,
+  // so that the search does not pay one global-memory round trip per probe.
+  const bool cdf_smem = forced_dp <= 0 && ndp <= 64;
+  if (cdf_smem && (int)threadIdx.x < ndp) s_cdf[threadIdx.x] = cdf[threadIdx.x];
+  __syncthreads();
   if (threadIdx.x == 0) {
     int dp, b;
     if (forced_dp > 0) {
@@ -55,7 +61,8 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
       const unsigned long long r0 = c[0];
       while (lo < hi) {
         int mid = (lo + hi) >> 1;
-        if (r0 < cdf[mid]) hi = mid; else lo = mid + 1;
+        const unsigned long long cm = cdf_smem ? s_cdf[mid] : cdf[mid];
+        if (r0 < cm) hi = mid; else lo = mid + 1;
       }
       dp = lo + 1;
       b = 1 + (int)(((unsigned long long)c[1] * (unsigned long long)dp) >> 32);
@@ -90,15 +97,21 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
     if (lim > b - 1) cnt = (int)((lim - 1 - (b - 1)) / dp) + 1;
     row_ptr[r] = cnt;
   }
-  // Group by tile-column: count, prefix-sum, fill.  The running sum lives in shared memory when the
-  // grid is narrow enough (one thread scans it; a dependent chain through global memory would cost
-  // a round trip per column).
+  // Group by tile-column: count, prefix-sum, fill.  A warp takes a column at a time with its lanes across
+  // the tile-rows, so a column costs Tr/32 ballots instead of a serial walk; the running sum over the
+  // columns lives in shared memory when the grid is narrow enough (a dependent chain through global
+  // memory would cost a round trip per column).
   __shared__ int s_cnt[SCAN_CAP];
   const bool in_smem = Tc <= SCAN_CAP;
-  for (int c = threadIdx.x; c < Tc; c += SAMPLER_THREADS) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = SAMPLER_THREADS / 32;
+  auto kept = [&](int r, int c) {
+    const int lin = r * Tc + c - (b - 1);
+    return r < Tr && lin >= 0 && lin % dp == 0;
+  };
+  for (int c = warp; c < Tc; c += nwarps) {
     int cnt = 0;
-    for (int r = 0; r < Tr; ++r) cnt += ((r * Tc + c - (b - 1)) % dp == 0) && (r * Tc + c >= b - 1);
-    if (in_smem) s_cnt[c] = cnt; else col_ptr[c + 1] = cnt;
+    for (int r0 = 0; r0 < Tr; r0 += 32) cnt += __popc(__ballot_sync(0xffffffffu, kept(r0 + lane, c)));
+    if (lane == 0) { if (in_smem) s_cnt[c] = cnt; else col_ptr[c + 1] = cnt; }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -115,10 +128,14 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
     for (int c = threadIdx.x; c < Tc; c += SAMPLER_THREADS) col_ptr[c] = s_cnt[c];
     if (threadIdx.x == 0) col_ptr[Tc] = n_keep;
   }
-  for (int c = threadIdx.x; c < Tc; c += SAMPLER_THREADS) {
+  for (int c = warp; c < Tc; c += nwarps) {
     int o = in_smem ? s_cnt[c] : col_ptr[c];
-    for (int r = 0; r < Tr; ++r)
-      if ((r * Tc + c >= b - 1) && ((r * Tc + c - (b - 1)) % dp == 0)) col_idx[o++] = r;
+    for (int r0 = 0; r0 < Tr; r0 += 32) {
+      const bool k = kept(r0 + lane, c);
+      const unsigned m = __ballot_sync(0xffffffffu, k);
+      if (k) col_idx[o + __popc(m & ((1u << lane) - 1u))] = r0 + lane;  // ascending rows
+      o += __popc(m);
+    }
   }
 }
 
