@@ -195,6 +195,7 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->lstm_persistent = 1;
   if (const char* e = getenv("ARD_LSTM_PERSISTENT")) ctx->lstm_persistent = atoi(e) ? 1 : 0;
   ctx->d_grid_bar = nullptr;
+  ctx->d_lstm_partial = nullptr;
   if (const char* e = getenv("ARD_PDL")) ctx->use_pdl = atoi(e) ? 1 : 0;
   ctx->sk_min_blocks = 16;
   if (const char* e = getenv("ARD_STREAM_K")) ctx->stream_k = atoi(e);
@@ -234,7 +235,9 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
     if (cudaMalloc(&ctx->d_sk_ws, ws_bytes) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->d_sk_cnt), cnt_bytes) != cudaSuccess ||
         cudaMemset(ctx->d_sk_cnt, 0, cnt_bytes) != cudaSuccess ||
-        cudaMalloc(reinterpret_cast<void**>(&ctx->d_grid_bar), 256) != cudaSuccess) {
+        cudaMalloc(reinterpret_cast<void**>(&ctx->d_grid_bar), 256) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&ctx->d_lstm_partial), lstm_bwd_partial_bytes(ctx->sm_count)) != cudaSuccess) {
+      if (ctx->d_lstm_partial) cudaFree(ctx->d_lstm_partial);
       if (ctx->d_grid_bar) cudaFree(ctx->d_grid_bar);
       if (ctx->d_sk_ws) cudaFree(ctx->d_sk_ws);
       if (ctx->d_sk_cnt) cudaFree(ctx->d_sk_cnt);
@@ -259,6 +262,7 @@ ard_status ard_destroy(ard_ctx* ctx) {
   if (ctx->d_sk_ws) cudaFree(ctx->d_sk_ws);
   if (ctx->d_sk_cnt) cudaFree(ctx->d_sk_cnt);
   if (ctx->d_grid_bar) cudaFree(ctx->d_grid_bar);
+  if (ctx->d_lstm_partial) cudaFree(ctx->d_lstm_partial);
   if (ctx->d_status) cudaFree(ctx->d_status);
   delete ctx;
   return ARD_OK;
@@ -724,6 +728,38 @@ ard_status ard_lstm_gate_gemm(ard_ctx* ctx, const ard_pattern* pat, int B, int K
   return launch_lstm_tc(ctx, 0, t, s);
 }
 
+// Tensor-core form of the adjoint gate product over `kout` consecutive columns of [x | h]:
+//   out[:, k] (+)= sum_g sum_j dZ[:, g*ldz_gate + j] * Wcols[g*H + keep[j]][k],   k < kout,
+// where Wcols points at the first of those columns of the weight.  The caller has checked eligibility.
+static ard_status lstm_gate_gemm_bwd_tc(ard_ctx* ctx, const ard_pattern* pat, int B, int kout, int H, const void* dZ,
+                                        int ldz_gate, const void* Wcols, int ldw, float* out, int ldo, int accumulate,
+                                        cudaStream_t s) {
+  const char* Wc = reinterpret_cast<const char*>(Wcols);
+  const char* dZc = reinterpret_cast<const char*>(dZ);
+  TcArgs t;
+  GemmArgs g;
+  fill_common(g, ctx, pat, B, kout, H, 1.0f);
+  g.A0 = dZ; g.lda0 = 4 * ldz_gate; g.A1 = Wcols; g.lda1 = ldw; g.out = out; g.ldo = ldo;
+  g.flag0 = 1;
+  g.out_is_f32 = 1;
+  g.accumulate = accumulate ? 1 : 0;
+  t.g = g;
+  t.ts = ldz_gate;
+  t.bn = ctx->force_bn;
+  for (int gate = 0; gate < 4; ++gate) {
+    ard_status st = get_maps(ctx, dZc + (size_t)gate * ldz_gate * 2, B, H, 4 * ldz_gate, H, MAP_COMPACT_COLS,
+                             pat->dp_bound, 128, 64, &t.mapA4[gate]);
+    if (st != ARD_OK) return st;
+    st = get_maps(ctx, Wc + (size_t)gate * H * ldw * 2, H, kout, ldw, H, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64,
+                  &t.mapB4[gate]);
+    if (st != ARD_OK) return st;
+  }
+  t.mapA = t.mapA4[0];
+  t.mapB = t.mapB4[0];
+  t.mapA_indexed = t.mapB_indexed = 1;
+  return launch_lstm_tc(ctx, 1, t, s);
+}
+
 ard_status ard_lstm_gate_gemm_bwd(ard_ctx* ctx, const ard_pattern* pat, int B, int KH, int H, const void* dZ,
                                   int ldz_gate, const void* W, int ldw, float* dXH, int lddxh, int accumulate,
                                   void* cuda_stream) {
@@ -751,28 +787,7 @@ ard_status ard_lstm_gate_gemm_bwd(ard_ctx* ctx, const ard_pattern* pat, int B, i
     }
     return ARD_OK;
   }
-  TcArgs t;
-  GemmArgs g;
-  fill_common(g, ctx, pat, B, KH, H, 1.0f);
-  g.A0 = dZ; g.lda0 = 4 * ldz_gate; g.A1 = W; g.lda1 = ldw; g.out = dXH; g.ldo = lddxh;
-  g.flag0 = 1;
-  g.out_is_f32 = 1;
-  g.accumulate = accumulate ? 1 : 0;
-  t.g = g;
-  t.ts = ldz_gate;
-  t.bn = ctx->force_bn;
-  for (int gate = 0; gate < 4; ++gate) {
-    st = get_maps(ctx, dZc + (size_t)gate * ldz_gate * 2, B, H, 4 * ldz_gate, H, MAP_COMPACT_COLS, pat->dp_bound, 128, 64,
-                  &t.mapA4[gate]);
-    if (st != ARD_OK) return st;
-    st = get_maps(ctx, Wc + (size_t)gate * H * ldw * 2, H, KH, ldw, H, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64,
-                  &t.mapB4[gate]);
-    if (st != ARD_OK) return st;
-  }
-  t.mapA = t.mapA4[0];
-  t.mapB = t.mapB4[0];
-  t.mapA_indexed = t.mapB_indexed = 1;
-  return launch_lstm_tc(ctx, 1, t, s);
+  return lstm_gate_gemm_bwd_tc(ctx, pat, B, KH, H, dZ, ldz_gate, W, ldw, dXH, lddxh, accumulate, s);
 }
 
 ard_status ard_lstm_gates(ard_ctx* ctx, const ard_pattern* pat, ard_dtype h_dtype, int B, int H, float alpha,
@@ -858,8 +873,10 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
                       &mapW[gate]);
         if (st != ARD_OK) return st;
       }
-      return launch_lstm_forward_persistent(ctx, pat, T, B, I, H, I, H, I > 0 ? 1 : 0, alpha, mapXH, mapW, XH, bias, C,
-                                            G, s);
+      st = launch_lstm_forward_persistent(ctx, pat, T, B, I, H, I, H, I > 0 ? 1 : 0, alpha, mapXH, mapW, XH, bias, C,
+                                          G, s);
+      if (st != ARD_ERR_UNSUPPORTED) return st;
+      // not launchable as one kernel right now: the per-step path below recomputes everything
     }
   }
   for (int t = 0; t < T; ++t) {
@@ -881,7 +898,42 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
   if (T < 1 || B < 0 || I < 0 || H < 1) return ARD_ERR_INVALID_ARG;
   const int KH = I + H;
   __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(DZ);
-  for (int t = T - 1; t >= 0; --t) {
+  // One cooperative kernel for the recurrence of the whole sequence when the layer fits it, followed by the
+  // input half of d[x, h] as one product over all T*B rows; otherwise the two kernels per time step below.
+  bool recurrence_done = false;
+  if (ctx->lstm_persistent && ctx->path != ARD_PATH_CUDA_CORE && B >= 1 && I > 0) {
+    ard_status st = check_common(ctx, pat, B, KH, H);
+    if (st != ARD_OK) return st;
+    if (pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+    if (ldw < KH) return ARD_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const char* Wc = reinterpret_cast<const char*>(W);
+    const char* dZc = reinterpret_cast<const char*>(DZ);
+    if (tc_eligible(ctx, pat, ARD_BF16, T * B, KH, H, DZ, 4 * H, W, ldw, D, KH, 4) == ARD_OK &&
+        ((size_t)H * ldw * 2) % 16 == 0 && I % 8 == 0 && lstm_persistent_bwd_fits(ctx, B, H)) {
+      const CUtensorMap* mapDZ[4];
+      const CUtensorMap* mapW[4];
+      for (int gate = 0; gate < 4; ++gate) {
+        st = get_maps(ctx, dZc + (size_t)gate * H * 2, T * B, H, 4 * H, H, MAP_COMPACT_COLS, pat->dp_bound, 64, 64,
+                      &mapDZ[gate]);
+        if (st != ARD_OK) return st;
+        st = get_maps(ctx, Wc + (size_t)gate * H * ldw * 2, H, KH, ldw, H, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64,
+                      &mapW[gate]);
+        if (st != ARD_OK) return st;
+      }
+      st = launch_lstm_backward_persistent(ctx, pat, T, B, I, H, alpha, mapDZ, mapW, C, G, dH_last, D, dc, DZ, s);
+      if (st == ARD_OK) {
+        // dx_t for all t: the x halves of D are overwritten
+        st = lstm_gate_gemm_bwd_tc(ctx, pat, T * B, I, H, DZ, H, W, ldw, D, KH, 0, s);
+        if (st != ARD_OK) return st;
+        recurrence_done = true;
+      } else if (st != ARD_ERR_UNSUPPORTED) {
+        return st;
+      }
+    }
+  }
+  for (int t = T - 1; t >= 0 && !recurrence_done; --t) {
     const float* dh = (t == T - 1) ? dH_last : D + (size_t)(t + 1) * B * KH + I;
     const int lddh = (t == T - 1) ? H : KH;
     ard_status st = ard_lstm_gates_bwd(ctx, pat, ARD_BF16, B, H, alpha, G + (size_t)t * B * 4 * H,

@@ -75,6 +75,7 @@ struct ard_ctx {
   int reuse_compact;  // opt-in: consecutive backward calls share one compacted dY
   int lstm_persistent; // ard_lstm_forward: one cooperative kernel for the whole sequence when the layer fits
   unsigned int* d_grid_bar;  // arrival counter of that kernel's grid-wide barrier
+  float* d_lstm_partial;     // partial sums of the whole-sequence BPTT kernel, lstm_bwd_partial_bytes(sm_count)
   int use_pdl;        // launch kernels with programmatic stream serialization (see ard_launch)
   int stream_k;       // tensor-core row kernels: share the last, partial wave of tiles along the contraction
   int sk_min_blocks;  // fewest 64-wide contraction blocks worth a separate share
@@ -148,7 +149,13 @@ int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int dp_bound, int ts);
 ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s);
 ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStream_t s);
 
-// Whole-sequence LSTM forward in one cooperative kernel (lstm_persistent.cu).
+// Whole-sequence LSTM kernels (lstm_persistent.cu).
+size_t lstm_bwd_partial_bytes(int sm_count);
+bool lstm_persistent_bwd_fits(ard_ctx* ctx, int B, int H);
+ard_status launch_lstm_backward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                                           const CUtensorMap* const mapDZ[4], const CUtensorMap* const mapW[4],
+                                           const float* C, const float* G, const float* dH_last, float* D, float* dc,
+                                           void* DZ, cudaStream_t s);
 bool lstm_persistent_fits(ard_ctx* ctx, int B, int klen, int H);
 ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H,
                                           int kx0, int klen, int add_zx, float alpha, const CUtensorMap* mapXH, const CUtensorMap* const mapW[4],

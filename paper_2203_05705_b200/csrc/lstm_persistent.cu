@@ -342,6 +342,293 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
   }
 }
 
+
+// ======================================================================================================
+// Whole-sequence BPTT recurrence (Sec. 7), the counterpart of the kernel above.
+//
+// Per step t = T-1 .. 0 the recurrence needs  dh_t = upstream_t + dz_{t+1} . W_h  (contraction over the
+// 4 * n_keep kept gate rows, output over the hidden units), then the cell adjoint gives dz_t.  Every SM
+// would need all of dz_{t+1} if the output units were simply dealt out, so the product is cut both ways:
+// CTA (s, r) owns the 64 hidden-unit COLUMNS 64 s .. 64 s + 63 of the recurrent weight (all of them, kept
+// or not: the columns of a kept-unit set are strided and cannot be boxed) and the r-th eighth of the
+// contraction blocks; its slice of the weight (at most 8 boxes of 64 gate rows x 64 columns, MN-major B
+// operand straight from the neuron-major weight) stays in shared memory for the whole sequence.  A step is
+//   A. wait until dz_{t+1} is complete (grid barrier), TMA-load this CTA's blocks of it, multiply
+//      (tcgen05.mma M = 128, N = 64, four issuing warps with an accumulator each), park the 64-column
+//      partial sums in global memory, arrive;
+//   B. wait until all partial sums are there (grid barrier); the threads that own a kept unit among this
+//      CTA's 8 columns 64 s + 8 r .. + 7 add the 8 partial sums in a fixed order, add the upstream gradient,
+//      store the total (the caller's D holds it afterwards), apply the cell adjoint with dc in a register,
+//      store dz_t (bf16, the operand of the next step and of the weight-gradient products), arrive.
+// After t = 0 one more product gives the gradient of h_0.  The input half of d[x, h] and the weight
+// gradient are large products over all T*B rows that the caller runs afterwards.
+// Grid barriers are phases of one arrival counter: every CTA arrives exactly once per phase and only
+// after it has passed the previous phase, so the count p * (number of CTAs) identifies phase p.
+constexpr int LB_COLS = 64;    // weight columns (hidden units, kept or not) per CTA
+constexpr int LB_KPARTS = 8;   // CTAs sharing the contraction of one column slice
+constexpr int LB_OWN = LB_COLS / LB_KPARTS;  // columns whose cell adjoint this CTA computes
+constexpr int LB_MAX_BLOCKS = 8;             // contraction blocks of one CTA (64 gate rows each)
+constexpr int LB_W_BLOCK = 64 * LB_COLS * 2; // one resident weight box
+constexpr int LB_THREADS = 512;              // warps 0-10 adjoint (0-3 also read TMEM), 11 relay, 12-15 load + MMA
+constexpr int LB_MATH = 352;
+constexpr int LB_PAIRS_MAX = (128 * LB_OWN + LB_MATH - 1) / LB_MATH;
+
+struct LstmBwdParams {
+  const CUtensorMap* mapDZ[4];  // per gate: tables over (dp, b) of [T*B rows][n_keep columns], boxes 64 x 64
+  const CUtensorMap* mapW[4];   // per gate: tables of strided-row maps over [n_keep rows][I+H columns], boxes 64 x 64
+  const int32_t* hdr;
+  int T, B, I, H;
+  float alpha;
+  const float* C;        // [T+1][B][H] compact
+  const float* G;        // [T][B][4H]
+  const float* dH_last;  // [B][H] full width
+  float* D;              // [T][B][I+H]
+  float* dc;             // [B][H] compact, in/out
+  __nv_bfloat16* DZ;     // [T][B][4H]: gate blocks of width H, compact inside a block
+  float* partial;        // [CTA][128][64]
+  unsigned int* bar;
+  int* status;
+};
+
+__global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const LstmBwdParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - raw_addr);
+
+  const int KH = p.I + p.H;
+  const int row_boxes = (p.B + 63) / 64;
+  const uint32_t a_block = (uint32_t)row_boxes * LP_ROW_BOX;
+  const uint32_t sA = base;                                     // LB_MAX_BLOCKS blocks of dz
+  const uint32_t sW = base + LB_MAX_BLOCKS * a_block;            // LB_MAX_BLOCKS weight boxes (the MMA's 128-row read of
+                                                                 // the last dz block ends inside this region)
+  const uint32_t bar_base = sW + LB_MAX_BLOCKS * LB_W_BLOCK;     // gfull[4], tfull, wfull, hready, pready
+  auto gfull_bar = [&](int g) { return bar_base + 8u * g; };
+  const uint32_t tfull_bar = bar_base + 8u * LP_GROUPS;
+  const uint32_t wfull_bar = bar_base + 8u * (LP_GROUPS + 1);
+  const uint32_t hready_bar = bar_base + 8u * (LP_GROUPS + 2);   // dz of the previous step is complete
+  const uint32_t pready_bar = bar_base + 8u * (LP_GROUPS + 3);   // all partial sums of this step are parked
+  uint8_t* misc = smem + (bar_base - base) + 8 * (LP_GROUPS + 4);
+  volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int g = 0; g < LP_GROUPS; ++g) mbar_init(gfull_bar(g), 1);
+    mbar_init(tfull_bar, LP_GROUPS);
+    mbar_init(wfull_bar, 1);
+    mbar_init(hready_bar, 1);
+    mbar_init(pready_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 15) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_ptr_smem)), LP_GROUPS * LB_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_ptr_smem;
+  pdl_wait_prior_grids();
+
+  const int dp = p.hdr[HDR_DP], bb = p.hdr[HDR_B] - 1, n_keep = p.hdr[HDR_NKEEP];
+  const int e = p.hdr[HDR_MAPIDX];
+  const int n_cta = (int)gridDim.x;
+  const int s_idx = (int)blockIdx.x / LB_KPARTS, r_idx = (int)blockIdx.x % LB_KPARTS;
+  const int c0 = s_idx * LB_COLS;                       // first weight column (hidden unit) of the slice
+  const int nb = (n_keep + 63) / 64;                    // contraction blocks per gate
+  const int per = (4 * nb + LB_KPARTS - 1) / LB_KPARTS; // blocks per CTA (<= LB_MAX_BLOCKS, checked by the host)
+  const int blk0 = r_idx * per;
+  const int nblk = max(0, min(per, 4 * nb - blk0));     // this CTA's blocks blk0 .. blk0 + nblk - 1; block = gate * nb + jb
+  const int parts = (4 * nb + per - 1) / per;           // CTAs of a slice that have blocks
+  const int gsz = (nblk + LP_GROUPS - 1) / LP_GROUPS;   // blocks per loader / MMA warp
+  const int T = p.T;
+
+  if (warp == 11) {
+    // ===================== weight loader and barrier relay =====================
+    const int kb = lane;
+    if (kb < nblk) {
+      const int blk = blk0 + kb, g = blk / nb, jb = blk - g * nb;
+      tensormap_acquire(p.mapW[g] + e);
+      if (lane == 0) mbar_arrive_expect_tx(wfull_bar, (uint32_t)nblk * LB_W_BLOCK);
+      __syncwarp(__activemask());
+      tma_load_2d(sW + kb * LB_W_BLOCK, p.mapW[g] + e, wfull_bar, p.I + c0, jb * 64);
+    }
+    __syncwarp();
+    if (lane == 0) {
+      for (int ph = 1; ph <= 2 * T; ++ph) {
+        if (!grid_wait(p.bar, (unsigned)ph * (unsigned)n_cta, abort_flag, p.status)) break;
+        mbar_arrive((ph & 1) ? hready_bar : pready_bar);
+      }
+    }
+  } else if (warp >= 12) {
+    // ===================== loaders and MMA issuers (group g = warp - 12) =====================
+    const int g4 = warp - 12;
+    const int kb0 = g4 * gsz, kb1 = min(nblk, kb0 + gsz);
+    const int kb = kb0 + lane;
+    const bool mine = kb < kb1;
+    int gate = 0, jb = 0;
+    if (mine) {
+      const int blk = blk0 + kb;
+      gate = blk / nb;
+      jb = blk - gate * nb;
+      tensormap_acquire(p.mapDZ[gate] + e);
+    }
+    const uint32_t idesc = make_idesc(LB_COLS, false, true, 128);
+    bool ok = (lane != 0) || nblk == 0 || mbar_wait(wfull_bar, 0u, abort_flag, p.status);
+    for (int k = 1; k <= T; ++k) {
+      // dz of time index T - k is complete
+      if (ok && !mbar_wait(hready_bar, (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
+      if (!__all_sync(0xffffffffu, ok)) break;
+      if (kb0 < kb1) {
+        asm volatile("fence.proxy.async.global;" ::: "memory");  // generic-proxy stores of other CTAs -> TMA reads
+        if (lane == 0) mbar_arrive_expect_tx(gfull_bar(g4), (uint32_t)(kb1 - kb0) * a_block);
+        __syncwarp();
+        if (mine)
+          for (int rb = 0; rb < row_boxes; ++rb)
+            tma_load_2d(sA + kb * a_block + rb * LP_ROW_BOX, p.mapDZ[gate] + e, gfull_bar(g4), jb * 64,
+                        (T - k) * p.B + rb * 64);
+        if (lane == 0) {
+          if (!mbar_wait(gfull_bar(g4), (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
+          if (ok) {
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(g4 * LB_COLS);
+            for (int k2 = kb0; k2 < kb1; ++k2) {
+              const uint32_t a0 = sA + k2 * a_block, b0 = sW + k2 * LB_W_BLOCK;
+#pragma unroll
+              for (int s = 0; s < LP_BK / 16; ++s)  // A K-major: 32 bytes per step; B MN-major: 16 k-rows = 2048 bytes
+                tc_mma_bf16(d_tmem, make_desc(a0 + s * 32, 16, 1024), make_desc(b0 + s * 2048, 64 * LP_BK * 2, 1024), idesc,
+                            (k2 != kb0 || s != 0) ? 1u : 0u);
+            }
+          }
+        }
+      }
+      if (lane == 0 && ok && nblk > 0) {
+        if (kb0 < kb1) tc_commit(tfull_bar);
+        else mbar_arrive(tfull_bar);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ===================== partial sums and cell adjoint (warps 0-10) =====================
+    const int tid = threadIdx.x;  // 0 .. LB_MATH-1
+    const int npairs = p.B * LB_OWN;  // (batch row, owned column) pairs; pair q = row * 8 + cc
+    const size_t ldd = (size_t)KH;
+    float dcreg[LB_PAIRS_MAX];
+    int jj[LB_PAIRS_MAX];  // kept index of the pair's unit, -1 if the column is a dropped unit or out of range
+#pragma unroll
+    for (int i = 0; i < LB_PAIRS_MAX; ++i) {
+      const int q = tid + i * LB_MATH;
+      const int row = q >> 3, u = c0 + r_idx * LB_OWN + (q & 7);
+      const int rel = u - bb;
+      jj[i] = (q < npairs && u < p.H && rel >= 0 && rel % dp == 0) ? rel / dp : -1;
+      dcreg[i] = jj[i] >= 0 ? p.dc[(size_t)row * p.H + jj[i]] : 0.f;
+    }
+    float* my_partial = p.partial + (size_t)blockIdx.x * 128 * LB_COLS;
+    const float* slice_partial = p.partial + (size_t)(s_idx * LB_KPARTS) * 128 * LB_COLS;
+    bool ok = true;
+    for (int k = 0; k <= T && ok; ++k) {
+      const int t = T - 1 - k;  // time index whose dh is formed in this round (-1: the gradient of h_0)
+      if (k >= 1) {
+        // ---- phase A: park this CTA's partial sums ----
+        // Every CTA passes the previous phase before it arrives for this one, also a CTA that has no
+        // contraction blocks: the arrival count identifies a phase only if nobody is two arrivals ahead.
+        if (!mbar_wait(hready_bar, (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
+        if (ok && warp < 4 && nblk > 0) {
+          if (!mbar_wait(tfull_bar, (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
+          if (ok) {
+            tc_fence_after();
+            const int row = warp * 32 + lane;
+            const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
+            const int ngroups = (nblk + gsz - 1) / gsz;
+#pragma unroll 1
+            for (int half = 0; half < 2; ++half) {
+              uint32_t z[32], y[32];
+              tmem_ld32(t_row + (uint32_t)(half * 32), z);
+              tmem_ld_wait();
+              for (int c = 1; c < ngroups; ++c) {
+                tmem_ld32(t_row + (uint32_t)(c * LB_COLS + half * 32), y);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) z[i] = __float_as_uint(__uint_as_float(z[i]) + __uint_as_float(y[i]));
+              }
+              if (row < p.B) {
+                float4* dst = reinterpret_cast<float4*>(my_partial + (size_t)row * LB_COLS + half * 32);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                  __stcg(dst + i, make_float4(__uint_as_float(z[4 * i]), __uint_as_float(z[4 * i + 1]),
+                                              __uint_as_float(z[4 * i + 2]), __uint_as_float(z[4 * i + 3])));
+              }
+            }
+            tc_fence_before();
+          }
+        }
+        asm volatile("bar.sync 1, 352;" ::: "memory");
+        if (*abort_flag) { ok = false; break; }
+        if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
+        // ---- all partial sums of the slice are parked ----
+        if (!mbar_wait(pready_bar, (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
+        asm volatile("bar.sync 2, 352;" ::: "memory");
+        if (*abort_flag) { ok = false; break; }
+      }
+      // ---- phase B: total gradient of h_t, cell adjoint, dz_t ----
+#pragma unroll
+      for (int i = 0; i < LB_PAIRS_MAX; ++i) {
+        if (jj[i] < 0) continue;
+        const int q = tid + i * LB_MATH;
+        const int row = q >> 3, cc = r_idx * LB_OWN + (q & 7), u = c0 + cc, j = jj[i];
+        float rec = 0.f;
+        if (k >= 1)
+          for (int rp = 0; rp < parts; ++rp) rec += __ldcg(slice_partial + ((size_t)rp * 128 + row) * LB_COLS + cc);
+        if (t < 0) {  // gradient of h_0: added to what the caller left in the h half of D[0]
+          p.D[(size_t)row * ldd + p.I + u] += rec;
+          continue;
+        }
+        float dh;
+        if (t == T - 1) {
+          dh = p.dH_last[(size_t)row * p.H + u];
+        } else {
+          float* up = p.D + ((size_t)(t + 1) * p.B + row) * ldd + p.I + u;  // upstream gradient of h_t
+          dh = *up + rec;
+          *up = dh;
+        }
+        const float* gs = p.G + ((size_t)t * p.B + row) * 4 * p.H + j;
+        const float gi = gs[0], gf = gs[p.H], gg = gs[2 * p.H], go = gs[3 * p.H];
+        const float cp = p.C[((size_t)t * p.B + row) * p.H + j];
+        const float tc = tanh_fast(p.C[((size_t)(t + 1) * p.B + row) * p.H + j]);
+        const float d_o = dh * p.alpha * tc;
+        const float dcv = dcreg[i] + dh * p.alpha * go * (1.f - tc * tc);
+        dcreg[i] = dcv * gf;
+        __nv_bfloat16* dz = p.DZ + ((size_t)t * p.B + row) * 4 * p.H + j;
+        dz[0] = __float2bfloat16_rn(dcv * gg * gi * (1.f - gi));
+        dz[p.H] = __float2bfloat16_rn(dcv * cp * gf * (1.f - gf));
+        dz[2 * p.H] = __float2bfloat16_rn(dcv * gi * (1.f - gg * gg));
+        dz[3 * p.H] = __float2bfloat16_rn(d_o * go * (1.f - go));
+      }
+      if (t >= 0) {
+        asm volatile("bar.sync 1, 352;" ::: "memory");
+        if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
+      }
+    }
+    if (ok) {
+#pragma unroll
+      for (int i = 0; i < LB_PAIRS_MAX; ++i)
+        if (jj[i] >= 0) p.dc[(size_t)((tid + i * LB_MATH) >> 3) * p.H + jj[i]] = dcreg[i];
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 15) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, LP_GROUPS * LB_COLS);
+  }
+}
+
 }  // namespace
 
 // Dynamic shared memory for klen contraction columns and batch B: the row buffer, the weight slice, the
@@ -403,7 +690,77 @@ ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, 
   attr[0].val.cooperative = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  ARD_CUDA_OK(cudaLaunchKernelEx(&cfg, ard_lstm_forward_kernel, p));
+  const cudaError_t err = cudaLaunchKernelEx(&cfg, ard_lstm_forward_kernel, p);
+  if (err == cudaErrorCooperativeLaunchTooLarge || err == cudaErrorLaunchOutOfResources) {
+    // the device cannot hold all CTAs at once right now (SMs taken by another context, a smaller
+    // partition): nothing was enqueued, the caller falls back to the per-step path
+    (void)cudaGetLastError();
+    return ARD_ERR_UNSUPPORTED;
+  }
+  if (err != cudaSuccess) return ARD_ERR_CUDA;
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+// ---- whole-sequence BPTT recurrence ----
+static size_t lstm_bwd_smem_bytes(int B) {
+  return (size_t)LB_MAX_BLOCKS * ((B + 63) / 64) * LP_ROW_BOX + (size_t)LB_MAX_BLOCKS * LB_W_BLOCK + 8 * (LP_GROUPS + 4) + 16 + 1024;
+}
+
+size_t lstm_bwd_partial_bytes(int sm_count) { return (size_t)sm_count * 128 * LB_COLS * sizeof(float); }
+
+bool lstm_persistent_bwd_fits(ard_ctx* ctx, int B, int H) {
+  if (B < 1 || B > 128 || H < 1 || H > 1024) return false;  // at most 8 contraction blocks per CTA
+  if (ctx->d_lstm_partial == nullptr) return false;
+  if ((H + LB_COLS - 1) / LB_COLS * LB_KPARTS > ctx->sm_count) return false;  // one CTA per SM, all resident at once
+  static int probed[64] = {};
+  const int dev = ctx->device & 63;
+  if (probed[dev] == 0) {
+    int n = 0;
+    if (cudaFuncSetAttribute(ard_lstm_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, ard_lstm_backward_kernel, LB_THREADS, lstm_bwd_smem_bytes(128)) !=
+            cudaSuccess ||
+        n < 1)
+      probed[dev] = -1;
+    else
+      probed[dev] = 1;
+  }
+  return probed[dev] == 1;
+}
+
+ard_status launch_lstm_backward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                                           const CUtensorMap* const mapDZ[4], const CUtensorMap* const mapW[4],
+                                           const float* C, const float* G, const float* dH_last, float* D, float* dc,
+                                           void* DZ, cudaStream_t s) {
+  LstmBwdParams p;
+  for (int g = 0; g < 4; ++g) { p.mapDZ[g] = mapDZ[g]; p.mapW[g] = mapW[g]; }
+  p.hdr = pat->d_hdr;
+  p.T = T; p.B = B; p.I = I; p.H = H;
+  p.alpha = alpha;
+  p.C = C; p.G = G; p.dH_last = dH_last; p.D = D; p.dc = dc;
+  p.DZ = reinterpret_cast<__nv_bfloat16*>(DZ);
+  p.partial = ctx->d_lstm_partial;
+  p.bar = ctx->d_grid_bar;
+  p.status = ctx->d_status;
+  ARD_CUDA_OK(cudaMemsetAsync(ctx->d_grid_bar, 0, sizeof(unsigned int), s));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((H + LB_COLS - 1) / LB_COLS * LB_KPARTS);
+  cfg.blockDim = dim3(LB_THREADS);
+  cfg.dynamicSmemBytes = lstm_bwd_smem_bytes(B);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs resident: they wait for one another
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t err = cudaLaunchKernelEx(&cfg, ard_lstm_backward_kernel, p);
+  if (err == cudaErrorCooperativeLaunchTooLarge || err == cudaErrorLaunchOutOfResources) {
+    (void)cudaGetLastError();
+    return ARD_ERR_UNSUPPORTED;  // nothing was enqueued: the caller takes the per-step path
+  }
+  if (err != cudaSuccess) return ARD_ERR_CUDA;
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;

@@ -96,3 +96,53 @@ def test_layers_that_do_not_fit_use_the_per_step_path():
         assert OG.rel_fro(host(Hg), fw["Hs"]) <= TOL[ard.ARD_BF16]
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("T,B,I,H", [(5, 33, 128, 264), (3, 128, 64, 128), (4, 7, 192, 1024)])
+def test_persistent_bptt_matches_the_oracle_and_the_per_step_path(T, B, I, H):
+    """Whole-sequence BPTT kernel: dX, dW, dh_0, dc_0 against the oracle and against the per-step path."""
+    from paper_2203_05705_b200.lstm import LstmLayer
+    rng = np.random.default_rng(T * 100 + B)
+    W = inputs.bf16_round(rng.uniform(-0.08, 0.08, size=(I + H, 4 * H)).astype(np.float32))
+    X = inputs.bf16_round(rng.standard_normal((T, B, I)).astype(np.float32))
+    dH = (rng.standard_normal((T, B, H)) / 8).astype(np.float32)
+    Wnm = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+    ctx = Ctx(1 << 20)
+    try:
+        pat = ctx.pattern(ard.ARD_ROW, I + H, H)
+        for dp, b in [(1, 1), (2, 1), (3, 3), (16, 5)]:
+            ard.ard_pattern_set(ctx.h, pat, dp, b)
+            m = OP.row_mask(H, dp, b)
+            keep = OP.row_keep(H, dp, b)
+            alpha = 1.5
+            fw = OL.fwd(X, W, None, m, alpha)
+            bw = OL.bwd(fw, W, m, alpha, dH)
+            got = {}
+            for mode in (1, 0):
+                ard.ard_set_lstm_persistent(ctx.h, mode)
+                layer = LstmLayer(ctx.h, pat, T, B, I, H, Wnm)
+                layer.load_inputs(torch.from_numpy(X).to(BF).cuda())
+                layer.forward(alpha)
+                n0 = ard.ard_launch_count(ctx.h)
+                dX, dW = layer.backward(alpha, torch.from_numpy(dH).cuda())
+                torch.cuda.synchronize()
+                launches = ard.ard_launch_count(ctx.h) - n0
+                assert ard.ard_last_device_status(ctx.h) == 0
+                assert launches == (2 + 4 if mode else 2 * T + 4), (mode, launches)
+                got[mode] = (dX.clone(), dW.clone(), layer.D[0, :, I:].clone(), layer.dc.clone())
+                assert OG.rel_fro(host(dX), bw["dX"]) <= TOL[ard.ARD_BF16], (mode, dp, b)
+                assert OG.rel_fro(host(dW), bw["dW"].T) <= TOL[ard.ARD_BF16], (mode, dp, b)
+                dropped = torch.from_numpy(np.concatenate([g * H + np.where(m == 0)[0] for g in range(4)])).cuda()
+                assert bool(torch.all(dW[dropped, :] == 0))
+                kidx = torch.from_numpy(keep).cuda()
+                assert OG.rel_fro(host(layer.D[0, :, I:][:, kidx]), bw["dh0"][:, keep]) <= TOL[ard.ARD_BF16], (mode, dp, b)
+                assert OG.rel_fro(host(layer.dc[:, :len(keep)]), bw["dc0"][:, keep]) <= TOL[ard.ARD_BF16], (mode, dp, b)
+            kept = torch.from_numpy(keep).cuda()
+            n = len(keep)
+            # gradient of h_0 (kept units) and of c_0: both paths agree closely
+            a, c = got[1][2][:, kept], got[0][2][:, kept]
+            assert float((a - c).abs().max()) <= 2e-2 * max(1.0, float(c.abs().max())), (dp, b)
+            a, c = got[1][3][:, :n], got[0][3][:, :n]
+            assert float((a - c).abs().max()) <= 2e-2 * max(1.0, float(c.abs().max())), (dp, b)
+    finally:
+        ctx.close()
