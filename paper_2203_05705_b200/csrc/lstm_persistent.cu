@@ -531,6 +531,21 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
     bool ok = true;
     for (int k = 0; k <= T && ok; ++k) {
       const int t = T - 1 - k;  // time index whose dh is formed in this round (-1: the gradient of h_0)
+      // what does not depend on the recurrence is fetched before the waits: gate activations, cell states
+      float pg[LB_PAIRS_MAX][6];
+#pragma unroll
+      for (int i = 0; i < LB_PAIRS_MAX; ++i) {
+        if (jj[i] >= 0 && t >= 0) {
+          const int row = (tid + i * LB_MATH) >> 3, j = jj[i];
+          const float* gs = p.G + ((size_t)t * p.B + row) * 4 * p.H + j;
+          pg[i][0] = __ldcg(gs);
+          pg[i][1] = __ldcg(gs + p.H);
+          pg[i][2] = __ldcg(gs + 2 * p.H);
+          pg[i][3] = __ldcg(gs + 3 * p.H);
+          pg[i][4] = __ldcg(p.C + ((size_t)t * p.B + row) * p.H + j);
+          pg[i][5] = __ldcg(p.C + ((size_t)(t + 1) * p.B + row) * p.H + j);
+        }
+      }
       if (k >= 1) {
         // ---- phase A: park this CTA's partial sums ----
         // Every CTA passes the previous phase before it arrives for this one, also a CTA that has no
@@ -594,10 +609,9 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
           dh = *up + rec;
           *up = dh;
         }
-        const float* gs = p.G + ((size_t)t * p.B + row) * 4 * p.H + j;
-        const float gi = gs[0], gf = gs[p.H], gg = gs[2 * p.H], go = gs[3 * p.H];
-        const float cp = p.C[((size_t)t * p.B + row) * p.H + j];
-        const float tc = tanh_fast(p.C[((size_t)(t + 1) * p.B + row) * p.H + j]);
+        const float gi = pg[i][0], gf = pg[i][1], gg = pg[i][2], go = pg[i][3];
+        const float cp = pg[i][4];
+        const float tc = tanh_fast(pg[i][5]);
         const float d_o = dh * p.alpha * tc;
         const float dcv = dcreg[i] + dh * p.alpha * go * (1.f - tc * tc);
         dcreg[i] = dcv * gf;
