@@ -271,6 +271,33 @@ def run_lstm(args, wl):
     for i in range(ne):
         ard.ard_sample_pattern(ctx, pat, 0, inputs.BASE_SEED, 200000 + args.warmup + i, 4)
         nks_e.append(ard.ard_pattern_to_host(pat, 0)[2])
+    # dense library baseline for context: the same layer without dropout in torch.nn.LSTM (cuDNN), bf16
+    ms_lib = None
+    try:
+        ref = torch.nn.LSTM(I, H, num_layers=1, bias=True).to(device="cuda", dtype=bf)
+        Xr = X.clone().requires_grad_(True)
+        dHr = dH.to(bf)
+
+        def lib_seq():
+            for prm in ref.parameters():
+                prm.grad = None
+            Xr.grad = None
+            out, _ = ref(Xr)
+            out.backward(dHr)
+
+        for _ in range(args.warmup):
+            lib_seq()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        nl = max(5, steps // 4)
+        e0.record()
+        for _ in range(nl):
+            lib_seq()
+        e1.record()
+        torch.cuda.synchronize()
+        ms_lib = e0.elapsed_time(e1) / nl
+    except Exception as ex:  # the library baseline is context only
+        sys.stderr.write("torch.nn.LSTM baseline skipped: %r\n" % (ex,))
     peaks = load_peaks()
     cpu = None
     if not args.no_cpu_baseline:
@@ -303,8 +330,8 @@ def run_lstm(args, wl):
                      "frac": value / peaks["bf16_tflops"], "traffic": None,
                      "note": "35 dependent steps of a 64-row product: bound by per-step latency, not by the tensor pipe"},
         "cpu_baseline": cpu,
-        "detail": {"dense_ms_per_step": {"own_kernels_dp1": ms_dense / max(5, steps // 4)},
-                   "speedup_vs_dense": {str(p): (ms_dense / max(5, steps // 4)) / (ms / steps)},
+        "detail": {"dense_ms_per_step": {"own_kernels_dp1": ms_dense / max(5, steps // 4), "torch_nn_lstm": ms_lib},
+                   "speedup_vs_dense": {str(p): min(ms_dense / max(5, steps // 4), ms_lib or 1e30) / (ms / steps)},
                    "kept_fraction": {str(p): float(np.mean(nks)) / H}},
         "device_status": int(status),
     }

@@ -262,7 +262,14 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
  * the upstream gradient of h_{t-1} in the h half of D[t] (t >= 1); on return its x halves hold dx_t and the h
  * half of D[0] the gradient of h_0.  dH_last [B][H] fp32 is the gradient of h_{T-1}; dc [B][H] fp32 must be
  * zero on entry (or hold the gradient of c_T) and returns the gradient of c_0; DZ [T][B][4H] bf16 scratch;
- * dW [4H][I+H] fp32 receives the weight gradient (dropped units' rows zero). */
+ * dW [4H][I+H] fp32 receives the weight gradient (dropped units' rows zero).
+ * When the layer fits (B <= 128, H <= 1024, 8*ceil(H/64) <= number of SMs, operands aligned) and
+ * ard_set_lstm_persistent is on, the recurrence dh_{t-1} = upstream + dz_t W_h with the cell adjoint is ONE
+ * cooperative kernel (weight slices resident in shared memory, dc in registers, two bounded grid-wide
+ * synchronisations per step) and the x halves come from one product over all T*B rows; otherwise a loop
+ * in native code enqueues ard_lstm_gates_bwd and ard_lstm_gate_gemm_bwd per step.  In both cases the h
+ * halves of D[1..T-1] are overwritten (kept units: the total gradient of h_{t-1}; dropped units:
+ * unspecified), and the h half of D[0] is meaningful at kept units only. */
 ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
                              const void* XH, const void* W, int ldw, const float* C, const float* G,
                              const float* dH_last, float* D, float* dc, void* DZ, float* dW, void* cuda_stream);

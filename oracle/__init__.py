@@ -16,6 +16,8 @@ Pins (each lives in tests/test_oracle_*.py):
   lstm.*                   dp=1 == torch.nn.LSTM (fp64, forward and autograd gradients);
                            kept sub-network == torch.nn.LSTM of hidden size n_k; finite differences
   mlp_chain.*              finite differences of the scalar <dZ3, Z3>
+  mlp.*                    torch autograd (fp64) on the same network written with library ops; central
+                           differences; == mlp_chain without bias; compact-matrix form == masked full width
   search.*                 gradient vs central differences; stationary points lie in the Gibbs family
                            ln k_i = beta (i-1)/i + c with beta = -2 (k.p_u - p)/lambda; small-lambda limit ==
                            the maximum-entropy distribution at rate p; Eq. 2-3 in exact rationals
