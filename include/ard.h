@@ -63,6 +63,7 @@ typedef enum { ARD_OUT_COMPACT = 0, ARD_OUT_SCATTER_ZEROFILL = 1 } ard_outmode;
  * argument of ard_bwd_data (whose bit 0 keeps its meaning): */
 #define ARD_FLAG_OUT_F32 0x10    /* bf16 operands: write the result as fp32 (leading dimension in fp32 elements) */
 #define ARD_FLAG_ACCUMULATE 0x20 /* add the product to the existing output; not with ARD_OUT_SCATTER_ZEROFILL   */
+#define ARD_FLAG_RELU 0x40       /* ard_layer_fwd only: apply max(., 0) before the rescale                      */
 
 /* Selects the kernel family for ARD_BF16 calls.  AUTO picks the tcgen05 path when the shape and
  * alignment allow it and the CUDA-core path otherwise; the other two force one family (FORCE_TC
@@ -216,6 +217,106 @@ ard_status ard_bwd_data_static_scratch(ard_ctx* ctx, const ard_pattern* pat, ard
 ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, ard_dtype dW_dtype, int B, int K,
                           int N, float alpha, const void* X, int ldx, const void* dY, int lddy, int dy_is_compact,
                           void* dW, int lddw, int zero_fill_dropped, void* cuda_stream);
+
+/* ---- fused layer step (row patterns) ----------------------------------------------------------
+ * Sec. 3.2, last paragraph: a layer of a training iteration is the fully connected product, the
+ * activation and the dropout mask; under a pattern the mask disappears into the product.  Sec. 3.1:
+ * a dropped neuron also removes its column from the input matrix of the layer it feeds and the
+ * matching fan-in weights of that layer, so BOTH matrices of that layer's product are compact.
+ * (The paper prints no formula for the step; ReLU with relu'(0) = 0, a bias per neuron and the
+ * rescale after the activation are this library's reading.)
+ *
+ * For a layer with row pattern `pat` (N neurons, n kept) fed by a layer with row pattern `in_pat`
+ * (its N_dim == this layer's K; n_in kept), or by a full-width input (in_pat == NULL, n_in = K):
+ *
+ *   forward        A[:, j]  = alpha * act( sum_i X[:, i] * Wk[keep[j]][i] + bias[keep[j]] )     j < n
+ *   backward-data  dX[:, i] = alpha * sum_j dZ[:, j] * Wk[keep[j]][i]  (0 where act_prev[:, i] <= 0)  i < n_in
+ *   backward-weight dWk[keep[j]][i] = alpha * sum_r dZ[r][j] * X[r][i]                           i < n_in
+ *
+ * where, with in_pat, X [B][n_in], act_prev [B][n_in] and dX [B][n_in] are COMPACT over the feeding
+ * layer's kept neurons (column i = its i-th kept neuron; leading dimensions >= K so that any pattern
+ * fits) and Wk / dWk [N][K-wide rows] hold, in row keep[j], the fan-in weights of those kept neurons
+ * in columns 0..n_in-1: Wk is made from W by ard_compact_weight_cols once per iteration, dWk is
+ * expanded into dW by ard_expand_weight_grad_cols.  Without in_pat, Wk = W, dWk = dW and X is full
+ * width.  dZ is the gradient of the pre-activations Z = X Wk + bias (compact [B][n] when the compact
+ * bit is set).  To chain layers, call ard_layer_bwd_data of layer l+1 with alpha = alpha_l and
+ * act_prev = A_l: its result is dZ_l, compact, which layer l's backward calls take with alpha = 1.
+ * bias (fp32 [N], indexed by the original neuron) and act_prev may be NULL.  act_prev has the
+ * operand element type.  The output modes and flags are those of ard_fwd / ard_bwd_data /
+ * ard_bwd_weight (ARD_OUT_COMPACT, ARD_OUT_SCATTER_ZEROFILL, ARD_FLAG_OUT_F32; ARD_FLAG_RELU selects
+ * act = ReLU, otherwise the identity); ARD_FLAG_ACCUMULATE cannot be combined with bias, ReLU or
+ * act_prev.  With zero_fill_dropped, ard_layer_bwd_weight zeroes the rows of dropped neurons in
+ * columns 0..n_in-1 of dWk.  Tensor-core path: bf16, aligned as for ard_fwd, act_prev 16-byte
+ * aligned with ldact % 8 == 0; otherwise (and for ARD_F32) the CUDA-core path runs the same step. */
+ard_status ard_layer_fwd(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype, int B, int K,
+                         int N, float alpha, const void* X, int ldx, const void* Wk, int ldw, const float* bias,
+                         void* A, int lda, int outmode_and_flags, void* cuda_stream);
+ard_status ard_layer_bwd_data(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype, int B,
+                              int K, int N, float alpha, const void* dZ, int lddz, int dz_is_compact_and_flags,
+                              const void* Wk, int ldw, const void* act_prev, int ldact, void* dX, int lddx,
+                              void* cuda_stream);
+ard_status ard_layer_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
+                                ard_dtype dW_dtype, int B, int K, int N, float alpha, const void* X, int ldx,
+                                const void* dZ, int lddz, int dz_is_compact, void* dWk, int lddw,
+                                int zero_fill_dropped, void* cuda_stream);
+/* Wk[n][i] = W[n][keep_in[i]] for the kept neurons n of `pat` and i < n_in; columns n_in up to the next
+ * multiple of 64 (bounded by ldwk) are written as zero; rows of dropped neurons are not touched.
+ * W, Wk [N][K-wide rows] of element type `dtype`, ldw, ldwk >= K, W != Wk. */
+ard_status ard_compact_weight_cols(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
+                                   int K, int N, const void* W, int ldw, void* Wk, int ldwk, void* cuda_stream);
+/* dW[n][keep_in[i]] = dWk[n][i] for the kept neurons n and i < n_in.  zero_fill != 0: every other entry
+ * of dW [N][K] (dropped neurons, dropped inputs) is written as zero; otherwise it is left untouched. */
+ard_status ard_expand_weight_grad_cols(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
+                                       int K, int N, const void* dWk, int lddwk, void* dW, int lddw, int zero_fill,
+                                       void* cuda_stream);
+/* db[keep[j]] = sum over the B rows of dZ[:, j] (fp32, rows added in a fixed order); dZ of element type
+ * `dtype`, compact [B][n] or full width [B][N]; zero_fill_dropped != 0 zeroes db at dropped neurons. */
+ard_status ard_bias_grad(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int N, const void* dZ, int lddz,
+                         int dz_is_compact, float* db, int zero_fill_dropped, void* cuda_stream);
+/* ard_sample_pattern with the iteration taken from device memory: the pattern is drawn for iteration
+ * iteration_base + *iteration_counter (DEVICE uint64, owned by the caller, read when the kernel runs);
+ * with advance != 0 the kernel then adds one to the counter.  A training step captured once into a CUDA
+ * graph therefore draws a new pattern at every replay: let the last sampling call of the step advance. */
+ard_status ard_sample_pattern_counter(ard_ctx* ctx, ard_pattern* pat, int dist_id, uint64_t seed,
+                                      uint64_t iteration_base, uint64_t* iteration_counter, int advance,
+                                      uint32_t stream_id, void* cuda_stream);
+
+/* One training iteration of a stack of bf16 layers as one native call: draws the pattern of every layer
+ * that asks for one (stream id = layer index + 1, iteration = iteration_base + *iteration_counter, the
+ * last draw advances the counter), runs the forward chain with ard_layer_fwd and the backward chain with
+ * ard_layer_bwd_weight / ard_bias_grad / ard_layer_bwd_data.  A layer with compact_out != 0 writes its
+ * activations compact and the layer after it multiplies compact matrices on both sides (its weight is
+ * compacted into Wk first, its gradient expanded from dWk into dW); with compact_out == 0 activations and
+ * gradients between the two layers are full width.  The last layer must have compact_out == 0; dOut
+ * [B][N_last] is the gradient with respect to its output A (for a linear last layer: relu = 0, alpha = 1,
+ * pattern set dense with ard_pattern_set(1, 1) and sample = 0).  On return: layers[l].dW (dropped rows
+ * and columns zero), layers[l].db if not NULL, dX [B][K_0] if not NULL; A and dZ of every layer hold what
+ * the step computed.  `layers` is a HOST array; all pointers inside are DEVICE pointers owned by the caller;
+ * dimensions must satisfy the alignment rules of ard_fwd or the slower CUDA-core kernels run.  Enqueues
+ * only; allocates nothing once every buffer has been seen once (descriptor tables), so it can be
+ * captured into a CUDA graph after one ordinary call. */
+typedef struct ard_mlp_layer {
+  int K, N;          /* fan-in and neurons; K of layer l+1 == N of layer l                                  */
+  ard_pattern* pat;  /* row pattern over the N neurons (created with K_dim = K, N_dim = N)                  */
+  int sample;        /* != 0: draw a new pattern this iteration; 0: keep the one the pattern holds          */
+  int relu;          /* != 0: ReLU between the product and the rescale                                      */
+  int compact_out;   /* != 0: compact activations, compact matrices in the next layer                       */
+  int dW_is_f32;     /* element type of dW and dWk: fp32 (!= 0) or bf16                                      */
+  float alpha;       /* rescale of this layer's output, e.g. 1/(1-p)                                        */
+  int ldw;           /* leading dimension of W, Wk, dW, dWk (>= K)                                           */
+  const void* W;     /* bf16 [N][ldw]                                                                        */
+  const float* bias; /* fp32 [N] or NULL                                                                     */
+  void* Wk;          /* bf16 [N][ldw] scratch, needed when the previous layer has compact_out               */
+  void* A;           /* bf16 [B][N] activations (compact: columns 0..n-1)                                    */
+  void* dZ;          /* bf16 [B][N] gradient of the pre-activations, written by the layer above; not needed
+                        for the last layer                                                                   */
+  void* dWk;         /* [N][ldw] scratch of dW's type, needed when the previous layer has compact_out       */
+  void* dW;          /* [N][ldw] weight gradient                                                             */
+  float* db;         /* fp32 [N] bias gradient or NULL                                                       */
+} ard_mlp_layer;
+ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, int n_layers, int B, const void* X, int ldx,
+                        const void* dOut, int lddout, void* dX, int lddx, int dist_id, uint64_t seed,
+                        uint64_t iteration_base, uint64_t* iteration_counter, void* cuda_stream);
 
 /* ---- LSTM cell on the kept hidden units (Sec. 7: an LSTM step is again a matrix
  * product; one row pattern over the H hidden units serves every time step) -------------

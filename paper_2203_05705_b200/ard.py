@@ -22,7 +22,7 @@ ARD_ERR_UNSUPPORTED, ARD_ERR_CUDA, ARD_ERR_TIMEOUT, ARD_ERR_NOMEM = 5, 6, 7, 8
 ARD_F32, ARD_BF16 = 0, 1
 ARD_ROW, ARD_TILE = 0, 1
 ARD_OUT_COMPACT, ARD_OUT_SCATTER_ZEROFILL = 0, 1
-ARD_FLAG_OUT_F32, ARD_FLAG_ACCUMULATE = 0x10, 0x20
+ARD_FLAG_OUT_F32, ARD_FLAG_ACCUMULATE, ARD_FLAG_RELU = 0x10, 0x20, 0x40
 ARD_PATH_AUTO, ARD_PATH_CUDA_CORE, ARD_PATH_TENSOR_CORE = 0, 1, 2
 ARD_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -31,9 +31,19 @@ EXPORTS = [
     "ard_pattern_create", "ard_pattern_destroy", "ard_sample_pattern", "ard_pattern_set",
     "ard_pattern_to_host", "ard_pattern_tile_lists_to_host", "ard_fwd", "ard_bwd_data", "ard_bwd_weight",
     "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_set_lstm_persistent", "ard_lstm_forward", "ard_lstm_backward", "ard_last_device_status", "ard_status_string", "ard_launch_count",
+    "ard_layer_fwd", "ard_layer_bwd_data", "ard_layer_bwd_weight", "ard_compact_weight_cols",
+    "ard_expand_weight_grad_cols", "ard_bias_grad", "ard_sample_pattern_counter", "ard_mlp_step",
 ]
 
 _lib = None
+
+
+class MlpLayer(C.Structure):
+    """struct ard_mlp_layer of include/ard.h (device pointers as integers)."""
+    _fields_ = [("K", C.c_int), ("N", C.c_int), ("pat", C.c_void_p), ("sample", C.c_int), ("relu", C.c_int),
+                ("compact_out", C.c_int), ("dW_is_f32", C.c_int), ("alpha", C.c_float), ("ldw", C.c_int),
+                ("W", C.c_void_p), ("bias", C.c_void_p), ("Wk", C.c_void_p), ("A", C.c_void_p), ("dZ", C.c_void_p),
+                ("dWk", C.c_void_p), ("dW", C.c_void_p), ("db", C.c_void_p)]
 
 
 class ArdError(RuntimeError):
@@ -83,6 +93,14 @@ def lib():
         "ard_lstm_gates_bwd": [vp, vp, i32, i32, i32, f32, vp, vp, vp, i32, vp, i32, i32, vp, vp, i32, vp],
         "ard_last_device_status": [vp, vp],
         "ard_launch_count": [vp],
+        "ard_layer_fwd": [vp, vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, vp, i32, i32, vp],
+        "ard_layer_bwd_data": [vp, vp, vp, i32, i32, i32, i32, f32, vp, i32, i32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_layer_bwd_weight": [vp, vp, vp, i32, i32, i32, i32, i32, f32, vp, i32, vp, i32, i32, vp, i32, i32, vp],
+        "ard_compact_weight_cols": [vp, vp, vp, i32, i32, i32, vp, i32, vp, i32, vp],
+        "ard_expand_weight_grad_cols": [vp, vp, vp, i32, i32, i32, vp, i32, vp, i32, i32, vp],
+        "ard_bias_grad": [vp, vp, i32, i32, i32, vp, i32, i32, vp, i32, vp],
+        "ard_sample_pattern_counter": [vp, vp, i32, u64, u64, vp, i32, u32, vp],
+        "ard_mlp_step": [vp, P(MlpLayer), i32, i32, vp, i32, vp, i32, vp, i32, i32, u64, u64, vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -244,6 +262,70 @@ def ard_bwd_weight(ctx, pat, dtype, dW_dtype, B, K, N, alpha, X, ldx, dY, lddy, 
     _check(lib().ard_bwd_weight(ctx, pat, dtype, dW_dtype, B, K, N, alpha, _ptr(X), ldx, _ptr(dY), lddy,
                                 dy_is_compact, _ptr(dW), lddw, zero_fill_dropped, _stream(stream)),
            "ard_bwd_weight")
+
+
+def ard_layer_fwd(ctx, pat, in_pat, dtype, B, K, N, alpha, X, ldx, Wk, ldw, bias, A, lda, outmode_and_flags,
+                  stream=None):
+    _check(lib().ard_layer_fwd(ctx, pat, in_pat, dtype, B, K, N, alpha, _ptr(X), ldx, _ptr(Wk), ldw, _ptr(bias),
+                               _ptr(A), lda, outmode_and_flags, _stream(stream)), "ard_layer_fwd")
+
+
+def ard_layer_bwd_data(ctx, pat, in_pat, dtype, B, K, N, alpha, dZ, lddz, dz_is_compact_and_flags, Wk, ldw, act_prev,
+                       ldact, dX, lddx, stream=None):
+    _check(lib().ard_layer_bwd_data(ctx, pat, in_pat, dtype, B, K, N, alpha, _ptr(dZ), lddz, dz_is_compact_and_flags,
+                                    _ptr(Wk), ldw, _ptr(act_prev), ldact, _ptr(dX), lddx, _stream(stream)),
+           "ard_layer_bwd_data")
+
+
+def ard_layer_bwd_weight(ctx, pat, in_pat, dtype, dW_dtype, B, K, N, alpha, X, ldx, dZ, lddz, dz_is_compact, dWk, lddw,
+                         zero_fill_dropped, stream=None):
+    _check(lib().ard_layer_bwd_weight(ctx, pat, in_pat, dtype, dW_dtype, B, K, N, alpha, _ptr(X), ldx, _ptr(dZ), lddz,
+                                      dz_is_compact, _ptr(dWk), lddw, zero_fill_dropped, _stream(stream)),
+           "ard_layer_bwd_weight")
+
+
+def ard_compact_weight_cols(ctx, pat, in_pat, dtype, K, N, W, ldw, Wk, ldwk, stream=None):
+    _check(lib().ard_compact_weight_cols(ctx, pat, in_pat, dtype, K, N, _ptr(W), ldw, _ptr(Wk), ldwk, _stream(stream)),
+           "ard_compact_weight_cols")
+
+
+def ard_expand_weight_grad_cols(ctx, pat, in_pat, dtype, K, N, dWk, lddwk, dW, lddw, zero_fill, stream=None):
+    _check(lib().ard_expand_weight_grad_cols(ctx, pat, in_pat, dtype, K, N, _ptr(dWk), lddwk, _ptr(dW), lddw,
+                                             zero_fill, _stream(stream)), "ard_expand_weight_grad_cols")
+
+
+def ard_bias_grad(ctx, pat, dtype, B, N, dZ, lddz, dz_is_compact, db, zero_fill_dropped, stream=None):
+    _check(lib().ard_bias_grad(ctx, pat, dtype, B, N, _ptr(dZ), lddz, dz_is_compact, _ptr(db), zero_fill_dropped,
+                               _stream(stream)), "ard_bias_grad")
+
+
+def ard_sample_pattern_counter(ctx, pat, dist_id, seed, iteration_base, iteration_counter, advance, stream_id,
+                               stream=None):
+    _check(lib().ard_sample_pattern_counter(ctx, pat, dist_id, seed, iteration_base, _ptr(iteration_counter),
+                                            1 if advance else 0, stream_id, _stream(stream)),
+           "ard_sample_pattern_counter")
+
+
+def mlp_layers(layers):
+    """Marshals a list of dicts (keys = the fields of struct ard_mlp_layer; tensors or None for the
+    pointers) into a C array.  Keep the tensors alive while the array is in use."""
+    arr = (MlpLayer * len(layers))()
+    for i, d in enumerate(layers):
+        for name, ctype in MlpLayer._fields_:
+            v = d.get(name)
+            if ctype is C.c_void_p:
+                v = v.value if isinstance(v, C.c_void_p) else _ptr(v)
+            elif v is None:
+                v = 0
+            setattr(arr[i], name, v)
+    return arr
+
+
+def ard_mlp_step(ctx, layers, n_layers, B, X, ldx, dOut, lddout, dX, lddx, dist_id, seed, iteration_base,
+                 iteration_counter, stream=None):
+    """`layers`: the array made by mlp_layers()."""
+    _check(lib().ard_mlp_step(ctx, layers, n_layers, B, _ptr(X), ldx, _ptr(dOut), lddout, _ptr(dX), lddx, dist_id,
+                              seed, iteration_base, _ptr(iteration_counter), _stream(stream)), "ard_mlp_step")
 
 
 def ard_lstm_gate_gemm(ctx, pat, B, KH, H, XH, ldxh, W, ldw, Z, ldz_gate, stream=None):

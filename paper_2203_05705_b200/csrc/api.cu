@@ -137,6 +137,11 @@ void fill_common(GemmArgs& g, ard_ctx* ctx, const ard_pattern* pat, int B, int K
   g.out_is_f32 = 0;
   g.accumulate = 0;
   g.status = ctx->d_status;
+  g.hdr_in = nullptr;
+  g.bias = nullptr;
+  g.relu = 0;
+  g.act = nullptr;
+  g.ldact = 0;
 }
 
 // Can the tcgen05 path take this call?  (bf16 only; 16-byte aligned pointers and pitches; the
@@ -474,17 +479,28 @@ ard_status ard_pattern_tile_lists_to_host(const ard_pattern* pat, int32_t* col_p
 
 // ---------------------------------------------------------------------------------------------------
 
-ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N, float alpha,
-                   const void* X, int ldx, const void* W, int ldw, void* Y, int ldy, ard_outmode outmode,
-                   void* cuda_stream) {
+// Validates the pattern of the layer that feeds a fused layer step.
+static ard_status check_in_pattern(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, int K) {
+  if (in_pat == nullptr) return ARD_OK;
+  if (in_pat->ctx != ctx || in_pat->kind != ARD_ROW || pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+  if (in_pat->N_dim != K) return ARD_ERR_SHAPE;
+  return ARD_OK;
+}
+
+static ard_status fwd_impl(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype, int B, int K,
+                           int N, float alpha, const void* X, int ldx, const void* W, int ldw, const float* bias,
+                           int relu, void* Y, int ldy, int outmode, void* cuda_stream) {
   ard_status st = check_common(ctx, pat, B, K, N);
   if (st != ARD_OK) return st;
+  st = check_in_pattern(ctx, pat, in_pat, K);
+  if (st != ARD_OK) return st;
+  if ((bias != nullptr || relu) && pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
   if (!X || !W || !Y) return ARD_ERR_INVALID_ARG;
   if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
-  const int mode = (int)outmode & 0xF;
-  const bool out_f32 = dtype == ARD_F32 || ((int)outmode & ARD_FLAG_OUT_F32);
-  const bool accumulate = ((int)outmode & ARD_FLAG_ACCUMULATE) != 0;
-  if (((int)outmode & ~(0xF | ARD_FLAG_OUT_F32 | ARD_FLAG_ACCUMULATE)) != 0) return ARD_ERR_INVALID_ARG;
+  const int mode = outmode & 0xF;
+  const bool out_f32 = dtype == ARD_F32 || (outmode & ARD_FLAG_OUT_F32);
+  const bool accumulate = (outmode & ARD_FLAG_ACCUMULATE) != 0;
+  if ((outmode & ~(0xF | ARD_FLAG_OUT_F32 | ARD_FLAG_ACCUMULATE)) != 0) return ARD_ERR_INVALID_ARG;
   if (mode != ARD_OUT_COMPACT && mode != ARD_OUT_SCATTER_ZEROFILL) return ARD_ERR_INVALID_ARG;
   if (accumulate && mode == ARD_OUT_SCATTER_ZEROFILL && pat->kind == ARD_ROW) return ARD_ERR_INVALID_ARG;
   if (ldx < K || ldw < K || ldy < N) return ARD_ERR_SHAPE;
@@ -499,9 +515,14 @@ ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B,
   g.flag0 = pat->kind == ARD_ROW ? mode : 0;
   g.out_is_f32 = out_f32;
   g.accumulate = accumulate;
+  g.hdr_in = in_pat ? in_pat->d_hdr : nullptr;
+  g.bias = bias;
+  g.relu = relu ? 1 : 0;
+  if (accumulate && (bias != nullptr || relu)) return ARD_ERR_INVALID_ARG;
 
   ard_status el = ctx->path == ARD_PATH_CUDA_CORE ? ARD_ERR_UNSUPPORTED
                                                   : tc_eligible(ctx, pat, dtype, B, K, N, X, ldx, W, ldw, Y, ldy, es);
+  if (el == ARD_OK && in_pat && in_pat->dp_bound > ARD_MAX_NDP_TC) el = ARD_ERR_UNSUPPORTED;
   // the tensor-core scatter epilogue writes bf16 only
   if (el == ARD_OK && out_f32 && pat->kind == ARD_ROW && mode == ARD_OUT_SCATTER_ZEROFILL) el = ARD_ERR_UNSUPPORTED;
   if (el != ARD_OK) {
@@ -513,9 +534,15 @@ ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B,
   t.ts = pat->ts;
   t.bn = tc_pick_bn(ctx, pat->kind, OP_FWD, pat->dp_bound, pat->ts);
   // A = X, K-major boxes [128 rows][64 k];  B = kept neurons of W, K-major boxes [64 rows][64 k].
-  st = get_maps(ctx, X, B, K, ldx, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);
+  if (in_pat) {
+    // compact X: one descriptor per pattern of the feeding layer, whose extent ends at its kept count
+    st = get_maps(ctx, X, B, K, ldx, K, MAP_COMPACT_COLS, in_pat->dp_bound, 128, 64, &t.mapA);
+    t.mapA_indexed = 2;
+  } else {
+    st = get_maps(ctx, X, B, K, ldx, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);
+    t.mapA_indexed = 0;
+  }
   if (st != ARD_OK) return st;
-  t.mapA_indexed = 0;
   if (pat->kind == ARD_ROW) {
     st = get_maps(ctx, W, N, K, ldw, N, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64, &t.mapB);
     t.mapB_indexed = 1;
@@ -525,6 +552,22 @@ ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B,
   }
   if (st != ARD_OK) return st;
   return launch_gemm_tc(ctx, pat->kind, OP_FWD, t, s);
+}
+
+ard_status ard_fwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N, float alpha,
+                   const void* X, int ldx, const void* W, int ldw, void* Y, int ldy, ard_outmode outmode,
+                   void* cuda_stream) {
+  if (((int)outmode & ARD_FLAG_RELU) != 0) return ARD_ERR_INVALID_ARG;
+  return fwd_impl(ctx, pat, nullptr, dtype, B, K, N, alpha, X, ldx, W, ldw, nullptr, 0, Y, ldy, (int)outmode, cuda_stream);
+}
+
+ard_status ard_layer_fwd(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype, int B, int K,
+                         int N, float alpha, const void* X, int ldx, const void* W, int ldw, const float* bias, void* A,
+                         int lda, int outmode, void* cuda_stream) {
+  if (!pat || pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+  const int relu = (outmode & ARD_FLAG_RELU) ? 1 : 0;
+  return fwd_impl(ctx, pat, in_pat, dtype, B, K, N, alpha, X, ldx, W, ldw, bias, relu, A, lda, outmode & ~ARD_FLAG_RELU,
+                  cuda_stream);
 }
 
 // Produces the operand the tensor-core backward GEMMs read for dY: the caller's compact matrix, or
@@ -557,11 +600,14 @@ static ard_status compact_dy(ard_ctx* ctx, const ard_pattern* pat, int B, int N,
   return st;
 }
 
-ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N, float alpha,
-                        const void* dY, int lddy, int dy_is_compact, const void* W, int ldw, void* dX, int lddx,
-                        void* cuda_stream) {
+static ard_status bwd_data_impl(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype, int B,
+                                int K, int N, float alpha, const void* dY, int lddy, int dy_is_compact, const void* W,
+                                int ldw, const void* act, int ldact, void* dX, int lddx, void* cuda_stream) {
   ard_status st = check_common(ctx, pat, B, K, N);
   if (st != ARD_OK) return st;
+  st = check_in_pattern(ctx, pat, in_pat, K);
+  if (st != ARD_OK) return st;
+  if (act != nullptr && (pat->kind != ARD_ROW || ldact < 1)) return ARD_ERR_INVALID_ARG;
   if (!dY || !W || !dX) return ARD_ERR_INVALID_ARG;
   if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
   const int flags = dy_is_compact;
@@ -581,10 +627,16 @@ ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, i
   g.flag0 = dy_is_compact ? 1 : 0;
   g.out_is_f32 = out_f32;
   g.accumulate = (flags & ARD_FLAG_ACCUMULATE) != 0;
+  g.hdr_in = in_pat ? in_pat->d_hdr : nullptr;
+  g.act = act;
+  g.ldact = ldact;
+  if (g.accumulate && act != nullptr) return ARD_ERR_INVALID_ARG;
 
   ard_status el = ctx->path == ARD_PATH_CUDA_CORE
                       ? ARD_ERR_UNSUPPORTED
                       : tc_eligible(ctx, pat, dtype, B, K, N, dY, lddy, W, ldw, dX, lddx, es);
+  // the tensor-core epilogue reads the activations in 16-byte pieces
+  if (el == ARD_OK && act != nullptr && (!aligned16(act) || ldact % 8 != 0)) el = ARD_ERR_ALIGNMENT;
   if (el == ARD_OK && pat->kind == ARD_ROW && !dy_is_compact &&
       (size_t)B * ((N + 7) / 8 * 8) * 2 > ctx->workspace_bytes)
     el = ARD_ERR_NOMEM;
@@ -619,10 +671,28 @@ ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, i
   return launch_gemm_tc(ctx, pat->kind, OP_BWD_DATA, t, s);
 }
 
-ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, ard_dtype dW_dtype, int B, int K,
-                          int N, float alpha, const void* X, int ldx, const void* dY, int lddy, int dy_is_compact,
-                          void* dW, int lddw, int zero_fill_dropped, void* cuda_stream) {
+ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N, float alpha,
+                        const void* dY, int lddy, int dy_is_compact, const void* W, int ldw, void* dX, int lddx,
+                        void* cuda_stream) {
+  return bwd_data_impl(ctx, pat, nullptr, dtype, B, K, N, alpha, dY, lddy, dy_is_compact, W, ldw, nullptr, 0, dX, lddx,
+                       cuda_stream);
+}
+
+ard_status ard_layer_bwd_data(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype, int B,
+                              int K, int N, float alpha, const void* dZ, int lddz, int flags, const void* W, int ldw,
+                              const void* act, int ldact, void* dX, int lddx, void* cuda_stream) {
+  if (!pat || pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+  return bwd_data_impl(ctx, pat, in_pat, dtype, B, K, N, alpha, dZ, lddz, flags, W, ldw, act, ldact, dX, lddx,
+                       cuda_stream);
+}
+
+static ard_status bwd_weight_impl(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
+                                  ard_dtype dW_dtype, int B, int K, int N, float alpha, const void* X, int ldx,
+                                  const void* dY, int lddy, int dy_is_compact, void* dW, int lddw,
+                                  int zero_fill_dropped, void* cuda_stream) {
   ard_status st = check_common(ctx, pat, B, K, N);
+  if (st != ARD_OK) return st;
+  st = check_in_pattern(ctx, pat, in_pat, K);
   if (st != ARD_OK) return st;
   if (!X || !dY || !dW) return ARD_ERR_INVALID_ARG;
   if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
@@ -640,6 +710,7 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
   g.flag0 = dy_is_compact ? 1 : 0;
   g.flag1 = zero_fill_dropped ? 1 : 0;
   g.out_is_f32 = dW_dtype == ARD_F32;
+  g.hdr_in = in_pat ? in_pat->d_hdr : nullptr;
   // Empty batch: the gradient of every kept weight is zero; the CUDA-core kernel writes exactly that.
   if (B == 0) return launch_gemm_cc(ctx, pat->kind, OP_BWD_WEIGHT, dtype, g, pat->ts, s);
 
@@ -676,6 +747,77 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
   if (st != ARD_OK) return st;
   t.g = g;
   return launch_gemm_tc(ctx, pat->kind, OP_BWD_WEIGHT, t, s);
+}
+
+ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, ard_dtype dW_dtype, int B, int K,
+                          int N, float alpha, const void* X, int ldx, const void* dY, int lddy, int dy_is_compact,
+                          void* dW, int lddw, int zero_fill_dropped, void* cuda_stream) {
+  return bwd_weight_impl(ctx, pat, nullptr, dtype, dW_dtype, B, K, N, alpha, X, ldx, dY, lddy, dy_is_compact, dW, lddw,
+                         zero_fill_dropped, cuda_stream);
+}
+
+ard_status ard_layer_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
+                                ard_dtype dW_dtype, int B, int K, int N, float alpha, const void* X, int ldx,
+                                const void* dZ, int lddz, int dz_is_compact, void* dW, int lddw, int zero_fill_dropped,
+                                void* cuda_stream) {
+  if (!pat || pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+  return bwd_weight_impl(ctx, pat, in_pat, dtype, dW_dtype, B, K, N, alpha, X, ldx, dZ, lddz, dz_is_compact, dW, lddw,
+                         zero_fill_dropped, cuda_stream);
+}
+
+ard_status ard_compact_weight_cols(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
+                                   int K, int N, const void* W, int ldw, void* Wk, int ldwk, void* cuda_stream) {
+  ard_status st = check_common(ctx, pat, 0, K, N);
+  if (st != ARD_OK) return st;
+  if (!in_pat || !W || !Wk) return ARD_ERR_INVALID_ARG;
+  st = check_in_pattern(ctx, pat, in_pat, K);
+  if (st != ARD_OK) return st;
+  if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (ldw < K || ldwk < K) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  return launch_compact_weight_cols(ctx, pat->d_hdr, in_pat->d_hdr, W, ldw, Wk, ldwk, N, K, dtype == ARD_F32 ? 4 : 2,
+                                    (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_expand_weight_grad_cols(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
+                                       int K, int N, const void* dWk, int lddwk, void* dW, int lddw, int zero_fill,
+                                       void* cuda_stream) {
+  ard_status st = check_common(ctx, pat, 0, K, N);
+  if (st != ARD_OK) return st;
+  if (!in_pat || !dWk || !dW || dWk == dW) return ARD_ERR_INVALID_ARG;
+  st = check_in_pattern(ctx, pat, in_pat, K);
+  if (st != ARD_OK) return st;
+  if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (lddwk < K || lddw < K) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  return launch_expand_weight_grad_cols(ctx, pat->d_hdr, in_pat->d_hdr, dWk, lddwk, dW, lddw, N, K,
+                                        dtype == ARD_F32 ? 4 : 2, zero_fill, (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_bias_grad(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int N, const void* dZ, int lddz,
+                         int dz_is_compact, float* db, int zero_fill_dropped, void* cuda_stream) {
+  if (!ctx || !pat || pat->ctx != ctx || pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
+  if (B < 0 || N != pat->N_dim) return ARD_ERR_SHAPE;
+  if (!dZ || !db) return ARD_ERR_INVALID_ARG;
+  if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (lddz < (dz_is_compact ? 1 : N)) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  return launch_bias_grad(ctx, pat->d_hdr, dZ, lddz, dz_is_compact ? 1 : 0, dtype == ARD_BF16, B, N, db,
+                          zero_fill_dropped, (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_sample_pattern_counter(ard_ctx* ctx, ard_pattern* pat, int dist_id, uint64_t seed, uint64_t iteration_base,
+                                      uint64_t* iteration_counter, int advance, uint32_t stream_id,
+                                      void* cuda_stream) {
+  if (!ctx || !pat || pat->ctx != ctx || !iteration_counter) return ARD_ERR_INVALID_ARG;
+  if (dist_id < 0 || dist_id >= ARD_MAX_DISTRIBUTIONS) return ARD_ERR_INVALID_ARG;
+  const ArdDistribution& d = ctx->dist[dist_id];
+  if (d.ndp == 0 || d.ndp > pat->units) return ARD_ERR_DISTRIBUTION;
+  DeviceGuard guard(ctx->device);
+  pat->dp_bound = d.ndp;
+  pat->generation++;
+  return launch_sampler(ctx, pat, d.d_cdf, d.ndp, seed, iteration_base, stream_id, 0, 0, (cudaStream_t)cuda_stream,
+                        reinterpret_cast<unsigned long long*>(iteration_counter), advance ? 1 : 0);
 }
 
 // ---------------------------------------------------------------------------------------------------

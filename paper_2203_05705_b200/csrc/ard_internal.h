@@ -104,7 +104,7 @@ static inline int map_index_count(int dp_bound) { return dp_bound * (dp_bound + 
 // ---- launchers implemented in the .cu files -----------------------------------------------------
 ard_status launch_sampler(ard_ctx* ctx, ard_pattern* pat, const unsigned long long* d_cdf, int ndp,
                           uint64_t seed, uint64_t iteration, uint32_t stream_id, int forced_dp, int forced_b,
-                          cudaStream_t s);
+                          cudaStream_t s, unsigned long long* d_counter = nullptr, int advance = 0);
 
 struct GemmArgs {
   const int32_t* hdr;
@@ -126,6 +126,14 @@ struct GemmArgs {
   int out_is_f32;
   int accumulate;  // add to the existing output instead of overwriting it
   int* status;
+  // Fused layer step (row patterns).  hdr_in: header of the row pattern of the layer that produced the
+  // input; the input matrix and the weight then hold only that layer's kept columns (n_in of them), so
+  // the fan-in extent of the product is n_in instead of K.
+  const int32_t* hdr_in;
+  const float* bias;  // forward: added before the activation, indexed by the original neuron
+  int relu;           // forward: max(., 0) before the rescale
+  const void* act;    // backward-data: the output is zeroed where act <= 0 (operand element type, layout of dX)
+  int ldact;
 };
 
 enum GemmOp { OP_FWD = 0, OP_BWD_DATA = 1, OP_BWD_WEIGHT = 2 };
@@ -140,7 +148,7 @@ struct TcArgs {
   const CUtensorMap* mapB;
   const CUtensorMap* mapA4[4];  // LSTM gate products: one table per gate
   const CUtensorMap* mapB4[4];
-  int mapA_indexed, mapB_indexed;
+  int mapA_indexed, mapB_indexed;  // 0: a single descriptor, 1: table indexed by the pattern, 2: by the input pattern
   GemmArgs g;
   int ts;
   int bn;  // N tile: 64, 128 or 256
@@ -165,6 +173,15 @@ ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* i
                               void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, int skip_dense,
                               cudaStream_t s);
 
+// Layer-step helpers (aux_kernels.cu); elem_bytes 2 or 4.
+ard_status launch_compact_weight_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* hdr_in, const void* W, int ldw,
+                                      void* Wk, int ldwk, int N, int K, int elem_bytes, cudaStream_t s);
+ard_status launch_expand_weight_grad_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* hdr_in, const void* dWk,
+                                          int lddwk, void* dW, int lddw, int N, int K, int elem_bytes, int zero_fill,
+                                          cudaStream_t s);
+ard_status launch_bias_grad(ard_ctx* ctx, const int32_t* hdr, const void* dZ, int lddz, int dz_is_compact,
+                            int elem_bytes_is_bf16, int B, int N, float* db, int zero_fill, cudaStream_t s);
+
 ard_status launch_lstm_gates(ard_ctx* ctx, const ard_pattern* pat, ard_dtype h_dtype, int B, int H, float alpha,
                              const float* Z, int ldz_gate, const float* bias, const float* c_prev, int ldc, float* c,
                              void* h, int ldh, int h_scatter, float* gates_saved, cudaStream_t s);
@@ -185,6 +202,17 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 
+// While a stream is being captured into a CUDA graph the kernels are launched the ordinary way: replays
+// of a graph whose nodes were joined by programmatic edges were seen to read the pattern header of the
+// previous replay in some blocks of the kernel that follows the sampler (never seen in stream order), and
+// inside a graph the launch latency that the early start hides is small anyway.
+inline bool ard_pdl_allowed(const ard_ctx* ctx, cudaStream_t s) {
+  if (!ctx->use_pdl) return false;
+  cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &st) != cudaSuccess) return false;
+  return st == cudaStreamCaptureStatusNone;
+}
+
 template <typename... P, typename... A>
 inline cudaError_t ard_launch(const ard_ctx* ctx, void (*kern)(P...), dim3 grid, dim3 block, size_t smem,
                               cudaStream_t s, A... args) {
@@ -194,7 +222,7 @@ inline cudaError_t ard_launch(const ard_ctx* ctx, void (*kern)(P...), dim3 grid,
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
-  if (ctx->use_pdl) {
+  if (ard_pdl_allowed(ctx, s)) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;

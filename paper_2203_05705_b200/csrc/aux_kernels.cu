@@ -166,6 +166,104 @@ lstm_gates_bwd_kernel(const int32_t* __restrict__ hdr, int B, int H, float alpha
   dz[3 * ldz + j] = ZT(d_o * go * (1.f - go));
 }
 
+// ---- layer-step helpers (Sec. 3.1: the weight is compacted along the fan-in too when the layer that
+// feeds it ran under a row pattern) -----------------------------------------------------------------
+//
+// Wk[n][j] = W[n][b_in-1 + j*dp_in] for the kept neurons n of `hdr` and j < n_in; columns n_in up to the
+// next multiple of 64 (or ldwk) are written as zero, so that the last 64-wide contraction block of the
+// tensor-core forward product multiplies zeros.  Eight outputs per thread (one 16- or 32-byte store).
+template <typename T>
+__global__ void __launch_bounds__(256) compact_weight_cols_kernel(const int32_t* __restrict__ hdr,
+                                                                  const int32_t* __restrict__ hdr_in,
+                                                                  const T* __restrict__ W, int ldw, T* __restrict__ Wk,
+                                                                  int ldwk, int vec_ok) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
+  const int n_in = hdr_in[HDR_NKEEP], dpi = hdr_in[HDR_DP], bi = hdr_in[HDR_B] - 1;
+  const int padded = min(ldwk, (n_in + 63) / 64 * 64);
+  const int groups = (padded + 7) / 8;
+  for (int i = blockIdx.y; i < n_keep; i += gridDim.y) {
+    const size_t row = (size_t)bb + (size_t)i * dp;
+    const T* src = W + row * ldw + bi;
+    T* dst = Wk + row * ldwk;
+    for (int g = blockIdx.x * 256 + threadIdx.x; g < groups; g += gridDim.x * 256) {
+      const int j0 = g * 8;
+      __align__(16) T v[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) v[q] = (j0 + q < n_in) ? src[(size_t)(j0 + q) * dpi] : T(0.f);
+      if (vec_ok && j0 + 8 <= padded) {
+        if (sizeof(T) == 2) {
+          *reinterpret_cast<uint4*>(dst + j0) = *reinterpret_cast<const uint4*>(v);
+        } else {
+          reinterpret_cast<uint4*>(dst + j0)[0] = reinterpret_cast<const uint4*>(v)[0];
+          reinterpret_cast<uint4*>(dst + j0)[1] = reinterpret_cast<const uint4*>(v)[1];
+        }
+      } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          if (j0 + q < padded) dst[j0 + q] = v[q];
+      }
+    }
+  }
+}
+
+// The inverse for the gradient: dW[n][b_in-1 + j*dp_in] = dWk[n][j] for kept neurons n; with zero_fill
+// every other entry of dW [N][K] (dropped neurons, dropped inputs) is written as zero, without it they
+// are left alone.  One output row per blockIdx.y step, consecutive threads write consecutive columns.
+template <typename T>
+__global__ void __launch_bounds__(256) expand_weight_grad_cols_kernel(const int32_t* __restrict__ hdr,
+                                                                      const int32_t* __restrict__ hdr_in,
+                                                                      const T* __restrict__ dWk, int lddwk,
+                                                                      T* __restrict__ dW, int lddw, int N, int K,
+                                                                      int zero_fill) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
+  const int dpi = hdr_in[HDR_DP], bi = hdr_in[HDR_B] - 1;
+  for (int n = blockIdx.y; n < N; n += gridDim.y) {
+    const bool kept_row = n >= bb && (n - bb) % dp == 0;
+    if (!kept_row && !zero_fill) continue;
+    const T* src = dWk + (size_t)n * lddwk;
+    T* dst = dW + (size_t)n * lddw;
+    for (int k = blockIdx.x * 256 + threadIdx.x; k < K; k += gridDim.x * 256) {
+      const bool kept = kept_row && k >= bi && (k - bi) % dpi == 0;
+      if (kept) dst[k] = src[(k - bi) / dpi];
+      else if (zero_fill) dst[k] = T(0.f);
+    }
+  }
+}
+
+// Bias gradient of a layer step: db[n] = sum over the batch of dZ[:, n] for the kept neurons (Sec. 3.1:
+// a dropped neuron takes no part in the iteration); dropped entries are zeroed on request.
+// A block owns 32 consecutive neurons; its 8 row groups add their rows in a fixed order.
+template <typename T>
+__global__ void __launch_bounds__(256) bias_grad_kernel(const int32_t* __restrict__ hdr, const T* __restrict__ dZ,
+                                                        int lddz, int dz_is_compact, int B, int N,
+                                                        float* __restrict__ db, int zero_fill) {
+  __shared__ float part[8][33];
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int n = blockIdx.x * 32 + tx;
+  const bool kept = n < N && n >= bb && (n - bb) % dp == 0;
+  float acc = 0.f;
+  if (kept) {
+    const int col = dz_is_compact ? (n - bb) / dp : n;
+    for (int r = ty; r < B; r += 8) acc += (float)dZ[(size_t)r * lddz + col];
+  }
+  part[ty][tx] = acc;
+  __syncthreads();
+  if (ty == 0 && n < N) {
+    float sum = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) sum += part[q][tx];
+    if (kept) db[n] = sum;
+    else if (zero_fill) db[n] = 0.f;
+  }
+}
+
 }  // namespace
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,
@@ -221,6 +319,53 @@ ard_status launch_lstm_gates_bwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype
     ARD_CUDA_OK(ard_launch(ctx, lstm_gates_bwd_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, (const int32_t*)pat->d_hdr, B,
                            H, alpha, gates_saved, c_prev, c, ldc, dh, lddh, dh_scatter, dc_inout, (__nv_bfloat16*)dZ,
                            ldz_gate));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+ard_status launch_compact_weight_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* hdr_in, const void* W, int ldw,
+                                      void* Wk, int ldwk, int N, int K, int elem_bytes, cudaStream_t s) {
+  if (N == 0 || K == 0) return ARD_OK;
+  const int vec_ok = (reinterpret_cast<uintptr_t>(Wk) & 15) == 0 && ((size_t)ldwk * elem_bytes) % 16 == 0 && ldwk % 8 == 0;
+  dim3 grid((K / 8 + 255) / 256 > 0 ? (K / 8 + 255) / 256 : 1, N < 65535 ? N : 65535);
+  if (elem_bytes == 2)
+    ARD_CUDA_OK(ard_launch(ctx, compact_weight_cols_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, hdr, hdr_in,
+                           (const __nv_bfloat16*)W, ldw, (__nv_bfloat16*)Wk, ldwk, vec_ok));
+  else
+    ARD_CUDA_OK(ard_launch(ctx, compact_weight_cols_kernel<float>, grid, dim3(256), 0, s, hdr, hdr_in, (const float*)W,
+                           ldw, (float*)Wk, ldwk, vec_ok));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+ard_status launch_expand_weight_grad_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* hdr_in, const void* dWk,
+                                          int lddwk, void* dW, int lddw, int N, int K, int elem_bytes, int zero_fill,
+                                          cudaStream_t s) {
+  if (N == 0 || K == 0) return ARD_OK;
+  dim3 grid((K + 1023) / 1024, N < 65535 ? N : 65535);
+  if (elem_bytes == 2)
+    ARD_CUDA_OK(ard_launch(ctx, expand_weight_grad_cols_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, hdr, hdr_in,
+                           (const __nv_bfloat16*)dWk, lddwk, (__nv_bfloat16*)dW, lddw, N, K, zero_fill));
+  else
+    ARD_CUDA_OK(ard_launch(ctx, expand_weight_grad_cols_kernel<float>, grid, dim3(256), 0, s, hdr, hdr_in,
+                           (const float*)dWk, lddwk, (float*)dW, lddw, N, K, zero_fill));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+ard_status launch_bias_grad(ard_ctx* ctx, const int32_t* hdr, const void* dZ, int lddz, int dz_is_compact,
+                            int is_bf16, int B, int N, float* db, int zero_fill, cudaStream_t s) {
+  if (N == 0) return ARD_OK;
+  dim3 grid((N + 31) / 32);
+  if (is_bf16)
+    ARD_CUDA_OK(ard_launch(ctx, bias_grad_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, hdr, (const __nv_bfloat16*)dZ,
+                           lddz, dz_is_compact, B, N, db, zero_fill));
+  else
+    ARD_CUDA_OK(ard_launch(ctx, bias_grad_kernel<float>, grid, dim3(256), 0, s, hdr, (const float*)dZ, lddz,
+                           dz_is_compact, B, N, db, zero_fill));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;

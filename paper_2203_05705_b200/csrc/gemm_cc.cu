@@ -42,9 +42,11 @@ __global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts)
   const int m0 = blockIdx.y * T_M, n0 = blockIdx.x * T_N;
   const int32_t* klist = nullptr;  // tile patterns: contraction runs over ts-wide blocks klist[0..]
   if (KIND == 0) {
-    if (OP == OP_FWD) { M = g.B; N = n_keep; nk = g.K; }
-    else if (OP == OP_BWD_DATA) { M = g.B; N = g.K; nk = n_keep; }
-    else { M = n_keep; N = g.K; nk = g.B; }
+    // fan-in extent: all K inputs, or the kept outputs of the layer that produced the input
+    const int kin = g.hdr_in != nullptr ? g.hdr_in[HDR_NKEEP] : g.K;
+    if (OP == OP_FWD) { M = g.B; N = n_keep; nk = kin; }
+    else if (OP == OP_BWD_DATA) { M = g.B; N = kin; nk = n_keep; }
+    else { M = n_keep; N = kin; nk = g.B; }
   } else {
     if (OP == OP_FWD) {
       M = g.B; N = g.N;
@@ -149,7 +151,18 @@ __global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts)
       if (KIND == 0 && OP == OP_FWD) off = (size_t)m * g.ldo + (g.flag0 == ARD_OUT_SCATTER_ZEROFILL ? g.idx[n] : n);
       else if (KIND == 0 && OP == OP_BWD_WEIGHT) off = (size_t)g.idx[m] * g.ldo + n;
       else off = (size_t)m * g.ldo + n;
-      store_out(g.out, off, g.alpha * acc[i][j], g.out_is_f32, g.accumulate);
+      float v = acc[i][j];
+      if (KIND == 0 && OP == OP_FWD) {
+        // layer step: bias, then the activation, then the rescale (Sec. 3.2, last paragraph)
+        if (g.bias != nullptr) v += g.bias[g.idx[n]];
+        if (g.relu) v = fmaxf(v, 0.f);
+      }
+      v *= g.alpha;
+      if (KIND == 0 && OP == OP_BWD_DATA && g.act != nullptr) {
+        // adjoint of the producing layer's ReLU: nothing flows where its output was not positive
+        if (!(to_f<T>(reinterpret_cast<const T*>(g.act)[(size_t)m * g.ldact + n]) > 0.f)) v = 0.f;
+      }
+      store_out(g.out, off, v, g.out_is_f32, g.accumulate);
     }
 }
 

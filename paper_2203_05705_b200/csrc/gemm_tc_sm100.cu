@@ -90,6 +90,12 @@ struct TcParams {
   int sk_min_blocks;  // fewest contraction blocks worth a separate share
   int sk_min_gain;    // fewest contraction blocks sharing must take off the last wave to be used
   int* status;
+  // Fused layer step (kernels instantiated with FUSED): see GemmArgs.
+  const int32_t* hdr_in;
+  const float* bias;
+  int relu;
+  const void* act;
+  int ldact;
 };
 
 // CTAS = 2: a cluster of two CTAs shares one 256 x BN output tile; each CTA stages its own 128 rows
@@ -175,7 +181,8 @@ struct Sched {
     return kt - (rem * kt + S - 1) / S >= min_gain ? S : 0;
   }
 
-  __device__ void init(const TcParams& p, int rank_) {
+  // kin: fan-in extent of the row products (K, or the kept outputs of the layer that feeds this one)
+  __device__ void init(const TcParams& p, int rank_, int kin) {
     rank = rank_;
     workers = (int)gridDim.x / CTAS;
     dp = p.hdr[HDR_DP];
@@ -184,11 +191,11 @@ struct Sched {
     Tc = p.hdr[HDR_TC];
     subm = subn = 1;
     KT = sk_tiles = sk_S = sk_blocks = 0;
-    if (MODE == M_ROW_FWD) { M_gemm = p.B; N_gemm = n_keep; Kc = p.K; }
-    else if (MODE == M_ROW_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = n_keep; }
+    if (MODE == M_ROW_FWD) { M_gemm = p.B; N_gemm = n_keep; Kc = kin; }
+    else if (MODE == M_ROW_BWD_DATA) { M_gemm = p.B; N_gemm = kin; Kc = n_keep; }
     else if (MODE == M_LSTM_FWD) { M_gemm = p.B; N_gemm = ((n_keep + 63) / 64) * 256; Kc = p.K; }
     else if (MODE == M_LSTM_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 4 * (((n_keep + 63) / 64) * 64); }
-    else if (MODE == M_ROW_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = p.K; Kc = p.B; }
+    else if (MODE == M_ROW_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = kin; Kc = p.B; }
     else if (MODE == M_TILE_FWD || MODE == M_TILEC_FWD) { M_gemm = p.B; N_gemm = p.N; Kc = 0; }
     else if (MODE == M_TILE_BWD_DATA || MODE == M_TILEC_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 0; }
     else { M_gemm = p.N; N_gemm = p.K; Kc = p.B; }
@@ -523,7 +530,7 @@ __device__ __forceinline__ void zero_row32(void* out, size_t row_off, int col, i
 }
 
 // ---- the kernel -----------------------------------------------------------------------------------
-template <int BN, int MODE, int CTAS, bool SHARE>
+template <int BN, int MODE, int CTAS, bool SHARE, bool FUSED>
 __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcParams p) {
   using L = SmemLayout<BN, CTAS>;
   const uint32_t rank = (CTAS == 2) ? cluster_ctarank() : 0u;  // rank 0 leads the pair and issues its MMAs
@@ -578,7 +585,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   pdl_wait_prior_grids();
 
   Sched<BN, MODE, CTAS, SHARE> sch;
-  sch.init(p, (int)rank);
+  sch.init(p, (int)rank, (FUSED && p.hdr_in != nullptr) ? p.hdr_in[HDR_NKEEP] : p.K);
   if (is_class_mode(MODE) && !sch.dense) {
     // The producer reads one list entry per contraction block: keep the list in shared memory (the
     // staging area of the forward scatter epilogue is free in these modes) instead of paying a
@@ -603,8 +610,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
     // ===================== TMA producer =====================
     if (lane == 0) {
       const int e = p.hdr[HDR_MAPIDX];
-      const CUtensorMap* mapA = p.mapA + (p.mapA_indexed ? e : 0);
-      const CUtensorMap* mapB = p.mapB + (p.mapB_indexed ? e : 0);
+      // a table is indexed by this layer's pattern (1) or by the pattern of the layer that feeds it (2)
+      const int e_in = (FUSED && p.hdr_in != nullptr) ? p.hdr_in[HDR_MAPIDX] : 0;
+      const CUtensorMap* mapA = p.mapA + (p.mapA_indexed == 2 ? e_in : (p.mapA_indexed ? e : 0));
+      const CUtensorMap* mapB = p.mapB + (p.mapB_indexed == 2 ? e_in : (p.mapB_indexed ? e : 0));
       tensormap_acquire(mapA);
       tensormap_acquire(mapB);
       if (MODE == M_LSTM_FWD || MODE == M_LSTM_BWD_DATA) {
@@ -775,8 +784,41 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         if (oc < 0) return;                    // padding of a class tile
         const int n = oc + (ch & 1) * 32;      // output column of this chunk
         float v[32];
+        if (FUSED && MODE == M_ROW_FWD) {
+          // layer step: bias of the original neuron, activation, rescale (Sec. 3.2, last paragraph)
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = has_acc ? p.alpha * __uint_as_float(r[i]) : 0.f;
+          for (int i = 0; i < 32; ++i) {
+            float z = has_acc ? __uint_as_float(r[i]) : 0.f;
+            if (p.bias != nullptr && n + i < sch.n_keep) z += __ldg(p.bias + bb + (n + i) * dp);
+            if (p.relu) z = fmaxf(z, 0.f);
+            v[i] = p.alpha * z;
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = has_acc ? p.alpha * __uint_as_float(r[i]) : 0.f;
+        }
+        if (FUSED && MODE == M_ROW_BWD_DATA && p.act != nullptr && row_ok) {
+          // adjoint of the producing layer's ReLU: zero where its (saved) output was not positive
+          const __nv_bfloat16* arow = reinterpret_cast<const __nv_bfloat16*>(p.act) + (size_t)m * p.ldact + n;
+          const int na = min(32, sch.N_gemm - n);
+          if (na >= 32) {
+#pragma unroll
+            for (int q8 = 0; q8 < 4; ++q8) {
+              const uint4 a = __ldg(reinterpret_cast<const uint4*>(arow) + q8);
+              const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+              for (int h = 0; h < 8; ++h) {
+                // bf16 > 0: sign bit clear and magnitude non-zero
+                const uint32_t bits = (w[h >> 1] >> ((h & 1) * 16)) & 0xFFFFu;
+                if ((bits & 0x8000u) || (bits & 0x7FFFu) == 0u || (bits & 0x7FFFu) > 0x7F80u) v[q8 * 8 + h] = 0.f;
+              }
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (i < na && !(__bfloat162float(arow[i]) > 0.f)) v[i] = 0.f;
+          }
+        }
 
         if (MODE == M_ROW_FWD && p.scatter && dp > 1) {
           // Full-width rows: compact column j -> column b-1 + j*dp, zeros everywhere else
@@ -998,12 +1040,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
 }
 
 // max_tiles: tile count of the densest pattern
-template <int BN, int MODE, int CTAS, bool SHARE = false>
+template <int BN, int MODE, int CTAS, bool SHARE = false, bool FUSED = false>
 ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStream_t s) {
   using L = SmemLayout<BN, CTAS>;
   static bool attr_done[64] = {};
   static int max_clusters[64] = {};
-  auto kern = ard_gemm_tc_kernel<BN, MODE, CTAS, SHARE>;
+  auto kern = ard_gemm_tc_kernel<BN, MODE, CTAS, SHARE, FUSED>;
   const int dev = ctx->device & 63;
   if (!attr_done[dev]) {
     ARD_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL));
@@ -1036,7 +1078,7 @@ ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStrea
   if (workers < 1) workers = 1;
   if (workers * CTAS > ctx->sm_count) return ARD_ERR_UNSUPPORTED;  // the partial-sum scratch is sized per SM
   cfg.gridDim = dim3(workers * CTAS);
-  if (ctx->use_pdl) {
+  if (ard_pdl_allowed(ctx, s)) {
     attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
     cfg.numAttrs++;
@@ -1100,14 +1142,24 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
   p.sk_cnt = ctx->d_sk_cnt;
   p.sk_min_blocks = ctx->sk_min_blocks;
   p.sk_min_gain = ctx->sk_min_gain;
+  p.hdr_in = a.g.hdr_in;
+  p.bias = a.g.bias;
+  p.relu = a.g.relu;
+  p.act = a.g.act;
+  p.ldact = a.g.ldact;
+  // the layer-step variants are separate instantiations, so that the plain products carry none of their code
+  const bool fused = kind == ARD_ROW && (p.hdr_in != nullptr || p.bias != nullptr || p.relu != 0 || p.act != nullptr);
   const int bn = (kind == ARD_ROW) ? 256 : a.bn;
 
 #define ARD_TC_CASE(BN_, MODE_, TILES_) \
   if (bn == BN_) return launch_mode<BN_, MODE_, 1>(ctx, p, (TILES_), s);
 #define ARD_TC_ROW(MODE_, TILES_)                                                      \
+  if (fused) return launch_mode<256, MODE_, 1, false, true>(ctx, p, (TILES_), s);      \
   return share ? launch_mode<256, MODE_, 1, true>(ctx, p, (TILES_), s) : launch_mode<256, MODE_, 1, false>(ctx, p, (TILES_), s);
   // Row patterns with at least two 128-row tiles of output use CTA pairs (256-row tiles).
 #define ARD_TC_PAIR(MODE_, MROWS_, NCOLS_)                                                      \
+  if (ctx->use_pairs && (MROWS_) > BM && (p.force_bn == 0 || p.force_bn >= 128) && fused)       \
+    return launch_mode<256, MODE_, 2, false, true>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s);         \
   if (ctx->use_pairs && (MROWS_) > BM && (p.force_bn == 0 || p.force_bn >= 128))                \
     return share ? launch_mode<256, MODE_, 2, true>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s)         \
                  : launch_mode<256, MODE_, 2, false>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s);
@@ -1189,6 +1241,11 @@ ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStrea
   p.sk_cnt = nullptr;
   p.sk_min_blocks = 16;
   p.sk_min_gain = 1;
+  p.hdr_in = nullptr;
+  p.bias = nullptr;
+  p.relu = 0;
+  p.act = nullptr;
+  p.ldact = 0;
   const int mt = cdiv(p.B, BM);
   if (!backward) return launch_mode<256, M_LSTM_FWD, 1>(ctx, p, mt * cdiv(p.N, 64), s);
   return launch_mode<256, M_LSTM_BWD_DATA, 1>(ctx, p, mt * cdiv(p.K, 64), s);

@@ -1,0 +1,81 @@
+// One training iteration of a stack of fully connected layers under row patterns, as a sequence of the
+// library's own calls (Sec. 3.2, last paragraph: product -> activation -> dropout per layer; Sec. 3.1: a
+// layer fed by a dropped layer multiplies compact matrices on both sides; Sec. 3.4: a new pattern per
+// iteration).  Host code only: the order of the calls is all that lives here, every step runs in the
+// kernels behind them.  Nothing here synchronises or allocates, so the whole iteration can be captured
+// into a CUDA graph once its descriptor tables exist (run it once before capturing).
+#include "ard_internal.h"
+
+extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, int n_layers, int B, const void* X,
+                                   int ldx, const void* dOut, int lddout, void* dX, int lddx, int dist_id,
+                                   uint64_t seed, uint64_t iteration_base, uint64_t* iteration_counter,
+                                   void* cuda_stream) {
+  if (!ctx || !layers || n_layers < 1 || B < 0 || !X || !dOut) return ARD_ERR_INVALID_ARG;
+  const ard_dtype dt = ARD_BF16;
+  int last_sampled = -1;
+  for (int l = 0; l < n_layers; ++l) {
+    const ard_mlp_layer& y = layers[l];
+    if (!y.pat || !y.W || !y.A || !y.dW || y.K < 1 || y.N < 1) return ARD_ERR_INVALID_ARG;
+    if (l > 0 && layers[l - 1].N != y.K) return ARD_ERR_SHAPE;
+    if (l > 0 && layers[l - 1].compact_out && (!y.Wk || !y.dWk)) return ARD_ERR_INVALID_ARG;
+    if (l + 1 < n_layers && !y.dZ) return ARD_ERR_INVALID_ARG;
+    if (y.sample) last_sampled = l;
+  }
+  if (layers[n_layers - 1].compact_out) return ARD_ERR_INVALID_ARG;  // dOut is full width
+  if (last_sampled >= 0 && !iteration_counter) return ARD_ERR_INVALID_ARG;
+  ard_status st;
+  // ---- patterns of this iteration (stream id = layer index + 1) ----
+  for (int l = 0; l < n_layers; ++l) {
+    if (!layers[l].sample) continue;
+    st = ard_sample_pattern_counter(ctx, layers[l].pat, dist_id, seed, iteration_base, iteration_counter,
+                                    l == last_sampled, (uint32_t)(l + 1), cuda_stream);
+    if (st != ARD_OK) return st;
+  }
+  // ---- forward ----
+  for (int l = 0; l < n_layers; ++l) {
+    const ard_mlp_layer& y = layers[l];
+    const ard_pattern* in = (l > 0 && layers[l - 1].compact_out) ? layers[l - 1].pat : nullptr;
+    const void* in_act = l == 0 ? X : layers[l - 1].A;
+    const int ld_in = l == 0 ? ldx : layers[l - 1].N;
+    if (in) {
+      st = ard_compact_weight_cols(ctx, y.pat, in, dt, y.K, y.N, y.W, y.ldw, y.Wk, y.ldw, cuda_stream);
+      if (st != ARD_OK) return st;
+    }
+    const int mode = (y.compact_out ? ARD_OUT_COMPACT : ARD_OUT_SCATTER_ZEROFILL) | (y.relu ? ARD_FLAG_RELU : 0);
+    st = ard_layer_fwd(ctx, y.pat, in, dt, B, y.K, y.N, y.alpha, in_act, ld_in, in ? y.Wk : y.W, y.ldw, y.bias, y.A, y.N,
+                       mode, cuda_stream);
+    if (st != ARD_OK) return st;
+  }
+  // ---- backward ----
+  for (int l = n_layers - 1; l >= 0; --l) {
+    const ard_mlp_layer& y = layers[l];
+    const ard_pattern* in = (l > 0 && layers[l - 1].compact_out) ? layers[l - 1].pat : nullptr;
+    const void* in_act = l == 0 ? X : layers[l - 1].A;
+    const int ld_in = l == 0 ? ldx : layers[l - 1].N;
+    const void* dZ = l == n_layers - 1 ? dOut : y.dZ;
+    const int lddz = l == n_layers - 1 ? lddout : y.N;
+    const int dz_compact = (l == n_layers - 1) ? 0 : (y.compact_out ? 1 : 0);
+    const ard_dtype dwt = y.dW_is_f32 ? ARD_F32 : ARD_BF16;
+    st = ard_layer_bwd_weight(ctx, y.pat, in, dt, dwt, B, y.K, y.N, 1.0f, in_act, ld_in, dZ, lddz, dz_compact,
+                              in ? y.dWk : y.dW, y.ldw, 1, cuda_stream);
+    if (st != ARD_OK) return st;
+    if (in) {
+      st = ard_expand_weight_grad_cols(ctx, y.pat, in, dwt, y.K, y.N, y.dWk, y.ldw, y.dW, y.ldw, 1, cuda_stream);
+      if (st != ARD_OK) return st;
+    }
+    if (y.db) {
+      st = ard_bias_grad(ctx, y.pat, dt, B, y.N, dZ, lddz, dz_compact, y.db, 1, cuda_stream);
+      if (st != ARD_OK) return st;
+    }
+    if (l > 0) {
+      const ard_mlp_layer& prev = layers[l - 1];
+      st = ard_layer_bwd_data(ctx, y.pat, in, dt, B, y.K, y.N, prev.alpha, dZ, lddz, dz_compact, in ? y.Wk : y.W, y.ldw,
+                              prev.relu ? prev.A : nullptr, prev.N, prev.dZ, prev.N, cuda_stream);
+      if (st != ARD_OK) return st;
+    } else if (dX) {
+      st = ard_bwd_data(ctx, y.pat, dt, B, y.K, y.N, 1.0f, dZ, lddz, dz_compact, y.W, y.ldw, dX, lddx, cuda_stream);
+      if (st != ARD_OK) return st;
+    }
+  }
+  return ARD_OK;
+}

@@ -38,7 +38,7 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
                   int32_t* __restrict__ col_idx, int32_t* __restrict__ row_ptr, int32_t* __restrict__ row_idx,
                   const unsigned long long* __restrict__ cdf, int ndp, unsigned long long seed,
                   unsigned long long iteration, uint32_t stream_id, int forced_dp, int forced_b, int kind,
-                  int units, int Tr, int Tc, int ts) {
+                  int units, int Tr, int Tc, int ts, unsigned long long* __restrict__ counter, int advance) {
   __shared__ int s_dp, s_b;
   __shared__ unsigned long long s_cdf[64];
   pdl_launch_dependents();
@@ -54,6 +54,12 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
       dp = forced_dp;
       b = forced_b;
     } else {
+      // A device-resident counter lets a captured graph draw a fresh pattern at every replay.
+      if (counter != nullptr) {
+        const unsigned long long n = *counter;
+        iteration += n;
+        if (advance) *counter = n + 1ull;
+      }
       uint32_t c[4] = {(uint32_t)iteration, (uint32_t)(iteration >> 32), stream_id, 0u};
       philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
       // dp = smallest i with r0 < c_i; the table is non-decreasing and ends at 2^32.
@@ -142,11 +148,12 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
 }  // namespace
 
 ard_status launch_sampler(ard_ctx* ctx, ard_pattern* pat, const unsigned long long* d_cdf, int ndp, uint64_t seed,
-                          uint64_t iteration, uint32_t stream_id, int forced_dp, int forced_b, cudaStream_t s) {
+                          uint64_t iteration, uint32_t stream_id, int forced_dp, int forced_b, cudaStream_t s,
+                          unsigned long long* d_counter, int advance) {
   ARD_CUDA_OK(ard_launch(ctx, ard_sample_kernel, dim3(1), dim3(SAMPLER_THREADS), 0, s, pat->d_hdr, pat->d_idx,
                          pat->d_col_ptr, pat->d_col_idx, pat->d_row_ptr, pat->d_row_idx, d_cdf, ndp,
                          (unsigned long long)seed, (unsigned long long)iteration, stream_id, forced_dp, forced_b,
-                         (int)pat->kind, pat->units, pat->Tr, pat->Tc, pat->ts));
+                         (int)pat->kind, pat->units, pat->Tr, pat->Tc, pat->ts, d_counter, advance));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;
