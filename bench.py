@@ -41,6 +41,11 @@ WORKLOADS = {
     "mlp8192_tile": dict(config=5, B=4096, K=8192, N=8192, kind="tile", ts=128, p=0.5, n_dp=16),
     "mlp4096_tile": dict(config=3, B=1024, K=4096, N=4096, kind="tile", ts=64, p=0.5, n_dp=16),
     "mlp2048_row": dict(config=2, B=128, K=2048, N=2048, kind="row", ts=0, p=0.5, n_dp=16),
+    # whole training iteration of a stack of layers through ard_mlp_step (fused layer steps, compact matrices
+    # between the hidden layers, one CUDA graph per iteration): the 784-2048-2048-10 network of config 2 and a
+    # stack of large layers where the second hidden layer multiplies two compact matrices
+    "mlp2048_step": dict(config=2, dims=[784, 2048, 2048, 10], B=128, kind="mlp_step", p=0.5, n_dp=16),
+    "mlp8192_step": dict(config=5, dims=[8192, 8192, 8192, 1024], B=4096, kind="mlp_step", p=0.5, n_dp=16),
     # LSTM layer (config 4): a step is one sequence, forward + BPTT, one fresh pattern per sequence
     "lstm1024": dict(config=4, T=35, B=64, I=1024, H=1024, kind="lstm", p=0.5, n_dp=16),
 }
@@ -180,6 +185,10 @@ def run_reference(args, wl):
     """--impl reference: the CPU oracle on the host cores, bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
+        return
+    if wl["kind"] not in ("row", "tile"):
+        print(json.dumps({"impl": "reference", "unavailable": "the reference arm covers the single-layer workloads; "
+                          "for this one the oracle is timed in the cpu_baseline field of the ordinary run"}))
         return
     d = inputs.dense_layer(wl["config"], wl["B"], wl["K"], wl["N"], 1.0 / 90.0)
     rows = 64
@@ -340,6 +349,212 @@ def run_lstm(args, wl):
     ard.ard_destroy(ctx)
 
 
+def run_mlp_step(args, wl):
+    """A step is one training iteration of the whole stack: patterns drawn on the device, forward chain,
+    backward chain (weight, bias and input gradients), as ONE native call replayed from a CUDA graph."""
+    import torch
+    from paper_2203_05705_b200 import ard
+    dev_index = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(dev_index)
+    clocks = ClockSampler(dev_index)
+    dims, B, p, n_dp = wl["dims"], wl["B"], wl["p"], wl["n_dp"]
+    L = len(dims) - 1
+    bf = torch.bfloat16
+    alpha = 1.0 / (1.0 - p)
+    ctx = ard.ard_create(0, 2 * B * max(dims) + 4096)
+    ard.ard_set_compact_reuse(ctx, 1)
+    Kd = inputs.max_entropy_K(p, n_dp)
+    ard.ard_set_distribution(ctx, 0, Kd)
+    g = torch.Generator(device="cuda").manual_seed(inputs.BASE_SEED)
+    hX = torch.rand((B, dims[0]), generator=torch.Generator().manual_seed(1)).to(bf).pin_memory()
+    hdO = (torch.randn((B, dims[-1]), generator=torch.Generator().manual_seed(2)) / B).to(bf).pin_memory()
+    hOut = torch.empty((B, dims[-1]), dtype=bf).pin_memory()
+    X, dOut = hX.cuda(), hdO.cuda()
+
+    def make_stack(compact):
+        layers, keep = [], []
+        for l in range(L):
+            K, N = dims[l], dims[l + 1]
+            hidden = l < L - 1
+            d = dict(K=K, N=N, pat=ard.ard_pattern_create(ctx, ard.ARD_ROW, K, N, 0), sample=1 if hidden else 0,
+                     relu=1 if hidden else 0, compact_out=1 if (hidden and compact) else 0, dW_is_f32=0,
+                     alpha=alpha if hidden else 1.0, ldw=K,
+                     W=(torch.randn((N, K), device="cuda", generator=g) * (2.0 / K) ** 0.5).to(bf),
+                     bias=torch.zeros(N, device="cuda"), Wk=torch.zeros((N, K), dtype=bf, device="cuda"),
+                     A=torch.zeros((B, N), dtype=bf, device="cuda"), dZ=torch.zeros((B, N), dtype=bf, device="cuda"),
+                     dWk=torch.zeros((N, K), dtype=bf, device="cuda"), dW=torch.zeros((N, K), dtype=bf, device="cuda"),
+                     db=torch.zeros(N, device="cuda"))
+            layers.append(d)
+        ard.ard_pattern_set(ctx, layers[-1]["pat"], 1, 1)
+        return layers, ard.mlp_layers(layers)
+
+    counter = torch.zeros(1, dtype=torch.int64, device="cuda")
+    dX = torch.zeros((B, dims[0]), dtype=bf, device="cuda")
+    base = 7000
+
+    def eager(stack, sample=True):
+        ard.ard_mlp_step(ctx, stack[1], L, B, X, dims[0], dOut, dims[-1], dX, dims[0], 0, inputs.BASE_SEED, base, counter)
+
+    def graphed(stack):
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            eager(stack)                     # descriptor tables are built outside the capture
+        torch.cuda.synchronize()
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            eager(stack)
+        return gr
+
+    def timed(fn, n, warm):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1), t0, time.time()
+
+    compact = make_stack(1)
+    gr = graphed(compact)
+    steps, warm = args.steps, max(3, args.warmup)
+    # headline: graph replays of the compact chain; the realised patterns are read back afterwards by
+    # replaying the same iterations one call at a time
+    counter.zero_()
+    l0 = ard.ard_launch_count(ctx)
+    eager(compact)
+    torch.cuda.synchronize()
+    launches_per_step = int(ard.ard_launch_count(ctx) - l0)
+    counter.zero_()
+    ms, t0, t1 = timed(gr.replay, steps, warm)
+    clk = clocks.stop(t0, t1)
+    status = ard.ard_last_device_status(ctx)
+    # kept FLOPs of the timed iterations (iteration = base + warm + i; stream id = layer + 1)
+    def kept_flops(it):
+        n = [dims[0]]
+        for l in range(L - 1):
+            ard.ard_sample_pattern(ctx, compact[0][l]["pat"], 0, inputs.BASE_SEED, it, l + 1)
+            n.append(ard.ard_pattern_to_host(compact[0][l]["pat"], 0)[2])
+        n.append(dims[-1])
+        fl = 0.0
+        for l in range(L):
+            fl += 2.0 * B * n[l] * n[l + 1] * 3            # forward, weight gradient, input gradient
+        return fl, n
+    kept = 0.0
+    fracs = []
+    for i in range(steps):
+        f, n = kept_flops(base + warm + i)
+        kept += f
+        fracs.append([n[l + 1] / dims[l + 1] for l in range(L - 1)])
+    dense_flops = sum(2.0 * B * dims[l] * dims[l + 1] * 3 for l in range(L))
+    value = kept / (ms * 1e-3) / 1e12
+    detail = {"ms_per_step": {"graph_compact": ms / steps}}
+    if not args.quick:
+        n2 = max(5, steps // 4)
+        detail["ms_per_step"]["eager_compact"] = timed(lambda: eager(compact), n2, warm)[0] / n2
+        fullw = make_stack(0)
+        gr_f = graphed(fullw)
+        detail["ms_per_step"]["graph_full_width"] = timed(gr_f.replay, n2, warm)[0] / n2
+        detail["ms_per_step"]["eager_full_width"] = timed(lambda: eager(fullw), n2, warm)[0] / n2
+        # the same iteration at dp = 1 everywhere (nothing dropped), own kernels
+        for d in compact[0][:-1]:
+            d["sample"] = 0
+            ard.ard_pattern_set(ctx, d["pat"], 1, 1)
+        dense_stack = (compact[0], ard.mlp_layers(compact[0]))
+        gr_d = graphed(dense_stack)
+        detail["ms_per_step"]["graph_own_kernels_dp1"] = timed(gr_d.replay, n2, warm)[0] / n2
+        # library baseline: the same network with conventional dropout in torch (bf16 autograd), eager and graphed
+        Wt = [d["W"].clone().requires_grad_(True) for d in compact[0]]
+        bt = [d["bias"].to(bf).clone().requires_grad_(True) for d in compact[0]]
+        Xt = X.clone().requires_grad_(True)
+
+        def torch_step():
+            for t in Wt + bt + [Xt]:
+                t.grad = None
+            a = Xt
+            for l in range(L):
+                a = torch.nn.functional.linear(a, Wt[l], bt[l])
+                if l < L - 1:
+                    a = torch.nn.functional.dropout(torch.relu(a), p, True)
+            a.backward(dOut)
+
+        detail["ms_per_step"]["torch_eager_dropout"] = timed(torch_step, n2, warm)[0] / n2
+        try:
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                for _ in range(3):
+                    torch_step()
+            torch.cuda.synchronize()
+            gt = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gt):
+                torch_step()
+            detail["ms_per_step"]["torch_graph_dropout"] = timed(gt.replay, n2, warm)[0] / n2
+        except Exception as ex:
+            sys.stderr.write("torch graph baseline skipped: %r\n" % (ex,))
+        best_dense = min(v for k, v in detail["ms_per_step"].items() if k.startswith("torch") or k.endswith("dp1"))
+        detail["speedup_vs_dense"] = {str(p): best_dense / (ms / steps)}
+        # end to end: the input batch and the loss gradient come from pinned host memory and the network's
+        # output goes back every iteration
+        for d in compact[0][:-1]:
+            d["sample"] = 1
+        compact = (compact[0], ard.mlp_layers(compact[0]))
+
+        def e2e_step():
+            X.copy_(hX, non_blocking=True)
+            dOut.copy_(hdO, non_blocking=True)
+            eager(compact)
+            hOut.copy_(compact[0][-1]["A"], non_blocking=True)
+
+        counter.zero_()
+        ms_e = timed(e2e_step, n2, warm)[0] / n2
+        kept_e = sum(kept_flops(base + warm + i)[0] for i in range(n2))
+        e2e = {"value": kept_e / n2 / (ms_e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": hX.numel() * 2 + hdO.numel() * 2,
+               "d2h_bytes_per_step": hOut.numel() * 2, "ms_per_step": ms_e}
+    else:
+        e2e = None
+    peaks = load_peaks()
+    cpu = None
+    if not args.no_cpu_baseline and not args.quick:
+        from oracle import mlp as OM
+        from oracle import pattern as OP
+        rows = min(B, 256)
+        Ws = [d["W"].float().cpu().numpy().T.astype(np.float64) for d in compact[0]]
+        masks = [OP.row_mask(dims[l + 1], 2, 1) for l in range(L - 1)] + [np.ones(dims[-1])]
+        Xh = hX[:rows].float().numpy()
+        tc0 = time.perf_counter()
+        fw = OM.fwd(Xh, Ws, None, masks, [alpha] * (L - 1) + [1.0])
+        OM.bwd(fw, Ws, masks, [alpha] * (L - 1) + [1.0], hdO[:rows].float().numpy())
+        dt = time.perf_counter() - tc0
+        try:
+            from threadpoolctl import threadpool_info
+            threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        except Exception:
+            threads = os.cpu_count() or 1
+        n = [dims[0]] + [dims[l + 1] // 2 for l in range(L - 1)] + [dims[-1]]
+        cpu = {"value": sum(2.0 * rows * n[l] * n[l + 1] * 3 for l in range(L)) / dt / 1e12, "unit": UNIT, "cores": threads,
+               "kind": "oracle", "sample": "%d batch rows of one iteration, dp=2 on every hidden layer" % rows, "seconds": dt}
+    line = {
+        "metric": "MLP training iteration kept TFLOP/s (row patterns on the hidden layers, p=%s)" % p, "value": value,
+        "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "dims": dims, "B": B, "p": p, "n_dp": n_dp,
+                   "l2": "a fresh pattern every iteration; working set %.0f MB" % (sum(dims[l] * dims[l + 1] for l in range(L)) * 2 / 1e6)},
+        "dense_equiv_tflops": dense_flops * steps / (ms * 1e-3) / 1e12, "clocks": clk, "e2e": e2e,
+        "gpu_launches": launches_per_step * steps,
+        "roofline": {"bound": "tensor", "achieved": value, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": value / peaks["bf16_tflops"], "traffic": None,
+                     "note": "whole iteration incl. sampler, weight compaction, gradient expansion and bias gradients"},
+        "cpu_baseline": cpu,
+        "detail": dict(detail, kept_fraction_per_hidden_layer=[float(np.mean([f[l] for f in fracs])) for l in range(L - 1)],
+                       launches_per_step=launches_per_step),
+        "device_status": int(status),
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -355,6 +570,8 @@ def main():
         return run_reference(args, wl)
     if wl["kind"] == "lstm":
         return run_lstm(args, wl)
+    if wl["kind"] == "mlp_step":
+        return run_mlp_step(args, wl)
 
     import torch
     import torch.distributed as dist

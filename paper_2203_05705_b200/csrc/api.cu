@@ -202,6 +202,8 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->d_grid_bar = nullptr;
   ctx->d_lstm_partial = nullptr;
   if (const char* e = getenv("ARD_PDL")) ctx->use_pdl = atoi(e) ? 1 : 0;
+  ctx->pdl_in_capture = 0;
+  if (const char* e = getenv("ARD_PDL_CAPTURE")) ctx->pdl_in_capture = atoi(e) ? 1 : 0;
   ctx->sk_min_blocks = 16;
   if (const char* e = getenv("ARD_STREAM_K")) ctx->stream_k = atoi(e);
   ctx->sk_min_gain = 24;
@@ -509,7 +511,7 @@ static ard_status fwd_impl(ard_ctx* ctx, const ard_pattern* pat, const ard_patte
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int es = out_f32 ? 4 : 2;
 
-  GemmArgs g;
+  GemmArgs g = {};
   fill_common(g, ctx, pat, B, K, N, alpha);
   g.A0 = X; g.lda0 = ldx; g.A1 = W; g.lda1 = ldw; g.out = Y; g.ldo = ldy;
   g.flag0 = pat->kind == ARD_ROW ? mode : 0;
@@ -529,7 +531,7 @@ static ard_status fwd_impl(ard_ctx* ctx, const ard_pattern* pat, const ard_patte
     if (ctx->path == ARD_PATH_TENSOR_CORE) return el;
     return launch_gemm_cc(ctx, pat->kind, OP_FWD, dtype, g, pat->ts, s);
   }
-  TcArgs t;
+  TcArgs t = {};
   t.g = g;
   t.ts = pat->ts;
   t.bn = tc_pick_bn(ctx, pat->kind, OP_FWD, pat->dp_bound, pat->ts);
@@ -621,7 +623,7 @@ static ard_status bwd_data_impl(ard_ctx* ctx, const ard_pattern* pat, const ard_
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int es = out_f32 ? 4 : 2;
 
-  GemmArgs g;
+  GemmArgs g = {};
   fill_common(g, ctx, pat, B, K, N, alpha);
   g.A0 = dY; g.lda0 = lddy; g.A1 = W; g.lda1 = ldw; g.out = dX; g.ldo = lddx;
   g.flag0 = dy_is_compact ? 1 : 0;
@@ -644,7 +646,7 @@ static ard_status bwd_data_impl(ard_ctx* ctx, const ard_pattern* pat, const ard_
     if (ctx->path == ARD_PATH_TENSOR_CORE) return el;
     return launch_gemm_cc(ctx, pat->kind, OP_BWD_DATA, dtype, g, pat->ts, s);
   }
-  TcArgs t;
+  TcArgs t = {};
   t.ts = pat->ts;
   t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_DATA, pat->dp_bound, pat->ts);
   if (pat->kind == ARD_ROW) {
@@ -704,7 +706,7 @@ static ard_status bwd_weight_impl(ard_ctx* ctx, const ard_pattern* pat, const ar
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int es_out = dW_dtype == ARD_F32 ? 4 : 2;
 
-  GemmArgs g;
+  GemmArgs g = {};
   fill_common(g, ctx, pat, B, K, N, alpha);
   g.A0 = dY; g.lda0 = lddy; g.A1 = X; g.lda1 = ldx; g.out = dW; g.ldo = lddw;
   g.flag0 = dy_is_compact ? 1 : 0;
@@ -724,7 +726,7 @@ static ard_status bwd_weight_impl(ard_ctx* ctx, const ard_pattern* pat, const ar
     if (ctx->path == ARD_PATH_TENSOR_CORE) return el;
     return launch_gemm_cc(ctx, pat->kind, OP_BWD_WEIGHT, dtype, g, pat->ts, s);
   }
-  TcArgs t;
+  TcArgs t = {};
   t.ts = pat->ts;
   t.bn = tc_pick_bn(ctx, pat->kind, OP_BWD_WEIGHT, pat->dp_bound, pat->ts);
   if (pat->kind == ARD_ROW) {
@@ -848,8 +850,8 @@ ard_status ard_lstm_gate_gemm(ard_ctx* ctx, const ard_pattern* pat, int B, int K
     }
     return ARD_OK;
   }
-  TcArgs t;
-  GemmArgs g;
+  TcArgs t = {};
+  GemmArgs g = {};
   fill_common(g, ctx, pat, B, KH, H, 1.0f);
   g.A0 = XH; g.lda0 = ldxh; g.A1 = W; g.lda1 = ldw; g.out = Z; g.ldo = 4 * ldz_gate;
   g.out_is_f32 = 1;
@@ -878,8 +880,8 @@ static ard_status lstm_gate_gemm_bwd_tc(ard_ctx* ctx, const ard_pattern* pat, in
                                         cudaStream_t s) {
   const char* Wc = reinterpret_cast<const char*>(Wcols);
   const char* dZc = reinterpret_cast<const char*>(dZ);
-  TcArgs t;
-  GemmArgs g;
+  TcArgs t = {};
+  GemmArgs g = {};
   fill_common(g, ctx, pat, B, kout, H, 1.0f);
   g.A0 = dZ; g.lda0 = 4 * ldz_gate; g.A1 = Wcols; g.lda1 = ldw; g.out = out; g.ldo = ldo;
   g.flag0 = 1;
@@ -985,8 +987,8 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
       const CUtensorMap* mapW[4];
       // 1. The input half for all steps at once: G[t][:, g*H + j] = x_t . W[g*H + keep[j]][0:I]  (T*B rows).
       if (I > 0) {
-        TcArgs t;
-        GemmArgs g;
+        TcArgs t = {};
+        GemmArgs g = {};
         fill_common(g, ctx, pat, T * B, I, H, 1.0f);
         g.A0 = XH; g.lda0 = KH; g.A1 = W; g.lda1 = ldw; g.out = G; g.ldo = 4 * H;
         g.out_is_f32 = 1;

@@ -77,6 +77,7 @@ struct ard_ctx {
   unsigned int* d_grid_bar;  // arrival counter of that kernel's grid-wide barrier
   float* d_lstm_partial;     // partial sums of the whole-sequence BPTT kernel, lstm_bwd_partial_bytes(sm_count)
   int use_pdl;        // launch kernels with programmatic stream serialization (see ard_launch)
+  int pdl_in_capture; // ... also while the stream is being captured into a CUDA graph
   int stream_k;       // tensor-core row kernels: share the last, partial wave of tiles along the contraction
   int sk_min_blocks;  // fewest 64-wide contraction blocks worth a separate share
   int sk_min_gain;    // fewest blocks the sharing must save per worker to be used
@@ -197,6 +198,10 @@ ard_status launch_lstm_gates_bwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype
 // successor start early with pdl_launch_dependents() and (2) calls pdl_wait_prior_grids() before its
 // first access to global memory; that call returns once all earlier kernels of the stream have
 // completed and their writes are visible.  Both are no-ops for a kernel launched the ordinary way.
+// (3) Nothing an earlier kernel of the stream writes (pattern headers and lists, activations, gradients)
+// is read through the read-only data path (const __restrict__ parameters, __ldg): a block can be
+// resident long before its wait returns, and that path is not made coherent by the wait: a block of the
+// kernel that followed the sampler was seen to read the previous iteration's pattern header that way.
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -208,6 +213,7 @@ __device__ __forceinline__ void pdl_wait_prior_grids() { asm volatile("griddepco
 // inside a graph the launch latency that the early start hides is small anyway.
 inline bool ard_pdl_allowed(const ard_ctx* ctx, cudaStream_t s) {
   if (!ctx->use_pdl) return false;
+  if (ctx->pdl_in_capture) return true;
   cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(s, &st) != cudaSuccess) return false;
   return st == cudaStreamCaptureStatusNone;

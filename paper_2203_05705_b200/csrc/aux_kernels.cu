@@ -7,8 +7,8 @@ namespace {
 // dst[r][j] = src[r][keep[j]], j < n_keep.  The kept columns of a row pattern (Sec. 3.1) stride the
 // contiguous dimension, which a TMA box cannot do, so the tensor-core backward GEMMs read this copy.
 template <typename T>
-__global__ void __launch_bounds__(256) gather_cols_kernel(const int32_t* __restrict__ hdr, const T* __restrict__ src,
-                                                          int ld_src, T* __restrict__ dst, int ld_dst, int rows) {
+__global__ void __launch_bounds__(256) gather_cols_kernel(const int32_t* hdr, const T* src,
+                                                          int ld_src, T* dst, int ld_dst, int rows) {
   pdl_launch_dependents();
   pdl_wait_prior_grids();
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], b = hdr[HDR_B];
@@ -27,8 +27,8 @@ constexpr int GATHER_WARPS = 4;
 constexpr int GATHER_SPAN = 4096;  // staged source elements per warp (8 KiB)
 
 __global__ void __launch_bounds__(GATHER_WARPS * 32)
-gather_cols_staged_kernel(const int32_t* __restrict__ hdr, const uint16_t* __restrict__ src, int ld_src,
-                          uint16_t* __restrict__ dst, int ld_dst, int rows, int n_cols, int skip_dense) {
+gather_cols_staged_kernel(const int32_t* hdr, const uint16_t* src, int ld_src,
+                          uint16_t* dst, int ld_dst, int rows, int n_cols, int skip_dense) {
   __shared__ __align__(16) uint16_t smem[GATHER_WARPS][GATHER_SPAN + 8];
   pdl_launch_dependents();
   pdl_wait_prior_grids();
@@ -91,10 +91,10 @@ __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + __expf
 
 template <typename HT>
 __global__ void __launch_bounds__(256)
-lstm_gates_kernel(const int32_t* __restrict__ hdr, int B, int H, float alpha, const float* __restrict__ Z,
-                  int ldz, const float* __restrict__ bias, const float* __restrict__ c_prev, int ldc,
-                  float* __restrict__ c, HT* __restrict__ h, int ldh, int h_scatter,
-                  float* __restrict__ gates_saved) {
+lstm_gates_kernel(const int32_t* hdr, int B, int H, float alpha, const float* Z,
+                  int ldz, const float* bias, const float* c_prev, int ldc,
+                  float* c, HT* h, int ldh, int h_scatter,
+                  float* gates_saved) {
   pdl_launch_dependents();
   pdl_wait_prior_grids();
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], b = hdr[HDR_B];
@@ -139,10 +139,10 @@ lstm_gates_kernel(const int32_t* __restrict__ hdr, int B, int H, float alpha, co
 
 template <typename ZT>
 __global__ void __launch_bounds__(256)
-lstm_gates_bwd_kernel(const int32_t* __restrict__ hdr, int B, int H, float alpha,
-                      const float* __restrict__ gates_saved, const float* __restrict__ c_prev,
-                      const float* __restrict__ c, int ldc, const float* __restrict__ dh, int lddh, int dh_scatter,
-                      float* __restrict__ dc_inout, ZT* __restrict__ dZ, int ldz) {
+lstm_gates_bwd_kernel(const int32_t* hdr, int B, int H, float alpha,
+                      const float* gates_saved, const float* c_prev,
+                      const float* c, int ldc, const float* dh, int lddh, int dh_scatter,
+                      float* dc_inout, ZT* dZ, int ldz) {
   pdl_launch_dependents();
   pdl_wait_prior_grids();
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], b = hdr[HDR_B];
@@ -173,9 +173,9 @@ lstm_gates_bwd_kernel(const int32_t* __restrict__ hdr, int B, int H, float alpha
 // next multiple of 64 (or ldwk) are written as zero, so that the last 64-wide contraction block of the
 // tensor-core forward product multiplies zeros.  Eight outputs per thread (one 16- or 32-byte store).
 template <typename T>
-__global__ void __launch_bounds__(256) compact_weight_cols_kernel(const int32_t* __restrict__ hdr,
-                                                                  const int32_t* __restrict__ hdr_in,
-                                                                  const T* __restrict__ W, int ldw, T* __restrict__ Wk,
+__global__ void __launch_bounds__(256) compact_weight_cols_kernel(const int32_t* hdr,
+                                                                  const int32_t* hdr_in,
+                                                                  const T* W, int ldw, T* Wk,
                                                                   int ldwk, int vec_ok) {
   pdl_launch_dependents();
   pdl_wait_prior_grids();
@@ -212,10 +212,10 @@ __global__ void __launch_bounds__(256) compact_weight_cols_kernel(const int32_t*
 // every other entry of dW [N][K] (dropped neurons, dropped inputs) is written as zero, without it they
 // are left alone.  One output row per blockIdx.y step, consecutive threads write consecutive columns.
 template <typename T>
-__global__ void __launch_bounds__(256) expand_weight_grad_cols_kernel(const int32_t* __restrict__ hdr,
-                                                                      const int32_t* __restrict__ hdr_in,
-                                                                      const T* __restrict__ dWk, int lddwk,
-                                                                      T* __restrict__ dW, int lddw, int N, int K,
+__global__ void __launch_bounds__(256) expand_weight_grad_cols_kernel(const int32_t* hdr,
+                                                                      const int32_t* hdr_in,
+                                                                      const T* dWk, int lddwk,
+                                                                      T* dW, int lddw, int N, int K,
                                                                       int zero_fill) {
   pdl_launch_dependents();
   pdl_wait_prior_grids();
@@ -238,9 +238,9 @@ __global__ void __launch_bounds__(256) expand_weight_grad_cols_kernel(const int3
 // a dropped neuron takes no part in the iteration); dropped entries are zeroed on request.
 // A block owns 32 consecutive neurons; its 8 row groups add their rows in a fixed order.
 template <typename T>
-__global__ void __launch_bounds__(256) bias_grad_kernel(const int32_t* __restrict__ hdr, const T* __restrict__ dZ,
+__global__ void __launch_bounds__(256) bias_grad_kernel(const int32_t* hdr, const T* dZ,
                                                         int lddz, int dz_is_compact, int B, int N,
-                                                        float* __restrict__ db, int zero_fill) {
+                                                        float* db, int zero_fill) {
   __shared__ float part[8][33];
   pdl_launch_dependents();
   pdl_wait_prior_grids();

@@ -35,8 +35,11 @@ __global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts)
   pdl_wait_prior_grids();
   const int dp = g.hdr[HDR_DP], b = g.hdr[HDR_B], n_keep = g.hdr[HDR_NKEEP];
   const int Tc = g.hdr[HDR_TC];
-  const T* __restrict__ P0 = reinterpret_cast<const T*>(g.A0);
-  const T* __restrict__ P1 = reinterpret_cast<const T*>(g.A1);
+  // No __restrict__ / read-only loads on anything an earlier kernel of the stream wrote: this kernel may
+  // become resident before that kernel has finished (see pdl_wait_prior_grids), and the non-coherent
+  // load path may then serve a line another resident kernel brought in before the data was rewritten.
+  const T* P0 = reinterpret_cast<const T*>(g.A0);
+  const T* P1 = reinterpret_cast<const T*>(g.A1);
 
   int M, N, nk;
   const int m0 = blockIdx.y * T_M, n0 = blockIdx.x * T_N;

@@ -804,7 +804,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
           if (na >= 32) {
 #pragma unroll
             for (int q8 = 0; q8 < 4; ++q8) {
-              const uint4 a = __ldg(reinterpret_cast<const uint4*>(arow) + q8);
+              const uint4 a = reinterpret_cast<const uint4*>(arow)[q8];
               const uint32_t w[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
               for (int h = 0; h < 8; ++h) {

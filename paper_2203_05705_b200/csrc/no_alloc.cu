@@ -29,8 +29,8 @@ void* g_scratch_addr[MAX_DEVICES] = {};  // device address of g_static_scratch, 
 // written densely.  `dst` is the static scratch array.
 template <typename T>
 __global__ void __launch_bounds__(256)
-gather_into_static_scratch_kernel(const int32_t* __restrict__ hdr, const T* __restrict__ src, int ld_src,
-                                  T* __restrict__ dst, int ld_dst, int rows) {
+gather_into_static_scratch_kernel(const int32_t* hdr, const T* src, int ld_src,
+                                  T* dst, int ld_dst, int rows) {
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
   for (long long e = (long long)blockIdx.x * 256 + threadIdx.x; e < (long long)rows * n_keep;
        e += (long long)gridDim.x * 256) {
@@ -83,7 +83,7 @@ extern "C" ard_status ard_bwd_data_static_scratch(ard_ctx* ctx, const ard_patter
     ctx->launches++;
     if (cudaGetLastError() != cudaSuccess) st = ARD_ERR_CUDA;
     if (st == ARD_OK) {
-      GemmArgs g;
+      GemmArgs g = {};
       g.hdr = pat->d_hdr;
       g.idx = pat->d_idx;
       g.col_ptr = g.col_idx = g.row_ptr = g.row_idx = nullptr;
