@@ -202,7 +202,7 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->d_grid_bar = nullptr;
   ctx->d_lstm_partial = nullptr;
   if (const char* e = getenv("ARD_PDL")) ctx->use_pdl = atoi(e) ? 1 : 0;
-  ctx->pdl_in_capture = 0;
+  ctx->pdl_in_capture = 1;
   if (const char* e = getenv("ARD_PDL_CAPTURE")) ctx->pdl_in_capture = atoi(e) ? 1 : 0;
   ctx->sk_min_blocks = 16;
   if (const char* e = getenv("ARD_STREAM_K")) ctx->stream_k = atoi(e);

@@ -207,10 +207,8 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 
-// While a stream is being captured into a CUDA graph the kernels are launched the ordinary way: replays
-// of a graph whose nodes were joined by programmatic edges were seen to read the pattern header of the
-// previous replay in some blocks of the kernel that follows the sampler (never seen in stream order), and
-// inside a graph the launch latency that the early start hides is small anyway.
+// The attribute is also kept while a stream is being captured into a CUDA graph (the nodes are then joined
+// by programmatic edges); ARD_PDL_CAPTURE=0 launches the ordinary way during a capture.
 inline bool ard_pdl_allowed(const ard_ctx* ctx, cudaStream_t s) {
   if (!ctx->use_pdl) return false;
   if (ctx->pdl_in_capture) return true;

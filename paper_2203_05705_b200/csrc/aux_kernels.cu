@@ -264,6 +264,129 @@ __global__ void __launch_bounds__(256) bias_grad_kernel(const int32_t* hdr, cons
   }
 }
 
+// Wide form of the expansion for 16-byte aligned rows: a thread assembles 8 consecutive output columns
+// (one 16-byte store for bf16, two for fp32) from the at most 8 compact entries that fall into them.
+template <typename T>
+__global__ void __launch_bounds__(256) expand_weight_grad_cols_wide_kernel(const int32_t* hdr, const int32_t* hdr_in,
+                                                                           const T* dWk, int lddwk, T* dW, int lddw,
+                                                                           int N, int K, int zero_fill) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
+  const int dpi = hdr_in[HDR_DP], bi = hdr_in[HDR_B] - 1;
+  const int groups = K / 8;  // the caller guarantees K % 8 == 0
+  for (int n = blockIdx.y; n < N; n += gridDim.y) {
+    const bool kept_row = n >= bb && (n - bb) % dp == 0;
+    if (!kept_row && !zero_fill) continue;
+    const T* src = dWk + (size_t)n * lddwk;
+    T* dst = dW + (size_t)n * lddw;
+    for (int g = blockIdx.x * 256 + threadIdx.x; g < groups; g += gridDim.x * 256) {
+      const int k0 = g * 8;
+      __align__(16) T v[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) v[q] = T(0.f);
+      bool any = false;
+      if (kept_row) {
+        // first kept input at or after k0, then every dpi-th
+        int k = k0 <= bi ? bi : bi + ((k0 - bi + dpi - 1) / dpi) * dpi;
+        int j = (k - bi) / dpi;
+        for (; k < k0 + 8; k += dpi, ++j) {
+          const T x = src[j];
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            if (q == k - k0) v[q] = x;
+          any = true;
+        }
+      }
+      if (!any && !zero_fill) continue;
+      if (!zero_fill) {
+        // only the kept entries may be touched
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          if (k0 + q >= bi && (k0 + q - bi) % dpi == 0) dst[k0 + q] = v[q];
+      } else if (sizeof(T) == 2) {
+        *reinterpret_cast<uint4*>(dst + k0) = *reinterpret_cast<const uint4*>(v);
+      } else {
+        reinterpret_cast<uint4*>(dst + k0)[0] = reinterpret_cast<const uint4*>(v)[0];
+        reinterpret_cast<uint4*>(dst + k0)[1] = reinterpret_cast<const uint4*>(v)[1];
+      }
+    }
+  }
+}
+
+// Wide form of the bias gradient for compact 16-byte aligned bf16 dZ and many rows: the batch is cut into
+// gridDim.y slices; a block adds its slice of 256 compact columns (a lane owns 8 columns of a row, a warp
+// every eighth row of the slice), parks the 256 sums in scratch and the block that arrives last for its
+// columns adds the slices in slice order, so the result does not depend on the arrival order.
+constexpr int BIAS_WIDE_COLS = 256;
+
+__global__ void __launch_bounds__(256) bias_grad_wide_kernel(const int32_t* hdr, const __nv_bfloat16* dZ, int lddz,
+                                                             int compact, int B, int N, float* db, int zero_fill,
+                                                             float* partial, int* counters) {
+  __shared__ float red[8][BIAS_WIDE_COLS + 8];
+  __shared__ int s_last;
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
+  const int n_keep = compact ? hdr[HDR_NKEEP] : N;  // columns of dZ that are added (full width: all of them)
+  const int c0 = blockIdx.x * BIAS_WIDE_COLS;
+  if (c0 >= n_keep) return;
+  const int S = gridDim.y, y = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (compact && zero_fill && y == 0) {
+    // dropped neurons between this block's first kept neuron and the next block's (the last block: to N)
+    const int lo = c0 == 0 ? 0 : bb + c0 * dp;
+    const int hi = (c0 + BIAS_WIDE_COLS >= n_keep) ? N : bb + (c0 + BIAS_WIDE_COLS) * dp;
+    for (int o = lo + threadIdx.x; o < hi; o += 256)
+      if (!(o >= bb && (o - bb) % dp == 0)) db[o] = 0.f;
+  }
+  const int rows_per = (B + S - 1) / S;
+  const int r0 = y * rows_per, r1 = min(B, r0 + rows_per);
+  const int c = c0 + lane * 8;
+  float acc[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+  if (c < n_keep) {
+    for (int r = r0 + warp; r < r1; r += 8) {
+      const uint4 x = *reinterpret_cast<const uint4*>(dZ + (size_t)r * lddz + c);
+      const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        acc[2 * q] += __uint_as_float(w[q] << 16);
+        acc[2 * q + 1] += __uint_as_float(w[q] & 0xFFFF0000u);
+      }
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < 8; ++q) red[warp][lane * 8 + q] = acc[q];
+  __syncthreads();
+  const int col = threadIdx.x;  // one compact column per thread from here on
+  float sum = 0.f;
+#pragma unroll
+  for (int w8 = 0; w8 < 8; ++w8) sum += red[w8][col];
+  const int n_cols_total = gridDim.x * BIAS_WIDE_COLS;
+  __stcg(partial + (size_t)y * n_cols_total + c0 + col, sum);
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = (atomicAdd(counters + blockIdx.x, 1) == S - 1) ? 1 : 0;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  if (threadIdx.x == 0) counters[blockIdx.x] = 0;  // armed again for the next launch
+  if (c0 + col < n_keep) {
+    float total = 0.f;
+    for (int yy = 0; yy < S; ++yy) total += __ldcg(partial + (size_t)yy * n_cols_total + c0 + col);
+    if (compact) {
+      db[bb + (c0 + col) * dp] = total;
+    } else {
+      // full width: the sums of dropped columns (whose entries are never values) are discarded
+      const int o = c0 + col;
+      if (o >= bb && (o - bb) % dp == 0) db[o] = total;
+      else if (zero_fill) db[o] = 0.f;
+    }
+  }
+}
+
 }  // namespace
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,
@@ -344,6 +467,19 @@ ard_status launch_expand_weight_grad_cols(ard_ctx* ctx, const int32_t* hdr, cons
                                           int lddwk, void* dW, int lddw, int N, int K, int elem_bytes, int zero_fill,
                                           cudaStream_t s) {
   if (N == 0 || K == 0) return ARD_OK;
+  const bool wide = K % 8 == 0 && lddw % 8 == 0 && (reinterpret_cast<uintptr_t>(dW) & 15) == 0;
+  if (wide) {
+    dim3 gridw((K / 8 + 255) / 256, N < 65535 ? N : 65535);
+    if (elem_bytes == 2)
+      ARD_CUDA_OK(ard_launch(ctx, expand_weight_grad_cols_wide_kernel<__nv_bfloat16>, gridw, dim3(256), 0, s, hdr, hdr_in,
+                             (const __nv_bfloat16*)dWk, lddwk, (__nv_bfloat16*)dW, lddw, N, K, zero_fill));
+    else
+      ARD_CUDA_OK(ard_launch(ctx, expand_weight_grad_cols_wide_kernel<float>, gridw, dim3(256), 0, s, hdr, hdr_in,
+                             (const float*)dWk, lddwk, (float*)dW, lddw, N, K, zero_fill));
+    ctx->launches++;
+    ARD_CUDA_OK(cudaGetLastError());
+    return ARD_OK;
+  }
   dim3 grid((K + 1023) / 1024, N < 65535 ? N : 65535);
   if (elem_bytes == 2)
     ARD_CUDA_OK(ard_launch(ctx, expand_weight_grad_cols_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, hdr, hdr_in,
@@ -359,6 +495,21 @@ ard_status launch_expand_weight_grad_cols(ard_ctx* ctx, const int32_t* hdr, cons
 ard_status launch_bias_grad(ard_ctx* ctx, const int32_t* hdr, const void* dZ, int lddz, int dz_is_compact,
                             int is_bf16, int B, int N, float* db, int zero_fill, cudaStream_t s) {
   if (N == 0) return ARD_OK;
+  // many rows of compact, aligned bf16: the batch is cut into slices that are added in a fixed order
+  const int xblocks = (N + BIAS_WIDE_COLS - 1) / BIAS_WIDE_COLS;
+  int slices = B / 64;
+  if (slices > 32) slices = 32;
+  if (is_bf16 && N % 8 == 0 && slices >= 2 && lddz % 8 == 0 && (reinterpret_cast<uintptr_t>(dZ) & 15) == 0 &&
+      ctx->d_sk_ws != nullptr && (size_t)slices * xblocks * BIAS_WIDE_COLS * sizeof(float) <= sk_ws_bytes(ctx->sm_count) &&
+      (size_t)xblocks * sizeof(int) <= sk_cnt_bytes(ctx->sm_count)) {
+    ARD_CUDA_OK(ard_launch(ctx, bias_grad_wide_kernel, dim3(xblocks, slices), dim3(256), 0, s, hdr,
+                           (const __nv_bfloat16*)dZ, lddz, dz_is_compact, B, N, db, zero_fill,
+                           reinterpret_cast<float*>(ctx->d_sk_ws),
+                           ctx->d_sk_cnt));
+    ctx->launches++;
+    ARD_CUDA_OK(cudaGetLastError());
+    return ARD_OK;
+  }
   dim3 grid((N + 31) / 32);
   if (is_bf16)
     ARD_CUDA_OK(ard_launch(ctx, bias_grad_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, hdr, (const __nv_bfloat16*)dZ,

@@ -56,8 +56,9 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
     const int lddz = l == n_layers - 1 ? lddout : y.N;
     const int dz_compact = (l == n_layers - 1) ? 0 : (y.compact_out ? 1 : 0);
     const ard_dtype dwt = y.dW_is_f32 ? ARD_F32 : ARD_BF16;
+    // the expansion writes every entry of dW, so the compact gradient needs no zeros of its own
     st = ard_layer_bwd_weight(ctx, y.pat, in, dt, dwt, B, y.K, y.N, 1.0f, in_act, ld_in, dZ, lddz, dz_compact,
-                              in ? y.dWk : y.dW, y.ldw, 1, cuda_stream);
+                              in ? y.dWk : y.dW, y.ldw, in ? 0 : 1, cuda_stream);
     if (st != ARD_OK) return st;
     if (in) {
       st = ard_expand_weight_grad_cols(ctx, y.pat, in, dwt, y.K, y.N, y.dWk, y.ldw, y.dW, y.ldw, 1, cuda_stream);

@@ -122,6 +122,12 @@ def test_every_layer_step_call_matches_the_oracle(path, dtype, B, K, N):
             dbh = host(db)
             assert np.abs(dbh[keep] - db_ref).max() <= tol * max(1.0, np.abs(db_ref).max()), tag
             assert np.all(dbh[dropped] == 0), tag
+            # the same from a full-width gradient whose dropped columns hold NaN (never read as values)
+            dZfull = torch.full((B, N), float("nan"), dtype=tdtype(dtype), device="cuda")
+            dZfull[:, torch.from_numpy(keep).cuda()] = dZd[:, :n]
+            db2 = torch.full((N,), float("nan"), dtype=torch.float32, device="cuda")
+            ard.ard_bias_grad(ctx.h, pat, dtype, B, N, dZfull, N, 0, db2, 1)
+            assert torch.equal(db2, db), tag
             assert ard.ard_last_device_status(ctx.h) == 0
     finally:
         ctx.close()
