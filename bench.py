@@ -284,6 +284,7 @@ def run_lstm(args, wl):
     ms_lib = None
     try:
         ref = torch.nn.LSTM(I, H, num_layers=1, bias=True).to(device="cuda", dtype=bf)
+        ref.flatten_parameters()
         Xr = X.clone().requires_grad_(True)
         dHr = dH.to(bf)
 

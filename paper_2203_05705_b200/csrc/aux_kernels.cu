@@ -495,11 +495,12 @@ ard_status launch_expand_weight_grad_cols(ard_ctx* ctx, const int32_t* hdr, cons
 ard_status launch_bias_grad(ard_ctx* ctx, const int32_t* hdr, const void* dZ, int lddz, int dz_is_compact,
                             int is_bf16, int B, int N, float* db, int zero_fill, cudaStream_t s) {
   if (N == 0) return ARD_OK;
-  // many rows of compact, aligned bf16: the batch is cut into slices that are added in a fixed order
+  // 512 rows or more of aligned bf16: the batch is cut into slices that are added in a fixed order (with
+  // fewer rows the plain form below is faster: 2 us against 5 us at 128 rows)
   const int xblocks = (N + BIAS_WIDE_COLS - 1) / BIAS_WIDE_COLS;
   int slices = B / 64;
   if (slices > 32) slices = 32;
-  if (is_bf16 && N % 8 == 0 && slices >= 2 && lddz % 8 == 0 && (reinterpret_cast<uintptr_t>(dZ) & 15) == 0 &&
+  if (is_bf16 && N % 8 == 0 && slices >= 8 && lddz % 8 == 0 && (reinterpret_cast<uintptr_t>(dZ) & 15) == 0 &&
       ctx->d_sk_ws != nullptr && (size_t)slices * xblocks * BIAS_WIDE_COLS * sizeof(float) <= sk_ws_bytes(ctx->sm_count) &&
       (size_t)xblocks * sizeof(int) <= sk_cnt_bytes(ctx->sm_count)) {
     ARD_CUDA_OK(ard_launch(ctx, bias_grad_wide_kernel, dim3(xblocks, slices), dim3(256), 0, s, hdr,
