@@ -358,3 +358,72 @@ def test_mlp_step_784_2048_2048_10(compact, p):
             assert OG.rel_fro(host(dX), bw["dX"]) <= 0.1
     finally:
         ctx.close()
+
+
+def test_full_size_layer_with_compact_matrices_on_sampled_outputs():
+    """The second hidden layer of the 8192-wide stack the benchmark times (batch 4096, K = N = 8192, default
+    launch configuration): compact input, compact weight, fused bias + ReLU and ReLU adjoint.  The oracle
+    recomputes 128 batch rows of the activations and of the input gradient and 64 neurons of the weight
+    gradient; finiteness and the zero pattern are checked on the whole outputs."""
+    c5 = inputs.config5()
+    X, W, dY = c5["X"], c5["W"], c5["dY"]
+    B, K = X.shape
+    N = W.shape[1]
+    bf = torch.bfloat16
+    rng = np.random.default_rng(8)
+    bias = rng.uniform(-0.5, 0.5, N).astype(np.float32)
+    ctx = Ctx(4096)
+    try:
+        pat = ctx.pattern(ard.ARD_ROW, K, N)
+        in_pat = ctx.pattern(ard.ARD_ROW, 8, K)
+        Wd = torch.from_numpy(np.ascontiguousarray(W.T)).to(bf).cuda()
+        Xd = torch.from_numpy(X).to(bf).cuda()
+        dZd = torch.from_numpy(dY).to(bf).cuda()
+        act = inputs.bf16_round(rng.standard_normal((B, K)).astype(np.float32))
+        actd = torch.from_numpy(act).to(bf).cuda()
+        bias_d = torch.from_numpy(bias).cuda()
+        Wk = torch.empty((N, K), dtype=bf, device="cuda")
+        A = torch.empty((B, N), dtype=bf, device="cuda")
+        dX = torch.empty((B, K), dtype=bf, device="cuda")
+        dWk = torch.empty((N, K), dtype=bf, device="cuda")
+        dW = torch.empty((N, K), dtype=bf, device="cuda")
+        rows = np.arange(5, B, B // 128)[:128]
+        tol = TOL[ard.ARD_BF16]
+        for pin, pout in [((2, 1), (2, 2)), ((3, 2), (5, 1)), ((1, 1), (16, 7))]:
+            ard.ard_pattern_set(ctx.h, in_pat, *pin)
+            ard.ard_pattern_set(ctx.h, pat, *pout)
+            keep_in, keep = OP.row_keep(K, *pin), OP.row_keep(N, *pout)
+            n_in, n = len(keep_in), len(keep)
+            for t in (Wk, A, dX, dWk, dW):
+                t.fill_(float("nan"))
+            ard.ard_compact_weight_cols(ctx.h, pat, in_pat, ard.ARD_BF16, K, N, Wd, K, Wk, K)
+            ard.ard_layer_fwd(ctx.h, pat, in_pat, ard.ARD_BF16, B, K, N, 2.0, Xd, K, Wk, K, bias_d, A, N,
+                              ard.ARD_OUT_COMPACT | ard.ARD_FLAG_RELU)
+            ard.ard_layer_bwd_data(ctx.h, pat, in_pat, ard.ARD_BF16, B, K, N, 2.0, dZd, N, 1, Wk, K, actd, K, dX, K)
+            ard.ard_layer_bwd_weight(ctx.h, pat, in_pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, 1.0, Xd, K, dZd, N, 1,
+                                     dWk, K, 0)
+            ard.ard_expand_weight_grad_cols(ctx.h, pat, in_pat, ard.ARD_BF16, K, N, dWk, K, dW, K, 1)
+            torch.cuda.synchronize()
+            assert ard.ard_last_device_status(ctx.h) == 0
+            tag = (pin, pout)
+            ridx = torch.from_numpy(rows).cuda()
+            # forward: sampled batch rows (the compact input is the first n_in columns of X)
+            ref = OM.layer_fwd_compact(X[rows][:, :n_in], keep_in, W, bias, keep, 2.0)
+            assert OG.rel_fro(host(A[ridx])[:, :n], ref) <= tol, tag
+            # input gradient with the ReLU adjoint: sampled batch rows
+            _, _, dA_prev = OM.layer_bwd_compact(X[rows][:, :n_in], keep_in, W, keep, dY[rows][:, :n])
+            refdx = 2.0 * dA_prev * (act[rows][:, :n_in] > 0)
+            assert OG.rel_fro(host(dX[ridx])[:, :n_in], refdx) <= tol, tag
+            # weight gradient: sampled kept neurons, through the expansion
+            js = np.arange(1, n, max(1, n // 64))[:64]
+            refw = dY[:, js].astype(np.float64).T @ X[:, :n_in].astype(np.float64)      # [64 x n_in]
+            got = host(dW[torch.from_numpy(keep[js]).cuda()])
+            assert OG.rel_fro(got[:, keep_in], refw) <= tol, tag
+            # whole outputs: finite where written, zeros exactly where the pattern says
+            assert bool(torch.isfinite(A[:, :n]).all()) and bool(torch.isfinite(dX[:, :n_in]).all())
+            assert bool(torch.isfinite(dW).all())
+            mrow = torch.from_numpy(OP.row_mask(N, *pout) == 0).cuda()
+            mcol = torch.from_numpy(OP.row_mask(K, *pin) == 0).cuda()
+            assert bool(torch.all(dW[mrow, :] == 0)) and bool(torch.all(dW[:, mcol] == 0)), tag
+    finally:
+        ctx.close()
