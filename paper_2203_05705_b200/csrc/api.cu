@@ -1088,7 +1088,33 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
                                 1, cuda_stream);
     if (st != ARD_OK) return st;
   }
-  for (int g = 0; g < 4; ++g) {  // weight gradient: one product over all T*B rows per gate
+  // Weight gradient over all T*B rows: the four gate blocks in one tensor-core launch when the operands
+  // allow it (the M tiles of the four gates share one tile loop), else one product per gate.
+  if (ctx->path != ARD_PATH_CUDA_CORE && H % 8 == 0 &&
+      tc_eligible(ctx, pat, ARD_BF16, T * B, KH, H, DZ, 4 * H, XH, KH, dW, KH, 4) == ARD_OK) {
+    TcArgs t = {};
+    GemmArgs g = {};
+    fill_common(g, ctx, pat, T * B, KH, H, 1.0f);
+    g.A0 = DZ; g.lda0 = 4 * H; g.A1 = XH; g.lda1 = KH; g.out = dW; g.ldo = KH;
+    g.flag0 = 1;
+    g.flag1 = 1;  // rows of dropped units are written as zero
+    g.out_is_f32 = 1;
+    ard_status st = ARD_OK;
+    const char* dZc = reinterpret_cast<const char*>(DZ);
+    for (int gate = 0; gate < 4 && st == ARD_OK; ++gate)
+      st = get_maps(ctx, dZc + (size_t)gate * H * 2, T * B, H, 4 * H, H, MAP_COMPACT_COLS, pat->dp_bound, 64, 64,
+                    &t.mapA4[gate]);
+    if (st == ARD_OK) st = get_maps(ctx, XH, T * B, KH, KH, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);
+    if (st != ARD_OK) return st;
+    t.mapA = t.mapA4[0];
+    t.mapA_indexed = 1;
+    t.mapB_indexed = 0;
+    t.g = g;
+    t.ts = 0;
+    t.bn = ctx->force_bn;
+    return launch_lstm_tc(ctx, 2, t, (cudaStream_t)cuda_stream);
+  }
+  for (int g = 0; g < 4; ++g) {  // one product per gate
     ard_status st = ard_bwd_weight(ctx, pat, ARD_BF16, ARD_F32, T * B, KH, H, 1.0f, XH, KH, dz + (size_t)g * H, 4 * H,
                                    1, dW + (size_t)g * H * KH, KH, 1, cuda_stream);
     if (st != ARD_OK) return st;

@@ -45,11 +45,12 @@ enum TcMode {
   // LSTM gate products over the four gate blocks i|f|g|o of one weight in a single launch: the kept
   // units of gate g are the rows g*H + keep[j] of W, reached through one descriptor table per gate.
   M_LSTM_FWD = 9,       // Z[:, g*ldz + j] = [x,h] . W[g*H + keep[j], :]
-  M_LSTM_BWD_DATA = 10  // d[x,h] = sum_g dZ[:, g*ldz + j] . W[g*H + keep[j], :]
+  M_LSTM_BWD_DATA = 10, // d[x,h] = sum_g dZ[:, g*ldz + j] . W[g*H + keep[j], :]
+  M_LSTM_BWD_WEIGHT = 11 // dW[g*H + keep[j], :] = sum_rows dZ[:, g*ldz + j] . [x,h]   (M tiles: gate-major)
 };
 
 __host__ __device__ constexpr bool a_is_mn(int mode) {
-  return mode == M_ROW_BWD_WEIGHT || mode == M_TILE_BWD_WEIGHT || mode == M_TILEC_BWD_WEIGHT;
+  return mode == M_ROW_BWD_WEIGHT || mode == M_TILE_BWD_WEIGHT || mode == M_TILEC_BWD_WEIGHT || mode == M_LSTM_BWD_WEIGHT;
 }
 __host__ __device__ constexpr bool b_is_mn(int mode) {
   return mode != M_ROW_FWD && mode != M_TILE_FWD && mode != M_TILEC_FWD && mode != M_LSTM_FWD;
@@ -136,7 +137,8 @@ struct TileInfo {
   int nkb;         // number of 64-wide contraction blocks
   const int32_t* klist;  // tile patterns: kept block list for this output tile
   int kper;        // 64-blocks per pattern tile
-  int out_row0;    // tile bwd-weight: first output row (neuron)
+  int out_row0;    // tile bwd-weight: first output row (neuron); LSTM bwd-weight: first row of the tile's gate block
+  int gate;        // LSTM bwd-weight: gate of this tile
   int rows_valid;  // tile bwd-weight: rows of this tile that belong to the kept tile
   int bn;          // N extent of this tile (whole pair)
   int nbox;        // 64-wide B boxes this CTA stages
@@ -195,7 +197,7 @@ struct Sched {
     else if (MODE == M_ROW_BWD_DATA) { M_gemm = p.B; N_gemm = kin; Kc = n_keep; }
     else if (MODE == M_LSTM_FWD) { M_gemm = p.B; N_gemm = ((n_keep + 63) / 64) * 256; Kc = p.K; }
     else if (MODE == M_LSTM_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 4 * (((n_keep + 63) / 64) * 64); }
-    else if (MODE == M_ROW_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = kin; Kc = p.B; }
+    else if (MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = kin; Kc = p.B; }
     else if (MODE == M_TILE_FWD || MODE == M_TILEC_FWD) { M_gemm = p.B; N_gemm = p.N; Kc = 0; }
     else if (MODE == M_TILE_BWD_DATA || MODE == M_TILEC_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 0; }
     else { M_gemm = p.N; N_gemm = p.K; Kc = p.B; }
@@ -238,7 +240,9 @@ struct Sched {
       Nt = subn;
     } else {
       Mt = (M_gemm + BM * CTAS - 1) / (BM * CTAS);
-      if (MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA || MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_DATA) {
+      if (MODE == M_LSTM_BWD_WEIGHT) Mt *= 4;  // the M tiles of the four gate blocks, gate after gate
+      if (MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA || MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_DATA ||
+          MODE == M_LSTM_BWD_WEIGHT) {
         if (p.force_bn) {
           bn = p.force_bn;
         } else {
@@ -454,6 +458,13 @@ struct Sched {
     }
     ti.m0 = mt * BM * CTAS + rank * BM;  // this CTA's 128 rows of the tile
     ti.n0 = nt * bn;
+    ti.gate = 0;
+    if (MODE == M_LSTM_BWD_WEIGHT) {
+      const int mt_gate = Mt >> 2;
+      ti.gate = mt / mt_gate;
+      ti.m0 = (mt - ti.gate * mt_gate) * BM * CTAS + rank * BM;  // row inside the gate's compact block
+      ti.out_row0 = ti.gate * p.N;
+    }
     if (MODE == M_TILE_FWD) {
       const int c = ti.n0 / p.ts;
       ti.klist = p.col_idx + p.col_ptr[c];
@@ -623,6 +634,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
           if (MODE == M_LSTM_BWD_DATA) tensormap_acquire(p.mapA4[g] + e);
         }
       }
+      if (MODE == M_LSTM_BWD_WEIGHT) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) tensormap_acquire(p.mapA4[g] + e);
+      }
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -670,7 +685,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
           } else {
 #pragma unroll
             for (int i = 0; i < BM / 64; ++i)  // [64 k rows][64 m] per box
-              load(sA + i * (64 * BK * 2), mapA, ti.ax[i], kx);
+              load(sA + i * (64 * BK * 2), MODE == M_LSTM_BWD_WEIGHT ? p.mapA4[ti.gate] + e : mapA, ti.ax[i], kx);
           }
           // B always moves in 64-wide boxes: K-major [64 rows][64 k] stacked, MN-major [64 k][64 n].
           // In a pair this CTA stages the second half of the tile's B boxes if its rank is 1.
@@ -763,9 +778,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
       // Output row and validity by mode.
       bool row_ok;
       long long out_row;
-      if (MODE == M_ROW_BWD_WEIGHT) {
+      if (MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_WEIGHT) {
         row_ok = m < sch.M_gemm;
         out_row = (long long)bb + (long long)m * dp;
+        if (MODE == M_LSTM_BWD_WEIGHT) out_row += ti.out_row0;
       } else if (MODE == M_TILE_BWD_WEIGHT) {
         row_ok = row_in_tile < ti.rows_valid && m < sch.M_gemm;
         out_row = m;
@@ -903,11 +919,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
                                                    : min(32, sch.N_gemm - n));
           if (row_ok && nvalid > 0) {
             store_row32(p.out, (size_t)out_row * p.ldo, n, v, nvalid, p.out_is_f32, p.accumulate);
-            if (MODE == M_ROW_BWD_WEIGHT && p.zero_fill) {
+            if ((MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_WEIGHT) && p.zero_fill) {
               // Compact row m owns output rows [m*dp, (m+1)*dp); the last one also owns the tail.
-              const long long first = (long long)m * dp;
-              const long long lastrow =
-                  (m == sch.M_gemm - 1) ? (long long)p.N - 1 : min((long long)(m + 1) * dp - 1, (long long)p.N - 1);
+              const long long goff = (MODE == M_LSTM_BWD_WEIGHT) ? ti.out_row0 : 0;  // the gate's block of rows
+              const long long first = goff + (long long)m * dp;
+              const long long lastrow = goff + ((m == sch.M_gemm - 1) ? (long long)p.N - 1
+                                                                     : min((long long)(m + 1) * dp - 1, (long long)p.N - 1));
               for (long long rz = first; rz <= lastrow; ++rz)
                 if (rz != out_row) zero_row32(p.out, (size_t)rz * p.ldo, n, nvalid, p.out_is_f32);
             }
@@ -1248,5 +1265,12 @@ ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStrea
   p.ldact = 0;
   const int mt = cdiv(p.B, BM);
   if (!backward) return launch_mode<256, M_LSTM_FWD, 1>(ctx, p, mt * cdiv(p.N, 64), s);
+  if (backward == 2) {
+    // weight gradient of the four gate blocks: p.B = rows summed over, p.N = H units per gate
+    p.zero_fill = a.g.flag1;
+    if (ctx->use_pairs && p.N > BM && (p.force_bn == 0 || p.force_bn >= 128))
+      return launch_mode<256, M_LSTM_BWD_WEIGHT, 2>(ctx, p, 4 * cdiv(p.N, 2 * BM) * cdiv(p.K, 128), s);
+    return launch_mode<256, M_LSTM_BWD_WEIGHT, 1>(ctx, p, 4 * cdiv(p.N, BM) * cdiv(p.K, 64), s);
+  }
   return launch_mode<256, M_LSTM_BWD_DATA, 1>(ctx, p, mt * cdiv(p.K, 64), s);
 }

@@ -30,7 +30,7 @@ __device__ void philox4x32_10(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
   }
 }
 
-constexpr int SAMPLER_THREADS = 256;
+constexpr int SAMPLER_THREADS = 1024;  // tile patterns; row patterns launch 256 (fewer lists to fill)
 constexpr int SCAN_CAP = 2048;  // tile-columns whose running count fits in shared memory
 
 __global__ void __launch_bounds__(SAMPLER_THREADS)
@@ -40,6 +40,7 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
                   unsigned long long iteration, uint32_t stream_id, int forced_dp, int forced_b, int kind,
                   int units, int Tr, int Tc, int ts, unsigned long long* __restrict__ counter, int advance) {
   __shared__ int s_dp, s_b;
+  const int nthreads = (int)blockDim.x;
   __shared__ unsigned long long s_cdf[64];
   pdl_launch_dependents();
   pdl_wait_prior_grids();  // earlier kernels may still be reading the lists this kernel rewrites
@@ -91,12 +92,12 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
     hdr[HDR_MAPIDX] = dp * (dp - 1) / 2 + (b - 1);
   }
   // Eq. 1 on the 1-based unit index i = b + j*dp  ->  0-based b-1 + j*dp, ascending.
-  for (int j = threadIdx.x; j < n_keep; j += SAMPLER_THREADS) idx[j] = b - 1 + j * dp;
+  for (int j = threadIdx.x; j < n_keep; j += nthreads) idx[j] = b - 1 + j * dp;
   if (kind != ARD_TILE) return;
 
   // Tiles are numbered row-major, so the ascending list is already grouped by tile-row.
-  for (int j = threadIdx.x; j < n_keep; j += SAMPLER_THREADS) row_idx[j] = (b - 1 + j * dp) % Tc;
-  for (int r = threadIdx.x; r <= Tr; r += SAMPLER_THREADS) {
+  for (int j = threadIdx.x; j < n_keep; j += nthreads) row_idx[j] = (b - 1 + j * dp) % Tc;
+  for (int r = threadIdx.x; r <= Tr; r += nthreads) {
     // kept tiles with 0-based linear index < r*Tc
     const long long lim = (long long)r * Tc;  // count of j with b-1 + j*dp < lim
     int cnt = 0;
@@ -109,7 +110,7 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
   // memory would cost a round trip per column).
   __shared__ int s_cnt[SCAN_CAP];
   const bool in_smem = Tc <= SCAN_CAP;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = SAMPLER_THREADS / 32;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = nthreads / 32;
   auto kept = [&](int r, int c) {
     const int lin = r * Tc + c - (b - 1);
     return r < Tr && lin >= 0 && lin % dp == 0;
@@ -131,7 +132,7 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
   }
   __syncthreads();
   if (in_smem) {
-    for (int c = threadIdx.x; c < Tc; c += SAMPLER_THREADS) col_ptr[c] = s_cnt[c];
+    for (int c = threadIdx.x; c < Tc; c += nthreads) col_ptr[c] = s_cnt[c];
     if (threadIdx.x == 0) col_ptr[Tc] = n_keep;
   }
   for (int c = warp; c < Tc; c += nwarps) {
@@ -150,7 +151,7 @@ ard_sample_kernel(int32_t* __restrict__ hdr, int32_t* __restrict__ idx, int32_t*
 ard_status launch_sampler(ard_ctx* ctx, ard_pattern* pat, const unsigned long long* d_cdf, int ndp, uint64_t seed,
                           uint64_t iteration, uint32_t stream_id, int forced_dp, int forced_b, cudaStream_t s,
                           unsigned long long* d_counter, int advance) {
-  ARD_CUDA_OK(ard_launch(ctx, ard_sample_kernel, dim3(1), dim3(SAMPLER_THREADS), 0, s, pat->d_hdr, pat->d_idx,
+  ARD_CUDA_OK(ard_launch(ctx, ard_sample_kernel, dim3(1), dim3(pat->kind == ARD_TILE ? SAMPLER_THREADS : 256), 0, s, pat->d_hdr, pat->d_idx,
                          pat->d_col_ptr, pat->d_col_idx, pat->d_row_ptr, pat->d_row_idx, d_cdf, ndp,
                          (unsigned long long)seed, (unsigned long long)iteration, stream_id, forced_dp, forced_b,
                          (int)pat->kind, pat->units, pat->Tr, pat->Tc, pat->ts, d_counter, advance));
