@@ -169,6 +169,114 @@ __global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts)
     }
 }
 
+// ---- layers with at most 16 neurons (an output layer) -----------------------------------------------
+// The tiled kernel above would give such a layer a handful of CTAs, each walking the whole fan-in alone.
+// Forward: one CTA per batch row; every thread walks a strided share of the fan-in with one accumulator
+// per kept neuron, then the CTA adds the shares (fixed order).  Backward-weight: 32 fan-in columns per CTA,
+// the batch rows dealt to its 8 warps, one accumulator per kept neuron, warp sums added in warp order.
+constexpr int SKINNY_N = 16;
+
+template <typename T>
+__global__ void __launch_bounds__(256) skinny_fwd_kernel(GemmArgs g) {
+  __shared__ float part[8][SKINNY_N];
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int n_keep = g.hdr[HDR_NKEEP];
+  const int kin = g.hdr_in != nullptr ? g.hdr_in[HDR_NKEEP] : g.K;
+  const int m = blockIdx.x;
+  const T* X = reinterpret_cast<const T*>(g.A0) + (size_t)m * g.lda0;
+  const T* W = reinterpret_cast<const T*>(g.A1);
+  float acc[SKINNY_N];
+#pragma unroll
+  for (int n = 0; n < SKINNY_N; ++n) acc[n] = 0.f;
+  int rows[SKINNY_N];
+#pragma unroll
+  for (int n = 0; n < SKINNY_N; ++n) rows[n] = n < n_keep ? g.idx[n] : 0;
+  for (int k = threadIdx.x; k < kin; k += 256) {
+    const float x = to_f<T>(X[k]);
+#pragma unroll
+    for (int n = 0; n < SKINNY_N; ++n)
+      if (n < n_keep) acc[n] = fmaf(x, to_f<T>(W[(size_t)rows[n] * g.lda1 + k]), acc[n]);
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int n = 0; n < SKINNY_N; ++n) {
+    float v = acc[n];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if (lane == 0) part[warp][n] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < n_keep) {
+    const int n = threadIdx.x;
+    float v = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) v += part[w][n];
+    if (g.bias != nullptr) v += g.bias[g.idx[n]];
+    if (g.relu) v = fmaxf(v, 0.f);
+    v *= g.alpha;
+    const size_t off = (size_t)m * g.ldo + (g.flag0 == ARD_OUT_SCATTER_ZEROFILL ? g.idx[n] : n);
+    store_out(g.out, off, v, g.out_is_f32, g.accumulate);
+  }
+  if (g.flag0 == ARD_OUT_SCATTER_ZEROFILL && threadIdx.x >= 32 && threadIdx.x < 32 + g.N) {
+    // full-width output: the dropped neurons' entries of this row are zero (no separate clearing pass)
+    const int o = threadIdx.x - 32, dp = g.hdr[HDR_DP], bb = g.hdr[HDR_B] - 1;
+    if (!(o >= bb && (o - bb) % dp == 0)) store_out(g.out, (size_t)m * g.ldo + o, 0.f, g.out_is_f32);
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) skinny_bwd_weight_kernel(GemmArgs g) {
+  // 32 fan-in columns per CTA; its 8 warps take every eighth batch row and their sums are added in warp order
+  __shared__ float part[8][SKINNY_N][33];
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int n_keep = g.hdr[HDR_NKEEP];
+  const int kin = g.hdr_in != nullptr ? g.hdr_in[HDR_NKEEP] : g.K;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int k = blockIdx.x * 32 + lane;
+  if (blockIdx.x * 32 >= kin) return;
+  const T* dY = reinterpret_cast<const T*>(g.A0);
+  const T* X = reinterpret_cast<const T*>(g.A1);
+  int cols[SKINNY_N];
+#pragma unroll
+  for (int n = 0; n < SKINNY_N; ++n) cols[n] = n < n_keep ? (g.flag0 ? n : g.idx[n]) : 0;
+  float acc[SKINNY_N];
+#pragma unroll
+  for (int n = 0; n < SKINNY_N; ++n) acc[n] = 0.f;
+  if (k < kin) {
+#pragma unroll 4
+    for (int r = warp; r < g.B; r += 8) {
+      const float x = to_f<T>(X[(size_t)r * g.lda1 + k]);
+      const T* dy = dY + (size_t)r * g.lda0;
+#pragma unroll
+      for (int n = 0; n < SKINNY_N; ++n)
+        if (n < n_keep) acc[n] = fmaf(to_f<T>(dy[cols[n]]), x, acc[n]);
+    }
+  }
+#pragma unroll
+  for (int n = 0; n < SKINNY_N; ++n) part[warp][n][lane] = acc[n];
+  __syncthreads();
+  // 32 columns x up to 16 neurons = up to 512 outputs for 256 threads
+  for (int o = threadIdx.x; o < 32 * n_keep; o += 256) {
+    const int n = o >> 5, c = o & 31;
+    const int kk = blockIdx.x * 32 + c;
+    if (kk >= kin) continue;
+    float v = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) v += part[w][n][c];
+    store_out(g.out, (size_t)g.idx[n] * g.ldo + kk, g.alpha * v, g.out_is_f32, g.accumulate);
+  }
+  if (g.flag1) {
+    // rows of dropped neurons, this CTA's 32 columns
+    const int dp = g.hdr[HDR_DP], bb = g.hdr[HDR_B] - 1;
+    for (int o = threadIdx.x; o < 32 * g.N; o += 256) {
+      const int row = o >> 5, kk = blockIdx.x * 32 + (o & 31);
+      if (kk < kin && !(row >= bb && (row - bb) % dp == 0)) store_out(g.out, (size_t)row * g.ldo + kk, 0.f, g.out_is_f32);
+    }
+  }
+}
+
 template <typename T, int KIND, int OP>
 void launch_one(const ard_ctx* ctx, const GemmArgs& a, int ts, int Mmax, int Nmax, cudaStream_t s) {
   dim3 grid((Nmax + T_N - 1) / T_N, (Mmax + T_M - 1) / T_M);
@@ -197,14 +305,26 @@ ard_status launch_gemm_cc(ard_ctx* ctx, ard_kind kind, GemmOp op, ard_dtype dtyp
   if ((a.B == 0 && op != OP_BWD_WEIGHT) || a.K == 0 || a.N == 0) return ARD_OK;
   const size_t es_out = a.out_is_f32 ? 4 : 2;
   // Row patterns: dropped outputs are cleared by a strided memset before the kept ones are written.
-  if (kind == ARD_ROW && op == OP_FWD && a.flag0 == ARD_OUT_SCATTER_ZEROFILL) {
+  const bool small_layer = kind == ARD_ROW && a.N <= SKINNY_N && (op == OP_FWD ? a.B > 0 : op == OP_BWD_WEIGHT);
+  if (small_layer) {
+    // the kernels for a handful of neurons write their own zeros
+  } else if (kind == ARD_ROW && op == OP_FWD && a.flag0 == ARD_OUT_SCATTER_ZEROFILL) {
     ARD_CUDA_OK(cudaMemset2DAsync(a.out, (size_t)a.ldo * es_out, 0, (size_t)a.N * es_out, a.B, s));
   }
-  if (kind == ARD_ROW && op == OP_BWD_WEIGHT && a.flag1) {
+  if (!small_layer && kind == ARD_ROW && op == OP_BWD_WEIGHT && a.flag1) {
     ARD_CUDA_OK(cudaMemset2DAsync(a.out, (size_t)a.ldo * es_out, 0, (size_t)a.K * es_out, a.N, s));
   }
-  if (dtype == ARD_F32) dispatch<float>(ctx, kind, op, a, ts, s);
-  else dispatch<__nv_bfloat16>(ctx, kind, op, a, ts, s);
+  if (kind == ARD_ROW && a.N <= SKINNY_N && op == OP_FWD && a.B > 0) {
+    if (dtype == ARD_F32) (void)ard_launch(ctx, skinny_fwd_kernel<float>, dim3(a.B), dim3(256), 0, s, a);
+    else (void)ard_launch(ctx, skinny_fwd_kernel<__nv_bfloat16>, dim3(a.B), dim3(256), 0, s, a);
+  } else if (kind == ARD_ROW && a.N <= SKINNY_N && op == OP_BWD_WEIGHT) {
+    if (dtype == ARD_F32) (void)ard_launch(ctx, skinny_bwd_weight_kernel<float>, dim3((a.K + 31) / 32), dim3(256), 0, s, a);
+    else (void)ard_launch(ctx, skinny_bwd_weight_kernel<__nv_bfloat16>, dim3((a.K + 31) / 32), dim3(256), 0, s, a);
+  } else if (dtype == ARD_F32) {
+    dispatch<float>(ctx, kind, op, a, ts, s);
+  } else {
+    dispatch<__nv_bfloat16>(ctx, kind, op, a, ts, s);
+  }
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;

@@ -38,6 +38,8 @@ def _dev(a, dtype, ld, fill=float("nan")):
     (ard.ARD_PATH_TENSOR_CORE, ard.ARD_BF16, 100, 1024, 264),    # one M tile, several contraction blocks
     (ard.ARD_PATH_CUDA_CORE, ard.ARD_BF16, 37, 90, 70),
     (ard.ARD_PATH_CUDA_CORE, ard.ARD_F32, 37, 90, 70),
+    (ard.ARD_PATH_AUTO, ard.ARD_BF16, 130, 1000, 10),            # an output layer: the kernels for <= 16 neurons
+    (ard.ARD_PATH_AUTO, ard.ARD_F32, 33, 300, 16),
 ])
 def test_every_layer_step_call_matches_the_oracle(path, dtype, B, K, N):
     rng = np.random.default_rng(B * 7 + K)
