@@ -203,6 +203,10 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->d_lstm_partial = nullptr;
   if (const char* e = getenv("ARD_PDL")) ctx->use_pdl = atoi(e) ? 1 : 0;
   ctx->pdl_in_capture = 1;
+  ctx->mlp_two_streams = 1;
+  if (const char* e = getenv("ARD_MLP_STREAMS")) ctx->mlp_two_streams = atoi(e) >= 2 ? 1 : 0;
+  ctx->side_stream = nullptr;
+  ctx->n_ev = 0;
   if (const char* e = getenv("ARD_PDL_CAPTURE")) ctx->pdl_in_capture = atoi(e) ? 1 : 0;
   ctx->sk_min_blocks = 16;
   if (const char* e = getenv("ARD_STREAM_K")) ctx->stream_k = atoi(e);
@@ -271,6 +275,8 @@ ard_status ard_destroy(ard_ctx* ctx) {
   if (ctx->d_grid_bar) cudaFree(ctx->d_grid_bar);
   if (ctx->d_lstm_partial) cudaFree(ctx->d_lstm_partial);
   if (ctx->d_status) cudaFree(ctx->d_status);
+  for (int i = 0; i < ctx->n_ev; ++i) cudaEventDestroy(ctx->ev[i]);
+  if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
   delete ctx;
   return ARD_OK;
 }

@@ -65,6 +65,8 @@ enum MapVariant {
   MAP_COMPACT_COLS = 2   // per (dp,b): all rows, cols 0..n_keep-1 of a compact matrix
 };
 
+constexpr int ARD_MLP_EVENTS = 72;  // fork + forward + join and one per layer each way, up to 32 layers
+
 struct ard_ctx {
   int device;
   int sm_count;
@@ -92,6 +94,12 @@ struct ard_ctx {
   unsigned long long launches;
   unsigned long long epoch;   // bumped by every public GEMM call
   void* encode_fn;  // cuTensorMapEncodeTiled, resolved at run time
+  // ard_mlp_step: the weight-side work of an iteration (weight compaction, weight and bias gradients) runs on
+  // a second stream, forked from and joined back into the caller's stream with these events
+  int mlp_two_streams;
+  cudaStream_t side_stream;
+  cudaEvent_t ev[ARD_MLP_EVENTS];
+  int n_ev;  // events created so far (0: none yet)
 };
 
 // Shared tail of the tensor-core row kernels: every CTA owns two slots, each holding the fp32 partial

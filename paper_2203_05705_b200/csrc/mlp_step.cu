@@ -6,6 +6,19 @@
 // into a CUDA graph once its descriptor tables exist (run it once before capturing).
 #include "ard_internal.h"
 
+namespace {
+struct DeviceGuardLite {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuardLite(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuardLite() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+}  // namespace
+
 extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, int n_layers, int B, const void* X,
                                    int ldx, const void* dOut, int lddout, void* dX, int lddx, int dist_id,
                                    uint64_t seed, uint64_t iteration_base, uint64_t* iteration_counter,
@@ -24,6 +37,39 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
   if (layers[n_layers - 1].compact_out) return ARD_ERR_INVALID_ARG;  // dOut is full width
   if (last_sampled >= 0 && !iteration_counter) return ARD_ERR_INVALID_ARG;
   ard_status st;
+  cudaStream_t main_s = (cudaStream_t)cuda_stream;
+  // Two streams: everything the activations and their gradients wait for stays on the caller's stream;
+  // weight compaction and the weight / bias gradients, which nothing downstream of them in the iteration
+  // reads, run beside it on the context's second stream (forked after the patterns are drawn, joined at the
+  // end, so the caller sees one ordered stream).  Needs compact matrices between all hidden layers: the
+  // full-width form gathers through the context workspace, which the two streams would share.
+  bool two = ctx->mlp_two_streams && n_layers >= 2 && n_layers <= 32;
+  for (int l = 0; l + 1 < n_layers && two; ++l) two = layers[l].compact_out != 0;
+  if (two && ctx->n_ev == 0) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(main_s, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
+      two = false;  // first use inside a capture: nothing may be created now
+    } else {
+      DeviceGuardLite guard(ctx->device);
+      if (cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        ctx->side_stream = nullptr;
+        two = false;
+      }
+      for (int i = 0; two && i < ARD_MLP_EVENTS; ++i) {
+        if (cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) != cudaSuccess) two = false;
+        else ctx->n_ev = i + 1;
+      }
+    }
+  }
+  if (two && ctx->n_ev < ARD_MLP_EVENTS) two = false;
+  cudaStream_t side_s = two ? ctx->side_stream : main_s;
+  void* side = (void*)side_s;
+  // event slots: 0 fork, 1 forward done, 2 join, 3 + l weight of layer l compacted, 35 + l dZ of layer l ready
+  auto after = [&](cudaStream_t waiter, cudaStream_t producer, int slot) -> bool {
+    if (!two) return true;
+    return cudaEventRecord(ctx->ev[slot], producer) == cudaSuccess &&
+           cudaStreamWaitEvent(waiter, ctx->ev[slot], 0) == cudaSuccess;
+  };
   // ---- patterns of this iteration (stream id = layer index + 1) ----
   for (int l = 0; l < n_layers; ++l) {
     if (!layers[l].sample) continue;
@@ -32,12 +78,23 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
     if (st != ARD_OK) return st;
   }
   // ---- forward ----
+  if (!after(side_s, main_s, 0)) return ARD_ERR_CUDA;  // fork: the second stream starts behind the samplers
+  if (two) {
+    for (int l = 1; l < n_layers; ++l) {  // all weight compactions, beside the first layer's product
+      const ard_mlp_layer& y = layers[l];
+      st = ard_compact_weight_cols(ctx, y.pat, layers[l - 1].pat, dt, y.K, y.N, y.W, y.ldw, y.Wk, y.ldw, side);
+      if (st != ARD_OK) return st;
+      if (cudaEventRecord(ctx->ev[3 + l], side_s) != cudaSuccess) return ARD_ERR_CUDA;
+    }
+  }
   for (int l = 0; l < n_layers; ++l) {
     const ard_mlp_layer& y = layers[l];
     const ard_pattern* in = (l > 0 && layers[l - 1].compact_out) ? layers[l - 1].pat : nullptr;
     const void* in_act = l == 0 ? X : layers[l - 1].A;
     const int ld_in = l == 0 ? ldx : layers[l - 1].N;
-    if (in) {
+    if (in && two) {
+      if (cudaStreamWaitEvent(main_s, ctx->ev[3 + l], 0) != cudaSuccess) return ARD_ERR_CUDA;
+    } else if (in) {
       st = ard_compact_weight_cols(ctx, y.pat, in, dt, y.K, y.N, y.W, y.ldw, y.Wk, y.ldw, cuda_stream);
       if (st != ARD_OK) return st;
     }
@@ -47,6 +104,7 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
     if (st != ARD_OK) return st;
   }
   // ---- backward ----
+  if (!after(side_s, main_s, 1)) return ARD_ERR_CUDA;  // the second stream reads the activations from here on
   for (int l = n_layers - 1; l >= 0; --l) {
     const ard_mlp_layer& y = layers[l];
     const ard_pattern* in = (l > 0 && layers[l - 1].compact_out) ? layers[l - 1].pat : nullptr;
@@ -57,15 +115,17 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
     const int dz_compact = (l == n_layers - 1) ? 0 : (y.compact_out ? 1 : 0);
     const ard_dtype dwt = y.dW_is_f32 ? ARD_F32 : ARD_BF16;
     // the expansion writes every entry of dW, so the compact gradient needs no zeros of its own
+    // weight side (second stream when there are two): needs dZ of this layer, which the layer above wrote
+    if (two && l < n_layers - 1 && cudaStreamWaitEvent(side_s, ctx->ev[35 + l], 0) != cudaSuccess) return ARD_ERR_CUDA;
     st = ard_layer_bwd_weight(ctx, y.pat, in, dt, dwt, B, y.K, y.N, 1.0f, in_act, ld_in, dZ, lddz, dz_compact,
-                              in ? y.dWk : y.dW, y.ldw, in ? 0 : 1, cuda_stream);
+                              in ? y.dWk : y.dW, y.ldw, in ? 0 : 1, side);
     if (st != ARD_OK) return st;
     if (in) {
-      st = ard_expand_weight_grad_cols(ctx, y.pat, in, dwt, y.K, y.N, y.dWk, y.ldw, y.dW, y.ldw, 1, cuda_stream);
+      st = ard_expand_weight_grad_cols(ctx, y.pat, in, dwt, y.K, y.N, y.dWk, y.ldw, y.dW, y.ldw, 1, side);
       if (st != ARD_OK) return st;
     }
     if (y.db) {
-      st = ard_bias_grad(ctx, y.pat, dt, B, y.N, dZ, lddz, dz_compact, y.db, 1, cuda_stream);
+      st = ard_bias_grad(ctx, y.pat, dt, B, y.N, dZ, lddz, dz_compact, y.db, 1, side);
       if (st != ARD_OK) return st;
     }
     if (l > 0) {
@@ -73,10 +133,12 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
       st = ard_layer_bwd_data(ctx, y.pat, in, dt, B, y.K, y.N, prev.alpha, dZ, lddz, dz_compact, in ? y.Wk : y.W, y.ldw,
                               prev.relu ? prev.A : nullptr, prev.N, prev.dZ, prev.N, cuda_stream);
       if (st != ARD_OK) return st;
+      if (two && cudaEventRecord(ctx->ev[35 + l - 1], main_s) != cudaSuccess) return ARD_ERR_CUDA;
     } else if (dX) {
       st = ard_bwd_data(ctx, y.pat, dt, B, y.K, y.N, 1.0f, dZ, lddz, dz_compact, y.W, y.ldw, dX, lddx, cuda_stream);
       if (st != ARD_OK) return st;
     }
   }
+  if (!after(main_s, side_s, 2)) return ARD_ERR_CUDA;  // join
   return ARD_OK;
 }

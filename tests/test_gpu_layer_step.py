@@ -429,3 +429,54 @@ def test_full_size_layer_with_compact_matrices_on_sampled_outputs():
             assert bool(torch.all(dW[mrow, :] == 0)) and bool(torch.all(dW[:, mcol] == 0)), tag
     finally:
         ctx.close()
+
+
+def test_mlp_step_replayed_from_a_graph_equals_the_same_iterations_called_one_by_one():
+    """The iteration forks its weight-side work onto a second stream; captured once and replayed, it must draw
+    the next pattern every time and give the bits the one-by-one calls give."""
+    dims, B, p = [784, 2048, 2048, 10], 128, 0.5
+    rng = np.random.default_rng(23)
+    ctx = Ctx(4096)
+    try:
+        ard.ard_set_distribution(ctx.h, 0, inputs.max_entropy_K(p, 16))
+        layers, arr, _, _ = _stack(ctx, dims, B, p, 1, rng)
+        L = len(layers)
+        counter = torch.zeros(1, dtype=torch.int64, device="cuda")
+        X, dOut = inputs.config2_step(0)
+        Xd = torch.from_numpy(X).to(torch.bfloat16).cuda()
+        dOd = torch.from_numpy(dOut).to(torch.bfloat16).cuda()
+        dX = torch.zeros((B, dims[0]), dtype=torch.bfloat16, device="cuda")
+
+        def step():
+            ard.ard_mlp_step(ctx.h, arr, L, B, Xd, dims[0], dOd, dims[-1], dX, dims[0], 0, inputs.BASE_SEED, 900, counter)
+
+        def snapshot():
+            torch.cuda.synchronize()
+            out = [dX.clone(), layers[-1]["A"].clone()]
+            for d in layers:
+                out += [d["dW"].clone(), d["db"].clone()]
+            return out, [tuple(ard.ard_pattern_to_host(d["pat"], 0)[:2]) for d in layers]
+
+        side = torch.cuda.Stream()
+        ref = []
+        with torch.cuda.stream(side):
+            for _ in range(4):
+                step()
+                ref.append(snapshot())
+        counter.zero_()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        for it in range(4):
+            for d in layers:                                        # stale results must not pass for fresh ones
+                d["dW"].fill_(float("nan"))
+            graph.replay()
+            got, pats = snapshot()
+            assert int(counter.item()) == it + 1
+            assert pats == ref[it][1], it
+            for a, c in zip(got, ref[it][0]):
+                assert torch.equal(a, c), it
+        assert len({tuple(r[1]) for r in ref}) > 1                 # the patterns did change
+        assert ard.ard_last_device_status(ctx.h) == 0
+    finally:
+        ctx.close()
