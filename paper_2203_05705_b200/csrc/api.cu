@@ -206,6 +206,7 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->mlp_two_streams = 1;
   if (const char* e = getenv("ARD_MLP_STREAMS")) ctx->mlp_two_streams = atoi(e) >= 2 ? 1 : 0;
   ctx->side_stream = nullptr;
+  ctx->aux_stream = nullptr;
   ctx->n_ev = 0;
   if (const char* e = getenv("ARD_PDL_CAPTURE")) ctx->pdl_in_capture = atoi(e) ? 1 : 0;
   ctx->sk_min_blocks = 16;
@@ -277,6 +278,7 @@ ard_status ard_destroy(ard_ctx* ctx) {
   if (ctx->d_status) cudaFree(ctx->d_status);
   for (int i = 0; i < ctx->n_ev; ++i) cudaEventDestroy(ctx->ev[i]);
   if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
+  if (ctx->aux_stream) cudaStreamDestroy(ctx->aux_stream);
   delete ctx;
   return ARD_OK;
 }

@@ -65,7 +65,7 @@ enum MapVariant {
   MAP_COMPACT_COLS = 2   // per (dp,b): all rows, cols 0..n_keep-1 of a compact matrix
 };
 
-constexpr int ARD_MLP_EVENTS = 72;  // fork + forward + join and one per layer each way, up to 32 layers
+constexpr int ARD_MLP_EVENTS = 104;  // fork, forward done, two joins, and three per layer (up to 32 layers)
 
 struct ard_ctx {
   int device;
@@ -98,6 +98,7 @@ struct ard_ctx {
   // a second stream, forked from and joined back into the caller's stream with these events
   int mlp_two_streams;
   cudaStream_t side_stream;
+  cudaStream_t aux_stream;  // expansion of the weight gradients and bias gradients
   cudaEvent_t ev[ARD_MLP_EVENTS];
   int n_ev;  // events created so far (0: none yet)
 };

@@ -38,10 +38,10 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
   if (last_sampled >= 0 && !iteration_counter) return ARD_ERR_INVALID_ARG;
   ard_status st;
   cudaStream_t main_s = (cudaStream_t)cuda_stream;
-  // Two streams: everything the activations and their gradients wait for stays on the caller's stream;
-  // weight compaction and the weight / bias gradients, which nothing downstream of them in the iteration
-  // reads, run beside it on the context's second stream (forked after the patterns are drawn, joined at the
-  // end, so the caller sees one ordered stream).  Needs compact matrices between all hidden layers: the
+  // Three streams: everything the activations and their gradients wait for stays on the caller's stream;
+  // weight compaction and the weight gradients, which nothing downstream of them in the iteration reads,
+  // run beside it on the context's second stream, the expansion of those gradients and the bias gradients
+  // on a third (forked after the patterns are drawn, joined at the end: the caller sees one ordered stream).  Needs compact matrices between all hidden layers: the
   // full-width form gathers through the context workspace, which the two streams would share.
   bool two = ctx->mlp_two_streams && n_layers >= 2 && n_layers <= 32;
   for (int l = 0; l + 1 < n_layers && two; ++l) two = layers[l].compact_out != 0;
@@ -55,6 +55,10 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
         ctx->side_stream = nullptr;
         two = false;
       }
+      if (two && cudaStreamCreateWithFlags(&ctx->aux_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        ctx->aux_stream = nullptr;
+        two = false;
+      }
       for (int i = 0; two && i < ARD_MLP_EVENTS; ++i) {
         if (cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) != cudaSuccess) two = false;
         else ctx->n_ev = i + 1;
@@ -63,8 +67,11 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
   }
   if (two && ctx->n_ev < ARD_MLP_EVENTS) two = false;
   cudaStream_t side_s = two ? ctx->side_stream : main_s;
+  cudaStream_t aux_s = two ? ctx->aux_stream : main_s;
   void* side = (void*)side_s;
-  // event slots: 0 fork, 1 forward done, 2 join, 3 + l weight of layer l compacted, 35 + l dZ of layer l ready
+  void* aux = (void*)aux_s;
+  // event slots: 0 fork, 1 forward done, 2 join, 3 + l weight of layer l compacted, 35 + l dZ of layer l ready,
+  // 67 join of the third stream, 68 + l compact weight gradient of layer l ready
   auto after = [&](cudaStream_t waiter, cudaStream_t producer, int slot) -> bool {
     if (!two) return true;
     return cudaEventRecord(ctx->ev[slot], producer) == cudaSuccess &&
@@ -104,7 +111,8 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
     if (st != ARD_OK) return st;
   }
   // ---- backward ----
-  if (!after(side_s, main_s, 1)) return ARD_ERR_CUDA;  // the second stream reads the activations from here on
+  if (!after(side_s, main_s, 1)) return ARD_ERR_CUDA;  // the other streams read the activations from here on
+  if (two && cudaStreamWaitEvent(aux_s, ctx->ev[1], 0) != cudaSuccess) return ARD_ERR_CUDA;
   for (int l = n_layers - 1; l >= 0; --l) {
     const ard_mlp_layer& y = layers[l];
     const ard_pattern* in = (l > 0 && layers[l - 1].compact_out) ? layers[l - 1].pat : nullptr;
@@ -120,12 +128,15 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
     st = ard_layer_bwd_weight(ctx, y.pat, in, dt, dwt, B, y.K, y.N, 1.0f, in_act, ld_in, dZ, lddz, dz_compact,
                               in ? y.dWk : y.dW, y.ldw, in ? 0 : 1, side);
     if (st != ARD_OK) return st;
+    // third stream: expansion of this layer's gradient and its bias gradient (both off everybody's path)
     if (in) {
-      st = ard_expand_weight_grad_cols(ctx, y.pat, in, dwt, y.K, y.N, y.dWk, y.ldw, y.dW, y.ldw, 1, side);
+      if (!after(aux_s, side_s, 68 + l)) return ARD_ERR_CUDA;
+      st = ard_expand_weight_grad_cols(ctx, y.pat, in, dwt, y.K, y.N, y.dWk, y.ldw, y.dW, y.ldw, 1, aux);
       if (st != ARD_OK) return st;
     }
     if (y.db) {
-      st = ard_bias_grad(ctx, y.pat, dt, B, y.N, dZ, lddz, dz_compact, y.db, 1, side);
+      if (two && l < n_layers - 1 && cudaStreamWaitEvent(aux_s, ctx->ev[35 + l], 0) != cudaSuccess) return ARD_ERR_CUDA;
+      st = ard_bias_grad(ctx, y.pat, dt, B, y.N, dZ, lddz, dz_compact, y.db, 1, aux);
       if (st != ARD_OK) return st;
     }
     if (l > 0) {
@@ -140,5 +151,6 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
     }
   }
   if (!after(main_s, side_s, 2)) return ARD_ERR_CUDA;  // join
+  if (!after(main_s, aux_s, 67)) return ARD_ERR_CUDA;
   return ARD_OK;
 }
