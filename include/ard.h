@@ -293,8 +293,13 @@ ard_status ard_sample_pattern_counter(ard_ctx* ctx, ard_pattern* pat, int dist_i
  * and columns zero), layers[l].db if not NULL, dX [B][K_0] if not NULL; A and dZ of every layer hold what
  * the step computed.  `layers` is a HOST array; all pointers inside are DEVICE pointers owned by the caller;
  * dimensions must satisfy the alignment rules of ard_fwd or the slower CUDA-core kernels run.  Enqueues
- * only; allocates nothing once every buffer has been seen once (descriptor tables), so it can be
- * captured into a CUDA graph after one ordinary call. */
+ * only; allocates nothing once every buffer has been seen once (descriptor tables, two internal streams
+ * and their events), so it can be captured into a CUDA graph after one ordinary call.  When every hidden
+ * layer has compact_out != 0 the weight compactions, weight gradients, gradient expansions and bias
+ * gradients are enqueued on two streams owned by the context, forked from `cuda_stream` after the patterns
+ * are drawn and joined back into it before the call returns: to the caller (and to a capture) all work of
+ * the call is ordered on `cuda_stream`, but the buffers of `layers` must not be touched by other streams
+ * while the iteration runs. */
 typedef struct ard_mlp_layer {
   int K, N;          /* fan-in and neurons; K of layer l+1 == N of layer l                                  */
   ard_pattern* pat;  /* row pattern over the N neurons (created with K_dim = K, N_dim = N)                  */
