@@ -161,6 +161,27 @@ ard_status tc_eligible(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, in
 
 }  // namespace
 
+bool ard_side_streams(ard_ctx* ctx, cudaStream_t main) {
+  if (ctx->n_ev == ARD_MLP_EVENTS && ctx->side_stream && ctx->aux_stream) return true;
+  if (ctx->n_ev != 0) return false;  // an earlier attempt failed half way
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(main, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return false;
+  DeviceGuard guard(ctx->device);
+  if (cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking) != cudaSuccess) {
+    ctx->side_stream = nullptr;
+    return false;
+  }
+  if (cudaStreamCreateWithFlags(&ctx->aux_stream, cudaStreamNonBlocking) != cudaSuccess) {
+    ctx->aux_stream = nullptr;
+    return false;
+  }
+  for (int i = 0; i < ARD_MLP_EVENTS; ++i) {
+    if (cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) != cudaSuccess) return false;
+    ctx->n_ev = i + 1;
+  }
+  return true;
+}
+
 extern "C" {
 
 const char* ard_status_string(ard_status s) {

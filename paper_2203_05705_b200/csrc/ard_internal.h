@@ -111,6 +111,10 @@ static inline size_t sk_cnt_bytes(int sm_count) { return (size_t)sm_count * 8 * 
 
 static inline int map_index_count(int dp_bound) { return dp_bound * (dp_bound + 1) / 2; }
 
+// Creates the context's second and third stream and their events on first use; false if they do not exist
+// and cannot be created now (`main` is being captured into a graph: nothing may be created then).
+bool ard_side_streams(ard_ctx* ctx, cudaStream_t main);
+
 // ---- launchers implemented in the .cu files -----------------------------------------------------
 ard_status launch_sampler(ard_ctx* ctx, ard_pattern* pat, const unsigned long long* d_cdf, int ndp,
                           uint64_t seed, uint64_t iteration, uint32_t stream_id, int forced_dp, int forced_b,

@@ -6,18 +6,6 @@
 // into a CUDA graph once its descriptor tables exist (run it once before capturing).
 #include "ard_internal.h"
 
-namespace {
-struct DeviceGuardLite {
-  int prev = -1;
-  bool switched = false;
-  explicit DeviceGuardLite(int dev) {
-    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
-  }
-  ~DeviceGuardLite() {
-    if (switched) cudaSetDevice(prev);
-  }
-};
-}  // namespace
 
 extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, int n_layers, int B, const void* X,
                                    int ldx, const void* dOut, int lddout, void* dX, int lddx, int dist_id,
@@ -45,27 +33,7 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
   // full-width form gathers through the context workspace, which the two streams would share.
   bool two = ctx->mlp_two_streams && n_layers >= 2 && n_layers <= 32;
   for (int l = 0; l + 1 < n_layers && two; ++l) two = layers[l].compact_out != 0;
-  if (two && ctx->n_ev == 0) {
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(main_s, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
-      two = false;  // first use inside a capture: nothing may be created now
-    } else {
-      DeviceGuardLite guard(ctx->device);
-      if (cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking) != cudaSuccess) {
-        ctx->side_stream = nullptr;
-        two = false;
-      }
-      if (two && cudaStreamCreateWithFlags(&ctx->aux_stream, cudaStreamNonBlocking) != cudaSuccess) {
-        ctx->aux_stream = nullptr;
-        two = false;
-      }
-      for (int i = 0; two && i < ARD_MLP_EVENTS; ++i) {
-        if (cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) != cudaSuccess) two = false;
-        else ctx->n_ev = i + 1;
-      }
-    }
-  }
-  if (two && ctx->n_ev < ARD_MLP_EVENTS) two = false;
+  if (two && !ard_side_streams(ctx, main_s)) two = false;
   cudaStream_t side_s = two ? ctx->side_stream : main_s;
   cudaStream_t aux_s = two ? ctx->aux_stream : main_s;
   void* side = (void*)side_s;
