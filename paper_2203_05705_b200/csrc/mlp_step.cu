@@ -91,7 +91,10 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
     const int dz_compact = (l == n_layers - 1) ? 0 : (y.compact_out ? 1 : 0);
     const ard_dtype dwt = y.dW_is_f32 ? ARD_F32 : ARD_BF16;
     // the expansion writes every entry of dW, so the compact gradient needs no zeros of its own
-    // weight side (second stream when there are two): needs dZ of this layer, which the layer above wrote
+    // weight side (second stream when there are two): needs dZ of this layer, which the layer above wrote.
+    // (The last layer's dOut is full width: if its pattern is not dense, both its backward products compact
+    // it into the context workspace, each on its own stream; they write the same values from the same
+    // source, so the overlap is harmless.)
     if (two && l < n_layers - 1 && cudaStreamWaitEvent(side_s, ctx->ev[35 + l], 0) != cudaSuccess) return ARD_ERR_CUDA;
     st = ard_layer_bwd_weight(ctx, y.pat, in, dt, dwt, B, y.K, y.N, 1.0f, in_act, ld_in, dZ, lddz, dz_compact,
                               in ? y.dWk : y.dW, y.ldw, in ? 0 : 1, side);
