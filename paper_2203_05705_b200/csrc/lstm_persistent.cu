@@ -589,25 +589,44 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
         if (*abort_flag) { ok = false; break; }
       }
       // ---- phase B: total gradient of h_t, cell adjoint, dz_t ----
+      // All loads of all owned (row, unit) pairs are issued before the first is consumed: the partial sums
+      // come from L2 and a chain of dependent round trips would cost more than the whole product.
+      float recs[LB_PAIRS_MAX], ups[LB_PAIRS_MAX];
+#pragma unroll
+      for (int i = 0; i < LB_PAIRS_MAX; ++i) {
+        recs[i] = 0.f;
+        ups[i] = 0.f;
+        if (jj[i] < 0) continue;
+        const int q = tid + i * LB_MATH;
+        const int row = q >> 3, cc = r_idx * LB_OWN + (q & 7), u = c0 + cc;
+        float part[LB_KPARTS];
+#pragma unroll
+        for (int rp = 0; rp < LB_KPARTS; ++rp)
+          part[rp] = (k >= 1 && rp < parts) ? __ldcg(slice_partial + ((size_t)rp * 128 + row) * LB_COLS + cc) : 0.f;
+        if (t >= 0)
+          ups[i] = (t == T - 1) ? p.dH_last[(size_t)row * p.H + u]
+                                : __ldcg(p.D + ((size_t)(t + 1) * p.B + row) * ldd + p.I + u);
+        float rec = 0.f;
+#pragma unroll
+        for (int rp = 0; rp < LB_KPARTS; ++rp) rec += part[rp];  // fixed order: same bits every launch
+        recs[i] = rec;
+      }
 #pragma unroll
       for (int i = 0; i < LB_PAIRS_MAX; ++i) {
         if (jj[i] < 0) continue;
         const int q = tid + i * LB_MATH;
         const int row = q >> 3, cc = r_idx * LB_OWN + (q & 7), u = c0 + cc, j = jj[i];
-        float rec = 0.f;
-        if (k >= 1)
-          for (int rp = 0; rp < parts; ++rp) rec += __ldcg(slice_partial + ((size_t)rp * 128 + row) * LB_COLS + cc);
+        const float rec = recs[i];
         if (t < 0) {  // gradient of h_0: added to what the caller left in the h half of D[0]
           p.D[(size_t)row * ldd + p.I + u] += rec;
           continue;
         }
         float dh;
         if (t == T - 1) {
-          dh = p.dH_last[(size_t)row * p.H + u];
+          dh = ups[i];
         } else {
-          float* up = p.D + ((size_t)(t + 1) * p.B + row) * ldd + p.I + u;  // upstream gradient of h_t
-          dh = *up + rec;
-          *up = dh;
+          dh = ups[i] + rec;  // upstream gradient of h_t plus the recurrent part
+          p.D[((size_t)(t + 1) * p.B + row) * ldd + p.I + u] = dh;
         }
         const float gi = pg[i][0], gf = pg[i][1], gg = pg[i][2], go = pg[i][3];
         const float cp = pg[i][4];
