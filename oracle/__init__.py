@@ -18,6 +18,9 @@ Pins (each lives in tests/test_oracle_*.py):
   mlp_chain.*              finite differences of the scalar <dZ3, Z3>
   mlp.*                    torch autograd (fp64) on the same network written with library ops; central
                            differences; == mlp_chain without bias; compact-matrix form == masked full width
+  cnn.*                    decisions that do not depend on the sample; binomial law of the region decision;
+                           drop rates of the row sampler; worked row example of Sec. 5.2.1; masked product ==
+                           product of the dense small matrix; brute force; adjoint identities
   search.*                 gradient vs central differences; stationary points lie in the Gibbs family
                            ln k_i = beta (i-1)/i + c with beta = -2 (k.p_u - p)/lambda; small-lambda limit ==
                            the maximum-entropy distribution at rate p; Eq. 2-3 in exact rationals
@@ -25,6 +28,7 @@ Pins (each lives in tests/test_oracle_*.py):
 Parity unpinned (the paper fixes no value to compare with): the constants of the
 distribution search (the body of Algorithm 1 is not printed: loss form, lambda, step size, start and
 stopping rule are a reading, see search.py) and therefore the authors' own K, the tile
-linearisation order beyond the first tile of the worked example, the LSTM
+linearisation order beyond the first tile of the worked example, every constant of the
+sensitivity prediction (region shape, which values are sampled, k, t, threshold, m, n: see cnn.py), the LSTM
 reading (which units are dropped, gate order) and the rescale convention.
 """

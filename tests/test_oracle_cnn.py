@@ -1,0 +1,93 @@
+"""Pins for oracle/cnn.py (sensitivity prediction and row-based sensitivity-aware dropout, Sec. 5.1 / 5.2.1).
+
+The paper fixes no numbers for this part, so the pins are what the mathematics fixes: the decision rule on
+regions whose answer does not depend on the sample (all values above / below the threshold), the binomial law
+of the decision for a region with a known fraction above the threshold, the drop rate of the row sampler, the
+worked row example of Sec. 5.2.1, the equality of the masked product with the product of the dense small
+matrix, brute-force loops and the adjoint identities.
+"""
+import numpy as np
+import pytest
+from scipy import stats
+
+from oracle import cnn as C
+
+
+def test_regions_that_do_not_depend_on_the_sample():
+    A = np.zeros((12, 40))
+    A[0:4] = 1.0                       # region 0 (x = 4): every value above the threshold
+    A[8:12, ::2] = 1.0                 # region 2: exactly half of the values above
+    for it in range(5):
+        s0, c0, n0 = C.region_sensitive(A, 0, 4, 0.3, 0.5, 0.5, 7, it, 3)
+        s1, c1, n1 = C.region_sensitive(A, 1, 4, 0.3, 0.5, 0.5, 7, it, 3)
+        assert s0 and c0 == n0 == C.n_samples(0.3, 4, 40) == 48
+        assert (not s1) and c1 == 0
+    P, sens = C.sensitivity_mask(A, 4, 0.3, 0.5, 0.5, 0.2, 0.8, 7, 0, 3)
+    assert sens[0] and not sens[1]
+    assert P[0] == C.quantise_probability(0.2) and P[1] == C.quantise_probability(0.8)
+
+
+def test_ragged_last_region_counts_missing_rows_as_below():
+    A = np.ones((5, 16))               # x = 4: region 1 has one real row of four
+    fr = []
+    for it in range(200):
+        _, c, s = C.region_sensitive(A, 1, 4, 0.5, 0.5, 0.5, 1, it, 0)
+        fr.append(c / s)
+    assert abs(np.mean(fr) - 0.25) < 0.02          # a quarter of the positions exist
+
+
+def test_decision_follows_the_binomial_law():
+    rng = np.random.default_rng(0)
+    x, Kc, f = 2, 64, 0.45
+    A = (rng.random((x, Kc)) < f).astype(np.float64)
+    frac = A.mean()
+    s = C.n_samples(0.25, x, Kc)
+    need = C.needed(0.5, s)
+    hits = sum(C.region_sensitive(A, 0, x, 0.25, 0.5, 0.5, 11, it, 0)[0] for it in range(1500))
+    p_theory = stats.binom.sf(need - 1, s, frac)
+    sd = np.sqrt(p_theory * (1 - p_theory) / 1500)
+    assert abs(hits / 1500 - p_theory) < 4 * sd + 1e-3
+
+
+def test_row_sampler_rates_and_extremes():
+    M, x = 4000, 8
+    P = np.array([C.quantise_probability(0.2), C.quantise_probability(0.8)] * (M // x // 2), dtype=np.uint64)
+    keep = C.draw_rows(P, x, M, 5, 9, 2)
+    m = C.row_mask(M, keep).reshape(-1, x)
+    low, high = 1 - m[0::2].mean(), 1 - m[1::2].mean()
+    assert abs(low - 0.2) < 4 * np.sqrt(0.2 * 0.8 / (M / 2)) and abs(high - 0.8) < 4 * np.sqrt(0.2 * 0.8 / (M / 2))
+    assert np.all(np.diff(keep) > 0)
+    assert len(C.draw_rows(np.zeros(M // x, dtype=np.uint64), x, M, 5, 9, 2)) == M      # probability 0: nothing dropped
+    assert len(C.draw_rows(np.full(M // x, C.quantise_probability(1.0), dtype=np.uint64), x, M, 5, 9, 2)) <= 1
+    # a pure function of (seed, iteration, stream): same draw twice, different draw for another iteration
+    assert np.array_equal(keep, C.draw_rows(P, x, M, 5, 9, 2))
+    assert not np.array_equal(keep, C.draw_rows(P, x, M, 5, 10, 2))
+
+
+def test_worked_row_example_and_the_dense_small_matrix():
+    """Sec. 5.2.1: six rows, the second, fifth and sixth dropped; the kept rows fill the same rows of Y."""
+    rng = np.random.default_rng(3)
+    A, W = rng.standard_normal((6, 9)), rng.standard_normal((9, 4))
+    keep = np.array([0, 2, 3])
+    Y = C.fwd(A, W, keep, 1.5)
+    assert np.all(Y[[1, 4, 5]] == 0)
+    np.testing.assert_allclose(Y[keep], 1.5 * A[keep] @ W, rtol=1e-13)
+    np.testing.assert_allclose(Y, C.fwd_compact(A, W, keep, 1.5), rtol=1e-13, atol=1e-15)
+    # brute force
+    for r in range(6):
+        for n in range(4):
+            ref = 1.5 * sum(A[r, k] * W[k, n] for k in range(9)) if r in keep else 0.0
+            assert abs(Y[r, n] - ref) < 1e-12
+
+
+def test_backward_products_are_the_adjoints():
+    rng = np.random.default_rng(4)
+    M, Kc, N = 17, 11, 7
+    A, W, dY = rng.standard_normal((M, Kc)), rng.standard_normal((Kc, N)), rng.standard_normal((M, N))
+    keep = np.array([1, 2, 5, 9, 16])
+    lhs = float((C.fwd(A, W, keep, 1.3) * dY).sum())
+    assert abs(lhs - float((A * C.bwd_data(dY, W, keep, 1.3)).sum())) < 1e-10
+    assert abs(lhs - float((W * C.bwd_weight(A, dY, keep, 1.3)).sum())) < 1e-10
+    dropped = np.setdiff1d(np.arange(M), keep)
+    assert np.all(C.bwd_data(dY, W, keep)[dropped] == 0)
+    np.testing.assert_allclose(C.bwd_weight(A, dY, keep, 1.0), A[keep].T @ dY[keep], rtol=1e-12, atol=1e-13)
