@@ -43,6 +43,7 @@ extern "C" {
 
 typedef struct ard_ctx ard_ctx;         /* owns distributions, workspace, descriptor cache, status word */
 typedef struct ard_pattern ard_pattern; /* handle of a device-resident pattern (header + index lists)   */
+typedef struct ard_rows ard_rows;       /* handle of a device-resident list of kept input-matrix rows   */
 
 typedef enum {
   ARD_OK = 0,
@@ -322,6 +323,38 @@ typedef struct ard_mlp_layer {
 ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, int n_layers, int B, const void* X, int ldx,
                         const void* dOut, int lddout, void* dX, int lddx, int dist_id, uint64_t seed,
                         uint64_t iteration_base, uint64_t* iteration_counter, void* cuda_stream);
+
+/* ---- row-based sensitivity-aware dropout of a convolution layer's input matrix (Sec. 5.1, 5.2.1) ----
+ * The layer is the product Y = A W of its input matrix A [M][Kc] (im2col of the input feature map: M
+ * output positions, Kc = C*k*k; making A is a library routine outside this interface) with the filters
+ * W [N][Kc] (neuron-major as everywhere here).  Sec. 5.1 predicts per region of A whether it is sensitive
+ * and gives it a low (sensitive) or a high dropout probability; Sec. 5.2.1 draws, per iteration, which rows
+ * of A are dropped, multiplies only the kept rows and fills the results back into the same rows of Y.
+ * The paper fixes neither the region shape nor which values are sampled nor any constant; this library's
+ * reading: regions of `region_rows` consecutive rows by the whole width; sample d of region g is word
+ * (d mod 4) of the Philox4x32-10 block with key (seed) and counter (iteration low, iteration high, g,
+ * stream_id * 65536 + d div 4), at position floor(word * region_rows*Kc / 2^32) of the region (row-major;
+ * positions below the last row of A count as not exceeding); s = max(1, floor(k_frac*region_rows*Kc + 1/2))
+ * samples; sensitive iff at least max(1, ceil(t_frac * s)) sampled values are > threshold; a probability p
+ * is the integer min(floor(p 2^32), 2^32 - 1); row r is dropped iff word 0 of the block with counter
+ * (iteration low, iteration high, r, stream_id * 65536 + 65535) is below its region's integer.
+ * stream_id < 65536.  Everything stays on the device; ard_rows_to_host is for tests. */
+ard_status ard_rows_create(ard_ctx* ctx, ard_rows** rows, int M, int region_rows);
+ard_status ard_rows_destroy(ard_rows* rows);
+/* Sec. 5.1: writes the dropout probability of every region (m_prob if sensitive, else n_prob).
+ * A [M][Kc] (lda) of element type dtype.  Asynchronous. */
+ard_status ard_sensitivity_predict(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc,
+                                   double k_frac, double t_frac, float threshold, double m_prob, double n_prob,
+                                   uint64_t seed, uint64_t iteration, uint32_t stream_id, void* cuda_stream);
+/* The same probability for every region (tests; p = 0 keeps every row).  Asynchronous. */
+ard_status ard_rows_set_probability(ard_ctx* ctx, ard_rows* rows, double p, void* cuda_stream);
+/* Sec. 5.2.1: draws the dropped rows and writes the ascending list of kept rows.  Asynchronous. */
+ard_status ard_rows_sample(ard_ctx* ctx, ard_rows* rows, uint64_t seed, uint64_t iteration, uint32_t stream_id,
+                           void* cuda_stream);
+/* Test / debug: synchronises; n_keep, the kept rows (at most idx_capacity) and the per-region integers
+ * (ceil(M / region_rows) entries) to HOST buffers; idx and region_probability may be NULL. */
+ard_status ard_rows_to_host(const ard_rows* rows, int32_t* n_keep, int32_t* idx, size_t idx_capacity,
+                            uint32_t* region_probability, void* cuda_stream);
 
 /* ---- LSTM cell on the kept hidden units (Sec. 7: an LSTM step is again a matrix
  * product; one row pattern over the H hidden units serves every time step) -------------

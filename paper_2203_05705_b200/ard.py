@@ -33,6 +33,8 @@ EXPORTS = [
     "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_set_lstm_persistent", "ard_lstm_forward", "ard_lstm_backward", "ard_last_device_status", "ard_status_string", "ard_launch_count",
     "ard_layer_fwd", "ard_layer_bwd_data", "ard_layer_bwd_weight", "ard_compact_weight_cols",
     "ard_expand_weight_grad_cols", "ard_bias_grad", "ard_sample_pattern_counter", "ard_mlp_step",
+    "ard_rows_create", "ard_rows_destroy", "ard_sensitivity_predict", "ard_rows_set_probability", "ard_rows_sample",
+    "ard_rows_to_host",
 ]
 
 _lib = None
@@ -101,6 +103,13 @@ def lib():
         "ard_bias_grad": [vp, vp, i32, i32, i32, vp, i32, i32, vp, i32, vp],
         "ard_sample_pattern_counter": [vp, vp, i32, u64, u64, vp, i32, u32, vp],
         "ard_mlp_step": [vp, P(MlpLayer), i32, i32, vp, i32, vp, i32, vp, i32, i32, u64, u64, vp, vp],
+        "ard_rows_create": [vp, P(vp), i32, i32],
+        "ard_rows_destroy": [vp],
+        "ard_sensitivity_predict": [vp, vp, i32, vp, i32, i32, C.c_double, C.c_double, f32, C.c_double, C.c_double, u64, u64,
+                                    u32, vp],
+        "ard_rows_set_probability": [vp, vp, C.c_double, vp],
+        "ard_rows_sample": [vp, vp, u64, u64, u32, vp],
+        "ard_rows_to_host": [vp, P(C.c_int32), P(C.c_int32), sz, P(C.c_uint32), vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -326,6 +335,41 @@ def ard_mlp_step(ctx, layers, n_layers, B, X, ldx, dOut, lddout, dX, lddx, dist_
     """`layers`: the array made by mlp_layers()."""
     _check(lib().ard_mlp_step(ctx, layers, n_layers, B, _ptr(X), ldx, _ptr(dOut), lddout, _ptr(dX), lddx, dist_id,
                               seed, iteration_base, _ptr(iteration_counter), _stream(stream)), "ard_mlp_step")
+
+
+def ard_rows_create(ctx, M, region_rows):
+    h = C.c_void_p()
+    _check(lib().ard_rows_create(ctx, C.byref(h), M, region_rows), "ard_rows_create")
+    return h
+
+
+def ard_rows_destroy(rows):
+    _check(lib().ard_rows_destroy(rows), "ard_rows_destroy")
+
+
+def ard_sensitivity_predict(ctx, rows, dtype, A, lda, Kc, k_frac, t_frac, threshold, m_prob, n_prob, seed, iteration,
+                            stream_id, stream=None):
+    _check(lib().ard_sensitivity_predict(ctx, rows, dtype, _ptr(A), lda, Kc, k_frac, t_frac, threshold, m_prob, n_prob,
+                                         seed, iteration, stream_id, _stream(stream)), "ard_sensitivity_predict")
+
+
+def ard_rows_set_probability(ctx, rows, p, stream=None):
+    _check(lib().ard_rows_set_probability(ctx, rows, p, _stream(stream)), "ard_rows_set_probability")
+
+
+def ard_rows_sample(ctx, rows, seed, iteration, stream_id, stream=None):
+    _check(lib().ard_rows_sample(ctx, rows, seed, iteration, stream_id, _stream(stream)), "ard_rows_sample")
+
+
+def ard_rows_to_host(rows, M, regions=0, stream=None):
+    """Returns (n_keep, kept rows, per-region integers or None)."""
+    nk = C.c_int32()
+    idx = np.zeros(max(M, 1), dtype=np.int32)
+    P = np.zeros(regions, dtype=np.uint32) if regions else None
+    _check(lib().ard_rows_to_host(rows, C.byref(nk), idx.ctypes.data_as(C.POINTER(C.c_int32)), M,
+                                  P.ctypes.data_as(C.POINTER(C.c_uint32)) if regions else None, _stream(stream)),
+           "ard_rows_to_host")
+    return nk.value, idx[:nk.value].copy(), P
 
 
 def ard_lstm_gate_gemm(ctx, pat, B, KH, H, XH, ldxh, W, ldw, Z, ldz_gate, stream=None):

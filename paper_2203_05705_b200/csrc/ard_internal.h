@@ -39,6 +39,17 @@ struct ard_pattern {
   int32_t* d_row_idx;  // tile only: [units]
 };
 
+// Device-resident list of the kept rows of an input matrix with M rows (Sec. 5.2.1) and the per-region
+// dropout probabilities it is drawn from (Sec. 5.1).  d_hdr mimics a pattern header (dp = b = 1, n_keep).
+struct ard_rows {
+  ard_ctx* ctx;
+  int M, x, regions;
+  int32_t* d_hdr;    // HDR_WORDS
+  int32_t* d_idx;    // kept rows, ascending, capacity M
+  uint8_t* d_flag;   // 1 = kept, per row
+  uint32_t* d_P;     // per region: dropped iff the row's random word is below this
+};
+
 struct ArdDistribution {
   int ndp = 0;
   unsigned long long* d_cdf = nullptr;  // device: ndp entries
@@ -186,6 +197,16 @@ ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,
                               void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, int skip_dense,
                               cudaStream_t s);
+
+// Sensitivity-aware row dropout (rows.cu).
+ard_status launch_sensitivity(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc, int samples,
+                              int need, float threshold, uint32_t P_sens, uint32_t P_insens, uint64_t seed,
+                              uint64_t iteration, uint32_t stream_id, cudaStream_t s);
+ard_status launch_fill_probability(ard_ctx* ctx, ard_rows* rows, uint32_t P, cudaStream_t s);
+ard_status launch_rows_sample(ard_ctx* ctx, ard_rows* rows, uint64_t seed, uint64_t iteration, uint32_t stream_id,
+                              cudaStream_t s);
+ard_status launch_zero_dropped_rows(ard_ctx* ctx, const ard_rows* rows, void* out, int ld_bytes, int row_bytes,
+                                    cudaStream_t s);
 
 // Layer-step helpers (aux_kernels.cu); elem_bytes 2 or 4.
 ard_status launch_compact_weight_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* hdr_in, const void* W, int ldw,

@@ -1,0 +1,305 @@
+// Row-based sensitivity-aware dropout of a convolution layer's input matrix (Sec. 5.1, Sec. 5.2.1):
+// sensitivity prediction per region, one Bernoulli draw per row, compaction of the kept rows into a
+// device-resident list.  Nothing returns to the host; the products that follow read the list.
+#include "ard_internal.h"
+
+namespace {
+
+__device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+  const uint32_t hi0 = __umulhi(M0, c[0]), lo0 = M0 * c[0];
+  const uint32_t hi1 = __umulhi(M1, c[2]), lo1 = M1 * c[2];
+  const uint32_t n0 = hi1 ^ c[1] ^ k0, n2 = hi0 ^ c[3] ^ k1;
+  c[0] = n0;
+  c[1] = lo1;
+  c[2] = n2;
+  c[3] = lo0;
+}
+
+__device__ __forceinline__ void philox4x32_10(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    philox_round(c, k0, k1);
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+}
+
+template <typename T> __device__ __forceinline__ float val_f(T v);
+template <> __device__ __forceinline__ float val_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float val_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Sec. 5.1, steps 2-4.  One warp per region of x rows by the whole width: lane l draws the Philox blocks
+// l, l + 32, ... (four samples each), looks the sampled entries up and counts those above the threshold.
+template <typename T>
+__global__ void __launch_bounds__(256) sensitivity_kernel(const T* A, int lda, int M, int Kc, int x, int regions,
+                                                          int samples, int need, float threshold, uint32_t P_sens,
+                                                          uint32_t P_insens, unsigned long long seed,
+                                                          unsigned long long iteration, uint32_t stream_id,
+                                                          uint32_t* P_region) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int lane = threadIdx.x & 31;
+  const int g = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (g >= regions) return;
+  const unsigned long long size = (unsigned long long)x * (unsigned long long)Kc;
+  const int blocks = (samples + 3) >> 2;
+  int count = 0;
+  for (int q = lane; q < blocks; q += 32) {
+    uint32_t c[4] = {(uint32_t)iteration, (uint32_t)(iteration >> 32), (uint32_t)g, (stream_id << 16) | (uint32_t)q};
+    philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      if (4 * q + w >= samples) break;
+      const unsigned long long pos = ((unsigned long long)c[w] * size) >> 32;
+      const long long row = (long long)g * x + (long long)(pos / (unsigned long long)Kc);
+      const int col = (int)(pos % (unsigned long long)Kc);
+      if (row < M && val_f<T>(A[(size_t)row * lda + col]) > threshold) ++count;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) count += __shfl_xor_sync(0xffffffffu, count, o);
+  if (lane == 0) P_region[g] = count >= need ? P_sens : P_insens;
+}
+
+__global__ void __launch_bounds__(256) fill_probability_kernel(uint32_t* P_region, int regions, uint32_t P) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  for (int g = blockIdx.x * 256 + threadIdx.x; g < regions; g += gridDim.x * 256) P_region[g] = P;
+}
+
+// Sec. 5.2.1: row r is dropped iff its Philox word is below the probability of its region.  One CTA: every
+// thread draws a contiguous run of rows, the CTA scans the kept counts and every thread then writes the
+// kept rows of its run, so the list comes out ascending.  hdr mimics a pattern header (dp = b = 1).
+constexpr int ROWS_THREADS = 1024;
+
+__global__ void __launch_bounds__(ROWS_THREADS) rows_sample_kernel(int32_t* hdr, int32_t* idx, uint8_t* kept_flag,
+                                                                   const uint32_t* P_region, int M, int x,
+                                                                   unsigned long long seed, unsigned long long iteration,
+                                                                   uint32_t stream_id) {
+  __shared__ int s_warp[32];
+  __shared__ int s_total;
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per = (M + ROWS_THREADS - 1) / ROWS_THREADS;
+  const int r0 = tid * per, r1 = min(M, r0 + per);
+  int mine = 0;
+  for (int r = r0; r < r1; ++r) {
+    uint32_t c[4] = {(uint32_t)iteration, (uint32_t)(iteration >> 32), (uint32_t)r, (stream_id << 16) | 0xFFFFu};
+    philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+    const bool keep = !(c[0] < P_region[r / x]);
+    kept_flag[r] = keep ? 1 : 0;
+    mine += keep ? 1 : 0;
+  }
+  // exclusive scan of `mine` over the CTA
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int v = s_warp[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, v, o);
+      if (lane >= o) v += u;
+    }
+    s_warp[lane] = v;  // inclusive over warps
+    if (lane == 31) s_total = v;
+  }
+  __syncthreads();
+  int out = incl - mine + (warp > 0 ? s_warp[warp - 1] : 0);
+  for (int r = r0; r < r1; ++r)
+    if (kept_flag[r]) idx[out++] = r;
+  if (tid == 0) {
+    hdr[HDR_KIND] = 2;
+    hdr[HDR_DP] = 1;
+    hdr[HDR_B] = 1;
+    hdr[HDR_NKEEP] = s_total;
+    hdr[HDR_UNITS] = M;
+    hdr[HDR_TR] = 0;
+    hdr[HDR_TC] = 0;
+    hdr[HDR_TS] = 0;
+    hdr[HDR_MAPIDX] = 0;
+  }
+}
+
+// Dropped rows of an output matrix are zero (Sec. 5.2.1: only the kept rows are filled back).
+__global__ void __launch_bounds__(256) zero_dropped_rows_kernel(const uint8_t* kept_flag, int M, void* out, int ld_bytes,
+                                                                int row_bytes) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  for (int r = blockIdx.x; r < M; r += gridDim.x) {
+    if (kept_flag[r]) continue;
+    char* row = reinterpret_cast<char*>(out) + (size_t)r * ld_bytes;
+    if ((row_bytes & 15) == 0 && (ld_bytes & 15) == 0 && (reinterpret_cast<uintptr_t>(out) & 15) == 0) {
+      for (int o = threadIdx.x * 16; o < row_bytes; o += 256 * 16) *reinterpret_cast<uint4*>(row + o) = make_uint4(0, 0, 0, 0);
+    } else {
+      for (int o = threadIdx.x * 2; o < row_bytes; o += 256 * 2) *reinterpret_cast<uint16_t*>(row + o) = 0;
+    }
+  }
+}
+
+}  // namespace
+
+ard_status launch_sensitivity(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc, int samples,
+                              int need, float threshold, uint32_t P_sens, uint32_t P_insens, uint64_t seed,
+                              uint64_t iteration, uint32_t stream_id, cudaStream_t s) {
+  const int regions = rows->regions;
+  dim3 grid((regions + 7) / 8);
+  if (dtype == ARD_F32)
+    ARD_CUDA_OK(ard_launch(ctx, sensitivity_kernel<float>, grid, dim3(256), 0, s, (const float*)A, lda, rows->M, Kc, rows->x,
+                           regions, samples, need, threshold, P_sens, P_insens, (unsigned long long)seed,
+                           (unsigned long long)iteration, stream_id, rows->d_P));
+  else
+    ARD_CUDA_OK(ard_launch(ctx, sensitivity_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, (const __nv_bfloat16*)A, lda,
+                           rows->M, Kc, rows->x, regions, samples, need, threshold, P_sens, P_insens,
+                           (unsigned long long)seed, (unsigned long long)iteration, stream_id, rows->d_P));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+ard_status launch_fill_probability(ard_ctx* ctx, ard_rows* rows, uint32_t P, cudaStream_t s) {
+  ARD_CUDA_OK(ard_launch(ctx, fill_probability_kernel, dim3((rows->regions + 255) / 256), dim3(256), 0, s, rows->d_P,
+                         rows->regions, P));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+ard_status launch_rows_sample(ard_ctx* ctx, ard_rows* rows, uint64_t seed, uint64_t iteration, uint32_t stream_id,
+                              cudaStream_t s) {
+  ARD_CUDA_OK(ard_launch(ctx, rows_sample_kernel, dim3(1), dim3(ROWS_THREADS), 0, s, rows->d_hdr, rows->d_idx, rows->d_flag,
+                         (const uint32_t*)rows->d_P, rows->M, rows->x, (unsigned long long)seed,
+                         (unsigned long long)iteration, stream_id));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+ard_status launch_zero_dropped_rows(ard_ctx* ctx, const ard_rows* rows, void* out, int ld_bytes, int row_bytes,
+                                    cudaStream_t s) {
+  if (rows->M == 0 || row_bytes == 0) return ARD_OK;
+  const int grid = rows->M < ctx->sm_count * 16 ? rows->M : ctx->sm_count * 16;
+  ARD_CUDA_OK(ard_launch(ctx, zero_dropped_rows_kernel, dim3(grid), dim3(256), 0, s, (const uint8_t*)rows->d_flag, rows->M,
+                         out, ld_bytes, row_bytes));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+// ---- C ABI -----------------------------------------------------------------------------------------
+namespace {
+struct DevGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DevGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DevGuard() {
+    if (switched) cudaSetDevice(prev);
+  }
+};
+
+uint32_t quantise_probability(double p) {
+  const double v = floor(p * 4294967296.0);
+  return v >= 4294967295.0 ? 4294967295u : (uint32_t)v;
+}
+}  // namespace
+
+extern "C" {
+
+ard_status ard_rows_create(ard_ctx* ctx, ard_rows** out, int M, int region_rows) {
+  if (!ctx || !out || M < 1 || region_rows < 1) return ARD_ERR_INVALID_ARG;
+  *out = nullptr;
+  DevGuard guard(ctx->device);
+  ard_rows* r = new (std::nothrow) ard_rows();
+  if (!r) return ARD_ERR_NOMEM;
+  r->ctx = ctx;
+  r->M = M;
+  r->x = region_rows;
+  r->regions = (M + region_rows - 1) / region_rows;
+  r->d_hdr = nullptr; r->d_idx = nullptr; r->d_flag = nullptr; r->d_P = nullptr;
+  // one allocation: header | kept list (padded to 64 entries: the products read whole 64-row blocks of it) | P | flags
+  const size_t n_idx = ((size_t)M + 63) / 64 * 64 + 64;
+  const size_t bytes = sizeof(int32_t) * (HDR_WORDS + n_idx) + sizeof(uint32_t) * r->regions + (size_t)M;
+  char* base = nullptr;
+  if (cudaMalloc(reinterpret_cast<void**>(&base), bytes) != cudaSuccess) {
+    delete r;
+    return ARD_ERR_NOMEM;
+  }
+  cudaMemset(base, 0, bytes);
+  r->d_hdr = reinterpret_cast<int32_t*>(base);
+  r->d_idx = r->d_hdr + HDR_WORDS;
+  r->d_P = reinterpret_cast<uint32_t*>(r->d_idx + n_idx);
+  r->d_flag = reinterpret_cast<uint8_t*>(r->d_P + r->regions);
+  *out = r;
+  return ARD_OK;
+}
+
+ard_status ard_rows_destroy(ard_rows* rows) {
+  if (!rows) return ARD_ERR_INVALID_ARG;
+  DevGuard guard(rows->ctx->device);
+  cudaDeviceSynchronize();
+  cudaFree(rows->d_hdr);
+  delete rows;
+  return ARD_OK;
+}
+
+ard_status ard_sensitivity_predict(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc,
+                                   double k_frac, double t_frac, float threshold, double m_prob, double n_prob,
+                                   uint64_t seed, uint64_t iteration, uint32_t stream_id, void* cuda_stream) {
+  if (!ctx || !rows || rows->ctx != ctx || !A) return ARD_ERR_INVALID_ARG;
+  if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (Kc < 1 || lda < Kc) return ARD_ERR_SHAPE;
+  if (!(k_frac > 0.0 && k_frac <= 1.0) || !(t_frac >= 0.0 && t_frac <= 1.0)) return ARD_ERR_INVALID_ARG;
+  if (!(m_prob >= 0.0 && m_prob <= 1.0) || !(n_prob >= 0.0 && n_prob <= 1.0) || stream_id > 0xFFFFu) return ARD_ERR_INVALID_ARG;
+  const double sd = floor(k_frac * (double)rows->x * (double)Kc + 0.5);
+  const long long samples = sd < 1.0 ? 1 : (long long)sd;
+  if ((samples + 3) / 4 > 65535) return ARD_ERR_UNSUPPORTED;  // the block index shares a counter word with the stream id
+  const double nd = ceil(t_frac * (double)samples - 1e-9);
+  const int need = nd < 1.0 ? 1 : (int)nd;
+  DevGuard guard(ctx->device);
+  return launch_sensitivity(ctx, rows, dtype, A, lda, Kc, (int)samples, need, threshold, quantise_probability(m_prob),
+                            quantise_probability(n_prob), seed, iteration, stream_id, (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_rows_set_probability(ard_ctx* ctx, ard_rows* rows, double p, void* cuda_stream) {
+  if (!ctx || !rows || rows->ctx != ctx || !(p >= 0.0 && p <= 1.0)) return ARD_ERR_INVALID_ARG;
+  DevGuard guard(ctx->device);
+  return launch_fill_probability(ctx, rows, quantise_probability(p), (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_rows_sample(ard_ctx* ctx, ard_rows* rows, uint64_t seed, uint64_t iteration, uint32_t stream_id,
+                           void* cuda_stream) {
+  if (!ctx || !rows || rows->ctx != ctx || stream_id > 0xFFFFu) return ARD_ERR_INVALID_ARG;
+  DevGuard guard(ctx->device);
+  return launch_rows_sample(ctx, rows, seed, iteration, stream_id, (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_rows_to_host(const ard_rows* rows, int32_t* n_keep, int32_t* idx, size_t idx_capacity,
+                            uint32_t* region_probability, void* cuda_stream) {
+  if (!rows) return ARD_ERR_INVALID_ARG;
+  DevGuard guard(rows->ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  int32_t hdr[HDR_WORDS];
+  ARD_CUDA_OK(cudaMemcpyAsync(hdr, rows->d_hdr, sizeof(hdr), cudaMemcpyDeviceToHost, s));
+  ARD_CUDA_OK(cudaStreamSynchronize(s));
+  if (n_keep) *n_keep = hdr[HDR_NKEEP];
+  if (idx && idx_capacity > 0) {
+    const size_t n = (size_t)hdr[HDR_NKEEP] < idx_capacity ? (size_t)hdr[HDR_NKEEP] : idx_capacity;
+    ARD_CUDA_OK(cudaMemcpyAsync(idx, rows->d_idx, n * sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  }
+  if (region_probability)
+    ARD_CUDA_OK(cudaMemcpyAsync(region_probability, rows->d_P, (size_t)rows->regions * sizeof(uint32_t),
+                                cudaMemcpyDeviceToHost, s));
+  ARD_CUDA_OK(cudaStreamSynchronize(s));
+  return ARD_OK;
+}
+
+}  // extern "C"
