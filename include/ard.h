@@ -351,6 +351,23 @@ ard_status ard_rows_set_probability(ard_ctx* ctx, ard_rows* rows, double p, void
 /* Sec. 5.2.1: draws the dropped rows and writes the ascending list of kept rows.  Asynchronous. */
 ard_status ard_rows_sample(ard_ctx* ctx, ard_rows* rows, uint64_t seed, uint64_t iteration, uint32_t stream_id,
                            void* cuda_stream);
+/* The three products over the kept rows (bf16 operands on the tensor cores, fp32 accumulation), with
+ * keep = the list drawn by ard_rows_sample, A [M][K] (lda; K = Kc), W [N][K] (ldw), Y / dY [M][N], dA [M][K]:
+ *   ard_rows_fwd         Y[r, :]  = alpha * A[r, :] W^T   for kept rows r, zero for dropped rows
+ *   ard_rows_bwd_data    dA[r, :] = alpha * dY[r, :] W    for kept rows r, zero for dropped rows
+ *   ard_rows_bwd_weight  dW = alpha * sum over kept rows r of dY[r, :]^T A[r, :]   (dW [N][K], dW_dtype)
+ * Only the kept rows of A / dY are fetched: the loading warp of the kernel follows the list with 16-byte
+ * asynchronous copies (an index list has no stride a TMA box could follow).  Requires 16-byte aligned
+ * pointers, leading dimensions that are multiples of 8 elements and K, N multiples of 8
+ * (ARD_ERR_ALIGNMENT otherwise: there is no second kernel family for this part).  M must equal the M of
+ * `rows`.  Asynchronous. */
+ard_status ard_rows_fwd(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha, const void* A, int lda,
+                        const void* W, int ldw, void* Y, int ldy, void* cuda_stream);
+ard_status ard_rows_bwd_data(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha, const void* dY,
+                             int lddy, const void* W, int ldw, void* dA, int ldda, void* cuda_stream);
+ard_status ard_rows_bwd_weight(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N, float alpha,
+                               const void* A, int lda, const void* dY, int lddy, void* dW, int lddw,
+                               void* cuda_stream);
 /* Test / debug: synchronises; n_keep, the kept rows (at most idx_capacity) and the per-region integers
  * (ceil(M / region_rows) entries) to HOST buffers; idx and region_probability may be NULL. */
 ard_status ard_rows_to_host(const ard_rows* rows, int32_t* n_keep, int32_t* idx, size_t idx_capacity,

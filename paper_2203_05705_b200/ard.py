@@ -34,7 +34,7 @@ EXPORTS = [
     "ard_layer_fwd", "ard_layer_bwd_data", "ard_layer_bwd_weight", "ard_compact_weight_cols",
     "ard_expand_weight_grad_cols", "ard_bias_grad", "ard_sample_pattern_counter", "ard_mlp_step",
     "ard_rows_create", "ard_rows_destroy", "ard_sensitivity_predict", "ard_rows_set_probability", "ard_rows_sample",
-    "ard_rows_to_host",
+    "ard_rows_to_host", "ard_rows_fwd", "ard_rows_bwd_data", "ard_rows_bwd_weight",
 ]
 
 _lib = None
@@ -110,6 +110,9 @@ def lib():
         "ard_rows_set_probability": [vp, vp, C.c_double, vp],
         "ard_rows_sample": [vp, vp, u64, u64, u32, vp],
         "ard_rows_to_host": [vp, P(C.c_int32), P(C.c_int32), sz, P(C.c_uint32), vp],
+        "ard_rows_fwd": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_rows_bwd_data": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_rows_bwd_weight": [vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -370,6 +373,21 @@ def ard_rows_to_host(rows, M, regions=0, stream=None):
                                   P.ctypes.data_as(C.POINTER(C.c_uint32)) if regions else None, _stream(stream)),
            "ard_rows_to_host")
     return nk.value, idx[:nk.value].copy(), P
+
+
+def ard_rows_fwd(ctx, rows, M, K, N, alpha, A, lda, W, ldw, Y, ldy, stream=None):
+    _check(lib().ard_rows_fwd(ctx, rows, M, K, N, alpha, _ptr(A), lda, _ptr(W), ldw, _ptr(Y), ldy, _stream(stream)),
+           "ard_rows_fwd")
+
+
+def ard_rows_bwd_data(ctx, rows, M, K, N, alpha, dY, lddy, W, ldw, dA, ldda, stream=None):
+    _check(lib().ard_rows_bwd_data(ctx, rows, M, K, N, alpha, _ptr(dY), lddy, _ptr(W), ldw, _ptr(dA), ldda,
+                                   _stream(stream)), "ard_rows_bwd_data")
+
+
+def ard_rows_bwd_weight(ctx, rows, dW_dtype, M, K, N, alpha, A, lda, dY, lddy, dW, lddw, stream=None):
+    _check(lib().ard_rows_bwd_weight(ctx, rows, dW_dtype, M, K, N, alpha, _ptr(A), lda, _ptr(dY), lddy, _ptr(dW), lddw,
+                                     _stream(stream)), "ard_rows_bwd_weight")
 
 
 def ard_lstm_gate_gemm(ctx, pat, B, KH, H, XH, ldxh, W, ldw, Z, ldz_gate, stream=None):

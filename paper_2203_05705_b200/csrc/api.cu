@@ -1151,6 +1151,85 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
   return ARD_OK;
 }
 
+// ---- products over the kept rows of a convolution layer's input matrix (Sec. 5.2.1) -----------------
+static ard_status rows_check(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, const void* p0, int ld0,
+                             const void* p1, int ld1, const void* po, int ldo, int out_es) {
+  if (!ctx || !rows || rows->ctx != ctx || !p0 || !p1 || !po) return ARD_ERR_INVALID_ARG;
+  ctx->epoch++;
+  if (M != rows->M || K < 1 || N < 1) return ARD_ERR_SHAPE;
+  if (ctx->encode_fn == nullptr) return ARD_ERR_UNSUPPORTED;
+  if (!aligned16(p0) || !aligned16(p1) || !aligned16(po)) return ARD_ERR_ALIGNMENT;
+  if (ld0 % 8 || ld1 % 8 || ((size_t)ldo * out_es) % 16 || K % 8 || N % 8) return ARD_ERR_ALIGNMENT;
+  return ARD_OK;
+}
+
+ard_status ard_rows_fwd(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha, const void* A, int lda,
+                        const void* W, int ldw, void* Y, int ldy, void* cuda_stream) {
+  ard_status st = rows_check(ctx, rows, M, K, N, A, lda, W, ldw, Y, ldy, 2);
+  if (st != ARD_OK) return st;
+  if (lda < K || ldw < K || ldy < N) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  TcArgs t = {};
+  GemmArgs g = {};
+  g.hdr = rows->d_hdr;
+  g.B = M; g.K = K; g.N = N;
+  g.alpha = alpha;
+  g.out = Y; g.ldo = ldy;
+  g.status = ctx->d_status;
+  st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);  // boxes [64 neurons][64 k]
+  if (st != ARD_OK) return st;
+  t.g = g;
+  t.bn = ctx->force_bn;
+  st = launch_zero_dropped_rows(ctx, rows, Y, ldy * 2, N * 2, s);
+  if (st != ARD_OK) return st;
+  return launch_rows_tc(ctx, OP_FWD, t, rows->d_idx, A, lda, nullptr, 0, s);
+}
+
+ard_status ard_rows_bwd_data(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha, const void* dY,
+                             int lddy, const void* W, int ldw, void* dA, int ldda, void* cuda_stream) {
+  ard_status st = rows_check(ctx, rows, M, K, N, dY, lddy, W, ldw, dA, ldda, 2);
+  if (st != ARD_OK) return st;
+  if (lddy < N || ldw < K || ldda < K) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  TcArgs t = {};
+  GemmArgs g = {};
+  g.hdr = rows->d_hdr;
+  g.B = M; g.K = K; g.N = N;
+  g.alpha = alpha;
+  g.out = dA; g.ldo = ldda;
+  g.status = ctx->d_status;
+  st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);  // read MN-major: boxes [64 neurons][64 k]
+  if (st != ARD_OK) return st;
+  t.g = g;
+  t.bn = ctx->force_bn;
+  st = launch_zero_dropped_rows(ctx, rows, dA, ldda * 2, K * 2, s);
+  if (st != ARD_OK) return st;
+  return launch_rows_tc(ctx, OP_BWD_DATA, t, rows->d_idx, dY, lddy, nullptr, 0, s);
+}
+
+ard_status ard_rows_bwd_weight(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N, float alpha,
+                               const void* A, int lda, const void* dY, int lddy, void* dW, int lddw,
+                               void* cuda_stream) {
+  if (dW_dtype != ARD_F32 && dW_dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  ard_status st = rows_check(ctx, rows, M, K, N, A, lda, dY, lddy, dW, lddw, dW_dtype == ARD_F32 ? 4 : 2);
+  if (st != ARD_OK) return st;
+  if (lda < K || lddy < N || lddw < K) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  TcArgs t = {};
+  GemmArgs g = {};
+  g.hdr = rows->d_hdr;
+  g.B = M; g.K = K; g.N = N;
+  g.alpha = alpha;
+  g.out = dW; g.ldo = lddw;
+  g.out_is_f32 = dW_dtype == ARD_F32;
+  g.status = ctx->d_status;
+  t.g = g;
+  t.bn = ctx->force_bn;
+  return launch_rows_tc(ctx, OP_BWD_WEIGHT, t, rows->d_idx, dY, lddy, A, lda, (cudaStream_t)cuda_stream);
+}
+
 ard_status ard_last_device_status(ard_ctx* ctx, void* cuda_stream) {
   if (!ctx) return ARD_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);

@@ -46,15 +46,23 @@ enum TcMode {
   // units of gate g are the rows g*H + keep[j] of W, reached through one descriptor table per gate.
   M_LSTM_FWD = 9,       // Z[:, g*ldz + j] = [x,h] . W[g*H + keep[j], :]
   M_LSTM_BWD_DATA = 10, // d[x,h] = sum_g dZ[:, g*ldz + j] . W[g*H + keep[j], :]
-  M_LSTM_BWD_WEIGHT = 11 // dW[g*H + keep[j], :] = sum_rows dZ[:, g*ldz + j] . [x,h]   (M tiles: gate-major)
+  M_LSTM_BWD_WEIGHT = 11, // dW[g*H + keep[j], :] = sum_rows dZ[:, g*ldz + j] . [x,h]   (M tiles: gate-major)
+  // Products over an index list of kept ROWS of the input matrix (Sec. 5.2.1).  The kept rows follow no
+  // stride, so the producer warp gathers them with 16-byte cp.async copies into the same swizzled layout a
+  // TMA box would have produced; the weight still arrives by TMA.
+  M_ROWS_FWD = 12,        // Y[idx[j], :]  = A[idx[j], :] . W^T          (A gathered, K-major)
+  M_ROWS_BWD_DATA = 13,   // dA[idx[j], :] = dY[idx[j], :] . W           (dY gathered, K-major)
+  M_ROWS_BWD_WEIGHT = 14  // dW[n, :] = sum_j dY[idx[j], n] A[idx[j], :] (both gathered, MN-major)
 };
 
 __host__ __device__ constexpr bool a_is_mn(int mode) {
-  return mode == M_ROW_BWD_WEIGHT || mode == M_TILE_BWD_WEIGHT || mode == M_TILEC_BWD_WEIGHT || mode == M_LSTM_BWD_WEIGHT;
+  return mode == M_ROW_BWD_WEIGHT || mode == M_TILE_BWD_WEIGHT || mode == M_TILEC_BWD_WEIGHT ||
+         mode == M_LSTM_BWD_WEIGHT || mode == M_ROWS_BWD_WEIGHT;
 }
 __host__ __device__ constexpr bool b_is_mn(int mode) {
-  return mode != M_ROW_FWD && mode != M_TILE_FWD && mode != M_TILEC_FWD && mode != M_LSTM_FWD;
+  return mode != M_ROW_FWD && mode != M_TILE_FWD && mode != M_TILEC_FWD && mode != M_LSTM_FWD && mode != M_ROWS_FWD;
 }
+__host__ __device__ constexpr bool is_rows_mode(int mode) { return mode >= M_ROWS_FWD && mode <= M_ROWS_BWD_WEIGHT; }
 __host__ __device__ constexpr bool is_class_mode(int mode) { return mode >= M_TILEC_FWD && mode <= M_TILEC_BWD_WEIGHT; }
 __host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 4 : (bn == 128 ? 6 : 8); }
 __host__ __device__ constexpr int tmem_cols_for(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }
@@ -97,6 +105,12 @@ struct TcParams {
   int relu;
   const void* act;
   int ldact;
+  // Row-list products: the kept-row list and the matrices the producer gathers from.
+  const int32_t* ridx;
+  const __nv_bfloat16* gA;  // forward: A; backward-data: dY; backward-weight: dY
+  int ldgA;
+  const __nv_bfloat16* gB;  // backward-weight: A
+  int ldgB;
 };
 
 // CTAS = 2: a cluster of two CTAs shares one 256 x BN output tile; each CTA stages its own 128 rows
@@ -198,6 +212,9 @@ struct Sched {
     else if (MODE == M_LSTM_FWD) { M_gemm = p.B; N_gemm = ((n_keep + 63) / 64) * 256; Kc = p.K; }
     else if (MODE == M_LSTM_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 4 * (((n_keep + 63) / 64) * 64); }
     else if (MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = kin; Kc = p.B; }
+    else if (MODE == M_ROWS_FWD) { M_gemm = n_keep; N_gemm = p.N; Kc = p.K; }
+    else if (MODE == M_ROWS_BWD_DATA) { M_gemm = n_keep; N_gemm = p.K; Kc = p.N; }
+    else if (MODE == M_ROWS_BWD_WEIGHT) { M_gemm = p.N; N_gemm = p.K; Kc = n_keep; }
     else if (MODE == M_TILE_FWD || MODE == M_TILEC_FWD) { M_gemm = p.B; N_gemm = p.N; Kc = 0; }
     else if (MODE == M_TILE_BWD_DATA || MODE == M_TILEC_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 0; }
     else { M_gemm = p.N; N_gemm = p.K; Kc = p.B; }
@@ -242,7 +259,7 @@ struct Sched {
       Mt = (M_gemm + BM * CTAS - 1) / (BM * CTAS);
       if (MODE == M_LSTM_BWD_WEIGHT) Mt *= 4;  // the M tiles of the four gate blocks, gate after gate
       if (MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA || MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_DATA ||
-          MODE == M_LSTM_BWD_WEIGHT) {
+          MODE == M_LSTM_BWD_WEIGHT || is_rows_mode(MODE)) {
         if (p.force_bn) {
           bn = p.force_bn;
         } else {
@@ -567,7 +584,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(full_bar(s), 1);
+      // row-list products: lane 0's arrival (with the TMA byte count) plus one arrival per gathering lane
+      mbar_init(full_bar(s), is_rows_mode(MODE) ? 33 : 1);
       mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -617,7 +635,110 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   }
   const int w0 = (int)blockIdx.x / CTAS;  // first tile of this CTA (pair)
 
-  if (warp == 0) {
+  if (warp == 0 && is_rows_mode(MODE)) {
+    // ===================== gathering producer (all 32 lanes) =====================
+    const CUtensorMap* mapB = p.mapB;
+    if (MODE != M_ROWS_BWD_WEIGHT && lane == 0) tensormap_acquire(mapB);
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    Unit un;
+    for (int i = 0; ok && sch.unit(w0, i, un); ++i) {
+      const TileInfo ti = sch.tile(p, un.t);
+      // K-major gathered operand: this lane owns rows lane, lane + 32, lane + 64, lane + 96 of the tile
+      const __nv_bfloat16* rowp[4] = {nullptr, nullptr, nullptr, nullptr};
+      if (MODE != M_ROWS_BWD_WEIGHT) {
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const int m = ti.m0 + lane + 32 * q4;
+          if (m < sch.M_gemm) rowp[q4] = p.gA + (size_t)p.ridx[m] * p.ldgA;
+        }
+      }
+      for (int kb = 0; kb < ti.nkb; ++kb) {
+        // backward-weight: the two contraction rows of this block that the lane owns
+        const __nv_bfloat16 *ja[2] = {nullptr, nullptr}, *jb[2] = {nullptr, nullptr};
+        if (MODE == M_ROWS_BWD_WEIGHT) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int j = kb * BK + lane + 32 * h;
+            if (j < sch.Kc) {
+              const size_t r = (size_t)p.ridx[j];
+              ja[h] = p.gA + r * p.ldgA;
+              jb[h] = p.gB + r * p.ldgB;
+            }
+          }
+        }
+        int good = 1;
+        if (lane == 0) good = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status) ? 1 : 0;
+        good = __shfl_sync(0xffffffffu, good, 0);
+        if (!good) { ok = false; break; }
+        const uint32_t sA = base + stage * L::STAGE_BYTES;
+        const uint32_t sB = sA + L::A_BYTES;
+        const int kx = kb * BK;
+        if (lane == 0) {
+          if (MODE == M_ROWS_BWD_WEIGHT) {
+            mbar_arrive(full_bar(stage));
+          } else {
+            mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(ti.nbox * 64 * BK * 2));
+#pragma unroll
+            for (int bxi = 0; bxi < 4; ++bxi) {
+              if (bxi < ti.nbox) {
+                if (MODE == M_ROWS_FWD) tma_load_2d(sB + bxi * (64 * BK * 2), mapB, full_bar(stage), kx, ti.bx[bxi]);
+                else tma_load_2d(sB + bxi * (64 * BK * 2), mapB, full_bar(stage), ti.bx[bxi], kx);
+              }
+            }
+          }
+        }
+        if (MODE != M_ROWS_BWD_WEIGHT) {
+          // [128 rows][64 k], 128 bytes per row, 16-byte chunk c of row r at chunk c ^ (r & 7)
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int r = lane + 32 * q4;
+            const uint32_t drow = sA + (uint32_t)r * 128u;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              const int k = kx + 8 * c;
+              const bool in = rowp[q4] != nullptr && k < sch.Kc;
+              cp_async_16(drow + (uint32_t)((c ^ (r & 7)) << 4), in ? (const void*)(rowp[q4] + k) : (const void*)p.gA,
+                          in ? 16u : 0u);
+            }
+          }
+        } else {
+          // boxes of [64 contraction rows][64 columns]: A operand = dY columns m0.., B operand = A columns n0..
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int jr = lane + 32 * h;
+            const uint32_t sw = (uint32_t)(jr & 7);
+#pragma unroll
+            for (int bxi = 0; bxi < BM / 64; ++bxi) {
+              const uint32_t drow = sA + (uint32_t)bxi * (64 * BK * 2) + (uint32_t)jr * 128u;
+#pragma unroll
+              for (int c = 0; c < 8; ++c) {
+                const int col = ti.ax[bxi] + 8 * c;
+                const bool in = ja[h] != nullptr && col < sch.M_gemm;
+                cp_async_16(drow + (((uint32_t)c ^ sw) << 4), in ? (const void*)(ja[h] + col) : (const void*)p.gA, in ? 16u : 0u);
+              }
+            }
+#pragma unroll
+            for (int bxi = 0; bxi < 4; ++bxi) {
+              if (bxi < ti.nbox) {
+                const uint32_t drow = sB + (uint32_t)bxi * (64 * BK * 2) + (uint32_t)jr * 128u;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                  const int col = ti.bx[bxi] + 8 * c;
+                  const bool in = jb[h] != nullptr && col < sch.N_gemm;
+                  cp_async_16(drow + (((uint32_t)c ^ sw) << 4), in ? (const void*)(jb[h] + col) : (const void*)p.gA,
+                              in ? 16u : 0u);
+                }
+              }
+            }
+          }
+        }
+        cp_async_mbar_arrive_noinc(full_bar(stage));
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0) {
       const int e = p.hdr[HDR_MAPIDX];
@@ -723,6 +844,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+          if (is_rows_mode(MODE)) {
+            // the gathered operand was written by ordinary asynchronous copies (generic proxy)
+            fence_proxy_async_smem();
+            tc_fence_after();
+          }
           // This thread's instruction stream is what feeds the tensor pipe: the descriptors of a block are
           // the stage's descriptor plus a constant per 16-deep step (the start-address field counts 16-byte
           // units: K-major 32 bytes = 2 per step, MN-major 16 k-rows = 2048 bytes = 128 per step).
@@ -782,6 +908,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         row_ok = m < sch.M_gemm;
         out_row = (long long)bb + (long long)m * dp;
         if (MODE == M_LSTM_BWD_WEIGHT) out_row += ti.out_row0;
+      } else if (MODE == M_ROWS_FWD || MODE == M_ROWS_BWD_DATA) {
+        row_ok = m < sch.M_gemm;
+        out_row = row_ok ? (long long)p.ridx[m] : 0;  // the results go back to the rows they came from
       } else if (MODE == M_TILE_BWD_WEIGHT) {
         row_ok = row_in_tile < ti.rows_valid && m < sch.M_gemm;
         out_row = m;
@@ -1227,6 +1356,36 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
 #undef ARD_TC_ROW
 #undef ARD_TC_PAIR
   return ARD_ERR_UNSUPPORTED;
+}
+
+// Products over a list of kept rows (Sec. 5.2.1).  Single-CTA tiles: the gathering lanes arrive on their own
+// CTA's barrier.
+ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_t* ridx, const void* gA, int ldgA,
+                          const void* gB, int ldgB, cudaStream_t s) {
+  TcParams p = {};
+  p.mapA = nullptr;
+  p.mapB = a.mapB;
+  p.hdr = a.g.hdr;
+  p.B = a.g.B;
+  p.K = a.g.K;
+  p.N = a.g.N;
+  p.alpha = a.g.alpha;
+  p.out = a.g.out;
+  p.ldo = a.g.ldo;
+  p.out_is_f32 = a.g.out_is_f32;
+  p.status = a.g.status;
+  p.force_bn = a.bn;
+  p.band_m = ctx->band_m;
+  p.sk_min_blocks = 16;
+  p.sk_min_gain = 1;
+  p.ridx = ridx;
+  p.gA = reinterpret_cast<const __nv_bfloat16*>(gA);
+  p.ldgA = ldgA;
+  p.gB = reinterpret_cast<const __nv_bfloat16*>(gB);
+  p.ldgB = ldgB;
+  if (op == OP_FWD) return launch_mode<256, M_ROWS_FWD, 1>(ctx, p, cdiv(p.B, BM) * cdiv(p.N, 64), s);
+  if (op == OP_BWD_DATA) return launch_mode<256, M_ROWS_BWD_DATA, 1>(ctx, p, cdiv(p.B, BM) * cdiv(p.K, 64), s);
+  return launch_mode<256, M_ROWS_BWD_WEIGHT, 1>(ctx, p, cdiv(p.N, BM) * cdiv(p.K, 64), s);
 }
 
 // LSTM gate products (single CTA per tile; the batch of a recurrent step is small).

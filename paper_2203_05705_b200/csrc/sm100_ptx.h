@@ -199,3 +199,17 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn, bool b_mn, i
 }
 
 }  // namespace
+
+// ---- non-bulk asynchronous copies (row gathers: a TMA box cannot follow an index list) -------------------
+// 16 bytes global -> shared; src_bytes = 0 writes zeros and reads nothing.
+__device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
+}
+// Arrives on the barrier once all earlier cp.async of this thread have landed; the barrier's expected count
+// must already include this arrival.
+__device__ __forceinline__ void cp_async_mbar_arrive_noinc(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+// Orders what the generic proxy wrote to shared memory (and this thread has observed) before later reads of
+// the async proxy (tcgen05.mma operands).
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

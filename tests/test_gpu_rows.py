@@ -57,3 +57,87 @@ def test_prediction_and_row_list_are_bit_exact(M, Kc, x, dtype):
         torch.cuda.synchronize()
         ard.ard_rows_destroy(rows)
         ctx.close()
+
+
+@pytest.mark.parametrize("M,K,N", [(300, 328, 520), (1000, 64, 72), (130, 1160, 264), (64, 72, 8)])
+def test_products_over_the_kept_rows_match_the_oracle(M, K, N):
+    """Forward, backward-data and backward-weight over the drawn rows; NaN wherever the kernels must write
+    (so a row left out shows) and in the rows of the operands that must not be read."""
+    rng = np.random.default_rng(M + K)
+    A = inputs.bf16_round(rng.standard_normal((M, K)).astype(np.float32))
+    W = inputs.bf16_round((rng.standard_normal((K, N)) / np.sqrt(K)).astype(np.float32))      # math orientation
+    dY = inputs.bf16_round(rng.standard_normal((M, N)).astype(np.float32))
+    ctx = Ctx(4096)
+    rows = ard.ard_rows_create(ctx.h, M, 3)
+    try:
+        Wd = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+        tol = TOL[ard.ARD_BF16]
+        for it, p in enumerate([0.0, 0.3, 0.5, 0.9, 0.999]):
+            ard.ard_rows_set_probability(ctx.h, rows, p)
+            ard.ard_rows_sample(ctx.h, rows, 7, it, 1)
+            n_keep, keep, _ = ard.ard_rows_to_host(rows, M)
+            Pq = np.full((M + 2) // 3, OC.quantise_probability(p), dtype=np.uint64)
+            assert np.array_equal(keep, OC.draw_rows(Pq, 3, M, 7, it, 1))
+            dropped = np.setdiff1d(np.arange(M), keep)
+            # operands: dropped rows hold NaN -- they must never be fetched
+            Ad = torch.from_numpy(A).to(BF).cuda()
+            dYd = torch.from_numpy(dY).to(BF).cuda()
+            if len(dropped):
+                Ad[torch.from_numpy(dropped).cuda()] = float("nan")
+                dYd[torch.from_numpy(dropped).cuda()] = float("nan")
+            Y = torch.full((M, N), float("nan"), dtype=BF, device="cuda")
+            dA = torch.full((M, K), float("nan"), dtype=BF, device="cuda")
+            dW = torch.full((N, K), float("nan"), dtype=torch.float32, device="cuda")
+            ard.ard_rows_fwd(ctx.h, rows, M, K, N, 1.5, Ad, K, Wd, K, Y, N)
+            ard.ard_rows_bwd_data(ctx.h, rows, M, K, N, 1.5, dYd, N, Wd, K, dA, K)
+            ard.ard_rows_bwd_weight(ctx.h, rows, ard.ARD_F32, M, K, N, 1.5, Ad, K, dYd, N, dW, K)
+            torch.cuda.synchronize()
+            assert ard.ard_last_device_status(ctx.h) == 0
+            tag = (M, K, N, p, n_keep)
+            Yh, dAh, dWh = host(Y), host(dA), host(dW)
+            assert np.all(Yh[dropped] == 0) and np.all(dAh[dropped] == 0), tag
+            if n_keep:
+                assert OG.rel_fro(Yh, OC.fwd(A, W, keep, 1.5)) <= tol, tag
+                assert OG.rel_fro(dAh, OC.bwd_data(dY, W, keep, 1.5)) <= tol, tag
+                assert OG.rel_fro(dWh, OC.bwd_weight(A, dY, keep, 1.5).T) <= tol, tag
+            else:
+                assert np.all(Yh == 0) and np.all(dAh == 0) and np.all(dWh == 0), tag
+    finally:
+        torch.cuda.synchronize()
+        ard.ard_rows_destroy(rows)
+        ctx.close()
+
+
+def test_repeated_launches_give_the_same_bits():
+    """The gathered operand reaches the tensor cores through ordinary asynchronous copies; a missing ordering
+    between those writes and the MMA reads would show as run-to-run differences."""
+    M, K, N = 2048, 1152, 256
+    rng = np.random.default_rng(5)
+    A = torch.from_numpy(inputs.bf16_round(rng.standard_normal((M, K)).astype(np.float32))).to(BF).cuda()
+    W = torch.from_numpy(inputs.bf16_round((rng.standard_normal((N, K)) / 34).astype(np.float32))).to(BF).cuda()
+    dY = torch.from_numpy(inputs.bf16_round(rng.standard_normal((M, N)).astype(np.float32))).to(BF).cuda()
+    ctx = Ctx(4096)
+    rows = ard.ard_rows_create(ctx.h, M, 1)
+    try:
+        ard.ard_rows_set_probability(ctx.h, rows, 0.4)
+        ard.ard_rows_sample(ctx.h, rows, 3, 0, 0)
+        ref = None
+        for rep in range(20):
+            Y = torch.zeros((M, N), dtype=BF, device="cuda")
+            dA = torch.zeros((M, K), dtype=BF, device="cuda")
+            dW = torch.zeros((N, K), dtype=torch.float32, device="cuda")
+            ard.ard_rows_fwd(ctx.h, rows, M, K, N, 1.0, A, K, W, K, Y, N)
+            ard.ard_rows_bwd_data(ctx.h, rows, M, K, N, 1.0, dY, N, W, K, dA, K)
+            ard.ard_rows_bwd_weight(ctx.h, rows, ard.ARD_F32, M, K, N, 1.0, A, K, dY, N, dW, K)
+            torch.cuda.synchronize()
+            cur = (Y, dA, dW)
+            if ref is None:
+                ref = cur
+            else:
+                for a, c in zip(cur, ref):
+                    assert torch.equal(a, c), rep
+        assert ard.ard_last_device_status(ctx.h) == 0
+    finally:
+        torch.cuda.synchronize()
+        ard.ard_rows_destroy(rows)
+        ctx.close()
