@@ -46,6 +46,10 @@ WORKLOADS = {
     # stack of large layers where the second hidden layer multiplies two compact matrices
     "mlp2048_step": dict(config=2, dims=[784, 2048, 2048, 10], B=128, kind="mlp_step", p=0.5, n_dp=16),
     "mlp8192_step": dict(config=5, dims=[8192, 8192, 8192, 1024], B=4096, kind="mlp_step", p=0.5, n_dp=16),
+    # a convolution layer as the product of its im2col input matrix with the filters, rows of the input matrix
+    # dropped by predicted sensitivity (Sec. 5.1, 5.2.1): 3x3 filters, 256 -> 512 channels, 32768 output positions
+    "conv_rows": dict(config=5, M=32768, K=2304, N=512, kind="conv_rows", region_rows=8, k_frac=0.05, t_frac=0.3,
+                      threshold=0.5, m_prob=0.2, n_prob=0.8),
     # LSTM layer (config 4): a step is one sequence, forward + BPTT, one fresh pattern per sequence
     "lstm1024": dict(config=4, T=35, B=64, I=1024, H=1024, kind="lstm", p=0.5, n_dp=16),
 }
@@ -556,6 +560,129 @@ def run_mlp_step(args, wl):
     print(json.dumps(line))
 
 
+def run_conv_rows(args, wl):
+    """A step = sensitivity prediction + row sampling + the three products over the kept rows of the input matrix."""
+    import torch
+    from paper_2203_05705_b200 import ard
+    dev_index = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(dev_index)
+    clocks = ClockSampler(dev_index)
+    M, K, N, x = wl["M"], wl["K"], wl["N"], wl["region_rows"]
+    bf = torch.bfloat16
+    g = torch.Generator(device="cuda").manual_seed(inputs.BASE_SEED)
+    # post-ReLU-like input matrix with quiet and busy regions, so that both kinds of region occur
+    level = torch.tensor([0.1, 1.0, 4.0], device="cuda")[torch.randint(0, 3, (M // x,), device="cuda", generator=g)]
+    A = (torch.relu(torch.randn((M, K), device="cuda", generator=g)) * level.repeat_interleave(x)[:, None]).to(bf)
+    W = (torch.randn((N, K), device="cuda", generator=g) / K ** 0.5).to(bf)
+    dY = torch.randn((M, N), device="cuda", generator=g).to(bf)
+    Y = torch.empty((M, N), dtype=bf, device="cuda")
+    dA = torch.empty((M, K), dtype=bf, device="cuda")
+    dW = torch.empty((N, K), dtype=bf, device="cuda")
+    hA, hdY = A.cpu().pin_memory(), dY.cpu().pin_memory()
+    hY = torch.empty((M, N), dtype=bf).pin_memory()
+    ctx = ard.ard_create(0, 4096)
+    rows = ard.ard_rows_create(ctx, M, x)
+
+    def step(it, dense=False, host=False):
+        if host:
+            A.copy_(hA, non_blocking=True)
+            dY.copy_(hdY, non_blocking=True)
+        if dense:
+            ard.ard_rows_set_probability(ctx, rows, 0.0)
+        else:
+            ard.ard_sensitivity_predict(ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["t_frac"], wl["threshold"],
+                                        wl["m_prob"], wl["n_prob"], inputs.BASE_SEED, it, 0)
+        ard.ard_rows_sample(ctx, rows, inputs.BASE_SEED, it, 0)
+        ard.ard_rows_fwd(ctx, rows, M, K, N, 1.0, A, K, W, K, Y, N)
+        ard.ard_rows_bwd_data(ctx, rows, M, K, N, 1.0, dY, N, W, K, dA, K)
+        ard.ard_rows_bwd_weight(ctx, rows, ard.ARD_BF16, M, K, N, 1.0, A, K, dY, N, dW, K)
+        if host:
+            hY.copy_(Y, non_blocking=True)
+
+    def timed(fn, n, warm):
+        for w in range(warm):
+            fn(w)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record()
+        for i in range(n):
+            fn(warm + i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1), t0, time.time()
+
+    steps, warm = args.steps, max(3, args.warmup)
+    l0 = ard.ard_launch_count(ctx)
+    ms, t0, t1 = timed(step, steps, warm)
+    launches = (ard.ard_launch_count(ctx) - l0) * steps // (steps + warm)
+    clk = clocks.stop(t0, t1)
+    status = ard.ard_last_device_status(ctx)
+    kept_rows = []
+    for i in range(steps):
+        ard.ard_sensitivity_predict(ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["t_frac"], wl["threshold"],
+                                    wl["m_prob"], wl["n_prob"], inputs.BASE_SEED, warm + i, 0)
+        ard.ard_rows_sample(ctx, rows, inputs.BASE_SEED, warm + i, 0)
+        kept_rows.append(ard.ard_rows_to_host(rows, 0)[0])
+    kept = sum(3 * 2.0 * nk * K * N for nk in kept_rows)
+    value = kept / (ms * 1e-3) / 1e12
+    detail = {"ms_per_step": {"ours": ms / steps}, "kept_row_fraction": float(np.mean(kept_rows)) / M}
+    e2e = None
+    if not args.quick:
+        n2 = max(5, steps // 4)
+        detail["ms_per_step"]["own_kernels_all_rows"] = timed(lambda it: step(it, dense=True), n2, warm)[0] / n2
+
+        def torch_step(it):
+            torch.matmul(A, W.t(), out=Y)
+            torch.matmul(dY, W, out=dA)
+            torch.matmul(dY.t(), A, out=dW)
+
+        detail["ms_per_step"]["torch_matmul_dense"] = timed(torch_step, n2, warm)[0] / n2
+        detail["speedup_vs_dense"] = min(detail["ms_per_step"]["own_kernels_all_rows"],
+                                         detail["ms_per_step"]["torch_matmul_dense"]) / (ms / steps)
+        ms_e = timed(lambda it: step(it + 100000, host=True), n2, warm)[0] / n2
+        e2e = {"value": float(np.mean(kept_rows)) * 3 * 2.0 * K * N / (ms_e * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": hA.numel() * 2 + hdY.numel() * 2, "d2h_bytes_per_step": hY.numel() * 2,
+               "ms_per_step": ms_e}
+    peaks = load_peaks()
+    cpu = None
+    if not args.no_cpu_baseline and not args.quick:
+        from oracle import cnn as OC
+        Mh = 2048
+        Ah, Wh, dYh = A[:Mh].float().cpu().numpy(), W.float().cpu().numpy().T, dY[:Mh].float().cpu().numpy()
+        keep = np.arange(0, Mh, 2)
+        tc0 = time.perf_counter()
+        OC.fwd(Ah, Wh, keep)
+        OC.bwd_data(dYh, Wh, keep)
+        OC.bwd_weight(Ah, dYh, keep)
+        dt = time.perf_counter() - tc0
+        try:
+            from threadpoolctl import threadpool_info
+            threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        except Exception:
+            threads = os.cpu_count() or 1
+        cpu = {"value": 3 * 2.0 * len(keep) * K * N / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": "%d of %d rows of the input matrix, every second one kept (the oracle multiplies the masked full matrix)" % (Mh, M),
+               "seconds": dt}
+    line = {
+        "metric": "convolution layer (im2col product) fwd+bwd kept TFLOP/s, rows dropped by predicted sensitivity",
+        "value": value, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms / steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, **{k: wl[k] for k in ("M", "K", "N", "region_rows", "k_frac", "t_frac",
+                                                                       "threshold", "m_prob", "n_prob")},
+                   "l2": "working set %.0f MB per step" % ((2 * M * K + 2 * M * N + 2 * N * K) * 2 / 1e6)},
+        "dense_equiv_tflops": 3 * 2.0 * M * K * N * steps / (ms * 1e-3) / 1e12, "clocks": clk, "e2e": e2e,
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "achieved": value, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": value / peaks["bf16_tflops"], "traffic": None,
+                     "note": "whole step incl. sensitivity prediction, row sampling and zero fill of the dropped rows"},
+        "cpu_baseline": cpu, "detail": detail, "device_status": int(status),
+    }
+    print(json.dumps(line))
+    ard.ard_rows_destroy(rows)
+    ard.ard_destroy(ctx)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -573,6 +700,8 @@ def main():
         return run_lstm(args, wl)
     if wl["kind"] == "mlp_step":
         return run_mlp_step(args, wl)
+    if wl["kind"] == "conv_rows":
+        return run_conv_rows(args, wl)
 
     import torch
     import torch.distributed as dist

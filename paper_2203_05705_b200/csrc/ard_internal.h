@@ -46,6 +46,8 @@ struct ard_rows {
   int M, x, regions;
   int32_t* d_hdr;    // HDR_WORDS
   int32_t* d_idx;    // kept rows, ascending, capacity M
+  int32_t* d_stage;  // sampler scratch: the kept rows of every 2048-row slice, compacted per slice
+  int32_t* d_counts; // sampler scratch: kept rows per slice
   uint8_t* d_flag;   // 1 = kept, per row
   uint32_t* d_P;     // per region: dropped iff the row's random word is below this
 };

@@ -27,6 +27,8 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;  // 64 bf16 = 128 bytes = one swizzle row
 constexpr int TC_THREADS = 320;  // warp 0 producer, warp 1 MMA, warps 2..9 epilogue
+constexpr int ROWS_GATHER_WARPS = 4;  // row-list products: warp 0 and warps 10..12 gather (one warp cannot issue enough copies)
+constexpr int TC_THREADS_ROWS = TC_THREADS + 32 * (ROWS_GATHER_WARPS - 1);
 constexpr int EPI_WARPS = 8;
 
 enum TcMode {
@@ -63,6 +65,7 @@ __host__ __device__ constexpr bool b_is_mn(int mode) {
   return mode != M_ROW_FWD && mode != M_TILE_FWD && mode != M_TILEC_FWD && mode != M_LSTM_FWD && mode != M_ROWS_FWD;
 }
 __host__ __device__ constexpr bool is_rows_mode(int mode) { return mode >= M_ROWS_FWD && mode <= M_ROWS_BWD_WEIGHT; }
+__host__ __device__ constexpr int tc_threads(int mode) { return is_rows_mode(mode) ? TC_THREADS_ROWS : TC_THREADS; }
 __host__ __device__ constexpr bool is_class_mode(int mode) { return mode >= M_TILEC_FWD && mode <= M_TILEC_BWD_WEIGHT; }
 __host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 4 : (bn == 128 ? 6 : 8); }
 __host__ __device__ constexpr int tmem_cols_for(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }
@@ -559,7 +562,7 @@ __device__ __forceinline__ void zero_row32(void* out, size_t row_off, int col, i
 
 // ---- the kernel -----------------------------------------------------------------------------------
 template <int BN, int MODE, int CTAS, bool SHARE, bool FUSED>
-__global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcParams p) {
+__global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const TcParams p) {
   using L = SmemLayout<BN, CTAS>;
   const uint32_t rank = (CTAS == 2) ? cluster_ctarank() : 0u;  // rank 0 leads the pair and issues its MMAs
   constexpr int STAGES = L::STAGES;
@@ -584,8 +587,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      // row-list products: lane 0's arrival (with the TMA byte count) plus one arrival per gathering lane
-      mbar_init(full_bar(s), is_rows_mode(MODE) ? 33 : 1);
+      // row-list products: one arrival with the TMA byte count plus one arrival per gathering lane
+      mbar_init(full_bar(s), is_rows_mode(MODE) ? 1 + 32 * ROWS_GATHER_WARPS : 1);
       mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -635,38 +638,47 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
   }
   const int w0 = (int)blockIdx.x / CTAS;  // first tile of this CTA (pair)
 
-  if (warp == 0 && is_rows_mode(MODE)) {
-    // ===================== gathering producer (all 32 lanes) =====================
+  if (is_rows_mode(MODE) && (warp == 0 || warp >= 10)) {
+    // ===================== gathering producers (4 warps, all lanes) =====================
+    const int gw = warp == 0 ? 0 : warp - 9;  // 0..3: which quarter of the gathered rows this warp fetches
     const CUtensorMap* mapB = p.mapB;
-    if (MODE != M_ROWS_BWD_WEIGHT && lane == 0) tensormap_acquire(mapB);
+    if (MODE != M_ROWS_BWD_WEIGHT && warp == 0 && lane == 0) tensormap_acquire(mapB);
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     Unit un;
+    // Eight consecutive lanes fetch the eight 16-byte chunks of one row (one 128-byte line), so a warp
+    // instruction asks for four whole lines instead of 32 scattered sectors (the load unit's tag stage was
+    // the limit with one row per lane).  The rows' global addresses are worked out once (per tile, or per
+    // contraction block for the backward-weight product) by the lane that read the list entry and kept in a
+    // small shared-memory table (the staging area of the scatter epilogue is unused in these modes).
+    const int sub = lane >> 3, ch = lane & 7;
+    // this warp's slice of the table: [32] row addresses, or [2 parities][2 operands][16] for backward-weight
+    unsigned long long* rowtab = reinterpret_cast<unsigned long long*>(smem + L::STG_OFF) + gw * 64;
     for (int i = 0; ok && sch.unit(w0, i, un); ++i) {
       const TileInfo ti = sch.tile(p, un.t);
-      // K-major gathered operand: this lane owns rows lane, lane + 32, lane + 64, lane + 96 of the tile
-      const __nv_bfloat16* rowp[4] = {nullptr, nullptr, nullptr, nullptr};
       if (MODE != M_ROWS_BWD_WEIGHT) {
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          const int m = ti.m0 + lane + 32 * q4;
-          if (m < sch.M_gemm) rowp[q4] = p.gA + (size_t)p.ridx[m] * p.ldgA;
-        }
+        __syncwarp();
+        const int m = ti.m0 + gw * 32 + lane;  // this warp fetches tile rows gw*32 .. gw*32 + 31
+        rowtab[lane] = m < sch.M_gemm ? (unsigned long long)(p.gA + (size_t)p.ridx[m] * p.ldgA) : 0ull;
+        __syncwarp();
       }
+      // backward-weight: list entries of contraction rows lane, lane + 32 of the current block; the next
+      // block's are fetched while this one is being issued (a dependent global load per block otherwise)
+      // (lanes 0..15 own the 16 contraction rows gw*16 .. gw*16 + 15 of a block)
+      int jcur = -1;
+      if (MODE == M_ROWS_BWD_WEIGHT && lane < 16 && gw * 16 + lane < sch.Kc) jcur = p.ridx[gw * 16 + lane];
       for (int kb = 0; kb < ti.nkb; ++kb) {
-        // backward-weight: the two contraction rows of this block that the lane owns
-        const __nv_bfloat16 *ja[2] = {nullptr, nullptr}, *jb[2] = {nullptr, nullptr};
+        int jnext = -1;
+        unsigned long long* tabA = rowtab + (kb & 1) * 32;  // [16] addresses in dY, then [16] in A
         if (MODE == M_ROWS_BWD_WEIGHT) {
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int j = kb * BK + lane + 32 * h;
-            if (j < sch.Kc) {
-              const size_t r = (size_t)p.ridx[j];
-              ja[h] = p.gA + r * p.ldgA;
-              jb[h] = p.gB + r * p.ldgB;
-            }
+          if (lane < 16) {
+            tabA[lane] = jcur >= 0 ? (unsigned long long)(p.gA + (size_t)jcur * p.ldgA) : 0ull;
+            tabA[16 + lane] = jcur >= 0 ? (unsigned long long)(p.gB + (size_t)jcur * p.ldgB) : 0ull;
+            const int j = (kb + 1) * BK + gw * 16 + lane;
+            if (kb + 1 < ti.nkb && j < sch.Kc) jnext = p.ridx[j];
           }
+          __syncwarp();  // the table entries are read by other lanes below
         }
         int good = 1;
         if (lane == 0) good = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status) ? 1 : 0;
@@ -675,7 +687,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         const uint32_t sA = base + stage * L::STAGE_BYTES;
         const uint32_t sB = sA + L::A_BYTES;
         const int kx = kb * BK;
-        if (lane == 0) {
+        if (warp == 0 && lane == 0) {
           if (MODE == M_ROWS_BWD_WEIGHT) {
             mbar_arrive(full_bar(stage));
           } else {
@@ -691,50 +703,43 @@ __global__ void __launch_bounds__(TC_THREADS, 1) ard_gemm_tc_kernel(const TcPara
         }
         if (MODE != M_ROWS_BWD_WEIGHT) {
           // [128 rows][64 k], 128 bytes per row, 16-byte chunk c of row r at chunk c ^ (r & 7)
+          const int k = kx + 8 * ch;
+          const bool kin = k < sch.Kc;
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const int r = lane + 32 * q4;
-            const uint32_t drow = sA + (uint32_t)r * 128u;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              const int k = kx + 8 * c;
-              const bool in = rowp[q4] != nullptr && k < sch.Kc;
-              cp_async_16(drow + (uint32_t)((c ^ (r & 7)) << 4), in ? (const void*)(rowp[q4] + k) : (const void*)p.gA,
-                          in ? 16u : 0u);
-            }
+          for (int q = 0; q < 8; ++q) {
+            const int rl = 4 * q + sub, r = gw * 32 + rl;
+            const unsigned long long bp = rowtab[rl];
+            const bool in = bp != 0ull && kin;
+            cp_async_16(sA + (uint32_t)r * 128u + (uint32_t)((ch ^ (r & 7)) << 4),
+                        in ? (const void*)(bp + (unsigned long long)k * 2ull) : (const void*)p.gA, in ? 16u : 0u);
           }
         } else {
           // boxes of [64 contraction rows][64 columns]: A operand = dY columns m0.., B operand = A columns n0..
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int jr = lane + 32 * h;
-            const uint32_t sw = (uint32_t)(jr & 7);
+          for (int q = 0; q < 4; ++q) {
+            const int jl = 4 * q + sub, jr = gw * 16 + jl;
+            const unsigned long long pa = tabA[jl], pb = tabA[16 + jl];
+            const uint32_t off = (uint32_t)jr * 128u + (uint32_t)((ch ^ (jr & 7)) << 4);
 #pragma unroll
             for (int bxi = 0; bxi < BM / 64; ++bxi) {
-              const uint32_t drow = sA + (uint32_t)bxi * (64 * BK * 2) + (uint32_t)jr * 128u;
-#pragma unroll
-              for (int c = 0; c < 8; ++c) {
-                const int col = ti.ax[bxi] + 8 * c;
-                const bool in = ja[h] != nullptr && col < sch.M_gemm;
-                cp_async_16(drow + (((uint32_t)c ^ sw) << 4), in ? (const void*)(ja[h] + col) : (const void*)p.gA, in ? 16u : 0u);
-              }
+              const int col = ti.ax[bxi] + 8 * ch;
+              const bool in = pa != 0ull && col < sch.M_gemm;
+              cp_async_16(sA + (uint32_t)bxi * (64 * BK * 2) + off,
+                          in ? (const void*)(pa + (unsigned long long)col * 2ull) : (const void*)p.gA, in ? 16u : 0u);
             }
 #pragma unroll
             for (int bxi = 0; bxi < 4; ++bxi) {
               if (bxi < ti.nbox) {
-                const uint32_t drow = sB + (uint32_t)bxi * (64 * BK * 2) + (uint32_t)jr * 128u;
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                  const int col = ti.bx[bxi] + 8 * c;
-                  const bool in = jb[h] != nullptr && col < sch.N_gemm;
-                  cp_async_16(drow + (((uint32_t)c ^ sw) << 4), in ? (const void*)(jb[h] + col) : (const void*)p.gA,
-                              in ? 16u : 0u);
-                }
+                const int col = ti.bx[bxi] + 8 * ch;
+                const bool in = pb != 0ull && col < sch.N_gemm;
+                cp_async_16(sB + (uint32_t)bxi * (64 * BK * 2) + off,
+                            in ? (const void*)(pb + (unsigned long long)col * 2ull) : (const void*)p.gA, in ? 16u : 0u);
               }
             }
           }
         }
         cp_async_mbar_arrive_noinc(full_bar(stage));
+        jcur = jnext;
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
@@ -1198,7 +1203,7 @@ ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStrea
     attr_done[dev] = true;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.blockDim = dim3(TC_THREADS);
+  cfg.blockDim = dim3(tc_threads(MODE));
   cfg.dynamicSmemBytes = L::TOTAL;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];

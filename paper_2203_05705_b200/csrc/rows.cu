@@ -68,31 +68,33 @@ __global__ void __launch_bounds__(256) fill_probability_kernel(uint32_t* P_regio
   for (int g = blockIdx.x * 256 + threadIdx.x; g < regions; g += gridDim.x * 256) P_region[g] = P;
 }
 
-// Sec. 5.2.1: row r is dropped iff its Philox word is below the probability of its region.  One CTA: every
-// thread draws a contiguous run of rows, the CTA scans the kept counts and every thread then writes the
-// kept rows of its run, so the list comes out ascending.  hdr mimics a pattern header (dp = b = 1).
-constexpr int ROWS_THREADS = 1024;
+// Sec. 5.2.1: row r is dropped iff its Philox word is below the probability of its region.  Two launches:
+// every CTA draws 2048 consecutive rows (8 per thread), scans the kept counts and parks its kept rows,
+// compacted, in a staging array together with its count; then every CTA adds the counts of the CTAs before
+// it and copies its run to its place in the list, which therefore comes out ascending.  hdr mimics a
+// pattern header (dp = b = 1).
+constexpr int ROWS_PER_CTA = 2048;
 
-__global__ void __launch_bounds__(ROWS_THREADS) rows_sample_kernel(int32_t* hdr, int32_t* idx, uint8_t* kept_flag,
-                                                                   const uint32_t* P_region, int M, int x,
-                                                                   unsigned long long seed, unsigned long long iteration,
-                                                                   uint32_t stream_id) {
-  __shared__ int s_warp[32];
-  __shared__ int s_total;
+__global__ void __launch_bounds__(256) rows_draw_kernel(int32_t* stage, int32_t* counts, uint8_t* kept_flag,
+                                                        const uint32_t* P_region, int M, int x, unsigned long long seed,
+                                                        unsigned long long iteration, uint32_t stream_id) {
+  __shared__ int s_warp[8];
   pdl_launch_dependents();
   pdl_wait_prior_grids();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int per = (M + ROWS_THREADS - 1) / ROWS_THREADS;
-  const int r0 = tid * per, r1 = min(M, r0 + per);
+  const int r0 = blockIdx.x * ROWS_PER_CTA + tid * 8;
+  unsigned keepbits = 0;
   int mine = 0;
-  for (int r = r0; r < r1; ++r) {
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const int r = r0 + q;
+    if (r >= M) break;
     uint32_t c[4] = {(uint32_t)iteration, (uint32_t)(iteration >> 32), (uint32_t)r, (stream_id << 16) | 0xFFFFu};
     philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
     const bool keep = !(c[0] < P_region[r / x]);
     kept_flag[r] = keep ? 1 : 0;
-    mine += keep ? 1 : 0;
+    if (keep) { keepbits |= 1u << q; ++mine; }
   }
-  // exclusive scan of `mine` over the CTA
   int incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -101,25 +103,44 @@ __global__ void __launch_bounds__(ROWS_THREADS) rows_sample_kernel(int32_t* hdr,
   }
   if (lane == 31) s_warp[warp] = incl;
   __syncthreads();
-  if (warp == 0) {
-    int v = s_warp[lane];
+  int before = 0;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int u = __shfl_up_sync(0xffffffffu, v, o);
-      if (lane >= o) v += u;
-    }
-    s_warp[lane] = v;  // inclusive over warps
-    if (lane == 31) s_total = v;
+  for (int w = 0; w < 8; ++w)
+    if (w < warp) before += s_warp[w];
+  int out = blockIdx.x * ROWS_PER_CTA + before + incl - mine;
+#pragma unroll
+  for (int q = 0; q < 8; ++q)
+    if (keepbits & (1u << q)) stage[out++] = r0 + q;
+  if (tid == 255) counts[blockIdx.x] = before + incl;
+}
+
+__global__ void __launch_bounds__(256) rows_compact_kernel(int32_t* hdr, int32_t* idx, const int32_t* stage,
+                                                           const int32_t* counts, int M) {
+  __shared__ int s_part[8];
+  __shared__ int s_base;
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int sum = 0;
+  for (int b = tid; b < (int)blockIdx.x; b += 256) sum += counts[b];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if (lane == 0) s_part[warp] = sum;
+  __syncthreads();
+  if (tid == 0) {
+    int v = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) v += s_part[w];
+    s_base = v;
   }
   __syncthreads();
-  int out = incl - mine + (warp > 0 ? s_warp[warp - 1] : 0);
-  for (int r = r0; r < r1; ++r)
-    if (kept_flag[r]) idx[out++] = r;
-  if (tid == 0) {
+  const int base = s_base, n = counts[blockIdx.x];
+  for (int j = tid; j < n; j += 256) idx[base + j] = stage[blockIdx.x * ROWS_PER_CTA + j];
+  if (blockIdx.x == gridDim.x - 1 && tid == 0) {
     hdr[HDR_KIND] = 2;
     hdr[HDR_DP] = 1;
     hdr[HDR_B] = 1;
-    hdr[HDR_NKEEP] = s_total;
+    hdr[HDR_NKEEP] = base + n;
     hdr[HDR_UNITS] = M;
     hdr[HDR_TR] = 0;
     hdr[HDR_TC] = 0;
@@ -174,10 +195,13 @@ ard_status launch_fill_probability(ard_ctx* ctx, ard_rows* rows, uint32_t P, cud
 
 ard_status launch_rows_sample(ard_ctx* ctx, ard_rows* rows, uint64_t seed, uint64_t iteration, uint32_t stream_id,
                               cudaStream_t s) {
-  ARD_CUDA_OK(ard_launch(ctx, rows_sample_kernel, dim3(1), dim3(ROWS_THREADS), 0, s, rows->d_hdr, rows->d_idx, rows->d_flag,
+  const int nb = (rows->M + ROWS_PER_CTA - 1) / ROWS_PER_CTA;
+  ARD_CUDA_OK(ard_launch(ctx, rows_draw_kernel, dim3(nb), dim3(256), 0, s, rows->d_stage, rows->d_counts, rows->d_flag,
                          (const uint32_t*)rows->d_P, rows->M, rows->x, (unsigned long long)seed,
                          (unsigned long long)iteration, stream_id));
-  ctx->launches++;
+  ARD_CUDA_OK(ard_launch(ctx, rows_compact_kernel, dim3(nb), dim3(256), 0, s, rows->d_hdr, rows->d_idx,
+                         (const int32_t*)rows->d_stage, (const int32_t*)rows->d_counts, rows->M));
+  ctx->launches += 2;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;
 }
@@ -227,7 +251,8 @@ ard_status ard_rows_create(ard_ctx* ctx, ard_rows** out, int M, int region_rows)
   r->d_hdr = nullptr; r->d_idx = nullptr; r->d_flag = nullptr; r->d_P = nullptr;
   // one allocation: header | kept list (padded to 64 entries: the products read whole 64-row blocks of it) | P | flags
   const size_t n_idx = ((size_t)M + 63) / 64 * 64 + 64;
-  const size_t bytes = sizeof(int32_t) * (HDR_WORDS + n_idx) + sizeof(uint32_t) * r->regions + (size_t)M;
+  const size_t n_cta = ((size_t)M + 2047) / 2048;
+  const size_t bytes = sizeof(int32_t) * (HDR_WORDS + 2 * n_idx + n_cta) + sizeof(uint32_t) * r->regions + (size_t)M;
   char* base = nullptr;
   if (cudaMalloc(reinterpret_cast<void**>(&base), bytes) != cudaSuccess) {
     delete r;
@@ -236,7 +261,9 @@ ard_status ard_rows_create(ard_ctx* ctx, ard_rows** out, int M, int region_rows)
   cudaMemset(base, 0, bytes);
   r->d_hdr = reinterpret_cast<int32_t*>(base);
   r->d_idx = r->d_hdr + HDR_WORDS;
-  r->d_P = reinterpret_cast<uint32_t*>(r->d_idx + n_idx);
+  r->d_stage = r->d_idx + n_idx;
+  r->d_counts = r->d_stage + n_idx;
+  r->d_P = reinterpret_cast<uint32_t*>(r->d_counts + n_cta);
   r->d_flag = reinterpret_cast<uint8_t*>(r->d_P + r->regions);
   *out = r;
   return ARD_OK;
