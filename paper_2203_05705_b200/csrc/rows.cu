@@ -45,17 +45,24 @@ __global__ void __launch_bounds__(256) sensitivity_kernel(const T* A, int lda, i
   const unsigned long long size = (unsigned long long)x * (unsigned long long)Kc;
   const int blocks = (samples + 3) >> 2;
   int count = 0;
+  // The entries are scattered over the region (one 32-byte sector per sample), so the loop is bound by how
+  // many loads are in flight: the four loads of a block are issued before any is compared, two blocks per pass.
+#pragma unroll 2
   for (int q = lane; q < blocks; q += 32) {
     uint32_t c[4] = {(uint32_t)iteration, (uint32_t)(iteration >> 32), (uint32_t)g, (stream_id << 16) | (uint32_t)q};
     philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+    float v[4];
 #pragma unroll
     for (int w = 0; w < 4; ++w) {
-      if (4 * q + w >= samples) break;
-      const unsigned long long pos = ((unsigned long long)c[w] * size) >> 32;
-      const long long row = (long long)g * x + (long long)(pos / (unsigned long long)Kc);
-      const int col = (int)(pos % (unsigned long long)Kc);
-      if (row < M && val_f<T>(A[(size_t)row * lda + col]) > threshold) ++count;
+      const unsigned int pos = (unsigned int)(((unsigned long long)c[w] * size) >> 32);  // < x*Kc < 2^32
+      const unsigned int roff = pos / (unsigned int)Kc;
+      const long long row = (long long)g * x + roff;
+      const int col = (int)(pos - roff * (unsigned int)Kc);
+      const bool in = 4 * q + w < samples && row < M;
+      v[w] = in ? val_f<T>(A[(size_t)row * lda + col]) : -INFINITY;  // nothing exceeds the threshold there
     }
+#pragma unroll
+    for (int w = 0; w < 4; ++w) count += v[w] > threshold ? 1 : 0;
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) count += __shfl_xor_sync(0xffffffffu, count, o);
@@ -289,6 +296,7 @@ ard_status ard_sensitivity_predict(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype
   const double sd = floor(k_frac * (double)rows->x * (double)Kc + 0.5);
   const long long samples = sd < 1.0 ? 1 : (long long)sd;
   if ((samples + 3) / 4 > 65535) return ARD_ERR_UNSUPPORTED;  // the block index shares a counter word with the stream id
+  if ((double)rows->x * (double)Kc >= 4294967296.0) return ARD_ERR_UNSUPPORTED;  // positions are 32-bit
   const double nd = ceil(t_frac * (double)samples - 1e-9);
   const int need = nd < 1.0 ? 1 : (int)nd;
   DevGuard guard(ctx->device);
