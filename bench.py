@@ -6,9 +6,12 @@ then the forward, backward-data and backward-weight GEMMs of the layer over the 
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-Prints ONE JSON line (rank 0).  Workload `mlp8192_row` is the large MLP layer of the paper's
+Prints ONE JSON line (rank 0).  Workload `mlp8192_row` (the default) is the large MLP layer of the paper's
 Table-1 sweep scaled to B200: W 8192x8192 bf16, batch 4096, row pattern, p = 0.5, K = the
-maximum-entropy distribution over periods 1..16.
+maximum-entropy distribution over periods 1..16.  Other workloads (`--workload`): `mlp8192_tile`,
+`mlp4096_tile`, `mlp2048_row` (single layers), `lstm1024` (a step is a whole sequence, forward + BPTT),
+`mlp2048_step` / `mlp8192_step` (a step is a whole training iteration of a stack of layers, replayed from a
+CUDA graph), `conv_rows` (a convolution layer as an im2col product with rows dropped by predicted sensitivity).
 """
 from __future__ import annotations
 
