@@ -768,7 +768,10 @@ static ard_status bwd_weight_impl(ard_ctx* ctx, const ard_pattern* pat, const ar
     st = get_maps(ctx, dyc, B, N, ldc, N, MAP_COMPACT_COLS, pat->dp_bound, 64, 64, &t.mapA, dense, dense_ld);
     t.mapA_indexed = 1;
   } else {
-    if (zero_fill_dropped) ARD_CUDA_OK(cudaMemset2DAsync(dW, (size_t)lddw * es_out, 0, (size_t)K * es_out, N, s));
+    if (zero_fill_dropped) {
+      st = launch_zero_dropped_tiles(ctx, pat, dW, lddw, es_out, s);
+      if (st != ARD_OK) return st;
+    }
     st = get_maps(ctx, dY, B, N, lddy, 0, MAP_PLAIN, 0, 64, 64, &t.mapA);
     t.mapA_indexed = 0;
   }

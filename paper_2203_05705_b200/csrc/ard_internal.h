@@ -212,6 +212,9 @@ ard_status launch_rows_sample(ard_ctx* ctx, ard_rows* rows, uint64_t seed, uint6
 ard_status launch_zero_dropped_rows(ard_ctx* ctx, const ard_rows* rows, void* out, int ld_bytes, int row_bytes,
                                     cudaStream_t s);
 
+ard_status launch_zero_dropped_tiles(ard_ctx* ctx, const ard_pattern* pat, void* dW, int lddw, int elem_bytes,
+                                     cudaStream_t s);
+
 // Layer-step helpers (aux_kernels.cu); elem_bytes 2 or 4.
 ard_status launch_compact_weight_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* hdr_in, const void* W, int ldw,
                                       void* Wk, int ldwk, int N, int K, int elem_bytes, cudaStream_t s);

@@ -387,6 +387,37 @@ __global__ void __launch_bounds__(256) bias_grad_wide_kernel(const int32_t* hdr,
   }
 }
 
+// Tile patterns, backward-weight: the dropped tiles of dW are zero (Sec. 3.2).  One CTA per dropped tile
+// (kept tiles are written by the product and skipped here), so a dense pattern costs nothing and a
+// pattern of period dp writes (dp-1)/dp of dW instead of all of it.
+__global__ void __launch_bounds__(256) zero_dropped_tiles_kernel(const int32_t* hdr, void* dW, int lddw, int ts, int Tr,
+                                                                 int Tc, int elem_bytes) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
+  if (dp == 1) return;
+  const int row_bytes = ts * elem_bytes;
+  const bool wide = (row_bytes & 15) == 0 && (((size_t)lddw * elem_bytes) & 15) == 0 && (reinterpret_cast<uintptr_t>(dW) & 15) == 0;
+  for (int lin = blockIdx.x; lin < Tr * Tc; lin += gridDim.x) {
+    if (lin >= bb && (lin - bb) % dp == 0) continue;  // kept
+    const int r = lin / Tc, c = lin - r * Tc;         // tile-row along the fan-in, tile-column along the neurons
+    char* base = reinterpret_cast<char*>(dW) + ((size_t)c * ts * lddw + (size_t)r * ts) * elem_bytes;
+    if (wide) {
+      const int per_row = row_bytes >> 4;
+      for (int e = threadIdx.x; e < ts * per_row; e += 256) {
+        const int n = e / per_row, q = e - n * per_row;
+        *reinterpret_cast<uint4*>(base + (size_t)n * lddw * elem_bytes + (size_t)q * 16) = make_uint4(0, 0, 0, 0);
+      }
+    } else {
+      const int per_row = row_bytes >> 1;
+      for (int e = threadIdx.x; e < ts * per_row; e += 256) {
+        const int n = e / per_row, q = e - n * per_row;
+        *reinterpret_cast<uint16_t*>(base + (size_t)n * lddw * elem_bytes + (size_t)q * 2) = 0;
+      }
+    }
+  }
+}
+
 }  // namespace
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,
@@ -518,6 +549,18 @@ ard_status launch_bias_grad(ard_ctx* ctx, const int32_t* hdr, const void* dZ, in
   else
     ARD_CUDA_OK(ard_launch(ctx, bias_grad_kernel<float>, grid, dim3(256), 0, s, hdr, (const float*)dZ, lddz,
                            dz_is_compact, B, N, db, zero_fill));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+ard_status launch_zero_dropped_tiles(ard_ctx* ctx, const ard_pattern* pat, void* dW, int lddw, int elem_bytes,
+                                     cudaStream_t s) {
+  const int tiles = pat->Tr * pat->Tc;
+  if (tiles == 0) return ARD_OK;
+  const int grid = tiles < ctx->sm_count * 32 ? tiles : ctx->sm_count * 32;
+  ARD_CUDA_OK(ard_launch(ctx, zero_dropped_tiles_kernel, dim3(grid), dim3(256), 0, s, (const int32_t*)pat->d_hdr, dW, lddw,
+                         pat->ts, pat->Tr, pat->Tc, elem_bytes));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;
