@@ -110,3 +110,17 @@ def test_host_side_distribution_search_matches_the_oracle(built):
             ard.ard_search_distribution(*args)
     with pytest.raises(ard.ArdError):
         ard.ard_search_distribution(0.5, 16, lam=0.0)
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 on its own (no C++ or CUDA types)."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no gcc")
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "ard.h"\nint main(void) { ard_mlp_layer l; ard_status s = ARD_OK; (void)l; return (int)s; }\n')
+    r = subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-I",
+                        os.path.join(ROOT, "include"), str(src)], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
