@@ -46,15 +46,24 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
            cudaStreamWaitEvent(waiter, ctx->ev[slot], 0) == cudaSuccess;
   };
   // ---- patterns of this iteration (stream id = layer index + 1) ----
+  // With several streams only the first layer's pattern is drawn on the caller's stream (its product is the
+  // first thing that stream runs); the others are drawn on the second stream, ahead of the compactions that
+  // need them.  The draws stay ordered (they share the iteration counter, the last one advances it).
   for (int l = 0; l < n_layers; ++l) {
-    if (!layers[l].sample) continue;
+    if (!layers[l].sample || (two && l > 0)) continue;
     st = ard_sample_pattern_counter(ctx, layers[l].pat, dist_id, seed, iteration_base, iteration_counter,
                                     l == last_sampled, (uint32_t)(l + 1), cuda_stream);
     if (st != ARD_OK) return st;
   }
   // ---- forward ----
-  if (!after(side_s, main_s, 0)) return ARD_ERR_CUDA;  // fork: the second stream starts behind the samplers
+  if (!after(side_s, main_s, 0)) return ARD_ERR_CUDA;  // fork: the second stream starts behind the first sampler
   if (two) {
+    for (int l = 1; l < n_layers; ++l) {
+      if (!layers[l].sample) continue;
+      st = ard_sample_pattern_counter(ctx, layers[l].pat, dist_id, seed, iteration_base, iteration_counter,
+                                      l == last_sampled, (uint32_t)(l + 1), side);
+      if (st != ARD_OK) return st;
+    }
     for (int l = 1; l < n_layers; ++l) {  // all weight compactions, beside the first layer's product
       const ard_mlp_layer& y = layers[l];
       st = ard_compact_weight_cols(ctx, y.pat, layers[l - 1].pat, dt, y.K, y.N, y.W, y.ldw, y.Wk, y.ldw, side);
