@@ -935,11 +935,14 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
         const int n = oc + (ch & 1) * 32;      // output column of this chunk
         float v[32];
         if (FUSED && MODE == M_ROW_FWD) {
-          // layer step: bias of the original neuron, activation, rescale (Sec. 3.2, last paragraph)
+          // layer step: bias of the original neuron, activation, rescale (Sec. 3.2, last paragraph).
+          // Lane l fetches the bias of column n + l once; the row loop takes it from there by shuffle (32
+          // loads per thread and chunk otherwise, all of them on the critical path of a single-wave launch).
+          float bl = 0.f;
+          if (p.bias != nullptr && n + lane < sch.n_keep) bl = __ldg(p.bias + bb + (n + lane) * dp);
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            float z = has_acc ? __uint_as_float(r[i]) : 0.f;
-            if (p.bias != nullptr && n + i < sch.n_keep) z += __ldg(p.bias + bb + (n + i) * dp);
+            float z = (has_acc ? __uint_as_float(r[i]) : 0.f) + __shfl_sync(0xffffffffu, bl, i);
             if (p.relu) z = fmaxf(z, 0.f);
             v[i] = p.alpha * z;
           }
