@@ -236,9 +236,11 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
  *
  * where, with in_pat, X [B][n_in], act_prev [B][n_in] and dX [B][n_in] are COMPACT over the feeding
  * layer's kept neurons (column i = its i-th kept neuron; leading dimensions >= K so that any pattern
- * fits) and Wk / dWk [N][K-wide rows] hold, in row keep[j], the fan-in weights of those kept neurons
- * in columns 0..n_in-1: Wk is made from W by ard_compact_weight_cols once per iteration, dWk is
- * expanded into dW by ard_expand_weight_grad_cols.  Without in_pat, Wk = W, dWk = dW and X is full
+ * fits) and Wk / dWk are PACKED in both dimensions: row j holds the j-th kept neuron of `pat`, column i
+ * the weight from the i-th kept neuron of the feeding layer (buffers of [N][K-wide rows] so that any
+ * pair of patterns fits): Wk is made from W by ard_compact_weight_cols once per iteration, dWk is
+ * expanded into dW by ard_expand_weight_grad_cols; in the formulas above read Wk[j][i] for
+ * Wk[keep[j]][i].  Without in_pat, Wk = W, dWk = dW (rows at the neurons' own positions) and X is full
  * width.  dZ is the gradient of the pre-activations Z = X Wk + bias (compact [B][n] when the compact
  * bit is set).  To chain layers, call ard_layer_bwd_data of layer l+1 with alpha = alpha_l and
  * act_prev = A_l: its result is dZ_l, compact, which layer l's backward calls take with alpha = 1.
@@ -246,8 +248,8 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
  * operand element type.  The output modes and flags are those of ard_fwd / ard_bwd_data /
  * ard_bwd_weight (ARD_OUT_COMPACT, ARD_OUT_SCATTER_ZEROFILL, ARD_FLAG_OUT_F32; ARD_FLAG_RELU selects
  * act = ReLU, otherwise the identity); ARD_FLAG_ACCUMULATE cannot be combined with bias, ReLU or
- * act_prev.  With zero_fill_dropped, ard_layer_bwd_weight zeroes the rows of dropped neurons in
- * columns 0..n_in-1 of dWk.  Tensor-core path: bf16, aligned as for ard_fwd, act_prev 16-byte
+ * act_prev.  zero_fill_dropped applies without in_pat only (a packed dWk has no rows of dropped neurons:
+ * ARD_ERR_INVALID_ARG if both are given; the expansion writes the zeros of dW).  Tensor-core path: bf16, aligned as for ard_fwd, act_prev 16-byte
  * aligned with ldact % 8 == 0; otherwise (and for ARD_F32) the CUDA-core path runs the same step. */
 ard_status ard_layer_fwd(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype, int B, int K,
                          int N, float alpha, const void* X, int ldx, const void* Wk, int ldw, const float* bias,
@@ -260,12 +262,12 @@ ard_status ard_layer_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, const ard_
                                 ard_dtype dW_dtype, int B, int K, int N, float alpha, const void* X, int ldx,
                                 const void* dZ, int lddz, int dz_is_compact, void* dWk, int lddw,
                                 int zero_fill_dropped, void* cuda_stream);
-/* Wk[n][i] = W[n][keep_in[i]] for the kept neurons n of `pat` and i < n_in; columns n_in up to the next
- * multiple of 64 (bounded by ldwk) are written as zero; rows of dropped neurons are not touched.
- * W, Wk [N][K-wide rows] of element type `dtype`, ldw, ldwk >= K, W != Wk. */
+/* Wk[j][i] = W[keep[j]][keep_in[i]] for j < n, i < n_in; columns n_in up to the next multiple of 64
+ * (bounded by ldwk) and rows n up to the next multiple of 64 (bounded by N) are written as zero, nothing
+ * else is touched.  W, Wk [N][K-wide rows] of element type `dtype`, ldw, ldwk >= K, W != Wk. */
 ard_status ard_compact_weight_cols(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
                                    int K, int N, const void* W, int ldw, void* Wk, int ldwk, void* cuda_stream);
-/* dW[n][keep_in[i]] = dWk[n][i] for the kept neurons n and i < n_in.  zero_fill != 0: every other entry
+/* dW[keep[j]][keep_in[i]] = dWk[j][i] for j < n and i < n_in.  zero_fill != 0: every other entry
  * of dW [N][K] (dropped neurons, dropped inputs) is written as zero; otherwise it is left untouched. */
 ard_status ard_expand_weight_grad_cols(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
                                        int K, int N, const void* dWk, int lddwk, void* dW, int lddw, int zero_fill,

@@ -574,10 +574,11 @@ static ard_status fwd_impl(ard_ctx* ctx, const ard_pattern* pat, const ard_patte
     t.mapA_indexed = 0;
   }
   if (st != ARD_OK) return st;
-  if (pat->kind == ARD_ROW) {
+  if (pat->kind == ARD_ROW && !in_pat) {
     st = get_maps(ctx, W, N, K, ldw, N, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64, &t.mapB);
     t.mapB_indexed = 1;
   } else {
+    // tile patterns; or the weight packed by ard_compact_weight_cols: its kept rows are rows 0..n_keep-1
     st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);
     t.mapB_indexed = 0;
   }
@@ -688,8 +689,13 @@ static ard_status bwd_data_impl(ard_ctx* ctx, const ard_pattern* pat, const ard_
     st = get_maps(ctx, dyc, B, N, ldc, N, MAP_COMPACT_COLS, pat->dp_bound, 128, 64, &t.mapA, dense, dense_ld);
     if (st != ARD_OK) return st;
     t.mapA_indexed = 1;
-    st = get_maps(ctx, W, N, K, ldw, N, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64, &t.mapB);
-    t.mapB_indexed = 1;
+    if (in_pat) {  // packed weight: rows 0..n_keep-1 (zero rows up to the next multiple of 64)
+      st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);
+      t.mapB_indexed = 0;
+    } else {
+      st = get_maps(ctx, W, N, K, ldw, N, MAP_STRIDED_ROWS, pat->dp_bound, 64, 64, &t.mapB);
+      t.mapB_indexed = 1;
+    }
   } else {
     st = get_maps(ctx, dY, B, N, lddy, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);
     if (st != ARD_OK) return st;
@@ -742,6 +748,7 @@ static ard_status bwd_weight_impl(ard_ctx* ctx, const ard_pattern* pat, const ar
   g.flag1 = zero_fill_dropped ? 1 : 0;
   g.out_is_f32 = dW_dtype == ARD_F32;
   g.hdr_in = in_pat ? in_pat->d_hdr : nullptr;
+  if (in_pat && zero_fill_dropped) return ARD_ERR_INVALID_ARG;  // the packed gradient has no rows of dropped neurons
   // Empty batch: the gradient of every kept weight is zero; the CUDA-core kernel writes exactly that.
   if (B == 0) return launch_gemm_cc(ctx, pat->kind, OP_BWD_WEIGHT, dtype, g, pat->ts, s);
 

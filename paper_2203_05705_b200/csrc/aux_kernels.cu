@@ -169,29 +169,34 @@ lstm_gates_bwd_kernel(const int32_t* hdr, int B, int H, float alpha,
 // ---- layer-step helpers (Sec. 3.1: the weight is compacted along the fan-in too when the layer that
 // feeds it ran under a row pattern) -----------------------------------------------------------------
 //
-// Wk[n][j] = W[n][b_in-1 + j*dp_in] for the kept neurons n of `hdr` and j < n_in; columns n_in up to the
-// next multiple of 64 (or ldwk) are written as zero, so that the last 64-wide contraction block of the
-// tensor-core forward product multiplies zeros.  Eight outputs per thread (one 16- or 32-byte store).
+// Wk[j][i] = W[keep[j]][keep_in[i]], compact in both dimensions (row j = j-th kept neuron of `hdr`, i < n_in).
+// Columns n_in up to the next multiple of 64 (or ldwk) and rows n_keep up to the next multiple of 64 (or N)
+// are written as zero, so that the last 64-deep contraction block of the forward and of the backward-data
+// product multiplies zeros.  Rows are packed (and not left at their neuron's position) because the products
+// read them in boxes of 64 rows: with a period of 8 and a 16 KiB pitch the rows of a box would be 128 KiB
+// apart, which halves the speed of the box loads.  Eight outputs per thread (one 16- or 32-byte store).
 template <typename T>
 __global__ void __launch_bounds__(256) compact_weight_cols_kernel(const int32_t* hdr,
                                                                   const int32_t* hdr_in,
                                                                   const T* W, int ldw, T* Wk,
-                                                                  int ldwk, int vec_ok) {
+                                                                  int ldwk, int N, int vec_ok) {
   pdl_launch_dependents();
   pdl_wait_prior_grids();
   const int n_keep = hdr[HDR_NKEEP], dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
   const int n_in = hdr_in[HDR_NKEEP], dpi = hdr_in[HDR_DP], bi = hdr_in[HDR_B] - 1;
   const int padded = min(ldwk, (n_in + 63) / 64 * 64);
+  const int rows_padded = min(N, (n_keep + 63) / 64 * 64);
   const int groups = (padded + 7) / 8;
-  for (int i = blockIdx.y; i < n_keep; i += gridDim.y) {
+  for (int i = blockIdx.y; i < rows_padded; i += gridDim.y) {
+    const bool real = i < n_keep;
     const size_t row = (size_t)bb + (size_t)i * dp;
-    const T* src = W + row * ldw + bi;
-    T* dst = Wk + row * ldwk;
+    const T* src = W + (real ? row : 0) * ldw + bi;
+    T* dst = Wk + (size_t)i * ldwk;
     for (int g = blockIdx.x * 256 + threadIdx.x; g < groups; g += gridDim.x * 256) {
       const int j0 = g * 8;
       __align__(16) T v[8];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) v[q] = (j0 + q < n_in) ? src[(size_t)(j0 + q) * dpi] : T(0.f);
+      for (int q = 0; q < 8; ++q) v[q] = (real && j0 + q < n_in) ? src[(size_t)(j0 + q) * dpi] : T(0.f);
       if (vec_ok && j0 + 8 <= padded) {
         if (sizeof(T) == 2) {
           *reinterpret_cast<uint4*>(dst + j0) = *reinterpret_cast<const uint4*>(v);
@@ -208,7 +213,7 @@ __global__ void __launch_bounds__(256) compact_weight_cols_kernel(const int32_t*
   }
 }
 
-// The inverse for the gradient: dW[n][b_in-1 + j*dp_in] = dWk[n][j] for kept neurons n; with zero_fill
+// The inverse for the gradient: dW[keep[j]][keep_in[i]] = dWk[j][i]; with zero_fill
 // every other entry of dW [N][K] (dropped neurons, dropped inputs) is written as zero, without it they
 // are left alone.  One output row per blockIdx.y step, consecutive threads write consecutive columns.
 template <typename T>
@@ -224,7 +229,7 @@ __global__ void __launch_bounds__(256) expand_weight_grad_cols_kernel(const int3
   for (int n = blockIdx.y; n < N; n += gridDim.y) {
     const bool kept_row = n >= bb && (n - bb) % dp == 0;
     if (!kept_row && !zero_fill) continue;
-    const T* src = dWk + (size_t)n * lddwk;
+    const T* src = dWk + (size_t)(kept_row ? (n - bb) / dp : 0) * lddwk;  // packed row of this neuron
     T* dst = dW + (size_t)n * lddw;
     for (int k = blockIdx.x * 256 + threadIdx.x; k < K; k += gridDim.x * 256) {
       const bool kept = kept_row && k >= bi && (k - bi) % dpi == 0;
@@ -278,7 +283,7 @@ __global__ void __launch_bounds__(256) expand_weight_grad_cols_wide_kernel(const
   for (int n = blockIdx.y; n < N; n += gridDim.y) {
     const bool kept_row = n >= bb && (n - bb) % dp == 0;
     if (!kept_row && !zero_fill) continue;
-    const T* src = dWk + (size_t)n * lddwk;
+    const T* src = dWk + (size_t)(kept_row ? (n - bb) / dp : 0) * lddwk;  // packed row of this neuron
     T* dst = dW + (size_t)n * lddw;
     for (int g = blockIdx.x * 256 + threadIdx.x; g < groups; g += gridDim.x * 256) {
       const int k0 = g * 8;
@@ -485,10 +490,10 @@ ard_status launch_compact_weight_cols(ard_ctx* ctx, const int32_t* hdr, const in
   dim3 grid((K / 8 + 255) / 256 > 0 ? (K / 8 + 255) / 256 : 1, N < 65535 ? N : 65535);
   if (elem_bytes == 2)
     ARD_CUDA_OK(ard_launch(ctx, compact_weight_cols_kernel<__nv_bfloat16>, grid, dim3(256), 0, s, hdr, hdr_in,
-                           (const __nv_bfloat16*)W, ldw, (__nv_bfloat16*)Wk, ldwk, vec_ok));
+                           (const __nv_bfloat16*)W, ldw, (__nv_bfloat16*)Wk, ldwk, N, vec_ok));
   else
     ARD_CUDA_OK(ard_launch(ctx, compact_weight_cols_kernel<float>, grid, dim3(256), 0, s, hdr, hdr_in, (const float*)W,
-                           ldw, (float*)Wk, ldwk, vec_ok));
+                           ldw, (float*)Wk, ldwk, N, vec_ok));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;

@@ -118,8 +118,9 @@ __global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts)
       if (gn < N && gk < nk) {
         size_t off;
         if (KIND == 0) {
-          if (OP == OP_FWD) off = (size_t)g.idx[gn] * g.lda1 + gk;
-          else if (OP == OP_BWD_DATA) off = (size_t)g.idx[gk] * g.lda1 + gn;
+          // with a feeding pattern the weight is packed in both dimensions (row j = j-th kept neuron)
+          if (OP == OP_FWD) off = (size_t)(g.hdr_in != nullptr ? gn : g.idx[gn]) * g.lda1 + gk;
+          else if (OP == OP_BWD_DATA) off = (size_t)(g.hdr_in != nullptr ? gk : g.idx[gk]) * g.lda1 + gn;
           else off = (size_t)gk * g.lda1 + gn;
         } else {
           const size_t kidx = (OP == OP_BWD_WEIGHT) ? (size_t)gk : (size_t)klist[gk / ts] * ts + gk % ts;
@@ -152,7 +153,7 @@ __global__ void __launch_bounds__(CC_THREADS) gemm_cc_kernel(GemmArgs g, int ts)
       if (m >= M || n >= N) continue;
       size_t off;
       if (KIND == 0 && OP == OP_FWD) off = (size_t)m * g.ldo + (g.flag0 == ARD_OUT_SCATTER_ZEROFILL ? g.idx[n] : n);
-      else if (KIND == 0 && OP == OP_BWD_WEIGHT) off = (size_t)g.idx[m] * g.ldo + n;
+      else if (KIND == 0 && OP == OP_BWD_WEIGHT) off = (size_t)(g.hdr_in != nullptr ? m : g.idx[m]) * g.ldo + n;
       else off = (size_t)m * g.ldo + n;
       float v = acc[i][j];
       if (KIND == 0 && OP == OP_FWD) {
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(256) skinny_fwd_kernel(GemmArgs g) {
   for (int n = 0; n < SKINNY_N; ++n) acc[n] = 0.f;
   int rows[SKINNY_N];
 #pragma unroll
-  for (int n = 0; n < SKINNY_N; ++n) rows[n] = n < n_keep ? g.idx[n] : 0;
+  for (int n = 0; n < SKINNY_N; ++n) rows[n] = n < n_keep ? (g.hdr_in != nullptr ? n : g.idx[n]) : 0;
   for (int k = threadIdx.x; k < kin; k += 256) {
     const float x = to_f<T>(X[k]);
 #pragma unroll
@@ -265,7 +266,7 @@ __global__ void __launch_bounds__(256) skinny_bwd_weight_kernel(GemmArgs g) {
     float v = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) v += part[w][n][c];
-    store_out(g.out, (size_t)g.idx[n] * g.ldo + kk, g.alpha * v, g.out_is_f32, g.accumulate);
+    store_out(g.out, (size_t)(g.hdr_in != nullptr ? n : g.idx[n]) * g.ldo + kk, g.alpha * v, g.out_is_f32, g.accumulate);
   }
   if (g.flag1) {
     // rows of dropped neurons, this CTA's 32 columns

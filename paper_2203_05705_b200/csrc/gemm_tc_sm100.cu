@@ -912,6 +912,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
       if (MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_WEIGHT) {
         row_ok = m < sch.M_gemm;
         out_row = (long long)bb + (long long)m * dp;
+        if (FUSED && MODE == M_ROW_BWD_WEIGHT && p.hdr_in != nullptr) out_row = m;  // packed gradient rows
         if (MODE == M_LSTM_BWD_WEIGHT) out_row += ti.out_row0;
       } else if (MODE == M_ROWS_FWD || MODE == M_ROWS_BWD_DATA) {
         row_ok = m < sch.M_gemm;

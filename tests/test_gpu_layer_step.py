@@ -64,12 +64,12 @@ def test_every_layer_step_call_matches_the_oracle(path, dtype, B, K, N):
             # ---- weight compaction along the fan-in ----
             Wk = torch.full((N, K), float("nan"), dtype=tdtype(dtype), device="cuda")
             ard.ard_compact_weight_cols(ctx.h, pat, in_pat, dtype, K, N, Wd, K, Wk, K)
-            Wkh = host(Wk)
-            assert np.array_equal(Wkh[np.ix_(keep, np.arange(n_in))], W.T.astype(np.float64)[np.ix_(keep, keep_in)]), tag
-            pad = min(K, (n_in + 63) // 64 * 64)
-            assert np.all(Wkh[keep][:, n_in:pad] == 0), tag
+            Wkh = host(Wk)                                         # packed in both dimensions
+            assert np.array_equal(Wkh[:n, :n_in], W.T.astype(np.float64)[np.ix_(keep, keep_in)]), tag
+            pad, pad_rows = min(K, (n_in + 63) // 64 * 64), min(N, (n + 63) // 64 * 64)
+            assert np.all(Wkh[:n, n_in:pad] == 0) and np.all(Wkh[n:pad_rows, :pad] == 0), tag
+            assert np.all(np.isnan(Wkh[pad_rows:])) and np.all(np.isnan(Wkh[:, pad:])), tag   # nothing else is touched
             dropped = np.setdiff1d(np.arange(N), keep)
-            assert np.all(np.isnan(Wkh[dropped])), tag             # rows of dropped neurons are not touched
 
             # ---- forward: compact input, bias, ReLU; compact and full-width output ----
             Xc = _rnd(rng, (B, n_in), dtype)
@@ -109,15 +109,15 @@ def test_every_layer_step_call_matches_the_oracle(path, dtype, B, K, N):
             # ---- backward-weight on compact operands, expansion, bias gradient ----
             dWc_ref, db_ref, _ = OM.layer_bwd_compact(Xc, keep_in, W, keep, dZc)       # [n_in x n], [n]
             dWk = torch.full((N, K), float("nan"), dtype=torch.float32, device="cuda")
-            ard.ard_layer_bwd_weight(ctx.h, pat, in_pat, dtype, ard.ARD_F32, B, K, N, 1.0, Xd, K, dZd, N, 1, dWk, K, 1)
-            dWkh = host(dWk)
-            assert OG.rel_fro(dWkh[np.ix_(keep, np.arange(n_in))], dWc_ref.T) <= tol, tag
-            assert np.all(dWkh[dropped][:, :n_in] == 0), tag
+            ard.ard_layer_bwd_weight(ctx.h, pat, in_pat, dtype, ard.ARD_F32, B, K, N, 1.0, Xd, K, dZd, N, 1, dWk, K, 0)
+            dWkh = host(dWk)                                       # packed like Wk
+            assert OG.rel_fro(dWkh[:n, :n_in], dWc_ref.T) <= tol, tag
+            assert np.all(np.isnan(dWkh[n:])) and np.all(np.isnan(dWkh[:, n_in:])), tag
             dW = torch.full((N, K), float("nan"), dtype=torch.float32, device="cuda")
             ard.ard_expand_weight_grad_cols(ctx.h, pat, in_pat, ard.ARD_F32, K, N, dWk, K, dW, K, 1)
             dWh = host(dW)
             full = np.zeros((N, K))
-            full[np.ix_(keep, keep_in)] = dWkh[np.ix_(keep, np.arange(n_in))]
+            full[np.ix_(keep, keep_in)] = dWkh[:n, :n_in]
             assert np.array_equal(dWh, full), tag
             db = torch.full((N,), float("nan"), dtype=torch.float32, device="cuda")
             ard.ard_bias_grad(ctx.h, pat, dtype, B, N, dZd, N, 1, db, 1)
