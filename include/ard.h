@@ -90,8 +90,10 @@ ard_status ard_set_path(ard_ctx* ctx, ard_path path);
  * gathering again (ard_bwd_data followed by ard_bwd_weight of the same layer then gather once).
  * Enable only if dY is not written between such calls.  Default: off. */
 ard_status ard_set_compact_reuse(ard_ctx* ctx, int enable);
-/* Tuning / test knob of the tensor-core path: forces the N extent of the output tile (64, 128 or
- * 256; 0 restores the built-in choice).  A forced value a product cannot use is ignored for it. */
+/* Tuning / test knob of the tensor-core path: forces the N extent of the output tile (a multiple of
+ * 32 from 64 to 256; 0 restores the built-in choice, which for row patterns picks the width with the
+ * fewest waves x time per tile on the device).  A forced value a product cannot use is ignored for
+ * it. */
 ard_status ard_set_tile_n(ard_ctx* ctx, int bn);
 /* Optional schedule of the tensor-core path for row patterns.  The output tiles of a product are
  * dealt to the SMs (or SM pairs) in waves.  With enable != 0, when the tile count leaves a partial

@@ -332,7 +332,7 @@ ard_status ard_set_lstm_persistent(ard_ctx* ctx, int enable) {
 }
 
 ard_status ard_set_tile_n(ard_ctx* ctx, int bn) {
-  if (!ctx || (bn != 0 && bn != 64 && bn != 128 && bn != 256)) return ARD_ERR_INVALID_ARG;
+  if (!ctx || (bn != 0 && (bn < 64 || bn > 256 || bn % 32 != 0))) return ARD_ERR_INVALID_ARG;
   ctx->force_bn = bn;
   return ARD_OK;
 }
@@ -736,7 +736,7 @@ static ard_status bwd_weight_impl(ard_ctx* ctx, const ard_pattern* pat, const ar
   if (dW_dtype != ARD_F32 && dW_dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
   if (dtype == ARD_F32 && dW_dtype != ARD_F32) return ARD_ERR_INVALID_ARG;
   if (dy_is_compact && pat->kind != ARD_ROW) return ARD_ERR_INVALID_ARG;
-  if (ldx < K || lddy < N || lddw < K) return ARD_ERR_SHAPE;
+  if (ldx < K || lddy < (dy_is_compact ? 1 : N) || lddw < K) return ARD_ERR_SHAPE;
   DeviceGuard guard(ctx->device);
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int es_out = dW_dtype == ARD_F32 ? 4 : 2;

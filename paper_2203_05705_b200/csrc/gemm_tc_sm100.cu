@@ -90,7 +90,7 @@ struct TcParams {
   int out_is_f32;
   int scatter;    // row fwd: full-width output with zero fill
   int zero_fill;  // row bwd-weight: write zeros to dropped rows
-  int force_bn;   // row modes: 0 = choose the N tile on the device, else 64 / 128 / 256
+  int force_bn;   // row modes: 0 = choose the N tile on the device, else a multiple of 32 in 64 .. 256
   int accumulate; // plain stores add to the existing output
   int band_m;     // M-tiles per raster band (0: one band)
   // Shared tiles (row modes): when the tile count is not a multiple of the worker count, the tiles
@@ -266,15 +266,23 @@ struct Sched {
         if (p.force_bn) {
           bn = p.force_bn;
         } else {
-          // Fewest (waves x time per tile).  Narrow tiles re-read the A operand more often and use
-          // narrower instructions: a 128-wide tile is charged 0.7 and a 64-wide one 0.55 of the time of
-          // a 256-wide tile (measured on dense problems).  Ties go to the wider tile.
+          // Fewest (waves x time per tile).  Narrow tiles re-read the A operand more often and use narrower
+          // instructions; the time of a tile relative to a 256-wide one, measured per wave on dense
+          // problems: pairs 0.92 / 0.83 / 0.78 / 0.76 at 224 / 192 / 160 / 128 columns, single CTAs 0.7 at
+          // 128 and 0.55 at 64.  Ties go to the wider tile.
+          // The forward products try every multiple of 32 columns (the instruction takes any multiple of
+          // 16; B still arrives in 64-row boxes, the last one partly unused).  Where B is read along its
+          // contiguous dimension (both backward products) only 256 / 128 / 64 keep every box on a 128-byte
+          // line; other widths were measured up to 20 % slower per tile there and are not tried.
           // Shared tiles cost each worker its share of their contraction plus some of the reduction.
+          constexpr bool FLEX = (MODE == M_ROW_FWD || MODE == M_ROWS_FWD);
           const int kt = (Kc + BK - 1) / BK;
           int best_cost = 0x7fffffff;
-          for (int cand = BN; cand >= 64 * CTAS; cand >>= 1) {
+          for (int cand = BN; cand >= 64 * CTAS; cand = FLEX ? cand - 32 : cand >> 1) {
             const int tiles = Mt * ((N_gemm + cand - 1) / cand);
-            const int w16 = 16 * (cand == 256 ? 100 : (cand == 128 ? 70 : 55));
+            const int wpair = cand == 256 ? 100 : (cand == 224 ? 92 : (cand == 192 ? 83 : (cand == 160 ? 78 : 76)));
+            const int wone = cand == 256 ? 100 : (cand == 128 ? 70 : (cand == 64 ? 55 : 40 + (60 * cand) / 256));
+            const int w16 = 16 * ((CTAS == 2 && FLEX) ? wpair : wone);
             const int full = tiles / workers, rem = tiles % workers;
             const int S = (SK_MODE && p.sk_ws != nullptr && kt > 0)
                               ? sharing_workers(full, rem, kt, workers, p.sk_min_blocks, p.sk_min_gain) : 0;
@@ -427,7 +435,7 @@ struct Sched {
     TileInfo ti = plain_tile(p, t);
     // affine block coordinates
     ti.bn = bn;
-    ti.nbox = bn / CTAS / 64;
+    ti.nbox = (bn / CTAS + 63) / 64;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       ti.bx[i] = ti.n0 + rank * (bn / CTAS) + 64 * i;

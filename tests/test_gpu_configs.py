@@ -125,7 +125,8 @@ def test_config5_sampled_outputs(kind, ts):
         dW = torch.empty((N, K), dtype=BF, device="cuda")
         rows = np.arange(7, B, B // 128)[:128]
         cols = np.arange(3, N, N // 128)[:128]
-        for dp, b in [(1, 1), (2, 2), (5, 3), (16, 7)]:
+        # periods 3, 5, 7, 12 make the forward product pick output tiles 224, 192, 160, 192 columns wide
+        for dp, b in [(1, 1), (2, 2), (3, 1), (5, 3), (7, 2), (12, 5), (16, 7)]:
             ard.ard_pattern_set(ctx.h, pat, dp, b)
             Y.fill_(float("nan")); dX.fill_(float("nan")); dW.fill_(float("nan"))
             ard.ard_fwd(ctx.h, pat, ard.ARD_BF16, B, K, N, 2.0, dXd, K, dWd, K, Y, N, ard.ARD_OUT_SCATTER_ZEROFILL)

@@ -29,7 +29,7 @@ def _layer(B, K, N, seed, wscale):
     return X, W, dY
 
 
-@pytest.mark.parametrize("bn", [128, 256, 64])
+@pytest.mark.parametrize("bn", [128, 256, 64, 224, 192, 160, 96])
 def test_row_tensor_core(ctx, bn):
     B, K, N = 300, 520, 1000
     X, W, dY = _layer(B, K, N, 1, 0.05)
