@@ -564,7 +564,8 @@ def run_mlp_step(args, wl):
 
 
 def run_conv_rows(args, wl):
-    """A step = sensitivity prediction + row sampling + the three products over the kept rows of the input matrix."""
+    """A step = sensitivity prediction + row sampling + gathering the kept rows of the input matrix and of the output
+    gradient + the three products on the gathered matrices (results filled back into the kept rows)."""
     import torch
     from paper_2203_05705_b200 import ard
     dev_index = int(os.environ.get("LOCAL_RANK", "0"))
@@ -585,8 +586,11 @@ def run_conv_rows(args, wl):
     hY = torch.empty((M, N), dtype=bf).pin_memory()
     ctx = ard.ard_create(0, 4096)
     rows = ard.ard_rows_create(ctx, M, x)
+    cap = (M + 63) // 64 * 64
+    Ak = torch.zeros((cap, K), dtype=bf, device="cuda")    # the dense small matrices of Sec. 5.2.1
+    dYk = torch.zeros((cap, N), dtype=bf, device="cuda")
 
-    def step(it, dense=False, host=False):
+    def step(it, dense=False, host=False, gathered=True):
         if host:
             A.copy_(hA, non_blocking=True)
             dY.copy_(hdY, non_blocking=True)
@@ -596,9 +600,19 @@ def run_conv_rows(args, wl):
             ard.ard_sensitivity_predict(ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["t_frac"], wl["threshold"],
                                         wl["m_prob"], wl["n_prob"], inputs.BASE_SEED, it, 0)
         ard.ard_rows_sample(ctx, rows, inputs.BASE_SEED, it, 0)
-        ard.ard_rows_fwd(ctx, rows, M, K, N, 1.0, A, K, W, K, Y, N)
-        ard.ard_rows_bwd_data(ctx, rows, M, K, N, 1.0, dY, N, W, K, dA, K)
-        ard.ard_rows_bwd_weight(ctx, rows, ard.ARD_BF16, M, K, N, 1.0, A, K, dY, N, dW, K)
+        if gathered:
+            # gather the kept rows once per operand, multiply dense, fill back; the gathered input serves the
+            # forward product and the weight gradient
+            ard.ard_rows_gather(ctx, rows, M, K, A, K, Ak, K)
+            ard.ard_rows_fwd_compact(ctx, rows, M, K, N, 1.0, Ak, K, W, K, Y, N)
+            ard.ard_rows_gather(ctx, rows, M, N, dY, N, dYk, N)
+            ard.ard_rows_bwd_data_compact(ctx, rows, M, K, N, 1.0, dYk, N, W, K, dA, K)
+            ard.ard_rows_bwd_weight_compact(ctx, rows, ard.ARD_BF16, M, K, N, 1.0, Ak, K, dYk, N, dW, K)
+        else:
+            # the producer warps of the GEMM kernel follow the list themselves
+            ard.ard_rows_fwd(ctx, rows, M, K, N, 1.0, A, K, W, K, Y, N)
+            ard.ard_rows_bwd_data(ctx, rows, M, K, N, 1.0, dY, N, W, K, dA, K)
+            ard.ard_rows_bwd_weight(ctx, rows, ard.ARD_BF16, M, K, N, 1.0, A, K, dY, N, dW, K)
         if host:
             hY.copy_(Y, non_blocking=True)
 
@@ -634,6 +648,21 @@ def run_conv_rows(args, wl):
     if not args.quick:
         n2 = max(5, steps // 4)
         detail["ms_per_step"]["own_kernels_all_rows"] = timed(lambda it: step(it, dense=True), n2, warm)[0] / n2
+        detail["ms_per_step"]["gather_inside_the_gemm_kernels"] = timed(lambda it: step(it, gathered=False), n2, warm)[0] / n2
+        # per stage, serialised (one stage per timed loop)
+        stage = {}
+        stage["sensitivity_predict"] = lambda it: ard.ard_sensitivity_predict(
+            ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["t_frac"], wl["threshold"], wl["m_prob"], wl["n_prob"],
+            inputs.BASE_SEED, 1, 0)
+        stage["rows_sample"] = lambda it: ard.ard_rows_sample(ctx, rows, inputs.BASE_SEED, 1, 0)
+        stage["gather_A"] = lambda it: ard.ard_rows_gather(ctx, rows, M, K, A, K, Ak, K)
+        stage["gather_dY"] = lambda it: ard.ard_rows_gather(ctx, rows, M, N, dY, N, dYk, N)
+        stage["fwd(+zero rows)"] = lambda it: ard.ard_rows_fwd_compact(ctx, rows, M, K, N, 1.0, Ak, K, W, K, Y, N)
+        stage["bwd_data(+zero rows)"] = lambda it: ard.ard_rows_bwd_data_compact(ctx, rows, M, K, N, 1.0, dYk, N, W, K, dA, K)
+        stage["bwd_weight"] = lambda it: ard.ard_rows_bwd_weight_compact(ctx, rows, ard.ARD_BF16, M, K, N, 1.0, Ak, K, dYk,
+                                                                         N, dW, K)
+        step(1)
+        detail["us_per_stage"] = {k: round(timed(f, n2, warm)[0] / n2 * 1e3, 1) for k, f in stage.items()}
 
         def torch_step(it):
             torch.matmul(A, W.t(), out=Y)

@@ -372,6 +372,27 @@ ard_status ard_rows_bwd_data(ard_ctx* ctx, const ard_rows* rows, int M, int K, i
 ard_status ard_rows_bwd_weight(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N, float alpha,
                                const void* A, int lda, const void* dY, int lddy, void* dW, int lddw,
                                void* cuda_stream);
+/* The same products through the dense, small matrices of Sec. 5.2.1 (step 2), for layers large enough that an
+ * extra pass over the kept rows pays: ard_rows_gather copies the kept rows of src [M][width] (ld_src) to the top
+ * of dst (ld_dst): row j of dst is row keep[j] of src, and the rows from n_keep up to the next multiple of 64 are
+ * zero.  dst must hold ceil(M / 64) * 64 rows (any list fits); bf16 elements, width a multiple of 8, 16-byte
+ * aligned pointers, leading dimensions multiples of 8.  The products then read their row operands (Ak = gathered
+ * A, dYk = gathered dY, both [ceil(M/64)*64][.]) with TMA like any dense matrix, take the number of rows from the
+ * list on the device and write forward / backward-data results back to rows keep[j] of Y / dA (dropped rows
+ * zero); the weight gradient's contraction runs over the list's rows and, having few output tiles and a long
+ * contraction, is cut along the contraction and shared by all SMs (fp32 partial sums added in a fixed order).
+ * A compact copy made for the forward product serves the weight gradient of the same iteration.  Results equal
+ * those of ard_rows_fwd / _bwd_data / _bwd_weight.  Same argument rules; asynchronous. */
+ard_status ard_rows_gather(ard_ctx* ctx, const ard_rows* rows, int M, int width, const void* src, int ld_src, void* dst,
+                           int ld_dst, void* cuda_stream);
+ard_status ard_rows_fwd_compact(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha, const void* Ak,
+                                int ldak, const void* W, int ldw, void* Y, int ldy, void* cuda_stream);
+ard_status ard_rows_bwd_data_compact(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha,
+                                     const void* dYk, int lddyk, const void* W, int ldw, void* dA, int ldda,
+                                     void* cuda_stream);
+ard_status ard_rows_bwd_weight_compact(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N,
+                                       float alpha, const void* Ak, int ldak, const void* dYk, int lddyk, void* dW,
+                                       int lddw, void* cuda_stream);
 /* Test / debug: synchronises; n_keep, the kept rows (at most idx_capacity) and the per-region integers
  * (ceil(M / region_rows) entries) to HOST buffers; idx and region_probability may be NULL. */
 ard_status ard_rows_to_host(const ard_rows* rows, int32_t* n_keep, int32_t* idx, size_t idx_capacity,

@@ -35,6 +35,7 @@ EXPORTS = [
     "ard_expand_weight_grad_cols", "ard_bias_grad", "ard_sample_pattern_counter", "ard_mlp_step",
     "ard_rows_create", "ard_rows_destroy", "ard_sensitivity_predict", "ard_rows_set_probability", "ard_rows_sample",
     "ard_rows_to_host", "ard_rows_fwd", "ard_rows_bwd_data", "ard_rows_bwd_weight",
+    "ard_rows_gather", "ard_rows_fwd_compact", "ard_rows_bwd_data_compact", "ard_rows_bwd_weight_compact",
 ]
 
 _lib = None
@@ -113,6 +114,10 @@ def lib():
         "ard_rows_fwd": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_rows_bwd_data": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_rows_bwd_weight": [vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_rows_gather": [vp, vp, i32, i32, vp, i32, vp, i32, vp],
+        "ard_rows_fwd_compact": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_rows_bwd_data_compact": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_rows_bwd_weight_compact": [vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -388,6 +393,26 @@ def ard_rows_bwd_data(ctx, rows, M, K, N, alpha, dY, lddy, W, ldw, dA, ldda, str
 def ard_rows_bwd_weight(ctx, rows, dW_dtype, M, K, N, alpha, A, lda, dY, lddy, dW, lddw, stream=None):
     _check(lib().ard_rows_bwd_weight(ctx, rows, dW_dtype, M, K, N, alpha, _ptr(A), lda, _ptr(dY), lddy, _ptr(dW), lddw,
                                      _stream(stream)), "ard_rows_bwd_weight")
+
+
+def ard_rows_gather(ctx, rows, M, width, src, ld_src, dst, ld_dst, stream=None):
+    _check(lib().ard_rows_gather(ctx, rows, M, width, _ptr(src), ld_src, _ptr(dst), ld_dst, _stream(stream)),
+           "ard_rows_gather")
+
+
+def ard_rows_fwd_compact(ctx, rows, M, K, N, alpha, Ak, ldak, W, ldw, Y, ldy, stream=None):
+    _check(lib().ard_rows_fwd_compact(ctx, rows, M, K, N, alpha, _ptr(Ak), ldak, _ptr(W), ldw, _ptr(Y), ldy,
+                                      _stream(stream)), "ard_rows_fwd_compact")
+
+
+def ard_rows_bwd_data_compact(ctx, rows, M, K, N, alpha, dYk, lddyk, W, ldw, dA, ldda, stream=None):
+    _check(lib().ard_rows_bwd_data_compact(ctx, rows, M, K, N, alpha, _ptr(dYk), lddyk, _ptr(W), ldw, _ptr(dA), ldda,
+                                           _stream(stream)), "ard_rows_bwd_data_compact")
+
+
+def ard_rows_bwd_weight_compact(ctx, rows, dW_dtype, M, K, N, alpha, Ak, ldak, dYk, lddyk, dW, lddw, stream=None):
+    _check(lib().ard_rows_bwd_weight_compact(ctx, rows, dW_dtype, M, K, N, alpha, _ptr(Ak), ldak, _ptr(dYk), lddyk,
+                                             _ptr(dW), lddw, _stream(stream)), "ard_rows_bwd_weight_compact")
 
 
 def ard_lstm_gate_gemm(ctx, pat, B, KH, H, XH, ldxh, W, ldw, Z, ldz_gate, stream=None):

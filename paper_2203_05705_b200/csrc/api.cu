@@ -1240,6 +1240,103 @@ ard_status ard_rows_bwd_weight(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_
   return launch_rows_tc(ctx, OP_BWD_WEIGHT, t, rows->d_idx, dY, lddy, A, lda, (cudaStream_t)cuda_stream);
 }
 
+// ---- the same products on compact operands (the dense small matrices of Sec. 5.2.1, step 2) ----------
+ard_status ard_rows_gather(ard_ctx* ctx, const ard_rows* rows, int M, int width, const void* src, int ld_src, void* dst,
+                           int ld_dst, void* cuda_stream) {
+  if (!ctx || !rows || rows->ctx != ctx || !src || !dst) return ARD_ERR_INVALID_ARG;
+  ctx->epoch++;
+  if (M != rows->M || width < 1 || ld_src < width || ld_dst < width) return ARD_ERR_SHAPE;
+  if (!aligned16(src) || !aligned16(dst) || width % 8 || ld_src % 8 || ld_dst % 8) return ARD_ERR_ALIGNMENT;
+  DeviceGuard guard(ctx->device);
+  return launch_rows_gather(ctx, rows, src, ld_src * 2, dst, ld_dst * 2, width * 2, (cudaStream_t)cuda_stream);
+}
+
+static int rows_capacity(int M) { return (M + 63) / 64 * 64; }
+
+ard_status ard_rows_fwd_compact(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha, const void* Ak,
+                                int ldak, const void* W, int ldw, void* Y, int ldy, void* cuda_stream) {
+  ard_status st = rows_check(ctx, rows, M, K, N, Ak, ldak, W, ldw, Y, ldy, 2);
+  if (st != ARD_OK) return st;
+  if (ldak < K || ldw < K || ldy < N) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  TcArgs t = {};
+  GemmArgs g = {};
+  g.hdr = rows->d_hdr;
+  g.B = M; g.K = K; g.N = N;
+  g.alpha = alpha;
+  g.out = Y; g.ldo = ldy;
+  g.flag0 = ARD_OUT_COMPACT;
+  g.status = ctx->d_status;
+  g.ext_mode = 1;
+  g.ridx = rows->d_idx;
+  st = get_maps(ctx, Ak, rows_capacity(M), K, ldak, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);  // [128 rows][64 k]
+  if (st != ARD_OK) return st;
+  st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);  // [64 neurons][64 k]
+  if (st != ARD_OK) return st;
+  t.g = g;
+  t.bn = ctx->force_bn;
+  st = launch_zero_dropped_rows(ctx, rows, Y, ldy * 2, N * 2, s);
+  if (st != ARD_OK) return st;
+  return launch_gemm_tc(ctx, ARD_ROW, OP_FWD, t, s);
+}
+
+ard_status ard_rows_bwd_data_compact(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha, const void* dYk,
+                                     int lddyk, const void* W, int ldw, void* dA, int ldda, void* cuda_stream) {
+  ard_status st = rows_check(ctx, rows, M, K, N, dYk, lddyk, W, ldw, dA, ldda, 2);
+  if (st != ARD_OK) return st;
+  if (lddyk < N || ldw < K || ldda < K) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  TcArgs t = {};
+  GemmArgs g = {};
+  g.hdr = rows->d_hdr;
+  g.B = M; g.K = K; g.N = N;
+  g.alpha = alpha;
+  g.out = dA; g.ldo = ldda;
+  g.flag0 = 1;
+  g.status = ctx->d_status;
+  g.ext_mode = 1;
+  g.ridx = rows->d_idx;
+  st = get_maps(ctx, dYk, rows_capacity(M), N, lddyk, 0, MAP_PLAIN, 0, 128, 64, &t.mapA);  // [128 rows][64 n]
+  if (st != ARD_OK) return st;
+  st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);  // read MN-major: [64 neurons][64 k]
+  if (st != ARD_OK) return st;
+  t.g = g;
+  t.bn = ctx->force_bn;
+  st = launch_zero_dropped_rows(ctx, rows, dA, ldda * 2, K * 2, s);
+  if (st != ARD_OK) return st;
+  return launch_gemm_tc(ctx, ARD_ROW, OP_BWD_DATA, t, s);
+}
+
+ard_status ard_rows_bwd_weight_compact(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N,
+                                       float alpha, const void* Ak, int ldak, const void* dYk, int lddyk, void* dW,
+                                       int lddw, void* cuda_stream) {
+  if (dW_dtype != ARD_F32 && dW_dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  ard_status st = rows_check(ctx, rows, M, K, N, Ak, ldak, dYk, lddyk, dW, lddw, dW_dtype == ARD_F32 ? 4 : 2);
+  if (st != ARD_OK) return st;
+  if (ldak < K || lddyk < N || lddw < K) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  TcArgs t = {};
+  GemmArgs g = {};
+  g.hdr = rows->d_hdr;
+  g.B = M; g.K = K; g.N = N;
+  g.alpha = alpha;
+  g.out = dW; g.ldo = lddw;
+  g.flag0 = 1;
+  g.out_is_f32 = dW_dtype == ARD_F32;
+  g.status = ctx->d_status;
+  g.ext_mode = 2;
+  // both operands read along the rows of the list: boxes [64 list rows][64 columns]
+  st = get_maps(ctx, dYk, rows_capacity(M), N, lddyk, 0, MAP_PLAIN, 0, 64, 64, &t.mapA);
+  if (st != ARD_OK) return st;
+  st = get_maps(ctx, Ak, rows_capacity(M), K, ldak, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);
+  if (st != ARD_OK) return st;
+  t.g = g;
+  t.bn = ctx->force_bn;
+  return launch_gemm_tc(ctx, ARD_ROW, OP_BWD_WEIGHT, t, (cudaStream_t)cuda_stream);
+}
+
 ard_status ard_last_device_status(ard_ctx* ctx, void* cuda_stream) {
   if (!ctx) return ARD_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);

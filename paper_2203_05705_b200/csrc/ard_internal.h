@@ -161,6 +161,11 @@ struct GemmArgs {
   int relu;           // forward: max(., 0) before the rescale
   const void* act;    // backward-data: the output is zeroed where act <= 0 (operand element type, layout of dX)
   int ldact;
+  // Row-list products on compact operands (Sec. 5.2.1): hdr is the row list's header, the layer is dense.
+  // ext_mode 1: hdr's count is the row extent of A and of the output, output row m goes to row ridx[m];
+  // ext_mode 2: hdr's count is the length of the contraction (weight gradient).
+  int ext_mode;
+  const int32_t* ridx;
 };
 
 enum GemmOp { OP_FWD = 0, OP_BWD_DATA = 1, OP_BWD_WEIGHT = 2 };
@@ -209,6 +214,8 @@ ard_status launch_sensitivity(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, con
 ard_status launch_fill_probability(ard_ctx* ctx, ard_rows* rows, uint32_t P, cudaStream_t s);
 ard_status launch_rows_sample(ard_ctx* ctx, ard_rows* rows, uint64_t seed, uint64_t iteration, uint32_t stream_id,
                               cudaStream_t s);
+ard_status launch_rows_gather(ard_ctx* ctx, const ard_rows* rows, const void* src, int ld_src_bytes, void* dst,
+                              int ld_dst_bytes, int row_bytes, cudaStream_t s);
 ard_status launch_zero_dropped_rows(ard_ctx* ctx, const ard_rows* rows, void* out, int ld_bytes, int row_bytes,
                                     cudaStream_t s);
 

@@ -116,6 +116,11 @@ struct TcParams {
   int ldgA;
   const __nv_bfloat16* gB;  // backward-weight: A
   int ldgB;
+  // Row-list products on compact operands (FUSED row kernels): hdr is the row list's header, the layer itself is
+  // dense.  1: the row extent of A and of the output is hdr[HDR_NKEEP] and output row m goes to row ridx[m]
+  // (forward, backward-data); 2: the contraction runs over hdr[HDR_NKEEP] rows (backward-weight).
+  int ext_mode;
+  int sk_any;  // shared tiles also when the tiles do not fill one wave (long contractions, few tiles)
 };
 
 // CTAS = 2: a cluster of two CTAs shares one 256 x BN output tile; each CTA stages its own 128 rows
@@ -195,28 +200,32 @@ struct Sched {
   // Workers that would share the `rem` tiles left over by `full` complete waves (0: not worth it).
   // The shared tiles are computed first, so that parking and adding their partial sums overlaps the
   // contraction of the tiles that follow; without a complete wave there is nothing to hide behind.
-  __device__ static int sharing_workers(int full, int rem, int kt, int nworkers, int min_blocks, int min_gain) {
-    if (rem == 0 || full == 0) return 0;
+  __device__ static int sharing_workers(int full, int rem, int kt, int nworkers, int min_blocks, int min_gain,
+                                        int any = 0) {
+    if (rem == 0 || (full == 0 && !any)) return 0;
     const int S = min(nworkers, rem * kt / min_blocks);
     if (S <= rem) return 0;
     return kt - (rem * kt + S - 1) / S >= min_gain ? S : 0;
   }
 
   // kin: fan-in extent of the row products (K, or the kept outputs of the layer that feeds this one)
-  __device__ void init(const TcParams& p, int rank_, int kin) {
+  // ext_mode: see TcParams (0 unless the kernel was instantiated with FUSED)
+  __device__ void init(const TcParams& p, int rank_, int kin, int ext_mode = 0) {
     rank = rank_;
     workers = (int)gridDim.x / CTAS;
     dp = p.hdr[HDR_DP];
     b = p.hdr[HDR_B];
     n_keep = p.hdr[HDR_NKEEP];
+    const int ext = n_keep;  // length of the row list when hdr is a row list's header
+    if (ext_mode) { dp = 1; b = 1; n_keep = p.N; }
     Tc = p.hdr[HDR_TC];
     subm = subn = 1;
     KT = sk_tiles = sk_S = sk_blocks = 0;
-    if (MODE == M_ROW_FWD) { M_gemm = p.B; N_gemm = n_keep; Kc = kin; }
-    else if (MODE == M_ROW_BWD_DATA) { M_gemm = p.B; N_gemm = kin; Kc = n_keep; }
+    if (MODE == M_ROW_FWD) { M_gemm = ext_mode ? ext : p.B; N_gemm = n_keep; Kc = kin; }
+    else if (MODE == M_ROW_BWD_DATA) { M_gemm = ext_mode ? ext : p.B; N_gemm = kin; Kc = n_keep; }
     else if (MODE == M_LSTM_FWD) { M_gemm = p.B; N_gemm = ((n_keep + 63) / 64) * 256; Kc = p.K; }
     else if (MODE == M_LSTM_BWD_DATA) { M_gemm = p.B; N_gemm = p.K; Kc = 4 * (((n_keep + 63) / 64) * 64); }
-    else if (MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = kin; Kc = p.B; }
+    else if (MODE == M_ROW_BWD_WEIGHT || MODE == M_LSTM_BWD_WEIGHT) { M_gemm = n_keep; N_gemm = kin; Kc = ext_mode ? ext : p.B; }
     else if (MODE == M_ROWS_FWD) { M_gemm = n_keep; N_gemm = p.N; Kc = p.K; }
     else if (MODE == M_ROWS_BWD_DATA) { M_gemm = n_keep; N_gemm = p.K; Kc = p.N; }
     else if (MODE == M_ROWS_BWD_WEIGHT) { M_gemm = p.N; N_gemm = p.K; Kc = n_keep; }
@@ -287,7 +296,7 @@ struct Sched {
             const int w16 = 16 * ((CTAS == 2 && FLEX) ? wpair : wone);
             const int full = tiles / workers, rem = tiles % workers;
             const int S = (SK_MODE && p.sk_ws != nullptr && kt > 0)
-                              ? sharing_workers(full, rem, kt, workers, p.sk_min_blocks, p.sk_min_gain) : 0;
+                              ? sharing_workers(full, rem, kt, workers, p.sk_min_blocks, p.sk_min_gain, p.sk_any) : 0;
             int cost = full * w16;
             if (S > 0) cost += (((rem * kt + S - 1) / max(S, 1)) + p.sk_min_gain / 2) * w16 / max(kt, 1);
             else if (rem > 0) cost += w16;
@@ -302,7 +311,7 @@ struct Sched {
     sk_tiles = sk_S = sk_blocks = 0;
     if (SK_MODE && p.sk_ws != nullptr && KT > 0) {
       const int rem = total % workers;
-      const int S = sharing_workers(total / workers, rem, KT, workers, p.sk_min_blocks, p.sk_min_gain);
+      const int S = sharing_workers(total / workers, rem, KT, workers, p.sk_min_blocks, p.sk_min_gain, p.sk_any);
       if (S > 0) { sk_tiles = rem; sk_S = S; sk_blocks = rem * KT; }
     }
   }
@@ -632,7 +641,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
   pdl_wait_prior_grids();
 
   Sched<BN, MODE, CTAS, SHARE> sch;
-  sch.init(p, (int)rank, (FUSED && p.hdr_in != nullptr) ? p.hdr_in[HDR_NKEEP] : p.K);
+  sch.init(p, (int)rank, (FUSED && p.hdr_in != nullptr) ? p.hdr_in[HDR_NKEEP] : p.K, FUSED ? p.ext_mode : 0);
   if (is_class_mode(MODE) && !sch.dense) {
     // The producer reads one list entry per contraction block: keep the list in shared memory (the
     // staging area of the forward scatter epilogue is free in these modes) instead of paying a
@@ -945,14 +954,13 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
       } else {
         row_ok = m < sch.M_gemm;
         out_row = m;
+        // compact operand of a row list: the results go back to the rows the operand was gathered from
+        if (FUSED && (MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA) && p.ridx != nullptr && row_ok) out_row = p.ridx[m];
       }
 
-      // One 32-column chunk of this thread's accumulator row, already loaded into r[].
-      auto emit = [&](const uint32_t (&r)[32], int ch) {
-        const int oc = sel4(ti.ocol, ch >> 1);
-        if (oc < 0) return;                    // padding of a class tile
-        const int n = oc + (ch & 1) * 32;      // output column of this chunk
-        float v[32];
+      // The values of one 32-column chunk of this thread's accumulator row (already loaded into r[]), whose
+      // first output column is n: rescale, and for the layer-step kernels bias / activation / ReLU adjoint.
+      auto values = [&](const uint32_t (&r)[32], int n, float (&v)[32]) {
         if (FUSED && MODE == M_ROW_FWD) {
           // layer step: bias of the original neuron, activation, rescale (Sec. 3.2, last paragraph).
           // Lane l fetches the bias of column n + l once; the row loop takes it from there by shuffle (32
@@ -991,6 +999,16 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
               if (i < na && !(__bfloat162float(arow[i]) > 0.f)) v[i] = 0.f;
           }
         }
+
+      };
+
+      // One 32-column chunk of this thread's accumulator row, already loaded into r[].
+      auto emit = [&](const uint32_t (&r)[32], int ch) {
+        const int oc = sel4(ti.ocol, ch >> 1);
+        if (oc < 0) return;                    // padding of a class tile
+        const int n = oc + (ch & 1) * 32;      // output column of this chunk
+        float v[32];
+        values(r, n, v);
 
         if (MODE == M_ROW_FWD && p.scatter && dp > 1) {
           // Full-width rows: compact column j -> column b-1 + j*dp, zeros everywhere else
@@ -1173,6 +1191,37 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
       } else {
         // Software pipeline over this warp's chunks: the TMEM load of chunk i+1 is in flight while
         // chunk i is converted and stored.
+        // bf16 rows written plainly go out two chunks at a time through the warp's staging block, so that a
+        // store instruction writes four whole 128-byte lines (eight lanes per row) instead of 16 bytes in each
+        // of 32 rows: with a short contraction the epilogue is what a tile waits for, and the scattered form
+        // kept it at 6.4 us per 256 x 256 tile where the products and loads need 4.1.
+        constexpr bool PAIR_MODES = MODE == M_ROW_FWD || MODE == M_ROW_BWD_DATA || MODE == M_ROW_BWD_WEIGHT ||
+                                    (is_class_mode(MODE) && PLAIN);
+        const bool pair_ok = PAIR_MODES && !p.out_is_f32 && !p.accumulate && !(MODE == M_ROW_FWD && p.scatter && dp > 1) &&
+                             !(MODE == M_ROW_BWD_WEIGHT && p.zero_fill);
+        const unsigned okmask = __ballot_sync(0xffffffffu, row_ok);
+        uint32_t* stw = reinterpret_cast<uint32_t*>(stg);
+        auto stage_half = [&](const uint32_t (&r)[32], int n, int half2) {
+          float v[32];
+          values(r, n, v);
+          uint32_t* sw = stw + lane * 33 + half2 * 16;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) sw[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+        };
+        auto flush_pair = [&](int n) {  // 32 rows x 64 columns starting at output column n
+          __syncwarp();
+          const int piece = lane & 7;
+#pragma unroll
+          for (int it8 = 0; it8 < 8; ++it8) {
+            const int rr = it8 * 4 + (lane >> 3);
+            const long long orow = __shfl_sync(0xffffffffu, out_row, rr);
+            const uint32_t* q = stw + rr * 33 + piece * 4;
+            const uint4 w = make_uint4(q[0], q[1], q[2], q[3]);
+            if ((okmask >> rr) & 1u)
+              *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)orow * p.ldo + n + piece * 8) = w;
+          }
+          __syncwarp();
+        };
         uint32_t ra[32], rb[32];
         if (has_acc && ch_lo < ch_hi) tmem_ld32(t_row + (uint32_t)(ch_lo * 32), ra);
 #pragma unroll 1
@@ -1181,13 +1230,21 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
             tmem_ld_wait();
             if (ch + 1 < ch_hi) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), rb);
           }
-          emit(ra, ch);
+          const int oc = sel4(ti.ocol, ch >> 1);
+          const bool paired = pair_ok && (ch & 1) == 0 && ch + 1 < ch_hi && oc >= 0 && oc + 64 <= sch.N_gemm;
+          if (paired) stage_half(ra, oc, 0);
+          else emit(ra, ch);
           if (ch + 1 < ch_hi) {
             if (has_acc) {
               tmem_ld_wait();
               if (ch + 2 < ch_hi) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), ra);
             }
-            emit(rb, ch + 1);
+            if (paired) {
+              stage_half(rb, oc + 32, 1);
+              flush_pair(oc);
+            } else {
+              emit(rb, ch + 1);
+            }
           }
         }
       }
@@ -1288,7 +1345,7 @@ int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int dp_bound, int ts) {
 }
 
 ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s) {
-  TcParams p;
+  TcParams p = {};
   p.mapA = a.mapA;
   p.mapB = a.mapB;
   p.mapA_indexed = a.mapA_indexed;
@@ -1323,9 +1380,20 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
   p.relu = a.g.relu;
   p.act = a.g.act;
   p.ldact = a.g.ldact;
+  p.ext_mode = a.g.ext_mode;
+  p.ridx = a.g.ridx;
   // the layer-step variants are separate instantiations, so that the plain products carry none of their code
-  const bool fused = kind == ARD_ROW && (p.hdr_in != nullptr || p.bias != nullptr || p.relu != 0 || p.act != nullptr);
+  const bool fused = kind == ARD_ROW && (p.hdr_in != nullptr || p.bias != nullptr || p.relu != 0 || p.act != nullptr ||
+                                         p.ext_mode != 0);
   const int bn = (kind == ARD_ROW) ? 256 : a.bn;
+  if (kind == ARD_ROW && op == OP_BWD_WEIGHT && p.ext_mode == 2 && ctx->use_pairs && p.N > BM &&
+      (p.force_bn == 0 || p.force_bn >= 128) && ctx->d_sk_ws != nullptr) {
+    // Weight gradient over a row list's compact operands: few output tiles (channels x fan-in) and a contraction
+    // as long as the list, so the tiles are always cut along the contraction and shared by all SMs.
+    p.sk_ws = reinterpret_cast<float4*>(ctx->d_sk_ws);
+    p.sk_any = 1;
+    return launch_mode<256, M_ROW_BWD_WEIGHT, 2, true, true>(ctx, p, 1 << 30, s);  // every SM takes a share
+  }
 
 #define ARD_TC_CASE(BN_, MODE_, TILES_) \
   if (bn == BN_) return launch_mode<BN_, MODE_, 1>(ctx, p, (TILES_), s);
@@ -1420,7 +1488,7 @@ ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_
 
 // LSTM gate products (single CTA per tile; the batch of a recurrent step is small).
 ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStream_t s) {
-  TcParams p;
+  TcParams p = {};
   p.mapA = a.mapA;
   p.mapB = a.mapB;
   for (int g = 0; g < 4; ++g) { p.mapA4[g] = a.mapA4[g]; p.mapB4[g] = a.mapB4[g]; }

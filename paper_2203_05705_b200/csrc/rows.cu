@@ -172,7 +172,50 @@ __global__ void __launch_bounds__(256) zero_dropped_rows_kernel(const uint8_t* k
   }
 }
 
+// The dense, small input matrix of Sec. 5.2.1 (step 2): row j of dst is row idx[j] of src, j < n_keep; the rows
+// up to the next multiple of 64 are zero, so that a contraction over the list can run in whole 64-row blocks.
+// One warp per row, 16-byte pieces, a few of them in flight per lane.
+__global__ void __launch_bounds__(256) rows_gather_kernel(const int32_t* hdr, const int32_t* idx, const uint4* src,
+                                                          size_t ld_src16, uint4* dst, size_t ld_dst16, int row16) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int n_keep = hdr[HDR_NKEEP];
+  const int n_pad = (n_keep + 63) / 64 * 64;
+  const int lane = threadIdx.x & 31;
+  const int warps = (int)gridDim.x * 8;
+  for (int j = (int)blockIdx.x * 8 + (threadIdx.x >> 5); j < n_pad; j += warps) {
+    uint4* d = dst + (size_t)j * ld_dst16;
+    if (j < n_keep) {
+      const uint4* sp = src + (size_t)idx[j] * ld_src16;
+      for (int c = lane; c < row16; c += 128) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (c + 32 * u < row16) v[u] = sp[c + 32 * u];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (c + 32 * u < row16) d[c + 32 * u] = v[u];
+      }
+    } else {
+      for (int c = lane; c < row16; c += 32) d[c] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+}
+
 }  // namespace
+
+ard_status launch_rows_gather(ard_ctx* ctx, const ard_rows* rows, const void* src, int ld_src_bytes, void* dst,
+                              int ld_dst_bytes, int row_bytes, cudaStream_t s) {
+  if (rows->M == 0 || row_bytes == 0) return ARD_OK;
+  const int want = (rows->M + 7) / 8;
+  const int grid = want < ctx->sm_count * 8 ? want : ctx->sm_count * 8;
+  ARD_CUDA_OK(ard_launch(ctx, rows_gather_kernel, dim3(grid), dim3(256), 0, s, (const int32_t*)rows->d_hdr,
+                         (const int32_t*)rows->d_idx, (const uint4*)src, (size_t)(ld_src_bytes / 16), (uint4*)dst,
+                         (size_t)(ld_dst_bytes / 16), row_bytes / 16));
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
 
 ard_status launch_sensitivity(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc, int samples,
                               int need, float threshold, uint32_t P_sens, uint32_t P_insens, uint64_t seed,

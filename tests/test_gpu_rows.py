@@ -108,6 +108,101 @@ def test_products_over_the_kept_rows_match_the_oracle(M, K, N):
         ctx.close()
 
 
+@pytest.mark.parametrize("M,K,N", [(300, 328, 520), (1000, 64, 72), (130, 1160, 264), (64, 72, 8), (2100, 520, 384)])
+def test_products_on_gathered_rows_match_the_oracle(M, K, N):
+    """The same three products through the dense small matrices of Sec. 5.2.1: gather the kept rows, multiply,
+    fill back.  The compact buffers start as NaN, so rows the gather must write (kept rows and the zero rows up
+    to the next multiple of 64) show if they are missing, and nothing past them may be read into a result."""
+    rng = np.random.default_rng(M + K + 1)
+    A = inputs.bf16_round(rng.standard_normal((M, K)).astype(np.float32))
+    W = inputs.bf16_round((rng.standard_normal((K, N)) / np.sqrt(K)).astype(np.float32))      # math orientation
+    dY = inputs.bf16_round(rng.standard_normal((M, N)).astype(np.float32))
+    ctx = Ctx(4096)
+    rows = ard.ard_rows_create(ctx.h, M, 3)
+    cap = (M + 63) // 64 * 64
+    try:
+        Wd = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+        Ad = torch.from_numpy(A).to(BF).cuda()
+        dYd = torch.from_numpy(dY).to(BF).cuda()
+        tol = TOL[ard.ARD_BF16]
+        for it, p in enumerate([0.0, 0.3, 0.5, 0.9, 0.999]):
+            ard.ard_rows_set_probability(ctx.h, rows, p)
+            ard.ard_rows_sample(ctx.h, rows, 11, it, 2)
+            n_keep, keep, _ = ard.ard_rows_to_host(rows, M)
+            dropped = np.setdiff1d(np.arange(M), keep)
+            Ak = torch.full((cap, K), float("nan"), dtype=BF, device="cuda")
+            dYk = torch.full((cap, N), float("nan"), dtype=BF, device="cuda")
+            ard.ard_rows_gather(ctx.h, rows, M, K, Ad, K, Ak, K)
+            ard.ard_rows_gather(ctx.h, rows, M, N, dYd, N, dYk, N)
+            torch.cuda.synchronize()
+            pad = (n_keep + 63) // 64 * 64
+            assert torch.equal(Ak[:n_keep], Ad[torch.from_numpy(keep).long().cuda()])          # bit-exact copy
+            assert bool(torch.all(Ak[n_keep:pad] == 0)) and bool(torch.all(dYk[n_keep:pad] == 0))
+            assert bool(torch.isnan(Ak[pad:]).all())                                           # nothing else written
+            Y = torch.full((M, N), float("nan"), dtype=BF, device="cuda")
+            dA = torch.full((M, K), float("nan"), dtype=BF, device="cuda")
+            dW = torch.full((N, K), float("nan"), dtype=torch.float32, device="cuda")
+            dWb = torch.full((N, K), float("nan"), dtype=BF, device="cuda")
+            ard.ard_rows_fwd_compact(ctx.h, rows, M, K, N, 1.5, Ak, K, Wd, K, Y, N)
+            ard.ard_rows_bwd_data_compact(ctx.h, rows, M, K, N, 1.5, dYk, N, Wd, K, dA, K)
+            ard.ard_rows_bwd_weight_compact(ctx.h, rows, ard.ARD_F32, M, K, N, 1.5, Ak, K, dYk, N, dW, K)
+            ard.ard_rows_bwd_weight_compact(ctx.h, rows, ard.ARD_BF16, M, K, N, 1.5, Ak, K, dYk, N, dWb, K)
+            torch.cuda.synchronize()
+            assert ard.ard_last_device_status(ctx.h) == 0
+            tag = (M, K, N, p, n_keep)
+            Yh, dAh, dWh, dWbh = host(Y), host(dA), host(dW), host(dWb)
+            assert np.all(Yh[dropped] == 0) and np.all(dAh[dropped] == 0), tag
+            if n_keep:
+                assert OG.rel_fro(Yh, OC.fwd_compact(A, W, keep, 1.5)) <= tol, tag
+                assert OG.rel_fro(dAh, OC.bwd_data(dY, W, keep, 1.5)) <= tol, tag
+                assert OG.rel_fro(dWh, OC.bwd_weight(A, dY, keep, 1.5).T) <= tol, tag
+                assert OG.rel_fro(dWbh, OC.bwd_weight(A, dY, keep, 1.5).T) <= tol, tag
+            else:
+                assert np.all(Yh == 0) and np.all(dAh == 0) and np.all(dWh == 0) and np.all(dWbh == 0), tag
+    finally:
+        torch.cuda.synchronize()
+        ard.ard_rows_destroy(rows)
+        ctx.close()
+
+
+def test_shared_weight_gradient_on_gathered_rows_is_reproducible():
+    """A long list and few output tiles: the weight gradient's tiles are cut along the contraction and shared by
+    all SMs; the partial sums are added in a fixed order, so every launch gives the same bits."""
+    M, K, N = 20000, 576, 512
+    rng = np.random.default_rng(9)
+    A = torch.from_numpy(inputs.bf16_round(rng.standard_normal((M, K)).astype(np.float32))).to(BF).cuda()
+    dY = torch.from_numpy(inputs.bf16_round(rng.standard_normal((M, N)).astype(np.float32))).to(BF).cuda()
+    ctx = Ctx(4096)
+    rows = ard.ard_rows_create(ctx.h, M, 1)
+    cap = (M + 63) // 64 * 64
+    try:
+        ard.ard_rows_set_probability(ctx.h, rows, 0.45)
+        ard.ard_rows_sample(ctx.h, rows, 3, 0, 0)
+        n_keep, keep, _ = ard.ard_rows_to_host(rows, M)
+        Ak = torch.zeros((cap, K), dtype=BF, device="cuda")
+        dYk = torch.zeros((cap, N), dtype=BF, device="cuda")
+        ard.ard_rows_gather(ctx.h, rows, M, K, A, K, Ak, K)
+        ard.ard_rows_gather(ctx.h, rows, M, N, dY, N, dYk, N)
+        ref = None
+        for rep in range(10):
+            dW = torch.full((N, K), float("nan"), dtype=torch.float32, device="cuda")
+            ard.ard_rows_bwd_weight_compact(ctx.h, rows, ard.ARD_F32, M, K, N, 1.0, Ak, K, dYk, N, dW, K)
+            torch.cuda.synchronize()
+            if ref is None:
+                ref = dW
+                kk = torch.from_numpy(keep).long().cuda()
+                want = dY[kk].double().T @ A[kk].double()                      # library matmul in fp64 on the same bits
+                err = float((dW.double() - want).norm() / want.norm())
+                assert err <= 1e-5, err                                        # fp32 accumulation of exact bf16 products
+            else:
+                assert torch.equal(dW, ref), rep
+        assert ard.ard_last_device_status(ctx.h) == 0
+    finally:
+        torch.cuda.synchronize()
+        ard.ard_rows_destroy(rows)
+        ctx.close()
+
+
 def test_repeated_launches_give_the_same_bits():
     """The gathered operand reaches the tensor cores through ordinary asynchronous copies; a missing ordering
     between those writes and the MMA reads would show as run-to-run differences."""
