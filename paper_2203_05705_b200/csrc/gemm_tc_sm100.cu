@@ -281,19 +281,19 @@ struct Sched {
           // instructions; the time of a tile relative to a 256-wide one, measured per wave on dense
           // problems: pairs 0.92 / 0.83 / 0.78 / 0.76 at 224 / 192 / 160 / 128 columns, single CTAs 0.7 at
           // 128 and 0.55 at 64.  Ties go to the wider tile.
-          // The forward products try every multiple of 32 columns (the instruction takes any multiple of
-          // 16; B still arrives in 64-row boxes, the last one partly unused).  Where B is read along its
+          // The forward products of CTA pairs try every multiple of 32 columns (the instruction takes any
+          // multiple of 16; B still arrives in 64-row boxes, the last one partly unused).  Where B is read along its
           // contiguous dimension (both backward products) only 256 / 128 / 64 keep every box on a 128-byte
           // line; other widths were measured up to 20 % slower per tile there and are not tried.
           // Shared tiles cost each worker its share of their contraction plus some of the reduction.
-          constexpr bool FLEX = (MODE == M_ROW_FWD || MODE == M_ROWS_FWD);
+          constexpr bool FLEX = CTAS == 2 && MODE == M_ROW_FWD;  // single CTAs: small, latency-bound problems
           const int kt = (Kc + BK - 1) / BK;
           int best_cost = 0x7fffffff;
           for (int cand = BN; cand >= 64 * CTAS; cand = FLEX ? cand - 32 : cand >> 1) {
             const int tiles = Mt * ((N_gemm + cand - 1) / cand);
             const int wpair = cand == 256 ? 100 : (cand == 224 ? 92 : (cand == 192 ? 83 : (cand == 160 ? 78 : 76)));
-            const int wone = cand == 256 ? 100 : (cand == 128 ? 70 : (cand == 64 ? 55 : 40 + (60 * cand) / 256));
-            const int w16 = 16 * ((CTAS == 2 && FLEX) ? wpair : wone);
+            const int wone = cand == 256 ? 100 : (cand == 128 ? 70 : 55);
+            const int w16 = 16 * (FLEX ? wpair : wone);
             const int full = tiles / workers, rem = tiles % workers;
             const int S = (SK_MODE && p.sk_ws != nullptr && kt > 0)
                               ? sharing_workers(full, rem, kt, workers, p.sk_min_blocks, p.sk_min_gain, p.sk_any) : 0;
