@@ -19,24 +19,29 @@ __global__ void __launch_bounds__(256) gather_cols_kernel(const int32_t* hdr, co
   for (int r = blockIdx.y; r < rows; r += gridDim.y) dst[(size_t)r * ld_dst + j] = src[(size_t)r * ld_src + col];
 }
 
-// Faster form for 2-byte elements with 16-byte aligned rows.  Each warp owns a private slice of
+// Faster form for 2-byte elements with 16-byte aligned rows.  Each warp owns two private slices of
 // shared memory: one bulk copy (the copy engine, not the load unit, whose queue holds about 20 KB of
-// 16-byte requests per SM) brings the source span of a pass, the warp compacts the slice in place and
-// writes it out with 16-byte stores.  No block-wide barrier, so the warps of a block overlap each
-// other's latency.  The wait on the copy is bounded; a timeout sets *status and ends the warp.
+// 16-byte requests per SM) brings the source span of a pass into one slice while the warp compacts the
+// other slice in place and writes it out with 16-byte stores.  No block-wide barrier, so the warps of a
+// block overlap each other's latency.  The wait on a copy is bounded; a timeout sets *status and ends
+// the warp.
 // With skip_dense != 0 a dense pattern (dp = 1) is left alone: the GEMM then reads the original matrix.
 constexpr int GATHER_WARPS = 4;
-constexpr int GATHER_SPAN = 4096;  // staged source elements per warp (8 KiB)
+constexpr int GATHER_SPAN = 2048;  // staged source elements per slice (4 KiB)
+
+struct GatherItem {
+  int r, j0, nout, a0, off, count, n16;
+};
 
 __global__ void __launch_bounds__(GATHER_WARPS * 32)
 gather_cols_staged_kernel(const int32_t* hdr, const uint16_t* src, int ld_src,
                           uint16_t* dst, int ld_dst, int rows, int n_cols, int skip_dense, int* status) {
-  __shared__ __align__(128) uint16_t smem[GATHER_WARPS][GATHER_SPAN + 64];
-  __shared__ __align__(8) uint64_t bars[GATHER_WARPS];
+  __shared__ __align__(128) uint16_t smem[GATHER_WARPS][2][GATHER_SPAN + 64];
+  __shared__ __align__(8) uint64_t bars[GATHER_WARPS][2];
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-  const uint32_t bar = smem_u32(&bars[wib]);
   if (lane == 0) {
-    mbar_init(bar, 1);
+    mbar_init(smem_u32(&bars[wib][0]), 1);
+    mbar_init(smem_u32(&bars[wib][1]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
@@ -46,7 +51,7 @@ gather_cols_staged_kernel(const int32_t* hdr, const uint16_t* src, int ld_src,
   if (skip_dense && dp == 1) return;
   const long long warp_id = (long long)blockIdx.x * GATHER_WARPS + wib;
   const long long n_warps = (long long)gridDim.x * GATHER_WARPS;
-  // outputs per warp pass (multiple of 8): whatever the period, a pass keeps the whole staging slice in flight
+  // outputs per warp pass (multiple of 8): whatever the period, a pass fills its staging slice
   const int outs = ((GATHER_SPAN - 8) / dp) & ~7;
   if (outs < 8) {
     // period too long for the staging slice: element-wise copy
@@ -56,38 +61,67 @@ gather_cols_staged_kernel(const int32_t* hdr, const uint16_t* src, int ld_src,
     }
     return;
   }
-  uint16_t* buf = smem[wib];
-  uint32_t phase = 0;
   const int chunks = (n_keep + outs - 1) / outs;
-  for (long long item = warp_id; item < (long long)rows * chunks; item += n_warps) {
-    const int r = (int)(item / chunks), ch = (int)(item - (long long)r * chunks);
-    const int j0 = ch * outs;
-    const int nout = min(outs, n_keep - j0);
-    const int s0 = bb + j0 * dp;  // first source column
-    const int a0 = s0 & ~7;       // 16-byte aligned start
-    const int count = bb + (j0 + nout - 1) * dp - a0 + 1;  // <= n_cols - a0
-    const uint16_t* srow = src + (size_t)r * ld_src;
+  const long long total = (long long)rows * chunks;
+  auto describe = [&](long long item) {
+    GatherItem g;
+    g.r = (int)(item / chunks);
+    const int ch = (int)(item - (long long)g.r * chunks);
+    g.j0 = ch * outs;
+    g.nout = min(outs, n_keep - g.j0);
+    const int s0 = bb + g.j0 * dp;  // first source column
+    g.a0 = s0 & ~7;                 // 16-byte aligned start
+    g.off = s0 - g.a0;
+    g.count = bb + (g.j0 + g.nout - 1) * dp - g.a0 + 1;  // <= n_cols - a0
     // whole 16-byte pieces inside the row go through the copy engine, a ragged end (< 8 elements) by lanes
-    const int n16 = min((count + 7) & ~7, (n_cols - a0) & ~7);
-    if (lane == 0 && n16 > 0) {
-      mbar_arrive_expect_tx(bar, (uint32_t)n16 * 2u);
+    g.n16 = min((g.count + 7) & ~7, (n_cols - g.a0) & ~7);
+    return g;
+  };
+  // starts the copy of an item into a slice; every lane's earlier accesses to the slice were fenced
+  auto fetch = [&](const GatherItem& g, int slot) {
+    uint16_t* buf = smem[wib][slot];
+    const uint16_t* srow = src + (size_t)g.r * ld_src;
+    if (lane == 0 && g.n16 > 0) {
+      const uint32_t bar = smem_u32(&bars[wib][slot]);
+      mbar_arrive_expect_tx(bar, (uint32_t)g.n16 * 2u);
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(smem_u32(buf)), "l"(srow + a0), "r"((uint32_t)n16 * 2u), "r"(bar)
+                   ::"r"(smem_u32(buf)), "l"(srow + g.a0), "r"((uint32_t)g.n16 * 2u), "r"(bar)
                    : "memory");
     }
-    for (int i = n16 + lane; i < count; i += 32) buf[i] = srow[a0 + i];
-    if (n16 > 0) {
-      bool ok = mbar_try_wait(bar, phase);
-      for (int poll = 0; poll < 4000 && !ok; ++poll) ok = mbar_try_wait_hint(bar, phase, 1000000u);
+    for (int i = g.n16 + lane; i < g.count; i += 32) buf[i] = srow[g.a0 + i];
+  };
+  uint32_t phase[2] = {0u, 0u};
+  long long item = warp_id;
+  if (item >= total) return;
+  GatherItem cur = describe(item);
+  fetch(cur, 0);
+  for (int k = 0;; ++k) {
+    const int slot = k & 1;
+    const long long next_item = item + n_warps;
+    GatherItem nxt = cur;
+    if (next_item < total) {
+      nxt = describe(next_item);
+      fetch(nxt, slot ^ 1);
+    }
+    if (cur.n16 > 0) {
+      const uint32_t bar = smem_u32(&bars[wib][slot]);
+      bool ok = mbar_try_wait(bar, phase[slot]);
+      for (int poll = 0; poll < 4000 && !ok; ++poll) ok = mbar_try_wait_hint(bar, phase[slot], 1000000u);
       if (!ok) {
         if (lane == 0) atomicMax(status, (int)ARD_ERR_TIMEOUT);
+        if (next_item < total && nxt.n16 > 0) {  // the copy into the other slice: give it the same time, then leave
+          const uint32_t bar2 = smem_u32(&bars[wib][slot ^ 1]);
+          bool done = false;
+          for (int poll = 0; poll < 4000 && !done; ++poll) done = mbar_try_wait_hint(bar2, phase[slot ^ 1], 1000000u);
+        }
         return;
       }
-      phase ^= 1u;
+      phase[slot] ^= 1u;
     }
     __syncwarp();
-    const int off = s0 - a0;
-    uint16_t* drow = dst + (size_t)r * ld_dst + j0;
+    uint16_t* buf = smem[wib][slot];
+    const int off = cur.off, nout = cur.nout;
+    uint16_t* drow = dst + (size_t)cur.r * ld_dst + cur.j0;
     // Compact the slice in place, consecutive lanes taking consecutive outputs (a lane that took eight
     // outputs in a row read shared memory at a stride of 16 * dp bytes: up to 32 lanes on one bank).  Output
     // j lands at element j <= off + j * dp, and the sources of a batch are all in registers before any of
@@ -114,8 +148,11 @@ gather_cols_staged_kernel(const int32_t* hdr, const uint16_t* src, int ld_src,
         for (int i = t * 8; i < nout; ++i) drow[i] = buf[i];
       }
     }
-    fence_proxy_async_smem();  // this lane's accesses to the slice, before the next pass's copy overwrites it
+    fence_proxy_async_smem();  // this lane's accesses to the slice, before a later pass's copy overwrites it
     __syncwarp();
+    if (next_item >= total) break;
+    item = next_item;
+    cur = nxt;
   }
 }
 
