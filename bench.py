@@ -33,7 +33,7 @@ from paper_2203_05705_b200 import inputs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of ard_gemm_tc_kernel, averaged over the three
 # GEMMs of one dense (dp = 1) step of this workload, from the ncu capture summarised under profiles/.
-DRAM_TRAFFIC_PER_LAUNCH = 579.0e6   # bytes (fwd 678.4 MB, bwd-data 675.6 MB, bwd-weight 383.3 MB)
+DRAM_TRAFFIC_PER_LAUNCH = 581.0e6   # bytes (fwd 679.5 MB, bwd-data 674.4 MB, bwd-weight 390.3 MB)
 
 METRIC = "layer fwd+bwd kept TFLOP/s (row pattern, p=0.5)"
 UNIT = "TFLOP/s"
