@@ -138,6 +138,10 @@ struct SmemLayout {
   static constexpr int TOTAL = MISC_OFF + 16 + 1024;         // + slack for manual 1024-byte alignment
 };
 
+// Class modes: bytes of the staging area that hold the kept-tile list and the class table.
+constexpr int CLASS_LIST_BYTES = 16384;
+static_assert(CLASS_LIST_BYTES + EPI_WARPS * 32 * 17 * 4 <= EPI_WARPS * 32 * 33 * 4, "class staging does not fit");
+
 // Element i of a 4-entry array without dynamic indexing (keeps the array in registers).
 __device__ __forceinline__ int sel4(const int (&a)[4], int i) {
   return i == 0 ? a[0] : (i == 1 ? a[1] : (i == 2 ? a[2] : a[3]));
@@ -646,12 +650,13 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
     // The producer reads one list entry per contraction block: keep the list in shared memory (the
     // staging area of the forward scatter epilogue is free in these modes) instead of paying a
     // global-memory round trip on its critical path.
-    // The last KiB of that area holds the per-class table (first item, list offset, length, members).
+    // The list and the per-class table (first item, list offset, length, members; one KiB) share the first
+    // CLASS_LIST_BYTES of that area; the rest is the epilogue warps' staging (32 rows x 17 words each).
     const int n_list = p.hdr[HDR_NKEEP];
-    int4* tab = reinterpret_cast<int4*>(smem + L::STG_OFF + L::STG_BYTES - 1024);
+    int4* tab = reinterpret_cast<int4*>(smem + L::STG_OFF + CLASS_LIST_BYTES - 1024);
     int* total_smem = reinterpret_cast<int*>(smem + L::MISC_OFF + 8);
     int32_t* slist = reinterpret_cast<int32_t*>(smem + L::STG_OFF);
-    const bool fits = n_list * 4 <= L::STG_BYTES - 1024;
+    const bool fits = n_list * 4 <= CLASS_LIST_BYTES - 1024;
     if (threadIdx.x == 0) sch.build_class_table(p, tab, total_smem);
     if (fits)
       for (int i = threadIdx.x; i < n_list; i += TC_THREADS) slist[i] = sch.list[i];
@@ -1200,13 +1205,44 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
         const bool pair_ok = PAIR_MODES && !p.out_is_f32 && !p.accumulate && !(MODE == M_ROW_FWD && p.scatter && dp > 1) &&
                              !(MODE == M_ROW_BWD_WEIGHT && p.zero_fill);
         const unsigned okmask = __ballot_sync(0xffffffffu, row_ok);
-        uint32_t* stw = reinterpret_cast<uint32_t*>(stg);
+        // The class tiling keeps its list in the first part of the staging area: its warps stage one chunk
+        // (32 rows x 17 words) behind it and write 64-byte row segments, four lanes per row.
+        constexpr bool CLASS_LIST = is_class_mode(MODE) && !PLAIN;
+        constexpr int SW = CLASS_LIST ? 17 : 33;  // words per staged row
+        uint32_t* stw = CLASS_LIST ? reinterpret_cast<uint32_t*>(smem + L::STG_OFF + CLASS_LIST_BYTES) + (warp - 2) * (32 * 17)
+                                   : reinterpret_cast<uint32_t*>(stg);
+        const bool one_ok = CLASS_LIST && !p.out_is_f32 && !p.accumulate;
         auto stage_half = [&](const uint32_t (&r)[32], int n, int half2) {
           float v[32];
           values(r, n, v);
-          uint32_t* sw = stw + lane * 33 + half2 * 16;
+          uint32_t* sw = stw + lane * SW + half2 * 16;
 #pragma unroll
           for (int i = 0; i < 16; ++i) sw[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+        };
+        auto flush_one = [&](int n) {  // 32 rows x 32 columns starting at output column n
+          __syncwarp();
+          const int piece = lane & 3;
+#pragma unroll
+          for (int it4 = 0; it4 < 4; ++it4) {
+            const int rr = it4 * 8 + (lane >> 2);
+            const long long orow = __shfl_sync(0xffffffffu, out_row, rr);
+            const uint32_t* q = stw + rr * SW + piece * 4;
+            const uint4 w = make_uint4(q[0], q[1], q[2], q[3]);
+            if ((okmask >> rr) & 1u)
+              *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)orow * p.ldo + n + piece * 8) = w;
+          }
+          __syncwarp();
+        };
+        // one chunk of a class tile: staged and written in row segments, or the per-thread form
+        auto emit_class = [&](const uint32_t (&r)[32], int ch) {
+          const int oc1 = sel4(ti.ocol, ch >> 1);
+          if (one_ok && oc1 >= 0) {
+            const int n = oc1 + (ch & 1) * 32;
+            stage_half(r, n, 0);
+            flush_one(n);
+          } else {
+            emit(r, ch);
+          }
         };
         auto flush_pair = [&](int n) {  // 32 rows x 64 columns starting at output column n
           __syncwarp();
@@ -1215,7 +1251,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
           for (int it8 = 0; it8 < 8; ++it8) {
             const int rr = it8 * 4 + (lane >> 3);
             const long long orow = __shfl_sync(0xffffffffu, out_row, rr);
-            const uint32_t* q = stw + rr * 33 + piece * 4;
+            const uint32_t* q = stw + rr * SW + piece * 4;
             const uint4 w = make_uint4(q[0], q[1], q[2], q[3]);
             if ((okmask >> rr) & 1u)
               *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + (size_t)orow * p.ldo + n + piece * 8) = w;
@@ -1233,6 +1269,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
           const int oc = sel4(ti.ocol, ch >> 1);
           const bool paired = pair_ok && (ch & 1) == 0 && ch + 1 < ch_hi && oc >= 0 && oc + 64 <= sch.N_gemm;
           if (paired) stage_half(ra, oc, 0);
+          else if (CLASS_LIST) emit_class(ra, ch);
           else emit(ra, ch);
           if (ch + 1 < ch_hi) {
             if (has_acc) {
@@ -1242,6 +1279,8 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
             if (paired) {
               stage_half(rb, oc + 32, 1);
               flush_pair(oc);
+            } else if (CLASS_LIST) {
+              emit_class(rb, ch + 1);
             } else {
               emit(rb, ch + 1);
             }
