@@ -203,6 +203,72 @@ def test_shared_weight_gradient_on_gathered_rows_is_reproducible():
         ctx.close()
 
 
+def test_benchmark_layer_on_sampled_outputs():
+    """The convolution layer the benchmark times (3 x 3, 256 -> 512 channels, 32768 output positions, regions of 8
+    rows), in its launch configuration: gathered operands, CTA pairs, shared weight-gradient tiles.  The oracle
+    recomputes the sensitivity decision of sampled regions, the whole kept-row list, sampled rows of Y and dA
+    and sampled channels of dW; the zero rows and finiteness are checked over the whole outputs."""
+    M, K, N, x = 32768, 2304, 512, 8
+    kf, tf, thr, mp, npb = 0.05, 0.3, 0.5, 0.2, 0.8
+    rng = np.random.default_rng(2025)
+    A = _input_matrix(rng, M, K, x)
+    W = inputs.bf16_round((rng.standard_normal((K, N)) / np.sqrt(K)).astype(np.float32))      # math orientation
+    dY = inputs.bf16_round(rng.standard_normal((M, N)).astype(np.float32))
+    ctx = Ctx(4096)
+    rows = ard.ard_rows_create(ctx.h, M, x)
+    cap = (M + 63) // 64 * 64
+    try:
+        Ad = torch.from_numpy(A).to(BF).cuda()
+        dYd = torch.from_numpy(dY).to(BF).cuda()
+        Wd = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+        # Sec. 5.1 on sampled regions (integer decisions: exact)
+        ard.ard_sensitivity_predict(ctx.h, rows, ard.ARD_BF16, Ad, K, K, kf, tf, thr, mp, npb, 5, 3, 1)
+        _, _, P = ard.ard_rows_to_host(rows, M, M // x)
+        Pm, Pn = OC.quantise_probability(mp), OC.quantise_probability(npb)
+        for g in range(5, M // x, (M // x) // 40):
+            sens, _, _ = OC.region_sensitive(A, g, x, kf, tf, thr, 5, 3, 1)
+            assert int(P[g]) == (Pm if sens else Pn), g
+        assert 0 < int(np.sum(P == Pm)) < M // x                     # both kinds of region occur
+        # Sec. 5.2.1 with one probability for every region: the whole list against the oracle
+        ard.ard_rows_set_probability(ctx.h, rows, 0.46)
+        ard.ard_rows_sample(ctx.h, rows, 5, 3, 1)
+        n_keep, keep, _ = ard.ard_rows_to_host(rows, M)
+        Pq = np.full(M // x, OC.quantise_probability(0.46), dtype=np.uint64)
+        assert np.array_equal(keep, OC.draw_rows(Pq, x, M, 5, 3, 1))
+        dropped = np.setdiff1d(np.arange(M), keep)
+        Ak = torch.full((cap, K), float("nan"), dtype=BF, device="cuda")
+        dYk = torch.full((cap, N), float("nan"), dtype=BF, device="cuda")
+        Y = torch.full((M, N), float("nan"), dtype=BF, device="cuda")
+        dA = torch.full((M, K), float("nan"), dtype=BF, device="cuda")
+        dW = torch.full((N, K), float("nan"), dtype=BF, device="cuda")
+        ard.ard_rows_gather(ctx.h, rows, M, K, Ad, K, Ak, K)
+        ard.ard_rows_fwd_compact(ctx.h, rows, M, K, N, 1.25, Ak, K, Wd, K, Y, N)
+        ard.ard_rows_gather(ctx.h, rows, M, N, dYd, N, dYk, N)
+        ard.ard_rows_bwd_data_compact(ctx.h, rows, M, K, N, 1.25, dYk, N, Wd, K, dA, K)
+        ard.ard_rows_bwd_weight_compact(ctx.h, rows, ard.ARD_BF16, M, K, N, 1.25, Ak, K, dYk, N, dW, K)
+        torch.cuda.synchronize()
+        assert ard.ard_last_device_status(ctx.h) == 0
+        # whole outputs: finite, dropped rows exactly zero
+        assert bool(torch.isfinite(Y).all()) and bool(torch.isfinite(dA).all()) and bool(torch.isfinite(dW).all())
+        dd = torch.from_numpy(dropped).long().cuda()
+        assert bool(torch.all(Y[dd] == 0)) and bool(torch.all(dA[dd] == 0))
+        # sampled rows (kept and dropped) of Y and dA
+        sel = np.concatenate([keep[:: max(1, len(keep) // 96)][:96], dropped[:: max(1, len(dropped) // 32)][:32]])
+        local_keep = np.flatnonzero(np.isin(sel, keep))
+        sd = torch.from_numpy(sel).long().cuda()
+        tol = TOL[ard.ARD_BF16]
+        assert OG.rel_fro(host(Y[sd]), OC.fwd(A[sel], W, local_keep, 1.25)) <= tol
+        assert OG.rel_fro(host(dA[sd]), OC.bwd_data(dY[sel], W, local_keep, 1.25)) <= tol
+        # sampled channels of dW: the contraction runs over every kept row
+        cols = np.arange(3, N, N // 48)[:48]
+        want = OC.bwd_weight(A[keep], dY[keep][:, cols], np.arange(len(keep)), 1.25).T       # [48][K]
+        assert OG.rel_fro(host(dW[torch.from_numpy(cols).long().cuda()]), want) <= tol
+    finally:
+        torch.cuda.synchronize()
+        ard.ard_rows_destroy(rows)
+        ctx.close()
+
+
 def test_repeated_launches_give_the_same_bits():
     """The gathered operand reaches the tensor cores through ordinary asynchronous copies; a missing ordering
     between those writes and the MMA reads would show as run-to-run differences."""
