@@ -927,6 +927,59 @@ def main():
         detail["kept_fraction"][str(pp)] = float(np.mean([nk / units for (_, _, nk) in pats_p]))
     detail["ideal_speedup"] = {str(pp): 1.0 / (1.0 - pp) for pp in (0.3, 0.5, 0.7)}
 
+    # ---- the same step as one CUDA graph: sampler on a device counter + ard_layer_products (the three products
+    # enqueued side by side on the context's streams); the dense torch step replayed from a graph beside it ----
+    if world == 1:
+        gstream = torch.cuda.Stream()
+        counter = torch.zeros(1, dtype=torch.int64, device="cuda")
+        reps = 10
+
+        def graph_ms(body, n_replays):
+            with torch.cuda.stream(gstream):
+                for _ in range(3):
+                    body()
+                torch.cuda.synchronize()
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=gstream):
+                    for _ in range(reps):
+                        body()
+                for _ in range(3):
+                    gr.replay()
+                torch.cuda.synchronize()
+                a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                for _ in range(n_replays):
+                    gr.replay()
+                b2.record()
+                torch.cuda.synchronize()
+            return a.elapsed_time(b2) / (n_replays * reps)
+
+        n_replays = max(2, args.steps // reps)
+        side, side_kept = {}, {}
+        for pp in (0.3, 0.5, 0.7):
+            def body(pp=pp):
+                gs = gstream.cuda_stream
+                ard.ard_sample_pattern_counter(ctx, pat, dist_ids[pp], seed, 30000, counter, 1, rank, gs)
+                ard.ard_layer_products(ctx, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, 1.0 / (1.0 - pp), X, K, W, K, dY, N,
+                                       Y, N, ard.ARD_OUT_SCATTER_ZEROFILL, dX, K, dW, K, 0, gs)
+            counter.zero_()
+            side[str(pp)] = graph_ms(body, n_replays)
+            # iterations of the timed replays: 3 eager calls and 3 replays of `reps` steps came before them
+            first = 30000 + 3 + 3 * reps
+            pats_g = kept_units_of(pp, range(first, first + n_replays * reps))
+            side_kept[str(pp)] = float(np.mean([nk / units for (_, _, nk) in pats_g]))
+        Wt_ = W.t()
+
+        def torch_body():
+            torch.matmul(X, Wt_, out=Y)
+            torch.matmul(dY, W, out=dX)
+            torch.matmul(dY.t(), X, out=dW)
+
+        torch_graph = graph_ms(torch_body, n_replays)
+        detail["graph_side_by_side"] = {"ms_per_step": side, "kept_fraction": side_kept,
+                                        "torch_matmul_graph_ms": torch_graph,
+                                        "speedup_vs_dense": {k2: torch_graph / v for k2, v in side.items()}}
+
     # ---- end to end through the C ABI with host buffers ----
     h2d = hX.numel() * 2 + hdY.numel() * 2
     d2h = hY.numel() * 2

@@ -221,6 +221,20 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
                           int N, float alpha, const void* X, int ldx, const void* dY, int lddy, int dy_is_compact,
                           void* dW, int lddw, int zero_fill_dropped, void* cuda_stream);
 
+/* The three products of one layer in one iteration behind one call: the same results as ard_fwd, ard_bwd_data
+ * (full-width dY) and ard_bwd_weight (full-width dY) with these arguments, but enqueued so that they may run
+ * side by side: the forward product on the caller's stream, the backward products on streams the context
+ * owns (a tile pattern: one each; a row pattern: both on one, sharing the compact copy of dY), joined back
+ * into the caller's stream before the call returns.  The products depend only on X, W, dY and the pattern
+ * (Sec. 3.1, 3.2), and on small layers one of them leaves most SMs idle.  The first call on a context creates
+ * the streams (make it before any stream capture); the call itself can be captured into a CUDA graph.
+ * Inputs must not be written, and outputs not read, by other work until the caller's stream has passed the
+ * call.  With ARD_MLP_STREAMS=1 in the environment everything stays on the caller's stream.  Asynchronous. */
+ard_status ard_layer_products(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, ard_dtype dW_dtype, int B, int K,
+                              int N, float alpha, const void* X, int ldx, const void* W, int ldw, const void* dY,
+                              int lddy, void* Y, int ldy, ard_outmode outmode, void* dX, int lddx, void* dW, int lddw,
+                              int zero_fill_dropped, void* cuda_stream);
+
 /* ---- fused layer step (row patterns) ----------------------------------------------------------
  * Sec. 3.2, last paragraph: a layer of a training iteration is the fully connected product, the
  * activation and the dropout mask; under a pattern the mask disappears into the product.  Sec. 3.1:

@@ -35,7 +35,7 @@ EXPORTS = [
     "ard_expand_weight_grad_cols", "ard_bias_grad", "ard_sample_pattern_counter", "ard_mlp_step",
     "ard_rows_create", "ard_rows_destroy", "ard_sensitivity_predict", "ard_rows_set_probability", "ard_rows_sample",
     "ard_rows_to_host", "ard_rows_fwd", "ard_rows_bwd_data", "ard_rows_bwd_weight",
-    "ard_rows_gather", "ard_rows_fwd_compact", "ard_rows_bwd_data_compact", "ard_rows_bwd_weight_compact",
+    "ard_layer_products", "ard_rows_gather", "ard_rows_fwd_compact", "ard_rows_bwd_data_compact", "ard_rows_bwd_weight_compact",
 ]
 
 _lib = None
@@ -114,6 +114,8 @@ def lib():
         "ard_rows_fwd": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_rows_bwd_data": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_rows_bwd_weight": [vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_layer_products": [vp, vp, i32, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp, i32, i32, vp, i32, vp,
+                               i32, i32, vp],
         "ard_rows_gather": [vp, vp, i32, i32, vp, i32, vp, i32, vp],
         "ard_rows_fwd_compact": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_rows_bwd_data_compact": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
@@ -393,6 +395,13 @@ def ard_rows_bwd_data(ctx, rows, M, K, N, alpha, dY, lddy, W, ldw, dA, ldda, str
 def ard_rows_bwd_weight(ctx, rows, dW_dtype, M, K, N, alpha, A, lda, dY, lddy, dW, lddw, stream=None):
     _check(lib().ard_rows_bwd_weight(ctx, rows, dW_dtype, M, K, N, alpha, _ptr(A), lda, _ptr(dY), lddy, _ptr(dW), lddw,
                                      _stream(stream)), "ard_rows_bwd_weight")
+
+
+def ard_layer_products(ctx, pat, dtype, dW_dtype, B, K, N, alpha, X, ldx, W, ldw, dY, lddy, Y, ldy, outmode, dX, lddx,
+                       dW, lddw, zero_fill_dropped, stream=None):
+    _check(lib().ard_layer_products(ctx, pat, dtype, dW_dtype, B, K, N, alpha, _ptr(X), ldx, _ptr(W), ldw, _ptr(dY),
+                                    lddy, _ptr(Y), ldy, outmode, _ptr(dX), lddx, _ptr(dW), lddw, zero_fill_dropped,
+                                    _stream(stream)), "ard_layer_products")
 
 
 def ard_rows_gather(ctx, rows, M, width, src, ld_src, dst, ld_dst, stream=None):

@@ -797,6 +797,56 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
                          zero_fill_dropped, cuda_stream);
 }
 
+// The three products of one layer and one iteration, which depend only on X, W, dY and the pattern, enqueued so
+// that they can run side by side: on small layers a product occupies a fraction of the SMs (and a tile pattern
+// whose period divides the tile-column count concentrates the forward product's work in 1/dp of its output
+// tiles), so the other two fill the idle ones.
+ard_status ard_layer_products(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, ard_dtype dW_dtype, int B, int K,
+                              int N, float alpha, const void* X, int ldx, const void* W, int ldw, const void* dY,
+                              int lddy, void* Y, int ldy, ard_outmode outmode, void* dX, int lddx, void* dW, int lddw,
+                              int zero_fill_dropped, void* cuda_stream) {
+  if (!ctx || !pat) return ARD_ERR_INVALID_ARG;
+  if (((int)outmode & ARD_FLAG_RELU) != 0) return ARD_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const bool streams = ctx->mlp_two_streams && ard_side_streams(ctx, s);
+  if (!streams) {
+    // one stream: the calls in order, the second backward product reusing the first one's compact dY
+    const int reuse = ctx->reuse_compact;
+    ctx->reuse_compact = 1;
+    ard_status st = fwd_impl(ctx, pat, nullptr, dtype, B, K, N, alpha, X, ldx, W, ldw, nullptr, 0, Y, ldy, (int)outmode, s);
+    if (st == ARD_OK)
+      st = bwd_data_impl(ctx, pat, nullptr, dtype, B, K, N, alpha, dY, lddy, 0, W, ldw, nullptr, 0, dX, lddx, s);
+    if (st == ARD_OK)
+      st = bwd_weight_impl(ctx, pat, nullptr, dtype, dW_dtype, B, K, N, alpha, X, ldx, dY, lddy, 0, dW, lddw,
+                           zero_fill_dropped, s);
+    ctx->reuse_compact = reuse;
+    return st;
+  }
+  DeviceGuard guard(ctx->device);
+  cudaStream_t side = ctx->side_stream, aux = ctx->aux_stream;
+  // A row pattern's backward products share the compact copy of dY in the context workspace, so they stay on
+  // one stream; a tile pattern's three products are independent.
+  const bool three = pat->kind == ARD_TILE;
+  ARD_CUDA_OK(cudaEventRecord(ctx->ev[100], s));
+  ARD_CUDA_OK(cudaStreamWaitEvent(side, ctx->ev[100], 0));
+  if (three) ARD_CUDA_OK(cudaStreamWaitEvent(aux, ctx->ev[100], 0));
+  ard_status st = fwd_impl(ctx, pat, nullptr, dtype, B, K, N, alpha, X, ldx, W, ldw, nullptr, 0, Y, ldy, (int)outmode, s);
+  const int reuse = ctx->reuse_compact;
+  ctx->reuse_compact = 1;
+  ard_status st2 = bwd_data_impl(ctx, pat, nullptr, dtype, B, K, N, alpha, dY, lddy, 0, W, ldw, nullptr, 0, dX, lddx, side);
+  ard_status st3 = bwd_weight_impl(ctx, pat, nullptr, dtype, dW_dtype, B, K, N, alpha, X, ldx, dY, lddy, 0, dW, lddw,
+                                   zero_fill_dropped, three ? aux : side);
+  ctx->reuse_compact = reuse;
+  // join whatever was enqueued, also after an error, so that a capture is not left forked
+  ARD_CUDA_OK(cudaEventRecord(ctx->ev[101], side));
+  ARD_CUDA_OK(cudaStreamWaitEvent(s, ctx->ev[101], 0));
+  if (three) {
+    ARD_CUDA_OK(cudaEventRecord(ctx->ev[102], aux));
+    ARD_CUDA_OK(cudaStreamWaitEvent(s, ctx->ev[102], 0));
+  }
+  return st != ARD_OK ? st : (st2 != ARD_OK ? st2 : st3);
+}
+
 ard_status ard_layer_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, const ard_pattern* in_pat, ard_dtype dtype,
                                 ard_dtype dW_dtype, int B, int K, int N, float alpha, const void* X, int ldx,
                                 const void* dZ, int lddz, int dz_is_compact, void* dW, int lddw, int zero_fill_dropped,

@@ -246,3 +246,44 @@ def test_lstm_gate_products_against_per_gate_calls(ctx):
         finally:
             ard.ard_set_path(ctx.h, ard.ARD_PATH_AUTO)
     assert ard.ard_last_device_status(ctx.h) == 0
+
+
+@pytest.mark.parametrize("kind,ts,shape", [("row", 0, (300, 520, 1000)), ("tile", 64, (200, 192, 320)),
+                                            ("row", 0, (70, 100, 90))])
+def test_three_products_side_by_side(ctx, kind, ts, shape):
+    """ard_layer_products: the forward and the two backward products of a layer enqueued on the context's own
+    streams and joined again; against the oracle, eagerly and replayed from a CUDA graph (outputs start as
+    NaN, so a product that was not joined before the read shows)."""
+    import torch
+    from oracle import gemm as OG
+    from gpu_helpers import dev, host, nan_buf, oracle_mask
+    B, K, N = shape
+    X, W, dY = _layer(B, K, N, 21, 0.05)
+    akind = ard.ARD_ROW if kind == "row" else ard.ARD_TILE
+    pat = ctx.pattern(akind, K, N, ts)
+    Xd, Wd, dYd = dev(X, ard.ARD_BF16, K), dev(W.T, ard.ARD_BF16, K), dev(dY, ard.ARD_BF16, N)
+    bf = torch.bfloat16
+    for dp, b in [(1, 1), (2, 2), (3, 1), (8, 5)]:
+        ard.ard_pattern_set(ctx.h, pat, dp, b)
+        mask = oracle_mask(akind, K, N, ts, dp, b)
+        want = (OG.fwd(X, W, mask, 1.5), OG.bwd_data(dY, W, mask, 1.5), OG.bwd_weight(X, dY, mask, 1.5).T)
+
+        def call(stream=None):
+            ard.ard_layer_products(ctx.h, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, 1.5, Xd, K, Wd, K, dYd, N, Y, N,
+                                   ard.ARD_OUT_SCATTER_ZEROFILL, dX, K, dW, K, 1, stream)
+
+        for mode in ("eager", "graph"):
+            Y, dX, dW = nan_buf(B, N, bf), nan_buf(B, K, bf), nan_buf(N, K, bf)
+            if mode == "eager":
+                call()
+            else:
+                s = torch.cuda.Stream()
+                with torch.cuda.stream(s):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=s):
+                        call(s.cuda_stream)
+                    g.replay()
+            torch.cuda.synchronize()
+            assert ard.ard_last_device_status(ctx.h) == 0
+            for got, w, name in zip((Y, dX, dW), want, ("fwd", "bwd_data", "bwd_weight")):
+                assert OG.rel_fro(host(got), w) <= TOL[ard.ARD_BF16], (kind, dp, b, mode, name)
