@@ -407,6 +407,16 @@ ard_status ard_rows_bwd_data_compact(ard_ctx* ctx, const ard_rows* rows, int M, 
 ard_status ard_rows_bwd_weight_compact(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N,
                                        float alpha, const void* Ak, int ldak, const void* dYk, int lddyk, void* dW,
                                        int lddw, void* cuda_stream);
+/* Both gathers and the three products of one iteration in one call: Ak and dYk (ceil(M/64)*64 rows each) are
+ * written, then Y, dA and dW as by the three calls above.  The output-gradient half (gather of dY,
+ * backward-data) runs on a stream the context owns beside the input half (gather of A, forward) on the caller's
+ * stream; the weight gradient waits for both gathered matrices; everything is joined into the caller's stream
+ * before the call returns.  The first call on a context creates the stream (make it before any stream
+ * capture); with ARD_MLP_STREAMS=1 in the environment everything stays on the caller's stream.  Asynchronous. */
+ard_status ard_rows_products(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N, float alpha,
+                             const void* A, int lda, const void* W, int ldw, const void* dY, int lddy, void* Ak,
+                             int ldak, void* dYk, int lddyk, void* Y, int ldy, void* dA, int ldda, void* dW, int lddw,
+                             void* cuda_stream);
 /* Test / debug: synchronises; n_keep, the kept rows (at most idx_capacity) and the per-region integers
  * (ceil(M / region_rows) entries) to HOST buffers; idx and region_probability may be NULL. */
 ard_status ard_rows_to_host(const ard_rows* rows, int32_t* n_keep, int32_t* idx, size_t idx_capacity,

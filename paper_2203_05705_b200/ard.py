@@ -35,7 +35,7 @@ EXPORTS = [
     "ard_expand_weight_grad_cols", "ard_bias_grad", "ard_sample_pattern_counter", "ard_mlp_step",
     "ard_rows_create", "ard_rows_destroy", "ard_sensitivity_predict", "ard_rows_set_probability", "ard_rows_sample",
     "ard_rows_to_host", "ard_rows_fwd", "ard_rows_bwd_data", "ard_rows_bwd_weight",
-    "ard_layer_products", "ard_rows_gather", "ard_rows_fwd_compact", "ard_rows_bwd_data_compact", "ard_rows_bwd_weight_compact",
+    "ard_layer_products", "ard_rows_products", "ard_rows_gather", "ard_rows_fwd_compact", "ard_rows_bwd_data_compact", "ard_rows_bwd_weight_compact",
 ]
 
 _lib = None
@@ -116,6 +116,8 @@ def lib():
         "ard_rows_bwd_weight": [vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_layer_products": [vp, vp, i32, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp, i32, i32, vp, i32, vp,
                                i32, i32, vp],
+        "ard_rows_products": [vp, vp, i32, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp,
+                              i32, vp, i32, vp],
         "ard_rows_gather": [vp, vp, i32, i32, vp, i32, vp, i32, vp],
         "ard_rows_fwd_compact": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_rows_bwd_data_compact": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp],
@@ -402,6 +404,13 @@ def ard_layer_products(ctx, pat, dtype, dW_dtype, B, K, N, alpha, X, ldx, W, ldw
     _check(lib().ard_layer_products(ctx, pat, dtype, dW_dtype, B, K, N, alpha, _ptr(X), ldx, _ptr(W), ldw, _ptr(dY),
                                     lddy, _ptr(Y), ldy, outmode, _ptr(dX), lddx, _ptr(dW), lddw, zero_fill_dropped,
                                     _stream(stream)), "ard_layer_products")
+
+
+def ard_rows_products(ctx, rows, dW_dtype, M, K, N, alpha, A, lda, W, ldw, dY, lddy, Ak, ldak, dYk, lddyk, Y, ldy, dA,
+                      ldda, dW, lddw, stream=None):
+    _check(lib().ard_rows_products(ctx, rows, dW_dtype, M, K, N, alpha, _ptr(A), lda, _ptr(W), ldw, _ptr(dY), lddy,
+                                   _ptr(Ak), ldak, _ptr(dYk), lddyk, _ptr(Y), ldy, _ptr(dA), ldda, _ptr(dW), lddw,
+                                   _stream(stream)), "ard_rows_products")
 
 
 def ard_rows_gather(ctx, rows, M, width, src, ld_src, dst, ld_dst, stream=None):

@@ -7,6 +7,7 @@
 #include <new>
 
 #include "ard_internal.h"
+#include <initializer_list>
 
 namespace {
 
@@ -1385,6 +1386,41 @@ ard_status ard_rows_bwd_weight_compact(ard_ctx* ctx, const ard_rows* rows, ard_d
   t.g = g;
   t.bn = ctx->force_bn;
   return launch_gemm_tc(ctx, ARD_ROW, OP_BWD_WEIGHT, t, (cudaStream_t)cuda_stream);
+}
+
+// Gathers and the three products of one iteration in one call, the output-gradient half (gather of dY,
+// backward-data) on the context's side stream beside the input half (gather of A, forward); the weight gradient
+// waits for both gathered matrices.  Each product fills the GPU here, but its dependent launches leave tails and
+// ramps that the other half covers.
+ard_status ard_rows_products(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N, float alpha,
+                             const void* A, int lda, const void* W, int ldw, const void* dY, int lddy, void* Ak,
+                             int ldak, void* dYk, int lddyk, void* Y, int ldy, void* dA, int ldda, void* dW, int lddw,
+                             void* cuda_stream) {
+  if (!ctx || !rows || rows->ctx != ctx) return ARD_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const bool streams = ctx->mlp_two_streams && ard_side_streams(ctx, s);
+  cudaStream_t side = streams ? ctx->side_stream : s;
+  DeviceGuard guard(ctx->device);
+  if (streams) {
+    ARD_CUDA_OK(cudaEventRecord(ctx->ev[100], s));
+    ARD_CUDA_OK(cudaStreamWaitEvent(side, ctx->ev[100], 0));
+  }
+  ard_status st = ard_rows_gather(ctx, rows, M, N, dY, lddy, dYk, lddyk, side);
+  if (streams) ARD_CUDA_OK(cudaEventRecord(ctx->ev[101], side));
+  ard_status st2 = st == ARD_OK ? ard_rows_bwd_data_compact(ctx, rows, M, K, N, alpha, dYk, lddyk, W, ldw, dA, ldda, side) : st;
+  ard_status st3 = ard_rows_gather(ctx, rows, M, K, A, lda, Ak, ldak, s);
+  if (streams) ARD_CUDA_OK(cudaStreamWaitEvent(s, ctx->ev[101], 0));
+  ard_status st4 = (st == ARD_OK && st3 == ARD_OK)
+                       ? ard_rows_bwd_weight_compact(ctx, rows, dW_dtype, M, K, N, alpha, Ak, ldak, dYk, lddyk, dW, lddw, s)
+                       : (st != ARD_OK ? st : st3);
+  ard_status st5 = st3 == ARD_OK ? ard_rows_fwd_compact(ctx, rows, M, K, N, alpha, Ak, ldak, W, ldw, Y, ldy, s) : st3;
+  if (streams) {  // join whatever was enqueued, also after an error, so that a capture is not left forked
+    ARD_CUDA_OK(cudaEventRecord(ctx->ev[102], side));
+    ARD_CUDA_OK(cudaStreamWaitEvent(s, ctx->ev[102], 0));
+  }
+  for (ard_status r : {st, st2, st3, st4, st5})
+    if (r != ARD_OK) return r;
+  return ARD_OK;
 }
 
 ard_status ard_last_device_status(ard_ctx* ctx, void* cuda_stream) {

@@ -159,6 +159,17 @@ def test_products_on_gathered_rows_match_the_oracle(M, K, N):
                 assert OG.rel_fro(dWbh, OC.bwd_weight(A, dY, keep, 1.5).T) <= tol, tag
             else:
                 assert np.all(Yh == 0) and np.all(dAh == 0) and np.all(dWh == 0) and np.all(dWbh == 0), tag
+            # both gathers and the three products behind one call (two streams inside): the same bits
+            Ak2 = torch.full((cap, K), float("nan"), dtype=BF, device="cuda")
+            dYk2 = torch.full((cap, N), float("nan"), dtype=BF, device="cuda")
+            Y2 = torch.full((M, N), float("nan"), dtype=BF, device="cuda")
+            dA2 = torch.full((M, K), float("nan"), dtype=BF, device="cuda")
+            dW2 = torch.full((N, K), float("nan"), dtype=torch.float32, device="cuda")
+            ard.ard_rows_products(ctx.h, rows, ard.ARD_F32, M, K, N, 1.5, Ad, K, Wd, K, dYd, N, Ak2, K, dYk2, N, Y2, N,
+                                  dA2, K, dW2, K)
+            torch.cuda.synchronize()
+            assert ard.ard_last_device_status(ctx.h) == 0
+            assert torch.equal(Y2, Y) and torch.equal(dA2, dA) and torch.equal(dW2, dW), tag
     finally:
         torch.cuda.synchronize()
         ard.ard_rows_destroy(rows)
