@@ -140,7 +140,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // TMA load issued inside a CTA pair: the data lands in this CTA, the byte count is reported to the
-// mbarrier at `bar_cluster`, which may live in the peer CTA.  No multicast.
+// mbarrier at `bar_cluster`, which may live in the peer CTA.  The data goes to this CTA only.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int x,
                                                  int y) {
   asm volatile(
