@@ -135,7 +135,7 @@ struct SmemLayout {
   static constexpr int STG_BYTES = EPI_WARPS * 32 * 33 * 4;
   static constexpr int BAR_OFF = STG_OFF + STG_BYTES;        // full[S], empty[S], tfull[2], tempty[2]
   static constexpr int MISC_OFF = BAR_OFF + (2 * STAGES + 4) * 8;
-  static constexpr int TOTAL = MISC_OFF + 16 + 1024;         // + slack for manual 1024-byte alignment
+  static constexpr int TOTAL = MISC_OFF + 32 + 1024;         // + slack for manual 1024-byte alignment
 };
 
 // Class modes: bytes of the staging area that hold the kept-tile list and the class table.
@@ -187,6 +187,7 @@ struct Sched {
   int workers;             // CTAs (or CTA pairs) sharing the tile loop
   // class modes
   int Tr, nclass, cstep;   // tile-rows; number of classes; distance between members of a class
+  int h_items, light_q;    // class form: items of classes that keep something come first; see unit()
   const int32_t* list;     // kept-tile list the class modes walk (a shared-memory copy when it fits)
   const int4* ctab;        // per class {first item, list offset, list length, members} (shared memory)
   int qn, qm;              // pattern tiles per output tile along N and along M
@@ -239,6 +240,8 @@ struct Sched {
     bn = BN;
     Tr = p.hdr[HDR_TR];
     nclass = cstep = qn = qm = 1;
+    h_items = 0x7fffffff;
+    light_q = 1;
     list = (MODE == M_TILEC_BWD_DATA) ? p.row_idx : p.col_idx;
     ctab = nullptr;
     lts = 31 - __clz(p.ts > 0 ? p.ts : 1);
@@ -350,10 +353,36 @@ struct Sched {
         return true;
       }
     }
-    const int first = SK_MODE ? sk_tiles : 0;
-    u.t = first + w + (i - n_shared) * workers;
     u.kb0 = 0;
     u.kb1 = -1;
+    if (is_class_mode(MODE) && h_items < total) {
+      // Some classes keep nothing: their items only write zeros and cost a fraction of the others.  The others
+      // go round first; then the zero items go, light_q apiece, to the workers that got one item less in
+      // that round, and only what is left of them is dealt to everybody.  (In plain round-robin order a
+      // forward product whose period divides the tile-column count ran its few long items on workers that
+      // afterwards still took their full share of the zero items.)
+      const int a = h_items / workers, rem = h_items - a * workers;
+      const int a_w = a + (w < rem ? 1 : 0);
+      if (i < a_w) {
+        u.t = w + i * workers;
+        return true;
+      }
+      const int ip = i - a_w, n_light = total - h_items;
+      int j;
+      if (rem == 0) {
+        j = w + ip * workers;
+      } else {
+        const int n_less = workers - rem;                  // workers rem .. workers-1
+        const int first_part = min(n_light, n_less * light_q);
+        int n1 = 0;                                         // zero items this worker takes in the first part
+        if (w >= rem && first_part > w - rem) n1 = min(light_q, (first_part - (w - rem) + n_less - 1) / n_less);
+        j = ip < n1 ? (w - rem) + ip * n_less : first_part + w + (ip - n1) * workers;
+      }
+      u.t = h_items + j;
+      return j < n_light;
+    }
+    const int first = SK_MODE ? sk_tiles : 0;
+    u.t = first + w + (i - n_shared) * workers;
     return u.t < total;
   }
 
@@ -367,16 +396,30 @@ struct Sched {
     return Mt * ((cnt + qn - 1) / qn);
   }
   // One thread fills the per-class table in shared memory (at most 64 classes); callers synchronise.
-  __device__ void build_class_table(const TcParams& p, int4* tab, int* total_out) const {
+  // Classes that keep something come first, the empty ones (whose items only write zeros) after them; an entry
+  // is {first item, list offset, list length, members | class << 16}.  out[0] = number of items, out[1] = items
+  // of the non-empty classes, out[2] = how many zero items cost about as much as one of the others.
+  __device__ void build_class_table(const TcParams& p, int4* tab, int* out) const {
     const int32_t* ptr = (MODE == M_TILEC_BWD_DATA) ? p.row_ptr : p.col_ptr;
-    int run = 0;
-    for (int c = 0; c < nclass; ++c) {
-      const int off = ptr[c], len = ptr[c + 1] - off;
-      const int cnt = class_members(c);
-      tab[c] = make_int4(run, off, len, cnt);
-      run += class_items(cnt, len);
+    int run = 0, slot = 0, heavy = 0;
+    long long blocks = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+      for (int c = 0; c < nclass; ++c) {
+        const int off = ptr[c], len = ptr[c + 1] - off;
+        if ((len == 0) != (pass == 1)) continue;
+        const int cnt = class_members(c);
+        const int items = class_items(cnt, len);
+        tab[slot++] = make_int4(run, off, len, cnt | (c << 16));
+        run += items;
+        blocks += (long long)items * len * (p.ts >> 6);
+      }
+      if (pass == 0) heavy = run;
     }
-    *total_out = run;
+    out[0] = run;
+    out[1] = heavy;
+    // an item that only writes zeros takes about as long as 14 contraction blocks
+    const int avg = heavy > 0 ? (int)(blocks / heavy) : 0;
+    out[2] = min(64, max(1, (avg + 14) / 14));
   }
   __device__ TileInfo class_tile(const TcParams& p, int t) const {
     TileInfo ti;
@@ -386,11 +429,11 @@ struct Sched {
     ti.rows_valid = BM;
     ti.n0 = 0;
     const int tmask = p.ts - 1;   // the pattern tile size is a power of two here
-    int c = nclass - 1;
-    while (c > 0 && ctab[c].x > t) --c;  // class whose item range holds t
-    const int4 ce = ctab[c];
+    int sl = nclass - 1;
+    while (sl > 0 && ctab[sl].x > t) --sl;  // table entry whose item range holds t
+    const int4 ce = ctab[sl];
     t -= ce.x;
-    const int cnt = ce.w;
+    const int cnt = ce.w & 0xffff, c = ce.w >> 16;
     const int lsub = lts - 6;     // log2 of the 64-wide boxes per pattern tile
     int nm;                       // pattern tiles along N in this output tile
     if (MODE == M_TILEC_BWD_WEIGHT) {
@@ -654,7 +697,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
     // CLASS_LIST_BYTES of that area; the rest is the epilogue warps' staging (32 rows x 17 words each).
     const int n_list = p.hdr[HDR_NKEEP];
     int4* tab = reinterpret_cast<int4*>(smem + L::STG_OFF + CLASS_LIST_BYTES - 1024);
-    int* total_smem = reinterpret_cast<int*>(smem + L::MISC_OFF + 8);
+    int* total_smem = reinterpret_cast<int*>(smem + L::MISC_OFF + 8);  // [3]: items, items of non-empty classes, light_q
     int32_t* slist = reinterpret_cast<int32_t*>(smem + L::STG_OFF);
     const bool fits = n_list * 4 <= CLASS_LIST_BYTES - 1024;
     if (threadIdx.x == 0) sch.build_class_table(p, tab, total_smem);
@@ -662,7 +705,9 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
       for (int i = threadIdx.x; i < n_list; i += TC_THREADS) slist[i] = sch.list[i];
     __syncthreads();
     sch.ctab = tab;
-    sch.total = *total_smem;
+    sch.total = total_smem[0];
+    sch.h_items = total_smem[1];
+    sch.light_q = total_smem[2];
     if (fits) sch.list = slist;
   }
   const int w0 = (int)blockIdx.x / CTAS;  // first tile of this CTA (pair)
