@@ -21,6 +21,10 @@ Pins (each lives in tests/test_oracle_*.py):
   cnn.*                    decisions that do not depend on the sample; binomial law of the region decision;
                            drop rates of the row sampler; worked row example of Sec. 5.2.1; masked product ==
                            product of the dense small matrix; brute force; adjoint identities
+  cnn_blocks.*             block decisions that do not depend on the sample; one block per group == the row
+                           variant's region; binomial law of a block's count; the bound on sensitive blocks per
+                           group; drop rates of the two labels; loops over kept blocks; all kept == plain product;
+                           adjoint identities
   search.*                 gradient vs central differences; stationary points lie in the Gibbs family
                            ln k_i = beta (i-1)/i + c with beta = -2 (k.p_u - p)/lambda; small-lambda limit ==
                            the maximum-entropy distribution at rate p; Eq. 2-3 in exact rationals
@@ -29,6 +33,6 @@ Parity unpinned (the paper fixes no value to compare with): the constants of the
 distribution search (the body of Algorithm 1 is not printed: loss form, lambda, step size, start and
 stopping rule are a reading, see search.py) and therefore the authors' own K, the tile
 linearisation order beyond the first tile of the worked example, every constant of the
-sensitivity prediction (region shape, which values are sampled, k, t, threshold, m, n: see cnn.py), the LSTM
+sensitivity prediction (region shape, which values are sampled, k, t, threshold, m, n: see cnn.py; the balancing rule of the block variant: see cnn_blocks.py), the LSTM
 reading (which units are dropped, gate order) and the rescale convention.
 """
