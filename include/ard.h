@@ -44,6 +44,7 @@ extern "C" {
 typedef struct ard_ctx ard_ctx;         /* owns distributions, workspace, descriptor cache, status word */
 typedef struct ard_pattern ard_pattern; /* handle of a device-resident pattern (header + index lists)   */
 typedef struct ard_rows ard_rows;       /* handle of a device-resident list of kept input-matrix rows   */
+typedef struct ard_blocks ard_blocks;   /* handle of a device-resident set of kept input-matrix blocks  */
 
 typedef enum {
   ARD_OK = 0,
@@ -421,6 +422,59 @@ ard_status ard_rows_products(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dt
  * (ceil(M / region_rows) entries) to HOST buffers; idx and region_probability may be NULL. */
 ard_status ard_rows_to_host(const ard_rows* rows, int32_t* n_keep, int32_t* idx, size_t idx_capacity,
                             uint32_t* region_probability, void* cuda_stream);
+
+/* ---- block-based sensitivity-aware dropout of a convolution layer's input matrix (Sec. 5.1, 5.2.2) ----
+ * The input matrix A [M][Kc] is cut into ts x ts blocks; the Q = Kc/ts blocks that share their rows are a
+ * group, there are G = M/ts groups (ts divides M and Kc; the tensor-core products need ts a multiple of 64).
+ * A block is the dropout granularity.  Sec. 5.2.2 bounds the number of sensitive blocks per group so that
+ * all groups keep nearly the same amount of work.  The paper fixes no constant, and the figure that shows the
+ * balancing is not available; this library's reading: the prediction of Sec. 5.1 with one block as the
+ * region (s = max(1, floor(k_frac*ts*ts + 1/2)) samples; sample d of block g*Q + j is word (d mod 4) of the
+ * Philox4x32-10 block with key (seed) and counter (iteration low, iteration high, g*Q + j,
+ * stream_id * 65536 + d div 4), at position floor(word * ts*ts / 2^32) of the block, row-major; a block passes
+ * iff at least max(1, ceil(t_frac * s)) sampled values are > threshold); of a group's passing blocks the
+ * `cap` with the highest counts are sensitive (equal counts: lower j first); block g*Q + j is dropped iff
+ * word 0 of the Philox block with counter (iteration low, iteration high, g*Q + j, stream_id * 65536 + 65535)
+ * is below min(floor(p 2^32), 2^32 - 1), p = m_prob for a sensitive block, n_prob otherwise.
+ * stream_id < 65536.  Everything stays on the device; ard_blocks_to_host is for tests. */
+ard_status ard_blocks_create(ard_ctx* ctx, ard_blocks** blocks, int M, int Kc, int ts);
+ard_status ard_blocks_destroy(ard_blocks* blocks);
+/* Counts and labels of all blocks.  A [M][Kc] (lda) on the device, element type dtype.  Asynchronous. */
+ard_status ard_blocks_predict(ard_ctx* ctx, ard_blocks* blocks, ard_dtype dtype, const void* A, int lda, double k_frac,
+                              double t_frac, float threshold, int cap, uint64_t seed, uint64_t iteration,
+                              uint32_t stream_id, void* cuda_stream);
+/* The same label for every block (tests; with ard_blocks_sample(m_prob = n_prob = 0) everything is kept). */
+ard_status ard_blocks_set_label(ard_ctx* ctx, ard_blocks* blocks, int sensitive, void* cuda_stream);
+/* Draws the dropped blocks and writes the kept blocks' index lists (those of a tile pattern over [Kc x M]
+ * with tile (r, c) = (block j, group g), all ascending).  Asynchronous. */
+ard_status ard_blocks_sample(ard_ctx* ctx, ard_blocks* blocks, double m_prob, double n_prob, uint64_t seed,
+                             uint64_t iteration, uint32_t stream_id, void* cuda_stream);
+/* The three products over the kept blocks (bf16 operands on the tensor cores, fp32 accumulation; only kept
+ * blocks of A are fetched).  W [N][Kc] (ldw) are the filters, neuron-major as everywhere here.  The output
+ * matrix and its gradient are held TRANSPOSED, Yt / dYt [N][M] (one row per output channel, the layout of
+ * the layer's output feature map), because the products are the tile-pattern products of Sec. 3.2 with the
+ * filters as the batch operand and A as the masked matrix:
+ *   ard_blocks_fwd         Yt = alpha * W (A .* mask)^T
+ *   ard_blocks_bwd_weight  dW = alpha * dYt (A .* mask)                       dW [N][Kc] (lddw), bf16
+ *   ard_blocks_bwd_input   dA = alpha * (dYt^T W) .* mask                     dA [M][Kc] (ldda), dA_dtype;
+ *                          dropped blocks are written as zero if zero_fill_dropped != 0, else left untouched
+ * Requires 16-byte aligned pointers, leading dimensions that are multiples of 8 elements, N >= 1
+ * (ARD_ERR_ALIGNMENT / ARD_ERR_UNSUPPORTED otherwise: there is no second kernel family for this part).
+ * Asynchronous. */
+ard_status ard_blocks_fwd(ard_ctx* ctx, const ard_blocks* blocks, int N, float alpha, const void* A, int lda,
+                          const void* W, int ldw, void* Yt, int ldyt, void* cuda_stream);
+ard_status ard_blocks_bwd_weight(ard_ctx* ctx, const ard_blocks* blocks, int N, float alpha, const void* A, int lda,
+                                 const void* dYt, int lddyt, void* dW, int lddw, void* cuda_stream);
+ard_status ard_blocks_bwd_input(ard_ctx* ctx, const ard_blocks* blocks, ard_dtype dA_dtype, int N, float alpha,
+                                const void* dYt, int lddyt, const void* W, int ldw, void* dA, int ldda,
+                                int zero_fill_dropped, void* cuda_stream);
+/* Test / debug: synchronises; per block g*Q + j its count, label and kept flag to HOST buffers of G*Q entries
+ * (any may be NULL). */
+ard_status ard_blocks_to_host(const ard_blocks* blocks, int32_t* counts, uint8_t* sensitive, uint8_t* keep,
+                              void* cuda_stream);
+/* The tile pattern that holds the lists (for ard_pattern_to_host / ard_pattern_tile_lists_to_host); owned by
+ * `blocks`. */
+const ard_pattern* ard_blocks_pattern(const ard_blocks* blocks);
 
 /* ---- LSTM cell on the kept hidden units (Sec. 7: an LSTM step is again a matrix
  * product; one row pattern over the H hidden units serves every time step) -------------

@@ -36,6 +36,8 @@ EXPORTS = [
     "ard_rows_create", "ard_rows_destroy", "ard_sensitivity_predict", "ard_rows_set_probability", "ard_rows_sample",
     "ard_rows_to_host", "ard_rows_fwd", "ard_rows_bwd_data", "ard_rows_bwd_weight",
     "ard_layer_products", "ard_rows_products", "ard_rows_gather", "ard_rows_fwd_compact", "ard_rows_bwd_data_compact", "ard_rows_bwd_weight_compact",
+    "ard_blocks_create", "ard_blocks_destroy", "ard_blocks_predict", "ard_blocks_set_label", "ard_blocks_sample",
+    "ard_blocks_fwd", "ard_blocks_bwd_weight", "ard_blocks_bwd_input", "ard_blocks_to_host", "ard_blocks_pattern",
 ]
 
 _lib = None
@@ -104,6 +106,15 @@ def lib():
         "ard_bias_grad": [vp, vp, i32, i32, i32, vp, i32, i32, vp, i32, vp],
         "ard_sample_pattern_counter": [vp, vp, i32, u64, u64, vp, i32, u32, vp],
         "ard_mlp_step": [vp, P(MlpLayer), i32, i32, vp, i32, vp, i32, vp, i32, i32, u64, u64, vp, vp],
+        "ard_blocks_create": [vp, P(vp), i32, i32, i32],
+        "ard_blocks_destroy": [vp],
+        "ard_blocks_predict": [vp, vp, i32, vp, i32, C.c_double, C.c_double, f32, i32, u64, u64, u32, vp],
+        "ard_blocks_set_label": [vp, vp, i32, vp],
+        "ard_blocks_sample": [vp, vp, C.c_double, C.c_double, u64, u64, u32, vp],
+        "ard_blocks_fwd": [vp, vp, i32, f32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_blocks_bwd_weight": [vp, vp, i32, f32, vp, i32, vp, i32, vp, i32, vp],
+        "ard_blocks_bwd_input": [vp, vp, i32, i32, f32, vp, i32, vp, i32, vp, i32, i32, vp],
+        "ard_blocks_to_host": [vp, P(C.c_int32), P(C.c_uint8), P(C.c_uint8), vp],
         "ard_rows_create": [vp, P(vp), i32, i32],
         "ard_rows_destroy": [vp],
         "ard_sensitivity_predict": [vp, vp, i32, vp, i32, i32, C.c_double, C.c_double, f32, C.c_double, C.c_double, u64, u64,
@@ -128,6 +139,8 @@ def lib():
         fn.argtypes = args
         fn.restype = i32
     L.ard_launch_count.restype = u64
+    L.ard_blocks_pattern.argtypes = [vp]
+    L.ard_blocks_pattern.restype = vp
     L.ard_status_string.argtypes = [i32]
     L.ard_status_string.restype = C.c_char_p
     _lib = L
@@ -347,6 +360,61 @@ def ard_mlp_step(ctx, layers, n_layers, B, X, ldx, dOut, lddout, dX, lddx, dist_
     """`layers`: the array made by mlp_layers()."""
     _check(lib().ard_mlp_step(ctx, layers, n_layers, B, _ptr(X), ldx, _ptr(dOut), lddout, _ptr(dX), lddx, dist_id,
                               seed, iteration_base, _ptr(iteration_counter), _stream(stream)), "ard_mlp_step")
+
+
+def ard_blocks_create(ctx, M, Kc, ts):
+    h = C.c_void_p()
+    _check(lib().ard_blocks_create(ctx, C.byref(h), M, Kc, ts), "ard_blocks_create")
+    return h
+
+
+def ard_blocks_destroy(blocks):
+    _check(lib().ard_blocks_destroy(blocks), "ard_blocks_destroy")
+
+
+def ard_blocks_predict(ctx, blocks, dtype, A, lda, k_frac, t_frac, threshold, cap, seed, iteration, stream_id,
+                       stream=None):
+    _check(lib().ard_blocks_predict(ctx, blocks, dtype, _ptr(A), lda, k_frac, t_frac, threshold, cap, seed, iteration,
+                                    stream_id, _stream(stream)), "ard_blocks_predict")
+
+
+def ard_blocks_set_label(ctx, blocks, sensitive, stream=None):
+    _check(lib().ard_blocks_set_label(ctx, blocks, sensitive, _stream(stream)), "ard_blocks_set_label")
+
+
+def ard_blocks_sample(ctx, blocks, m_prob, n_prob, seed, iteration, stream_id, stream=None):
+    _check(lib().ard_blocks_sample(ctx, blocks, m_prob, n_prob, seed, iteration, stream_id, _stream(stream)),
+           "ard_blocks_sample")
+
+
+def ard_blocks_fwd(ctx, blocks, N, alpha, A, lda, W, ldw, Yt, ldyt, stream=None):
+    _check(lib().ard_blocks_fwd(ctx, blocks, N, alpha, _ptr(A), lda, _ptr(W), ldw, _ptr(Yt), ldyt, _stream(stream)),
+           "ard_blocks_fwd")
+
+
+def ard_blocks_bwd_weight(ctx, blocks, N, alpha, A, lda, dYt, lddyt, dW, lddw, stream=None):
+    _check(lib().ard_blocks_bwd_weight(ctx, blocks, N, alpha, _ptr(A), lda, _ptr(dYt), lddyt, _ptr(dW), lddw,
+                                       _stream(stream)), "ard_blocks_bwd_weight")
+
+
+def ard_blocks_bwd_input(ctx, blocks, dA_dtype, N, alpha, dYt, lddyt, W, ldw, dA, ldda, zero_fill_dropped, stream=None):
+    _check(lib().ard_blocks_bwd_input(ctx, blocks, dA_dtype, N, alpha, _ptr(dYt), lddyt, _ptr(W), ldw, _ptr(dA), ldda,
+                                      zero_fill_dropped, _stream(stream)), "ard_blocks_bwd_input")
+
+
+def ard_blocks_to_host(blocks, n_blocks, stream=None):
+    """Returns (counts, sensitive, keep), one entry per block g*Q + j."""
+    counts = np.zeros(n_blocks, dtype=np.int32)
+    sens = np.zeros(n_blocks, dtype=np.uint8)
+    keep = np.zeros(n_blocks, dtype=np.uint8)
+    _check(lib().ard_blocks_to_host(blocks, counts.ctypes.data_as(C.POINTER(C.c_int32)),
+                                    sens.ctypes.data_as(C.POINTER(C.c_uint8)), keep.ctypes.data_as(C.POINTER(C.c_uint8)),
+                                    _stream(stream)), "ard_blocks_to_host")
+    return counts, sens, keep
+
+
+def ard_blocks_pattern(blocks):
+    return C.c_void_p(lib().ard_blocks_pattern(blocks))
 
 
 def ard_rows_create(ctx, M, region_rows):
