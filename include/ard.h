@@ -423,6 +423,22 @@ ard_status ard_rows_products(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dt
 ard_status ard_rows_to_host(const ard_rows* rows, int32_t* n_keep, int32_t* idx, size_t idx_capacity,
                             uint32_t* region_probability, void* cuda_stream);
 
+/* Sec. 5.3, Eq. 12-14: the dropout probability of every training epoch, on the host in fp64 (no context or GPU
+ * needed): low at the start, rising, lower again towards the end, with the shape of the skew-normal density
+ *   f(y) = (2/sigma) phi((y-mu)/sigma) Phi(lambda (y-mu)/sigma)                                     (Eq. 12)
+ * whose parameters follow from a prescribed expectation and variance through
+ *   E = mu + mu0 sigma, mu0 = sqrt(2/pi) lambda / sqrt(1+lambda^2);  D = (1 - mu0^2) sigma^2       (Eq. 13, 14).
+ * The paper does not say what the axis or the scale of the curve are; this library's reading: the axis is the
+ * epoch number e = 0..n_epochs-1, mean_epoch and var_epoch are E and D along it, and
+ *   p_out[e] = min(p_max, p_total * n_epochs * f(e) / sum_e' f(e')),
+ * so the mean over the epochs is p_total unless an entry was clipped.  A training loop passes p_out[e] (or a
+ * pair of values derived from it) as the probabilities of ard_sensitivity_predict / ard_blocks_sample.
+ * p_out: HOST array of n_epochs doubles.  Errors: ARD_ERR_INVALID_ARG (NULL, n_epochs < 1, probabilities
+ * outside [0,1], var_epoch <= 0, non-finite arguments), ARD_ERR_UNSUPPORTED (the curve underflows to zero on
+ * every epoch). */
+ard_status ard_dropout_schedule(int n_epochs, double p_total, double mean_epoch, double var_epoch, double lambda,
+                                double p_max, double* p_out);
+
 /* ---- block-based sensitivity-aware dropout of a convolution layer's input matrix (Sec. 5.1, 5.2.2) ----
  * The input matrix A [M][Kc] is cut into ts x ts blocks; the Q = Kc/ts blocks that share their rows are a
  * group, there are G = M/ts groups (ts divides M and Kc; the tensor-core products need ts a multiple of 64).

@@ -25,6 +25,8 @@ Pins (each lives in tests/test_oracle_*.py):
                            variant's region; binomial law of a block's count; the bound on sensitive blocks per
                            group; drop rates of the two labels; loops over kept blocks; all kept == plain product;
                            adjoint identities
+  schedule.*               Eq. 12 == the library's skew-normal density, integrates to one; Eq. 13-14 by numerical
+                           integration; shape 0 == normal; prescribed mean of the scaled curve; one maximum
   search.*                 gradient vs central differences; stationary points lie in the Gibbs family
                            ln k_i = beta (i-1)/i + c with beta = -2 (k.p_u - p)/lambda; small-lambda limit ==
                            the maximum-entropy distribution at rate p; Eq. 2-3 in exact rationals
@@ -33,6 +35,7 @@ Parity unpinned (the paper fixes no value to compare with): the constants of the
 distribution search (the body of Algorithm 1 is not printed: loss form, lambda, step size, start and
 stopping rule are a reading, see search.py) and therefore the authors' own K, the tile
 linearisation order beyond the first tile of the worked example, every constant of the
-sensitivity prediction (region shape, which values are sampled, k, t, threshold, m, n: see cnn.py; the balancing rule of the block variant: see cnn_blocks.py), the LSTM
+sensitivity prediction (region shape, which values are sampled, k, t, threshold, m, n: see cnn.py; the balancing rule of the block variant: see cnn_blocks.py; axis and scale of the dropout-probability curve over the
+epochs: see schedule.py), the LSTM
 reading (which units are dropped, gate order) and the rescale convention.
 """

@@ -37,7 +37,7 @@ EXPORTS = [
     "ard_rows_to_host", "ard_rows_fwd", "ard_rows_bwd_data", "ard_rows_bwd_weight",
     "ard_layer_products", "ard_rows_products", "ard_rows_gather", "ard_rows_fwd_compact", "ard_rows_bwd_data_compact", "ard_rows_bwd_weight_compact",
     "ard_blocks_create", "ard_blocks_destroy", "ard_blocks_predict", "ard_blocks_set_label", "ard_blocks_sample",
-    "ard_blocks_fwd", "ard_blocks_bwd_weight", "ard_blocks_bwd_input", "ard_blocks_to_host", "ard_blocks_pattern",
+    "ard_blocks_fwd", "ard_blocks_bwd_weight", "ard_blocks_bwd_input", "ard_blocks_to_host", "ard_blocks_pattern", "ard_dropout_schedule",
 ]
 
 _lib = None
@@ -106,6 +106,7 @@ def lib():
         "ard_bias_grad": [vp, vp, i32, i32, i32, vp, i32, i32, vp, i32, vp],
         "ard_sample_pattern_counter": [vp, vp, i32, u64, u64, vp, i32, u32, vp],
         "ard_mlp_step": [vp, P(MlpLayer), i32, i32, vp, i32, vp, i32, vp, i32, i32, u64, u64, vp, vp],
+        "ard_dropout_schedule": [i32, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, P(C.c_double)],
         "ard_blocks_create": [vp, P(vp), i32, i32, i32],
         "ard_blocks_destroy": [vp],
         "ard_blocks_predict": [vp, vp, i32, vp, i32, C.c_double, C.c_double, f32, i32, u64, u64, u32, vp],
@@ -360,6 +361,13 @@ def ard_mlp_step(ctx, layers, n_layers, B, X, ldx, dOut, lddout, dX, lddx, dist_
     """`layers`: the array made by mlp_layers()."""
     _check(lib().ard_mlp_step(ctx, layers, n_layers, B, _ptr(X), ldx, _ptr(dOut), lddout, _ptr(dX), lddx, dist_id,
                               seed, iteration_base, _ptr(iteration_counter), _stream(stream)), "ard_mlp_step")
+
+
+def ard_dropout_schedule(n_epochs, p_total, mean_epoch, var_epoch, lam, p_max=1.0):
+    out = np.zeros(max(n_epochs, 1), dtype=np.float64)
+    _check(lib().ard_dropout_schedule(n_epochs, p_total, mean_epoch, var_epoch, lam, p_max,
+                                      out.ctypes.data_as(C.POINTER(C.c_double))), "ard_dropout_schedule")
+    return out[:n_epochs]
 
 
 def ard_blocks_create(ctx, M, Kc, ts):

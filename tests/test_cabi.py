@@ -112,6 +112,23 @@ def test_host_side_distribution_search_matches_the_oracle(built):
         ard.ard_search_distribution(0.5, 16, lam=0.0)
 
 
+def test_host_side_dropout_schedule_matches_the_oracle(built):
+    """Sec. 5.3 on the host: the library's curve against the oracle's statement of Eq. 12-14, and the rejections."""
+    import numpy as np
+    from oracle import schedule as OSch
+    from paper_2203_05705_b200 import ard
+    for n, p, E, D, lam, pmax in [(60, 0.4, 35.0, 150.0, -3.0, 1.0), (30, 0.5, 12.0, 20.0, 2.0, 0.7), (10, 0.3, 4.5, 9.0, 0.0, 1.0),
+                                  (200, 0.6, 120.0, 900.0, -6.0, 0.9), (1, 0.25, 0.0, 1.0, 1.0, 1.0)]:
+        got = ard.ard_dropout_schedule(n, p, E, D, lam, pmax)
+        want = np.asarray(OSch.schedule(n, p, E, D, lam, pmax))
+        assert np.abs(got - want).max() <= 1e-12, (n, p, E, D, lam)
+        assert got.max() <= pmax
+    for args in [(0, 0.4, 1.0, 1.0, 0.0), (10, 1.4, 1.0, 1.0, 0.0), (10, 0.4, 1.0, 0.0, 0.0), (10, 0.4, float("nan"), 1.0, 0.0),
+                 (10, 0.4, 1e6, 1.0, 0.0)]:
+        with pytest.raises(ard.ArdError):
+            ard.ard_dropout_schedule(*args)
+
+
 def test_header_is_plain_c(tmp_path):
     """The boundary is a C ABI: the header must compile as C99 on its own (no C++ or CUDA types)."""
     import shutil
