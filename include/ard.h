@@ -484,6 +484,13 @@ ard_status ard_blocks_bwd_weight(ard_ctx* ctx, const ard_blocks* blocks, int N, 
 ard_status ard_blocks_bwd_input(ard_ctx* ctx, const ard_blocks* blocks, ard_dtype dA_dtype, int N, float alpha,
                                 const void* dYt, int lddyt, const void* W, int ldw, void* dA, int ldda,
                                 int zero_fill_dropped, void* cuda_stream);
+/* The three products of one iteration behind one call, enqueued side by side on the context's streams as by
+ * ard_layer_products (same first-call and capture rules), joined into the caller's stream before the call
+ * returns; results as by the three calls above.  Asynchronous. */
+ard_status ard_blocks_products(ard_ctx* ctx, const ard_blocks* blocks, ard_dtype dA_dtype, int N, float alpha,
+                               const void* A, int lda, const void* W, int ldw, const void* dYt, int lddyt, void* Yt,
+                               int ldyt, void* dW, int lddw, void* dA, int ldda, int zero_fill_dropped,
+                               void* cuda_stream);
 /* Test / debug: synchronises; per block g*Q + j its count, label and kept flag to HOST buffers of G*Q entries
  * (any may be NULL). */
 ard_status ard_blocks_to_host(const ard_blocks* blocks, int32_t* counts, uint8_t* sensitive, uint8_t* keep,

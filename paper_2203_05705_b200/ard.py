@@ -37,7 +37,7 @@ EXPORTS = [
     "ard_rows_to_host", "ard_rows_fwd", "ard_rows_bwd_data", "ard_rows_bwd_weight",
     "ard_layer_products", "ard_rows_products", "ard_rows_gather", "ard_rows_fwd_compact", "ard_rows_bwd_data_compact", "ard_rows_bwd_weight_compact",
     "ard_blocks_create", "ard_blocks_destroy", "ard_blocks_predict", "ard_blocks_set_label", "ard_blocks_sample",
-    "ard_blocks_fwd", "ard_blocks_bwd_weight", "ard_blocks_bwd_input", "ard_blocks_to_host", "ard_blocks_pattern", "ard_dropout_schedule",
+    "ard_blocks_fwd", "ard_blocks_bwd_weight", "ard_blocks_bwd_input", "ard_blocks_to_host", "ard_blocks_pattern", "ard_dropout_schedule", "ard_blocks_products",
 ]
 
 _lib = None
@@ -115,6 +115,7 @@ def lib():
         "ard_blocks_fwd": [vp, vp, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_blocks_bwd_weight": [vp, vp, i32, f32, vp, i32, vp, i32, vp, i32, vp],
         "ard_blocks_bwd_input": [vp, vp, i32, i32, f32, vp, i32, vp, i32, vp, i32, i32, vp],
+        "ard_blocks_products": [vp, vp, i32, i32, f32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, vp, i32, i32, vp],
         "ard_blocks_to_host": [vp, P(C.c_int32), P(C.c_uint8), P(C.c_uint8), vp],
         "ard_rows_create": [vp, P(vp), i32, i32],
         "ard_rows_destroy": [vp],
@@ -408,6 +409,13 @@ def ard_blocks_bwd_weight(ctx, blocks, N, alpha, A, lda, dYt, lddyt, dW, lddw, s
 def ard_blocks_bwd_input(ctx, blocks, dA_dtype, N, alpha, dYt, lddyt, W, ldw, dA, ldda, zero_fill_dropped, stream=None):
     _check(lib().ard_blocks_bwd_input(ctx, blocks, dA_dtype, N, alpha, _ptr(dYt), lddyt, _ptr(W), ldw, _ptr(dA), ldda,
                                       zero_fill_dropped, _stream(stream)), "ard_blocks_bwd_input")
+
+
+def ard_blocks_products(ctx, blocks, dA_dtype, N, alpha, A, lda, W, ldw, dYt, lddyt, Yt, ldyt, dW, lddw, dA, ldda,
+                        zero_fill_dropped, stream=None):
+    _check(lib().ard_blocks_products(ctx, blocks, dA_dtype, N, alpha, _ptr(A), lda, _ptr(W), ldw, _ptr(dYt), lddyt,
+                                     _ptr(Yt), ldyt, _ptr(dW), lddw, _ptr(dA), ldda, zero_fill_dropped, _stream(stream)),
+           "ard_blocks_products")
 
 
 def ard_blocks_to_host(blocks, n_blocks, stream=None):

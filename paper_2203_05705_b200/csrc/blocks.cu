@@ -416,6 +416,28 @@ ard_status ard_blocks_bwd_input(ard_ctx* ctx, const ard_blocks* b, ard_dtype dA_
                         cuda_stream);
 }
 
+ard_status ard_blocks_products(ard_ctx* ctx, const ard_blocks* b, ard_dtype dA_dtype, int N, float alpha, const void* A,
+                               int lda, const void* W, int ldw, const void* dYt, int lddyt, void* Yt, int ldyt, void* dW,
+                               int lddw, void* dA, int ldda, int zero_fill_dropped, void* cuda_stream) {
+  if (!ctx || !b || b->ctx != ctx || !dA) return ARD_ERR_INVALID_ARG;
+  if (dA_dtype != ARD_F32 && dA_dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (ldda < b->Kc || N < 1) return ARD_ERR_SHAPE;
+  DevGuard guard(ctx->device);
+  if (zero_fill_dropped) {
+    // on the caller's stream, before the fork: the input gradient's stream waits for it
+    const int es = dA_dtype == ARD_F32 ? 4 : 2;
+    const int nblocks = b->G * b->Q;
+    const int grid = nblocks < ctx->sm_count * 32 ? nblocks : ctx->sm_count * 32;
+    ARD_CUDA_OK(ard_launch(ctx, zero_dropped_blocks_kernel, dim3(grid), dim3(256), 0, (cudaStream_t)cuda_stream,
+                           (const uint8_t*)b->d_keep, nblocks, b->Q, b->ts, dA, ldda * es, es));
+    ctx->launches++;
+    ARD_CUDA_OK(cudaGetLastError());
+  }
+  PathGuard path(ctx);
+  return ard_layer_products(ctx, b->pat, ARD_BF16, dA_dtype, N, b->Kc, b->M, alpha, W, ldw, A, lda, dYt, lddyt, Yt, ldyt,
+                            ARD_OUT_SCATTER_ZEROFILL, dW, lddw, dA, ldda, 0, cuda_stream);
+}
+
 ard_status ard_blocks_to_host(const ard_blocks* b, int32_t* counts, uint8_t* sensitive, uint8_t* keep,
                               void* cuda_stream) {
   if (!b) return ARD_ERR_INVALID_ARG;

@@ -104,8 +104,14 @@ def test_products_over_the_kept_blocks_match_the_oracle(M, Kc, N, ts):
             ard.ard_blocks_bwd_weight(ctx.h, blocks, N, 1.5, Ad, Kc, dYt, M, dW, Kc)
             ard.ard_blocks_bwd_input(ctx.h, blocks, ard.ARD_F32, N, 1.5, dYt, M, Wd, Kc, dA, Kc, 1)
             ard.ard_blocks_bwd_input(ctx.h, blocks, ard.ARD_BF16, N, 1.5, dYt, M, Wd, Kc, dA2, Kc, 0)
+            # the same through the one-call form
+            Yt3 = torch.full((N, ldy), float("nan"), dtype=BF, device="cuda")
+            dW3 = torch.full((N, Kc), float("nan"), dtype=BF, device="cuda")
+            dA3 = torch.full((M, Kc), float("nan"), dtype=torch.float32, device="cuda")
+            ard.ard_blocks_products(ctx.h, blocks, ard.ARD_F32, N, 1.5, Ad, Kc, Wd, Kc, dYt, M, Yt3, ldy, dW3, Kc, dA3, Kc, 1)
             torch.cuda.synchronize()
             assert ard.ard_last_device_status(ctx.h) == 0
+            assert torch.equal(Yt3[:, :M], Yt[:, :M]) and torch.equal(dW3, dW) and torch.equal(dA3, dA)
             tag = (M, Kc, N, ts, p, int(keep.sum()))
             Yh, dWh, dAh, dA2h = host(Yt)[:, :M].T, host(dW).T, host(dA), host(dA2)
             assert np.all(dAh[~mask] == 0), tag
