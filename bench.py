@@ -11,7 +11,8 @@ Table-1 sweep scaled to B200: W 8192x8192 bf16, batch 4096, row pattern, p = 0.5
 maximum-entropy distribution over periods 1..16.  Other workloads (`--workload`): `mlp8192_tile`,
 `mlp4096_tile`, `mlp2048_row` (single layers), `lstm1024` (a step is a whole sequence, forward + BPTT),
 `mlp2048_step` / `mlp8192_step` (a step is a whole training iteration of a stack of layers, replayed from a
-CUDA graph), `conv_rows` (a convolution layer as an im2col product with rows dropped by predicted sensitivity).
+CUDA graph), `conv_rows` (a convolution layer as an im2col product with rows dropped by predicted sensitivity),
+`conv_blocks` (the same layer with blocks of the input matrix dropped).
 """
 from __future__ import annotations
 
@@ -53,6 +54,9 @@ WORKLOADS = {
     # dropped by predicted sensitivity (Sec. 5.1, 5.2.1): 3x3 filters, 256 -> 512 channels, 32768 output positions
     "conv_rows": dict(config=5, M=32768, K=2304, N=512, kind="conv_rows", region_rows=8, k_frac=0.05, t_frac=0.3,
                       threshold=0.5, m_prob=0.2, n_prob=0.8),
+    # the same layer with blocks of the input matrix as the dropout granularity (Sec. 5.2.2)
+    "conv_blocks": dict(config=5, M=32768, K=2304, N=512, kind="conv_blocks", ts=128, k_frac=0.05, t_frac=0.3,
+                        threshold=0.5, cap=6, m_prob=0.2, n_prob=0.8),
     # LSTM layer (config 4): a step is one sequence, forward + BPTT, one fresh pattern per sequence
     "lstm1024": dict(config=4, T=35, B=64, I=1024, H=1024, kind="lstm", p=0.5, n_dp=16),
 }
@@ -730,6 +734,138 @@ def run_conv_rows(args, wl):
     ard.ard_destroy(ctx)
 
 
+def run_conv_blocks(args, wl):
+    """A step = per-block sensitivity counts + labels (at most `cap` sensitive blocks per group) + block draws +
+    index lists + the three products over the kept blocks of the input matrix, through ard_blocks_products."""
+    import torch
+    from paper_2203_05705_b200 import ard
+    dev_index = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(dev_index)
+    clocks = ClockSampler(dev_index)
+    M, K, N, ts = wl["M"], wl["K"], wl["N"], wl["ts"]
+    G, Q = M // ts, K // ts
+    bf = torch.bfloat16
+    g = torch.Generator(device="cuda").manual_seed(inputs.BASE_SEED)
+    # post-ReLU-like input matrix with quiet and busy blocks, so that both labels occur
+    level = torch.tensor([0.1, 1.0, 4.0], device="cuda")[torch.randint(0, 3, (G, Q), device="cuda", generator=g)]
+    A = (torch.relu(torch.randn((M, K), device="cuda", generator=g))
+         * level.repeat_interleave(ts, 0).repeat_interleave(ts, 1)).to(bf)
+    W = (torch.randn((N, K), device="cuda", generator=g) / K ** 0.5).to(bf)
+    dYt = torch.randn((N, M), device="cuda", generator=g).to(bf)       # output gradient, one row per channel
+    Yt = torch.empty((N, M), dtype=bf, device="cuda")
+    dA = torch.empty((M, K), dtype=bf, device="cuda")
+    dW = torch.empty((N, K), dtype=bf, device="cuda")
+    hA, hdY = A.cpu().pin_memory(), dYt.cpu().pin_memory()
+    hY = torch.empty((N, M), dtype=bf).pin_memory()
+    ctx = ard.ard_create(0, 4096)
+    blocks = ard.ard_blocks_create(ctx, M, K, ts)
+
+    def sample(it):
+        ard.ard_blocks_predict(ctx, blocks, ard.ARD_BF16, A, K, wl["k_frac"], wl["t_frac"], wl["threshold"], wl["cap"],
+                               inputs.BASE_SEED, it, 0)
+        ard.ard_blocks_sample(ctx, blocks, wl["m_prob"], wl["n_prob"], inputs.BASE_SEED, it, 0)
+
+    def products():
+        ard.ard_blocks_products(ctx, blocks, ard.ARD_BF16, N, 1.0, A, K, W, K, dYt, M, Yt, M, dW, K, dA, K, 1)
+
+    def step(it, host=False, dense=False):
+        if host:
+            A.copy_(hA, non_blocking=True)
+            dYt.copy_(hdY, non_blocking=True)
+        if dense:
+            ard.ard_blocks_set_label(ctx, blocks, 1)
+            ard.ard_blocks_sample(ctx, blocks, 0.0, 0.0, inputs.BASE_SEED, it, 0)
+        else:
+            sample(it)
+        products()
+        if host:
+            hY.copy_(Yt, non_blocking=True)
+
+    def timed(fn, n, warm):
+        for w in range(warm):
+            fn(w)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record()
+        for i in range(n):
+            fn(warm + i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1), t0, time.time()
+
+    steps, warm = args.steps, max(3, args.warmup)
+    l0 = ard.ard_launch_count(ctx)
+    ms, t0, t1 = timed(step, steps, warm)
+    launches = (ard.ard_launch_count(ctx) - l0) * steps // (steps + warm)
+    clk = clocks.stop(t0, t1)
+    status = ard.ard_last_device_status(ctx)
+    kept_blocks = []
+    for i in range(steps):
+        sample(warm + i)
+        kept_blocks.append(int(ard.ard_blocks_to_host(blocks, G * Q)[2].sum()))
+    flops_per_block = 3 * 2.0 * ts * ts * N
+    value = sum(kept_blocks) * flops_per_block / (ms * 1e-3) / 1e12
+    detail = {"ms_per_step": {"ours": ms / steps}, "kept_block_fraction": float(np.mean(kept_blocks)) / (G * Q)}
+    e2e = None
+    if not args.quick:
+        n2 = max(5, steps // 4)
+        detail["ms_per_step"]["own_kernels_all_blocks"] = timed(lambda it: step(it, dense=True), n2, warm)[0] / n2
+        detail["us_per_stage"] = {"predict+sample": round(timed(sample, n2, warm)[0] / n2 * 1e3, 1)}
+        sample(1)
+        detail["us_per_stage"]["products"] = round(timed(lambda it: products(), n2, warm)[0] / n2 * 1e3, 1)
+
+        def torch_step(it):
+            torch.matmul(W, A.t(), out=Yt)
+            torch.matmul(dYt, A, out=dW)
+            torch.matmul(dYt.t(), W, out=dA)
+
+        detail["ms_per_step"]["torch_matmul_dense"] = timed(torch_step, n2, warm)[0] / n2
+        detail["speedup_vs_dense"] = min(detail["ms_per_step"]["own_kernels_all_blocks"],
+                                         detail["ms_per_step"]["torch_matmul_dense"]) / (ms / steps)
+        ms_e = timed(lambda it: step(it + 100000, host=True), n2, warm)[0] / n2
+        e2e = {"value": float(np.mean(kept_blocks)) * flops_per_block / (ms_e * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": hA.numel() * 2 + hdY.numel() * 2, "d2h_bytes_per_step": hY.numel() * 2,
+               "ms_per_step": ms_e}
+    peaks = load_peaks()
+    cpu = None
+    if not args.no_cpu_baseline and not args.quick:
+        from oracle import cnn_blocks as OB
+        Mh = 2048
+        Ah, Wh, dYh = A[:Mh].float().cpu().numpy(), W.float().cpu().numpy().T, dYt[:, :Mh].float().cpu().numpy().T
+        keep = (np.add.outer(np.arange(Mh // ts), np.arange(Q)) % 2 == 0)
+        tc0 = time.perf_counter()
+        OB.fwd(Ah, Wh, keep, ts)
+        OB.bwd_input(dYh, Wh, keep, ts)
+        OB.bwd_weight(Ah, dYh, keep, ts)
+        dt = time.perf_counter() - tc0
+        try:
+            from threadpoolctl import threadpool_info
+            threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        except Exception:
+            threads = os.cpu_count() or 1
+        cpu = {"value": int(keep.sum()) * flops_per_block / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": "%d of %d rows of the input matrix, every second block kept (the oracle multiplies the masked full matrix)" % (Mh, M),
+               "seconds": dt}
+    line = {
+        "metric": "convolution layer (im2col product) fwd+bwd kept TFLOP/s, blocks dropped by predicted sensitivity",
+        "value": value, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms / steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, **{k: wl[k] for k in ("M", "K", "N", "ts", "k_frac", "t_frac", "threshold",
+                                                                       "cap", "m_prob", "n_prob")},
+                   "l2": "working set %.0f MB per step" % ((2 * M * K + 2 * M * N + 2 * N * K) * 2 / 1e6)},
+        "dense_equiv_tflops": 3 * 2.0 * M * K * N * steps / (ms * 1e-3) / 1e12, "clocks": clk, "e2e": e2e,
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "achieved": value, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": value / peaks["bf16_tflops"], "traffic": None,
+                     "note": "whole step incl. sensitivity counts, labels, block draws, lists and zero fill of the dropped blocks"},
+        "cpu_baseline": cpu, "detail": detail, "device_status": int(status),
+    }
+    print(json.dumps(line))
+    ard.ard_blocks_destroy(blocks)
+    ard.ard_destroy(ctx)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -749,6 +885,8 @@ def main():
         return run_mlp_step(args, wl)
     if wl["kind"] == "conv_rows":
         return run_conv_rows(args, wl)
+    if wl["kind"] == "conv_blocks":
+        return run_conv_blocks(args, wl)
 
     import torch
     import torch.distributed as dist
