@@ -445,9 +445,11 @@ ard_status ard_dropout_schedule(int n_epochs, double p_total, double mean_epoch,
  * A block is the dropout granularity.  Sec. 5.2.2 bounds the number of sensitive blocks per group so that
  * all groups keep nearly the same amount of work.  The paper fixes no constant, and the figure that shows the
  * balancing is not available; this library's reading: the prediction of Sec. 5.1 with one block as the
- * region (s = max(1, floor(k_frac*ts*ts + 1/2)) samples; sample d of block g*Q + j is word (d mod 4) of the
- * Philox4x32-10 block with key (seed) and counter (iteration low, iteration high, g*Q + j,
- * stream_id * 65536 + d div 4), at position floor(word * ts*ts / 2^32) of the block, row-major; a block passes
+ * region, its random k_frac of the values taken in runs of c = gcd(ts, 32) neighbouring values of a row (what
+ * one memory transaction delivers): of the block's Cn = ts*ts/c runs, n_c = max(1, floor(k_frac*Cn + 1/2))
+ * are drawn with replacement, s = n_c*c values are looked at; run d of block g*Q + j is chosen by word
+ * (d mod 4) of the Philox4x32-10 block with key (seed) and counter (iteration low, iteration high, g*Q + j,
+ * stream_id * 65536 + d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major; a block passes
  * iff at least max(1, ceil(t_frac * s)) sampled values are > threshold); of a group's passing blocks the
  * `cap` with the highest counts are sensitive (equal counts: lower j first); block g*Q + j is dropped iff
  * word 0 of the Philox block with counter (iteration low, iteration high, g*Q + j, stream_id * 65536 + 65535)

@@ -10,11 +10,13 @@ number, after which every group keeps nearly the same amount of work.
 
 Readings (the paper fixes none of this, and the figure that shows the balancing is not available;
 PARITY UNPINNED):
-  * prediction is that of Sec. 5.1 with one block as the region: s = max(1, floor(k * ts*ts + 1/2)) values of
-    the block, drawn with replacement; sample d is word (d mod 4) of the Philox4x32-10 block with key (seed)
-    and counter (iteration low, iteration high, g*Q + j, stream_id * 65536 + d div 4); its position inside
-    the block is floor(word * ts*ts / 2^32), row-major; the block passes iff at least
-    max(1, ceil(t * s)) sampled values exceed the threshold;
+  * prediction is that of Sec. 5.1 with one block as the region, and the random k% of its values are taken in
+    runs of c = gcd(ts, 32) neighbouring values of a row (a run is what one memory transaction delivers;
+    isolated values would cost a transaction each): a block has Cn = ts*ts/c runs, n_c = max(1, floor(k * Cn +
+    1/2)) of them are drawn with replacement, s = n_c * c values are looked at; run d is chosen by word
+    (d mod 4) of the Philox4x32-10 block with key (seed) and counter (iteration low, iteration high, g*Q + j,
+    stream_id * 65536 + d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major; the block
+    passes iff at least max(1, ceil(t * s)) of the values looked at exceed the threshold;
   * the bound: in every group at most `cap` blocks are labelled sensitive, namely the passing blocks with
     the highest counts (equal counts: the lower block index first);
   * a probability p becomes the integer P = min(floor(p * 2^32), 2^32 - 1); block (g, j) is dropped iff word 0
@@ -33,8 +35,18 @@ from .pattern import philox4x32_10, MASK32
 TWO32 = 1 << 32
 
 
+def run_length(ts):
+    return math.gcd(ts, 32)
+
+
+def n_runs(k_frac, ts):
+    """How many runs of a block are drawn."""
+    return max(1, int(math.floor(k_frac * (ts * ts // run_length(ts)) + 0.5)))
+
+
 def n_samples(k_frac, ts):
-    return max(1, int(math.floor(k_frac * ts * ts + 0.5)))
+    """How many values of a block are looked at."""
+    return n_runs(k_frac, ts) * run_length(ts)
 
 
 def needed(t_frac, s):
@@ -49,18 +61,23 @@ def block_count(A, g, j, ts, k_frac, threshold, seed, iteration, stream_id):
     """Sec. 5.1, step 2 for block j of group g: how many of the sampled values exceed the threshold."""
     A = np.asarray(A)
     Q = A.shape[1] // ts
-    s = n_samples(k_frac, ts)
-    assert (s + 3) // 4 <= 65535
+    c = run_length(ts)
+    Cn = ts * ts // c
+    per_row = ts // c
+    n_c = n_runs(k_frac, ts)
+    assert (n_c + 3) // 4 <= 65535
     count = 0
-    for q in range((s + 3) // 4):
+    for q in range((n_c + 3) // 4):
         words = philox4x32_10((iteration & MASK32, (iteration >> 32) & MASK32, g * Q + j,
                                ((stream_id << 16) | q) & MASK32), (seed & MASK32, (seed >> 32) & MASK32))
         for w in range(4):
-            if 4 * q + w >= s:
+            if 4 * q + w >= n_c:
                 break
-            pos = (words[w] * ts * ts) >> 32
-            if float(A[g * ts + pos // ts, j * ts + pos % ts]) > threshold:
-                count += 1
+            run = (words[w] * Cn) >> 32
+            row, col = g * ts + run // per_row, j * ts + (run % per_row) * c
+            for e in range(c):
+                if float(A[row, col + e]) > threshold:
+                    count += 1
     return count
 
 

@@ -44,11 +44,14 @@ template <typename T> __device__ __forceinline__ float val_f(T v);
 template <> __device__ __forceinline__ float val_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float val_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-// Sec. 5.1, step 2 with a block as the region.  One warp per block (g, j): lane l draws the Philox blocks
-// l, l + 32, ... (four samples each) and counts the sampled entries above the threshold.
+// Sec. 5.1, step 2 with a block as the region.  The sampled values are taken in runs of c = gcd(ts, 32)
+// neighbouring values of a row: a run is what one memory transaction delivers (64 bytes of bf16), where
+// isolated values cost a transaction each and made this kernel read more than the kept blocks themselves.
+// One warp per block (g, j); lane l takes the runs l, l + 32, ...: run d is chosen by word (d mod 4) of the
+// Philox block (d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major inside the block.
 template <typename T>
-__global__ void __launch_bounds__(256) block_count_kernel(const T* A, int lda, int ts, int Q, int nblocks, int samples,
-                                                          float threshold, unsigned long long seed,
+__global__ void __launch_bounds__(256) block_count_kernel(const T* A, int lda, int ts, int Q, int nblocks, int c,
+                                                          int n_runs, float threshold, unsigned long long seed,
                                                           unsigned long long iteration, uint32_t stream_id,
                                                           int32_t* counts) {
   pdl_launch_dependents();
@@ -58,23 +61,30 @@ __global__ void __launch_bounds__(256) block_count_kernel(const T* A, int lda, i
   if (blk >= nblocks) return;
   const int g = blk / Q, j = blk - g * Q;
   const T* base = A + (size_t)g * ts * lda + (size_t)j * ts;
-  const unsigned long long size = (unsigned long long)ts * (unsigned long long)ts;
-  const int pblocks = (samples + 3) >> 2;
+  const unsigned int per_row = (unsigned int)(ts / c);
+  const unsigned long long Cn = (unsigned long long)ts * per_row;
+  // 16-byte pieces when every run starts on a 16-byte boundary
+  constexpr int VEC = 16 / (int)sizeof(T);
+  const bool wide = (c % VEC) == 0 && ((size_t)lda * sizeof(T)) % 16 == 0 && (reinterpret_cast<uintptr_t>(A) & 15) == 0 &&
+                    ((size_t)ts * sizeof(T)) % 16 == 0;
   int count = 0;
-#pragma unroll 2
-  for (int q = lane; q < pblocks; q += 32) {
-    uint32_t c[4] = {(uint32_t)iteration, (uint32_t)(iteration >> 32), (uint32_t)blk, (stream_id << 16) | (uint32_t)q};
-    philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
-    float v[4];
+  for (int d = lane; d < n_runs; d += 32) {
+    uint32_t w[4] = {(uint32_t)iteration, (uint32_t)(iteration >> 32), (uint32_t)blk, (stream_id << 16) | (uint32_t)(d >> 2)};
+    philox4x32_10(w, (uint32_t)seed, (uint32_t)(seed >> 32));
+    const uint32_t word = (d & 3) == 0 ? w[0] : ((d & 3) == 1 ? w[1] : ((d & 3) == 2 ? w[2] : w[3]));
+    const unsigned int run = (unsigned int)(((unsigned long long)word * Cn) >> 32);  // < Cn
+    const unsigned int roff = run / per_row;
+    const T* p = base + (size_t)roff * lda + (size_t)(run - roff * per_row) * c;
+    if (wide) {
+      for (int e = 0; e < c; e += VEC) {
+        const uint4 v = *reinterpret_cast<const uint4*>(p + e);
+        const T* t = reinterpret_cast<const T*>(&v);
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const unsigned int pos = (unsigned int)(((unsigned long long)c[w] * size) >> 32);  // < ts*ts
-      const unsigned int roff = pos / (unsigned int)ts;
-      const unsigned int col = pos - roff * (unsigned int)ts;
-      v[w] = 4 * q + w < samples ? val_f<T>(base[(size_t)roff * lda + col]) : -INFINITY;
+        for (int u = 0; u < VEC; ++u) count += val_f<T>(t[u]) > threshold ? 1 : 0;
+      }
+    } else {
+      for (int e = 0; e < c; ++e) count += val_f<T>(p[e]) > threshold ? 1 : 0;
     }
-#pragma unroll
-    for (int w = 0; w < 4; ++w) count += v[w] > threshold ? 1 : 0;
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) count += __shfl_xor_sync(0xffffffffu, count, o);
@@ -322,21 +332,26 @@ ard_status ard_blocks_predict(ard_ctx* ctx, ard_blocks* b, ard_dtype dtype, cons
   if (lda < b->Kc) return ARD_ERR_SHAPE;
   if (!(k_frac > 0.0) || k_frac > 1.0 || !(t_frac >= 0.0) || t_frac > 1.0 || cap < 0 || stream_id >= 65536u)
     return ARD_ERR_INVALID_ARG;
-  const double sd = floor(k_frac * (double)b->ts * (double)b->ts + 0.5);
-  const int samples = sd < 1.0 ? 1 : (int)sd;
-  if ((samples + 3) / 4 > 65535) return ARD_ERR_UNSUPPORTED;
-  const double nd = ceil(t_frac * samples - 1e-9);
+  int c = b->ts, r32 = 32;
+  while (r32) { const int t = c % r32; c = r32; r32 = t; }  // c = gcd(ts, 32): values per run
+  const long long Cn = (long long)b->ts * (b->ts / c);
+  const double rd = floor(k_frac * (double)Cn + 0.5);
+  const long long n_runs_ll = rd < 1.0 ? 1 : (long long)rd;
+  if ((n_runs_ll + 3) / 4 > 65535) return ARD_ERR_UNSUPPORTED;
+  const int n_runs = (int)n_runs_ll;
+  const long long samples = n_runs_ll * c;
+  const double nd = ceil(t_frac * (double)samples - 1e-9);
   const int need = nd < 1.0 ? 1 : (int)nd;
   DevGuard guard(ctx->device);
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int nblocks = b->G * b->Q;
   if (dtype == ARD_F32)
     ARD_CUDA_OK(ard_launch(ctx, block_count_kernel<float>, dim3((nblocks + 7) / 8), dim3(256), 0, s, (const float*)A, lda,
-                           b->ts, b->Q, nblocks, samples, threshold, (unsigned long long)seed,
+                           b->ts, b->Q, nblocks, c, n_runs, threshold, (unsigned long long)seed,
                            (unsigned long long)iteration, stream_id, b->d_count));
   else
     ARD_CUDA_OK(ard_launch(ctx, block_count_kernel<__nv_bfloat16>, dim3((nblocks + 7) / 8), dim3(256), 0, s,
-                           (const __nv_bfloat16*)A, lda, b->ts, b->Q, nblocks, samples, threshold,
+                           (const __nv_bfloat16*)A, lda, b->ts, b->Q, nblocks, c, n_runs, threshold,
                            (unsigned long long)seed, (unsigned long long)iteration, stream_id, b->d_count));
   ARD_CUDA_OK(ard_launch(ctx, block_label_kernel, dim3((nblocks + 255) / 256), dim3(256), 0, s,
                          (const int32_t*)b->d_count, b->Q, nblocks, need, cap, b->d_sens));

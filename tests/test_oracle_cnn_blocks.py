@@ -1,15 +1,14 @@
 """Pins for oracle/cnn_blocks.py (block-based sensitivity-aware dropout, Sec. 5.1 / 5.2.2).
 
 The paper fixes no numbers for this part; the pins are what the mathematics fixes: decisions that do not depend
-on the sample, agreement with the row variant's region decision where a block IS a region (one block per
-group), the binomial law of a block's count, the bound on sensitive blocks per group and which blocks it
+on the sample, that the sampled runs are whole, lie inside their block and are drawn uniformly, the binomial law of a
+block's count over runs, the bound on sensitive blocks per group and which blocks it
 picks, the drop rates of the two labels, brute-force loops over kept blocks, the all-kept case against a
 plain matrix product, and the adjoint identities.
 """
 import numpy as np
 from scipy import stats
 
-from oracle import cnn as R
 from oracle import cnn_blocks as C
 
 
@@ -19,33 +18,52 @@ def test_counts_that_do_not_depend_on_the_sample():
     A[0:4, 4:8] = 1.0                  # block (0, 1): every value above the threshold
     for it in range(4):
         counts, sens = C.predict(A, ts, 0.5, 0.5, 0.5, 3, 7, it, 2)
-        assert counts[0, 1] == C.n_samples(0.5, ts) == 8
+        assert counts[0, 1] == C.n_samples(0.5, ts) == 8      # two runs of four values
         assert counts.sum() == 8
         assert sens[0, 1] and sens.sum() == 1
 
 
-def test_one_block_per_group_is_the_row_variants_region():
-    # Kc = ts: a block covers x = ts whole rows, which is a region of the row variant with the same id
-    rng = np.random.default_rng(1)
+def test_runs_are_whole_and_inside_the_block():
+    # values encode their own position: a count over a block whose ONLY large values sit in one run of another
+    # block, or straddle a run boundary, must never see part of a run
+    ts = 8                                   # run length gcd(8, 32) = 8: a run is a whole row of the block
+    assert C.run_length(ts) == 8 and C.run_length(64) == 32 and C.run_length(48) == 16 and C.run_length(7) == 1
+    A = np.zeros((ts, 2 * ts))
+    A[:, :ts] = 1.0                          # block 0 all above, block 1 all below
+    for it in range(20):
+        assert C.block_count(A, 0, 0, ts, 0.5, 0.5, 1, it, 0) == C.n_samples(0.5, ts) == 32
+        assert C.block_count(A, 0, 1, ts, 0.5, 0.5, 1, it, 0) == 0
+    B = np.zeros((ts, ts))
+    B[3, :] = 1.0                            # exactly one run above: every draw contributes 0 or 8
+    counts = {C.block_count(B, 0, 0, ts, 0.5, 0.5, 2, it, 0) for it in range(200)}
+    assert all(c % 8 == 0 for c in counts) and len(counts) > 1
+
+
+def test_runs_are_drawn_uniformly():
+    # one run of the block above the threshold: it is hit with probability 1/Cn per draw
     ts = 8
-    A = rng.random((4 * ts, ts))
-    for g in range(4):
-        c = C.block_count(A, g, 0, ts, 0.4, 0.5, 99, 5, 3)
-        _, c_row, s_row = R.region_sensitive(A, g, ts, 0.4, 0.5, 0.5, 99, 5, 3)
-        assert s_row == C.n_samples(0.4, ts)
-        assert c == c_row
+    B = np.zeros((ts, ts))
+    n_c = C.n_runs(1.0, ts)                  # 8 draws per count
+    hits = np.zeros(ts)
+    for r in range(ts):
+        B[:] = 0.0
+        B[r, :] = 1.0
+        hits[r] = sum(C.block_count(B, 0, 0, ts, 1.0, 0.5, 5, it, 1) for it in range(300)) / 8
+    expect = 300 * n_c / ts
+    assert np.all(np.abs(hits - expect) < 4.5 * np.sqrt(expect))
 
 
-def test_count_follows_the_binomial_law():
+def test_count_follows_the_binomial_law_over_runs():
     rng = np.random.default_rng(0)
     ts = 8
     A = np.zeros((ts, 2 * ts))
-    A[:, ts:] = (rng.random((ts, ts)) < 0.4)
-    frac = A[:, ts:].mean()
-    s = C.n_samples(0.5, ts)
-    c = np.array([C.block_count(A, 0, 1, ts, 0.5, 0.5, 3, it, 0) for it in range(800)])
-    assert abs(c.mean() - s * frac) < 4 * np.sqrt(s * frac * (1 - frac) / 800)
-    assert abs(c.var() - s * frac * (1 - frac)) < 0.25 * s * frac * (1 - frac)
+    above = rng.random(ts) < 0.4             # whole runs (rows of block 1) above the threshold
+    A[above, ts:] = 1.0
+    frac = above.mean()
+    n_c = C.n_runs(0.5, ts)
+    c = np.array([C.block_count(A, 0, 1, ts, 0.5, 0.5, 3, it, 0) for it in range(800)]) / 8
+    assert abs(c.mean() - n_c * frac) < 4 * np.sqrt(n_c * frac * (1 - frac) / 800)
+    assert abs(c.var() - n_c * frac * (1 - frac)) < 0.25 * n_c * frac * (1 - frac)
 
 
 def test_bound_on_sensitive_blocks_picks_the_highest_counts():
