@@ -171,40 +171,65 @@ __device__ void block_exclusive_scan(int32_t* ptr, int n, int* s_warp /* [33] */
 // The kept blocks as the lists of a tile pattern with Tr = Q tile-rows (blocks along Kc) and Tc = G
 // tile-columns (groups): idx = r*G + c ascending; grouped by tile-column (col_ptr, col_idx = r ascending)
 // and by tile-row (row_ptr, row_idx = c ascending).  One CTA: the lists are a few thousand entries.
-__global__ void __launch_bounds__(LIST_THREADS) block_lists_kernel(const uint8_t* keep, int G, int Q, int ts, int kind,
+// draw != 0: the CTA first draws the kept flags itself (small block counts: saves a launch).
+// in_smem != 0: the flags and the two pointer arrays live in shared memory while the lists are built (every
+// phase otherwise waits for a round trip to global memory); the pointer arrays are copied out at the end.
+__global__ void __launch_bounds__(LIST_THREADS) block_lists_kernel(uint8_t* keep, const uint8_t* sens, int draw, int in_smem,
+                                                                   uint32_t P_sens, uint32_t P_insens,
+                                                                   unsigned long long seed, unsigned long long iteration,
+                                                                   uint32_t stream_id, int G, int Q, int ts, int kind,
                                                                    int32_t* hdr, int32_t* idx, int32_t* col_ptr,
                                                                    int32_t* col_idx, int32_t* row_ptr, int32_t* row_idx) {
   __shared__ int s_warp[33];
+  extern __shared__ int32_t s_dyn[];
   pdl_launch_dependents();
   pdl_wait_prior_grids();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = LIST_THREADS / 32;
+  const int nblocks = G * Q;
+  int32_t* cp = in_smem ? s_dyn : col_ptr;
+  int32_t* rp = in_smem ? s_dyn + (G + 1) : row_ptr;
+  uint8_t* s_keep = reinterpret_cast<uint8_t*>(s_dyn + (G + 1) + (Q + 1));
+  const uint8_t* kp = in_smem ? s_keep : keep;
+  if (draw) {
+    for (int blk = tid; blk < nblocks; blk += LIST_THREADS) {
+      uint32_t c[4] = {(uint32_t)iteration, (uint32_t)(iteration >> 32), (uint32_t)blk, (stream_id << 16) | 0xFFFFu};
+      philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+      const uint8_t k = (c[0] < (sens[blk] ? P_sens : P_insens)) ? 0 : 1;
+      keep[blk] = k;
+      if (in_smem) s_keep[blk] = k;
+    }
+    __syncthreads();
+  } else if (in_smem) {
+    for (int blk = tid; blk < nblocks; blk += LIST_THREADS) s_keep[blk] = keep[blk];
+    __syncthreads();
+  }
   // counts per group (a warp per group, lanes across its blocks) and per tile-row (lanes across the groups)
   for (int g = warp; g < G; g += nwarps) {
     int cnt = 0;
-    for (int j0 = 0; j0 < Q; j0 += 32) cnt += __popc(__ballot_sync(0xffffffffu, j0 + lane < Q && keep[g * Q + j0 + lane]));
-    if (lane == 0) col_ptr[g] = cnt;
+    for (int j0 = 0; j0 < Q; j0 += 32) cnt += __popc(__ballot_sync(0xffffffffu, j0 + lane < Q && kp[g * Q + j0 + lane]));
+    if (lane == 0) cp[g] = cnt;
   }
   for (int j = warp; j < Q; j += nwarps) {
     int cnt = 0;
-    for (int g0 = 0; g0 < G; g0 += 32) cnt += __popc(__ballot_sync(0xffffffffu, g0 + lane < G && keep[(g0 + lane) * Q + j]));
-    if (lane == 0) row_ptr[j] = cnt;
+    for (int g0 = 0; g0 < G; g0 += 32) cnt += __popc(__ballot_sync(0xffffffffu, g0 + lane < G && kp[(g0 + lane) * Q + j]));
+    if (lane == 0) rp[j] = cnt;
   }
   __syncthreads();
-  block_exclusive_scan(col_ptr, G, s_warp);
-  block_exclusive_scan(row_ptr, Q, s_warp);
+  block_exclusive_scan(cp, G, s_warp);
+  block_exclusive_scan(rp, Q, s_warp);
   for (int g = warp; g < G; g += nwarps) {
-    int o = col_ptr[g];
+    int o = cp[g];
     for (int j0 = 0; j0 < Q; j0 += 32) {
-      const bool k = j0 + lane < Q && keep[g * Q + j0 + lane];
+      const bool k = j0 + lane < Q && kp[g * Q + j0 + lane];
       const unsigned m = __ballot_sync(0xffffffffu, k);
       if (k) col_idx[o + __popc(m & ((1u << lane) - 1u))] = j0 + lane;
       o += __popc(m);
     }
   }
   for (int j = warp; j < Q; j += nwarps) {
-    int o = row_ptr[j];
+    int o = rp[j];
     for (int g0 = 0; g0 < G; g0 += 32) {
-      const bool k = g0 + lane < G && keep[(g0 + lane) * Q + j];
+      const bool k = g0 + lane < G && kp[(g0 + lane) * Q + j];
       const unsigned m = __ballot_sync(0xffffffffu, k);
       if (k) {
         const int at = o + __popc(m & ((1u << lane) - 1u));
@@ -214,11 +239,15 @@ __global__ void __launch_bounds__(LIST_THREADS) block_lists_kernel(const uint8_t
       o += __popc(m);
     }
   }
+  if (in_smem) {
+    for (int g = tid; g <= G; g += LIST_THREADS) col_ptr[g] = cp[g];
+    for (int j = tid; j <= Q; j += LIST_THREADS) row_ptr[j] = rp[j];
+  }
   if (tid == 0) {
     hdr[HDR_KIND] = kind;
     hdr[HDR_DP] = 1;   // no period: the list kernels never use it
     hdr[HDR_B] = 1;
-    hdr[HDR_NKEEP] = row_ptr[Q];
+    hdr[HDR_NKEEP] = rp[Q];
     hdr[HDR_UNITS] = G * Q;
     hdr[HDR_TR] = Q;
     hdr[HDR_TC] = G;
@@ -380,14 +409,23 @@ ard_status ard_blocks_sample(ard_ctx* ctx, ard_blocks* b, double m_prob, double 
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int nblocks = b->G * b->Q;
   ard_pattern* p = b->pat;
-  ARD_CUDA_OK(ard_launch(ctx, block_draw_kernel, dim3((nblocks + 255) / 256), dim3(256), 0, s, (const uint8_t*)b->d_sens,
-                         nblocks, quantise_probability(m_prob), quantise_probability(n_prob), (unsigned long long)seed,
-                         (unsigned long long)iteration, stream_id, b->d_keep));
-  ARD_CUDA_OK(ard_launch(ctx, block_lists_kernel, dim3(1), dim3(LIST_THREADS), 0, s, (const uint8_t*)b->d_keep, b->G, b->Q,
-                         b->ts, (int)ARD_TILE, p->d_hdr, p->d_idx, p->d_col_ptr, p->d_col_idx, p->d_row_ptr, p->d_row_idx));
+  const uint32_t Pm = quantise_probability(m_prob), Pn = quantise_probability(n_prob);
+  // few blocks: the list kernel's CTA draws them itself; the flags and pointer arrays in shared memory if they fit
+  const int fused = nblocks <= 65536 ? 1 : 0;
+  const size_t smem = ((size_t)(b->G + 1) + (size_t)(b->Q + 1)) * sizeof(int32_t) + (size_t)nblocks;
+  const int in_smem = smem <= 40960 ? 1 : 0;
+  if (!fused) {
+    ARD_CUDA_OK(ard_launch(ctx, block_draw_kernel, dim3((nblocks + 255) / 256), dim3(256), 0, s, (const uint8_t*)b->d_sens,
+                           nblocks, Pm, Pn, (unsigned long long)seed, (unsigned long long)iteration, stream_id, b->d_keep));
+    ctx->launches++;
+  }
+  ARD_CUDA_OK(ard_launch(ctx, block_lists_kernel, dim3(1), dim3(LIST_THREADS), in_smem ? smem : 0, s, b->d_keep,
+                         (const uint8_t*)b->d_sens, fused, in_smem, Pm, Pn, (unsigned long long)seed,
+                         (unsigned long long)iteration, stream_id, b->G, b->Q, b->ts, (int)ARD_TILE, p->d_hdr, p->d_idx,
+                         p->d_col_ptr, p->d_col_idx, p->d_row_ptr, p->d_row_idx));
+  ctx->launches++;
   p->dp_bound = IRREGULAR_DP_BOUND;
   p->generation++;
-  ctx->launches += 2;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;
 }

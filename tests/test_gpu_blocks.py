@@ -132,6 +132,33 @@ def test_products_over_the_kept_blocks_match_the_oracle(M, Kc, N, ts):
         ctx.close()
 
 
+@pytest.mark.parametrize("G,Q", [(200, 256), (280, 256), (3, 1), (1, 40)])
+def test_draws_and_lists_on_other_grid_sizes(G, Q):
+    """Block counts beyond what the list kernel keeps in shared memory (51200) and beyond what it draws itself
+    (71680), and degenerate grids: the same flags and lists as the oracle."""
+    ts = 8
+    ctx = Ctx(4096)
+    blocks = ard.ard_blocks_create(ctx.h, G * ts, Q * ts, ts)
+    try:
+        pat = ard.ard_blocks_pattern(blocks)
+        ard.ard_blocks_set_label(ctx.h, blocks, 0)
+        for it, p in enumerate([0.5, 0.97]):
+            ard.ard_blocks_sample(ctx.h, blocks, 0.0, p, 21, it, 9)
+            _, _, keep = ard.ard_blocks_to_host(blocks, G * Q)
+            ko = OB.draw_blocks(np.zeros((G, Q), bool), 0.0, p, 21, it, 9)
+            assert np.array_equal(keep.reshape(G, Q).astype(bool), ko)
+            idx, col_ptr, col_idx, row_ptr, row_idx = OB.block_lists(ko)
+            _, _, n_keep, didx = ard.ard_pattern_to_host(pat, G * Q)
+            assert n_keep == len(idx) and np.array_equal(didx, idx)
+            cp, ci, rp, ri = ard.ard_pattern_tile_lists_to_host(pat, Q, G)
+            assert np.array_equal(cp, col_ptr) and np.array_equal(ci, col_idx)
+            assert np.array_equal(rp, row_ptr) and np.array_equal(ri, row_idx)
+    finally:
+        torch.cuda.synchronize()
+        ard.ard_blocks_destroy(blocks)
+        ctx.close()
+
+
 def test_argument_checks():
     ctx = Ctx(4096)
     try:
