@@ -350,10 +350,12 @@ ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, int n_layers,
  * and gives it a low (sensitive) or a high dropout probability; Sec. 5.2.1 draws, per iteration, which rows
  * of A are dropped, multiplies only the kept rows and fills the results back into the same rows of Y.
  * The paper fixes neither the region shape nor which values are sampled nor any constant; this library's
- * reading: regions of `region_rows` consecutive rows by the whole width; sample d of region g is word
- * (d mod 4) of the Philox4x32-10 block with key (seed) and counter (iteration low, iteration high, g,
- * stream_id * 65536 + d div 4), at position floor(word * region_rows*Kc / 2^32) of the region (row-major;
- * positions below the last row of A count as not exceeding); s = max(1, floor(k_frac*region_rows*Kc + 1/2))
+ * reading: regions of `region_rows` consecutive rows by the whole width; the random k_frac of a region's values
+ * is taken in runs of c = gcd(Kc, 32) neighbouring values of a row (what one memory transaction delivers): of the
+ * region's Cn = region_rows*Kc/c runs, n_c = max(1, floor(k_frac*Cn + 1/2)) are drawn with replacement; run d of
+ * region g is chosen by word (d mod 4) of the Philox4x32-10 block with key (seed) and counter (iteration low,
+ * iteration high, g, stream_id * 65536 + d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major
+ * (runs below the last row of A count as not exceeding); s = n_c*c
  * samples; sensitive iff at least max(1, ceil(t_frac * s)) sampled values are > threshold; a probability p
  * is the integer min(floor(p 2^32), 2^32 - 1); row r is dropped iff word 0 of the block with counter
  * (iteration low, iteration high, r, stream_id * 65536 + 65535) is below its region's integer.

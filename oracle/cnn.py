@@ -11,11 +11,14 @@ probabilities, multiplies only the kept rows and writes the results to the same 
 
 Readings (the paper fixes none of this; PARITY UNPINNED):
   * regions: x consecutive rows by the whole width of A (the row is the granularity of Sec. 5.2.1);
-  * the sampled values are drawn with replacement: sample d of region g is word (d mod 4) of the Philox4x32-10
-    block with key (seed) and counter (iteration low, iteration high, g, stream_id * 65536 + d div 4); its
-    position inside the region is floor(word * x*Kc / 2^32), row-major; positions below the last row of A
-    (ragged last region) count as not exceeding;
-  * s = max(1, floor(k * x * Kc + 1/2)) samples; sensitive iff the count is >= max(1, ceil(t * s));
+  * the random k% of a region's values are taken in runs of c = gcd(Kc, 32) neighbouring values of a row (a run
+    is what one memory transaction delivers; isolated values would cost a transaction each): the region has
+    Cn = x*Kc/c runs, n_c = max(1, floor(k * Cn + 1/2)) of them are drawn with replacement, s = n_c * c values
+    are looked at; run d of region g is chosen by word (d mod 4) of the Philox4x32-10 block with key (seed) and
+    counter (iteration low, iteration high, g, stream_id * 65536 + d div 4) as run number
+    floor(word * Cn / 2^32), runs numbered row-major; runs below the last row of A (ragged last region) count
+    as not exceeding;
+  * sensitive iff the count of values above the threshold is >= max(1, ceil(t * s));
   * a probability p becomes the integer P = min(floor(p * 2^32), 2^32 - 1); row r is dropped iff word 0 of the
     block with counter (iteration low, iteration high, r, stream_id * 65536 + 65535) is < P of its region;
   * no rescale is mentioned: alpha is an explicit argument, as for the other patterns;
@@ -33,8 +36,18 @@ TWO32 = 1 << 32
 MAX_BLOCKS = 65535
 
 
+def run_length(Kc):
+    return math.gcd(Kc, 32)
+
+
+def n_runs(k_frac, x, Kc):
+    """How many runs of a region are drawn."""
+    return max(1, int(math.floor(k_frac * (x * (Kc // run_length(Kc))) + 0.5)))
+
+
 def n_samples(k_frac, x, Kc):
-    return max(1, int(math.floor(k_frac * x * Kc + 0.5)))
+    """How many values of a region are looked at."""
+    return n_runs(k_frac, x, Kc) * run_length(Kc)
 
 
 def needed(t_frac, s):
@@ -50,19 +63,22 @@ def region_sensitive(A, g, x, k_frac, t_frac, threshold, seed, iteration, stream
     A = np.asarray(A)
     M, Kc = A.shape
     s = n_samples(k_frac, x, Kc)
-    assert (s + 3) // 4 <= MAX_BLOCKS
-    size = x * Kc
+    c = run_length(Kc)
+    per_row = Kc // c
+    Cn = x * per_row
+    n_c = n_runs(k_frac, x, Kc)
+    assert (n_c + 3) // 4 <= MAX_BLOCKS
     count = 0
-    for q in range((s + 3) // 4):
+    for q in range((n_c + 3) // 4):
         words = philox4x32_10((iteration & MASK32, (iteration >> 32) & MASK32, g, ((stream_id << 16) | q) & MASK32),
                               (seed & MASK32, (seed >> 32) & MASK32))
         for w in range(4):
-            if 4 * q + w >= s:
+            if 4 * q + w >= n_c:
                 break
-            pos = (words[w] * size) >> 32
-            row, col = g * x + pos // Kc, pos % Kc
-            if row < M and float(A[row, col]) > threshold:
-                count += 1
+            run = (words[w] * Cn) >> 32
+            row, col = g * x + run // per_row, (run % per_row) * c
+            if row < M:
+                count += int(np.count_nonzero(np.asarray(A[row, col:col + c], dtype=np.float64) > threshold))
     return count >= needed(t_frac, s), count, s
 
 

@@ -208,8 +208,8 @@ ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* i
                               cudaStream_t s);
 
 // Sensitivity-aware row dropout (rows.cu).
-ard_status launch_sensitivity(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc, int samples,
-                              int need, float threshold, uint32_t P_sens, uint32_t P_insens, uint64_t seed,
+ard_status launch_sensitivity(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc, int c,
+                              int n_runs, int need, float threshold, uint32_t P_sens, uint32_t P_insens, uint64_t seed,
                               uint64_t iteration, uint32_t stream_id, cudaStream_t s);
 ard_status launch_fill_probability(ard_ctx* ctx, ard_rows* rows, uint32_t P, cudaStream_t s);
 ard_status launch_rows_sample(ard_ctx* ctx, ard_rows* rows, uint64_t seed, uint64_t iteration, uint32_t stream_id,

@@ -36,17 +36,41 @@ def test_ragged_last_region_counts_missing_rows_as_below():
     assert abs(np.mean(fr) - 0.25) < 0.02          # a quarter of the positions exist
 
 
-def test_decision_follows_the_binomial_law():
+def test_decision_follows_the_binomial_law_over_runs():
+    # whole runs (32 neighbouring values of a row) above or below the threshold: the count is 32 times a binomial
+    # variable over the drawn runs
     rng = np.random.default_rng(0)
-    x, Kc, f = 2, 64, 0.45
-    A = (rng.random((x, Kc)) < f).astype(np.float64)
-    frac = A.mean()
-    s = C.n_samples(0.25, x, Kc)
-    need = C.needed(0.5, s)
-    hits = sum(C.region_sensitive(A, 0, x, 0.25, 0.5, 0.5, 11, it, 0)[0] for it in range(1500))
-    p_theory = stats.binom.sf(need - 1, s, frac)
+    x, Kc = 8, 64
+    assert C.run_length(Kc) == 32 and C.run_length(200) == 8 and C.run_length(33) == 1
+    above = np.zeros(16, dtype=bool)
+    above[rng.choice(16, 6, replace=False)] = True
+    A = np.repeat(above.reshape(x, 2), 32, axis=1).astype(np.float64)
+    n_c = C.n_runs(0.5, x, Kc)
+    s = C.n_samples(0.5, x, Kc)
+    assert n_c == 8 and s == 256
+    need_runs = -(-C.needed(0.5, s) // 32)
+    res = [C.region_sensitive(A, 0, x, 0.5, 0.5, 0.5, 11, it, 0) for it in range(1500)]
+    assert all(c % 32 == 0 and n == s for _, c, n in res)
+    hits = sum(r[0] for r in res)
+    p_theory = stats.binom.sf(need_runs - 1, n_c, 6 / 16)
     sd = np.sqrt(p_theory * (1 - p_theory) / 1500)
     assert abs(hits / 1500 - p_theory) < 4 * sd + 1e-3
+    mean_runs = np.mean([c for _, c, _ in res]) / 32
+    assert abs(mean_runs - n_c * 6 / 16) < 4 * np.sqrt(n_c * (6 / 16) * (10 / 16) / 1500)
+
+
+def test_runs_are_drawn_uniformly_and_stay_in_their_region():
+    x, Kc = 2, 16                                  # runs of 16: a run is a whole row; region 1 = rows 2, 3
+    n_c = C.n_runs(1.0, x, Kc)
+    assert n_c == 2
+    hits = np.zeros(6)
+    for r in range(6):
+        A = np.zeros((6, Kc))
+        A[r] = 1.0
+        hits[r] = sum(C.region_sensitive(A, 1, x, 1.0, 0.5, 0.5, 5, it, 1)[1] for it in range(400)) / 16
+    assert hits[0] == hits[1] == hits[4] == hits[5] == 0          # other regions' rows are never looked at
+    expect = 400 * n_c / 2
+    assert np.all(np.abs(hits[2:4] - expect) < 4.5 * np.sqrt(expect / 2))
 
 
 def test_row_sampler_rates_and_extremes():
