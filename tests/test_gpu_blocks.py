@@ -159,6 +159,76 @@ def test_draws_and_lists_on_other_grid_sizes(G, Q):
         ctx.close()
 
 
+def test_benchmark_layer_on_sampled_outputs():
+    """The convolution layer the benchmark times (3 x 3, 256 -> 512 channels, 32768 output positions, 128 x 128
+    blocks, at most 6 sensitive blocks per group), in its launch configuration (ard_blocks_products).  The oracle
+    recomputes counts and labels of sampled groups, every draw and the whole lists, the output rows and the
+    input-gradient rows of sampled groups and sampled channels of the weight gradient; finiteness and the zero
+    blocks are checked over the whole outputs."""
+    M, K, N, ts, cap = 32768, 2304, 512, 128, 6
+    kf, tf, thr, mp, npb = 0.05, 0.3, 0.5, 0.2, 0.8
+    G, Q = M // ts, K // ts
+    rng = np.random.default_rng(2026)
+    A = _input_matrix(rng, M, K, ts)
+    W = inputs.bf16_round((rng.standard_normal((K, N)) / np.sqrt(K)).astype(np.float32))      # math orientation
+    dY = inputs.bf16_round(rng.standard_normal((M, N)).astype(np.float32))
+    ctx = Ctx(4096)
+    blocks = ard.ard_blocks_create(ctx.h, M, K, ts)
+    try:
+        Ad = torch.from_numpy(A).to(BF).cuda()
+        Wd = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+        dYt = torch.from_numpy(np.ascontiguousarray(dY.T)).to(BF).cuda()
+        ard.ard_blocks_predict(ctx.h, blocks, ard.ARD_BF16, Ad, K, kf, tf, thr, cap, 5, 3, 1)
+        ard.ard_blocks_sample(ctx.h, blocks, mp, npb, 5, 3, 1)
+        counts, sens, keep = ard.ard_blocks_to_host(blocks, G * Q)
+        counts, sens, keep = counts.reshape(G, Q), sens.reshape(G, Q).astype(bool), keep.reshape(G, Q).astype(bool)
+        need = OB.needed(tf, OB.n_samples(kf, ts))
+        groups = list(range(3, G, G // 24))
+        for g in groups:
+            co = [OB.block_count(A, g, j, ts, kf, thr, 5, 3, 1) for j in range(Q)]
+            assert counts[g].tolist() == co, g
+            assert np.array_equal(sens[g], OB.label_group(co, need, cap)), g
+        assert (sens.sum(1) <= cap).all() and 0 < sens.sum() < G * Q
+        # every draw and the whole lists, from the device's labels
+        ko = OB.draw_blocks(sens, mp, npb, 5, 3, 1)
+        assert np.array_equal(keep, ko)
+        idx, col_ptr, col_idx, row_ptr, row_idx = OB.block_lists(ko)
+        pat = ard.ard_blocks_pattern(blocks)
+        _, _, n_keep, didx = ard.ard_pattern_to_host(pat, G * Q)
+        assert n_keep == len(idx) and np.array_equal(didx, idx)
+        cp, ci, rp, ri = ard.ard_pattern_tile_lists_to_host(pat, Q, G)
+        assert np.array_equal(cp, col_ptr) and np.array_equal(ci, col_idx)
+        assert np.array_equal(rp, row_ptr) and np.array_equal(ri, row_idx)
+        # products: dropped blocks of A hold NaN, outputs start as NaN
+        mask_t = torch.from_numpy(ko).cuda().repeat_interleave(ts, 0).repeat_interleave(ts, 1)
+        Ad[~mask_t] = float("nan")
+        Yt = torch.full((N, M), float("nan"), dtype=BF, device="cuda")
+        dW = torch.full((N, K), float("nan"), dtype=BF, device="cuda")
+        dA = torch.full((M, K), float("nan"), dtype=BF, device="cuda")
+        ard.ard_blocks_products(ctx.h, blocks, ard.ARD_BF16, N, 1.25, Ad, K, Wd, K, dYt, M, Yt, M, dW, K, dA, K, 1)
+        torch.cuda.synchronize()
+        assert ard.ard_last_device_status(ctx.h) == 0
+        assert bool(torch.isfinite(Yt).all()) and bool(torch.isfinite(dW).all()) and bool(torch.isfinite(dA).all())
+        assert bool(torch.all(dA[~mask_t] == 0))
+        tol = TOL[ard.ARD_BF16]
+        for g in groups[::3]:
+            rs = slice(g * ts, (g + 1) * ts)
+            kg = ko[g:g + 1]
+            assert OG.rel_fro(host(Yt[:, rs]).T, OB.fwd(A[rs], W, kg, ts, 1.25)) <= tol, g
+            assert OG.rel_fro(host(dA[rs]), OB.bwd_input(dY[rs], W, kg, ts, 1.25)) <= tol, g
+        # sampled channels of dW: the contraction runs over every group
+        cols = np.arange(3, N, N // 32)[:32]
+        want = np.zeros((K, len(cols)))
+        for g in range(G):
+            rs = slice(g * ts, (g + 1) * ts)
+            want += OB.bwd_weight(A[rs], dY[rs][:, cols], ko[g:g + 1], ts, 1.25)
+        assert OG.rel_fro(host(dW[torch.from_numpy(cols).long().cuda()]).T, want) <= tol
+    finally:
+        torch.cuda.synchronize()
+        ard.ard_blocks_destroy(blocks)
+        ctx.close()
+
+
 def test_argument_checks():
     ctx = Ctx(4096)
     try:
