@@ -1519,12 +1519,17 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
     return pairs ? launch_mode<256, M_TILEC_BWD_WEIGHT, 2>(ctx, p, many, s)
                  : launch_mode<256, M_TILEC_BWD_WEIGHT, 1>(ctx, p, many, s);
   } else {
+    // List form with at least two 128-row tiles of output and 128-wide pattern tiles: CTA pairs (256 x 128
+    // tiles; each CTA stages half of the kept block, the instruction is the wide one).
+    const bool pairs = ctx->use_pairs && p.B > BM && bn == 128;
     if (op == OP_FWD) {
       const int mt = cdiv(p.B, BM);
+      if (pairs) return launch_mode<128, M_TILE_FWD, 2>(ctx, p, cdiv(p.B, 2 * BM) * cdiv(p.N, 128), s);
       ARD_TC_CASE(128, M_TILE_FWD, mt * cdiv(p.N, 128))
       ARD_TC_CASE(64, M_TILE_FWD, mt * cdiv(p.N, 64))
     } else if (op == OP_BWD_DATA) {
       const int mt = cdiv(p.B, BM);
+      if (pairs) return launch_mode<128, M_TILE_BWD_DATA, 2>(ctx, p, cdiv(p.B, 2 * BM) * cdiv(p.K, 128), s);
       ARD_TC_CASE(128, M_TILE_BWD_DATA, mt * cdiv(p.K, 128))
       ARD_TC_CASE(64, M_TILE_BWD_DATA, mt * cdiv(p.K, 64))
     } else {
