@@ -477,12 +477,19 @@ ard_status ard_blocks_products(ard_ctx* ctx, const ard_blocks* b, ard_dtype dA_d
   if (ldda < b->Kc || N < 1) return ARD_ERR_SHAPE;
   DevGuard guard(ctx->device);
   if (zero_fill_dropped) {
-    // on the caller's stream, before the fork: the input gradient's stream waits for it
+    // On the stream that will run the input gradient (the context's third stream when ard_layer_products forks),
+    // so that clearing the dropped blocks runs beside the forward product instead of ahead of everything.
+    cudaStream_t s = (cudaStream_t)cuda_stream, zs = s;
+    if (ctx->mlp_two_streams && ard_side_streams(ctx, s)) {
+      ARD_CUDA_OK(cudaEventRecord(ctx->ev[103], s));
+      ARD_CUDA_OK(cudaStreamWaitEvent(ctx->aux_stream, ctx->ev[103], 0));
+      zs = ctx->aux_stream;
+    }
     const int es = dA_dtype == ARD_F32 ? 4 : 2;
     const int nblocks = b->G * b->Q;
     const int grid = nblocks < ctx->sm_count * 32 ? nblocks : ctx->sm_count * 32;
-    ARD_CUDA_OK(ard_launch(ctx, zero_dropped_blocks_kernel, dim3(grid), dim3(256), 0, (cudaStream_t)cuda_stream,
-                           (const uint8_t*)b->d_keep, nblocks, b->Q, b->ts, dA, ldda * es, es));
+    ARD_CUDA_OK(ard_launch(ctx, zero_dropped_blocks_kernel, dim3(grid), dim3(256), 0, zs, (const uint8_t*)b->d_keep, nblocks,
+                           b->Q, b->ts, dA, ldda * es, es));
     ctx->launches++;
     ARD_CUDA_OK(cudaGetLastError());
   }
