@@ -7,7 +7,6 @@ picks, the drop rates of the two labels, brute-force loops over kept blocks, the
 plain matrix product, and the adjoint identities.
 """
 import numpy as np
-from scipy import stats
 
 from oracle import cnn_blocks as C
 
