@@ -107,7 +107,10 @@ ard_status ard_set_tile_n(ard_ctx* ctx, int bn);
  * (default 24).  0 keeps the current value of either.
  * Default: disabled.  On a B200 the parked partial sums and the later start of the shared tiles'
  * epilogues cost about what the better balance saves (a few percent either way, depending on the
- * period), and the forward product with zero fill gets slower. */
+ * period), and the forward product with zero fill gets slower.
+ * The partial sums live in one scratch per context, so the schedule needs the context's row products to run
+ * one after the other: the calls that enqueue several products side by side (ard_layer_products,
+ * ard_rows_products, ard_mlp_step on several streams) switch it off for their own launches. */
 ard_status ard_set_shared_tail(ard_ctx* ctx, int enable, int min_blocks, int min_gain_blocks);
 
 /* Sec. 3.3: the distribution K = {k_i}, i = 1..ndp, over the periods dp, sum k_i = 1.
@@ -208,7 +211,8 @@ ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, i
  *   starting any stream capture.  Every call on a device shares the one array, which keeps the
  *   previous call's contents (all entries that are read are rewritten first; nothing needs
  *   clearing).  Calls that overlap on the GPU (other streams, other host threads) race on it:
- *   serialise them. */
+ *   serialise them.  The looked-up address is cached per device in a plain host array without a lock: host
+ *   threads that make the first call at the same time all store the same value, which is harmless. */
 #define ARD_STATIC_SCRATCH_BYTES (8u << 20)
 ard_status ard_bwd_data_static_scratch(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N,
                                        float alpha, const void* dY, int lddy, const void* W, int ldw, void* dX,
@@ -351,22 +355,30 @@ ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, int n_layers,
  * of A are dropped, multiplies only the kept rows and fills the results back into the same rows of Y.
  * The paper fixes neither the region shape nor which values are sampled nor any constant; this library's
  * reading: regions of `region_rows` consecutive rows by the whole width; the random k_frac of a region's values
- * is taken in runs of c = gcd(Kc, 32) neighbouring values of a row (what one memory transaction delivers): of the
- * region's Cn = region_rows*Kc/c runs, n_c = max(1, floor(k_frac*Cn + 1/2)) are drawn with replacement; run d of
- * region g is chosen by word (d mod 4) of the Philox4x32-10 block with key (seed) and counter (iteration low,
- * iteration high, g, stream_id * 65536 + d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major
- * (runs below the last row of A count as not exceeding); s = n_c*c
- * samples; sensitive iff at least max(1, ceil(t_frac * s)) sampled values are > threshold; a probability p
+ * is drawn in runs of c = run_len neighbouring values of a row.  run_len = 1 is the text's statement: every
+ * sampled value is drawn on its own, one random word per value.  A larger run_len (it must divide Kc;
+ * gcd(Kc, 32) makes a run what one memory transaction delivers) is a departure from Sec. 5.1 that the caller
+ * asks for by name: neighbouring values of an im2col matrix are correlated, so the clustered sample is a
+ * different statistic, but it costs a fraction of the memory traffic.  Of the region's Cn = region_rows*Kc/c
+ * runs, n_c = max(1, floor(k_frac*Cn + 1/2)) are drawn with replacement; run d of region g is chosen by word
+ * (d mod 4) of the Philox4x32-10 block with key (seed) and counter (iteration low, iteration high, g,
+ * stream_id * 65536 + d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major (runs below the
+ * last row of A count as not exceeding); s = n_c*c samples; sensitive iff at least max(1, ceil(t_frac * s))
+ * sampled values are > threshold, the product taken exactly (t_frac is the binary fraction the double holds,
+ * so 0.3 of 10 samples needs 3 and 0.1 of 10 needs 2); a probability p
  * is the integer min(floor(p 2^32), 2^32 - 1); row r is dropped iff word 0 of the block with counter
  * (iteration low, iteration high, r, stream_id * 65536 + 65535) is below its region's integer.
  * stream_id < 65536.  Everything stays on the device; ard_rows_to_host is for tests. */
 ard_status ard_rows_create(ard_ctx* ctx, ard_rows** rows, int M, int region_rows);
 ard_status ard_rows_destroy(ard_rows* rows);
 /* Sec. 5.1: writes the dropout probability of every region (m_prob if sensitive, else n_prob).
- * A [M][Kc] (lda) of element type dtype.  Asynchronous. */
+ * A [M][Kc] (lda) of element type dtype.  run_len: see above (1 = independent values).  Errors:
+ * ARD_ERR_INVALID_ARG (run_len < 1 or not a divisor of Kc, fractions outside their ranges, stream_id >= 65536),
+ * ARD_ERR_UNSUPPORTED (more than 262140 runs per region).  Asynchronous. */
 ard_status ard_sensitivity_predict(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc,
-                                   double k_frac, double t_frac, float threshold, double m_prob, double n_prob,
-                                   uint64_t seed, uint64_t iteration, uint32_t stream_id, void* cuda_stream);
+                                   double k_frac, int run_len, double t_frac, float threshold, double m_prob,
+                                   double n_prob, uint64_t seed, uint64_t iteration, uint32_t stream_id,
+                                   void* cuda_stream);
 /* The same probability for every region (tests; p = 0 keeps every row).  Asynchronous. */
 ard_status ard_rows_set_probability(ard_ctx* ctx, ard_rows* rows, double p, void* cuda_stream);
 /* Sec. 5.2.1: draws the dropped rows and writes the ascending list of kept rows.  Asynchronous. */
@@ -447,12 +459,14 @@ ard_status ard_dropout_schedule(int n_epochs, double p_total, double mean_epoch,
  * A block is the dropout granularity.  Sec. 5.2.2 bounds the number of sensitive blocks per group so that
  * all groups keep nearly the same amount of work.  The paper fixes no constant, and the figure that shows the
  * balancing is not available; this library's reading: the prediction of Sec. 5.1 with one block as the
- * region, its random k_frac of the values taken in runs of c = gcd(ts, 32) neighbouring values of a row (what
- * one memory transaction delivers): of the block's Cn = ts*ts/c runs, n_c = max(1, floor(k_frac*Cn + 1/2))
+ * region, its random k_frac of the values drawn in runs of c = run_len neighbouring values of a row (run_len = 1,
+ * every value on its own, is the text's statement; a larger run_len, a divisor of ts, is the departure described
+ * for ard_sensitivity_predict): of the block's Cn = ts*ts/c runs, n_c = max(1, floor(k_frac*Cn + 1/2))
  * are drawn with replacement, s = n_c*c values are looked at; run d of block g*Q + j is chosen by word
  * (d mod 4) of the Philox4x32-10 block with key (seed) and counter (iteration low, iteration high, g*Q + j,
  * stream_id * 65536 + d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major; a block passes
- * iff at least max(1, ceil(t_frac * s)) sampled values are > threshold); of a group's passing blocks the
+ * iff at least max(1, ceil(t_frac * s)) sampled values are > threshold, the product taken exactly); of a
+ * group's passing blocks the
  * `cap` with the highest counts are sensitive (equal counts: lower j first); block g*Q + j is dropped iff
  * word 0 of the Philox block with counter (iteration low, iteration high, g*Q + j, stream_id * 65536 + 65535)
  * is below min(floor(p 2^32), 2^32 - 1), p = m_prob for a sensitive block, n_prob otherwise.
@@ -461,7 +475,7 @@ ard_status ard_blocks_create(ard_ctx* ctx, ard_blocks** blocks, int M, int Kc, i
 ard_status ard_blocks_destroy(ard_blocks* blocks);
 /* Counts and labels of all blocks.  A [M][Kc] (lda) on the device, element type dtype.  Asynchronous. */
 ard_status ard_blocks_predict(ard_ctx* ctx, ard_blocks* blocks, ard_dtype dtype, const void* A, int lda, double k_frac,
-                              double t_frac, float threshold, int cap, uint64_t seed, uint64_t iteration,
+                              int run_len, double t_frac, float threshold, int cap, uint64_t seed, uint64_t iteration,
                               uint32_t stream_id, void* cuda_stream);
 /* The same label for every block (tests; with ard_blocks_sample(m_prob = n_prob = 0) everything is kept). */
 ard_status ard_blocks_set_label(ard_ctx* ctx, ard_blocks* blocks, int sensitive, void* cuda_stream);

@@ -11,14 +11,17 @@ probabilities, multiplies only the kept rows and writes the results to the same 
 
 Readings (the paper fixes none of this; PARITY UNPINNED):
   * regions: x consecutive rows by the whole width of A (the row is the granularity of Sec. 5.2.1);
-  * the random k% of a region's values are taken in runs of c = gcd(Kc, 32) neighbouring values of a row (a run
-    is what one memory transaction delivers; isolated values would cost a transaction each): the region has
-    Cn = x*Kc/c runs, n_c = max(1, floor(k * Cn + 1/2)) of them are drawn with replacement, s = n_c * c values
-    are looked at; run d of region g is chosen by word (d mod 4) of the Philox4x32-10 block with key (seed) and
-    counter (iteration low, iteration high, g, stream_id * 65536 + d div 4) as run number
-    floor(word * Cn / 2^32), runs numbered row-major; runs below the last row of A (ragged last region) count
-    as not exceeding;
-  * sensitive iff the count of values above the threshold is >= max(1, ceil(t * s));
+  * the random k% of a region's values: every sampled value is drawn on its own, uniformly over the region's
+    x*Kc positions and with replacement, one Philox word per value (`run_len` = 1, the default, is the text's
+    statement).  `run_len` = c > 1 is an explicit departure, offered because a memory transaction delivers
+    neighbouring values: the positions are then drawn as runs of c neighbouring values of a row (c divides Kc).
+    In both cases the region has Cn = x*Kc/c runs, n_c = max(1, floor(k * Cn + 1/2)) of them are drawn,
+    s = n_c * c values are looked at; run d of region g is chosen by word (d mod 4) of the Philox4x32-10 block
+    with key (seed) and counter (iteration low, iteration high, g, stream_id * 65536 + d div 4) as run number
+    floor(word * Cn / 2^32), runs numbered row-major; positions below the last row of A (ragged last region)
+    count as not exceeding;
+  * sensitive iff the count of values above the threshold is >= max(1, ceil(t * s)), the product taken
+    exactly (t is the binary fraction the caller's double holds, s an integer);
   * a probability p becomes the integer P = min(floor(p * 2^32), 2^32 - 1); row r is dropped iff word 0 of the
     block with counter (iteration low, iteration high, r, stream_id * 65536 + 65535) is < P of its region;
   * no rescale is mentioned: alpha is an explicit argument, as for the other patterns;
@@ -27,6 +30,7 @@ Readings (the paper fixes none of this; PARITY UNPINNED):
 from __future__ import annotations
 
 import math
+from fractions import Fraction
 
 import numpy as np
 
@@ -36,37 +40,41 @@ TWO32 = 1 << 32
 MAX_BLOCKS = 65535
 
 
-def run_length(Kc):
+def transaction_run(Kc):
+    """The run length at which every run of bf16 / fp32 values is one aligned piece of a row: gcd(Kc, 32).
+    Not the default: pass it as `run_len` to ask for the clustered sample."""
     return math.gcd(Kc, 32)
 
 
-def n_runs(k_frac, x, Kc):
-    """How many runs of a region are drawn."""
-    return max(1, int(math.floor(k_frac * (x * (Kc // run_length(Kc))) + 0.5)))
+def n_runs(k_frac, x, Kc, run_len=1):
+    """How many runs of a region are drawn (run_len = 1: how many values)."""
+    assert run_len >= 1 and Kc % run_len == 0
+    return max(1, int(math.floor(k_frac * (x * (Kc // run_len)) + 0.5)))
 
 
-def n_samples(k_frac, x, Kc):
+def n_samples(k_frac, x, Kc, run_len=1):
     """How many values of a region are looked at."""
-    return n_runs(k_frac, x, Kc) * run_length(Kc)
+    return n_runs(k_frac, x, Kc, run_len) * run_len
 
 
 def needed(t_frac, s):
-    return max(1, int(math.ceil(t_frac * s - 1e-9)))
+    """Smallest count that reaches the fraction t of s sampled values: max(1, ceil(t * s)) in exact arithmetic."""
+    return max(1, math.ceil(Fraction(t_frac) * s))
 
 
 def quantise_probability(p):
     return min(int(math.floor(p * TWO32)), TWO32 - 1)
 
 
-def region_sensitive(A, g, x, k_frac, t_frac, threshold, seed, iteration, stream_id):
+def region_sensitive(A, g, x, k_frac, t_frac, threshold, seed, iteration, stream_id, run_len=1):
     """Sec. 5.1, steps 2-3 for region g.  Returns (sensitive, count, samples)."""
     A = np.asarray(A)
     M, Kc = A.shape
-    s = n_samples(k_frac, x, Kc)
-    c = run_length(Kc)
+    s = n_samples(k_frac, x, Kc, run_len)
+    c = run_len
     per_row = Kc // c
     Cn = x * per_row
-    n_c = n_runs(k_frac, x, Kc)
+    n_c = n_runs(k_frac, x, Kc, run_len)
     assert (n_c + 3) // 4 <= MAX_BLOCKS
     count = 0
     for q in range((n_c + 3) // 4):
@@ -82,7 +90,7 @@ def region_sensitive(A, g, x, k_frac, t_frac, threshold, seed, iteration, stream
     return count >= needed(t_frac, s), count, s
 
 
-def sensitivity_mask(A, x, k_frac, t_frac, threshold, m_prob, n_prob, seed, iteration, stream_id):
+def sensitivity_mask(A, x, k_frac, t_frac, threshold, m_prob, n_prob, seed, iteration, stream_id, run_len=1):
     """Sec. 5.1, step 4: the dropout probability of every region, as the integers the sampler compares with
     (sensitive regions get m_prob, the others n_prob; n_prob > m_prob)."""
     M = np.asarray(A).shape[0]
@@ -91,7 +99,7 @@ def sensitivity_mask(A, x, k_frac, t_frac, threshold, m_prob, n_prob, seed, iter
     out = np.empty(regions, dtype=np.uint64)
     sens = np.empty(regions, dtype=bool)
     for g in range(regions):
-        sens[g], _, _ = region_sensitive(A, g, x, k_frac, t_frac, threshold, seed, iteration, stream_id)
+        sens[g], _, _ = region_sensitive(A, g, x, k_frac, t_frac, threshold, seed, iteration, stream_id, run_len)
         out[g] = Pm if sens[g] else Pn
     return out, sens
 

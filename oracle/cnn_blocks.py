@@ -10,13 +10,16 @@ number, after which every group keeps nearly the same amount of work.
 
 Readings (the paper fixes none of this, and the figure that shows the balancing is not available;
 PARITY UNPINNED):
-  * prediction is that of Sec. 5.1 with one block as the region, and the random k% of its values are taken in
-    runs of c = gcd(ts, 32) neighbouring values of a row (a run is what one memory transaction delivers;
-    isolated values would cost a transaction each): a block has Cn = ts*ts/c runs, n_c = max(1, floor(k * Cn +
-    1/2)) of them are drawn with replacement, s = n_c * c values are looked at; run d is chosen by word
-    (d mod 4) of the Philox4x32-10 block with key (seed) and counter (iteration low, iteration high, g*Q + j,
-    stream_id * 65536 + d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major; the block
-    passes iff at least max(1, ceil(t * s)) of the values looked at exceed the threshold;
+  * prediction is that of Sec. 5.1 with one block as the region: every sampled value is drawn on its own,
+    uniformly over the block's ts*ts positions and with replacement, one Philox word per value (`run_len` = 1,
+    the default, is the text's statement).  `run_len` = c > 1 is an explicit departure, offered because a memory
+    transaction delivers neighbouring values: the positions are then drawn as runs of c neighbouring values of
+    a row (c divides ts).  In both cases a block has Cn = ts*ts/c runs, n_c = max(1, floor(k * Cn + 1/2)) of
+    them are drawn, s = n_c * c values are looked at; run d is chosen by word (d mod 4) of the Philox4x32-10
+    block with key (seed) and counter (iteration low, iteration high, g*Q + j, stream_id * 65536 + d div 4) as
+    run number floor(word * Cn / 2^32), runs numbered row-major; the block passes iff at least
+    max(1, ceil(t * s)) of the values looked at exceed the threshold, the product taken exactly (t is the
+    binary fraction the caller's double holds);
   * the bound: in every group at most `cap` blocks are labelled sensitive, namely the passing blocks with
     the highest counts (equal counts: the lower block index first);
   * a probability p becomes the integer P = min(floor(p * 2^32), 2^32 - 1); block (g, j) is dropped iff word 0
@@ -27,6 +30,7 @@ PARITY UNPINNED):
 from __future__ import annotations
 
 import math
+from fractions import Fraction
 
 import numpy as np
 
@@ -35,36 +39,40 @@ from .pattern import philox4x32_10, MASK32
 TWO32 = 1 << 32
 
 
-def run_length(ts):
+def transaction_run(ts):
+    """The run length at which every run of bf16 / fp32 values is one aligned piece of a row: gcd(ts, 32).
+    Not the default: pass it as `run_len` to ask for the clustered sample."""
     return math.gcd(ts, 32)
 
 
-def n_runs(k_frac, ts):
-    """How many runs of a block are drawn."""
-    return max(1, int(math.floor(k_frac * (ts * ts // run_length(ts)) + 0.5)))
+def n_runs(k_frac, ts, run_len=1):
+    """How many runs of a block are drawn (run_len = 1: how many values)."""
+    assert run_len >= 1 and ts % run_len == 0
+    return max(1, int(math.floor(k_frac * (ts * ts // run_len) + 0.5)))
 
 
-def n_samples(k_frac, ts):
+def n_samples(k_frac, ts, run_len=1):
     """How many values of a block are looked at."""
-    return n_runs(k_frac, ts) * run_length(ts)
+    return n_runs(k_frac, ts, run_len) * run_len
 
 
 def needed(t_frac, s):
-    return max(1, int(math.ceil(t_frac * s - 1e-9)))
+    """Smallest count that reaches the fraction t of s sampled values: max(1, ceil(t * s)) in exact arithmetic."""
+    return max(1, math.ceil(Fraction(t_frac) * s))
 
 
 def quantise_probability(p):
     return min(int(math.floor(p * TWO32)), TWO32 - 1)
 
 
-def block_count(A, g, j, ts, k_frac, threshold, seed, iteration, stream_id):
+def block_count(A, g, j, ts, k_frac, threshold, seed, iteration, stream_id, run_len=1):
     """Sec. 5.1, step 2 for block j of group g: how many of the sampled values exceed the threshold."""
     A = np.asarray(A)
     Q = A.shape[1] // ts
-    c = run_length(ts)
+    c = run_len
     Cn = ts * ts // c
     per_row = ts // c
-    n_c = n_runs(k_frac, ts)
+    n_c = n_runs(k_frac, ts, run_len)
     assert (n_c + 3) // 4 <= 65535
     count = 0
     for q in range((n_c + 3) // 4):
@@ -96,18 +104,18 @@ def label_group(counts, need, cap):
     return sens
 
 
-def predict(A, ts, k_frac, t_frac, threshold, cap, seed, iteration, stream_id):
+def predict(A, ts, k_frac, t_frac, threshold, cap, seed, iteration, stream_id, run_len=1):
     """Counts [G][Q] and sensitivity labels [G][Q] of all blocks."""
     A = np.asarray(A)
     M, Kc = A.shape
     assert M % ts == 0 and Kc % ts == 0
     G, Q = M // ts, Kc // ts
-    need = needed(t_frac, n_samples(k_frac, ts))
+    need = needed(t_frac, n_samples(k_frac, ts, run_len))
     counts = np.zeros((G, Q), dtype=np.int64)
     sens = np.zeros((G, Q), dtype=bool)
     for g in range(G):
         for j in range(Q):
-            counts[g, j] = block_count(A, g, j, ts, k_frac, threshold, seed, iteration, stream_id)
+            counts[g, j] = block_count(A, g, j, ts, k_frac, threshold, seed, iteration, stream_id, run_len)
         sens[g] = label_group(counts[g], need, cap)
     return counts, sens
 

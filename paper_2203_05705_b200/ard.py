@@ -109,7 +109,7 @@ def lib():
         "ard_dropout_schedule": [i32, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, P(C.c_double)],
         "ard_blocks_create": [vp, P(vp), i32, i32, i32],
         "ard_blocks_destroy": [vp],
-        "ard_blocks_predict": [vp, vp, i32, vp, i32, C.c_double, C.c_double, f32, i32, u64, u64, u32, vp],
+        "ard_blocks_predict": [vp, vp, i32, vp, i32, C.c_double, i32, C.c_double, f32, i32, u64, u64, u32, vp],
         "ard_blocks_set_label": [vp, vp, i32, vp],
         "ard_blocks_sample": [vp, vp, C.c_double, C.c_double, u64, u64, u32, vp],
         "ard_blocks_fwd": [vp, vp, i32, f32, vp, i32, vp, i32, vp, i32, vp],
@@ -119,7 +119,7 @@ def lib():
         "ard_blocks_to_host": [vp, P(C.c_int32), P(C.c_uint8), P(C.c_uint8), vp],
         "ard_rows_create": [vp, P(vp), i32, i32],
         "ard_rows_destroy": [vp],
-        "ard_sensitivity_predict": [vp, vp, i32, vp, i32, i32, C.c_double, C.c_double, f32, C.c_double, C.c_double, u64, u64,
+        "ard_sensitivity_predict": [vp, vp, i32, vp, i32, i32, C.c_double, i32, C.c_double, f32, C.c_double, C.c_double, u64, u64,
                                     u32, vp],
         "ard_rows_set_probability": [vp, vp, C.c_double, vp],
         "ard_rows_sample": [vp, vp, u64, u64, u32, vp],
@@ -381,10 +381,10 @@ def ard_blocks_destroy(blocks):
     _check(lib().ard_blocks_destroy(blocks), "ard_blocks_destroy")
 
 
-def ard_blocks_predict(ctx, blocks, dtype, A, lda, k_frac, t_frac, threshold, cap, seed, iteration, stream_id,
+def ard_blocks_predict(ctx, blocks, dtype, A, lda, k_frac, run_len, t_frac, threshold, cap, seed, iteration, stream_id,
                        stream=None):
-    _check(lib().ard_blocks_predict(ctx, blocks, dtype, _ptr(A), lda, k_frac, t_frac, threshold, cap, seed, iteration,
-                                    stream_id, _stream(stream)), "ard_blocks_predict")
+    _check(lib().ard_blocks_predict(ctx, blocks, dtype, _ptr(A), lda, k_frac, run_len, t_frac, threshold, cap, seed,
+                                    iteration, stream_id, _stream(stream)), "ard_blocks_predict")
 
 
 def ard_blocks_set_label(ctx, blocks, sensitive, stream=None):
@@ -443,10 +443,10 @@ def ard_rows_destroy(rows):
     _check(lib().ard_rows_destroy(rows), "ard_rows_destroy")
 
 
-def ard_sensitivity_predict(ctx, rows, dtype, A, lda, Kc, k_frac, t_frac, threshold, m_prob, n_prob, seed, iteration,
-                            stream_id, stream=None):
-    _check(lib().ard_sensitivity_predict(ctx, rows, dtype, _ptr(A), lda, Kc, k_frac, t_frac, threshold, m_prob, n_prob,
-                                         seed, iteration, stream_id, _stream(stream)), "ard_sensitivity_predict")
+def ard_sensitivity_predict(ctx, rows, dtype, A, lda, Kc, k_frac, run_len, t_frac, threshold, m_prob, n_prob, seed,
+                            iteration, stream_id, stream=None):
+    _check(lib().ard_sensitivity_predict(ctx, rows, dtype, _ptr(A), lda, Kc, k_frac, run_len, t_frac, threshold, m_prob,
+                                         n_prob, seed, iteration, stream_id, _stream(stream)), "ard_sensitivity_predict")
 
 
 def ard_rows_set_probability(ctx, rows, p, stream=None):

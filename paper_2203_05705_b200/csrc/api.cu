@@ -810,6 +810,14 @@ ard_status ard_layer_products(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dt
   if (((int)outmode & ARD_FLAG_RELU) != 0) return ARD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const bool streams = ctx->mlp_two_streams && ard_side_streams(ctx, s);
+  SharedTailOff tail_guard(ctx, streams);
+  // The compact copy of dY is shared by this call's two backward products only: whatever an earlier call left in
+  // the workspace is never taken for it (same buffer, new contents), and nothing is left for a later call.
+  struct ForgetGather {
+    ard_ctx* c;
+    explicit ForgetGather(ard_ctx* c_) : c(c_) { c->last_gather.src = nullptr; }
+    ~ForgetGather() { c->last_gather.src = nullptr; }
+  } forget(ctx);
   if (!streams) {
     // one stream: the calls in order, the second backward product reusing the first one's compact dY
     const int reuse = ctx->reuse_compact;
@@ -1399,6 +1407,7 @@ ard_status ard_rows_products(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dt
   if (!ctx || !rows || rows->ctx != ctx) return ARD_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const bool streams = ctx->mlp_two_streams && ard_side_streams(ctx, s);
+  SharedTailOff tail_guard(ctx, streams);
   cudaStream_t side = streams ? ctx->side_stream : s;
   DeviceGuard guard(ctx->device);
   if (streams) {

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <math.h>
 #include <stdint.h>
 
 #include <vector>
@@ -122,11 +123,31 @@ struct ard_ctx {
 static inline size_t sk_ws_bytes(int sm_count) { return (size_t)sm_count * 2 * 128 * 256 * sizeof(float); }
 static inline size_t sk_cnt_bytes(int sm_count) { return (size_t)sm_count * 8 * sizeof(int); }
 
+// max(1, ceil(t * s)) with the product taken exactly (Sec. 5.1, step 3: "at least t% of the sampled values").
+// t * s as a double is off by at most half a unit in the last place, which only matters when the rounded product
+// is an integer; the fused multiply-add gives the sign of what the rounding dropped.  Needs s < 2^31, 0 <= t <= 1.
+static inline long long ard_exact_need(double t, long long s) {
+  const double prod = t * (double)s;
+  const double err = fma(t, (double)s, -prod);
+  double c = ceil(prod);
+  if (c == prod && err > 0.0) c += 1.0;
+  return c < 1.0 ? 1 : (long long)c;
+}
+
 static inline int map_index_count(int dp_bound) { return dp_bound * (dp_bound + 1) / 2; }
 
 // Creates the context's second and third stream and their events on first use; false if they do not exist
 // and cannot be created now (`main` is being captured into a graph: nothing may be created then).
 bool ard_side_streams(ard_ctx* ctx, cudaStream_t main);
+
+// The shared tail of the row kernels parks partial sums in ONE scratch per context, so it must stay off while
+// products of the same context run side by side on several streams: calls that fork hold one of these.
+struct SharedTailOff {
+  ard_ctx* ctx;
+  int saved;
+  SharedTailOff(ard_ctx* c, bool forked) : ctx(c), saved(c->stream_k) { if (forked) c->stream_k = 0; }
+  ~SharedTailOff() { ctx->stream_k = saved; }
+};
 
 // ---- launchers implemented in the .cu files -----------------------------------------------------
 ard_status launch_sampler(ard_ctx* ctx, ard_pattern* pat, const unsigned long long* d_cdf, int ndp,

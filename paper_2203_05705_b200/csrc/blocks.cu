@@ -44,9 +44,10 @@ template <typename T> __device__ __forceinline__ float val_f(T v);
 template <> __device__ __forceinline__ float val_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float val_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-// Sec. 5.1, step 2 with a block as the region.  The sampled values are taken in runs of c = gcd(ts, 32)
-// neighbouring values of a row: a run is what one memory transaction delivers (64 bytes of bf16), where
-// isolated values cost a transaction each and made this kernel read more than the kept blocks themselves.
+// Sec. 5.1, step 2 with a block as the region.  The sampled values are taken in runs of c neighbouring values of
+// a row.  c = 1 is the text's statement (every value drawn on its own) and the default of the entry point; with
+// c = gcd(ts, 32) a run is what one memory transaction delivers (64 bytes of bf16), where isolated values cost a
+// transaction each and make this kernel read more than the kept blocks themselves.
 // One warp per block (g, j); lane l takes the runs l, l + 32, ...: run d is chosen by word (d mod 4) of the
 // Philox block (d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major inside the block.
 template <typename T>
@@ -354,23 +355,23 @@ ard_status ard_blocks_destroy(ard_blocks* b) {
 }
 
 ard_status ard_blocks_predict(ard_ctx* ctx, ard_blocks* b, ard_dtype dtype, const void* A, int lda, double k_frac,
-                              double t_frac, float threshold, int cap, uint64_t seed, uint64_t iteration,
+                              int run_len, double t_frac, float threshold, int cap, uint64_t seed, uint64_t iteration,
                               uint32_t stream_id, void* cuda_stream) {
   if (!ctx || !b || b->ctx != ctx || !A) return ARD_ERR_INVALID_ARG;
   if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
   if (lda < b->Kc) return ARD_ERR_SHAPE;
   if (!(k_frac > 0.0) || k_frac > 1.0 || !(t_frac >= 0.0) || t_frac > 1.0 || cap < 0 || stream_id >= 65536u)
     return ARD_ERR_INVALID_ARG;
-  int c = b->ts, r32 = 32;
-  while (r32) { const int t = c % r32; c = r32; r32 = t; }  // c = gcd(ts, 32): values per run
+  if (run_len < 1 || b->ts % run_len != 0) return ARD_ERR_INVALID_ARG;
+  const int c = run_len;  // values per run
   const long long Cn = (long long)b->ts * (b->ts / c);
   const double rd = floor(k_frac * (double)Cn + 0.5);
   const long long n_runs_ll = rd < 1.0 ? 1 : (long long)rd;
   if ((n_runs_ll + 3) / 4 > 65535) return ARD_ERR_UNSUPPORTED;
   const int n_runs = (int)n_runs_ll;
   const long long samples = n_runs_ll * c;
-  const double nd = ceil(t_frac * (double)samples - 1e-9);
-  const int need = nd < 1.0 ? 1 : (int)nd;
+  if (samples >= (1ll << 31)) return ARD_ERR_UNSUPPORTED;
+  const int need = (int)ard_exact_need(t_frac, samples);
   DevGuard guard(ctx->device);
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int nblocks = b->G * b->Q;

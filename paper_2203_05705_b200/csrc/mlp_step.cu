@@ -34,6 +34,7 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
   bool two = ctx->mlp_two_streams && n_layers >= 2 && n_layers <= 32;
   for (int l = 0; l + 1 < n_layers && two; ++l) two = layers[l].compact_out != 0;
   if (two && !ard_side_streams(ctx, main_s)) two = false;
+  SharedTailOff tail_guard(ctx, two);
   cudaStream_t side_s = two ? ctx->side_stream : main_s;
   cudaStream_t aux_s = two ? ctx->aux_stream : main_s;
   void* side = (void*)side_s;

@@ -29,9 +29,10 @@ template <typename T> __device__ __forceinline__ float val_f(T v);
 template <> __device__ __forceinline__ float val_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float val_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-// Sec. 5.1, steps 2-4.  The sampled values are taken in runs of c = gcd(Kc, 32) neighbouring values of a row: a
-// run is what one memory transaction delivers (64 bytes of bf16), where isolated values cost a transaction each
-// (3.8 M scattered reads and 208 MB of DRAM traffic per prediction on a 32768 x 2304 matrix, 41 us).
+// Sec. 5.1, steps 2-4.  The sampled values are taken in runs of c neighbouring values of a row.  c = 1 is the
+// text's statement (every value drawn on its own) and the default of the entry point; with c = gcd(Kc, 32) a run is
+// what one memory transaction delivers (64 bytes of bf16), where isolated values cost a transaction each
+// (3.8 M scattered reads and 208 MB of DRAM traffic per prediction on a 32768 x 2304 matrix, 41 us against 11).
 // One warp per region of x rows by the whole width; lane l takes the runs l, l + 32, ...: run d is chosen by word
 // (d mod 4) of the Philox block (d div 4) as run number floor(word * Cn / 2^32), runs numbered row-major.
 template <typename T>
@@ -336,23 +337,24 @@ ard_status ard_rows_destroy(ard_rows* rows) {
 }
 
 ard_status ard_sensitivity_predict(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc,
-                                   double k_frac, double t_frac, float threshold, double m_prob, double n_prob,
-                                   uint64_t seed, uint64_t iteration, uint32_t stream_id, void* cuda_stream) {
+                                   double k_frac, int run_len, double t_frac, float threshold, double m_prob,
+                                   double n_prob, uint64_t seed, uint64_t iteration, uint32_t stream_id,
+                                   void* cuda_stream) {
   if (!ctx || !rows || rows->ctx != ctx || !A) return ARD_ERR_INVALID_ARG;
   if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
   if (Kc < 1 || lda < Kc) return ARD_ERR_SHAPE;
   if (!(k_frac > 0.0 && k_frac <= 1.0) || !(t_frac >= 0.0 && t_frac <= 1.0)) return ARD_ERR_INVALID_ARG;
   if (!(m_prob >= 0.0 && m_prob <= 1.0) || !(n_prob >= 0.0 && n_prob <= 1.0) || stream_id > 0xFFFFu) return ARD_ERR_INVALID_ARG;
-  int c = Kc, r32 = 32;
-  while (r32) { const int t = c % r32; c = r32; r32 = t; }  // c = gcd(Kc, 32): values per run
+  if (run_len < 1 || Kc % run_len != 0) return ARD_ERR_INVALID_ARG;
+  const int c = run_len;  // values per run
   const double Cn = (double)rows->x * (double)(Kc / c);
   if (Cn >= 4294967296.0) return ARD_ERR_UNSUPPORTED;  // run numbers are 32-bit
   const double rd = floor(k_frac * Cn + 0.5);
   const long long n_runs = rd < 1.0 ? 1 : (long long)rd;
   if ((n_runs + 3) / 4 > 65535) return ARD_ERR_UNSUPPORTED;  // the block index shares a counter word with the stream id
   const long long samples = n_runs * c;
-  const double nd = ceil(t_frac * (double)samples - 1e-9);
-  const int need = nd < 1.0 ? 1 : (int)nd;
+  if (samples >= (1ll << 31)) return ARD_ERR_UNSUPPORTED;
+  const int need = (int)ard_exact_need(t_frac, samples);
   DevGuard guard(ctx->device);
   return launch_sensitivity(ctx, rows, dtype, A, lda, Kc, c, (int)n_runs, need, threshold, quantise_probability(m_prob),
                             quantise_probability(n_prob), seed, iteration, stream_id, (cudaStream_t)cuda_stream);

@@ -2,8 +2,7 @@
 implementation used by the tests.
 
 This module holds none of the method's arithmetic: it only draws tensors with
-the shapes and value distributions of the paper's MLP / LSTM workloads (Sec. 7)
-and builds the pattern distribution K that is an *input* of the hot path.
+the shapes and value distributions of the paper's MLP / LSTM workloads (Sec. 7).
 It imports neither the CUDA binding nor that reference implementation.
 """
 from __future__ import annotations
@@ -32,36 +31,6 @@ def bf16_to_f32(bits: np.ndarray) -> np.ndarray:
 def bf16_round(x: np.ndarray) -> np.ndarray:
     """fp32 array holding values exactly representable in bf16."""
     return bf16_to_f32(bf16_bits(x)).reshape(np.shape(x))
-
-
-def max_entropy_K(p: float, n_dp: int) -> np.ndarray:
-    """The distribution over periods dp = 1..n_dp used for every benchmark and
-    test: the maximum-entropy distribution whose global dropout rate
-    sum_i k_i (i-1)/i equals p, i.e. k_i proportional to exp(beta (i-1)/i),
-    beta found by bisection.  It stands in for the output of the paper's
-    SGD-based search (Sec. 3.3), whose loss rewards exactly these two things
-    (rate error and entropy) but whose constants are not printed."""
-    if n_dp < 2:
-        raise ValueError("need at least two periods")
-    pu = np.array([(i - 1) / i for i in range(1, n_dp + 1)], dtype=np.float64)
-    if not (0.0 < p < pu[-1]):
-        raise ValueError("target rate must lie in (0, (n_dp-1)/n_dp)")
-
-    def rate(beta):
-        w = np.exp(beta * (pu - pu.max())) if beta > 0 else np.exp(beta * pu)
-        k = w / w.sum()
-        return float(k @ pu), k
-
-    lo, hi = -200.0, 200.0
-    for _ in range(200):
-        mid = 0.5 * (lo + hi)
-        r, _k = rate(mid)
-        if r < p:
-            lo = mid
-        else:
-            hi = mid
-    _r, k = rate(0.5 * (lo + hi))
-    return k / k.sum()
 
 
 # ---------------------------------------------------------------------------

@@ -4,6 +4,7 @@ import os
 import re
 
 import pytest
+from distributions import max_entropy_K
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -72,7 +73,7 @@ def test_host_side_quantiser_matches_the_oracle(built):
     import numpy as np
     from oracle import pattern as OP
     from paper_2203_05705_b200 import ard, inputs
-    cases = [inputs.max_entropy_K(p, n) for p, n in [(0.3, 16), (0.5, 16), (0.7, 16), (0.5, 8), (0.9, 64)]]
+    cases = [max_entropy_K(p, n) for p, n in [(0.3, 16), (0.5, 16), (0.7, 16), (0.5, 8), (0.9, 64)]]
     cases += [[1.0], [0.25, 0.0, 0.5, 0.0, 0.25], [0.0, 0.0, 1.0], [1e-12, 1.0 - 1e-12]]
     rng = np.random.default_rng(0)
     for _ in range(20):

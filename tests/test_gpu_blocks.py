@@ -39,11 +39,13 @@ def test_counts_labels_draws_and_lists_are_bit_exact(M, Kc, ts, dtype):
         pat = ard.ard_blocks_pattern(blocks)
         cases = [(0.02, 0.3, 0.5, max(1, Q // 2), 0.2, 0.8), (0.05, 0.25, 0.1, 1, 0.0, 1.0), (0.03, 0.4, 0.3, Q, 0.35, 0.65),
                  (0.02, 0.3, 0.5, 0, 0.1, 0.5)]
-        for it, (k, t, thr, cap, mp, npb) in enumerate(cases):
-            ard.ard_blocks_predict(ctx.h, blocks, dtype, Ad, Kc + 8, k, t, thr, cap, 99, it, 5)
+        # every case with run length 1 (each value drawn on its own: the statement of Sec. 5.1) and in the run form
+        cases = [c + (rl,) for rl in (1, OB.transaction_run(ts)) for c in cases]
+        for it, (k, t, thr, cap, mp, npb, rl) in enumerate(cases):
+            ard.ard_blocks_predict(ctx.h, blocks, dtype, Ad, Kc + 8, k, rl, t, thr, cap, 99, it, 5)
             ard.ard_blocks_sample(ctx.h, blocks, mp, npb, 99, it, 5)
             counts, sens, keep = ard.ard_blocks_to_host(blocks, G * Q)
-            co, so = OB.predict(A, ts, k, t, thr, cap, 99, it, 5)
+            co, so = OB.predict(A, ts, k, t, thr, cap, 99, it, 5, run_len=rl)
             assert np.array_equal(counts.reshape(G, Q), co), it
             assert np.array_equal(sens.reshape(G, Q).astype(bool), so), it
             if 0 < cap < Q:
@@ -178,7 +180,7 @@ def test_benchmark_layer_on_sampled_outputs():
         Ad = torch.from_numpy(A).to(BF).cuda()
         Wd = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
         dYt = torch.from_numpy(np.ascontiguousarray(dY.T)).to(BF).cuda()
-        ard.ard_blocks_predict(ctx.h, blocks, ard.ARD_BF16, Ad, K, kf, tf, thr, cap, 5, 3, 1)
+        ard.ard_blocks_predict(ctx.h, blocks, ard.ARD_BF16, Ad, K, kf, 1, tf, thr, cap, 5, 3, 1)
         ard.ard_blocks_sample(ctx.h, blocks, mp, npb, 5, 3, 1)
         counts, sens, keep = ard.ard_blocks_to_host(blocks, G * Q)
         counts, sens, keep = counts.reshape(G, Q), sens.reshape(G, Q).astype(bool), keep.reshape(G, Q).astype(bool)
@@ -237,9 +239,13 @@ def test_argument_checks():
         blocks = ard.ard_blocks_create(ctx.h, 128, 128, 64)
         A = torch.zeros((128, 128), dtype=BF, device="cuda")
         with pytest.raises(ard.ArdError):
-            ard.ard_blocks_predict(ctx.h, blocks, ard.ARD_BF16, A, 64, 0.1, 0.5, 0.5, 1, 0, 0, 0)      # lda < Kc
+            ard.ard_blocks_predict(ctx.h, blocks, ard.ARD_BF16, A, 64, 0.1, 1, 0.5, 0.5, 1, 0, 0, 0)      # lda < Kc
         with pytest.raises(ard.ArdError):
-            ard.ard_blocks_predict(ctx.h, blocks, ard.ARD_BF16, A, 128, 0.1, 0.5, 0.5, 1, 0, 0, 1 << 16)
+            ard.ard_blocks_predict(ctx.h, blocks, ard.ARD_BF16, A, 128, 0.1, 1, 0.5, 0.5, 1, 0, 0, 1 << 16)
+        with pytest.raises(ard.ArdError):
+            ard.ard_blocks_predict(ctx.h, blocks, ard.ARD_BF16, A, 128, 0.1, 48, 0.5, 0.5, 1, 0, 0, 0)    # 48 does not divide 64
+        with pytest.raises(ard.ArdError):
+            ard.ard_blocks_predict(ctx.h, blocks, ard.ARD_BF16, A, 128, 0.1, 0, 0.5, 0.5, 1, 0, 0, 0)
         with pytest.raises(ard.ArdError):
             ard.ard_blocks_sample(ctx.h, blocks, 0.2, 1.5, 0, 0, 0)
         ard.ard_blocks_destroy(blocks)

@@ -8,6 +8,7 @@ import pytest
 
 from paper_2203_05705_b200 import ard, inputs
 from gpu_helpers import Ctx, run_three_gemms, assert_ok, TOL
+from distributions import max_entropy_K
 
 pytestmark = pytest.mark.gpu
 
@@ -68,7 +69,7 @@ def test_row_sampled_patterns_auto_path(ctx):
     from oracle import pattern as OP
     B, K, N = 128, 784, 2048                         # first hidden layer of the 784-2048-2048-10 MLP
     X, W, dY = _layer(B, K, N, 3, np.sqrt(2.0 / K))
-    Kd = inputs.max_entropy_K(0.5, 16)
+    Kd = max_entropy_K(0.5, 16)
     cdf = OP.quantise_K(Kd)
     ard.ard_set_distribution(ctx.h, 0, Kd)
     pat = ctx.pattern(ard.ARD_ROW, K, N)

@@ -5,6 +5,7 @@ import pytest
 from oracle import pattern as OP
 from paper_2203_05705_b200 import ard, inputs
 from gpu_helpers import Ctx, run_three_gemms, assert_ok, TOL
+from distributions import max_entropy_K
 
 pytestmark = pytest.mark.gpu
 
@@ -30,7 +31,7 @@ def test_config1_all_patterns(ctx):
 
 def test_config1_sampled_iterations(ctx):
     c1 = inputs.config1()
-    K = inputs.max_entropy_K(c1["p"], c1["n_dp"])
+    K = max_entropy_K(c1["p"], c1["n_dp"])
     cdf = OP.quantise_K(K)
     ard.ard_set_distribution(ctx.h, 0, K)
     pat = ctx.pattern(ard.ARD_ROW, 784, 256)

@@ -16,6 +16,7 @@ from oracle import mlp as OM
 from oracle import pattern as OP
 from paper_2203_05705_b200 import ard, inputs
 from gpu_helpers import Ctx, host, tdtype, TOL
+from distributions import max_entropy_K
 
 pytestmark = pytest.mark.gpu
 
@@ -200,7 +201,7 @@ def test_a_captured_step_draws_a_new_pattern_at_every_replay():
     rng = np.random.default_rng(4)
     W = _rnd(rng, (K, N), dtype, 1.0 / np.sqrt(K))
     X = _rnd(rng, (B, K), dtype)
-    Kd = inputs.max_entropy_K(0.5, 8)
+    Kd = max_entropy_K(0.5, 8)
     cdf = OP.quantise_K(Kd)
     ctx = Ctx(1 << 20)
     try:
@@ -285,7 +286,7 @@ def test_mlp_step_784_2048_2048_10(compact, p):
     oracle's step on the same inputs with a tolerance for the bf16 activations in between."""
     dims, B = [784, 2048, 2048, 10], 128
     rng = np.random.default_rng(17)
-    Kd = inputs.max_entropy_K(p, 16)
+    Kd = max_entropy_K(p, 16)
     cdf = OP.quantise_K(Kd)
     ctx = Ctx(2 * B * 2048 + 4096)
     try:
@@ -438,7 +439,7 @@ def test_mlp_step_replayed_from_a_graph_equals_the_same_iterations_called_one_by
     rng = np.random.default_rng(23)
     ctx = Ctx(4096)
     try:
-        ard.ard_set_distribution(ctx.h, 0, inputs.max_entropy_K(p, 16))
+        ard.ard_set_distribution(ctx.h, 0, max_entropy_K(p, 16))
         layers, arr, _, _ = _stack(ctx, dims, B, p, 1, rng)
         L = len(layers)
         counter = torch.zeros(1, dtype=torch.int64, device="cuda")

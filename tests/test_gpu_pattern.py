@@ -6,6 +6,7 @@ import torch
 from oracle import pattern as OP
 from paper_2203_05705_b200 import ard, inputs
 from gpu_helpers import Ctx
+from distributions import max_entropy_K
 
 pytestmark = pytest.mark.gpu
 
@@ -19,7 +20,7 @@ def ctx():
 
 def test_cdf_table_matches_oracle(ctx):
     for i, (p, n) in enumerate([(0.3, 16), (0.5, 16), (0.7, 16), (0.5, 8)]):
-        K = inputs.max_entropy_K(p, n)
+        K = max_entropy_K(p, n)
         ard.ard_set_distribution(ctx.h, i, K)
         assert ard.ard_get_distribution_cdf(ctx.h, i).tolist() == OP.quantise_K(K)
     K = [0.25, 0.0, 0.5, 0.0, 0.25]
@@ -29,7 +30,7 @@ def test_cdf_table_matches_oracle(ctx):
 
 @pytest.mark.parametrize("p,n_dp,N", [(0.5, 8, 256), (0.3, 16, 2048), (0.7, 16, 1000)])
 def test_sampled_row_patterns_bit_exact(ctx, p, n_dp, N):
-    K = inputs.max_entropy_K(p, n_dp)
+    K = max_entropy_K(p, n_dp)
     cdf = OP.quantise_K(K)
     ard.ard_set_distribution(ctx.h, 0, K)
     pat = ctx.pattern(ard.ARD_ROW, 64, N)
@@ -48,7 +49,7 @@ def test_sampled_row_patterns_bit_exact(ctx, p, n_dp, N):
 def test_sampler_statistics_many_counters(ctx):
     """10^5 counters: the device histogram of (dp, b) equals the oracle's exactly."""
     p, n_dp, N = 0.5, 16, 64
-    K = inputs.max_entropy_K(p, n_dp)
+    K = max_entropy_K(p, n_dp)
     cdf = OP.quantise_K(K)
     ard.ard_set_distribution(ctx.h, 1, K)
     pat = ctx.pattern(ard.ARD_ROW, 8, N)
@@ -60,7 +61,7 @@ def test_sampler_statistics_many_counters(ctx):
 
 
 def test_counter_is_stateless(ctx):
-    K = inputs.max_entropy_K(0.5, 8)
+    K = max_entropy_K(0.5, 8)
     ard.ard_set_distribution(ctx.h, 2, K)
     pat = ctx.pattern(ard.ARD_ROW, 8, 100)
     ard.ard_sample_pattern(ctx.h, pat, 2, 5, 17, 0)
@@ -92,7 +93,7 @@ def test_tile_lists_bit_exact(ctx, Kd, Nd, ts):
 
 
 def test_sampled_tile_pattern(ctx):
-    K = inputs.max_entropy_K(0.5, 16)
+    K = max_entropy_K(0.5, 16)
     cdf = OP.quantise_K(K)
     ard.ard_set_distribution(ctx.h, 3, K)
     pat = ctx.pattern(ard.ARD_TILE, 512, 512, 64)
@@ -117,7 +118,7 @@ def test_host_side_rejections(ctx):
         ard.ard_pattern_create(h, ard.ARD_TILE, 100, 64, 64)
     assert e.value.status == ard.ARD_ERR_SHAPE
     pat = ctx.pattern(ard.ARD_ROW, 8, 4)
-    ard.ard_set_distribution(h, 4, inputs.max_entropy_K(0.5, 8))
+    ard.ard_set_distribution(h, 4, max_entropy_K(0.5, 8))
     with pytest.raises(ard.ArdError) as e:                       # more periods than units (dp_max = M)
         ard.ard_sample_pattern(h, pat, 4, 0, 0, 0)
     assert e.value.status == ard.ARD_ERR_DISTRIBUTION

@@ -35,11 +35,14 @@ def test_prediction_and_row_list_are_bit_exact(M, Kc, x, dtype):
     rows = ard.ard_rows_create(ctx.h, M, x)
     try:
         regions = (M + x - 1) // x
-        for it, (k, t, thr, mp, npb) in enumerate([(0.3, 0.3, 0.5, 0.2, 0.8), (0.05, 0.25, 0.1, 0.0, 1.0), (1.0, 0.4, 0.3, 0.35, 0.65)]):
-            ard.ard_sensitivity_predict(ctx.h, rows, dtype, Ad, Kc + 8, Kc, k, t, thr, mp, npb, 99, it, 5)
+        # run length 1 (every value drawn on its own: the statement of Sec. 5.1) and the opt-in run form
+        cases = [(0.3, 0.3, 0.5, 0.2, 0.8, 1), (0.05, 0.25, 0.1, 0.0, 1.0, 1), (1.0, 0.4, 0.3, 0.35, 0.65, 1),
+                 (0.3, 0.3, 0.5, 0.2, 0.8, OC.transaction_run(Kc)), (0.05, 0.1, 0.1, 0.0, 1.0, OC.transaction_run(Kc))]
+        for it, (k, t, thr, mp, npb, rl) in enumerate(cases):
+            ard.ard_sensitivity_predict(ctx.h, rows, dtype, Ad, Kc + 8, Kc, k, rl, t, thr, mp, npb, 99, it, 5)
             ard.ard_rows_sample(ctx.h, rows, 99, it, 5)
             n_keep, idx, P = ard.ard_rows_to_host(rows, M, regions)
-            Po, sens = OC.sensitivity_mask(A, x, k, t, thr, mp, npb, 99, it, 5)
+            Po, sens = OC.sensitivity_mask(A, x, k, t, thr, mp, npb, 99, it, 5, run_len=rl)
             assert np.array_equal(P.astype(np.uint64), Po), (it, int((P.astype(np.uint64) != Po).sum()))
             assert 0 < sens.sum() < regions                      # the input has both kinds of region
             keep = OC.draw_rows(Po, x, M, 99, it, 5)
@@ -233,13 +236,14 @@ def test_benchmark_layer_on_sampled_outputs():
         dYd = torch.from_numpy(dY).to(BF).cuda()
         Wd = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
         # Sec. 5.1 on sampled regions (integer decisions: exact)
-        ard.ard_sensitivity_predict(ctx.h, rows, ard.ARD_BF16, Ad, K, K, kf, tf, thr, mp, npb, 5, 3, 1)
-        _, _, P = ard.ard_rows_to_host(rows, M, M // x)
         Pm, Pn = OC.quantise_probability(mp), OC.quantise_probability(npb)
-        for g in range(5, M // x, (M // x) // 40):
-            sens, _, _ = OC.region_sensitive(A, g, x, kf, tf, thr, 5, 3, 1)
-            assert int(P[g]) == (Pm if sens else Pn), g
-        assert 0 < int(np.sum(P == Pm)) < M // x                     # both kinds of region occur
+        for rl in (1, OC.transaction_run(K)):
+            ard.ard_sensitivity_predict(ctx.h, rows, ard.ARD_BF16, Ad, K, K, kf, rl, tf, thr, mp, npb, 5, 3, 1)
+            _, _, P = ard.ard_rows_to_host(rows, M, M // x)
+            for g in range(5, M // x, (M // x) // 40):
+                sens, _, _ = OC.region_sensitive(A, g, x, kf, tf, thr, 5, 3, 1, run_len=rl)
+                assert int(P[g]) == (Pm if sens else Pn), (g, rl)
+            assert 0 < int(np.sum(P == Pm)) < M // x                     # both kinds of region occur
         # Sec. 5.2.1 with one probability for every region: the whole list against the oracle
         ard.ard_rows_set_probability(ctx.h, rows, 0.46)
         ard.ard_rows_sample(ctx.h, rows, 5, 3, 1)

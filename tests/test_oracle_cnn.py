@@ -36,20 +36,59 @@ def test_ragged_last_region_counts_missing_rows_as_below():
     assert abs(np.mean(fr) - 0.25) < 0.02          # a quarter of the positions exist
 
 
+def test_default_draws_every_value_on_its_own():
+    """Sec. 5.1, step 2 says a random k% of the VALUES: with the default run length the sampled positions are
+    independent, so over a region whose values above the threshold sit side by side the count is binomial over
+    single values -- not a multiple of a run length, and with the variance of independent draws (a sample taken in
+    runs of c neighbours has c times that variance)."""
+    x, Kc = 4, 64
+    A = np.zeros((x, Kc))
+    A[1, 0:32] = 1.0                               # one aligned piece of 32 neighbouring values above
+    A[3, 32:64] = 1.0                              # and another
+    s = C.n_samples(0.25, x, Kc)
+    assert s == C.n_runs(0.25, x, Kc) == 64        # run_len = 1: a run is one value
+    f = 64 / (x * Kc)
+    res = np.array([C.region_sensitive(A, 0, x, 0.25, 0.5, 0.5, 3, it, 0)[1] for it in range(1200)])
+    assert np.any(res % 2 == 1) and len(set(res.tolist())) > 8
+    assert abs(res.mean() - s * f) < 4 * np.sqrt(s * f * (1 - f) / 1200)
+    assert abs(res.var() - s * f * (1 - f)) < 0.2 * s * f * (1 - f)
+    # two neighbouring positions are hit independently: P(both looked at) = P(one)^2 for single draws
+    B = np.zeros((x, Kc))
+    B[2, 10] = B[2, 11] = 1.0
+    one = 1 - (1 - 1 / (x * Kc)) ** s              # a given position is looked at at least once
+    both = 1 - 2 * (1 - 1 / (x * Kc)) ** s + (1 - 2 / (x * Kc)) ** s
+    cnt = np.array([C.region_sensitive(B, 0, x, 0.25, 0.5, 0.5, 9, it, 1)[1] for it in range(3000)])
+    B[2, 11] = 0.0
+    cnt_one = np.array([C.region_sensitive(B, 0, x, 0.25, 0.5, 0.5, 9, it, 1)[1] for it in range(3000)])
+    B[2, 10], B[2, 11] = 0.0, 1.0
+    cnt_other = np.array([C.region_sensitive(B, 0, x, 0.25, 0.5, 0.5, 9, it, 1)[1] for it in range(3000)])
+    p_both = np.mean((cnt_one > 0) & (cnt_other > 0))
+    assert abs(np.mean(cnt_one > 0) - one) < 4 * np.sqrt(one * (1 - one) / 3000)
+    assert abs(p_both - both) < 4 * np.sqrt(both * (1 - both) / 3000) + 2e-3   # runs of neighbours: p_both = one
+    assert np.array_equal(cnt, cnt_one + cnt_other)                              # same positions, whatever A holds
+
+
+def test_threshold_count_is_exact():
+    # ceil(t * s) with the product taken exactly: 0.3 (a little below 3/10 as a double) of 10 samples needs 3,
+    # 0.1 (a little above 1/10) of 10 needs 2, a half of 7 needs 4, and at least one value is always needed
+    assert C.needed(0.3, 10) == 3 and C.needed(0.1, 10) == 2 and C.needed(0.5, 7) == 4 and C.needed(0.5, 8) == 4
+    assert C.needed(0.0, 100) == 1 and C.needed(1.0, 100) == 100 and C.needed(0.25, 1 << 30) == 1 << 28
+
+
 def test_decision_follows_the_binomial_law_over_runs():
-    # whole runs (32 neighbouring values of a row) above or below the threshold: the count is 32 times a binomial
-    # variable over the drawn runs
+    # the opt-in run form: whole runs (32 neighbouring values of a row) above or below the threshold: the count is
+    # 32 times a binomial variable over the drawn runs
     rng = np.random.default_rng(0)
     x, Kc = 8, 64
-    assert C.run_length(Kc) == 32 and C.run_length(200) == 8 and C.run_length(33) == 1
+    assert C.transaction_run(Kc) == 32 and C.transaction_run(200) == 8 and C.transaction_run(33) == 1
     above = np.zeros(16, dtype=bool)
     above[rng.choice(16, 6, replace=False)] = True
     A = np.repeat(above.reshape(x, 2), 32, axis=1).astype(np.float64)
-    n_c = C.n_runs(0.5, x, Kc)
-    s = C.n_samples(0.5, x, Kc)
+    n_c = C.n_runs(0.5, x, Kc, 32)
+    s = C.n_samples(0.5, x, Kc, 32)
     assert n_c == 8 and s == 256
     need_runs = -(-C.needed(0.5, s) // 32)
-    res = [C.region_sensitive(A, 0, x, 0.5, 0.5, 0.5, 11, it, 0) for it in range(1500)]
+    res = [C.region_sensitive(A, 0, x, 0.5, 0.5, 0.5, 11, it, 0, run_len=32) for it in range(1500)]
     assert all(c % 32 == 0 and n == s for _, c, n in res)
     hits = sum(r[0] for r in res)
     p_theory = stats.binom.sf(need_runs - 1, n_c, 6 / 16)
@@ -61,13 +100,13 @@ def test_decision_follows_the_binomial_law_over_runs():
 
 def test_runs_are_drawn_uniformly_and_stay_in_their_region():
     x, Kc = 2, 16                                  # runs of 16: a run is a whole row; region 1 = rows 2, 3
-    n_c = C.n_runs(1.0, x, Kc)
+    n_c = C.n_runs(1.0, x, Kc, 16)
     assert n_c == 2
     hits = np.zeros(6)
     for r in range(6):
         A = np.zeros((6, Kc))
         A[r] = 1.0
-        hits[r] = sum(C.region_sensitive(A, 1, x, 1.0, 0.5, 0.5, 5, it, 1)[1] for it in range(400)) / 16
+        hits[r] = sum(C.region_sensitive(A, 1, x, 1.0, 0.5, 0.5, 5, it, 1, run_len=16)[1] for it in range(400)) / 16
     assert hits[0] == hits[1] == hits[4] == hits[5] == 0          # other regions' rows are never looked at
     expect = 400 * n_c / 2
     assert np.all(np.abs(hits[2:4] - expect) < 4.5 * np.sqrt(expect / 2))

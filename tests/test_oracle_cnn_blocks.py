@@ -17,24 +17,42 @@ def test_counts_that_do_not_depend_on_the_sample():
     A[0:4, 4:8] = 1.0                  # block (0, 1): every value above the threshold
     for it in range(4):
         counts, sens = C.predict(A, ts, 0.5, 0.5, 0.5, 3, 7, it, 2)
-        assert counts[0, 1] == C.n_samples(0.5, ts) == 8      # two runs of four values
+        assert counts[0, 1] == C.n_samples(0.5, ts) == 8      # eight single values
         assert counts.sum() == 8
         assert sens[0, 1] and sens.sum() == 1
+
+
+def test_default_draws_every_value_on_its_own():
+    """With the default run length the sampled positions of a block are independent single values: over a block
+    whose values above the threshold are one row, the count is binomial over single values (not a multiple of
+    the row length, variance of independent draws)."""
+    ts = 8
+    B = np.zeros((ts, ts))
+    B[3, :] = 1.0
+    s = C.n_samples(0.5, ts)
+    assert s == C.n_runs(0.5, ts) == 32
+    c = np.array([C.block_count(B, 0, 0, ts, 0.5, 0.5, 2, it, 0) for it in range(1500)])
+    f = 1 / ts
+    assert np.any(c % 8 != 0)
+    assert abs(c.mean() - s * f) < 4 * np.sqrt(s * f * (1 - f) / 1500)
+    assert abs(c.var() - s * f * (1 - f)) < 0.2 * s * f * (1 - f)      # runs of 8: eight times this
+    assert C.needed(0.3, 10) == 3 and C.needed(0.1, 10) == 2 and C.needed(0.5, 7) == 4 and C.needed(0.0, 5) == 1
 
 
 def test_runs_are_whole_and_inside_the_block():
     # values encode their own position: a count over a block whose ONLY large values sit in one run of another
     # block, or straddle a run boundary, must never see part of a run
     ts = 8                                   # run length gcd(8, 32) = 8: a run is a whole row of the block
-    assert C.run_length(ts) == 8 and C.run_length(64) == 32 and C.run_length(48) == 16 and C.run_length(7) == 1
+    assert (C.transaction_run(ts) == 8 and C.transaction_run(64) == 32 and C.transaction_run(48) == 16
+            and C.transaction_run(7) == 1)
     A = np.zeros((ts, 2 * ts))
     A[:, :ts] = 1.0                          # block 0 all above, block 1 all below
     for it in range(20):
-        assert C.block_count(A, 0, 0, ts, 0.5, 0.5, 1, it, 0) == C.n_samples(0.5, ts) == 32
-        assert C.block_count(A, 0, 1, ts, 0.5, 0.5, 1, it, 0) == 0
+        assert C.block_count(A, 0, 0, ts, 0.5, 0.5, 1, it, 0, run_len=8) == C.n_samples(0.5, ts, 8) == 32
+        assert C.block_count(A, 0, 1, ts, 0.5, 0.5, 1, it, 0, run_len=8) == 0
     B = np.zeros((ts, ts))
     B[3, :] = 1.0                            # exactly one run above: every draw contributes 0 or 8
-    counts = {C.block_count(B, 0, 0, ts, 0.5, 0.5, 2, it, 0) for it in range(200)}
+    counts = {C.block_count(B, 0, 0, ts, 0.5, 0.5, 2, it, 0, run_len=8) for it in range(200)}
     assert all(c % 8 == 0 for c in counts) and len(counts) > 1
 
 
@@ -42,12 +60,12 @@ def test_runs_are_drawn_uniformly():
     # one run of the block above the threshold: it is hit with probability 1/Cn per draw
     ts = 8
     B = np.zeros((ts, ts))
-    n_c = C.n_runs(1.0, ts)                  # 8 draws per count
+    n_c = C.n_runs(1.0, ts, 8)               # 8 draws per count
     hits = np.zeros(ts)
     for r in range(ts):
         B[:] = 0.0
         B[r, :] = 1.0
-        hits[r] = sum(C.block_count(B, 0, 0, ts, 1.0, 0.5, 5, it, 1) for it in range(300)) / 8
+        hits[r] = sum(C.block_count(B, 0, 0, ts, 1.0, 0.5, 5, it, 1, run_len=8) for it in range(300)) / 8
     expect = 300 * n_c / ts
     assert np.all(np.abs(hits - expect) < 4.5 * np.sqrt(expect))
 
@@ -59,8 +77,8 @@ def test_count_follows_the_binomial_law_over_runs():
     above = rng.random(ts) < 0.4             # whole runs (rows of block 1) above the threshold
     A[above, ts:] = 1.0
     frac = above.mean()
-    n_c = C.n_runs(0.5, ts)
-    c = np.array([C.block_count(A, 0, 1, ts, 0.5, 0.5, 3, it, 0) for it in range(800)]) / 8
+    n_c = C.n_runs(0.5, ts, 8)
+    c = np.array([C.block_count(A, 0, 1, ts, 0.5, 0.5, 3, it, 0, run_len=8) for it in range(800)]) / 8
     assert abs(c.mean() - n_c * frac) < 4 * np.sqrt(n_c * frac * (1 - frac) / 800)
     assert abs(c.var() - n_c * frac * (1 - frac)) < 0.25 * n_c * frac * (1 - frac)
 

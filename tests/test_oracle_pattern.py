@@ -7,6 +7,7 @@ import pytest
 
 from oracle import pattern as P
 from paper_2203_05705_b200 import inputs
+from distributions import max_entropy_K
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -94,7 +95,7 @@ def test_quantise_sums_to_one_and_zero_entries_never_drawn():
     seen = {P.draw(cdf, 7, it, 0)[0] for it in range(3000)}
     assert seen == {1, 3, 5}
     for p, n in [(0.3, 16), (0.5, 16), (0.7, 16), (0.5, 8)]:
-        k = inputs.max_entropy_K(p, n)
+        k = max_entropy_K(p, n)
         q = P.quantised_probabilities(P.quantise_K(k))
         assert sum(q) == 1 << 32
         assert max(abs(qi / 2**32 - ki) for qi, ki in zip(q, k)) < 2**-31
@@ -114,7 +115,7 @@ def test_exact_per_unit_drop_probability_equals_global_rate():
     """Eq. 2-3 as an exact identity in rationals: for every unit i,
     sum_dp k_dp * #{b : unit dropped}/dp == sum_dp k_dp (dp-1)/dp, for any N."""
     for N in (10, 37):
-        K = inputs.max_entropy_K(0.5, 8)
+        K = max_entropy_K(0.5, 8)
         q = P.quantised_probabilities(P.quantise_K(K))
         pg = sum(Fraction(qi, 1 << 32) * Fraction(dp - 1, dp) for dp, qi in enumerate(q, 1))
         for i in range(N):
@@ -128,7 +129,7 @@ def test_exact_per_unit_drop_probability_equals_global_rate():
 def test_monte_carlo_matches_bernoulli_rate():
     """Sampler end to end: empirical per-neuron drop rate -> target p; dp ~ K; b | dp uniform."""
     p, n_dp, N, S = 0.5, 8, 64, 20000
-    K = inputs.max_entropy_K(p, n_dp)
+    K = max_entropy_K(p, n_dp)
     cdf = P.quantise_K(K)
     drops = np.zeros(N)
     hist = np.zeros(n_dp + 1)
@@ -150,7 +151,7 @@ def test_monte_carlo_matches_bernoulli_rate():
 
 
 def test_draw_is_a_pure_function_of_the_counter():
-    cdf = P.quantise_K(inputs.max_entropy_K(0.3, 16))
+    cdf = P.quantise_K(max_entropy_K(0.3, 16))
     a = [P.draw(cdf, 5, it, 2) for it in range(50)]
     b = [P.draw(cdf, 5, it, 2) for it in reversed(range(50))][::-1]
     assert a == b

@@ -12,6 +12,7 @@ import pytest
 from oracle import search as OS
 from oracle import pattern as OP
 from paper_2203_05705_b200 import inputs
+from distributions import max_entropy_K
 
 
 def test_gradient_matches_central_differences():
@@ -47,7 +48,7 @@ def test_small_lambda_tends_to_the_maximum_entropy_distribution():
     errs = []
     for lam in (1e-1, 1e-2, 1e-3):
         K, _ = OS.search_K(0.5, 16, lam=lam, tol=1e-18)
-        ref = np.asarray(inputs.max_entropy_K(0.5, 16))
+        ref = np.asarray(max_entropy_K(0.5, 16))
         errs.append(np.abs(K - ref).max())
         assert abs(float(K @ OS.p_u(16)) - 0.5) <= 1.5 * lam     # |e| = lam |beta| / 2, |beta| < 3 here
     assert errs[0] > errs[1] > errs[2] and errs[2] <= 2e-3

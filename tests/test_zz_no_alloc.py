@@ -1,11 +1,14 @@
 """ard_bwd_data_static_scratch -- the entry point for callers that may not allocate device memory
 (frozen memory plan, host application owns the allocator, no device-wide sync allowed) -- must give
-what ard_bwd_data gives.  Collected last so that a failure here cannot hide another test's result.
+what the definition gives (the oracle's masked fp64 product) and what ard_bwd_data gives.  Collected last so that
+a failure here cannot hide another test's result.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import gemm as OG
+from oracle import pattern as OP
 from paper_2203_05705_b200 import ard, inputs
 
 pytestmark = pytest.mark.gpu
@@ -20,27 +23,36 @@ def _rel(a, b):
 
 
 @pytest.mark.parametrize("dtype", [ard.ARD_BF16, ard.ARD_F32])
-def test_two_calls_in_a_row_match_the_allocating_entry_point(dtype):
+@pytest.mark.parametrize("pads", [(0, 0), (8, 16)])
+def test_calls_in_a_row_match_the_definition_and_the_allocating_entry_point(dtype, pads):
     B, K, N = 200, 264, 520
+    lddy, lddx = N + pads[0], K + pads[1]           # also with rows that do not follow one another in memory
     td = torch.bfloat16 if dtype == ard.ARD_BF16 else torch.float32
     tol = TOL_BF16 if dtype == ard.ARD_BF16 else TOL_F32
     rng = np.random.default_rng(11)
-    W = torch.from_numpy(inputs.bf16_round((rng.standard_normal((N, K)) * 0.05).astype(np.float32))).to(td).cuda()
+    Wh = inputs.bf16_round((rng.standard_normal((N, K)) * 0.05).astype(np.float32))       # neuron-major
+    W = torch.from_numpy(Wh).to(td).cuda()
     ctx = ard.ard_create(0, 2 * B * N + 4096)
     pat = ard.ard_pattern_create(ctx, ard.ARD_ROW, K, N, 0)
     try:
-        # two different patterns and gradients back to back: the second call starts with the first
-        # call's data still in the shared scratch array
-        for call, (dp, b) in enumerate([(3, 2), (1, 1), (5, 5)]):
-            dY = torch.from_numpy(inputs.bf16_round(rng.standard_normal((B, N)).astype(np.float32))).to(td).cuda()
+        # different patterns and gradients back to back: every call after the first starts with the previous
+        # call's data still in the shared scratch array; (300, 7) keeps two neurons, (520, 520) only the last one
+        for call, (dp, b) in enumerate([(3, 2), (1, 1), (5, 5), (300, 7), (520, 520)]):
+            dYh = inputs.bf16_round(rng.standard_normal((B, N)).astype(np.float32))
+            dY = torch.full((B, lddy), float("nan"), dtype=td, device="cuda")
+            dY[:, :N] = torch.from_numpy(dYh).to(td)
             ard.ard_pattern_set(ctx, pat, dp, b)
-            ref = torch.full((B, K), float("nan"), dtype=td, device="cuda")
-            out = torch.full((B, K), float("nan"), dtype=td, device="cuda")
-            ard.ard_bwd_data(ctx, pat, dtype, B, K, N, 2.0, dY, N, 0, W, K, ref, K)
-            ard.ard_bwd_data_static_scratch(ctx, pat, dtype, B, K, N, 2.0, dY, N, W, K, out, K)
+            ref = torch.full((B, lddx), float("nan"), dtype=td, device="cuda")
+            out = torch.full((B, lddx), float("nan"), dtype=td, device="cuda")
+            ard.ard_bwd_data(ctx, pat, dtype, B, K, N, 2.0, dY, lddy, 0, W, K, ref, lddx)
+            ard.ard_bwd_data_static_scratch(ctx, pat, dtype, B, K, N, 2.0, dY, lddy, W, K, out, lddx)
             torch.cuda.synchronize()
-            assert bool(torch.isfinite(out).all()), (call, dp, b)
-            assert _rel(out, ref) <= tol, (call, dp, b, _rel(out, ref))
+            assert bool(torch.isfinite(out[:, :K]).all()), (call, dp, b)
+            assert bool(torch.isnan(out[:, K:]).all()), (call, dp, b)           # nothing written beyond the K columns
+            want = OG.bwd_data(dYh, Wh.T, OP.row_mask(N, dp, b), 2.0)            # the definition: masked fp64 product
+            err = OG.rel_fro(out[:, :K].double().cpu().numpy(), want)
+            assert err <= tol, (call, dp, b, err)
+            assert _rel(out[:, :K], ref[:, :K]) <= tol, (call, dp, b, _rel(out[:, :K], ref[:, :K]))
         assert ard.ard_last_device_status(ctx) == 0
     finally:
         torch.cuda.synchronize()
