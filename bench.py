@@ -33,8 +33,9 @@ sys.path.insert(0, ROOT)
 from paper_2203_05705_b200 import inputs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of ard_gemm_tc_kernel, averaged over the three
-# GEMMs of one dense (dp = 1) step of this workload, from the ncu capture summarised under profiles/.
-DRAM_TRAFFIC_PER_LAUNCH = 581.0e6   # bytes (fwd 679.5 MB, bwd-data 674.4 MB, bwd-weight 390.3 MB)
+# GEMMs of one step of the 8192 x 8192 layer at batch 4096, per period dp, from the ncu captures summarised
+# under profiles/ (dp = 1: fwd 679.5 MB, bwd-data 674.4 MB, bwd-weight 390.3 MB).
+DRAM_TRAFFIC_BY_DP = {"row": {1: 581.0e6}, "tile": {}}
 
 METRIC = "layer fwd+bwd kept TFLOP/s (row pattern, p=0.5)"
 UNIT = "TFLOP/s"
@@ -52,14 +53,36 @@ WORKLOADS = {
     "mlp8192_step": dict(config=5, dims=[8192, 8192, 8192, 1024], B=4096, kind="mlp_step", p=0.5, n_dp=16),
     # a convolution layer as the product of its im2col input matrix with the filters, rows of the input matrix
     # dropped by predicted sensitivity (Sec. 5.1, 5.2.1): 3x3 filters, 256 -> 512 channels, 32768 output positions
-    "conv_rows": dict(config=5, M=32768, K=2304, N=512, kind="conv_rows", region_rows=8, k_frac=0.05, t_frac=0.3,
-                      threshold=0.5, m_prob=0.2, n_prob=0.8),
+    # run_len = 32: the sampled values of the sensitivity prediction are taken in runs of 32 neighbours, a departure
+    # from Sec. 5.1 (which samples single values: --conv-run-len 1) chosen for its memory traffic
+    "conv_rows": dict(config=5, M=32768, K=2304, N=512, kind="conv_rows", region_rows=8, k_frac=0.05, run_len=32,
+                      t_frac=0.3, threshold=0.5, m_prob=0.2, n_prob=0.8),
     # the same layer with blocks of the input matrix as the dropout granularity (Sec. 5.2.2)
-    "conv_blocks": dict(config=5, M=32768, K=2304, N=512, kind="conv_blocks", ts=128, k_frac=0.05, t_frac=0.3,
-                        threshold=0.5, cap=6, m_prob=0.2, n_prob=0.8),
+    "conv_blocks": dict(config=5, M=32768, K=2304, N=512, kind="conv_blocks", ts=128, k_frac=0.05, run_len=32,
+                        t_frac=0.3, threshold=0.5, cap=6, m_prob=0.2, n_prob=0.8),
     # LSTM layer (config 4): a step is one sequence, forward + BPTT, one fresh pattern per sequence
     "lstm1024": dict(config=4, T=35, B=64, I=1024, H=1024, kind="lstm", p=0.5, n_dp=16),
 }
+
+def max_entropy_K(p, n_dp):
+    """K of every benchmark workload: over the periods dp = 1..n_dp, the distribution of greatest entropy whose
+    global dropout rate sum_i k_i (i-1)/i (Eq. 2-3) is p, i.e. k_i proportional to exp(beta (i-1)/i) with beta by
+    bisection.  It stands in for the output of the search of Sec. 3.3 (whose constants are not printed): K is an
+    input of the hot path, this is the workload recipe's choice of it."""
+    pu = np.array([(i - 1) / i for i in range(1, n_dp + 1)])
+    if n_dp < 2 or not (0.0 < p < pu[-1]):
+        raise ValueError("need n_dp >= 2 and 0 < p < (n_dp-1)/n_dp")
+    lo, hi = -200.0, 200.0
+    for _ in range(200):
+        beta = 0.5 * (lo + hi)
+        w = np.exp(beta * (pu - pu[-1])) if beta > 0 else np.exp(beta * pu)
+        k = w / w.sum()
+        if float(k @ pu) < p:
+            lo = beta
+        else:
+            hi = beta
+    return k / k.sum()
+
 
 # Measured peaks of this pool's B200s (driver-written file), else the documented fallback.
 def load_peaks():
@@ -215,7 +238,7 @@ def run_reference(args, wl):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, **{k: wl[k] for k in ("B", "K", "N", "kind", "p", "n_dp")}},
+        "config": layer_config(args, wl, 1),
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -239,7 +262,7 @@ def run_lstm(args, wl):
     X, dH = hX.cuda(), hdH.cuda()
     hH = torch.empty((T, B, H), dtype=bf).pin_memory()
     ctx = ard.ard_create(0, 2 * T * B * 4 * H + 4096)
-    ard.ard_set_distribution(ctx, 0, inputs.max_entropy_K(p, n_dp))
+    ard.ard_set_distribution(ctx, 0, max_entropy_K(p, n_dp))
     pat = ard.ard_pattern_create(ctx, ard.ARD_ROW, I + H, H, 0)
     layer = LstmLayer(ctx, pat, T, B, I, H, W)
     alpha = 1.0 / (1.0 - p)
@@ -375,7 +398,7 @@ def run_mlp_step(args, wl):
     alpha = 1.0 / (1.0 - p)
     ctx = ard.ard_create(0, 2 * B * max(dims) + 4096)
     ard.ard_set_compact_reuse(ctx, 1)
-    Kd = inputs.max_entropy_K(p, n_dp)
+    Kd = max_entropy_K(p, n_dp)
     ard.ard_set_distribution(ctx, 0, Kd)
     g = torch.Generator(device="cuda").manual_seed(inputs.BASE_SEED)
     hX = torch.rand((B, dims[0]), generator=torch.Generator().manual_seed(1)).to(bf).pin_memory()
@@ -602,7 +625,7 @@ def run_conv_rows(args, wl):
         if dense:
             ard.ard_rows_set_probability(ctx, rows, 0.0)
         else:
-            ard.ard_sensitivity_predict(ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["t_frac"], wl["threshold"],
+            ard.ard_sensitivity_predict(ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["run_len"], wl["t_frac"], wl["threshold"],
                                         wl["m_prob"], wl["n_prob"], inputs.BASE_SEED, it, 0)
         ard.ard_rows_sample(ctx, rows, inputs.BASE_SEED, it, 0)
         if gathered:
@@ -627,7 +650,7 @@ def run_conv_rows(args, wl):
         if host:
             A.copy_(hA, non_blocking=True)
             dY.copy_(hdY, non_blocking=True)
-        ard.ard_sensitivity_predict(ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["t_frac"], wl["threshold"],
+        ard.ard_sensitivity_predict(ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["run_len"], wl["t_frac"], wl["threshold"],
                                     wl["m_prob"], wl["n_prob"], inputs.BASE_SEED, it, 0)
         ard.ard_rows_sample(ctx, rows, inputs.BASE_SEED, it, 0)
         ard.ard_rows_products(ctx, rows, ard.ARD_BF16, M, K, N, 1.0, A, K, W, K, dY, N, Ak, K, dYk, N, Y, N, dA, K, dW, K)
@@ -655,7 +678,7 @@ def run_conv_rows(args, wl):
     status = ard.ard_last_device_status(ctx)
     kept_rows = []
     for i in range(steps):
-        ard.ard_sensitivity_predict(ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["t_frac"], wl["threshold"],
+        ard.ard_sensitivity_predict(ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["run_len"], wl["t_frac"], wl["threshold"],
                                     wl["m_prob"], wl["n_prob"], inputs.BASE_SEED, warm + i, 0)
         ard.ard_rows_sample(ctx, rows, inputs.BASE_SEED, warm + i, 0)
         kept_rows.append(ard.ard_rows_to_host(rows, 0)[0])
@@ -671,7 +694,10 @@ def run_conv_rows(args, wl):
         # per stage, serialised (one stage per timed loop)
         stage = {}
         stage["sensitivity_predict"] = lambda it: ard.ard_sensitivity_predict(
-            ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["t_frac"], wl["threshold"], wl["m_prob"], wl["n_prob"],
+            ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], wl["run_len"], wl["t_frac"], wl["threshold"], wl["m_prob"], wl["n_prob"],
+            inputs.BASE_SEED, 1, 0)
+        stage["sensitivity_predict_single_values"] = lambda it: ard.ard_sensitivity_predict(
+            ctx, rows, ard.ARD_BF16, A, K, K, wl["k_frac"], 1, wl["t_frac"], wl["threshold"], wl["m_prob"], wl["n_prob"],
             inputs.BASE_SEED, 1, 0)
         stage["rows_sample"] = lambda it: ard.ard_rows_sample(ctx, rows, inputs.BASE_SEED, 1, 0)
         stage["gather_A"] = lambda it: ard.ard_rows_gather(ctx, rows, M, K, A, K, Ak, K)
@@ -719,8 +745,10 @@ def run_conv_rows(args, wl):
         "metric": "convolution layer (im2col product) fwd+bwd kept TFLOP/s, rows dropped by predicted sensitivity",
         "value": value, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms / steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, **{k: wl[k] for k in ("M", "K", "N", "region_rows", "k_frac", "t_frac",
-                                                                       "threshold", "m_prob", "n_prob")},
+        "config": {"workload": args.workload, **{k: wl[k] for k in ("M", "K", "N", "region_rows", "k_frac", "run_len",
+                                                                       "t_frac", "threshold", "m_prob", "n_prob")},
+                   "sampling": ("single values, as Sec. 5.1 states" if wl["run_len"] == 1 else
+                                "runs of %d neighbouring values: a departure from Sec. 5.1" % wl["run_len"]),
                    "l2": "working set %.0f MB per step" % ((2 * M * K + 2 * M * N + 2 * N * K) * 2 / 1e6)},
         "dense_equiv_tflops": 3 * 2.0 * M * K * N * steps / (ms * 1e-3) / 1e12, "clocks": clk, "e2e": e2e,
         "gpu_launches": int(launches),
@@ -761,7 +789,7 @@ def run_conv_blocks(args, wl):
     blocks = ard.ard_blocks_create(ctx, M, K, ts)
 
     def sample(it):
-        ard.ard_blocks_predict(ctx, blocks, ard.ARD_BF16, A, K, wl["k_frac"], wl["t_frac"], wl["threshold"], wl["cap"],
+        ard.ard_blocks_predict(ctx, blocks, ard.ARD_BF16, A, K, wl["k_frac"], wl["run_len"], wl["t_frac"], wl["threshold"], wl["cap"],
                                inputs.BASE_SEED, it, 0)
         ard.ard_blocks_sample(ctx, blocks, wl["m_prob"], wl["n_prob"], inputs.BASE_SEED, it, 0)
 
@@ -851,8 +879,10 @@ def run_conv_blocks(args, wl):
         "metric": "convolution layer (im2col product) fwd+bwd kept TFLOP/s, blocks dropped by predicted sensitivity",
         "value": value, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warm, "ms_per_step": ms / steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, **{k: wl[k] for k in ("M", "K", "N", "ts", "k_frac", "t_frac", "threshold",
-                                                                       "cap", "m_prob", "n_prob")},
+        "config": {"workload": args.workload, **{k: wl[k] for k in ("M", "K", "N", "ts", "k_frac", "run_len", "t_frac",
+                                                                       "threshold", "cap", "m_prob", "n_prob")},
+                   "sampling": ("single values, as Sec. 5.1 states" if wl["run_len"] == 1 else
+                                "runs of %d neighbouring values: a departure from Sec. 5.1" % wl["run_len"]),
                    "l2": "working set %.0f MB per step" % ((2 * M * K + 2 * M * N + 2 * N * K) * 2 / 1e6)},
         "dense_equiv_tflops": 3 * 2.0 * M * K * N * steps / (ms * 1e-3) / 1e12, "clocks": clk, "e2e": e2e,
         "gpu_launches": int(launches),
@@ -867,6 +897,289 @@ def run_conv_blocks(args, wl):
     ard.ard_destroy(ctx)
 
 
+RATES = (0.3, 0.4, 0.5, 0.6, 0.7)       # the dropout rates of the large-layer sweep
+REPEATS = 5                              # timed regions per figure; the median is reported
+
+
+def layer_config(args, wl, world):
+    """The `config` object of a single-layer line; both arms (this library, the CPU reference) print the same."""
+    return {"workload": args.workload, "B": wl["B"], "K": wl["K"], "N": wl["N"], "kind": wl["kind"], "ts": wl["ts"],
+            "p": wl["p"], "n_dp": wl["n_dp"], "l2": "inputs larger than L2 (X, W, dY and outputs: ~0.5 GB per step)",
+            "replicas": world}
+
+
+class LayerBench:
+    """One layer (X, W, dY resident on the device), one context, one pattern object; every timing helper of the
+    single-layer workloads.  A step = draw a pattern on the device, forward (full-width output, dropped columns
+    written as zero), backward-data and backward-weight from the full-width dY (compacted once per step)."""
+
+    def __init__(self, torch, ard, args, wl, dev, rank, world, barrier, tensors=None):
+        self.torch, self.ard, self.args, self.wl = torch, ard, args, wl
+        self.rank, self.world, self.barrier = rank, world, barrier
+        B, K, N = wl["B"], wl["K"], wl["N"]
+        self.B, self.K, self.N, self.ts = B, K, N, wl["ts"]
+        self.kind = ard.ARD_ROW if wl["kind"] == "row" else ard.ARD_TILE
+        self.units = N if self.kind == ard.ARD_ROW else (K // wl["ts"]) * (N // wl["ts"])
+        bf = torch.bfloat16
+        if tensors is None:
+            d = inputs.dense_layer(wl["config"], B, K, N, 1.0 / 90.0 if wl["config"] == 5 else 1.0 / 64.0)
+            hX = torch.from_numpy(d["X"]).to(bf).pin_memory()
+            hdY = torch.from_numpy(d["dY"]).to(bf).pin_memory()
+            tensors = dict(host=d, hX=hX, hdY=hdY, X=hX.cuda(), dY=hdY.cuda(),
+                           W=torch.from_numpy(np.ascontiguousarray(d["W"].T)).to(bf).cuda(),     # neuron-major [N][K]
+                           Y=torch.empty((B, N), dtype=bf, device="cuda"), dX=torch.empty((B, K), dtype=bf, device="cuda"),
+                           dW=torch.zeros((N, K), dtype=bf, device="cuda"), hY=torch.empty((B, N), dtype=bf).pin_memory())
+        self.t = tensors
+        self.ctx = ard.ard_create(dev, 2 * B * N + 4096)
+        ard.ard_set_compact_reuse(self.ctx, 1)   # dY is not written between bwd-data and bwd-weight of a step
+        self.pat = ard.ard_pattern_create(self.ctx, self.kind, K, N, wl["ts"])
+        self.dist_ids, self.khat = {}, {}
+        for i, pp in enumerate(RATES):
+            Kd = max_entropy_K(pp, wl["n_dp"])
+            ard.ard_set_distribution(self.ctx, i, Kd)
+            cdf = np.asarray(ard.ard_quantise_distribution(Kd), dtype=np.float64)
+            self.dist_ids[pp] = i
+            self.khat[pp] = np.diff(np.concatenate([[0.0], cdf])) / 2.0 ** 32      # the distribution the sampler realises
+        self.seed = inputs.BASE_SEED
+        self.cs = torch.cuda.current_stream().cuda_stream
+        self.ptr = {k: tensors[k].data_ptr() for k in ("X", "W", "Y", "dY", "dX", "dW")}
+
+    def close(self):
+        self.ard.ard_pattern_destroy(self.pat)
+        self.ard.ard_destroy(self.ctx)
+
+    # ---- the calls of a step -----------------------------------------------------------------------
+    def gemms(self, alpha, ev=None, ptr=None, zero_fill=0):
+        ard, B, K, N, ctx, pat, cs = self.ard, self.B, self.K, self.N, self.ctx, self.pat, self.cs
+        q = ptr or self.ptr
+        if ev is not None:
+            ev[0].record()
+        ard.ard_fwd(ctx, pat, ard.ARD_BF16, B, K, N, alpha, q["X"], K, q["W"], K, q["Y"], N, ard.ARD_OUT_SCATTER_ZEROFILL, cs)
+        if ev is not None:
+            ev[1].record()
+        ard.ard_bwd_data(ctx, pat, ard.ARD_BF16, B, K, N, alpha, q["dY"], N, 0, q["W"], K, q["dX"], K, cs)
+        if ev is not None:
+            ev[2].record()
+        ard.ard_bwd_weight(ctx, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, alpha, q["X"], K, q["dY"], N, 0, q["dW"], K,
+                           zero_fill, cs)
+        if ev is not None:
+            ev[3].record()
+
+    def step(self, pp, it, ev=None, ptr=None):
+        self.ard.ard_sample_pattern(self.ctx, self.pat, self.dist_ids[pp], self.seed, it, self.rank, self.cs)
+        self.gemms(1.0 / (1.0 - pp), ev, ptr)
+
+    def patterns_of(self, pp, its):
+        """(dp, b, kept units) of the given iterations, read back from the device sampler outside any timed region."""
+        out = []
+        for it in its:
+            self.ard.ard_sample_pattern(self.ctx, self.pat, self.dist_ids[pp], self.seed, it, self.rank)
+            dp_, b_, nk, _ = self.ard.ard_pattern_to_host(self.pat, 0)
+            out.append((dp_, b_, nk))
+        return out
+
+    def flops_per_unit(self):
+        """FLOPs of ONE product per kept unit (a kept neuron, or a kept tile)."""
+        return 2.0 * self.B * self.K if self.kind == self.ard.ARD_ROW else 2.0 * self.B * self.ts ** 2
+
+    # ---- timed regions -----------------------------------------------------------------------------
+    def timed_steps(self, pp, its, per_kernel=False, ptrs=None):
+        """Times exactly len(its) steps between two barriers.  Returns (ms, per-kernel ms [steps][3] or None, wall)."""
+        torch = self.torch
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in its] if per_kernel else None
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.barrier()
+        w0 = time.time()
+        e0.record()
+        for i, it in enumerate(its):
+            self.step(pp, it, evs[i] if per_kernel else None, None if ptrs is None else ptrs[i % len(ptrs)])
+        e1.record()
+        self.barrier()
+        w1 = time.time()
+        per = None
+        if per_kernel:
+            per = [[evs[i][j].elapsed_time(evs[i][j + 1]) for j in range(3)] for i in range(len(its))]
+        return e0.elapsed_time(e1), per, (w0, w1)
+
+    def repeated(self, pp, first_it, per_kernel=False):
+        """Warm-up, then REPEATS timed regions over the SAME iterations (same patterns), so that the spread is the
+        machine's and not the draw's."""
+        a = self.args
+        for w in range(a.warmup):
+            self.step(pp, first_it + w)
+        its = list(range(first_it + a.warmup, first_it + a.warmup + a.steps))
+        runs = [self.timed_steps(pp, its, per_kernel) for _ in range(REPEATS)]
+        return its, runs
+
+    def time_fn(self, fn, n):
+        torch = self.torch
+        for _ in range(self.args.warmup):
+            fn()
+        out = []
+        for _ in range(REPEATS):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            self.barrier()
+            e0.record()
+            for _ in range(n):
+                fn()
+            e1.record()
+            self.barrier()
+            out.append(e0.elapsed_time(e1) / n)
+        return out
+
+    def dense_baselines(self):
+        """ms per dense step (median of REPEATS regions): this library's kernels at dp = 1, and torch.matmul."""
+        torch, t = self.torch, self.t
+        self.ard.ard_pattern_set(self.ctx, self.pat, 1, 1)
+        n = max(5, self.args.steps // 4)
+        own = self.time_fn(lambda: self.gemms(1.0), n)
+        X, dY, W = t["X"], t["dY"], t["W"]
+        Wt = W.t()
+
+        def lib():
+            torch.matmul(X, Wt); torch.matmul(dY, W); torch.matmul(dY.t(), X)
+
+        lib_ms = self.time_fn(lib, n)
+        return {"own_kernels_dp1": statistics.median(own), "torch_matmul": statistics.median(lib_ms),
+                "own_kernels_dp1_all": own, "torch_matmul_all": lib_ms}
+
+    def per_dp_table(self, peak_burst):
+        """Every (dp, b) of the distribution's support, forced with ard_pattern_set: per product and for the whole
+        step the median over b and REPEATS of the CUDA-event time.  bwd_data includes the compaction of the
+        full-width dY (once per step); bwd_weight reuses it; bwd_weight_zero_fill also writes the dropped rows."""
+        torch, ard = self.torch, self.ard
+        n_dp = self.wl["n_dp"]
+        names = ["sampler", "fwd", "bwd_data", "bwd_weight", "bwd_weight_zero_fill"]
+        table, step_by_dp, units_by_dp = {}, {}, {}
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+        for dp in range(1, n_dp + 1):
+            ms = {nm: [] for nm in names}
+            steps, kept = [], []
+            for b in range(1, dp + 1):
+                ard.ard_pattern_set(self.ctx, self.pat, dp, b, self.cs)
+                kept.append(self.ard.ard_pattern_to_host(self.pat, 0)[2])
+                for rep in range(REPEATS + 1):                    # the first pass warms up
+                    ev[0].record()
+                    ard.ard_pattern_set(self.ctx, self.pat, dp, b, self.cs)      # the sampler kernel, pattern forced
+                    self.gemms(2.0, ev[1:5])
+                    q = self.ptr
+                    ard.ard_bwd_weight(self.ctx, self.pat, ard.ARD_BF16, ard.ARD_BF16, self.B, self.K, self.N, 2.0, q["X"],
+                                       self.K, q["dY"], self.N, 0, q["dW"], self.K, 1, self.cs)
+                    ev[5].record()
+                    torch.cuda.synchronize()
+                    if rep == 0:
+                        continue
+                    for j, nm in enumerate(names):
+                        ms[nm].append(ev[j].elapsed_time(ev[j + 1]))
+                    steps.append(ev[0].elapsed_time(ev[4]))
+            fl = self.flops_per_unit() * float(np.mean(kept))
+            row = {"kept_units_mean": float(np.mean(kept)), "step_ms": statistics.median(steps)}
+            for nm in names:
+                m = statistics.median(ms[nm])
+                row[nm + "_ms"] = m
+                if nm != "sampler":
+                    row[nm + "_tflops"] = fl / (m * 1e-3) / 1e12
+                    row[nm + "_frac_of_burst"] = row[nm + "_tflops"] / peak_burst
+            table[str(dp)] = row
+            step_by_dp[dp] = float(np.mean(steps))            # mean over b and repeats: what an expectation needs
+            units_by_dp[dp] = float(np.mean(kept))
+        return table, step_by_dp, units_by_dp
+
+    def expectations(self, step_by_dp, units_by_dp, dense_ms):
+        """What the sampled figures estimate, without the sampling: E[step time] = sum_dp k^_dp t(dp) under the
+        quantised K of each rate, against the dense step; the ideal is 1/(1-p)."""
+        out = {}
+        for pp in RATES:
+            k = self.khat[pp]
+            t = sum(k[dp - 1] * step_by_dp[dp] for dp in step_by_dp)
+            u = sum(k[dp - 1] * units_by_dp[dp] for dp in step_by_dp)
+            out[str(pp)] = {"expected_ms_per_step": t, "expected_speedup": dense_ms / t, "ideal_speedup": 1.0 / (1.0 - pp),
+                            "fraction_of_ideal": dense_ms / t * (1.0 - pp),
+                            "expected_kept_tflops": 3 * self.flops_per_unit() * u / (t * 1e-3) / 1e12,
+                            "expected_kept_fraction": u / self.units}
+        return out
+
+    def headline(self, peaks):
+        """The timed regions the line's `value` comes from, and the roofline of the GEMM kernel inside them."""
+        a, wl = self.args, self.wl
+        p = wl["p"]
+        launches0 = self.ard.ard_launch_count(self.ctx)
+        its, runs = self.repeated(p, 0, per_kernel=True)
+        launches = (self.ard.ard_launch_count(self.ctx) - launches0) * a.steps // (a.steps * REPEATS + a.warmup)
+        status = self.ard.ard_last_device_status(self.ctx)
+        pats = self.patterns_of(p, its)
+        kept = [3 * self.flops_per_unit() * nk for (_, _, nk) in pats]
+        dense_flops = 3 * 2.0 * self.B * self.K * self.N * a.steps
+        ms_all = [r[0] for r in runs]
+        if self.world > 1:
+            # whole job: slowest rank per region, work of all ranks
+            agg = [aggregate_over_ranks(m, sum(kept), dense_flops, "cuda") for m in ms_all]
+            ms_all = [x[0] for x in agg]
+            kept_total, dense_total = agg[0][1], agg[0][2]
+        else:
+            kept_total, dense_total = sum(kept), dense_flops
+        values = [kept_total / (m * 1e-3) / 1e12 for m in ms_all]
+        order = sorted(range(REPEATS), key=lambda i: ms_all[i])
+        mid = order[REPEATS // 2]
+        per = np.array(runs[mid][1])                     # [steps][3] ms of the median region
+        gemm_ms = float(per.sum())
+        achieved = sum(kept) / (gemm_ms * 1e-3) / 1e12
+        per_op = {nm: {"ms_avg": float(per[:, j].mean()), "tflops": sum(kept) / 3.0 / (float(per[:, j].sum()) * 1e-3) / 1e12}
+                  for j, nm in enumerate(["fwd", "bwd_data", "bwd_weight"])}
+        wall = (runs[0][2][0], runs[-1][2][1])
+        return dict(its=its, pats=pats, ms=ms_all[mid], ms_all=ms_all, values=values, value=values[mid],
+                    dense_equiv=dense_total / (ms_all[mid] * 1e-3) / 1e12, launches=int(launches), status=int(status),
+                    achieved=achieved, per_op=per_op, wall=wall, kept=kept)
+
+
+def traffic_per_launch(lb, pats):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of ard_gemm_tc_kernel for the patterns of the timed
+    region: the per-period figures of the ncu captures summarised under profiles/ (average of the three products),
+    weighted by how often each period was drawn; None for a period that was not captured."""
+    tab = DRAM_TRAFFIC_BY_DP.get(lb.wl["kind"], {})
+    tot, n = 0.0, 0
+    for (dp, _, _) in pats:
+        if dp not in tab:
+            return None
+        tot += tab[dp]
+        n += 1
+    return tot / max(n, 1)
+
+
+def roofline_of(h, peaks, clk, lb):
+    # The timed regions are short (tens of ms each): if the SM clock stayed near its maximum the kernels ran in
+    # the burst regime and are held against the burst cuBLAS figure, otherwise against the sustained one.
+    burst = clk["sm_mhz"] is None or clk["sm_max_mhz"] is None or clk["sm_mhz"] >= 0.9 * clk["sm_max_mhz"]
+    peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+    a = h["achieved"]
+    return {"bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
+            "traffic": traffic_per_launch(lb, h["pats"]),
+            "traffic_unit": "bytes per launch, mean over the launches of the timed region (ncu captures per period)",
+            "peak_source": peaks["source"] + (" burst" if burst else " sustained") + " cuBLAS bf16 8192^3",
+            "frac_of_burst": a / peaks["bf16_tflops"], "frac_of_sustained": a / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_2250": a / 2250.0, "kernel": "ard_gemm_tc_kernel", "launches": 3 * lb.args.steps,
+            "per_op": h["per_op"]}
+
+
+def sweep_block(lb, peaks, dense):
+    """Per-period table, expectations under every rate of the sweep, and the sampled figures beside them."""
+    best_dense = min(dense["own_kernels_dp1"], dense["torch_matmul"])
+    table, step_by_dp, units_by_dp = lb.per_dp_table(peaks["bf16_tflops"])
+    exp = lb.expectations(step_by_dp, units_by_dp, best_dense)
+    sampled = {}
+    for pp in (0.3, 0.5, 0.7):
+        its, runs = lb.repeated(pp, 10000 + int(pp * 100) * 1000)
+        ms = statistics.median(r[0] for r in runs) / lb.args.steps
+        pats = lb.patterns_of(pp, its)
+        sampled[str(pp)] = {"ms_per_step": ms, "speedup_vs_dense": best_dense / ms,
+                            "kept_fraction": float(np.mean([nk / lb.units for (_, _, nk) in pats]))}
+    return {"per_dp": table, "expected": exp, "sampled": sampled,
+            "note": "per_dp: median over every offset b and %d repeats, pattern forced with ard_pattern_set; expected: "
+                    "sum over dp of k^_dp x mean step time, k^ = the quantised distribution; sampled: %d device-drawn "
+                    "steps per rate (a bimodal K makes these noisy; the expectations are the figures to read)"
+                    % (REPEATS, lb.args.steps)}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -876,8 +1189,14 @@ def main():
     ap.add_argument("--workload", default="mlp8192_row", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true", help="headline region only (for profiler captures)")
+    ap.add_argument("--conv-run-len", type=int, default=0,
+                    help="conv workloads: values per sampled run of the sensitivity prediction (1 = single values, "
+                         "the statement of Sec. 5.1; default: the workload's 32)")
+    ap.add_argument("--force-dp", type=int, default=0, help="profiler captures: time steps of this period only (b = 1)")
     args = ap.parse_args()
-    wl = WORKLOADS[args.workload]
+    wl = dict(WORKLOADS[args.workload])
+    if args.conv_run_len and "run_len" in wl:
+        wl["run_len"] = args.conv_run_len
     if args.impl == "reference":
         return run_reference(args, wl)
     if wl["kind"] == "lstm":
@@ -906,184 +1225,93 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    B, K, N, p, n_dp = wl["B"], wl["K"], wl["N"], wl["p"], wl["n_dp"]
-    kind = ard.ARD_ROW if wl["kind"] == "row" else ard.ARD_TILE
-    units = N if kind == ard.ARD_ROW else (K // wl["ts"]) * (N // wl["ts"])
-    d = inputs.dense_layer(wl["config"], B, K, N, 1.0 / 90.0 if wl["config"] == 5 else 1.0 / 64.0)
-    bf = torch.bfloat16
-    hX = torch.from_numpy(d["X"]).to(bf).pin_memory()
-    hdY = torch.from_numpy(d["dY"]).to(bf).pin_memory()
-    X = hX.cuda()
-    dY = hdY.cuda()
-    W = torch.from_numpy(np.ascontiguousarray(d["W"].T)).to(bf).cuda()     # neuron-major [N][K]
-    Y = torch.empty((B, N), dtype=bf, device="cuda")
-    dX = torch.empty((B, K), dtype=bf, device="cuda")
-    dW = torch.zeros((N, K), dtype=bf, device="cuda")
-    hY = torch.empty((B, N), dtype=bf).pin_memory()
-
-    ctx = ard.ard_create(local, 2 * B * N + 4096)
-    ard.ard_set_compact_reuse(ctx, 1)   # dY is not written between bwd-data and bwd-weight of a step
-    pat = ard.ard_pattern_create(ctx, kind, K, N, wl["ts"])
-    dist_ids = {}
-    for i, pp in enumerate((0.3, 0.5, 0.7)):
-        ard.ard_set_distribution(ctx, i, inputs.max_entropy_K(pp, n_dp))
-        dist_ids[pp] = i
-    seed = inputs.BASE_SEED
-
-    # raw handles, looked up once: the per-call cost of the binding matters for the small workloads
-    cs = torch.cuda.current_stream().cuda_stream
-    pX, pW, pY, pdY, pdX, pdW = (t.data_ptr() for t in (X, W, Y, dY, dX, dW))
-
-    def gemms(alpha, ev=None):
-        if ev is not None:
-            ev[0].record()
-        ard.ard_fwd(ctx, pat, ard.ARD_BF16, B, K, N, alpha, pX, K, pW, K, pY, N, ard.ARD_OUT_SCATTER_ZEROFILL, cs)
-        if ev is not None:
-            ev[1].record()
-        ard.ard_bwd_data(ctx, pat, ard.ARD_BF16, B, K, N, alpha, pdY, N, 0, pW, K, pdX, K, cs)
-        if ev is not None:
-            ev[2].record()
-        ard.ard_bwd_weight(ctx, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, alpha, pX, K, pdY, N, 0, pdW, K, 0, cs)
-        if ev is not None:
-            ev[3].record()
-
-    def step(pp, it, ev=None):
-        ard.ard_sample_pattern(ctx, pat, dist_ids[pp], seed, it, rank, cs)
-        gemms(1.0 / (1.0 - pp), ev)
-
-    def kept_units_of(pp, its):
-        """Host replay of the device sampler's counters, for FLOP accounting only (reads the pattern
-        back after the timed region)."""
-        out = []
-        for it in its:
-            ard.ard_sample_pattern(ctx, pat, dist_ids[pp], seed, it, rank)
-            dp_, b_, nk, _ = ard.ard_pattern_to_host(pat, 0)
-            out.append((dp_, b_, nk))
-        return out
-
-    wall = [0.0, 0.0]
-
-    def timed_run(pp, first_it, per_kernel=False):
-        for w in range(args.warmup):
-            step(pp, first_it + w)
-        its = list(range(first_it + args.warmup, first_it + args.warmup + args.steps))
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in its] if per_kernel else None
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        wall[0] = time.time()
-        e0.record()
-        for i, it in enumerate(its):
-            step(pp, it, evs[i] if per_kernel else None)
-        e1.record()
-        barrier()
-        wall[1] = time.time()
-        ms = e0.elapsed_time(e1)
-        per = None
-        if per_kernel:
-            per = [[evs[i][j].elapsed_time(evs[i][j + 1]) for j in range(3)] for i in range(len(its))]
-        return ms, its, per
-
-    def dense_run():
-        ard.ard_pattern_set(ctx, pat, 1, 1)
-        for _ in range(args.warmup):
-            gemms(1.0)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record()
-        for _ in range(args.steps):
-            gemms(1.0)
-        e1.record()
-        barrier()
-        return e0.elapsed_time(e1)
-
-    def torch_dense_run():
-        Wt = W.t()
-        for _ in range(args.warmup):
-            torch.matmul(X, Wt); torch.matmul(dY, W); torch.matmul(dY.t(), X)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        e0.record()
-        for _ in range(args.steps):
-            torch.matmul(X, Wt); torch.matmul(dY, W); torch.matmul(dY.t(), X)
-        e1.record()
-        barrier()
-        return e0.elapsed_time(e1)
-
-    # ---- the timed region the headline value comes from (p = 0.5) ----
-    launches0 = ard.ard_launch_count(ctx)
-    ms, its, per = timed_run(p, 0, per_kernel=True)
-    t_begin, t_end = wall
-    clk = clocks.stop(t_begin, t_end)
-    launches = (ard.ard_launch_count(ctx) - launches0) * args.steps // (args.steps + args.warmup)
-    status = ard.ard_last_device_status(ctx)
-    pats = kept_units_of(p, its)
-    if kind == ard.ARD_ROW:
-        kept_flops = [3 * 2.0 * B * K * nk for (_, _, nk) in pats]
-    else:
-        kept_flops = [3 * 2.0 * B * wl["ts"] ** 2 * nk for (_, _, nk) in pats]
-    dense_flops = 3 * 2.0 * B * K * N * args.steps
-    kept_tflops = sum(kept_flops) / (ms * 1e-3) / 1e12
-    dense_eq_tflops = dense_flops / (ms * 1e-3) / 1e12
-
-    # max over ranks, sum of work
-    if world > 1:
-        ms, kept_all, dense_all = aggregate_over_ranks(ms, sum(kept_flops), dense_flops, "cuda")
-        kept_tflops = kept_all / (ms * 1e-3) / 1e12
-        dense_eq_tflops = dense_all / (ms * 1e-3) / 1e12
-
-    # ---- roofline of the tcgen05 GEMM kernel (three launches per step) ----
+    lb = LayerBench(torch, ard, args, wl, local, rank, world, barrier)
+    B, K, N, p = wl["B"], wl["K"], wl["N"], wl["p"]
     peaks = load_peaks()
-    per = np.array(per)                                  # [steps][3] ms
-    gemm_ms = float(per.sum())
-    op_names = ["fwd", "bwd_data", "bwd_weight"]
-    per_op = {}
-    for j, nm in enumerate(op_names):
-        fl = sum(kept_flops) / 3.0
-        per_op[nm] = {"ms_avg": float(per[:, j].mean()), "tflops": fl / (float(per[:, j].sum()) * 1e-3) / 1e12}
-    achieved = sum(kept_flops) / (gemm_ms * 1e-3) / 1e12
-    # The timed region is short (tens of ms): if the SM clock stayed near its maximum the kernels ran in
-    # the burst regime and are held against the burst cuBLAS figure, otherwise against the sustained one.
-    burst = clk["sm_mhz"] is None or clk["sm_max_mhz"] is None or clk["sm_mhz"] >= 0.9 * clk["sm_max_mhz"]
-    peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
-    roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": DRAM_TRAFFIC_PER_LAUNCH, "traffic_unit": "bytes per launch (dense step)",
-                "peak_source": peaks["source"] + (" burst" if burst else " sustained") + " cuBLAS bf16 8192^3",
-                "frac_of_burst": achieved / peaks["bf16_tflops"],
-                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
-                "frac_of_nominal_2250": achieved / 2250.0, "kernel": "ard_gemm_tc_kernel",
-                "launches": 3 * args.steps, "per_op": per_op}
 
-    # ---- dense baselines and the other dropout rates (outside the headline region) ----
-    detail = {}
+    if args.force_dp:
+        # a handful of steps of one period, for a profiler capture of sparse draws
+        ard.ard_pattern_set(lb.ctx, lb.pat, args.force_dp, 1)
+        for _ in range(args.warmup + args.steps):
+            lb.gemms(2.0)
+        torch.cuda.synchronize()
+        if rank == 0:
+            print(json.dumps({"forced_dp": args.force_dp, "steps": args.steps, "status": int(ard.ard_last_device_status(lb.ctx))}))
+        lb.close()
+        return
+
+    # ---- the timed regions the headline value comes from (p = 0.5) ----
+    h = lb.headline(peaks)
+    clk = clocks.stop(*h["wall"])
+    roofline = roofline_of(h, peaks, clk, lb)
     if args.quick:
         if rank == 0:
-            print(json.dumps({"metric": METRIC, "value": kept_tflops, "unit": UNIT, "quick": True,
-                              "ms_per_step": ms / args.steps, "roofline": roofline, "clocks": clk}))
-        ard.ard_pattern_destroy(pat)
-        ard.ard_destroy(ctx)
+            print(json.dumps({"metric": METRIC, "value": h["value"], "unit": UNIT, "quick": True,
+                              "ms_per_step": h["ms"] / args.steps, "roofline": roofline, "clocks": clk}))
+        lb.close()
         return
-    dense_ms = dense_run()
-    torch_ms = torch_dense_run()
-    best_dense = min(dense_ms, torch_ms)
-    detail["dense_ms_per_step"] = {"own_kernels_dp1": dense_ms / args.steps, "torch_matmul": torch_ms / args.steps}
-    detail["dense_tflops"] = {"own_kernels_dp1": dense_flops / (dense_ms * 1e-3) / 1e12,
-                              "torch_matmul": dense_flops / (torch_ms * 1e-3) / 1e12}
-    detail["speedup_vs_dense"] = {}
-    detail["kept_fraction"] = {}
-    for pp in (0.3, 0.5, 0.7):
-        if pp == p:
-            ms_p, its_p = ms, its
-            pats_p = pats
-        else:
-            ms_p, its_p, _ = timed_run(pp, 10000)
-            pats_p = kept_units_of(pp, its_p)
-        detail["speedup_vs_dense"][str(pp)] = best_dense / ms_p
-        detail["kept_fraction"][str(pp)] = float(np.mean([nk / units for (_, _, nk) in pats_p]))
-    detail["ideal_speedup"] = {str(pp): 1.0 / (1.0 - pp) for pp in (0.3, 0.5, 0.7)}
+
+    # ---- dense baselines, the per-period table, expectations for the sweep's rates ----
+    detail = {}
+    dense = lb.dense_baselines()
+    dense_flops_step = 3 * 2.0 * B * K * N
+    detail["dense_ms_per_step"] = dense
+    detail["dense_tflops"] = {k2: dense_flops_step / (dense[k2] * 1e-3) / 1e12 for k2 in ("own_kernels_dp1", "torch_matmul")}
+    sw = sweep_block(lb, peaks, dense)
+    detail.update(sw)
+    detail["speedup_vs_dense"] = {k2: v["expected_speedup"] for k2, v in sw["expected"].items()}
+    detail["ideal_speedup"] = {k2: v["ideal_speedup"] for k2, v in sw["expected"].items()}
+    detail["repeats"] = {"n": REPEATS, "values": h["values"], "ms_per_step": [m / args.steps for m in h["ms_all"]],
+                         "spread": (max(h["values"]) - min(h["values"])) / h["value"]}
+
+    # ---- the other half of the large-layer sweep: the same layer under the 128 x 128 tile pattern ----
+    if args.workload == "mlp8192_row" and world == 1:
+        twl = WORKLOADS["mlp8192_tile"]
+        tb = LayerBench(torch, ard, args, twl, local, rank, world, barrier, tensors=lb.t)
+        th = tb.headline(peaks)
+        tdense = tb.dense_baselines()
+        tsw = sweep_block(tb, peaks, tdense)
+        detail["tile"] = {"workload": "mlp8192_tile", "ts": twl["ts"], "value": th["value"], "values": th["values"],
+                          "ms_per_step": th["ms"] / args.steps, "roofline_frac_of_burst": th["achieved"] / peaks["bf16_tflops"],
+                          "per_op": th["per_op"], "gpu_launches": th["launches"], "device_status": th["status"],
+                          "dense_ms_per_step": {k2: tdense[k2] for k2 in ("own_kernels_dp1", "torch_matmul")}, **tsw}
+        tb.close()
+
+    # ---- operands that move: the same steps with three rotating buffer sets, and with never-seen addresses ----
+    if world == 1:
+        t = lb.t
+        n_rot = max(8, min(args.steps, 48))
+        sets = [lb.ptr]
+        keep_alive = []
+        for _ in range(2):
+            extra = {k2: torch.empty_like(t[k2]) for k2 in ("X", "dY", "Y", "dX", "dW")}
+            extra["X"].copy_(t["X"]); extra["dY"].copy_(t["dY"])
+            keep_alive.append(extra)
+            sets.append({**lb.ptr, **{k2: v.data_ptr() for k2, v in extra.items()}})
+        its_r = list(range(40000, 40000 + n_rot))
+        for s_ in sets:
+            lb.step(p, 39999, None, s_)
+        fixed = statistics.median(lb.timed_steps(p, its_r)[0] for _ in range(3)) / n_rot
+        rot = statistics.median(lb.timed_steps(p, its_r, ptrs=sets)[0] for _ in range(3)) / n_rot
+        # never-seen addresses: one pool per operand, the base sliding by 256 bytes per step
+        pool = {k2: torch.empty(t[k2].numel() + 128 * (n_rot + 1), dtype=t[k2].dtype, device="cuda") for k2 in ("X", "dY")}
+        slide = []
+        for i in range(n_rot):
+            q = dict(lb.ptr)
+            for k2 in ("X", "dY"):
+                view = pool[k2][128 * i:128 * i + t[k2].numel()]
+                q[k2] = view.data_ptr()
+            slide.append(q)
+        pool["X"][:t["X"].numel()].copy_(t["X"].reshape(-1)); pool["dY"][:t["dY"].numel()].copy_(t["dY"].reshape(-1))
+        fresh = lb.timed_steps(p, its_r, ptrs=slide)[0] / n_rot
+        detail["moving_operands"] = {"ms_per_step_fixed_buffers": fixed, "ms_per_step_three_rotating_sets": rot,
+                                     "ms_per_step_new_addresses_every_step": fresh, "steps": n_rot}
+        del pool, keep_alive
 
     # ---- the same step as one CUDA graph: sampler on a device counter + ard_layer_products (the three products
     # enqueued side by side on the context's streams); the dense torch step replayed from a graph beside it ----
     if world == 1:
+        X, W, dY, Y, dX, dW = (lb.t[k2] for k2 in ("X", "W", "dY", "Y", "dX", "dW"))
         gstream = torch.cuda.Stream()
         counter = torch.zeros(1, dtype=torch.int64, device="cuda")
         reps = 10
@@ -1113,15 +1341,15 @@ def main():
         for pp in (0.3, 0.5, 0.7):
             def body(pp=pp):
                 gs = gstream.cuda_stream
-                ard.ard_sample_pattern_counter(ctx, pat, dist_ids[pp], seed, 30000, counter, 1, rank, gs)
-                ard.ard_layer_products(ctx, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, 1.0 / (1.0 - pp), X, K, W, K, dY, N,
+                ard.ard_sample_pattern_counter(lb.ctx, lb.pat, lb.dist_ids[pp], lb.seed, 30000, counter, 1, rank, gs)
+                ard.ard_layer_products(lb.ctx, lb.pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, 1.0 / (1.0 - pp), X, K, W, K, dY, N,
                                        Y, N, ard.ARD_OUT_SCATTER_ZEROFILL, dX, K, dW, K, 0, gs)
             counter.zero_()
             side[str(pp)] = graph_ms(body, n_replays)
             # iterations of the timed replays: 3 eager calls and 3 replays of `reps` steps came before them
             first = 30000 + 3 + 3 * reps
-            pats_g = kept_units_of(pp, range(first, first + n_replays * reps))
-            side_kept[str(pp)] = float(np.mean([nk / units for (_, _, nk) in pats_g]))
+            pats_g = lb.patterns_of(pp, range(first, first + n_replays * reps))
+            side_kept[str(pp)] = float(np.mean([nk / lb.units for (_, _, nk) in pats_g]))
         Wt_ = W.t()
 
         def torch_body():
@@ -1135,83 +1363,87 @@ def main():
                                         "speedup_vs_dense": {k2: torch_graph / v for k2, v in side.items()}}
 
     # ---- end to end through the C ABI with host buffers ----
+    t = lb.t
+    hX, hdY, hY = t["hX"], t["hdY"], t["hY"]
     h2d = hX.numel() * 2 + hdY.numel() * 2
     d2h = hY.numel() * 2
     e2e_steps = max(4, min(args.steps, 40))
-    # Three streams and two sets of device buffers: the copy-in of step i+1 and the copy-out of step i-1
-    # overlap the kernels of step i; every step still moves its own inputs and result over PCIe.
+    # Three streams and three sets of device buffers: the copy-in of step i+1 and the copy-out of step i-1
+    # overlap the kernels of step i; every step still moves its own inputs and result over PCIe, and the operands
+    # of consecutive steps sit at different addresses.
     s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
-    Xb = [X, torch.empty_like(X)]
-    dYb = [dY, torch.empty_like(dY)]
-    Yb = [Y, torch.empty_like(Y)]
+    NB = 3
+    Xb = [t["X"]] + [torch.empty_like(t["X"]) for _ in range(NB - 1)]
+    dYb = [t["dY"]] + [torch.empty_like(t["dY"]) for _ in range(NB - 1)]
+    Yb = [t["Y"]] + [torch.empty_like(t["Y"]) for _ in range(NB - 1)]
     al = 1.0 / (1.0 - p)
+    dXt, dWt, Wt2 = t["dX"], t["dW"], t["W"]
 
     def e2e_run(its_list):
         in_done, cmp_done, out_done = {}, {}, {}
         for i, it in enumerate(its_list):
-            k = i % 2
+            k = i % NB
             with torch.cuda.stream(s_in):
-                if i >= 2:
-                    s_in.wait_event(cmp_done[i - 2])          # buffers k are free again
+                if i >= NB:
+                    s_in.wait_event(cmp_done[i - NB])          # buffers k are free again
                 Xb[k].copy_(hX, non_blocking=True)
                 dYb[k].copy_(hdY, non_blocking=True)
                 in_done[i] = s_in.record_event()
             with torch.cuda.stream(s_cmp):
                 s_cmp.wait_event(in_done[i])
-                if i >= 2:
-                    s_cmp.wait_event(out_done[i - 2])         # Y[k] has been read out
-                ard.ard_sample_pattern(ctx, pat, dist_ids[p], seed, it, rank, s_cmp)
-                ard.ard_fwd(ctx, pat, ard.ARD_BF16, B, K, N, al, Xb[k], K, W, K, Yb[k], N,
-                            ard.ARD_OUT_SCATTER_ZEROFILL, s_cmp)
-                ard.ard_bwd_data(ctx, pat, ard.ARD_BF16, B, K, N, al, dYb[k], N, 0, W, K, dX, K, s_cmp)
-                ard.ard_bwd_weight(ctx, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, al, Xb[k], K, dYb[k], N, 0, dW, K,
-                                   0, s_cmp)
+                if i >= NB:
+                    s_cmp.wait_event(out_done[i - NB])         # Y[k] has been read out
+                sc = s_cmp.cuda_stream
+                ard.ard_sample_pattern(lb.ctx, lb.pat, lb.dist_ids[p], lb.seed, it, rank, sc)
+                ard.ard_fwd(lb.ctx, lb.pat, ard.ARD_BF16, B, K, N, al, Xb[k], K, Wt2, K, Yb[k], N,
+                            ard.ARD_OUT_SCATTER_ZEROFILL, sc)
+                ard.ard_bwd_data(lb.ctx, lb.pat, ard.ARD_BF16, B, K, N, al, dYb[k], N, 0, Wt2, K, dXt, K, sc)
+                ard.ard_bwd_weight(lb.ctx, lb.pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, al, Xb[k], K, dYb[k], N, 0, dWt, K,
+                                   0, sc)
                 cmp_done[i] = s_cmp.record_event()
             with torch.cuda.stream(s_out):
                 s_out.wait_event(cmp_done[i])
                 hY.copy_(Yb[k], non_blocking=True)
                 out_done[i] = s_out.record_event()
 
-    e2e_run([20000, 20001, 20002])                            # warm-up (also builds descriptor tables)
+    e2e_run([20000, 20001, 20002])                            # warm-up
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     its_e = list(range(20003, 20003 + e2e_steps))
-    for st in (s_in, s_cmp, s_out):
-        st.wait_stream(torch.cuda.current_stream())
-    e0.record(s_in)
-    e2e_run(its_e)
-    e1.record(s_out)
-    barrier()
-    ms_e = e0.elapsed_time(e1)
-    pats_e = kept_units_of(p, its_e)
-    fl_e = sum(3 * 2.0 * B * K * nk for (_, _, nk) in pats_e) if kind == ard.ARD_ROW else \
-        sum(3 * 2.0 * B * wl["ts"] ** 2 * nk for (_, _, nk) in pats_e)
-    e2e_val = fl_e / (ms_e * 1e-3) / 1e12 * world
-    e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-           "ms_per_step": ms_e / e2e_steps, "steps": e2e_steps,
-           "how": "C-ABI calls on a compute stream; pinned-host copies on two more streams, double-buffered"}
+    ms_e_all = []
+    for _ in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for st in (s_in, s_cmp, s_out):
+            st.wait_stream(torch.cuda.current_stream())
+        e0.record(s_in)
+        e2e_run(its_e)
+        e1.record(s_out)
+        barrier()
+        ms_e_all.append(e0.elapsed_time(e1))
+    ms_e = statistics.median(ms_e_all)
+    pats_e = lb.patterns_of(p, its_e)
+    fl_e = sum(3 * lb.flops_per_unit() * nk for (_, _, nk) in pats_e)
+    e2e = {"value": fl_e / (ms_e * 1e-3) / 1e12 * world, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "ms_per_step": ms_e / e2e_steps, "steps": e2e_steps, "repeats": len(ms_e_all),
+           "how": "C-ABI calls on a compute stream; pinned-host copies on two more streams, three buffer sets"}
 
     # ---- CPU baseline: the oracle on the host cores (rank 0, N = 1 only) ----
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        dt, fl, threads, sample = oracle_sample_seconds(wl, d, max(wl["B"], wl["N"]))   # one full step
+        dt, fl, threads, sample = oracle_sample_seconds(wl, t["host"], max(wl["B"], wl["N"]))   # one full step
         cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
                "seconds": dt}
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": kept_tflops, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "metric": METRIC, "value": h["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": h["ms"] / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "B": B, "K": K, "N": N, "kind": wl["kind"], "ts": wl["ts"], "p": p,
-                       "n_dp": n_dp, "l2": "inputs larger than L2 (X, W, dY and outputs: ~0.5 GB per step)",
-                       "replicas": world},
-            "dense_equiv_tflops": dense_eq_tflops, "clocks": clk, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "cpu_baseline": cpu, "detail": detail, "device_status": int(status),
+            "config": layer_config(args, wl, world),
+            "dense_equiv_tflops": h["dense_equiv"], "clocks": clk, "e2e": e2e, "gpu_launches": h["launches"],
+            "roofline": roofline, "cpu_baseline": cpu, "detail": detail, "device_status": h["status"],
         }
         print(json.dumps(line))
-    ard.ard_pattern_destroy(pat)
-    ard.ard_destroy(ctx)
+    lb.close()
     if world > 1:
         dist.destroy_process_group()
 
