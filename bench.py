@@ -932,6 +932,11 @@ class LayerBench:
         self.t = tensors
         self.ctx = ard.ard_create(dev, 2 * B * N + 4096)
         ard.ard_set_compact_reuse(self.ctx, 1)   # dY is not written between bwd-data and bwd-weight of a step
+        for kv in args.opt:
+            name, val = kv.split("=")
+            ard.ard_set_option(self.ctx, getattr(ard, "ARD_OPT_" + name.upper()), int(val))
+        if args.shared_tail:
+            ard.ard_set_shared_tail(self.ctx, 1, 0, 0)
         self.pat = ard.ard_pattern_create(self.ctx, self.kind, K, N, wl["ts"])
         self.dist_ids, self.khat = {}, {}
         for i, pp in enumerate(RATES):
@@ -1052,9 +1057,10 @@ class LayerBench:
         names = ["sampler", "fwd", "bwd_data", "bwd_weight", "bwd_weight_zero_fill"]
         table, step_by_dp, units_by_dp = {}, {}, {}
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+        self.dense_burst = {}
         for dp in range(1, n_dp + 1):
             ms = {nm: [] for nm in names}
-            steps, kept = [], []
+            steps, kept, prods = [], [], []
             for b in range(1, dp + 1):
                 ard.ard_pattern_set(self.ctx, self.pat, dp, b, self.cs)
                 kept.append(self.ard.ard_pattern_to_host(self.pat, 0)[2])
@@ -1072,6 +1078,21 @@ class LayerBench:
                     for j, nm in enumerate(names):
                         ms[nm].append(ev[j].elapsed_time(ev[j + 1]))
                     steps.append(ev[0].elapsed_time(ev[4]))
+                    prods.append(ev[1].elapsed_time(ev[4]))
+            if dp == 1:
+                # the dense layer, timed the same way (one pass between two synchronisations): this library's three
+                # products without a sampler, and torch.matmul
+                X, dY, W = self.t["X"], self.t["dY"], self.t["W"]
+                Wt = W.t()
+                lib = []
+                for rep in range(REPEATS + 1):
+                    ev[0].record()
+                    torch.matmul(X, Wt); torch.matmul(dY, W); torch.matmul(dY.t(), X)
+                    ev[1].record()
+                    torch.cuda.synchronize()
+                    if rep:
+                        lib.append(ev[0].elapsed_time(ev[1]))
+                self.dense_burst = {"own_kernels_dp1": statistics.median(prods), "torch_matmul": statistics.median(lib)}
             fl = self.flops_per_unit() * float(np.mean(kept))
             row = {"kept_units_mean": float(np.mean(kept)), "step_ms": statistics.median(steps)}
             for nm in names:
@@ -1162,10 +1183,12 @@ def roofline_of(h, peaks, clk, lb):
 
 
 def sweep_block(lb, peaks, dense):
-    """Per-period table, expectations under every rate of the sweep, and the sampled figures beside them."""
+    """Per-period table, expectations under every rate of the sweep, and the sampled figures beside them.  The
+    expectations are held against the dense step timed like the table's entries (single passes); the sampled
+    figures against the dense step timed like them (long loops, where the power cap lowers the clock)."""
     best_dense = min(dense["own_kernels_dp1"], dense["torch_matmul"])
     table, step_by_dp, units_by_dp = lb.per_dp_table(peaks["bf16_tflops"])
-    exp = lb.expectations(step_by_dp, units_by_dp, best_dense)
+    exp = lb.expectations(step_by_dp, units_by_dp, min(lb.dense_burst.values()))
     sampled = {}
     for pp in (0.3, 0.5, 0.7):
         its, runs = lb.repeated(pp, 10000 + int(pp * 100) * 1000)
@@ -1173,7 +1196,7 @@ def sweep_block(lb, peaks, dense):
         pats = lb.patterns_of(pp, its)
         sampled[str(pp)] = {"ms_per_step": ms, "speedup_vs_dense": best_dense / ms,
                             "kept_fraction": float(np.mean([nk / lb.units for (_, _, nk) in pats]))}
-    return {"per_dp": table, "expected": exp, "sampled": sampled,
+    return {"per_dp": table, "dense_ms_single_pass": lb.dense_burst, "expected": exp, "sampled": sampled,
             "note": "per_dp: median over every offset b and %d repeats, pattern forced with ard_pattern_set; expected: "
                     "sum over dp of k^_dp x mean step time, k^ = the quantised distribution; sampled: %d device-drawn "
                     "steps per rate (a bimodal K makes these noisy; the expectations are the figures to read)"
@@ -1192,6 +1215,10 @@ def main():
     ap.add_argument("--conv-run-len", type=int, default=0,
                     help="conv workloads: values per sampled run of the sensitivity prediction (1 = single values, "
                          "the statement of Sec. 5.1; default: the workload's 32)")
+    ap.add_argument("--opt", action="append", default=[], metavar="NAME=VALUE",
+                    help="tuning switch of the context, e.g. BAND_ROWS=8 (see ard_set_option); repeatable")
+    ap.add_argument("--shared-tail", action="store_true", help="row products share their left-over tiles (ard_set_shared_tail)")
+    ap.add_argument("--sweep-only", action="store_true", help="headline, dense baselines and the per-period table only")
     ap.add_argument("--force-dp", type=int, default=0, help="profiler captures: time steps of this period only (b = 1)")
     args = ap.parse_args()
     wl = dict(WORKLOADS[args.workload])
@@ -1263,6 +1290,13 @@ def main():
     detail["ideal_speedup"] = {k2: v["ideal_speedup"] for k2, v in sw["expected"].items()}
     detail["repeats"] = {"n": REPEATS, "values": h["values"], "ms_per_step": [m / args.steps for m in h["ms_all"]],
                          "spread": (max(h["values"]) - min(h["values"])) / h["value"]}
+
+    if args.sweep_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": h["value"], "unit": UNIT, "sweep_only": True, "options": args.opt,
+                              "ms_per_step": h["ms"] / args.steps, "roofline": roofline, "clocks": clk, "detail": detail}))
+        lb.close()
+        return
 
     # ---- the other half of the large-layer sweep: the same layer under the 128 x 128 tile pattern ----
     if args.workload == "mlp8192_row" and world == 1:

@@ -84,6 +84,17 @@ typedef enum { ARD_PATH_AUTO = 0, ARD_PATH_CUDA_CORE = 1, ARD_PATH_TENSOR_CORE =
 ard_status ard_create(ard_ctx** ctx, int device, size_t workspace_bytes);
 ard_status ard_destroy(ard_ctx* ctx);
 ard_status ard_set_path(ard_ctx* ctx, ard_path path);
+/* Tuning switches of a context (host state only; nothing is read from the environment).  Defaults in brackets.
+ *   ARD_OPT_PDL [1]               launch kernels with programmatic stream serialization
+ *   ARD_OPT_PDL_IN_CAPTURE [1]    ... also while the stream is being captured into a CUDA graph
+ *   ARD_OPT_SIDE_STREAMS [1]      ard_layer_products / ard_rows_products / ard_blocks_products / ard_mlp_step may
+ *                                 fork onto the context's own streams (0: everything on the caller's stream)
+ *   ARD_OPT_CTA_PAIRS [1]         tensor-core products with more than 128 output rows use pairs of SMs
+ *   ARD_OPT_BAND_ROWS [16]        raster band of the tensor-core tile order, in 128-row tiles (0: one band)
+ * Errors: ARD_ERR_INVALID_ARG (unknown option, negative value). */
+typedef enum { ARD_OPT_PDL = 0, ARD_OPT_PDL_IN_CAPTURE = 1, ARD_OPT_SIDE_STREAMS = 2, ARD_OPT_CTA_PAIRS = 3,
+               ARD_OPT_BAND_ROWS = 4 } ard_option;
+ard_status ard_set_option(ard_ctx* ctx, ard_option option, int value);
 /* Opt-in for training loops.  The tensor-core backward GEMMs of a row pattern read a compacted copy
  * of a full-width dY (kept columns only) that the library makes in the context workspace.  With
  * enable != 0, a backward call whose dY pointer, leading dimension, batch size, pattern sample and
@@ -234,7 +245,7 @@ ard_status ard_bwd_weight(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype,
  * (Sec. 3.1, 3.2), and on small layers one of them leaves most SMs idle.  The first call on a context creates
  * the streams (make it before any stream capture); the call itself can be captured into a CUDA graph.
  * Inputs must not be written, and outputs not read, by other work until the caller's stream has passed the
- * call.  With ARD_MLP_STREAMS=1 in the environment everything stays on the caller's stream.  Asynchronous. */
+ * call.  After ard_set_option(ctx, ARD_OPT_SIDE_STREAMS, 0) everything stays on the caller's stream.  Asynchronous. */
 ard_status ard_layer_products(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, ard_dtype dW_dtype, int B, int K,
                               int N, float alpha, const void* X, int ldx, const void* W, int ldw, const void* dY,
                               int lddy, void* Y, int ldy, ard_outmode outmode, void* dX, int lddx, void* dW, int lddw,
@@ -427,7 +438,8 @@ ard_status ard_rows_bwd_weight_compact(ard_ctx* ctx, const ard_rows* rows, ard_d
  * backward-data) runs on a stream the context owns beside the input half (gather of A, forward) on the caller's
  * stream; the weight gradient waits for both gathered matrices; everything is joined into the caller's stream
  * before the call returns.  The first call on a context creates the stream (make it before any stream
- * capture); with ARD_MLP_STREAMS=1 in the environment everything stays on the caller's stream.  Asynchronous. */
+ * capture); after ard_set_option(ctx, ARD_OPT_SIDE_STREAMS, 0) everything stays on the caller's stream.
+ * Asynchronous. */
 ard_status ard_rows_products(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N, float alpha,
                              const void* A, int lda, const void* W, int ldw, const void* dY, int lddy, void* Ak,
                              int ldak, void* dYk, int lddyk, void* Y, int ldy, void* dA, int ldda, void* dW, int lddw,

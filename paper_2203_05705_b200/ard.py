@@ -24,10 +24,11 @@ ARD_ROW, ARD_TILE = 0, 1
 ARD_OUT_COMPACT, ARD_OUT_SCATTER_ZEROFILL = 0, 1
 ARD_FLAG_OUT_F32, ARD_FLAG_ACCUMULATE, ARD_FLAG_RELU = 0x10, 0x20, 0x40
 ARD_PATH_AUTO, ARD_PATH_CUDA_CORE, ARD_PATH_TENSOR_CORE = 0, 1, 2
+ARD_OPT_PDL, ARD_OPT_PDL_IN_CAPTURE, ARD_OPT_SIDE_STREAMS, ARD_OPT_CTA_PAIRS, ARD_OPT_BAND_ROWS = range(5)
 ARD_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = [
-    "ard_create", "ard_destroy", "ard_set_path", "ard_set_tile_n", "ard_set_shared_tail", "ard_set_compact_reuse", "ard_set_distribution", "ard_quantise_distribution", "ard_search_distribution", "ard_get_distribution_cdf",
+    "ard_create", "ard_destroy", "ard_set_path", "ard_set_option", "ard_set_tile_n", "ard_set_shared_tail", "ard_set_compact_reuse", "ard_set_distribution", "ard_quantise_distribution", "ard_search_distribution", "ard_get_distribution_cdf",
     "ard_pattern_create", "ard_pattern_destroy", "ard_sample_pattern", "ard_pattern_set",
     "ard_pattern_to_host", "ard_pattern_tile_lists_to_host", "ard_fwd", "ard_bwd_data", "ard_bwd_weight",
     "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_set_lstm_persistent", "ard_lstm_forward", "ard_lstm_backward", "ard_last_device_status", "ard_status_string", "ard_launch_count",
@@ -77,6 +78,7 @@ def lib():
         "ard_set_shared_tail": [vp, i32, i32, i32],
         "ard_set_compact_reuse": [vp, i32],
         "ard_set_distribution": [vp, i32, P(C.c_double), i32],
+        "ard_set_option": [vp, i32, i32],
         "ard_quantise_distribution": [P(C.c_double), i32, P(u64)],
         "ard_search_distribution": [C.c_double, i32, C.c_double, C.c_double, i32, C.c_double, P(C.c_double), P(i32)],
         "ard_get_distribution_cdf": [vp, i32, P(u64), i32, P(i32)],
@@ -183,6 +185,10 @@ def ard_destroy(ctx):
 
 def ard_set_path(ctx, path):
     _check(lib().ard_set_path(ctx, path), "ard_set_path")
+
+
+def ard_set_option(ctx, option, value):
+    _check(lib().ard_set_option(ctx, option, value), "ard_set_option")
 
 
 def ard_set_compact_reuse(ctx, enable):

@@ -214,28 +214,19 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->force_bn = 0;
   ctx->band_m = 16;
   ctx->use_pairs = 1;
-  if (const char* e = getenv("ARD_USE_PAIRS")) ctx->use_pairs = atoi(e);
-  if (const char* e = getenv("ARD_BAND_M")) ctx->band_m = atoi(e);
   ctx->reuse_compact = 0;
   ctx->stream_k = 0;
   ctx->use_pdl = 1;
   ctx->lstm_persistent = 1;
-  if (const char* e = getenv("ARD_LSTM_PERSISTENT")) ctx->lstm_persistent = atoi(e) ? 1 : 0;
   ctx->d_grid_bar = nullptr;
   ctx->d_lstm_partial = nullptr;
-  if (const char* e = getenv("ARD_PDL")) ctx->use_pdl = atoi(e) ? 1 : 0;
   ctx->pdl_in_capture = 1;
   ctx->mlp_two_streams = 1;
-  if (const char* e = getenv("ARD_MLP_STREAMS")) ctx->mlp_two_streams = atoi(e) >= 2 ? 1 : 0;
   ctx->side_stream = nullptr;
   ctx->aux_stream = nullptr;
   ctx->n_ev = 0;
-  if (const char* e = getenv("ARD_PDL_CAPTURE")) ctx->pdl_in_capture = atoi(e) ? 1 : 0;
   ctx->sk_min_blocks = 16;
-  if (const char* e = getenv("ARD_STREAM_K")) ctx->stream_k = atoi(e);
   ctx->sk_min_gain = 24;
-  if (const char* e = getenv("ARD_SK_MIN_BLOCKS")) ctx->sk_min_blocks = atoi(e) > 0 ? atoi(e) : 16;
-  if (const char* e = getenv("ARD_SK_MIN_GAIN")) ctx->sk_min_gain = atoi(e) > 0 ? atoi(e) : 24;
   ctx->d_sk_ws = nullptr;
   ctx->d_sk_cnt = nullptr;
   ctx->last_gather = {nullptr, 0, 0, 0, nullptr, 0ull, nullptr};
@@ -309,6 +300,18 @@ ard_status ard_set_path(ard_ctx* ctx, ard_path path) {
   if (!ctx || path < ARD_PATH_AUTO || path > ARD_PATH_TENSOR_CORE) return ARD_ERR_INVALID_ARG;
   ctx->path = path;
   return ARD_OK;
+}
+
+ard_status ard_set_option(ard_ctx* ctx, ard_option option, int value) {
+  if (!ctx || value < 0) return ARD_ERR_INVALID_ARG;
+  switch (option) {
+    case ARD_OPT_PDL: ctx->use_pdl = value ? 1 : 0; return ARD_OK;
+    case ARD_OPT_PDL_IN_CAPTURE: ctx->pdl_in_capture = value ? 1 : 0; return ARD_OK;
+    case ARD_OPT_SIDE_STREAMS: ctx->mlp_two_streams = value ? 1 : 0; return ARD_OK;
+    case ARD_OPT_CTA_PAIRS: ctx->use_pairs = value ? 1 : 0; return ARD_OK;
+    case ARD_OPT_BAND_ROWS: ctx->band_m = value; return ARD_OK;
+  }
+  return ARD_ERR_INVALID_ARG;
 }
 
 ard_status ard_set_compact_reuse(ard_ctx* ctx, int enable) {

@@ -277,7 +277,7 @@ __device__ __forceinline__ void pdl_wait_prior_grids() { asm volatile("griddepco
 #endif
 
 // The attribute is also kept while a stream is being captured into a CUDA graph (the nodes are then joined
-// by programmatic edges); ARD_PDL_CAPTURE=0 launches the ordinary way during a capture.
+// by programmatic edges); ard_set_option(ctx, ARD_OPT_PDL_IN_CAPTURE, 0) launches the ordinary way during a capture.
 inline bool ard_pdl_allowed(const ard_ctx* ctx, cudaStream_t s) {
   if (!ctx->use_pdl) return false;
   if (ctx->pdl_in_capture) return true;
