@@ -433,7 +433,7 @@ def run_mlp_step(args, wl):
     def graphed(stack):
         s = torch.cuda.Stream()
         with torch.cuda.stream(s):
-            eager(stack)                     # descriptor tables are built outside the capture
+            eager(stack)                     # warm-up; the context creates its side streams outside the capture
         torch.cuda.synchronize()
         gr = torch.cuda.CUDAGraph()
         with torch.cuda.graph(gr):

@@ -16,9 +16,11 @@
  *   - `cuda_stream` is a cudaStream_t passed as void*.  Calls only enqueue work; they do not
  *     synchronise unless stated.  The pattern lives on the device: nothing about it returns to the
  *     host unless ard_pattern_to_host is called.
- *   - The library allocates device memory only in ard_create, ard_pattern_create and (once per new
- *     combination of operand pointer and shape) when it builds and caches TMA descriptor tables
- *     for the bf16 tensor-core path; everything is freed by the matching destroy call.
+ *   - The library allocates device memory only in its create calls (ard_create, ard_pattern_create,
+ *     ard_rows_create, ard_blocks_create) and frees it in the matching destroy call.  No product call
+ *     allocates, copies descriptors or synchronises: the TMA descriptors of the bf16 tensor-core path
+ *     are encoded on the host per call, travel as kernel parameters and are fitted to the sampled pattern
+ *     by the kernel itself, so operands may sit at a new address in every call.
  *   - A context's scratch memory and status word are shared by its calls: work enqueued through one
  *     context must be ordered (one stream, or streams ordered by events).  Use one context per
  *     concurrently running stream.
@@ -74,7 +76,7 @@ typedef enum { ARD_PATH_AUTO = 0, ARD_PATH_CUDA_CORE = 1, ARD_PATH_TENSOR_CORE =
 
 #define ARD_MAX_DISTRIBUTIONS 16
 #define ARD_MAX_NDP 4096      /* longest distribution accepted                                  */
-#define ARD_MAX_NDP_TC 32     /* longest period the tensor-core path keeps descriptor tables for */
+#define ARD_MAX_NDP_TC 32     /* longest distribution the tensor-core path takes (longer ones: CUDA cores)  */
 
 /* ---- context -------------------------------------------------------------------------------- */
 
@@ -210,9 +212,9 @@ ard_status ard_bwd_data(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, i
  * variant of ard_bwd_data, same result).  For callers that are not allowed to allocate device
  * memory when they run the layer: a process whose memory plan was frozen after start-up, a plug-in
  * inside an application that owns the allocator, or anyone who must avoid the device-wide
- * synchronisation of cudaMalloc / cudaFree.  ard_bwd_data can allocate (descriptor tables on first
- * use of new buffers); this call never does, and neither calls cudaMalloc / cudaFree nor any
- * allocating library routine.
+ * synchronisation of cudaMalloc / cudaFree.  ard_bwd_data compacts dY into the workspace that
+ * ard_create allocated (and fails with ARD_ERR_NOMEM when that workspace is too small); this call needs no
+ * workspace at all, and calls neither cudaMalloc / cudaFree nor any allocating library routine.
  *   Row patterns only, full-width dY [B][N] (lddy), W [N][K] (ldw), dX [B][K] (lddx); runs on the
  *   CUDA cores (fp32 accumulate) for both dtypes.  The compacted copy of dY is kept in a fixed
  *   array inside the library image: ARD_STATIC_SCRATCH_BYTES per GPU that loads the library, held
@@ -328,7 +330,7 @@ ard_status ard_sample_pattern_counter(ard_ctx* ctx, ard_pattern* pat, int dist_i
  * and columns zero), layers[l].db if not NULL, dX [B][K_0] if not NULL; A and dZ of every layer hold what
  * the step computed.  `layers` is a HOST array; all pointers inside are DEVICE pointers owned by the caller;
  * dimensions must satisfy the alignment rules of ard_fwd or the slower CUDA-core kernels run.  Enqueues
- * only; allocates nothing once every buffer has been seen once (descriptor tables, two internal streams
+ * only; allocates nothing after the context's first forking call (which creates two internal streams
  * and their events), so it can be captured into a CUDA graph after one ordinary call.  When every hidden
  * layer has compact_out != 0 the weight compactions, weight gradients, gradient expansions and bias
  * gradients are enqueued on two streams owned by the context, forked from `cuda_stream` after the patterns

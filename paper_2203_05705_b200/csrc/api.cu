@@ -48,76 +48,30 @@ bool encode_map(ard_ctx* ctx, CUtensorMap* out, const void* base, uint64_t cols,
   return r == CUDA_SUCCESS;
 }
 
-constexpr size_t MAX_CACHED_TABLES = 1024;
-
-// Returns a device table of descriptors for `base`; builds and caches it on first use.
+// Fills `out` with the descriptor of the whole matrix [rows][cols] at `base` (pitch ld elements, bf16) and with
+// what the kernel needs to specialise it to the sampled pattern (see TcMap).  Host work only: one encode, no
+// device memory, no copy, nothing cached, so operands may sit at a new address in every call and a call may be
+// captured into a CUDA graph like any other launch.  `units` and `dp_bound` describe the pattern the variant
+// follows; they are implied by the pattern header on the device and only checked here.
 ard_status get_maps(ard_ctx* ctx, const void* base, int rows, int cols, int ld, int units, int variant, int dp_bound,
-                    int box_rows, int box_cols, const CUtensorMap** out, const void* dense_base = nullptr,
-                    int dense_ld = 0) {
-  for (MapTable& t : ctx->maps) {
-    if (t.base == base && t.dense_base == dense_base && t.dense_ld == dense_ld && t.rows == rows && t.cols == cols && t.ld == ld && t.elem_bytes == units &&
-        t.variant == variant && t.dp_bound == dp_bound && t.box_rows == box_rows && t.box_cols == box_cols) {
-      t.epoch = ctx->epoch;
-      *out = t.d_maps;
-      return ARD_OK;
-    }
-  }
-  const int count = variant == MAP_PLAIN ? 1 : map_index_count(dp_bound);
-  std::vector<CUtensorMap> h(count);
-  const char* cbase = reinterpret_cast<const char*>(base);
-  if (variant == MAP_PLAIN) {
-    if (!encode_map(ctx, &h[0], base, cols, rows, (uint64_t)ld * 2, box_cols, box_rows)) return ARD_ERR_CUDA;
-  } else {
-    for (int dp = 1; dp <= dp_bound; ++dp)
-      for (int b = 1; b <= dp; ++b) {
-        int nk = units >= b ? (units - b) / dp + 1 : 1;
-        CUtensorMap* m = &h[dp * (dp - 1) / 2 + (b - 1)];
-        bool ok;
-        if (variant == MAP_STRIDED_ROWS) {
-          // kept neurons b-1, b-1+dp, ...: base moved to row b-1, pitch dp rows, exactly nk rows
-          ok = units >= b ? encode_map(ctx, m, cbase + (size_t)(b - 1) * ld * 2, cols, nk, (uint64_t)dp * ld * 2,
-                                       box_cols, box_rows)
-                          : encode_map(ctx, m, base, cols, 1, (uint64_t)ld * 2, box_cols, box_rows);
-        } else {
-          // compact matrix: all rows, columns 0..nk-1.  A dense pattern needs no compaction: its
-          // entry may point straight at the full-width matrix.
-          if (dp == 1 && dense_base != nullptr)
-            ok = encode_map(ctx, m, dense_base, nk, rows, (uint64_t)dense_ld * 2, box_cols, box_rows);
-          else
-            ok = encode_map(ctx, m, base, nk, rows, (uint64_t)ld * 2, box_cols, box_rows);
-        }
-        if (!ok) return ARD_ERR_CUDA;
-      }
-  }
-  if (ctx->maps.size() >= MAX_CACHED_TABLES) {
-    // Evict the table that has gone unused for the longest time, never one the running call already
-    // handed out.  cudaFree synchronises the device, so no kernel can still be reading it.
-    size_t victim = ctx->maps.size();
-    for (size_t i = 0; i < ctx->maps.size(); ++i)
-      if (ctx->maps[i].epoch != ctx->epoch && (victim == ctx->maps.size() || ctx->maps[i].epoch < ctx->maps[victim].epoch))
-        victim = i;
-    if (victim == ctx->maps.size()) return ARD_ERR_NOMEM;
-    cudaFree(ctx->maps[victim].d_maps);
-    ctx->maps.erase(ctx->maps.begin() + victim);
-  }
-  MapTable t;
-  t.base = base; t.dense_base = dense_base; t.dense_ld = dense_ld; t.rows = rows; t.cols = cols; t.ld = ld; t.elem_bytes = units; t.variant = variant;
-  t.dp_bound = dp_bound; t.box_rows = box_rows; t.box_cols = box_cols; t.count = count;
-  t.epoch = ctx->epoch;
-  t.d_maps = nullptr;
-  if (cudaMalloc(&t.d_maps, sizeof(CUtensorMap) * count) != cudaSuccess) return ARD_ERR_NOMEM;
-  if (cudaMemcpy(t.d_maps, h.data(), sizeof(CUtensorMap) * count, cudaMemcpyHostToDevice) != cudaSuccess) {
-    cudaFree(t.d_maps);
+                    int box_rows, int box_cols, TcMap* out, const void* dense_base = nullptr, int dense_ld = 0) {
+  (void)dp_bound;
+  if (variant == MAP_STRIDED_ROWS && units != rows) return ARD_ERR_INVALID_ARG;
+  if (variant == MAP_COMPACT_COLS && units != cols) return ARD_ERR_INVALID_ARG;
+  if (!encode_map(ctx, &out->tm, base, (uint64_t)cols, (uint64_t)rows, (uint64_t)ld * 2, (uint32_t)box_cols,
+                  (uint32_t)box_rows))
     return ARD_ERR_CUDA;
-  }
-  ctx->maps.push_back(t);
-  *out = t.d_maps;
+  out->base = base;
+  out->dense_base = dense_base;
+  out->ld = ld;
+  out->dense_ld = dense_ld;
+  out->variant = variant;
+  out->pad_ = 0;
   return ARD_OK;
 }
 
 ard_status check_common(ard_ctx* ctx, const ard_pattern* pat, int B, int K, int N) {
   if (!ctx || !pat) return ARD_ERR_INVALID_ARG;
-  ctx->epoch++;  // a new public call: descriptor tables it obtains stay pinned until it returns
   if (pat->ctx != ctx) return ARD_ERR_INVALID_ARG;
   if (B < 0 || K < 0 || N < 0) return ARD_ERR_INVALID_ARG;
   if (K != pat->K_dim || N != pat->N_dim) return ARD_ERR_SHAPE;
@@ -234,7 +188,7 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->d_workspace = nullptr;
   ctx->d_status = nullptr;
   ctx->launches = 0;
-  ctx->epoch = 1;
+  ctx->d_tm_slots = nullptr;
   ctx->encode_fn = nullptr;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return ARD_ERR_CUDA; }
@@ -260,10 +214,12 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
     if (cudaMalloc(&ctx->d_sk_ws, ws_bytes) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->d_sk_cnt), cnt_bytes) != cudaSuccess ||
         cudaMemset(ctx->d_sk_cnt, 0, cnt_bytes) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&ctx->d_tm_slots), tm_slots_bytes()) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->d_grid_bar), 256) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->d_lstm_partial), lstm_bwd_partial_bytes(ctx->sm_count)) != cudaSuccess) {
       if (ctx->d_lstm_partial) cudaFree(ctx->d_lstm_partial);
       if (ctx->d_grid_bar) cudaFree(ctx->d_grid_bar);
+      if (ctx->d_tm_slots) cudaFree(ctx->d_tm_slots);
       if (ctx->d_sk_ws) cudaFree(ctx->d_sk_ws);
       if (ctx->d_sk_cnt) cudaFree(ctx->d_sk_cnt);
       if (ctx->d_workspace) cudaFree(ctx->d_workspace);
@@ -280,7 +236,7 @@ ard_status ard_destroy(ard_ctx* ctx) {
   if (!ctx) return ARD_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   cudaDeviceSynchronize();
-  for (MapTable& t : ctx->maps) cudaFree(t.d_maps);
+  if (ctx->d_tm_slots) cudaFree(ctx->d_tm_slots);
   for (int i = 0; i < ARD_MAX_DISTRIBUTIONS; ++i)
     if (ctx->dist[i].d_cdf) cudaFree(ctx->dist[i].d_cdf);
   if (ctx->d_workspace) cudaFree(ctx->d_workspace);
@@ -1084,8 +1040,8 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
     if (tc_eligible(ctx, pat, ARD_BF16, B, KH, H, XH, KH, W, ldw, C, H, 4) == ARD_OK &&
         ((size_t)H * ldw * 2) % 16 == 0 && lstm_persistent_fits(ctx, B, H, H)) {
       cudaStream_t s = (cudaStream_t)cuda_stream;
-      const CUtensorMap* mapXH = nullptr;
-      const CUtensorMap* mapW[4];
+      TcMap mapXH;
+      TcMap mapW[4];
       // 1. The input half for all steps at once: G[t][:, g*H + j] = x_t . W[g*H + keep[j]][0:I]  (T*B rows).
       if (I > 0) {
         TcArgs t = {};
@@ -1157,8 +1113,8 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
     const char* dZc = reinterpret_cast<const char*>(DZ);
     if (tc_eligible(ctx, pat, ARD_BF16, T * B, KH, H, DZ, 4 * H, W, ldw, D, KH, 4) == ARD_OK &&
         ((size_t)H * ldw * 2) % 16 == 0 && I % 8 == 0 && lstm_persistent_bwd_fits(ctx, B, H)) {
-      const CUtensorMap* mapDZ[4];
-      const CUtensorMap* mapW[4];
+      TcMap mapDZ[4];
+      TcMap mapW[4];
       for (int gate = 0; gate < 4; ++gate) {
         st = get_maps(ctx, dZc + (size_t)gate * H * 2, T * B, H, 4 * H, H, MAP_COMPACT_COLS, pat->dp_bound, 64, 64,
                       &mapDZ[gate]);
@@ -1227,7 +1183,6 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
 static ard_status rows_check(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, const void* p0, int ld0,
                              const void* p1, int ld1, const void* po, int ldo, int out_es) {
   if (!ctx || !rows || rows->ctx != ctx || !p0 || !p1 || !po) return ARD_ERR_INVALID_ARG;
-  ctx->epoch++;
   if (M != rows->M || K < 1 || N < 1) return ARD_ERR_SHAPE;
   if (ctx->encode_fn == nullptr) return ARD_ERR_UNSUPPORTED;
   if (!aligned16(p0) || !aligned16(p1) || !aligned16(po)) return ARD_ERR_ALIGNMENT;
@@ -1306,7 +1261,6 @@ ard_status ard_rows_bwd_weight(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_
 ard_status ard_rows_gather(ard_ctx* ctx, const ard_rows* rows, int M, int width, const void* src, int ld_src, void* dst,
                            int ld_dst, void* cuda_stream) {
   if (!ctx || !rows || rows->ctx != ctx || !src || !dst) return ARD_ERR_INVALID_ARG;
-  ctx->epoch++;
   if (M != rows->M || width < 1 || ld_src < width || ld_dst < width) return ARD_ERR_SHAPE;
   if (!aligned16(src) || !aligned16(dst) || width % 8 || ld_src % 8 || ld_dst % 8) return ARD_ERR_ALIGNMENT;
   DeviceGuard guard(ctx->device);

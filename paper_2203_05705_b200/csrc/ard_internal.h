@@ -59,25 +59,37 @@ struct ArdDistribution {
   std::vector<unsigned long long> h_cdf;
 };
 
-// A cached table of TMA descriptors in device memory, one per (dp, b) pair (or a single one).
-struct MapTable {
-  const void* base;
-  const void* dense_base;  // MAP_COMPACT_COLS: matrix the dp = 1 entry points at (nullptr: same as base)
-  int dense_ld;
-  int rows, cols, ld, elem_bytes;
-  int box_rows, box_cols;
-  int variant;   // see MapVariant
-  int dp_bound;
-  CUtensorMap* d_maps;
-  int count;
-  unsigned long long epoch;  // public call that last used the table (tables of the running call are never evicted)
+enum MapVariant {
+  MAP_PLAIN = 0,         // the descriptor as encoded: [rows][cols], pitch ld
+  MAP_STRIDED_ROWS = 1,  // per pattern: rows b-1, b-1+dp, ... (n_keep of them), all cols
+  MAP_COMPACT_COLS = 2   // per pattern: all rows, cols 0..n_keep-1 of a compact matrix
 };
 
-enum MapVariant {
-  MAP_PLAIN = 0,         // one descriptor: [rows][cols], pitch ld
-  MAP_STRIDED_ROWS = 1,  // per (dp,b): rows b-1, b-1+dp, ... (n_keep of them), all cols
-  MAP_COMPACT_COLS = 2   // per (dp,b): all rows, cols 0..n_keep-1 of a compact matrix
+// A TMA descriptor handed to a kernel BY VALUE (a kernel parameter), with what the kernel needs to turn it into
+// the descriptor of the sampled pattern.  The host encodes the descriptor of the whole matrix and never learns
+// the pattern; the producer warp of the kernel rewrites the address, one extent and the row pitch for the (dp, b)
+// it reads from the pattern header (tensormap_specialise in sm100_ptx.h) and publishes the result in a slot of
+// the context's descriptor scratch that belongs to its SM.  Nothing is cached, allocated or copied per call.
+struct alignas(64) TcMap {
+  CUtensorMap tm;          // [rows][cols] of `base`, pitch ld: also what a dense pattern (dp = 1) reads
+  const void* base;
+  const void* dense_base;  // MAP_COMPACT_COLS: the matrix a dense pattern reads instead of `base` (nullptr: base)
+  int ld, dense_ld;        // elements
+  int variant;             // MapVariant
+  int pad_;
 };
+
+// Descriptor scratch of a context: one group of 128-byte slots per SM for the kernels that own their SM (the
+// tcgen05 product kernels: their shared memory leaves no room for a second block), and one group per block for the
+// whole-sequence LSTM kernels (cooperative launches of at most ARD_TM_LSTM_BLOCKS blocks, one at a time per
+// context).
+constexpr int ARD_TM_SM_MAX = 256;
+constexpr int ARD_TM_SLOTS = 16;
+constexpr int ARD_TM_LSTM_BLOCKS = 512;
+constexpr int ARD_TM_LSTM_SLOTS = 8;
+static inline size_t tm_slots_bytes() {
+  return ((size_t)ARD_TM_SM_MAX * ARD_TM_SLOTS + (size_t)ARD_TM_LSTM_BLOCKS * ARD_TM_LSTM_SLOTS) * sizeof(CUtensorMap);
+}
 
 constexpr int ARD_MLP_EVENTS = 104;  // fork, forward done, two joins, and three per layer (up to 32 layers)
 
@@ -104,9 +116,8 @@ struct ard_ctx {
   void* d_workspace;
   int* d_status;
   ArdDistribution dist[ARD_MAX_DISTRIBUTIONS];
-  std::vector<MapTable> maps;
+  CUtensorMap* d_tm_slots;  // descriptor scratch, tm_slots_bytes()
   unsigned long long launches;
-  unsigned long long epoch;   // bumped by every public GEMM call
   void* encode_fn;  // cuTensorMapEncodeTiled, resolved at run time
   // ard_mlp_step: the weight-side work of an iteration (weight compaction, weight and bias gradients) runs on
   // a second stream, forked from and joined back into the caller's stream with these events
@@ -133,8 +144,6 @@ static inline long long ard_exact_need(double t, long long s) {
   if (c == prod && err > 0.0) c += 1.0;
   return c < 1.0 ? 1 : (long long)c;
 }
-
-static inline int map_index_count(int dp_bound) { return dp_bound * (dp_bound + 1) / 2; }
 
 // Creates the context's second and third stream and their events on first use; false if they do not exist
 // and cannot be created now (`main` is being captured into a graph: nothing may be created then).
@@ -197,11 +206,11 @@ ard_status launch_gemm_cc(ard_ctx* ctx, ard_kind kind, GemmOp op, ard_dtype dtyp
 
 // tcgen05 family (bf16 operands, fp32 accumulate in TMEM).
 struct TcArgs {
-  const CUtensorMap* mapA;  // table or single descriptor
-  const CUtensorMap* mapB;
-  const CUtensorMap* mapA4[4];  // LSTM gate products: one table per gate
-  const CUtensorMap* mapB4[4];
-  int mapA_indexed, mapB_indexed;  // 0: a single descriptor, 1: table indexed by the pattern, 2: by the input pattern
+  TcMap mapA;
+  TcMap mapB;
+  TcMap mapA4[4];  // LSTM gate products: one descriptor per gate
+  TcMap mapB4[4];
+  int mapA_indexed, mapB_indexed;  // 0: used as encoded, 1: specialised to the pattern, 2: to the input pattern
   GemmArgs g;
   int ts;
   int bn;  // N tile: 64, 128 or 256
@@ -216,12 +225,12 @@ ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_
 size_t lstm_bwd_partial_bytes(int sm_count);
 bool lstm_persistent_bwd_fits(ard_ctx* ctx, int B, int H);
 ard_status launch_lstm_backward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
-                                           const CUtensorMap* const mapDZ[4], const CUtensorMap* const mapW[4],
+                                           const TcMap mapDZ[4], const TcMap mapW[4],
                                            const float* C, const float* G, const float* dH_last, float* D, float* dc,
                                            void* DZ, cudaStream_t s);
 bool lstm_persistent_fits(ard_ctx* ctx, int B, int klen, int H);
 ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H,
-                                          int kx0, int klen, int add_zx, float alpha, const CUtensorMap* mapXH, const CUtensorMap* const mapW[4],
+                                          int kx0, int klen, int add_zx, float alpha, const TcMap& mapXH, const TcMap mapW[4],
                                           void* XH, const float* bias, float* C, float* G, cudaStream_t s);
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,

@@ -73,10 +73,7 @@ __host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 4 : (b
 __host__ __device__ constexpr int tmem_cols_for(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }
 
 struct TcParams {
-  const CUtensorMap* mapA;
-  const CUtensorMap* mapB;
-  const CUtensorMap* mapA4[4];  // LSTM modes: one table per gate
-  const CUtensorMap* mapB4[4];
+  CUtensorMap* tm_slots;  // descriptor scratch of the context (ARD_TM_SLOTS slots per SM)
   int mapA_indexed, mapB_indexed;
   const int32_t* hdr;
   const int32_t* idx;
@@ -123,6 +120,15 @@ struct TcParams {
   int sk_any;  // shared tiles also when the tiles do not fill one wave (long contractions, few tiles)
 };
 
+// The descriptors travel by value behind the scalar parameters: A and B, and for the LSTM gate products one per
+// gate for either operand (maps[2 + g] for A, maps[6 + g] for B).
+template <int NM>
+struct TcParamsT : TcParams {
+  TcMap maps[NM];
+};
+__host__ __device__ constexpr bool is_lstm_mode(int mode) { return mode >= M_LSTM_FWD && mode <= M_LSTM_BWD_WEIGHT; }
+__host__ __device__ constexpr int nmaps(int mode) { return is_lstm_mode(mode) ? 10 : 2; }
+
 // CTAS = 2: a cluster of two CTAs shares one 256 x BN output tile; each CTA stages its own 128 rows
 // of A and half of the B rows, so a stage is smaller and the pipeline deeper.
 template <int BN, int CTAS = 1>
@@ -144,6 +150,9 @@ static_assert(CLASS_LIST_BYTES + EPI_WARPS * 32 * 17 * 4 <= EPI_WARPS * 32 * 33 
 
 // Element i of a 4-entry array without dynamic indexing (keeps the array in registers).
 __device__ __forceinline__ int sel4(const int (&a)[4], int i) {
+  return i == 0 ? a[0] : (i == 1 ? a[1] : (i == 2 ? a[2] : a[3]));
+}
+__device__ __forceinline__ const CUtensorMap* sel_map(const CUtensorMap* const (&a)[4], int i) {
   return i == 0 ? a[0] : (i == 1 ? a[1] : (i == 2 ? a[2] : a[3]));
 }
 
@@ -633,7 +642,8 @@ __device__ __forceinline__ void zero_row32(void* out, size_t row_off, int col, i
 
 // ---- the kernel -----------------------------------------------------------------------------------
 template <int BN, int MODE, int CTAS, bool SHARE, bool FUSED>
-__global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const TcParams p) {
+__global__ void __launch_bounds__(tc_threads(MODE), 1)
+ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
   using L = SmemLayout<BN, CTAS>;
   const uint32_t rank = (CTAS == 2) ? cluster_ctarank() : 0u;  // rank 0 leads the pair and issues its MMAs
   constexpr int STAGES = L::STAGES;
@@ -718,8 +728,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
   if (is_rows_mode(MODE) && (warp == 0 || warp >= 10)) {
     // ===================== gathering producers (4 warps, all lanes) =====================
     const int gw = warp == 0 ? 0 : warp - 9;  // 0..3: which quarter of the gathered rows this warp fetches
-    const CUtensorMap* mapB = p.mapB;
-    if (MODE != M_ROWS_BWD_WEIGHT && warp == 0 && lane == 0) tensormap_acquire(mapB);
+    const CUtensorMap* mapB = &p.maps[1].tm;  // the weight, as encoded
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
@@ -822,24 +831,44 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
     }
   } else if (warp == 0) {
     // ===================== TMA producer =====================
-    if (lane == 0) {
-      const int e = p.hdr[HDR_MAPIDX];
-      // a table is indexed by this layer's pattern (1) or by the pattern of the layer that feeds it (2)
-      const int e_in = (FUSED && p.hdr_in != nullptr) ? p.hdr_in[HDR_MAPIDX] : 0;
-      const CUtensorMap* mapA = p.mapA + (p.mapA_indexed == 2 ? e_in : (p.mapA_indexed ? e : 0));
-      const CUtensorMap* mapB = p.mapB + (p.mapB_indexed == 2 ? e_in : (p.mapB_indexed ? e : 0));
-      tensormap_acquire(mapA);
-      tensormap_acquire(mapB);
-      if (MODE == M_LSTM_FWD || MODE == M_LSTM_BWD_DATA) {
+    // The whole warp first turns the descriptors it was given into those of the sampled pattern (the first
+    // operand stage is free until the first load and serves as the 128-byte work area of each).
+    const int32_t* hin = (FUSED && p.hdr_in != nullptr) ? p.hdr_in : p.hdr;
+    const uint32_t smid = sm_id();
+    CUtensorMap* slots = p.tm_slots + (size_t)(smid < (uint32_t)ARD_TM_SM_MAX ? smid : 0u) * ARD_TM_SLOTS;
+    auto special = [&](int mi, int indexed, int slot) -> const CUtensorMap* {
+      const int32_t* h = indexed == 2 ? hin : p.hdr;
+      if (indexed == 0) return &p.maps[mi].tm;
+      return tensormap_specialise(&p.maps[mi], h[HDR_DP], h[HDR_B], h[HDR_NKEEP], smem + 128 * slot, slots + slot, lane);
+    };
+    const CUtensorMap* mapA = special(0, p.mapA_indexed, 0);
+    const CUtensorMap* mapB = special(1, p.mapB_indexed, 1);
+    const CUtensorMap* mapA4[4] = {mapA, mapA, mapA, mapA};
+    const CUtensorMap* mapB4[4] = {mapB, mapB, mapB, mapB};
+    if (is_lstm_mode(MODE)) {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        if (MODE == M_LSTM_BWD_DATA || MODE == M_LSTM_BWD_WEIGHT) mapA4[g] = special(2 + g, 1, 2 + g);
+        if (MODE == M_LSTM_FWD || MODE == M_LSTM_BWD_DATA) mapB4[g] = special(6 + g, 1, 6 + g);
+      }
+    }
+    fence_proxy_async_smem();  // the work area is about to be overwritten by asynchronous copies
+    if (smid >= (uint32_t)ARD_TM_SM_MAX) {  // more SMs than the scratch was laid out for: refuse rather than share a slot
+      if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (int)ARD_ERR_UNSUPPORTED); }
+    } else if (lane == 0) {
+      // only the rewritten copies live in global memory and need the tensor-map proxy's acquire; a descriptor
+      // used as encoded is read from the kernel's parameters
+      auto acquire = [&](const CUtensorMap* m, int mi) {
+        if (m != &p.maps[mi].tm) tensormap_acquire(m);
+      };
+      acquire(mapA, 0);
+      acquire(mapB, 1);
+      if (is_lstm_mode(MODE)) {
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-          tensormap_acquire(p.mapB4[g] + e);
-          if (MODE == M_LSTM_BWD_DATA) tensormap_acquire(p.mapA4[g] + e);
+          if (MODE == M_LSTM_BWD_DATA || MODE == M_LSTM_BWD_WEIGHT) acquire(mapA4[g], 2 + g);
+          if (MODE == M_LSTM_FWD || MODE == M_LSTM_BWD_DATA) acquire(mapB4[g], 6 + g);
         }
-      }
-      if (MODE == M_LSTM_BWD_WEIGHT) {
-#pragma unroll
-        for (int g = 0; g < 4; ++g) tensormap_acquire(p.mapA4[g] + e);
       }
       int stage = 0;
       uint32_t phase = 0;
@@ -881,21 +910,21 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
             const int nkg = ti.nkb >> 2;
             const int g = kb / nkg;
             kx = (kb - g * nkg) * BK;
-            mapBk = p.mapB4[g] + e;
-            load(sA, p.mapA4[g] + e, kx, ti.m0);
+            mapBk = mapB4[g];
+            load(sA, mapA4[g], kx, ti.m0);
           } else if (!A_MN) {
             load(sA, mapA, kx, ti.m0);  // [BM rows][64 k]
           } else {
 #pragma unroll
             for (int i = 0; i < BM / 64; ++i)  // [64 k rows][64 m] per box
-              load(sA + i * (64 * BK * 2), MODE == M_LSTM_BWD_WEIGHT ? p.mapA4[ti.gate] + e : mapA, ti.ax[i], kx);
+              load(sA + i * (64 * BK * 2), MODE == M_LSTM_BWD_WEIGHT ? sel_map(mapA4, ti.gate) : mapA, ti.ax[i], kx);
           }
           // B always moves in 64-wide boxes: K-major [64 rows][64 k] stacked, MN-major [64 k][64 n].
           // In a pair this CTA stages the second half of the tile's B boxes if its rank is 1.
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             if (i < ti.nbox) {
-              if (MODE == M_LSTM_FWD) load(sB + i * (64 * BK * 2), p.mapB4[i] + e, kx, ti.bx[i]);
+              if (MODE == M_LSTM_FWD) load(sB + i * (64 * BK * 2), mapB4[i], kx, ti.bx[i]);
               else if (!B_MN) load(sB + i * (64 * BK * 2), mapBk, kx, ti.bx[i]);
               else load(sB + i * (64 * BK * 2), mapBk, ti.bx[i], kx);
             }
@@ -1358,7 +1387,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) ard_gemm_tc_kernel(const 
 
 // max_tiles: tile count of the densest pattern
 template <int BN, int MODE, int CTAS, bool SHARE = false, bool FUSED = false>
-ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStream_t s) {
+ard_status launch_mode(ard_ctx* ctx, const TcParams& p, const TcMap* maps, int max_tiles, cudaStream_t s) {
   using L = SmemLayout<BN, CTAS>;
   static bool attr_done[64] = {};
   static int max_clusters[64] = {};
@@ -1400,7 +1429,10 @@ ard_status launch_mode(ard_ctx* ctx, const TcParams& p, int max_tiles, cudaStrea
     attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
     cfg.numAttrs++;
   }
-  TcParams pc = p;
+  TcParamsT<nmaps(MODE)> pc;
+  static_cast<TcParams&>(pc) = p;
+  pc.tm_slots = ctx->d_tm_slots;
+  for (int i = 0; i < nmaps(MODE); ++i) pc.maps[i] = maps[i];
   ARD_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, pc));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
@@ -1430,8 +1462,7 @@ int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int dp_bound, int ts) {
 
 ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s) {
   TcParams p = {};
-  p.mapA = a.mapA;
-  p.mapB = a.mapB;
+  const TcMap maps[2] = {a.mapA, a.mapB};
   p.mapA_indexed = a.mapA_indexed;
   p.mapB_indexed = a.mapB_indexed;
   p.hdr = a.g.hdr;
@@ -1476,21 +1507,21 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
     // as long as the list, so the tiles are always cut along the contraction and shared by all SMs.
     p.sk_ws = reinterpret_cast<float4*>(ctx->d_sk_ws);
     p.sk_any = 1;
-    return launch_mode<256, M_ROW_BWD_WEIGHT, 2, true, true>(ctx, p, 1 << 30, s);  // every SM takes a share
+    return launch_mode<256, M_ROW_BWD_WEIGHT, 2, true, true>(ctx, p, maps, 1 << 30, s);  // every SM takes a share
   }
 
 #define ARD_TC_CASE(BN_, MODE_, TILES_) \
-  if (bn == BN_) return launch_mode<BN_, MODE_, 1>(ctx, p, (TILES_), s);
+  if (bn == BN_) return launch_mode<BN_, MODE_, 1>(ctx, p, maps, (TILES_), s);
 #define ARD_TC_ROW(MODE_, TILES_)                                                      \
-  if (fused) return launch_mode<256, MODE_, 1, false, true>(ctx, p, (TILES_), s);      \
-  return share ? launch_mode<256, MODE_, 1, true>(ctx, p, (TILES_), s) : launch_mode<256, MODE_, 1, false>(ctx, p, (TILES_), s);
+  if (fused) return launch_mode<256, MODE_, 1, false, true>(ctx, p, maps, (TILES_), s);      \
+  return share ? launch_mode<256, MODE_, 1, true>(ctx, p, maps, (TILES_), s) : launch_mode<256, MODE_, 1, false>(ctx, p, maps, (TILES_), s);
   // Row patterns with at least two 128-row tiles of output use CTA pairs (256-row tiles).
 #define ARD_TC_PAIR(MODE_, MROWS_, NCOLS_)                                                      \
   if (ctx->use_pairs && (MROWS_) > BM && (p.force_bn == 0 || p.force_bn >= 128) && fused)       \
-    return launch_mode<256, MODE_, 2, false, true>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s);         \
+    return launch_mode<256, MODE_, 2, false, true>(ctx, p, maps, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s);         \
   if (ctx->use_pairs && (MROWS_) > BM && (p.force_bn == 0 || p.force_bn >= 128))                \
-    return share ? launch_mode<256, MODE_, 2, true>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s)         \
-                 : launch_mode<256, MODE_, 2, false>(ctx, p, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s);
+    return share ? launch_mode<256, MODE_, 2, true>(ctx, p, maps, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s)         \
+                 : launch_mode<256, MODE_, 2, false>(ctx, p, maps, cdiv((MROWS_), 2 * BM) * cdiv((NCOLS_), 128), s);
 
   if (kind == ARD_ROW) {
     if (op == OP_FWD) {
@@ -1512,24 +1543,24 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
     const int rows = (op == OP_BWD_WEIGHT) ? p.N : p.B;
     const bool pairs = ctx->use_pairs && rows > BM;
     if (op == OP_FWD)
-      return pairs ? launch_mode<256, M_TILEC_FWD, 2>(ctx, p, many, s) : launch_mode<256, M_TILEC_FWD, 1>(ctx, p, many, s);
+      return pairs ? launch_mode<256, M_TILEC_FWD, 2>(ctx, p, maps, many, s) : launch_mode<256, M_TILEC_FWD, 1>(ctx, p, maps, many, s);
     if (op == OP_BWD_DATA)
-      return pairs ? launch_mode<256, M_TILEC_BWD_DATA, 2>(ctx, p, many, s)
-                   : launch_mode<256, M_TILEC_BWD_DATA, 1>(ctx, p, many, s);
-    return pairs ? launch_mode<256, M_TILEC_BWD_WEIGHT, 2>(ctx, p, many, s)
-                 : launch_mode<256, M_TILEC_BWD_WEIGHT, 1>(ctx, p, many, s);
+      return pairs ? launch_mode<256, M_TILEC_BWD_DATA, 2>(ctx, p, maps, many, s)
+                   : launch_mode<256, M_TILEC_BWD_DATA, 1>(ctx, p, maps, many, s);
+    return pairs ? launch_mode<256, M_TILEC_BWD_WEIGHT, 2>(ctx, p, maps, many, s)
+                 : launch_mode<256, M_TILEC_BWD_WEIGHT, 1>(ctx, p, maps, many, s);
   } else {
     // List form with at least two 128-row tiles of output and 128-wide pattern tiles: CTA pairs (256 x 128
     // tiles; each CTA stages half of the kept block, the instruction is the wide one).
     const bool pairs = ctx->use_pairs && p.B > BM && bn == 128;
     if (op == OP_FWD) {
       const int mt = cdiv(p.B, BM);
-      if (pairs) return launch_mode<128, M_TILE_FWD, 2>(ctx, p, cdiv(p.B, 2 * BM) * cdiv(p.N, 128), s);
+      if (pairs) return launch_mode<128, M_TILE_FWD, 2>(ctx, p, maps, cdiv(p.B, 2 * BM) * cdiv(p.N, 128), s);
       ARD_TC_CASE(128, M_TILE_FWD, mt * cdiv(p.N, 128))
       ARD_TC_CASE(64, M_TILE_FWD, mt * cdiv(p.N, 64))
     } else if (op == OP_BWD_DATA) {
       const int mt = cdiv(p.B, BM);
-      if (pairs) return launch_mode<128, M_TILE_BWD_DATA, 2>(ctx, p, cdiv(p.B, 2 * BM) * cdiv(p.K, 128), s);
+      if (pairs) return launch_mode<128, M_TILE_BWD_DATA, 2>(ctx, p, maps, cdiv(p.B, 2 * BM) * cdiv(p.K, 128), s);
       ARD_TC_CASE(128, M_TILE_BWD_DATA, mt * cdiv(p.K, 128))
       ARD_TC_CASE(64, M_TILE_BWD_DATA, mt * cdiv(p.K, 64))
     } else {
@@ -1550,8 +1581,7 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
 ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_t* ridx, const void* gA, int ldgA,
                           const void* gB, int ldgB, cudaStream_t s) {
   TcParams p = {};
-  p.mapA = nullptr;
-  p.mapB = a.mapB;
+  const TcMap maps[2] = {a.mapB, a.mapB};  // only the weight arrives by TMA
   p.hdr = a.g.hdr;
   p.B = a.g.B;
   p.K = a.g.K;
@@ -1570,19 +1600,21 @@ ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_
   p.ldgA = ldgA;
   p.gB = reinterpret_cast<const __nv_bfloat16*>(gB);
   p.ldgB = ldgB;
-  if (op == OP_FWD) return launch_mode<256, M_ROWS_FWD, 1>(ctx, p, cdiv(p.B, BM) * cdiv(p.N, 64), s);
-  if (op == OP_BWD_DATA) return launch_mode<256, M_ROWS_BWD_DATA, 1>(ctx, p, cdiv(p.B, BM) * cdiv(p.K, 64), s);
-  return launch_mode<256, M_ROWS_BWD_WEIGHT, 1>(ctx, p, cdiv(p.N, BM) * cdiv(p.K, 64), s);
+  if (op == OP_FWD) return launch_mode<256, M_ROWS_FWD, 1>(ctx, p, maps, cdiv(p.B, BM) * cdiv(p.N, 64), s);
+  if (op == OP_BWD_DATA) return launch_mode<256, M_ROWS_BWD_DATA, 1>(ctx, p, maps, cdiv(p.B, BM) * cdiv(p.K, 64), s);
+  return launch_mode<256, M_ROWS_BWD_WEIGHT, 1>(ctx, p, maps, cdiv(p.N, BM) * cdiv(p.K, 64), s);
 }
 
 // LSTM gate products (single CTA per tile; the batch of a recurrent step is small).
 ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStream_t s) {
   TcParams p = {};
-  p.mapA = a.mapA;
-  p.mapB = a.mapB;
-  for (int g = 0; g < 4; ++g) { p.mapA4[g] = a.mapA4[g]; p.mapB4[g] = a.mapB4[g]; }
-  p.mapA_indexed = a.mapA_indexed;
-  p.mapB_indexed = a.mapB_indexed;
+  TcMap maps[10];
+  maps[0] = a.mapA;
+  maps[1] = a.mapB;
+  for (int g = 0; g < 4; ++g) { maps[2 + g] = a.mapA4[g]; maps[6 + g] = a.mapB4[g]; }
+  // the per-gate descriptors carry the pattern; A and B themselves are used only where they are plain
+  p.mapA_indexed = 0;
+  p.mapB_indexed = 0;
   p.hdr = a.g.hdr;
   p.idx = a.g.idx;
   p.col_ptr = p.col_idx = p.row_ptr = p.row_idx = nullptr;
@@ -1610,13 +1642,13 @@ ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStrea
   p.act = nullptr;
   p.ldact = 0;
   const int mt = cdiv(p.B, BM);
-  if (!backward) return launch_mode<256, M_LSTM_FWD, 1>(ctx, p, mt * cdiv(p.N, 64), s);
+  if (!backward) return launch_mode<256, M_LSTM_FWD, 1>(ctx, p, maps, mt * cdiv(p.N, 64), s);
   if (backward == 2) {
     // weight gradient of the four gate blocks: p.B = rows summed over, p.N = H units per gate
     p.zero_fill = a.g.flag1;
     if (ctx->use_pairs && p.N > BM && (p.force_bn == 0 || p.force_bn >= 128))
-      return launch_mode<256, M_LSTM_BWD_WEIGHT, 2>(ctx, p, 4 * cdiv(p.N, 2 * BM) * cdiv(p.K, 128), s);
-    return launch_mode<256, M_LSTM_BWD_WEIGHT, 1>(ctx, p, 4 * cdiv(p.N, BM) * cdiv(p.K, 64), s);
+      return launch_mode<256, M_LSTM_BWD_WEIGHT, 2>(ctx, p, maps, 4 * cdiv(p.N, 2 * BM) * cdiv(p.K, 128), s);
+    return launch_mode<256, M_LSTM_BWD_WEIGHT, 1>(ctx, p, maps, 4 * cdiv(p.N, BM) * cdiv(p.K, 64), s);
   }
-  return launch_mode<256, M_LSTM_BWD_DATA, 1>(ctx, p, mt * cdiv(p.K, 64), s);
+  return launch_mode<256, M_LSTM_BWD_DATA, 1>(ctx, p, maps, mt * cdiv(p.K, 64), s);
 }

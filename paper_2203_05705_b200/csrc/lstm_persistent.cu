@@ -46,8 +46,9 @@ constexpr int LP_ZS_BYTES = 128 * LP_ZS_LD * 4;
 constexpr int LP_PAIRS_MAX = (128 * LP_UNITS + LP_MATH - 1) / LP_MATH;  // (row, unit) pairs per thread
 
 struct LstmFwdParams {
-  const CUtensorMap* mapXH;    // [(T+1)*B][I+H], boxes of 64 rows x 64 columns
-  const CUtensorMap* mapW[4];  // per gate: table over (dp, b) of strided-row maps, boxes of 8 rows x 64 columns
+  TcMap mapXH;    // [(T+1)*B][I+H], boxes of 64 rows x 64 columns (used as encoded)
+  TcMap mapW[4];  // per gate: [H rows][I+H], boxes of 8 rows x 64 columns; specialised to the kept rows by the kernel
+  CUtensorMap* tm_slots;  // this launch's descriptor scratch: ARD_TM_LSTM_SLOTS slots per block
   const int32_t* hdr;
   int T, B, I, H;
   int kx0, klen;      // contraction columns [kx0, kx0 + klen) of [x | h] this kernel multiplies
@@ -89,7 +90,7 @@ __device__ bool grid_wait(const unsigned int* bar, unsigned int target, volatile
 __device__ __forceinline__ float sigmoid_fast(float x) { return 1.f / (1.f + __expf(-x)); }
 __device__ __forceinline__ float tanh_fast(float x) { return 1.f - 2.f / (1.f + __expf(2.f * x)); }
 
-__global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const LstmFwdParams p) {
+__global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const __grid_constant__ LstmFwdParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -151,19 +152,24 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
       // ===================== weight loader and barrier relay =====================
       // Loads the weight slice (lane = contraction block), then relays the grid barrier of every step to
       // the warps of this CTA through a shared-memory barrier.
-      const int e = p.hdr[HDR_MAPIDX];
-      const int kb = lane;
-      if (kb < nkb) {
+      // The gates' weight descriptors become those of the kept rows (the weight area, still empty, is the work area).
+      CUtensorMap* slots = p.tm_slots + (size_t)blockIdx.x * ARD_TM_LSTM_SLOTS;
+      const CUtensorMap* mapW[4];
 #pragma unroll
-        for (int g = 0; g < 4; ++g) tensormap_acquire(p.mapW[g] + e);
+      for (int g = 0; g < 4; ++g)
+        mapW[g] = tensormap_specialise(&p.mapW[g], dp, bb + 1, n_keep, smem + (sW - base) + 128 * g, slots + g, lane);
+      fence_proxy_async_smem();
+      const int kb = lane;
+      if (kb < nkb && dp > 1) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) tensormap_acquire(mapW[g]);
       }
       if (lane == 0) mbar_arrive_expect_tx(wfull_bar, (uint32_t)nkb * LP_W_BLOCK);
       __syncwarp();
       if (kb < nkb) {
 #pragma unroll
         for (int g = 0; g < 4; ++g)
-          tma_load_2d(sW + kb * LP_W_BLOCK + g * (LP_UNITS * LP_BK * 2), p.mapW[g] + e, wfull_bar, p.kx0 + kb * LP_BK,
-                      j0);
+          tma_load_2d(sW + kb * LP_W_BLOCK + g * (LP_UNITS * LP_BK * 2), mapW[g], wfull_bar, p.kx0 + kb * LP_BK, j0);
       }
       if (lane == 0) {
         for (int t = 1; t < p.T; ++t) {
@@ -184,7 +190,7 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
       const int kb0 = g * gsz, kb1 = min(nkb, kb0 + gsz);
       const int kb = kb0 + lane;
       const bool mine = kb < kb1;
-      if (mine) tensormap_acquire(p.mapXH);
+      const CUtensorMap* mapXH = &p.mapXH.tm;  // a kernel parameter, used as encoded
       const uint32_t idesc = make_idesc(LP_N, false, false, 128);
       bool ok = (lane != 0) || mbar_wait(wfull_bar, 0u, abort_flag, p.status);
       for (int t = 0; t < p.T; ++t) {
@@ -196,7 +202,7 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const L
         __syncwarp();
         auto issue = [&]() {
           for (int rb = 0; rb < row_boxes; ++rb)
-            tma_load_2d(sA + kb * a_block + rb * LP_ROW_BOX, p.mapXH, gfull_bar(g), p.kx0 + kb * LP_BK,
+            tma_load_2d(sA + kb * a_block + rb * LP_ROW_BOX, mapXH, gfull_bar(g), p.kx0 + kb * LP_BK,
                         t * p.B + rb * 64);
         };
         if (mine && kb < xblocks) issue();  // columns of x do not depend on the recurrence
@@ -374,8 +380,9 @@ constexpr int LB_MATH = 352;
 constexpr int LB_PAIRS_MAX = (128 * LB_OWN + LB_MATH - 1) / LB_MATH;
 
 struct LstmBwdParams {
-  const CUtensorMap* mapDZ[4];  // per gate: tables over (dp, b) of [T*B rows][n_keep columns], boxes 64 x 64
-  const CUtensorMap* mapW[4];   // per gate: tables of strided-row maps over [n_keep rows][I+H columns], boxes 64 x 64
+  TcMap mapDZ[4];  // per gate: [T*B rows][H columns], boxes 64 x 64; the kernel limits them to the n_keep compact columns
+  TcMap mapW[4];   // per gate: [H rows][I+H columns], boxes 64 x 64; the kernel turns them into the kept rows
+  CUtensorMap* tm_slots;  // this launch's descriptor scratch: ARD_TM_LSTM_SLOTS slots per block
   const int32_t* hdr;
   int T, B, I, H;
   float alpha;
@@ -390,7 +397,7 @@ struct LstmBwdParams {
   int* status;
 };
 
-__global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const LstmBwdParams p) {
+__global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const __grid_constant__ LstmBwdParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -434,7 +441,11 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
   pdl_wait_prior_grids();
 
   const int dp = p.hdr[HDR_DP], bb = p.hdr[HDR_B] - 1, n_keep = p.hdr[HDR_NKEEP];
-  const int e = p.hdr[HDR_MAPIDX];
+  // Descriptors of this pattern: slots 0-3 the gates' kept weight rows, 4-7 the gates' compact gradient columns.
+  // Warp 11 writes them (below) before its first arrival on hready_bar; the loading lanes acquire them after
+  // their first wait on that barrier.
+  CUtensorMap* slots = p.tm_slots + (size_t)blockIdx.x * ARD_TM_LSTM_SLOTS;
+  auto map_of = [&](const TcMap* m, int slot) -> const CUtensorMap* { return dp == 1 ? &m->tm : slots + slot; };
   const int n_cta = (int)gridDim.x;
   const int s_idx = (int)blockIdx.x / LB_KPARTS, r_idx = (int)blockIdx.x % LB_KPARTS;
   const int c0 = s_idx * LB_COLS;                       // first weight column (hidden unit) of the slice
@@ -448,13 +459,21 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
 
   if (warp == 11) {
     // ===================== weight loader and barrier relay =====================
+    // the weight area, still empty, is the work area of the eight descriptors
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      tensormap_specialise(&p.mapW[g], dp, bb + 1, n_keep, smem + (sW - base) + 128 * g, slots + g, lane);
+      tensormap_specialise(&p.mapDZ[g], dp, bb + 1, n_keep, smem + (sW - base) + 128 * (4 + g), slots + 4 + g, lane);
+    }
+    fence_proxy_async_smem();
     const int kb = lane;
     if (kb < nblk) {
       const int blk = blk0 + kb, g = blk / nb, jb = blk - g * nb;
-      tensormap_acquire(p.mapW[g] + e);
+      const CUtensorMap* mw = map_of(&p.mapW[g], g);
+      if (dp > 1) tensormap_acquire(mw);
       if (lane == 0) mbar_arrive_expect_tx(wfull_bar, (uint32_t)nblk * LB_W_BLOCK);
       __syncwarp(__activemask());
-      tma_load_2d(sW + kb * LB_W_BLOCK, p.mapW[g] + e, wfull_bar, p.I + c0, jb * 64);
+      tma_load_2d(sW + kb * LB_W_BLOCK, mw, wfull_bar, p.I + c0, jb * 64);
     }
     __syncwarp();
     if (lane == 0) {
@@ -474,21 +493,22 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
       const int blk = blk0 + kb;
       gate = blk / nb;
       jb = blk - gate * nb;
-      tensormap_acquire(p.mapDZ[gate] + e);
     }
+    const CUtensorMap* mdz = map_of(&p.mapDZ[gate], 4 + gate);
     const uint32_t idesc = make_idesc(LB_COLS, false, true, 128);
     bool ok = (lane != 0) || nblk == 0 || mbar_wait(wfull_bar, 0u, abort_flag, p.status);
     for (int k = 1; k <= T; ++k) {
       // dz of time index T - k is complete
       if (ok && !mbar_wait(hready_bar, (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
       if (!__all_sync(0xffffffffu, ok)) break;
+      if (k == 1 && mine && dp > 1) tensormap_acquire(mdz);  // written by warp 11 ahead of its first arrival on hready_bar
       if (kb0 < kb1) {
         asm volatile("fence.proxy.async.global;" ::: "memory");  // generic-proxy stores of other CTAs -> TMA reads
         if (lane == 0) mbar_arrive_expect_tx(gfull_bar(g4), (uint32_t)(kb1 - kb0) * a_block);
         __syncwarp();
         if (mine)
           for (int rb = 0; rb < row_boxes; ++rb)
-            tma_load_2d(sA + kb * a_block + rb * LP_ROW_BOX, p.mapDZ[gate] + e, gfull_bar(g4), jb * 64,
+            tma_load_2d(sA + kb * a_block + rb * LP_ROW_BOX, mdz, gfull_bar(g4), jb * 64,
                         (T - k) * p.B + rb * 64);
         if (lane == 0) {
           if (!mbar_wait(gfull_bar(g4), (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
@@ -695,11 +715,13 @@ bool lstm_persistent_fits(ard_ctx* ctx, int B, int klen, int H) {
 }
 
 ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H,
-                                          int kx0, int klen, int add_zx, float alpha, const CUtensorMap* mapXH, const CUtensorMap* const mapW[4],
+                                          int kx0, int klen, int add_zx, float alpha, const TcMap& mapXH, const TcMap mapW[4],
                                           void* XH, const float* bias, float* C, float* G, cudaStream_t s) {
+  if ((H + LP_UNITS - 1) / LP_UNITS > ARD_TM_LSTM_BLOCKS) return ARD_ERR_UNSUPPORTED;
   LstmFwdParams p;
   p.mapXH = mapXH;
   for (int g = 0; g < 4; ++g) p.mapW[g] = mapW[g];
+  p.tm_slots = ctx->d_tm_slots + (size_t)ARD_TM_SM_MAX * ARD_TM_SLOTS;
   p.hdr = pat->d_hdr;
   p.T = T; p.B = B; p.I = I; p.H = H;
   p.kx0 = kx0; p.klen = klen; p.add_zx = add_zx;
@@ -764,11 +786,13 @@ bool lstm_persistent_bwd_fits(ard_ctx* ctx, int B, int H) {
 }
 
 ard_status launch_lstm_backward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
-                                           const CUtensorMap* const mapDZ[4], const CUtensorMap* const mapW[4],
+                                           const TcMap mapDZ[4], const TcMap mapW[4],
                                            const float* C, const float* G, const float* dH_last, float* D, float* dc,
                                            void* DZ, cudaStream_t s) {
+  if ((H + LB_COLS - 1) / LB_COLS * LB_KPARTS > ARD_TM_LSTM_BLOCKS) return ARD_ERR_UNSUPPORTED;
   LstmBwdParams p;
   for (int g = 0; g < 4; ++g) { p.mapDZ[g] = mapDZ[g]; p.mapW[g] = mapW[g]; }
+  p.tm_slots = ctx->d_tm_slots + (size_t)ARD_TM_SM_MAX * ARD_TM_SLOTS;
   p.hdr = pat->d_hdr;
   p.T = T; p.B = B; p.I = I; p.H = H;
   p.alpha = alpha;

@@ -83,6 +83,53 @@ __device__ __forceinline__ void tensormap_acquire(const CUtensorMap* map) {
   asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(map) : "memory");
 }
 
+__device__ __forceinline__ uint32_t sm_id() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%smid;" : "=r"(r));
+  return r;
+}
+
+// Turns the whole-matrix descriptor `m` (a kernel parameter) into the descriptor of the pattern (dp, b, n_keep)
+// and returns the address the TMA instructions of this CTA should use: the parameter itself when nothing
+// changes (a plain descriptor, a dense pattern), else `slot` (global memory written by this CTA only), which
+// receives a copy whose address, extent and row pitch were replaced:
+//   MAP_STRIDED_ROWS  rows b-1, b-1+dp, ...: address + (b-1) rows, n_keep rows, pitch dp rows (Eq. 1);
+//   MAP_COMPACT_COLS  columns 0 .. n_keep-1 (beyond them TMA fills zeros); a dense pattern reads dense_base.
+// Called by all 32 lanes of ONE warp with the same arguments.  `stmp`: 128 bytes of shared memory, 128-byte
+// aligned, not in use by anyone else (callers pass the start of an operand stage before the first load).  Every
+// thread that later issues a copy through the returned address calls tensormap_acquire on it first.
+__device__ __forceinline__ const CUtensorMap* tensormap_specialise(const TcMap* m, int dp, int b, int n_keep,
+                                                                   uint8_t* stmp, CUtensorMap* slot, int lane) {
+  const int variant = m->variant;
+  const bool dense_elsewhere = variant == MAP_COMPACT_COLS && dp == 1 && m->dense_base != nullptr;
+  if (variant == MAP_PLAIN || (dp == 1 && !dense_elsewhere)) return &m->tm;
+  reinterpret_cast<uint32_t*>(stmp)[lane] = reinterpret_cast<const uint32_t*>(&m->tm)[lane];
+  __syncwarp();
+  const uint64_t sdesc = (uint64_t)smem_u32(stmp);
+  if (lane == 0) {
+    if (variant == MAP_STRIDED_ROWS) {
+      const uint64_t addr = reinterpret_cast<uint64_t>(m->base) + (uint64_t)(b - 1) * (uint64_t)m->ld * 2ull;
+      asm volatile("tensormap.replace.tile.global_address.shared::cta.b1024.b64 [%0], %1;" ::"l"(sdesc), "l"(addr) : "memory");
+      asm volatile("tensormap.replace.tile.global_dim.shared::cta.b1024.b32 [%0], 1, %1;" ::"l"(sdesc), "r"(n_keep) : "memory");
+      asm volatile("tensormap.replace.tile.global_stride.shared::cta.b1024.b64 [%0], 0, %1;"
+                   ::"l"(sdesc), "l"((uint64_t)dp * (uint64_t)m->ld * 2ull) : "memory");
+    } else {
+      if (dense_elsewhere) {
+        asm volatile("tensormap.replace.tile.global_address.shared::cta.b1024.b64 [%0], %1;"
+                     ::"l"(sdesc), "l"(reinterpret_cast<uint64_t>(m->dense_base)) : "memory");
+        asm volatile("tensormap.replace.tile.global_stride.shared::cta.b1024.b64 [%0], 0, %1;"
+                     ::"l"(sdesc), "l"((uint64_t)m->dense_ld * 2ull) : "memory");
+      }
+      asm volatile("tensormap.replace.tile.global_dim.shared::cta.b1024.b32 [%0], 0, %1;" ::"l"(sdesc), "r"(n_keep) : "memory");
+    }
+  }
+  __syncwarp();
+  // copy to global memory and release it to the tensor-map proxy at GPU scope (one fused, warp-wide instruction)
+  asm volatile("tensormap.cp_fenceproxy.global.shared::cta.tensormap::generic.release.gpu.sync.aligned [%0], [%1], 128;"
+               ::"l"(slot), "r"((uint32_t)sdesc) : "memory");
+  return slot;
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols)
                : "memory");

@@ -224,7 +224,7 @@ def test_a_captured_step_draws_a_new_pattern_at_every_replay():
 
         side = torch.cuda.Stream()
         with torch.cuda.stream(side):
-            step()                                                  # descriptor tables are built outside the capture
+            step()                                                  # the context creates its side streams outside the capture
         torch.cuda.synchronize()
         assert int(counter.item()) == 1
         counter.zero_()
