@@ -34,8 +34,9 @@ from paper_2203_05705_b200 import inputs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of ard_gemm_tc_kernel, averaged over the three
 # GEMMs of one step of the 8192 x 8192 layer at batch 4096, per period dp, from the ncu captures summarised
-# under profiles/ (dp = 1: fwd 679.5 MB, bwd-data 674.4 MB, bwd-weight 390.3 MB).
-DRAM_TRAFFIC_BY_DP = {"row": {1: 581.0e6}, "tile": {}}
+# under profiles/ (dp = 1: fwd 679.5 MB, bwd-data 674.4 MB, bwd-weight 390.3 MB; dp = 2, 4, 8, 16: the
+# sparse-draw capture).  Periods in between are interpolated linearly in 1/dp, the kept share of the layer.
+DRAM_TRAFFIC_BY_DP = {"row": {1: 581.0e6, 2: 257.0e6, 4: 130.8e6, 8: 71.3e6, 16: 60.5e6}, "tile": {}}
 
 METRIC = "layer fwd+bwd kept TFLOP/s (row pattern, p=0.5)"
 UNIT = "TFLOP/s"
@@ -1158,11 +1159,15 @@ def traffic_per_launch(lb, pats):
     region: the per-period figures of the ncu captures summarised under profiles/ (average of the three products),
     weighted by how often each period was drawn; None for a period that was not captured."""
     tab = DRAM_TRAFFIC_BY_DP.get(lb.wl["kind"], {})
+    if not tab:
+        return None
+    xs = sorted(1.0 / dp for dp in tab)
+    ys = [tab[round(1.0 / x)] for x in xs]
     tot, n = 0.0, 0
     for (dp, _, _) in pats:
-        if dp not in tab:
+        if 1.0 / dp < xs[0] or 1.0 / dp > xs[-1]:
             return None
-        tot += tab[dp]
+        tot += float(np.interp(1.0 / dp, xs, ys))
         n += 1
     return tot / max(n, 1)
 
@@ -1175,7 +1180,8 @@ def roofline_of(h, peaks, clk, lb):
     a = h["achieved"]
     return {"bound": "tensor", "achieved": a, "peak": peak, "unit": "TFLOP/s", "frac": a / peak,
             "traffic": traffic_per_launch(lb, h["pats"]),
-            "traffic_unit": "bytes per launch, mean over the launches of the timed region (ncu captures per period)",
+            "traffic_unit": "bytes per launch, mean over the launches of the timed region (ncu captures at dp = 1, 2, 4, "
+                            "8, 16, interpolated in 1/dp)",
             "peak_source": peaks["source"] + (" burst" if burst else " sustained") + " cuBLAS bf16 8192^3",
             "frac_of_burst": a / peaks["bf16_tflops"], "frac_of_sustained": a / peaks["bf16_tflops_sustained"],
             "frac_of_nominal_2250": a / 2250.0, "kernel": "ard_gemm_tc_kernel", "launches": 3 * lb.args.steps,
@@ -1262,6 +1268,7 @@ def main():
         for _ in range(args.warmup + args.steps):
             lb.gemms(2.0)
         torch.cuda.synchronize()
+        clocks.stop()            # ends the nvidia-smi child: a profiler waits for every child of the command
         if rank == 0:
             print(json.dumps({"forced_dp": args.force_dp, "steps": args.steps, "status": int(ard.ard_last_device_status(lb.ctx))}))
         lb.close()
