@@ -15,10 +15,13 @@ Pins (each lives in tests/test_oracle_*.py):
   gemm.*                   scalar triple loops on tiny shapes; dp=1 == numpy matmul; adjoint identity
   lstm.*                   dp=1 == torch.nn.LSTM (fp64, forward and autograd gradients);
                            kept sub-network == torch.nn.LSTM of hidden size n_k; finite differences
+  lstm_stack.*             torch.nn.LSTM modules (fp64) with the mask applied between them, forward and autograd
+                           gradients; central differences; dropped units' fan-in rows of the next layer get no gradient
   mlp_chain.*              finite differences of the scalar <dZ3, Z3>
   mlp.*                    torch autograd (fp64) on the same network written with library ops; central
                            differences; == mlp_chain without bias; compact-matrix form == masked full width
-  cnn.*                    decisions that do not depend on the sample; binomial law of the region decision;
+  cnn.*                    decisions that do not depend on the sample; binomial law of the region decision; single
+                           values drawn independently by default (variance and joint law of two positions);
                            drop rates of the row sampler; worked row example of Sec. 5.2.1; masked product ==
                            product of the dense small matrix; brute force; adjoint identities
   cnn_blocks.*             block decisions that do not depend on the sample; one block per group == the row
