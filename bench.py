@@ -9,7 +9,8 @@ then the forward, backward-data and backward-weight GEMMs of the layer over the 
 Prints ONE JSON line (rank 0).  Workload `mlp8192_row` (the default) is the large MLP layer of the paper's
 Table-1 sweep scaled to B200: W 8192x8192 bf16, batch 4096, row pattern, p = 0.5, K = the
 maximum-entropy distribution over periods 1..16.  Other workloads (`--workload`): `mlp8192_tile`,
-`mlp4096_tile`, `mlp2048_row` (single layers), `lstm1024` (a step is a whole sequence, forward + BPTT),
+`mlp4096_tile`, `mlp2048_row` (single layers), `lstm1024` (a step is a whole sequence, forward + BPTT), `lstm1024x2_out` (two stacked
+LSTM layers with dropout on the layer outputs only),
 `mlp2048_step` / `mlp8192_step` (a step is a whole training iteration of a stack of layers, replayed from a
 CUDA graph), `conv_rows` (a convolution layer as an im2col product with rows dropped by predicted sensitivity),
 `conv_blocks` (the same layer with blocks of the input matrix dropped).
@@ -63,6 +64,9 @@ WORKLOADS = {
                         t_frac=0.3, threshold=0.5, cap=6, m_prob=0.2, n_prob=0.8),
     # LSTM layer (config 4): a step is one sequence, forward + BPTT, one fresh pattern per sequence
     "lstm1024": dict(config=4, T=35, B=64, I=1024, H=1024, kind="lstm", p=0.5, n_dp=16),
+    # two stacked LSTM layers of that size with dropout on the layer outputs only (the non-recurrent connections):
+    # the second layer's input half contracts over the kept outputs of the first
+    "lstm1024x2_out": dict(config=4, T=35, B=64, dims=[1024, 1024, 1024], kind="lstm_stack", p=0.5, n_dp=16),
 }
 
 def max_entropy_K(p, n_dp):
@@ -382,6 +386,160 @@ def run_lstm(args, wl):
     }
     print(json.dumps(line))
     ard.ard_pattern_destroy(pat)
+    ard.ard_destroy(ctx)
+
+
+def run_lstm_stack(args, wl):
+    """A step is one sequence through the stack: a fresh pattern per layer, forward of all layers, BPTT of all layers."""
+    import torch
+    from paper_2203_05705_b200 import ard
+    from paper_2203_05705_b200.lstm import LstmStack
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    clocks = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+    T, B, dims, p, n_dp = wl["T"], wl["B"], wl["dims"], wl["p"], wl["n_dp"]
+    L = len(dims) - 1
+    bf = torch.bfloat16
+    Ws, Xs = [], None
+    for l in range(L):
+        c4 = inputs.config4(T, B, dims[l], dims[l + 1], l)
+        Ws.append(c4["W"])
+        if l == 0:
+            Xs = c4["X"]
+    dY = inputs.config4(T, B, dims[-2], dims[-1], 0)["dH"]
+    ctx = ard.ard_create(0, 2 * T * B * 4 * max(dims) + 4096)
+    ard.ard_set_distribution(ctx, 0, max_entropy_K(p, n_dp))
+    stack = LstmStack(ctx, T, B, dims, [torch.from_numpy(np.ascontiguousarray(W.T)).to(bf).cuda() for W in Ws])
+    hX = torch.from_numpy(Xs).to(bf).pin_memory()
+    hdY = torch.from_numpy(dY.reshape(T * B, -1)).to(bf).pin_memory()
+    X, dYc = hX.cuda(), hdY.cuda()
+    hY = torch.empty((T * B, dims[-1]), dtype=bf).pin_memory()
+    alphas = [1.0 / (1.0 - p)] * L
+
+    def seq(it, dense=False, host=False):
+        for l in range(L):
+            if dense:
+                ard.ard_pattern_set(ctx, stack.out_pats[l], 1, 1)
+            else:
+                ard.ard_sample_pattern(ctx, stack.out_pats[l], 0, inputs.BASE_SEED, it, 10 + l)
+        if host:
+            X.copy_(hX, non_blocking=True)
+            dYc.copy_(hdY, non_blocking=True)
+        Yc = stack.forward(X, alphas)
+        stack.backward(dYc, alphas)       # the first n_keep columns of dYc are read: a synthetic upstream gradient
+        if host:
+            hY.copy_(Yc, non_blocking=True)
+
+    def timed(n, first, **kw):
+        for w in range(args.warmup):
+            seq(first + w, **kw)
+        torch.cuda.synchronize()
+        out = []
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0 = time.time()
+            e0.record()
+            for i in range(n):
+                seq(first + args.warmup + i, **kw)
+            e1.record()
+            torch.cuda.synchronize()
+            out.append((e0.elapsed_time(e1), t0, time.time()))
+        out.sort()
+        return out[1]
+
+    def kept_flops(its):
+        tot, fr = 0.0, []
+        for it in its:
+            n_in = []
+            for l in range(L):
+                ard.ard_sample_pattern(ctx, stack.out_pats[l], 0, inputs.BASE_SEED, it, 10 + l)
+                n_in.append(ard.ard_pattern_to_host(stack.out_pats[l], 0)[2])
+            for l in range(L):
+                kin = dims[l] if l == 0 else n_in[l - 1]
+                tot += 3 * 2.0 * T * B * (kin + dims[l + 1]) * 4 * dims[l + 1]
+            fr.append([n_in[l] / dims[l + 1] for l in range(L)])
+        return tot, fr
+
+    steps = args.steps
+    l0 = ard.ard_launch_count(ctx)
+    ms, t0, t1 = timed(steps, 0)
+    launches = (ard.ard_launch_count(ctx) - l0) * steps // (3 * steps + args.warmup)
+    clk = clocks.stop(t0, t1)
+    status = ard.ard_last_device_status(ctx)
+    kept, fracs = kept_flops(range(args.warmup, args.warmup + steps))
+    dense_flops = sum(3 * 2.0 * T * B * (dims[l] + dims[l + 1]) * 4 * dims[l + 1] for l in range(L))
+    value = kept / (ms * 1e-3) / 1e12
+    n2 = max(5, steps // 4)
+    ms_dense = timed(n2, 100000, dense=True)[0] / n2
+    ms_e = timed(n2, 200000, host=True)[0] / n2
+    kept_e, _ = kept_flops(range(200000 + args.warmup, 200000 + args.warmup + n2))
+    ms_lib = None
+    try:
+        ref = torch.nn.LSTM(dims[0], dims[1], num_layers=L, bias=True, dropout=p).to(device="cuda", dtype=bf)
+        ref.train()
+        ref.flatten_parameters()
+        Xr = X.clone().requires_grad_(True)
+        dHr = dYc.reshape(T, B, -1)
+
+        def lib_seq():
+            for prm in ref.parameters():
+                prm.grad = None
+            Xr.grad = None
+            out, _ = ref(Xr)
+            out.backward(dHr)
+
+        for _ in range(args.warmup):
+            lib_seq()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n2):
+            lib_seq()
+        e1.record()
+        torch.cuda.synchronize()
+        ms_lib = e0.elapsed_time(e1) / n2
+    except Exception as ex:  # the library baseline is context only
+        sys.stderr.write("torch.nn.LSTM baseline skipped: %r\n" % (ex,))
+    peaks = load_peaks()
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import lstm_stack as OS
+        from oracle import pattern as OP
+        masks = [OP.row_mask(dims[l + 1], 2, 1) for l in range(L)]
+        tc0 = time.perf_counter()
+        fw = OS.fwd(Xs, Ws, None, masks, alphas)
+        OS.bwd(fw, Ws, masks, alphas, dY)
+        dt = time.perf_counter() - tc0
+        try:
+            from threadpoolctl import threadpool_info
+            threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        except Exception:
+            threads = os.cpu_count() or 1
+        fl = sum(3 * 2.0 * T * B * ((dims[l] if l == 0 else dims[l] // 2) + dims[l + 1]) * 4 * dims[l + 1] for l in range(L))
+        cpu = {"value": fl / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": "one full sequence through the stack, dp=2 on every layer's output", "seconds": dt}
+    best_dense = min(ms_dense, ms_lib or 1e30)
+    line = {
+        "metric": "stacked LSTM fwd+BPTT kept TFLOP/s (row pattern on every layer's outputs, p=%s)" % p, "value": value,
+        "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": args.warmup, "ms_per_step": ms / steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "T": T, "B": B, "dims": dims, "p": p, "n_dp": n_dp,
+                   "l2": "weights (%d MB) stay in L2 by design; a step is a whole sequence" % (sum(w.size for w in Ws) * 2 // 2 ** 20)},
+        "dense_equiv_tflops": dense_flops * steps / (ms * 1e-3) / 1e12, "clocks": clk,
+        "e2e": {"value": kept_e / n2 / (ms_e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": hX.numel() * 2 + hdY.numel() * 2,
+                "d2h_bytes_per_step": hY.numel() * 2, "ms_per_step": ms_e},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "achieved": value, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                     "frac": value / peaks["bf16_tflops"], "traffic": None,
+                     "note": "35 dependent steps of a 64-row product per layer: bound by per-step latency, not by the tensor "
+                             "pipe; only the input half of the upper layer shrinks with the pattern"},
+        "cpu_baseline": cpu,
+        "detail": {"dense_ms_per_step": {"own_kernels_dp1": ms_dense, "torch_nn_lstm_2_layers_dropout": ms_lib},
+                   "speedup_vs_dense": {str(p): best_dense / (ms / steps)},
+                   "kept_fraction_of_outputs": {str(p): [float(x) for x in np.mean(np.array(fracs), axis=0)]}},
+        "device_status": int(status),
+    }
+    print(json.dumps(line))
+    stack.close()
     ard.ard_destroy(ctx)
 
 
@@ -1234,6 +1392,8 @@ def main():
         return run_reference(args, wl)
     if wl["kind"] == "lstm":
         return run_lstm(args, wl)
+    if wl["kind"] == "lstm_stack":
+        return run_lstm_stack(args, wl)
     if wl["kind"] == "mlp_step":
         return run_mlp_step(args, wl)
     if wl["kind"] == "conv_rows":

@@ -588,6 +588,46 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
                              const void* XH, const void* W, int ldw, const float* C, const float* G,
                              const float* dH_last, float* D, float* dc, void* DZ, float* dW, void* cuda_stream);
 
+/* ---- stacked LSTM with dropout on the layer OUTPUTS only (second reading of the LSTM experiment of Sec. 7) ----
+ * The paper prints no LSTM equations; its LSTM networks are stacks of two and three layers.  In this reading every
+ * unit of a layer is computed at every step, the recurrent path is left alone, and a row pattern (Sec. 3.1, Eq. 1),
+ * one per layer and iteration, masks what the layer hands to its consumer:
+ *     y_t = alpha * m .* h_t.
+ * A dropped unit multiplies its fan-in row of the consumer's weight by zero (Sec. 3.1: the matching rows of the
+ * next layer's weight matrix), so the consumer contracts over kept units only: the layer's output leaves as the
+ * compact matrix Yc [T*B][n_keep] (ard_compact_cols of the h halves of XH), the input half of the next layer's gate
+ * product is ard_layer_fwd over Yc with that pattern as in_pat and the weight packed by ard_compact_weight_cols,
+ * and the recurrence runs from those pre-activations (ard_lstm_forward_from_gates).  Backward: the gradient of Yc
+ * is expanded to full width with the rescale (ard_expand_cols) into D / dH_last, ard_lstm_backward_recurrent gives
+ * the gate gradients DZ and the weight gradient of the recurrent half, and the input half is
+ * ard_layer_bwd_data / ard_layer_bwd_weight over the same compact operands.  The layers themselves use a pattern
+ * that stays dense (never sampled).  paper_2203_05705_b200/lstm.py (LstmStack) holds the buffers and the order of
+ * the calls.
+ *
+ * ard_lstm_forward_from_gates: ard_lstm_forward whose input half is already done: on entry G [T][B][4H] holds
+ *   x-part pre-activations of every step (fp32, e.g. written by ard_layer_fwd with ARD_FLAG_OUT_F32); the x halves
+ *   of XH are not read.  Only the one-kernel recurrence exists for this form: ARD_ERR_UNSUPPORTED when the layer
+ *   does not fit it (see ard_lstm_forward) or I < 1.
+ * ard_lstm_backward_recurrent: ard_lstm_backward without the input half: computes DZ and dW[:, I : I+H] (all 4H
+ *   rows; columns 0 .. I-1 of dW and the x halves of D are left untouched).  ARD_ERR_UNSUPPORTED when the layer
+ *   does not fit the one-kernel recurrence. */
+ard_status ard_lstm_forward_from_gates(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                                       void* XH, const void* W, int ldw, const float* bias, float* C, float* G,
+                                       void* cuda_stream);
+ard_status ard_lstm_backward_recurrent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                                       const void* XH, const void* W, int ldw, const float* C, const float* G,
+                                       const float* dH_last, float* D, float* dc, void* DZ, float* dW,
+                                       void* cuda_stream);
+/* Eq. 1 applied to the columns of a matrix.  ard_compact_cols: dst[r][j] = src[r][keep[j]], j < n_keep (the kept
+ * columns side by side; element type dtype).  ard_expand_cols, its adjoint with a rescale:
+ * dst[r][keep[j]] = alpha * src[r][j], every other column of dst [rows][N] zero (src of type src_dtype, dst fp32).
+ * pat: a row pattern over N units.  Errors: ARD_ERR_INVALID_ARG, ARD_ERR_SHAPE (N differs from the pattern's, leading
+ * dimensions too small).  Asynchronous. */
+ard_status ard_compact_cols(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int rows, int N, const void* src,
+                            int ld_src, void* dst, int ld_dst, void* cuda_stream);
+ard_status ard_expand_cols(ard_ctx* ctx, const ard_pattern* pat, ard_dtype src_dtype, int rows, int N, float alpha,
+                           const void* src, int ld_src, float* dst, int ld_dst, void* cuda_stream);
+
 /* Adjoint of ard_lstm_gates.  dh [B][lddh] (fp32; compact, or full width if dh_scatter != 0, in
  * which case only kept columns are read), dc_inout [B][ldc]: in = gradient arriving at c from the
  * next step, out = gradient w.r.t. c_prev.  dZ [B][4*ldz_gate] compact like Z, element type

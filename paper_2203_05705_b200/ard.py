@@ -31,7 +31,7 @@ EXPORTS = [
     "ard_create", "ard_destroy", "ard_set_path", "ard_set_option", "ard_set_tile_n", "ard_set_shared_tail", "ard_set_compact_reuse", "ard_set_distribution", "ard_quantise_distribution", "ard_search_distribution", "ard_get_distribution_cdf",
     "ard_pattern_create", "ard_pattern_destroy", "ard_sample_pattern", "ard_pattern_set",
     "ard_pattern_to_host", "ard_pattern_tile_lists_to_host", "ard_fwd", "ard_bwd_data", "ard_bwd_weight",
-    "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_set_lstm_persistent", "ard_lstm_forward", "ard_lstm_backward", "ard_last_device_status", "ard_status_string", "ard_launch_count",
+    "ard_bwd_data_static_scratch", "ard_lstm_gates", "ard_lstm_gates_bwd", "ard_lstm_gate_gemm", "ard_lstm_gate_gemm_bwd", "ard_set_lstm_persistent", "ard_lstm_forward", "ard_lstm_backward", "ard_lstm_forward_from_gates", "ard_lstm_backward_recurrent", "ard_compact_cols", "ard_expand_cols", "ard_last_device_status", "ard_status_string", "ard_launch_count",
     "ard_layer_fwd", "ard_layer_bwd_data", "ard_layer_bwd_weight", "ard_compact_weight_cols",
     "ard_expand_weight_grad_cols", "ard_bias_grad", "ard_sample_pattern_counter", "ard_mlp_step",
     "ard_rows_create", "ard_rows_destroy", "ard_sensitivity_predict", "ard_rows_set_probability", "ard_rows_sample",
@@ -96,6 +96,10 @@ def lib():
         "ard_lstm_gate_gemm_bwd": [vp, vp, i32, i32, i32, vp, i32, vp, i32, vp, i32, i32, vp],
         "ard_lstm_forward": [vp, vp, i32, i32, i32, i32, f32, vp, vp, i32, vp, vp, vp, vp, vp],
         "ard_lstm_backward": [vp, vp, i32, i32, i32, i32, f32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp],
+        "ard_lstm_forward_from_gates": [vp, vp, i32, i32, i32, i32, f32, vp, vp, i32, vp, vp, vp, vp],
+        "ard_lstm_backward_recurrent": [vp, vp, i32, i32, i32, i32, f32, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp],
+        "ard_compact_cols": [vp, vp, i32, i32, i32, vp, i32, vp, i32, vp],
+        "ard_expand_cols": [vp, vp, i32, i32, i32, f32, vp, i32, vp, i32, vp],
         "ard_lstm_gates": [vp, vp, i32, i32, i32, f32, vp, i32, vp, vp, i32, vp, vp, i32, i32, vp, vp],
         "ard_lstm_gates_bwd": [vp, vp, i32, i32, i32, f32, vp, vp, vp, i32, vp, i32, i32, vp, vp, i32, vp],
         "ard_last_device_status": [vp, vp],
@@ -542,6 +546,27 @@ def ard_lstm_backward(ctx, pat, T, B, I, H, alpha, XH, W, ldw, C, G, dH_last, D,
     _check(lib().ard_lstm_backward(ctx, pat, T, B, I, H, alpha, _ptr(XH), _ptr(W), ldw, _ptr(C), _ptr(G),
                                    _ptr(dH_last), _ptr(D), _ptr(dc), _ptr(DZ), _ptr(dW), _stream(stream)),
            "ard_lstm_backward")
+
+
+def ard_lstm_forward_from_gates(ctx, pat, T, B, I, H, alpha, XH, W, ldw, bias, C, G, stream=None):
+    _check(lib().ard_lstm_forward_from_gates(ctx, pat, T, B, I, H, alpha, _ptr(XH), _ptr(W), ldw, _ptr(bias), _ptr(C),
+                                             _ptr(G), _stream(stream)), "ard_lstm_forward_from_gates")
+
+
+def ard_lstm_backward_recurrent(ctx, pat, T, B, I, H, alpha, XH, W, ldw, C, G, dH_last, D, dc, DZ, dW, stream=None):
+    _check(lib().ard_lstm_backward_recurrent(ctx, pat, T, B, I, H, alpha, _ptr(XH), _ptr(W), ldw, _ptr(C), _ptr(G),
+                                             _ptr(dH_last), _ptr(D), _ptr(dc), _ptr(DZ), _ptr(dW), _stream(stream)),
+           "ard_lstm_backward_recurrent")
+
+
+def ard_compact_cols(ctx, pat, dtype, rows, N, src, ld_src, dst, ld_dst, stream=None):
+    _check(lib().ard_compact_cols(ctx, pat, dtype, rows, N, _ptr(src), ld_src, _ptr(dst), ld_dst, _stream(stream)),
+           "ard_compact_cols")
+
+
+def ard_expand_cols(ctx, pat, src_dtype, rows, N, alpha, src, ld_src, dst, ld_dst, stream=None):
+    _check(lib().ard_expand_cols(ctx, pat, src_dtype, rows, N, alpha, _ptr(src), ld_src, _ptr(dst), ld_dst,
+                                 _stream(stream)), "ard_expand_cols")
 
 
 def ard_lstm_gates(ctx, pat, h_dtype, B, H, alpha, Z, ldz_gate, bias, c_prev, ldc, c, h, ldh, h_scatter,

@@ -1020,10 +1020,12 @@ ard_status ard_lstm_gates_bwd(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dz
 }
 
 // Whole-sequence drivers: the time loop runs here, in native code, and only enqueues kernels.
-ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha, void* XH,
-                            const void* W, int ldw, const float* bias, float* C, float* G, float* Z,
-                            void* cuda_stream) {
-  if (!ctx || !pat || !XH || !W || !C || !G || !Z) return ARD_ERR_INVALID_ARG;
+// gates_ready: the input half of every step's pre-activations is already in G (the caller multiplied it, e.g. over
+// the kept outputs of the layer below); only the recurrence runs, which needs the one-kernel form.
+static ard_status lstm_forward_impl(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                                    void* XH, const void* W, int ldw, const float* bias, float* C, float* G, float* Z,
+                                    int gates_ready, void* cuda_stream) {
+  if (!ctx || !pat || !XH || !W || !C || !G || (!Z && !gates_ready)) return ARD_ERR_INVALID_ARG;
   if (T < 0 || B < 0 || I < 0 || H < 1) return ARD_ERR_INVALID_ARG;
   const int KH = I + H;
   __nv_bfloat16* xh = reinterpret_cast<__nv_bfloat16*>(XH);
@@ -1043,7 +1045,7 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
       TcMap mapXH;
       TcMap mapW[4];
       // 1. The input half for all steps at once: G[t][:, g*H + j] = x_t . W[g*H + keep[j]][0:I]  (T*B rows).
-      if (I > 0) {
+      if (I > 0 && !gates_ready) {
         TcArgs t = {};
         GemmArgs g = {};
         fill_common(g, ctx, pat, T * B, I, H, 1.0f);
@@ -1080,6 +1082,7 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
       // not launchable as one kernel right now: the per-step path below recomputes everything
     }
   }
+  if (gates_ready) return ARD_ERR_UNSUPPORTED;  // the per-step path multiplies [x, h] as one operand
   for (int t = 0; t < T; ++t) {
     __nv_bfloat16* xh_t = xh + (size_t)t * B * KH;
     __nv_bfloat16* h_out = xh + (size_t)(t + 1) * B * KH + I;  // h_t lands in the operand of step t+1
@@ -1092,9 +1095,25 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
   return ARD_OK;
 }
 
-ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
-                             const void* XH, const void* W, int ldw, const float* C, const float* G,
-                             const float* dH_last, float* D, float* dc, void* DZ, float* dW, void* cuda_stream) {
+ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha, void* XH,
+                            const void* W, int ldw, const float* bias, float* C, float* G, float* Z,
+                            void* cuda_stream) {
+  return lstm_forward_impl(ctx, pat, T, B, I, H, alpha, XH, W, ldw, bias, C, G, Z, 0, cuda_stream);
+}
+
+ard_status ard_lstm_forward_from_gates(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                                       void* XH, const void* W, int ldw, const float* bias, float* C, float* G,
+                                       void* cuda_stream) {
+  if (I < 1) return ARD_ERR_INVALID_ARG;
+  return lstm_forward_impl(ctx, pat, T, B, I, H, alpha, XH, W, ldw, bias, C, G, nullptr, 1, cuda_stream);
+}
+
+// recurrent_only: the recurrence (gate gradients DZ) and the weight gradient of the recurrent half,
+// dW[:, I : I+H]; the input half (dx and dW[:, 0 : I]) is left to the caller.  Needs the one-kernel form.
+static ard_status lstm_backward_impl(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                                     const void* XH, const void* W, int ldw, const float* C, const float* G,
+                                     const float* dH_last, float* D, float* dc, void* DZ, float* dW,
+                                     int recurrent_only, void* cuda_stream) {
   if (!ctx || !pat || !XH || !W || !C || !G || !dH_last || !D || !dc || !DZ || !dW) return ARD_ERR_INVALID_ARG;
   if (T < 1 || B < 0 || I < 0 || H < 1) return ARD_ERR_INVALID_ARG;
   const int KH = I + H;
@@ -1126,7 +1145,7 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
       st = launch_lstm_backward_persistent(ctx, pat, T, B, I, H, alpha, mapDZ, mapW, C, G, dH_last, D, dc, DZ, s);
       if (st == ARD_OK) {
         // dx_t for all t: the x halves of D are overwritten
-        st = lstm_gate_gemm_bwd_tc(ctx, pat, T * B, I, H, DZ, H, W, ldw, D, KH, 0, s);
+        if (!recurrent_only) st = lstm_gate_gemm_bwd_tc(ctx, pat, T * B, I, H, DZ, H, W, ldw, D, KH, 0, s);
         if (st != ARD_OK) return st;
         recurrence_done = true;
       } else if (st != ARD_ERR_UNSUPPORTED) {
@@ -1134,6 +1153,7 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
       }
     }
   }
+  if (recurrent_only && !recurrence_done) return ARD_ERR_UNSUPPORTED;
   for (int t = T - 1; t >= 0 && !recurrence_done; --t) {
     const float* dh = (t == T - 1) ? dH_last : D + (size_t)(t + 1) * B * KH + I;
     const int lddh = (t == T - 1) ? H : KH;
@@ -1147,12 +1167,18 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
   }
   // Weight gradient over all T*B rows: the four gate blocks in one tensor-core launch when the operands
   // allow it (the M tiles of the four gates share one tile loop), else one product per gate.
-  if (ctx->path != ARD_PATH_CUDA_CORE && H % 8 == 0 &&
-      tc_eligible(ctx, pat, ARD_BF16, T * B, KH, H, DZ, 4 * H, XH, KH, dW, KH, 4) == ARD_OK) {
+  // (recurrent_only: the columns of the h half alone -- operand, output and fan-in extent start at column I)
+  const int wcol0 = recurrent_only ? I : 0, wcols = recurrent_only ? H : KH;
+  const void* XHw = reinterpret_cast<const __nv_bfloat16*>(XH) + wcol0;
+  float* dWw = dW + wcol0;
+  const bool w_tc = ctx->path != ARD_PATH_CUDA_CORE && H % 8 == 0 && wcols % 8 == 0 && wcol0 % 8 == 0 &&
+                    tc_eligible(ctx, pat, ARD_BF16, T * B, KH, H, DZ, 4 * H, XH, KH, dW, KH, 4) == ARD_OK;
+  if (recurrent_only && !w_tc) return ARD_ERR_UNSUPPORTED;
+  if (w_tc) {
     TcArgs t = {};
     GemmArgs g = {};
-    fill_common(g, ctx, pat, T * B, KH, H, 1.0f);
-    g.A0 = DZ; g.lda0 = 4 * H; g.A1 = XH; g.lda1 = KH; g.out = dW; g.ldo = KH;
+    fill_common(g, ctx, pat, T * B, wcols, H, 1.0f);
+    g.A0 = DZ; g.lda0 = 4 * H; g.A1 = XHw; g.lda1 = KH; g.out = dWw; g.ldo = KH;
     g.flag0 = 1;
     g.flag1 = 1;  // rows of dropped units are written as zero
     g.out_is_f32 = 1;
@@ -1161,7 +1187,7 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
     for (int gate = 0; gate < 4 && st == ARD_OK; ++gate)
       st = get_maps(ctx, dZc + (size_t)gate * H * 2, T * B, H, 4 * H, H, MAP_COMPACT_COLS, pat->dp_bound, 64, 64,
                     &t.mapA4[gate]);
-    if (st == ARD_OK) st = get_maps(ctx, XH, T * B, KH, KH, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);
+    if (st == ARD_OK) st = get_maps(ctx, XHw, T * B, wcols, KH, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);
     if (st != ARD_OK) return st;
     t.mapA = t.mapA4[0];
     t.mapA_indexed = 1;
@@ -1177,6 +1203,39 @@ ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B,
     if (st != ARD_OK) return st;
   }
   return ARD_OK;
+}
+
+ard_status ard_lstm_backward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                             const void* XH, const void* W, int ldw, const float* C, const float* G,
+                             const float* dH_last, float* D, float* dc, void* DZ, float* dW, void* cuda_stream) {
+  return lstm_backward_impl(ctx, pat, T, B, I, H, alpha, XH, W, ldw, C, G, dH_last, D, dc, DZ, dW, 0, cuda_stream);
+}
+
+ard_status ard_lstm_backward_recurrent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
+                                       const void* XH, const void* W, int ldw, const float* C, const float* G,
+                                       const float* dH_last, float* D, float* dc, void* DZ, float* dW,
+                                       void* cuda_stream) {
+  return lstm_backward_impl(ctx, pat, T, B, I, H, alpha, XH, W, ldw, C, G, dH_last, D, dc, DZ, dW, 1, cuda_stream);
+}
+
+ard_status ard_compact_cols(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int rows, int N, const void* src,
+                            int ld_src, void* dst, int ld_dst, void* cuda_stream) {
+  if (!ctx || !pat || pat->ctx != ctx || pat->kind != ARD_ROW || !src || !dst) return ARD_ERR_INVALID_ARG;
+  if (dtype != ARD_F32 && dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (rows < 0 || N != pat->N_dim || ld_src < N || ld_dst < 1) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  return launch_gather_cols(ctx, pat->d_hdr, pat->d_idx, src, ld_src, dst, ld_dst, rows, dtype == ARD_F32 ? 4 : 2, N, 0,
+                            (cudaStream_t)cuda_stream);
+}
+
+ard_status ard_expand_cols(ard_ctx* ctx, const ard_pattern* pat, ard_dtype src_dtype, int rows, int N, float alpha,
+                           const void* src, int ld_src, float* dst, int ld_dst, void* cuda_stream) {
+  if (!ctx || !pat || pat->ctx != ctx || pat->kind != ARD_ROW || !src || !dst) return ARD_ERR_INVALID_ARG;
+  if (src_dtype != ARD_F32 && src_dtype != ARD_BF16) return ARD_ERR_INVALID_ARG;
+  if (rows < 0 || N != pat->N_dim || ld_src < 1 || ld_dst < N) return ARD_ERR_SHAPE;
+  DeviceGuard guard(ctx->device);
+  return launch_expand_cols(ctx, pat->d_hdr, src, ld_src, src_dtype == ARD_BF16, dst, ld_dst, rows, N, alpha,
+                            (cudaStream_t)cuda_stream);
 }
 
 // ---- products over the kept rows of a convolution layer's input matrix (Sec. 5.2.1) -----------------

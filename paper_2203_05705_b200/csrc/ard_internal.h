@@ -237,6 +237,9 @@ ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* i
                               void* dst, int ld_dst, int rows, int elem_bytes, int max_cols, int skip_dense,
                               cudaStream_t s);
 
+ard_status launch_expand_cols(ard_ctx* ctx, const int32_t* hdr, const void* src, int ld_src, int src_is_bf16, float* dst,
+                              int ld_dst, int rows, int N, float alpha, cudaStream_t s);
+
 // Sensitivity-aware row dropout (rows.cu).
 ard_status launch_sensitivity(ard_ctx* ctx, ard_rows* rows, ard_dtype dtype, const void* A, int lda, int Kc, int c,
                               int n_runs, int need, float threshold, uint32_t P_sens, uint32_t P_insens, uint64_t seed,

@@ -19,6 +19,30 @@ __global__ void __launch_bounds__(256) gather_cols_kernel(const int32_t* hdr, co
   for (int r = blockIdx.y; r < rows; r += gridDim.y) dst[(size_t)r * ld_dst + j] = src[(size_t)r * ld_src + col];
 }
 
+// The adjoint of the gather, with a rescale: dst[r][b-1 + j*dp] = alpha * src[r][j] for j < n_keep, every other
+// column of dst zero (fp32 out).  Used to hand a gradient that arrives over kept units only to a consumer that
+// wants it full width (the upstream gradient of an LSTM layer whose outputs were dropped).
+template <typename T>
+__global__ void __launch_bounds__(256) expand_cols_kernel(const int32_t* hdr, const T* src, int ld_src, float* dst,
+                                                          int ld_dst, int rows, int N, float alpha) {
+  pdl_launch_dependents();
+  pdl_wait_prior_grids();
+  const int dp = hdr[HDR_DP], bb = hdr[HDR_B] - 1;
+  const int c = blockIdx.x * 256 + threadIdx.x;
+  if (c >= N) return;
+  const int rel = c - bb;
+  const bool kept = rel >= 0 && rel % dp == 0;
+  const int j = kept ? rel / dp : 0;
+  for (int r = blockIdx.y; r < rows; r += gridDim.y) {
+    float v = 0.f;
+    if (kept) {
+      if (sizeof(T) == 2) v = alpha * __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(src)[(size_t)r * ld_src + j]);
+      else v = alpha * reinterpret_cast<const float*>(src)[(size_t)r * ld_src + j];
+    }
+    dst[(size_t)r * ld_dst + c] = v;
+  }
+}
+
 // Faster form for 2-byte elements with 16-byte aligned rows.  Each warp owns two private slices of
 // shared memory: one bulk copy (the copy engine, not the load unit, whose queue holds about 20 KB of
 // 16-byte requests per SM) brings the source span of a pass into one slice while the warp compacts the
@@ -513,6 +537,21 @@ ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* i
       ARD_CUDA_OK(ard_launch(ctx, gather_cols_kernel<uint32_t>, grid, dim3(256), 0, s, hdr, (const uint32_t*)src, ld_src,
                              (uint32_t*)dst, ld_dst, rows));
   }
+  ctx->launches++;
+  ARD_CUDA_OK(cudaGetLastError());
+  return ARD_OK;
+}
+
+ard_status launch_expand_cols(ard_ctx* ctx, const int32_t* hdr, const void* src, int ld_src, int src_is_bf16, float* dst,
+                              int ld_dst, int rows, int N, float alpha, cudaStream_t s) {
+  if (rows == 0 || N == 0) return ARD_OK;
+  dim3 grid((N + 255) / 256, rows < 2048 ? rows : 2048);
+  if (src_is_bf16)
+    ARD_CUDA_OK(ard_launch(ctx, expand_cols_kernel<uint16_t>, grid, dim3(256), 0, s, hdr, (const uint16_t*)src, ld_src, dst,
+                           ld_dst, rows, N, alpha));
+  else
+    ARD_CUDA_OK(ard_launch(ctx, expand_cols_kernel<float>, grid, dim3(256), 0, s, hdr, (const float*)src, ld_src, dst, ld_dst,
+                           rows, N, alpha));
   ctx->launches++;
   ARD_CUDA_OK(cudaGetLastError());
   return ARD_OK;
