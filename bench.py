@@ -1069,8 +1069,9 @@ def layer_config(args, wl, world):
 
 class LayerBench:
     """One layer (X, W, dY resident on the device), one context, one pattern object; every timing helper of the
-    single-layer workloads.  A step = draw a pattern on the device, forward (full-width output, dropped columns
-    written as zero), backward-data and backward-weight from the full-width dY (compacted once per step)."""
+    single-layer workloads.  A step = draw a pattern on the device, then ard_layer_products: forward (full-width
+    output, dropped columns written as zero), backward-data and backward-weight from the full-width dY (compacted
+    once per step), enqueued side by side on the caller's stream and one stream of the context."""
 
     def __init__(self, torch, ard, args, wl, dev, rank, world, barrier, tensors=None):
         self.torch, self.ard, self.args, self.wl = torch, ard, args, wl
@@ -1129,9 +1130,22 @@ class LayerBench:
         if ev is not None:
             ev[3].record()
 
+    def products(self, alpha, ptr=None, stream=None):
+        """The three products of the layer through the one call that enqueues them side by side."""
+        ard, B, K, N = self.ard, self.B, self.K, self.N
+        q = ptr or self.ptr
+        ard.ard_layer_products(self.ctx, self.pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, alpha, q["X"], K, q["W"], K, q["dY"], N,
+                               q["Y"], N, ard.ARD_OUT_SCATTER_ZEROFILL, q["dX"], K, q["dW"], K, 0,
+                               self.cs if stream is None else stream)
+
     def step(self, pp, it, ev=None, ptr=None):
+        """One step: draw the pattern on the device, then the layer's three products (ard_layer_products; with `ev`,
+        one call per product in sequence so that each can be timed)."""
         self.ard.ard_sample_pattern(self.ctx, self.pat, self.dist_ids[pp], self.seed, it, self.rank, self.cs)
-        self.gemms(1.0 / (1.0 - pp), ev, ptr)
+        if ev is not None:
+            self.gemms(1.0 / (1.0 - pp), ev, ptr)
+        else:
+            self.products(1.0 / (1.0 - pp), ptr)
 
     def patterns_of(self, pp, its):
         """(dp, b, kept units) of the given iterations, read back from the device sampler outside any timed region."""
@@ -1197,6 +1211,7 @@ class LayerBench:
         self.ard.ard_pattern_set(self.ctx, self.pat, 1, 1)
         n = max(5, self.args.steps // 4)
         own = self.time_fn(lambda: self.gemms(1.0), n)
+        own_one = self.time_fn(lambda: self.products(1.0), n)
         X, dY, W = t["X"], t["dY"], t["W"]
         Wt = W.t()
 
@@ -1204,8 +1219,9 @@ class LayerBench:
             torch.matmul(X, Wt); torch.matmul(dY, W); torch.matmul(dY.t(), X)
 
         lib_ms = self.time_fn(lib, n)
-        return {"own_kernels_dp1": statistics.median(own), "torch_matmul": statistics.median(lib_ms),
-                "own_kernels_dp1_all": own, "torch_matmul_all": lib_ms}
+        return {"own_kernels_dp1": min(statistics.median(own), statistics.median(own_one)),
+                "torch_matmul": statistics.median(lib_ms), "own_kernels_dp1_in_sequence_all": own,
+                "own_kernels_dp1_one_call_all": own_one, "torch_matmul_all": lib_ms}
 
     def per_dp_table(self, peak_burst):
         """Every (dp, b) of the distribution's support, forced with ard_pattern_set: per product and for the whole
@@ -1219,7 +1235,7 @@ class LayerBench:
         self.dense_burst = {}
         for dp in range(1, n_dp + 1):
             ms = {nm: [] for nm in names}
-            steps, kept, prods = [], [], []
+            steps, kept, prods, onecall = [], [], [], []
             for b in range(1, dp + 1):
                 ard.ard_pattern_set(self.ctx, self.pat, dp, b, self.cs)
                 kept.append(self.ard.ard_pattern_to_host(self.pat, 0)[2])
@@ -1238,6 +1254,18 @@ class LayerBench:
                         ms[nm].append(ev[j].elapsed_time(ev[j + 1]))
                     steps.append(ev[0].elapsed_time(ev[4]))
                     prods.append(ev[1].elapsed_time(ev[4]))
+                # the same step through ard_layer_products: the three products enqueued side by side
+                t = self.t
+                for rep in range(REPEATS + 1):
+                    ev[0].record()
+                    ard.ard_pattern_set(self.ctx, self.pat, dp, b, self.cs)
+                    ard.ard_layer_products(self.ctx, self.pat, ard.ARD_BF16, ard.ARD_BF16, self.B, self.K, self.N, 2.0, t["X"],
+                                           self.K, t["W"], self.K, t["dY"], self.N, t["Y"], self.N, ard.ARD_OUT_SCATTER_ZEROFILL,
+                                           t["dX"], self.K, t["dW"], self.K, 0, self.cs)
+                    ev[1].record()
+                    torch.cuda.synchronize()
+                    if rep:
+                        onecall.append(ev[0].elapsed_time(ev[1]))
             if dp == 1:
                 # the dense layer, timed the same way (one pass between two synchronisations): this library's three
                 # products without a sampler, and torch.matmul
@@ -1253,7 +1281,8 @@ class LayerBench:
                         lib.append(ev[0].elapsed_time(ev[1]))
                 self.dense_burst = {"own_kernels_dp1": statistics.median(prods), "torch_matmul": statistics.median(lib)}
             fl = self.flops_per_unit() * float(np.mean(kept))
-            row = {"kept_units_mean": float(np.mean(kept)), "step_ms": statistics.median(steps)}
+            row = {"kept_units_mean": float(np.mean(kept)), "step_ms": statistics.median(steps),
+                   "step_one_call_ms": statistics.median(onecall)}
             for nm in names:
                 m = statistics.median(ms[nm])
                 row[nm + "_ms"] = m
@@ -1262,6 +1291,10 @@ class LayerBench:
                     row[nm + "_frac_of_burst"] = row[nm + "_tflops"] / peak_burst
             table[str(dp)] = row
             step_by_dp[dp] = float(np.mean(steps))            # mean over b and repeats: what an expectation needs
+            self.onecall_by_dp = getattr(self, "onecall_by_dp", {})
+            self.onecall_by_dp[dp] = float(np.mean(onecall))
+            if dp == 1:
+                self.dense_burst["own_kernels_dp1_one_call"] = statistics.median(onecall)
             units_by_dp[dp] = float(np.mean(kept))
         return table, step_by_dp, units_by_dp
 
@@ -1284,8 +1317,11 @@ class LayerBench:
         a, wl = self.args, self.wl
         p = wl["p"]
         launches0 = self.ard.ard_launch_count(self.ctx)
-        its, runs = self.repeated(p, 0, per_kernel=True)
+        its, runs = self.repeated(p, 0)
         launches = (self.ard.ard_launch_count(self.ctx) - launches0) * a.steps // (a.steps * REPEATS + a.warmup)
+        # the same iterations once more with one call per product in sequence and an event between the calls: the
+        # per-kernel durations the roofline needs cannot be separated while the products overlap
+        seq_run = self.timed_steps(p, its, per_kernel=True)
         status = self.ard.ard_last_device_status(self.ctx)
         pats = self.patterns_of(p, its)
         kept = [3 * self.flops_per_unit() * nk for (_, _, nk) in pats]
@@ -1301,13 +1337,14 @@ class LayerBench:
         values = [kept_total / (m * 1e-3) / 1e12 for m in ms_all]
         order = sorted(range(REPEATS), key=lambda i: ms_all[i])
         mid = order[REPEATS // 2]
-        per = np.array(runs[mid][1])                     # [steps][3] ms of the median region
+        per = np.array(seq_run[1])                       # [steps][3] ms, products in sequence
         gemm_ms = float(per.sum())
         achieved = sum(kept) / (gemm_ms * 1e-3) / 1e12
         per_op = {nm: {"ms_avg": float(per[:, j].mean()), "tflops": sum(kept) / 3.0 / (float(per[:, j].sum()) * 1e-3) / 1e12}
                   for j, nm in enumerate(["fwd", "bwd_data", "bwd_weight"])}
-        wall = (runs[0][2][0], runs[-1][2][1])
+        wall = (runs[0][2][0], seq_run[2][1])
         return dict(its=its, pats=pats, ms=ms_all[mid], ms_all=ms_all, values=values, value=values[mid],
+                    ms_sequential=seq_run[0],
                     dense_equiv=dense_total / (ms_all[mid] * 1e-3) / 1e12, launches=int(launches), status=int(status),
                     achieved=achieved, per_op=per_op, wall=wall, kept=kept)
 
@@ -1343,7 +1380,10 @@ def roofline_of(h, peaks, clk, lb):
             "peak_source": peaks["source"] + (" burst" if burst else " sustained") + " cuBLAS bf16 8192^3",
             "frac_of_burst": a / peaks["bf16_tflops"], "frac_of_sustained": a / peaks["bf16_tflops_sustained"],
             "frac_of_nominal_2250": a / 2250.0, "kernel": "ard_gemm_tc_kernel", "launches": 3 * lb.args.steps,
-            "per_op": h["per_op"]}
+            "per_op": h["per_op"],
+            "how": "CUDA events between the three product calls of the same iterations issued in sequence right after the "
+                   "headline regions (in those the products overlap on two streams and have no separate durations); "
+                   "%.4f ms per step in sequence" % (h["ms_sequential"] / lb.args.steps)}
 
 
 def sweep_block(lb, peaks, dense):
@@ -1353,6 +1393,7 @@ def sweep_block(lb, peaks, dense):
     best_dense = min(dense["own_kernels_dp1"], dense["torch_matmul"])
     table, step_by_dp, units_by_dp = lb.per_dp_table(peaks["bf16_tflops"])
     exp = lb.expectations(step_by_dp, units_by_dp, min(lb.dense_burst.values()))
+    exp_one = lb.expectations(lb.onecall_by_dp, units_by_dp, min(lb.dense_burst.values()))
     sampled = {}
     for pp in (0.3, 0.5, 0.7):
         its, runs = lb.repeated(pp, 10000 + int(pp * 100) * 1000)
@@ -1360,7 +1401,8 @@ def sweep_block(lb, peaks, dense):
         pats = lb.patterns_of(pp, its)
         sampled[str(pp)] = {"ms_per_step": ms, "speedup_vs_dense": best_dense / ms,
                             "kept_fraction": float(np.mean([nk / lb.units for (_, _, nk) in pats]))}
-    return {"per_dp": table, "dense_ms_single_pass": lb.dense_burst, "expected": exp, "sampled": sampled,
+    return {"per_dp": table, "dense_ms_single_pass": lb.dense_burst, "expected": exp,
+            "expected_products_in_one_call": exp_one, "sampled": sampled,
             "note": "per_dp: median over every offset b and %d repeats, pattern forced with ard_pattern_set; expected: "
                     "sum over dp of k^_dp x mean step time, k^ = the quantised distribution; sampled: %d device-drawn "
                     "steps per rate (a bimodal K makes these noisy; the expectations are the figures to read)"
@@ -1453,7 +1495,7 @@ def main():
     detail["dense_tflops"] = {k2: dense_flops_step / (dense[k2] * 1e-3) / 1e12 for k2 in ("own_kernels_dp1", "torch_matmul")}
     sw = sweep_block(lb, peaks, dense)
     detail.update(sw)
-    detail["speedup_vs_dense"] = {k2: v["expected_speedup"] for k2, v in sw["expected"].items()}
+    detail["speedup_vs_dense"] = {k2: v["expected_speedup"] for k2, v in sw["expected_products_in_one_call"].items()}
     detail["ideal_speedup"] = {k2: v["ideal_speedup"] for k2, v in sw["expected"].items()}
     detail["repeats"] = {"n": REPEATS, "values": h["values"], "ms_per_step": [m / args.steps for m in h["ms_all"]],
                          "spread": (max(h["values"]) - min(h["values"])) / h["value"]}
@@ -1596,11 +1638,8 @@ def main():
                     s_cmp.wait_event(out_done[i - NB])         # Y[k] has been read out
                 sc = s_cmp.cuda_stream
                 ard.ard_sample_pattern(lb.ctx, lb.pat, lb.dist_ids[p], lb.seed, it, rank, sc)
-                ard.ard_fwd(lb.ctx, lb.pat, ard.ARD_BF16, B, K, N, al, Xb[k], K, Wt2, K, Yb[k], N,
-                            ard.ARD_OUT_SCATTER_ZEROFILL, sc)
-                ard.ard_bwd_data(lb.ctx, lb.pat, ard.ARD_BF16, B, K, N, al, dYb[k], N, 0, Wt2, K, dXt, K, sc)
-                ard.ard_bwd_weight(lb.ctx, lb.pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, al, Xb[k], K, dYb[k], N, 0, dWt, K,
-                                   0, sc)
+                ard.ard_layer_products(lb.ctx, lb.pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, al, Xb[k], K, Wt2, K, dYb[k], N,
+                                       Yb[k], N, ard.ARD_OUT_SCATTER_ZEROFILL, dXt, K, dWt, K, 0, sc)
                 cmp_done[i] = s_cmp.record_event()
             with torch.cuda.stream(s_out):
                 s_out.wait_event(cmp_done[i])
