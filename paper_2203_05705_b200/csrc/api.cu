@@ -1263,13 +1263,15 @@ ard_status ard_rows_fwd(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N,
   g.alpha = alpha;
   g.out = Y; g.ldo = ldy;
   g.status = ctx->d_status;
+  st = get_maps(ctx, A, M, K, lda, 0, MAP_PLAIN, 0, 1, 64, &t.mapA);   // gathered: one row of 64 k per piece
+  if (st != ARD_OK) return st;
   st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);  // boxes [64 neurons][64 k]
   if (st != ARD_OK) return st;
   t.g = g;
   t.bn = ctx->force_bn;
   st = launch_zero_dropped_rows(ctx, rows, Y, ldy * 2, N * 2, s);
   if (st != ARD_OK) return st;
-  return launch_rows_tc(ctx, OP_FWD, t, rows->d_idx, A, lda, nullptr, 0, s);
+  return launch_rows_tc(ctx, OP_FWD, t, rows->d_idx, s);
 }
 
 ard_status ard_rows_bwd_data(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha, const void* dY,
@@ -1286,13 +1288,15 @@ ard_status ard_rows_bwd_data(ard_ctx* ctx, const ard_rows* rows, int M, int K, i
   g.alpha = alpha;
   g.out = dA; g.ldo = ldda;
   g.status = ctx->d_status;
+  st = get_maps(ctx, dY, M, N, lddy, 0, MAP_PLAIN, 0, 1, 64, &t.mapA);  // gathered: one row of 64 n per piece
+  if (st != ARD_OK) return st;
   st = get_maps(ctx, W, N, K, ldw, 0, MAP_PLAIN, 0, 64, 64, &t.mapB);  // read MN-major: boxes [64 neurons][64 k]
   if (st != ARD_OK) return st;
   t.g = g;
   t.bn = ctx->force_bn;
   st = launch_zero_dropped_rows(ctx, rows, dA, ldda * 2, K * 2, s);
   if (st != ARD_OK) return st;
-  return launch_rows_tc(ctx, OP_BWD_DATA, t, rows->d_idx, dY, lddy, nullptr, 0, s);
+  return launch_rows_tc(ctx, OP_BWD_DATA, t, rows->d_idx, s);
 }
 
 ard_status ard_rows_bwd_weight(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N, float alpha,
@@ -1311,9 +1315,14 @@ ard_status ard_rows_bwd_weight(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_
   g.out = dW; g.ldo = lddw;
   g.out_is_f32 = dW_dtype == ARD_F32;
   g.status = ctx->d_status;
+  // both operands are gathered along the contraction: pieces of one list row by 64 columns
+  st = get_maps(ctx, dY, M, N, lddy, 0, MAP_PLAIN, 0, 1, 64, &t.mapA);
+  if (st != ARD_OK) return st;
+  st = get_maps(ctx, A, M, K, lda, 0, MAP_PLAIN, 0, 1, 64, &t.mapB);
+  if (st != ARD_OK) return st;
   t.g = g;
   t.bn = ctx->force_bn;
-  return launch_rows_tc(ctx, OP_BWD_WEIGHT, t, rows->d_idx, dY, lddy, A, lda, (cudaStream_t)cuda_stream);
+  return launch_rows_tc(ctx, OP_BWD_WEIGHT, t, rows->d_idx, (cudaStream_t)cuda_stream);
 }
 
 // ---- the same products on compact operands (the dense small matrices of Sec. 5.2.1, step 2) ----------

@@ -52,8 +52,8 @@ enum TcMode {
   M_LSTM_BWD_DATA = 10, // d[x,h] = sum_g dZ[:, g*ldz + j] . W[g*H + keep[j], :]
   M_LSTM_BWD_WEIGHT = 11, // dW[g*H + keep[j], :] = sum_rows dZ[:, g*ldz + j] . [x,h]   (M tiles: gate-major)
   // Products over an index list of kept ROWS of the input matrix (Sec. 5.2.1).  The kept rows follow no
-  // stride, so the producer warp gathers them with 16-byte cp.async copies into the same swizzled layout a
-  // TMA box would have produced; the weight still arrives by TMA.
+  // stride, so the producer warps fetch them four at a time with TMA gather instructions (tile::gather4), which
+  // fill a stage exactly as a box would; the weight arrives in ordinary boxes.
   M_ROWS_FWD = 12,        // Y[idx[j], :]  = A[idx[j], :] . W^T          (A gathered, K-major)
   M_ROWS_BWD_DATA = 13,   // dA[idx[j], :] = dY[idx[j], :] . W           (dY gathered, K-major)
   M_ROWS_BWD_WEIGHT = 14  // dW[n, :] = sum_j dY[idx[j], n] A[idx[j], :] (both gathered, MN-major)
@@ -107,12 +107,8 @@ struct TcParams {
   int relu;
   const void* act;
   int ldact;
-  // Row-list products: the kept-row list and the matrices the producer gathers from.
+  // Row-list products: the kept-row list (the matrices the producers gather from come as descriptors).
   const int32_t* ridx;
-  const __nv_bfloat16* gA;  // forward: A; backward-data: dY; backward-weight: dY
-  int ldgA;
-  const __nv_bfloat16* gB;  // backward-weight: A
-  int ldgB;
   // Row-list products on compact operands (FUSED row kernels): hdr is the row list's header, the layer itself is
   // dense.  1: the row extent of A and of the output is hdr[HDR_NKEEP] and output row m goes to row ridx[m]
   // (forward, backward-data); 2: the contraction runs over hdr[HDR_NKEEP] rows (backward-weight).
@@ -668,8 +664,7 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      // row-list products: one arrival with the TMA byte count plus one arrival per gathering lane
-      mbar_init(full_bar(s), is_rows_mode(MODE) ? 1 + 32 * ROWS_GATHER_WARPS : 1);
+      mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -726,46 +721,33 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
   auto roles = [&](auto plain_tag) {
   constexpr bool PLAIN = decltype(plain_tag)::value;
   if (is_rows_mode(MODE) && (warp == 0 || warp >= 10)) {
-    // ===================== gathering producers (4 warps, all lanes) =====================
-    const int gw = warp == 0 ? 0 : warp - 9;  // 0..3: which quarter of the gathered rows this warp fetches
-    const CUtensorMap* mapB = &p.maps[1].tm;  // the weight, as encoded
+    // ===================== gathering producers (4 warps) =====================
+    // An index list has no stride a TMA box could follow, but the TMA unit takes four arbitrary rows per
+    // instruction (tile::gather4 on a descriptor whose box is one row of 64 columns = 128 bytes high): the four
+    // 128-byte pieces land one after the other, and since the 128-byte swizzle is a function of the shared-memory
+    // address, a run of such instructions fills a stage exactly as one tall box would.  A stage takes 32 (forward,
+    // backward-data: 128 rows of the list) or 16 x (2 + boxes of B) instructions (backward-weight: 64 list rows of
+    // both operands); one thread paces at several hundred cycles per instruction, so they are dealt over the lanes
+    // of four warps.  Rows past the end of the list get an index outside the matrix: TMA fills zeros.
+    const int gw = warp == 0 ? 0 : warp - 9;  // 0..3
+    const CUtensorMap* mapG = &p.maps[0].tm;  // forward: A; backward-data: dY; backward-weight: dY (the A operand)
+    const CUtensorMap* mapB = &p.maps[1].tm;  // the weight (boxes), or for backward-weight A (gathered, the B operand)
+    const int oob = p.B;                      // the first row the gathered matrices do not have
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
     Unit un;
-    // Eight consecutive lanes fetch the eight 16-byte chunks of one row (one 128-byte line), so a warp
-    // instruction asks for four whole lines instead of 32 scattered sectors (the load unit's tag stage was
-    // the limit with one row per lane).  The rows' global addresses are worked out once (per tile, or per
-    // contraction block for the backward-weight product) by the lane that read the list entry and kept in a
-    // small shared-memory table (the staging area of the scatter epilogue is unused in these modes).
-    const int sub = lane >> 3, ch = lane & 7;
-    // this warp's slice of the table: [32] row addresses, or [2 parities][2 operands][16] for backward-weight
-    unsigned long long* rowtab = reinterpret_cast<unsigned long long*>(smem + L::STG_OFF) + gw * 64;
     for (int i = 0; ok && sch.unit(w0, i, un); ++i) {
       const TileInfo ti = sch.template tile<PLAIN>(p, un.t);
-      if (MODE != M_ROWS_BWD_WEIGHT) {
-        __syncwarp();
-        const int m = ti.m0 + gw * 32 + lane;  // this warp fetches tile rows gw*32 .. gw*32 + 31
-        rowtab[lane] = m < sch.M_gemm ? (unsigned long long)(p.gA + (size_t)p.ridx[m] * p.ldgA) : 0ull;
-        __syncwarp();
+      // forward / backward-data: lanes 0..7 of warp gw own the rows 4*(8*gw + lane) .. + 3 of the tile for all blocks
+      int r4[4] = {oob, oob, oob, oob};
+      if (MODE != M_ROWS_BWD_WEIGHT && lane < 8) {
+        const int m = ti.m0 + 4 * (8 * gw + lane);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (m + q < sch.M_gemm) r4[q] = p.ridx[m + q];
       }
-      // backward-weight: list entries of contraction rows lane, lane + 32 of the current block; the next
-      // block's are fetched while this one is being issued (a dependent global load per block otherwise)
-      // (lanes 0..15 own the 16 contraction rows gw*16 .. gw*16 + 15 of a block)
-      int jcur = -1;
-      if (MODE == M_ROWS_BWD_WEIGHT && lane < 16 && gw * 16 + lane < sch.Kc) jcur = p.ridx[gw * 16 + lane];
       for (int kb = 0; kb < ti.nkb; ++kb) {
-        int jnext = -1;
-        unsigned long long* tabA = rowtab + (kb & 1) * 32;  // [16] addresses in dY, then [16] in A
-        if (MODE == M_ROWS_BWD_WEIGHT) {
-          if (lane < 16) {
-            tabA[lane] = jcur >= 0 ? (unsigned long long)(p.gA + (size_t)jcur * p.ldgA) : 0ull;
-            tabA[16 + lane] = jcur >= 0 ? (unsigned long long)(p.gB + (size_t)jcur * p.ldgB) : 0ull;
-            const int j = (kb + 1) * BK + gw * 16 + lane;
-            if (kb + 1 < ti.nkb && j < sch.Kc) jnext = p.ridx[j];
-          }
-          __syncwarp();  // the table entries are read by other lanes below
-        }
         int good = 1;
         if (lane == 0) good = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status) ? 1 : 0;
         good = __shfl_sync(0xffffffffu, good, 0);
@@ -774,10 +756,8 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
         const uint32_t sB = sA + L::A_BYTES;
         const int kx = kb * BK;
         if (warp == 0 && lane == 0) {
-          if (MODE == M_ROWS_BWD_WEIGHT) {
-            mbar_arrive(full_bar(stage));
-          } else {
-            mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(ti.nbox * 64 * BK * 2));
+          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(L::A_BYTES + ti.nbox * 64 * BK * 2));
+          if (MODE != M_ROWS_BWD_WEIGHT) {
 #pragma unroll
             for (int bxi = 0; bxi < 4; ++bxi) {
               if (bxi < ti.nbox) {
@@ -788,44 +768,26 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
           }
         }
         if (MODE != M_ROWS_BWD_WEIGHT) {
-          // [128 rows][64 k], 128 bytes per row, 16-byte chunk c of row r at chunk c ^ (r & 7)
-          const int k = kx + 8 * ch;
-          const bool kin = k < sch.Kc;
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const int rl = 4 * q + sub, r = gw * 32 + rl;
-            const unsigned long long bp = rowtab[rl];
-            const bool in = bp != 0ull && kin;
-            cp_async_16(sA + (uint32_t)r * 128u + (uint32_t)((ch ^ (r & 7)) << 4),
-                        in ? (const void*)(bp + (unsigned long long)k * 2ull) : (const void*)p.gA, in ? 16u : 0u);
-          }
+          // [128 rows][64 k]: rows 4g .. 4g+3 at byte 512 g of the stage
+          if (lane < 8)
+            tma_gather4_2d(sA + (uint32_t)(8 * gw + lane) * 512u, mapG, full_bar(stage), kx, r4[0], r4[1], r4[2], r4[3]);
         } else {
-          // boxes of [64 contraction rows][64 columns]: A operand = dY columns m0.., B operand = A columns n0..
+          // boxes of [64 list rows][64 columns]; item = (group of four list rows g, box): 16 x (2 + nbox) of them
+          const int nitem = 16 * (2 + ti.nbox);
+          for (int it = gw * 32 + lane; it < nitem; it += 32 * ROWS_GATHER_WARPS) {
+            const int g = it & 15, bx = it >> 4;  // bx 0,1: the two 64-column boxes of dY; 2..: the boxes of A
+            const int j = kx + 4 * g;
+            int jr[4];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const int jl = 4 * q + sub, jr = gw * 16 + jl;
-            const unsigned long long pa = tabA[jl], pb = tabA[16 + jl];
-            const uint32_t off = (uint32_t)jr * 128u + (uint32_t)((ch ^ (jr & 7)) << 4);
-#pragma unroll
-            for (int bxi = 0; bxi < BM / 64; ++bxi) {
-              const int col = ti.ax[bxi] + 8 * ch;
-              const bool in = pa != 0ull && col < sch.M_gemm;
-              cp_async_16(sA + (uint32_t)bxi * (64 * BK * 2) + off,
-                          in ? (const void*)(pa + (unsigned long long)col * 2ull) : (const void*)p.gA, in ? 16u : 0u);
-            }
-#pragma unroll
-            for (int bxi = 0; bxi < 4; ++bxi) {
-              if (bxi < ti.nbox) {
-                const int col = ti.bx[bxi] + 8 * ch;
-                const bool in = pb != 0ull && col < sch.N_gemm;
-                cp_async_16(sB + (uint32_t)bxi * (64 * BK * 2) + off,
-                            in ? (const void*)(pb + (unsigned long long)col * 2ull) : (const void*)p.gA, in ? 16u : 0u);
-              }
-            }
+            for (int q = 0; q < 4; ++q) jr[q] = (j + q < sch.Kc) ? p.ridx[j + q] : oob;
+            if (bx < 2)
+              tma_gather4_2d(sA + (uint32_t)bx * (64 * BK * 2) + (uint32_t)g * 512u, mapG, full_bar(stage), ti.ax[bx], jr[0],
+                             jr[1], jr[2], jr[3]);
+            else
+              tma_gather4_2d(sB + (uint32_t)(bx - 2) * (64 * BK * 2) + (uint32_t)g * 512u, mapB, full_bar(stage),
+                             sel4(ti.bx, bx - 2), jr[0], jr[1], jr[2], jr[3]);
           }
         }
-        cp_async_mbar_arrive_noinc(full_bar(stage));
-        jcur = jnext;
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
@@ -955,11 +917,6 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
-          if (is_rows_mode(MODE)) {
-            // the gathered operand was written by ordinary asynchronous copies (generic proxy)
-            fence_proxy_async_smem();
-            tc_fence_after();
-          }
           // This thread's instruction stream is what feeds the tensor pipe: the descriptors of a block are
           // the stage's descriptor plus a constant per 16-deep step (the start-address field counts 16-byte
           // units: K-major 32 bytes = 2 per step, MN-major 16 k-rows = 2048 bytes = 128 per step).
@@ -1576,12 +1533,12 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
   return ARD_ERR_UNSUPPORTED;
 }
 
-// Products over a list of kept rows (Sec. 5.2.1).  Single-CTA tiles: the gathering lanes arrive on their own
-// CTA's barrier.
-ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_t* ridx, const void* gA, int ldgA,
-                          const void* gB, int ldgB, cudaStream_t s) {
+// Products over a list of kept rows (Sec. 5.2.1).  Single-CTA tiles.
+ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_t* ridx, cudaStream_t s) {
   TcParams p = {};
-  const TcMap maps[2] = {a.mapB, a.mapB};  // only the weight arrives by TMA
+  // mapA: the gathered operand (one-row boxes); mapB: the weight (64 x 64 boxes), or for the weight gradient the
+  // second gathered operand
+  const TcMap maps[2] = {a.mapA, a.mapB};
   p.hdr = a.g.hdr;
   p.B = a.g.B;
   p.K = a.g.K;
@@ -1596,10 +1553,6 @@ ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_
   p.sk_min_blocks = 16;
   p.sk_min_gain = 1;
   p.ridx = ridx;
-  p.gA = reinterpret_cast<const __nv_bfloat16*>(gA);
-  p.ldgA = ldgA;
-  p.gB = reinterpret_cast<const __nv_bfloat16*>(gB);
-  p.ldgB = ldgB;
   if (op == OP_FWD) return launch_mode<256, M_ROWS_FWD, 1>(ctx, p, maps, cdiv(p.B, BM) * cdiv(p.N, 64), s);
   if (op == OP_BWD_DATA) return launch_mode<256, M_ROWS_BWD_DATA, 1>(ctx, p, maps, cdiv(p.B, BM) * cdiv(p.K, 64), s);
   return launch_mode<256, M_ROWS_BWD_WEIGHT, 1>(ctx, p, maps, cdiv(p.N, BM) * cdiv(p.K, 64), s);
