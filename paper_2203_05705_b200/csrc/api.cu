@@ -1271,7 +1271,7 @@ ard_status ard_rows_fwd(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N,
   t.bn = ctx->force_bn;
   st = launch_zero_dropped_rows(ctx, rows, Y, ldy * 2, N * 2, s);
   if (st != ARD_OK) return st;
-  return launch_rows_tc(ctx, OP_FWD, t, rows->d_idx, s);
+  return launch_rows_tc(ctx, OP_FWD, t, rows->d_idx, nullptr, 0, nullptr, 0, s);
 }
 
 ard_status ard_rows_bwd_data(ard_ctx* ctx, const ard_rows* rows, int M, int K, int N, float alpha, const void* dY,
@@ -1296,7 +1296,7 @@ ard_status ard_rows_bwd_data(ard_ctx* ctx, const ard_rows* rows, int M, int K, i
   t.bn = ctx->force_bn;
   st = launch_zero_dropped_rows(ctx, rows, dA, ldda * 2, K * 2, s);
   if (st != ARD_OK) return st;
-  return launch_rows_tc(ctx, OP_BWD_DATA, t, rows->d_idx, s);
+  return launch_rows_tc(ctx, OP_BWD_DATA, t, rows->d_idx, nullptr, 0, nullptr, 0, s);
 }
 
 ard_status ard_rows_bwd_weight(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_dtype, int M, int K, int N, float alpha,
@@ -1315,14 +1315,13 @@ ard_status ard_rows_bwd_weight(ard_ctx* ctx, const ard_rows* rows, ard_dtype dW_
   g.out = dW; g.ldo = lddw;
   g.out_is_f32 = dW_dtype == ARD_F32;
   g.status = ctx->d_status;
-  // both operands are gathered along the contraction: pieces of one list row by 64 columns
-  st = get_maps(ctx, dY, M, N, lddy, 0, MAP_PLAIN, 0, 1, 64, &t.mapA);
-  if (st != ARD_OK) return st;
-  st = get_maps(ctx, A, M, K, lda, 0, MAP_PLAIN, 0, 1, 64, &t.mapB);
-  if (st != ARD_OK) return st;
+  // both operands are gathered along the contraction by the kernel's loading warps (plain pointers, no descriptor)
+  st = get_maps(ctx, dY, M, N, lddy, 0, MAP_PLAIN, 0, 1, 64, &t.mapA);   // placeholders: the kernel's parameter block
+  if (st != ARD_OK) return st;                                            // always carries two descriptors
+  t.mapB = t.mapA;
   t.g = g;
   t.bn = ctx->force_bn;
-  return launch_rows_tc(ctx, OP_BWD_WEIGHT, t, rows->d_idx, (cudaStream_t)cuda_stream);
+  return launch_rows_tc(ctx, OP_BWD_WEIGHT, t, rows->d_idx, dY, lddy, A, lda, (cudaStream_t)cuda_stream);
 }
 
 // ---- the same products on compact operands (the dense small matrices of Sec. 5.2.1, step 2) ----------

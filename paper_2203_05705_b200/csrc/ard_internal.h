@@ -218,7 +218,8 @@ struct TcArgs {
 int tc_pick_bn(ard_ctx* ctx, ard_kind kind, GemmOp op, int dp_bound, int ts);
 ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& a, cudaStream_t s);
 ard_status launch_lstm_tc(ard_ctx* ctx, int backward, const TcArgs& a, cudaStream_t s);
-ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_t* ridx, cudaStream_t s);
+ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_t* ridx, const void* gA, int ldgA,
+                          const void* gB, int ldgB, cudaStream_t s);
 
 // Whole-sequence LSTM kernels (lstm_persistent.cu).
 size_t lstm_bwd_partial_bytes(int sm_count);

@@ -107,8 +107,13 @@ struct TcParams {
   int relu;
   const void* act;
   int ldact;
-  // Row-list products: the kept-row list (the matrices the producers gather from come as descriptors).
+  // Row-list products: the kept-row list.  Forward and backward-data gather through descriptors; the weight
+  // gradient, whose two operands both follow the list, gathers with asynchronous copies from these matrices.
   const int32_t* ridx;
+  const __nv_bfloat16* gA;  // backward-weight: dY
+  int ldgA;
+  const __nv_bfloat16* gB;  // backward-weight: A
+  int ldgB;
   // Row-list products on compact operands (FUSED row kernels): hdr is the row list's header, the layer itself is
   // dense.  1: the row extent of A and of the output is hdr[HDR_NKEEP] and output row m goes to row ridx[m]
   // (forward, backward-data); 2: the contraction runs over hdr[HDR_NKEEP] rows (backward-weight).
@@ -664,7 +669,8 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(full_bar(s), 1);
+      // weight gradient over a row list: one arrival per gathering lane besides the producer's
+      mbar_init(full_bar(s), MODE == M_ROWS_BWD_WEIGHT ? 1 + 32 * ROWS_GATHER_WARPS : 1);
       mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -725,13 +731,13 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
     // An index list has no stride a TMA box could follow, but the TMA unit takes four arbitrary rows per
     // instruction (tile::gather4 on a descriptor whose box is one row of 64 columns = 128 bytes high): the four
     // 128-byte pieces land one after the other, and since the 128-byte swizzle is a function of the shared-memory
-    // address, a run of such instructions fills a stage exactly as one tall box would.  A stage takes 32 (forward,
-    // backward-data: 128 rows of the list) or 16 x (2 + boxes of B) instructions (backward-weight: 64 list rows of
-    // both operands); one thread paces at several hundred cycles per instruction, so they are dealt over the lanes
-    // of four warps.  Rows past the end of the list get an index outside the matrix: TMA fills zeros.
+    // address, a run of such instructions fills a stage exactly as one tall box would.  Forward and backward-data
+    // take 32 of them per stage (128 rows of the list); one thread paces at several hundred cycles per
+    // instruction, so they are dealt over lanes of four warps.  Rows past the end of the list get an index outside
+    // the matrix: TMA fills zeros.  (The weight gradient gathers differently, see below.)
     const int gw = warp == 0 ? 0 : warp - 9;  // 0..3
-    const CUtensorMap* mapG = &p.maps[0].tm;  // forward: A; backward-data: dY; backward-weight: dY (the A operand)
-    const CUtensorMap* mapB = &p.maps[1].tm;  // the weight (boxes), or for backward-weight A (gathered, the B operand)
+    const CUtensorMap* mapG = &p.maps[0].tm;  // forward: A; backward-data: dY
+    const CUtensorMap* mapB = &p.maps[1].tm;  // the weight (boxes)
     const int oob = p.B;                      // the first row the gathered matrices do not have
     int stage = 0;
     uint32_t phase = 0;
@@ -747,7 +753,28 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
         for (int q = 0; q < 4; ++q)
           if (m + q < sch.M_gemm) r4[q] = p.ridx[m + q];
       }
+      // Weight gradient: both operands follow the list along the contraction, 16 x (2 + boxes of B) gather
+      // instructions per block, and at the ~115 cycles a warp needs per instruction that is slower (378 us on the
+      // 32768 x 2304 x 512 layer) than 16-byte asynchronous copies straight into the swizzled layout (261 us): eight
+      // lanes fetch the eight chunks of one row, chunk c of row r goes to chunk c ^ (r & 7).  Lanes 0..15 of warp gw
+      // own the contraction rows gw*16 .. gw*16 + 15 of a block; the next block's list entries are fetched while
+      // this one is issued.
+      const int sub = lane >> 3, ch = lane & 7;
+      unsigned long long* rowtab = reinterpret_cast<unsigned long long*>(smem + L::STG_OFF) + gw * 64;
+      int jcur = -1;
+      if (MODE == M_ROWS_BWD_WEIGHT && lane < 16 && gw * 16 + lane < sch.Kc) jcur = p.ridx[gw * 16 + lane];
       for (int kb = 0; kb < ti.nkb; ++kb) {
+        int jnext = -1;
+        unsigned long long* tabA = rowtab + (kb & 1) * 32;  // [16] addresses in dY, then [16] in A
+        if (MODE == M_ROWS_BWD_WEIGHT) {
+          if (lane < 16) {
+            tabA[lane] = jcur >= 0 ? (unsigned long long)(p.gA + (size_t)jcur * p.ldgA) : 0ull;
+            tabA[16 + lane] = jcur >= 0 ? (unsigned long long)(p.gB + (size_t)jcur * p.ldgB) : 0ull;
+            const int j = (kb + 1) * BK + gw * 16 + lane;
+            if (kb + 1 < ti.nkb && j < sch.Kc) jnext = p.ridx[j];
+          }
+          __syncwarp();  // the table entries are read by other lanes below
+        }
         int good = 1;
         if (lane == 0) good = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status) ? 1 : 0;
         good = __shfl_sync(0xffffffffu, good, 0);
@@ -756,8 +783,10 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
         const uint32_t sB = sA + L::A_BYTES;
         const int kx = kb * BK;
         if (warp == 0 && lane == 0) {
-          mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(L::A_BYTES + ti.nbox * 64 * BK * 2));
-          if (MODE != M_ROWS_BWD_WEIGHT) {
+          if (MODE == M_ROWS_BWD_WEIGHT) {
+            mbar_arrive(full_bar(stage));
+          } else {
+            mbar_arrive_expect_tx(full_bar(stage), (uint32_t)(L::A_BYTES + ti.nbox * 64 * BK * 2));
 #pragma unroll
             for (int bxi = 0; bxi < 4; ++bxi) {
               if (bxi < ti.nbox) {
@@ -772,22 +801,32 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
           if (lane < 8)
             tma_gather4_2d(sA + (uint32_t)(8 * gw + lane) * 512u, mapG, full_bar(stage), kx, r4[0], r4[1], r4[2], r4[3]);
         } else {
-          // boxes of [64 list rows][64 columns]; item = (group of four list rows g, box): 16 x (2 + nbox) of them
-          const int nitem = 16 * (2 + ti.nbox);
-          for (int it = gw * 32 + lane; it < nitem; it += 32 * ROWS_GATHER_WARPS) {
-            const int g = it & 15, bx = it >> 4;  // bx 0,1: the two 64-column boxes of dY; 2..: the boxes of A
-            const int j = kx + 4 * g;
-            int jr[4];
+          // boxes of [64 contraction rows][64 columns]: A operand = dY columns m0.., B operand = A columns n0..
 #pragma unroll
-            for (int q = 0; q < 4; ++q) jr[q] = (j + q < sch.Kc) ? p.ridx[j + q] : oob;
-            if (bx < 2)
-              tma_gather4_2d(sA + (uint32_t)bx * (64 * BK * 2) + (uint32_t)g * 512u, mapG, full_bar(stage), ti.ax[bx], jr[0],
-                             jr[1], jr[2], jr[3]);
-            else
-              tma_gather4_2d(sB + (uint32_t)(bx - 2) * (64 * BK * 2) + (uint32_t)g * 512u, mapB, full_bar(stage),
-                             sel4(ti.bx, bx - 2), jr[0], jr[1], jr[2], jr[3]);
+          for (int q = 0; q < 4; ++q) {
+            const int jl = 4 * q + sub, jr = gw * 16 + jl;
+            const unsigned long long pa = tabA[jl], pb = tabA[16 + jl];
+            const uint32_t off = (uint32_t)jr * 128u + (uint32_t)((ch ^ (jr & 7)) << 4);
+#pragma unroll
+            for (int bxi = 0; bxi < BM / 64; ++bxi) {
+              const int col = ti.ax[bxi] + 8 * ch;
+              const bool in = pa != 0ull && col < sch.M_gemm;
+              cp_async_16(sA + (uint32_t)bxi * (64 * BK * 2) + off,
+                          in ? (const void*)(pa + (unsigned long long)col * 2ull) : (const void*)p.gA, in ? 16u : 0u);
+            }
+#pragma unroll
+            for (int bxi = 0; bxi < 4; ++bxi) {
+              if (bxi < ti.nbox) {
+                const int col = ti.bx[bxi] + 8 * ch;
+                const bool in = pb != 0ull && col < sch.N_gemm;
+                cp_async_16(sB + (uint32_t)bxi * (64 * BK * 2) + off,
+                            in ? (const void*)(pb + (unsigned long long)col * 2ull) : (const void*)p.gA, in ? 16u : 0u);
+              }
+            }
           }
+          cp_async_mbar_arrive_noinc(full_bar(stage));
         }
+        jcur = jnext;
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
@@ -917,6 +956,11 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
         for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+          if (MODE == M_ROWS_BWD_WEIGHT) {
+            // the gathered operands were written by ordinary asynchronous copies (generic proxy)
+            fence_proxy_async_smem();
+            tc_fence_after();
+          }
           // This thread's instruction stream is what feeds the tensor pipe: the descriptors of a block are
           // the stage's descriptor plus a constant per 16-deep step (the start-address field counts 16-byte
           // units: K-major 32 bytes = 2 per step, MN-major 16 k-rows = 2048 bytes = 128 per step).
@@ -1534,10 +1578,11 @@ ard_status launch_gemm_tc(ard_ctx* ctx, ard_kind kind, GemmOp op, const TcArgs& 
 }
 
 // Products over a list of kept rows (Sec. 5.2.1).  Single-CTA tiles.
-ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_t* ridx, cudaStream_t s) {
+ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_t* ridx, const void* gA, int ldgA,
+                          const void* gB, int ldgB, cudaStream_t s) {
   TcParams p = {};
-  // mapA: the gathered operand (one-row boxes); mapB: the weight (64 x 64 boxes), or for the weight gradient the
-  // second gathered operand
+  // forward, backward-data: mapA the gathered operand (one-row boxes), mapB the weight (64 x 64 boxes); the weight
+  // gradient takes its operands as plain pointers (gA = dY, gB = A) and uses neither
   const TcMap maps[2] = {a.mapA, a.mapB};
   p.hdr = a.g.hdr;
   p.B = a.g.B;
@@ -1553,6 +1598,10 @@ ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_
   p.sk_min_blocks = 16;
   p.sk_min_gain = 1;
   p.ridx = ridx;
+  p.gA = reinterpret_cast<const __nv_bfloat16*>(gA);
+  p.ldgA = ldgA;
+  p.gB = reinterpret_cast<const __nv_bfloat16*>(gB);
+  p.ldgB = ldgB;
   if (op == OP_FWD) return launch_mode<256, M_ROWS_FWD, 1>(ctx, p, maps, cdiv(p.B, BM) * cdiv(p.N, 64), s);
   if (op == OP_BWD_DATA) return launch_mode<256, M_ROWS_BWD_DATA, 1>(ctx, p, maps, cdiv(p.B, BM) * cdiv(p.K, 64), s);
   return launch_mode<256, M_ROWS_BWD_WEIGHT, 1>(ctx, p, maps, cdiv(p.N, BM) * cdiv(p.K, 64), s);
