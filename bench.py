@@ -648,6 +648,19 @@ def run_mlp_step(args, wl):
     detail = {"ms_per_step": {"graph_compact": ms / steps}}
     if not args.quick:
         n2 = max(5, steps // 4)
+        # cold L2: a 256 MB buffer is overwritten between the replays (the weights, 12 - 290 MB here, otherwise stay in
+        # the 126 MB L2 from one iteration to the next); the cost of the overwriting alone is timed and subtracted
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+        def cold_step():
+            flush.fill_(1)
+            gr.replay()
+
+        t_cold = timed(cold_step, n2, warm)[0] / n2
+        t_flush = timed(lambda: flush.fill_(1), n2, warm)[0] / n2
+        detail["ms_per_step"]["graph_compact_cold_l2"] = t_cold - t_flush
+        detail["ms_per_step"]["graph_compact_warm_l2"] = ms / steps
+        del flush
         detail["ms_per_step"]["eager_compact"] = timed(lambda: eager(compact), n2, warm)[0] / n2
         fullw = make_stack(0)
         gr_f = graphed(fullw)

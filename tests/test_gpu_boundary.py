@@ -132,3 +132,67 @@ def test_layer_products_with_the_shared_tail_enabled():
         assert ard.ard_last_device_status(ctx.h) == 0
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("dtype", [ard.ARD_BF16, ard.ARD_F32])
+def test_compact_and_expand_columns(dtype):
+    """ard_compact_cols / ard_expand_cols: Eq. 1 applied to the columns of a matrix and its adjoint with a rescale,
+    exact (copies and one multiplication) against the oracle's kept list."""
+    rows_, N, ld = 77, 200, 208
+    rng = np.random.default_rng(8)
+    src = inputs.bf16_round(rng.standard_normal((rows_, N)).astype(np.float32))
+    td = BF if dtype == ard.ARD_BF16 else torch.float32
+    ctx = Ctx(4096)
+    try:
+        pat = ctx.pattern(ard.ARD_ROW, 8, N)
+        S = torch.full((rows_, ld), float("nan"), dtype=td, device="cuda")
+        S[:, :N] = torch.from_numpy(src).to(td)
+        for dp, b in [(1, 1), (3, 2), (7, 7), (16, 9), (150, 30)]:
+            ard.ard_pattern_set(ctx.h, pat, dp, b)
+            keep = OP.row_keep(N, dp, b)
+            C = torch.full((rows_, ld), float("nan"), dtype=td, device="cuda")
+            ard.ard_compact_cols(ctx.h, pat, dtype, rows_, N, S, ld, C, ld)
+            got = host(C)
+            assert np.array_equal(got[:, :len(keep)], src[:, keep].astype(np.float64)), (dp, b)
+            assert np.all(np.isnan(got[:, len(keep):])), (dp, b)                  # nothing written beyond n_keep
+            E = torch.full((rows_, ld), float("nan"), dtype=torch.float32, device="cuda")
+            ard.ard_expand_cols(ctx.h, pat, dtype, rows_, N, 1.5, C, ld, E, ld)
+            want = np.zeros((rows_, N), dtype=np.float32)
+            want[:, keep] = np.float32(1.5) * src[:, keep]
+            got = host(E)
+            assert np.array_equal(got[:, :N], want.astype(np.float64)), (dp, b)
+            assert np.all(np.isnan(got[:, N:])), (dp, b)
+        with pytest.raises(ard.ArdError):
+            ard.ard_compact_cols(ctx.h, pat, dtype, rows_, N + 8, S, ld, C, ld)     # N differs from the pattern's
+    finally:
+        ctx.close()
+
+
+def test_options_are_validated_and_do_not_change_results():
+    B, K, N = 300, 512, 1024
+    X, W, dY = _layer(B, K, N, 51)
+    ctx = Ctx(2 * B * N + 4096)
+    try:
+        with pytest.raises(ard.ArdError):
+            ard.ard_set_option(ctx.h, 99, 1)
+        with pytest.raises(ard.ArdError):
+            ard.ard_set_option(ctx.h, ard.ARD_OPT_PDL, -1)
+        pat = ctx.pattern(ard.ARD_ROW, K, N)
+        ard.ard_pattern_set(ctx.h, pat, 3, 1)
+        mask = OP.row_mask(N, 3, 1)
+        Xd, Wd, dYd = dev(X, ard.ARD_BF16), dev(W.T, ard.ARD_BF16), dev(dY, ard.ARD_BF16)
+        want = (OG.fwd(X, W, mask, 2.0), OG.bwd_data(dY, W, mask, 2.0), OG.bwd_weight(X, dY, mask, 2.0).T)
+        for opts in [{}, {ard.ARD_OPT_PDL: 0}, {ard.ARD_OPT_SIDE_STREAMS: 0}, {ard.ARD_OPT_CTA_PAIRS: 0}, {ard.ARD_OPT_BAND_ROWS: 2}]:
+            for k, v in opts.items():
+                ard.ard_set_option(ctx.h, k, v)
+            Y, dX, dW = nan_buf(B, N, BF), nan_buf(B, K, BF), nan_buf(N, K, BF)
+            ard.ard_layer_products(ctx.h, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, 2.0, Xd, K, Wd, K, dYd, N, Y, N,
+                                   ard.ARD_OUT_SCATTER_ZEROFILL, dX, K, dW, K, 1)
+            torch.cuda.synchronize()
+            for got, w, name in zip((Y, dX, dW), want, ("fwd", "bwd_data", "bwd_weight")):
+                assert OG.rel_fro(host(got), w) <= TOL_BF16, (opts, name)
+            for k in opts:
+                ard.ard_set_option(ctx.h, k, 1 if k != ard.ARD_OPT_BAND_ROWS else 16)
+        assert ard.ard_last_device_status(ctx.h) == 0
+    finally:
+        ctx.close()
