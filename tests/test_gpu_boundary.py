@@ -196,3 +196,48 @@ def test_options_are_validated_and_do_not_change_results():
         assert ard.ard_last_device_status(ctx.h) == 0
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("kind,ts", [("row", 0), ("tile", 128)])
+def test_first_use_of_new_buffers_inside_a_stream_capture(kind, ts):
+    """No product call allocates, copies or synchronises, so the very first call on buffers the library has never
+    seen can be recorded into a CUDA graph (pattern drawn inside the graph from a device counter); the replays are
+    compared with the oracle."""
+    B, K, N = 384, 512, 1024
+    X, W, dY = _layer(B, K, N, 61)
+    akind = ard.ARD_ROW if kind == "row" else ard.ARD_TILE
+    from distributions import max_entropy_K
+    Kd = max_entropy_K(0.5, 8)
+    cdf = OP.quantise_K(Kd)
+    ctx = Ctx(2 * B * N + 4096)
+    try:
+        ard.ard_set_path(ctx.h, ard.ARD_PATH_TENSOR_CORE)
+        ard.ard_set_distribution(ctx.h, 0, Kd)
+        pat = ctx.pattern(akind, K, N, ts)
+        counter = torch.zeros(1, dtype=torch.int64, device="cuda")
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            Xd, Wd, dYd = dev(X, ard.ARD_BF16), dev(W.T, ard.ARD_BF16), dev(dY, ard.ARD_BF16)
+            Y, dX, dW = nan_buf(B, N, BF), nan_buf(B, K, BF), nan_buf(N, K, BF)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                cs = s.cuda_stream
+                ard.ard_sample_pattern_counter(ctx.h, pat, 0, 77, 500, counter, 1, 3, cs)
+                ard.ard_fwd(ctx.h, pat, ard.ARD_BF16, B, K, N, 2.0, Xd, K, Wd, K, Y, N, ard.ARD_OUT_SCATTER_ZEROFILL, cs)
+                ard.ard_bwd_data(ctx.h, pat, ard.ARD_BF16, B, K, N, 2.0, dYd, N, 0, Wd, K, dX, K, cs)
+                ard.ard_bwd_weight(ctx.h, pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, 2.0, Xd, K, dYd, N, 0, dW, K, 1, cs)
+            seen = set()
+            for it in range(6):
+                g.replay()
+                torch.cuda.synchronize()
+                dp, b = OP.draw(cdf, 77, 500 + it, 3)
+                seen.add(dp)
+                mask = OP.row_mask(N, dp, b) if kind == "row" else OP.tile_mask(K, N, ts, dp, b)
+                for got, want, name in ((Y, OG.fwd(X, W, mask, 2.0), "fwd"), (dX, OG.bwd_data(dY, W, mask, 2.0), "bwd_data"),
+                                        (dW, OG.bwd_weight(X, dY, mask, 2.0).T, "bwd_weight")):
+                    assert OG.rel_fro(host(got), want) <= TOL_BF16, (it, dp, b, name)
+            assert len(seen) >= 2
+        assert ard.ard_last_device_status(ctx.h) == 0
+    finally:
+        ctx.close()
