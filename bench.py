@@ -1236,6 +1236,19 @@ class LayerBench:
                 "torch_matmul": statistics.median(lib_ms), "own_kernels_dp1_in_sequence_all": own,
                 "own_kernels_dp1_one_call_all": own_one, "torch_matmul_all": lib_ms}
 
+    def algorithmic_bytes(self, op, kept_units):
+        """Bytes a product has to move at least (bf16): operands read once, output written once (Sec. 3.1 / 3.2:
+        only the kept part of the weight; the forward output is full width, the weight gradient's kept part)."""
+        B, K, N = self.B, self.K, self.N
+        if self.kind == self.ard.ARD_ROW:
+            nk = kept_units
+            return {"fwd": 2.0 * (B * K + nk * K + B * N), "bwd_data": 2.0 * (B * nk + nk * K + B * K),
+                    "bwd_weight": 2.0 * (B * K + B * nk + nk * K),
+                    "bwd_weight_zero_fill": 2.0 * (B * K + B * nk + N * K)}[op]
+        w = 2.0 * self.ts ** 2 * kept_units
+        return {"fwd": 2.0 * (B * K + B * N) + w, "bwd_data": 2.0 * (B * N + B * K) + w,
+                "bwd_weight": 2.0 * (B * K + B * N) + w, "bwd_weight_zero_fill": 2.0 * (B * K + B * N + N * K)}[op]
+
     def per_dp_table(self, peak_burst):
         """Every (dp, b) of the distribution's support, forced with ard_pattern_set: per product and for the whole
         step the median over b and REPEATS of the CUDA-event time.  bwd_data includes the compaction of the
@@ -1302,6 +1315,11 @@ class LayerBench:
                 if nm != "sampler":
                     row[nm + "_tflops"] = fl / (m * 1e-3) / 1e12
                     row[nm + "_frac_of_burst"] = row[nm + "_tflops"] / peak_burst
+                    # the roofline that binds this product: tensor time of its kept FLOPs or HBM time of its bytes
+                    t_tc = fl / (peak_burst * 1e12) * 1e3
+                    t_hbm = self.algorithmic_bytes(nm, float(np.mean(kept))) / (self.hbm_gbs * 1e9) * 1e3
+                    row[nm + "_bound"] = "hbm" if t_hbm > t_tc else "tensor"
+                    row[nm + "_frac_of_roofline"] = max(t_tc, t_hbm) / m
             table[str(dp)] = row
             step_by_dp[dp] = float(np.mean(steps))            # mean over b and repeats: what an expectation needs
             self.onecall_by_dp = getattr(self, "onecall_by_dp", {})
@@ -1404,6 +1422,7 @@ def sweep_block(lb, peaks, dense):
     expectations are held against the dense step timed like the table's entries (single passes); the sampled
     figures against the dense step timed like them (long loops, where the power cap lowers the clock)."""
     best_dense = min(dense["own_kernels_dp1"], dense["torch_matmul"])
+    lb.hbm_gbs = peaks["hbm_gbs"]
     table, step_by_dp, units_by_dp = lb.per_dp_table(peaks["bf16_tflops"])
     exp = lb.expectations(step_by_dp, units_by_dp, min(lb.dense_burst.values()))
     exp_one = lb.expectations(lb.onecall_by_dp, units_by_dp, min(lb.dense_burst.values()))
@@ -1415,6 +1434,8 @@ def sweep_block(lb, peaks, dense):
         sampled[str(pp)] = {"ms_per_step": ms, "speedup_vs_dense": best_dense / ms,
                             "kept_fraction": float(np.mean([nk / lb.units for (_, _, nk) in pats]))}
     return {"per_dp": table, "dense_ms_single_pass": lb.dense_burst, "expected": exp,
+            "per_dp_rooflines": "tensor: kept FLOPs / %.1f TFLOP/s; hbm: algorithmic bytes / %.1f GB/s (%s); a product's "
+                                "bound is the longer of the two" % (peaks["bf16_tflops"], peaks["hbm_gbs"], peaks["source"]),
             "expected_products_in_one_call": exp_one, "sampled": sampled,
             "note": "per_dp: median over every offset b and %d repeats, pattern forced with ard_pattern_set; expected: "
                     "sum over dp of k^_dp x mean step time, k^ = the quantised distribution; sampled: %d device-drawn "
