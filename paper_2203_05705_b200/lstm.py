@@ -78,6 +78,7 @@ class LstmStack:
             self.dYc.append(torch.zeros((T * B, H), dtype=bf, device="cuda"))
             self.Wk.append(torch.zeros((4 * H, I), dtype=bf, device="cuda") if l > 0 else None)
             self.dWk.append(torch.zeros((4 * H, I), dtype=f32, device="cuda") if l > 0 else None)
+        self.dh_last = [torch.zeros((B, dims[l + 1]), dtype=f32, device="cuda") for l in range(self.L)]
 
     def close(self):
         for p in self.out_pats + [q for q in self.gate_pats if q is not None] + [ly.pat for ly in self.layers]:
@@ -114,7 +115,7 @@ class LstmStack:
             # upstream gradient of h_t, full width with the rescale: h half of D[t+1] for t < T-1, dH_last for t = T-1
             ly.D.zero_()
             ly.dc.zero_()
-            dh_last = torch.empty((B, H), dtype=torch.float32, device="cuda")
+            dh_last = self.dh_last[l]
             if T > 1:
                 ard.ard_expand_cols(ctx, self.out_pats[l], ard.ARD_BF16, (T - 1) * B, H, alphas[l], dYc, H,
                                     ly.D.data_ptr() + (B * KH + I) * 4, KH)

@@ -43,7 +43,7 @@ def test_config2_mlp_chain_per_gemm(p):
         alpha = [1.0 / (1.0 - p), 1.0 / (1.0 - p), 1.0]
         B = 128
         worst = 0.0
-        for step in range(4):
+        for step in range(8):
             X, dZ3 = inputs.config2_step(step)
             masks = []
             for l in range(2):
@@ -151,8 +151,10 @@ def test_config5_sampled_outputs(kind, ts):
         dW = torch.empty((N, K), dtype=BF, device="cuda")
         rows = np.arange(7, B, B // 128)[:128]
         cols = np.arange(3, N, N // 128)[:128]
-        # periods 3, 5, 7, 12 make the forward product pick output tiles 224, 192, 160, 192 columns wide
-        for dp, b in [(1, 1), (2, 2), (3, 1), (5, 3), (7, 2), (12, 5), (16, 7)]:
+        # every period of the benchmark's distribution (3, 5, 7, 12 make the forward product pick output tiles 224,
+        # 192, 160, 192 columns wide), the offset varied with it
+        for dp, b in [(1, 1), (2, 2), (3, 1), (4, 4), (5, 3), (6, 1), (7, 2), (8, 5), (9, 9), (10, 3), (11, 6), (12, 5),
+                      (13, 1), (14, 14), (15, 8), (16, 7)]:
             ard.ard_pattern_set(ctx.h, pat, dp, b)
             Y.fill_(float("nan")); dX.fill_(float("nan")); dW.fill_(float("nan"))
             ard.ard_fwd(ctx.h, pat, ard.ARD_BF16, B, K, N, 2.0, dXd, K, dWd, K, Y, N, ard.ARD_OUT_SCATTER_ZEROFILL)
