@@ -99,8 +99,8 @@ void fill_common(GemmArgs& g, ard_ctx* ctx, const ard_pattern* pat, int B, int K
   g.ldact = 0;
 }
 
-// Can the tcgen05 path take this call?  (bf16 only; 16-byte aligned pointers and pitches; the
-// period bounded by the descriptor-table size.)
+// Can the tcgen05 path take this call?  (bf16 only; 16-byte aligned pointers and pitches; distributions of
+// at most ARD_MAX_NDP_TC periods.)
 ard_status tc_eligible(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, int B, int K, int N,
                        const void* p0, int ld0, const void* p1, int ld1, const void* po, int ldo, int out_es) {
   if (dtype != ARD_BF16) return ARD_ERR_UNSUPPORTED;

@@ -22,7 +22,7 @@ enum {
   HDR_TR = 5,
   HDR_TC = 6,
   HDR_TS = 7,
-  HDR_MAPIDX = 8,  // dp*(dp-1)/2 + (b-1): index into per-(dp,b) descriptor tables
+  HDR_MAPIDX = 8,  // dp*(dp-1)/2 + (b-1): the pattern's number among all (dp, b) pairs
   HDR_WORDS = 16
 };
 

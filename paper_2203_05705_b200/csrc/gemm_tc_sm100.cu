@@ -47,7 +47,7 @@ enum TcMode {
   M_TILEC_BWD_DATA = 7,
   M_TILEC_BWD_WEIGHT = 8,
   // LSTM gate products over the four gate blocks i|f|g|o of one weight in a single launch: the kept
-  // units of gate g are the rows g*H + keep[j] of W, reached through one descriptor table per gate.
+  // units of gate g are the rows g*H + keep[j] of W, reached through one descriptor per gate.
   M_LSTM_FWD = 9,       // Z[:, g*ldz + j] = [x,h] . W[g*H + keep[j], :]
   M_LSTM_BWD_DATA = 10, // d[x,h] = sum_g dZ[:, g*ldz + j] . W[g*H + keep[j], :]
   M_LSTM_BWD_WEIGHT = 11, // dW[g*H + keep[j], :] = sum_rows dZ[:, g*ldz + j] . [x,h]   (M tiles: gate-major)

@@ -3,7 +3,7 @@
 // layer fed by a dropped layer multiplies compact matrices on both sides; Sec. 3.4: a new pattern per
 // iteration).  Host code only: the order of the calls is all that lives here, every step runs in the
 // kernels behind them.  Nothing here synchronises or allocates, so the whole iteration can be captured
-// into a CUDA graph once its descriptor tables exist (run it once before capturing).
+// into a CUDA graph (after one ordinary call, in which the context creates the streams it forks onto).
 #include "ard_internal.h"
 
 

@@ -3,9 +3,8 @@
 // Who needs this: code that may not allocate device memory at the moment it calls the layer -- an
 // inference / training server that froze its memory plan after start-up, a plug-in running inside a
 // host application that owns the allocator, or a caller sitting on a stream whose owner forbids
-// cudaMalloc / cudaFree because both synchronise the whole device.  ard_bwd_data may allocate (the
-// context workspace was sized at ard_create, and the tensor-core path builds descriptor tables on
-// first use); this entry point never does.
+// cudaMalloc / cudaFree because both synchronise the whole device.  ard_bwd_data needs a context
+// workspace that ard_create allocated for it; this entry point needs none and never allocates.
 //
 // How: the compacted copy of dY (kept columns only) that the GEMM reads lives in a fixed array that
 // is part of the library image, so every GPU that loads libard.so carries ARD_STATIC_SCRATCH_BYTES
