@@ -366,30 +366,30 @@ struct Sched {
     u.kb0 = 0;
     u.kb1 = -1;
     if (is_class_mode(MODE) && h_items < total) {
-      // Some classes keep nothing: their items only write zeros and cost a fraction of the others.  The others
-      // go round first; then the zero items go, light_q apiece, to the workers that got one item less in
-      // that round, and only what is left of them is dealt to everybody.  (In plain round-robin order a
-      // forward product whose period divides the tile-column count ran its few long items on workers that
-      // afterwards still took their full share of the zero items.)
+      // Some classes keep nothing: their items only write zeros, take no part in the producer's and the MMA
+      // thread's loops and cost a fraction of the others.  The others are dealt round-robin; the zero items go,
+      // light_q apiece, to the workers that got one item less in that round, and only what is left of them is
+      // dealt to everybody.  (In plain round-robin order a forward product whose period divides the tile-column
+      // count ran its few long items on workers that afterwards still took their full share of the zero items.)
+      // Every worker takes its zero items FIRST: its epilogue warps write them while the first long item's
+      // products run, instead of after the last one.
       const int a = h_items / workers, rem = h_items - a * workers;
       const int a_w = a + (w < rem ? 1 : 0);
-      if (i < a_w) {
-        u.t = w + i * workers;
+      const int n_light = total - h_items;
+      const int n_less = workers - rem;                        // workers rem .. workers-1 got one item less
+      const int first_part = rem == 0 ? 0 : min(n_light, n_less * light_q);
+      int n1 = 0;                                               // zero items this worker takes in the first part
+      if (rem != 0 && w >= rem && first_part > w - rem) n1 = min(light_q, (first_part - (w - rem) + n_less - 1) / n_less);
+      const int rest = n_light - first_part;
+      const int n2 = rest > w ? (rest - w + workers - 1) / workers : 0;
+      if (i < n1 + n2) {
+        const int j = i < n1 ? (w - rem) + i * n_less : first_part + w + (i - n1) * workers;
+        u.t = h_items + j;
         return true;
       }
-      const int ip = i - a_w, n_light = total - h_items;
-      int j;
-      if (rem == 0) {
-        j = w + ip * workers;
-      } else {
-        const int n_less = workers - rem;                  // workers rem .. workers-1
-        const int first_part = min(n_light, n_less * light_q);
-        int n1 = 0;                                         // zero items this worker takes in the first part
-        if (w >= rem && first_part > w - rem) n1 = min(light_q, (first_part - (w - rem) + n_less - 1) / n_less);
-        j = ip < n1 ? (w - rem) + ip * n_less : first_part + w + (ip - n1) * workers;
-      }
-      u.t = h_items + j;
-      return j < n_light;
+      const int ih = i - (n1 + n2);
+      u.t = w + ih * workers;
+      return ih < a_w;
     }
     const int first = SK_MODE ? sk_tiles : 0;
     u.t = first + w + (i - n_shared) * workers;
@@ -945,12 +945,15 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
       int it = 0;
       bool ok = true;
       Unit un;
+      int nacc = 0;  // tiles that used an accumulator so far (a tile without contraction blocks uses none)
       for (; ok && sch.unit(w0, it, un); ++it) {
         const TileInfo ti = sch.template tile<PLAIN>(p, un.t);
         const int kb_begin = un.kb0, kb_end = un.kb1 < 0 ? ti.nkb : un.kb1;
+        if (kb_end <= kb_begin) continue;  // nothing to multiply: the epilogue warps write the zeros on their own
         const uint32_t idesc = make_idesc(ti.bn, A_MN, B_MN, BM * CTAS);
-        const int acc = it & 1;
-        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        const int acc = nacc & 1;
+        const uint32_t acc_phase = (uint32_t)(nacc >> 1) & 1u;
+        ++nacc;
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
@@ -981,13 +984,8 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        if (CTAS == 2) {
-          if (kb_end > kb_begin) tc_commit2(tfull_bar(acc), (uint16_t)3);
-          else { mbar_arrive(tfull_bar(acc)); mbar_arrive_cluster(mapa_u32(tfull_bar(acc), 1u)); }
-        } else {
-          if (kb_end > kb_begin) tc_commit(tfull_bar(acc));
-          else mbar_arrive(tfull_bar(acc));
-        }
+        if (CTAS == 2) tc_commit2(tfull_bar(acc), (uint16_t)3);
+        else tc_commit(tfull_bar(acc));
       }
     }
   } else {
@@ -998,16 +996,21 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
     float* stg = reinterpret_cast<float*>(smem + L::STG_OFF) + (warp - 2) * (32 * 33);
     const int dp = sch.dp, bb = sch.b - 1;
     const uint32_t magic_dp = (uint32_t)(0x100000000ull / (unsigned)dp) + 1u;  // exact x/dp for x < 2^16
-    int it = 0;
+    int it = 0, nacc = 0;
     bool ok = true;
     Unit un;
     for (; ok && sch.unit(w0, it, un); ++it) {
       const TileInfo ti = sch.template tile<PLAIN>(p, un.t);
-      const bool has_acc = (un.kb1 < 0 ? ti.nkb : un.kb1) > un.kb0;  // an empty contraction leaves zeros
-      const int acc = it & 1;
-      const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
-      tc_fence_after();
+      // An empty contraction leaves zeros: such a tile has no accumulator and no barrier traffic, these warps
+      // just write it (the same way as any other tile, from zeros instead of the accumulator).
+      const bool has_acc = (un.kb1 < 0 ? ti.nkb : un.kb1) > un.kb0;
+      const int acc = nacc & 1;
+      const uint32_t acc_phase = (uint32_t)(nacc >> 1) & 1u;
+      if (has_acc) {
+        ++nacc;
+        if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+      }
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
       const int m = ti.m0 + row_in_tile;
       const int nch = ti.bn / 32;  // 32-column chunks in this tile, split between the two warps of a quadrant
@@ -1364,7 +1367,7 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) {
+      if (lane == 0 && has_acc) {
         if (CTAS == 2) mbar_arrive_cluster(mapa_u32(tempty_bar(acc), 0u));  // the leader's barrier
         else mbar_arrive(tempty_bar(acc));
       }
