@@ -23,20 +23,50 @@ def test_philox_known_answers():
         assert list(P.philox4x32_10(ctr, key)) == out
 
 
+def _paper_examples():
+    """tests/golden/paper_examples.txt: the kept units the paper's worked examples name."""
+    out = []
+    with open(os.path.join(GOLD, "paper_examples.txt")) as f:
+        for line in f:
+            if not line.strip() or line.startswith("#"):
+                continue
+            head, tail = line.split("->")
+            out.append((head.split(), tail))
+    return out
+
+
 def test_paper_worked_examples():
-    # Sec. 3.1: dp=3, b=1 keeps rows 1, 4, 7 (1-based)
-    assert (P.row_keep(9, 3, 1) + 1).tolist() == [1, 4, 7]
-    # Sec. 3.2: dp=4, b=1 keeps tiles 1, 5, 9, 13
-    kept = P.tile_keep(4 * 2, 4 * 2, 2, 4, 1)          # 4x4 grid of 2x2 tiles
-    t = (kept[:, 0] * 4 + kept[:, 1] + 1).tolist()
-    assert t == [1, 5, 9, 13]
-    M = P.tile_mask(8, 8, 2, 4, 1)
-    assert M.sum() == 8 * 8 / 4                          # a quarter of the synapses survive
-    # Sec. 6: mask convention 1 = keep
-    m = np.zeros(6)
-    m[[0, 2, 3]] = 1
-    assert m.tolist() == [1, 0, 1, 1, 0, 0]
-    assert P.row_mask(6, 2, 1).tolist() == [1, 0, 1, 0, 1, 0]
+    seen = set()
+    for head, tail in _paper_examples():
+        kind = head[0]
+        seen.add(kind)
+        if kind == "row":        # Sec. 3.1: dp = 3, b = 1 keeps rows 1, 4, 7 (1-based)
+            dp, b, units = int(head[1]), int(head[2]), int(head[3])
+            assert (P.row_keep(units, dp, b) + 1).tolist() == [int(x) for x in tail.split()]
+            assert (np.flatnonzero(P.row_mask(units, dp, b)) + 1).tolist() == [int(x) for x in tail.split()]
+        elif kind == "tile":     # Sec. 3.2: dp = 4, b = 1 keeps tiles 1, 5, 9, 13 of a grid numbered row-major from 1
+            dp, b, units = int(head[1]), int(head[2]), int(head[3])
+            g = int(round(units ** 0.5))
+            kept = P.tile_keep(g * 2, g * 2, 2, dp, b)          # g x g grid of 2 x 2 tiles
+            assert (kept[:, 0] * g + kept[:, 1] + 1).tolist() == [int(x) for x in tail.split()]
+            M = P.tile_mask(g * 2, g * 2, 2, dp, b)
+            assert M.sum() == (g * 2) ** 2 / dp                  # a quarter of the synapses survive
+            # the mask is 1 exactly on the kept tiles
+            want = np.zeros((g, g))
+            want[kept[:, 0], kept[:, 1]] = 1
+            assert np.array_equal(M, np.kron(want, np.ones((2, 2))))
+        elif kind == "mask":     # Sec. 6: the mask has 1 where a row is KEPT (six rows, rows 1, 3, 4 kept)
+            units = int(head[1])
+            bits, rows = tail.split(":")
+            bits = [int(x) for x in bits.split()]
+            rows = [int(x) for x in rows.split()]
+            assert len(bits) == units and [i + 1 for i, v in enumerate(bits) if v == 1] == rows
+            # the oracle's masks follow that convention: ones at the kept units, and only there
+            for dp, b in [(2, 1), (3, 2), (6, 6)]:
+                m = P.row_mask(units, dp, b)
+                assert set(m.tolist()) <= {0.0, 1.0}
+                assert (np.flatnonzero(m == 1)).tolist() == P.row_keep(units, dp, b).tolist()
+    assert seen == {"row", "tile", "mask"}
 
 
 @pytest.mark.parametrize("N", [12, 256, 257, 1000])
