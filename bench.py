@@ -1144,12 +1144,14 @@ class LayerBench:
             ev[3].record()
 
     def products(self, alpha, ptr=None, stream=None):
-        """The three products of the layer through the one call that enqueues them side by side."""
+        """The three products of the layer through the one call that enqueues them side by side.  The weight
+        gradient writes the kept rows only (an optimiser that walks the kept rows needs no zeros) unless
+        self.zero_fill_dW is set, which also writes zeros to the rows of dropped neurons."""
         ard, B, K, N = self.ard, self.B, self.K, self.N
         q = ptr or self.ptr
         ard.ard_layer_products(self.ctx, self.pat, ard.ARD_BF16, ard.ARD_BF16, B, K, N, alpha, q["X"], K, q["W"], K, q["dY"], N,
-                               q["Y"], N, ard.ARD_OUT_SCATTER_ZEROFILL, q["dX"], K, q["dW"], K, 0,
-                               self.cs if stream is None else stream)
+                               q["Y"], N, ard.ARD_OUT_SCATTER_ZEROFILL, q["dX"], K, q["dW"], K,
+                               1 if getattr(self, "zero_fill_dW", False) else 0, self.cs if stream is None else stream)
 
     def step(self, pp, it, ev=None, ptr=None):
         """One step: draw the pattern on the device, then the layer's three products (ard_layer_products; with `ev`,
@@ -1533,6 +1535,11 @@ def main():
     detail["ideal_speedup"] = {k2: v["ideal_speedup"] for k2, v in sw["expected"].items()}
     detail["repeats"] = {"n": REPEATS, "values": h["values"], "ms_per_step": [m / args.steps for m in h["ms_all"]],
                          "spread": (max(h["values"]) - min(h["values"])) / h["value"]}
+    # the same iterations with the weight gradient also writing zeros to the rows of dropped neurons
+    lb.zero_fill_dW = True
+    zf = statistics.median(lb.timed_steps(p, h["its"])[0] for _ in range(3)) / args.steps
+    lb.zero_fill_dW = False
+    detail["ms_per_step_with_dW_zero_fill"] = zf
 
     if args.sweep_only:
         if rank == 0:
