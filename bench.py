@@ -1340,6 +1340,7 @@ class LayerBench:
             t = sum(k[dp - 1] * step_by_dp[dp] for dp in step_by_dp)
             u = sum(k[dp - 1] * units_by_dp[dp] for dp in step_by_dp)
             out[str(pp)] = {"expected_ms_per_step": t, "expected_speedup": dense_ms / t, "ideal_speedup": 1.0 / (1.0 - pp),
+                            "expected_speedup_vs_torch_matmul": self.dense_burst["torch_matmul"] / t,
                             "fraction_of_ideal": dense_ms / t * (1.0 - pp),
                             "expected_kept_tflops": 3 * self.flops_per_unit() * u / (t * 1e-3) / 1e12,
                             "expected_kept_fraction": u / self.units}
