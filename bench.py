@@ -543,6 +543,14 @@ def run_lstm_stack(args, wl):
     ard.ard_destroy(ctx)
 
 
+def apply_options(ctx, args):
+    """--opt NAME=VALUE: tuning switches of the context (ard_set_option)."""
+    from paper_2203_05705_b200 import ard
+    for kv in getattr(args, "opt", []):
+        name, val = kv.split("=")
+        ard.ard_set_option(ctx, getattr(ard, "ARD_OPT_" + name.upper()), int(val))
+
+
 def run_mlp_step(args, wl):
     """A step is one training iteration of the whole stack: patterns drawn on the device, forward chain,
     backward chain (weight, bias and input gradients), as ONE native call replayed from a CUDA graph."""
@@ -556,6 +564,7 @@ def run_mlp_step(args, wl):
     bf = torch.bfloat16
     alpha = 1.0 / (1.0 - p)
     ctx = ard.ard_create(0, 2 * B * max(dims) + 4096)
+    apply_options(ctx, args)
     ard.ard_set_compact_reuse(ctx, 1)
     Kd = max_entropy_K(p, n_dp)
     ard.ard_set_distribution(ctx, 0, Kd)
@@ -1105,9 +1114,7 @@ class LayerBench:
         self.t = tensors
         self.ctx = ard.ard_create(dev, 2 * B * N + 4096)
         ard.ard_set_compact_reuse(self.ctx, 1)   # dY is not written between bwd-data and bwd-weight of a step
-        for kv in args.opt:
-            name, val = kv.split("=")
-            ard.ard_set_option(self.ctx, getattr(ard, "ARD_OPT_" + name.upper()), int(val))
+        apply_options(self.ctx, args)
         if args.shared_tail:
             ard.ard_set_shared_tail(self.ctx, 1, 0, 0)
         self.pat = ard.ard_pattern_create(self.ctx, self.kind, K, N, wl["ts"])

@@ -15,7 +15,7 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libard.so")
 SOURCES = ["api.cu", "sampler.cu", "gemm_cc.cu", "gemm_tc_sm100.cu", "aux_kernels.cu", "no_alloc.cu",
-           "distribution_search.cu", "lstm_persistent.cu", "mlp_step.cu", "rows.cu", "blocks.cu", "dropout_schedule.cu"]
+           "distribution_search.cu", "lstm_persistent.cu", "mlp_step.cu", "mlp_persistent.cu", "rows.cu", "blocks.cu", "dropout_schedule.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]

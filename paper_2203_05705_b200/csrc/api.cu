@@ -116,6 +116,11 @@ ard_status tc_eligible(ard_ctx* ctx, const ard_pattern* pat, ard_dtype dtype, in
 
 }  // namespace
 
+ard_status ard_encode_tcmap(ard_ctx* ctx, const void* base, int rows, int cols, int ld, int units, int variant,
+                            int box_rows, int box_cols, TcMap* out) {
+  return get_maps(ctx, base, rows, cols, ld, units, variant, 0, box_rows, box_cols, out);
+}
+
 bool ard_side_streams(ard_ctx* ctx, cudaStream_t main) {
   if (ctx->n_ev == ARD_MLP_EVENTS && ctx->side_stream && ctx->aux_stream) return true;
   if (ctx->n_ev != 0) return false;  // an earlier attempt failed half way
@@ -176,6 +181,7 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->d_lstm_partial = nullptr;
   ctx->pdl_in_capture = 1;
   ctx->mlp_two_streams = 1;
+  ctx->mlp_persistent = 1;
   ctx->side_stream = nullptr;
   ctx->aux_stream = nullptr;
   ctx->n_ev = 0;
@@ -266,6 +272,7 @@ ard_status ard_set_option(ard_ctx* ctx, ard_option option, int value) {
     case ARD_OPT_SIDE_STREAMS: ctx->mlp_two_streams = value ? 1 : 0; return ARD_OK;
     case ARD_OPT_CTA_PAIRS: ctx->use_pairs = value ? 1 : 0; return ARD_OK;
     case ARD_OPT_BAND_ROWS: ctx->band_m = value; return ARD_OK;
+    case ARD_OPT_MLP_PERSISTENT: ctx->mlp_persistent = value ? 1 : 0; return ARD_OK;
   }
   return ARD_ERR_INVALID_ARG;
 }

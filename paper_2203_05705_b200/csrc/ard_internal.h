@@ -122,6 +122,7 @@ struct ard_ctx {
   // ard_mlp_step: the weight-side work of an iteration (weight compaction, weight and bias gradients) runs on
   // a second stream, forked from and joined back into the caller's stream with these events
   int mlp_two_streams;
+  int mlp_persistent;  // ard_mlp_step: the whole iteration in one cooperative kernel when the stack fits it
   cudaStream_t side_stream;
   cudaStream_t aux_stream;  // expansion of the weight gradients and bias gradients
   cudaEvent_t ev[ARD_MLP_EVENTS];
@@ -159,6 +160,14 @@ struct SharedTailOff {
 };
 
 // ---- launchers implemented in the .cu files -----------------------------------------------------
+// One whole-matrix descriptor (see TcMap): [rows][cols] bf16 at `base`, pitch ld, boxes of box_rows x box_cols.
+ard_status ard_encode_tcmap(ard_ctx* ctx, const void* base, int rows, int cols, int ld, int units, int variant,
+                            int box_rows, int box_cols, TcMap* out);
+// The iteration of ard_mlp_step in one cooperative kernel; ARD_ERR_UNSUPPORTED (nothing enqueued) when the
+// stack does not fit it.
+ard_status launch_mlp_persistent(ard_ctx* ctx, const ard_mlp_layer* layers, int n_layers, int B, const void* X, int ldx,
+                                 const void* dOut, int lddout, void* dX, int lddx, int dist_id, uint64_t seed,
+                                 uint64_t iteration_base, uint64_t* iteration_counter, cudaStream_t s);
 ard_status launch_sampler(ard_ctx* ctx, ard_pattern* pat, const unsigned long long* d_cdf, int ndp,
                           uint64_t seed, uint64_t iteration, uint32_t stream_id, int forced_dp, int forced_b,
                           cudaStream_t s, unsigned long long* d_counter = nullptr, int advance = 0);

@@ -26,6 +26,12 @@ extern "C" ard_status ard_mlp_step(ard_ctx* ctx, const ard_mlp_layer* layers, in
   if (last_sampled >= 0 && !iteration_counter) return ARD_ERR_INVALID_ARG;
   ard_status st;
   cudaStream_t main_s = (cudaStream_t)cuda_stream;
+  // A small stack (batch of at most 128 rows, a narrow output layer) runs as one cooperative kernel.
+  if (ctx->mlp_persistent && ctx->path != ARD_PATH_CUDA_CORE) {
+    st = launch_mlp_persistent(ctx, layers, n_layers, B, X, ldx, dOut, lddout, dX, lddx, dist_id, seed, iteration_base,
+                               iteration_counter, main_s);
+    if (st != ARD_ERR_UNSUPPORTED) return st;
+  }
   // Three streams: everything the activations and their gradients wait for stays on the caller's stream;
   // weight compaction and the weight gradients, which nothing downstream of them in the iteration reads,
   // run beside it on the context's second stream, the expansion of those gradients and the bias gradients

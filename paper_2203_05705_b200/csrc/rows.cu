@@ -2,28 +2,9 @@
 // sensitivity prediction per region, one Bernoulli draw per row, compaction of the kept rows into a
 // device-resident list.  Nothing returns to the host; the products that follow read the list.
 #include "ard_internal.h"
+#include "philox.h"
 
 namespace {
-
-__device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
-  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
-  const uint32_t hi0 = __umulhi(M0, c[0]), lo0 = M0 * c[0];
-  const uint32_t hi1 = __umulhi(M1, c[2]), lo1 = M1 * c[2];
-  const uint32_t n0 = hi1 ^ c[1] ^ k0, n2 = hi0 ^ c[3] ^ k1;
-  c[0] = n0;
-  c[1] = lo1;
-  c[2] = n2;
-  c[3] = lo0;
-}
-
-__device__ __forceinline__ void philox4x32_10(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    philox_round(c, k0, k1);
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
-  }
-}
 
 template <typename T> __device__ __forceinline__ float val_f(T v);
 template <> __device__ __forceinline__ float val_f<float>(float v) { return v; }

@@ -5,30 +5,9 @@
 // all threads then write the header and the lists the GEMM kernels read.  Nothing returns to the
 // host, so the GEMMs that follow on the same stream need no synchronisation.
 #include "ard_internal.h"
+#include "philox.h"
 
 namespace {
-
-__device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
-  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
-  uint32_t hi0 = __umulhi(M0, c[0]), lo0 = M0 * c[0];
-  uint32_t hi1 = __umulhi(M1, c[2]), lo1 = M1 * c[2];
-  uint32_t n0 = hi1 ^ c[1] ^ k0;
-  uint32_t n2 = hi0 ^ c[3] ^ k1;
-  c[0] = n0;
-  c[1] = lo1;
-  c[2] = n2;
-  c[3] = lo0;
-}
-
-__device__ void philox4x32_10(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
-  const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    philox_round(c, k0, k1);
-    k0 += W0;
-    k1 += W1;
-  }
-}
 
 constexpr int SAMPLER_THREADS = 1024;  // tile patterns; row patterns launch 256 (fewer lists to fill)
 constexpr int SCAN_CAP = 2048;  // tile-columns whose running count fits in shared memory
