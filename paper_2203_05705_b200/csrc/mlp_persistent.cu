@@ -77,7 +77,7 @@ constexpr int MP_BAR_OFF = MP_SDO_OFF + 128 * MP_SMALL_N * 4;
 constexpr int MP_NBARS = 2 * MP_STAGES + MP_NI + 1;
 constexpr int MP_CDF_OFF = (MP_BAR_OFF + 8 * MP_NBARS + 15) / 16 * 16;
 constexpr int MP_MISC_OFF = MP_CDF_OFF + 64 * 8;
-constexpr int MP_SMEM = MP_MISC_OFF + 512 + 1024;   // + slack for the 1024-byte alignment of the ring
+constexpr int MP_SMEM = MP_MISC_OFF + 128 + 2 * (MP_MAX_LAYERS - 1) * 2 * 80 + 64 + 1024;   // + slack for the 1024-byte alignment of the ring
 static_assert(MP_SMEM <= 227 * 1024, "shared memory of the iteration kernel");
 
 enum { JT_F = 0, JT_BD = 1, JT_BW = 2 };
@@ -128,11 +128,14 @@ struct MpParams {
 
 struct LayerRt { int dp, bb, n, npad; };  // period, offset - 1, kept neurons, the latter rounded up to 64
 
+constexpr int MP_MAX_MINE = 24;  // most tiles of one product a CTA can be dealt (checked on the host)
 struct GemmJob {
   int type, l;
   int items, nkb, nt, ntn;
-  int base;  // first index in the stage's item numbering
+  int mine;                  // tiles of this CTA
+  short tile[MP_MAX_MINE];   // their numbers
 };
+static_assert(sizeof(GemmJob) <= 80, "room per product in shared memory");
 
 __device__ __forceinline__ unsigned int mp_ld_acquire(const unsigned int* p) {
   unsigned int v;
@@ -198,9 +201,13 @@ __device__ __forceinline__ void store16_bf16(__nv_bfloat16* dst, const float (&v
 // block is reached through a generic pointer, i.e. by loads that go to the L2 instead of the constant bank, a
 // memory round trip per field on the critical path of every stage.
 
-// The products of stage st, written by one thread into shared memory.
-__device__ __forceinline__ int mp_make_jobs(const MpParams& p, const LayerRt* rt, int H, int G, int st, GemmJob* job) {
-  int njobs = 0, next_base = 0;
+// The products of stage st and the tiles of this CTA, written by one thread into shared memory (all stages are set
+// up at the start of the kernel).  Tiles are dealt round-robin.  A stage with two products deals the second one (the
+// weight gradient: many short tiles) past the CTAs that hold a tile of the first (the input gradient: few tiles
+// with a long contraction) for as many rounds as that tile is worth, when enough other CTAs are left.
+__device__ __forceinline__ int mp_make_jobs(const MpParams& p, const LayerRt* rt, int H, int G, int cta, int st,
+                                            GemmJob* job) {
+  int njobs = 0;
   if (st < H) {
     const int l = st;
     GemmJob& j = job[njobs++];
@@ -209,7 +216,6 @@ __device__ __forceinline__ int mp_make_jobs(const MpParams& p, const LayerRt* rt
     j.items = (rt[l].n + j.nt - 1) / j.nt;
     j.nkb = l == 0 ? (p.layer[0].K + MP_BK - 1) / MP_BK : rt[l - 1].npad / MP_BK;
     j.ntn = 1;
-    j.base = next_base; next_base += j.items;
   } else {
     const int l = H - 1 - (st - H);
     const int nin = l == 0 ? p.layer[0].K : rt[l - 1].n;
@@ -220,7 +226,6 @@ __device__ __forceinline__ int mp_make_jobs(const MpParams& p, const LayerRt* rt
       j.items = (nin + 63) / 64;
       j.nkb = rt[l].npad / MP_BK;
       j.ntn = 1;
-      j.base = next_base; next_base += j.items;
     }
     GemmJob& j = job[njobs++];
     j.type = JT_BW; j.l = l;
@@ -228,19 +233,44 @@ __device__ __forceinline__ int mp_make_jobs(const MpParams& p, const LayerRt* rt
     j.ntn = (nin + 63) / 64;
     j.items = ((rt[l].n + 127) / 128) * j.ntn;
     j.nkb = (p.B + MP_BK - 1) / MP_BK;
-    j.base = next_base; next_base += j.items;
+  }
+  // first product: tile cta, cta + G, ...
+  {
+    GemmJob& j = job[0];
+    j.mine = 0;
+    for (int i = cta; i < j.items && j.mine < MP_MAX_MINE; i += G) j.tile[j.mine++] = (short)i;
+  }
+  if (njobs > 1) {
+    GemmJob& j = job[1];
+    const int nbd = min(job[0].items, G);
+    int skip = min(4, job[0].nkb / 8);           // rounds in which the holders of a long tile are passed over
+    if ((G - nbd) * 2 < G) skip = 0;
+    j.mine = 0;
+    int next = 0;                                 // first tile of the current round
+    for (int r = 0; next < j.items && j.mine < MP_MAX_MINE; ++r) {
+      if (r < skip) {
+        if (cta >= nbd && next + (cta - nbd) < j.items) j.tile[j.mine++] = (short)(next + (cta - nbd));
+        next += G - nbd;
+      } else {
+        // the rounds after that start behind the long tiles' holders, so that those come last
+        const int slot = cta >= nbd ? cta - nbd : cta + (G - nbd);
+        if (next + slot < j.items) j.tile[j.mine++] = (short)(next + slot);
+        next += G;
+      }
+    }
   }
   return njobs;
 }
 
-// CUDA-core work of forward stage st, done by the MP_CC_THREADS threads `ct` of every CTA.  Every loop here is
-// bound by memory latency: a thread issues a batch of independent loads before it uses the first.
-__device__ __forceinline__ void mp_forward_jobs(const MpParams& p, const LayerRt* rt, int H, int st, int cta, int G, int ct) {
-  const int gthreads = G * MP_CC_THREADS, gtid = cta * MP_CC_THREADS + ct;
-  if (st == 0) {
+// CUDA-core work of stage 0, done by thread gtid of gthreads: the CUDA-core warps of every CTA (ct = 0 .. MP_CC_THREADS-1
+// inside the CTA) and, in the CTAs that have no tile of the first product, the other warps too (ct = -1).  Every
+// loop here is bound by memory latency: a thread issues a batch of independent loads before it uses the first.
+__device__ __forceinline__ void mp_forward_jobs(const MpParams& p, const LayerRt* rt, int H, int cta, int G, int ct,
+                                                int gtid, int gthreads) {
+  {
     // (a) headers and kept lists of the patterns, as the sampler kernel leaves them: the last CTAs, one per layer
     const int l = G - 1 - cta;
-    if (l < H && p.layer[l].sample) {
+    if (ct >= 0 && l < H && p.layer[l].sample) {
       const MpLayer& y = p.layer[l];
       if (ct == 0) {
         y.hdr[HDR_KIND] = ARD_ROW;
@@ -532,10 +562,10 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(smem + MP_MISC_OFF);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + MP_MISC_OFF + 4);
   volatile int* stop_flag = reinterpret_cast<volatile int*>(smem + MP_MISC_OFF + 8);
-  volatile int* s_njobs = reinterpret_cast<volatile int*>(smem + MP_MISC_OFF + 12);
+  volatile int* s_njobs = reinterpret_cast<volatile int*>(smem + MP_MISC_OFF + 96);  // [stage]
   LayerRt* s_rt = reinterpret_cast<LayerRt*>(smem + MP_MISC_OFF + 16);  // [MP_MAX_LAYERS]
   unsigned long long* s_count = reinterpret_cast<unsigned long long*>(smem + MP_MISC_OFF + 16 + 16 * MP_MAX_LAYERS);
-  GemmJob* job = reinterpret_cast<GemmJob*>(smem + MP_MISC_OFF + 128);  // [2], written by thread 0
+  GemmJob* jobs = reinterpret_cast<GemmJob*>(smem + MP_MISC_OFF + 128);  // [stage][2]
 
   // A block-wide barrier counts a warp once, whichever of its lanes execute it: every warp first waits for its own
   // lanes (the lanes of the producer warp and lane 0 of the issuing warps come out of their loops one by one).
@@ -614,14 +644,14 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
   // the patterns and the stage's products are read from shared memory: indexed by layer they would otherwise sit
   // in local memory, for whose lines the 200 KB of shared memory leave almost no L1
   const LayerRt* rt = s_rt;
-  if (tid == 0) *s_njobs = mp_make_jobs(p, rt, H, G, 0, job);
+  if (tid < 2 * H) s_njobs[tid] = mp_make_jobs(p, rt, H, G, cta, tid, jobs + 2 * tid);
   block_sync();
 
   // per-role running counters: contraction blocks and tiles this CTA has been through
   int gblk = 0, git = 0;
   unsigned int barrier_no = 0;
   const int n_stages = 2 * H;
-  const int nt0 = job[0].nt;  // tile width of layer 0
+  const int nt0 = jobs[0].nt;  // tile width of layer 0
 
   // The first layer's weight is read in place: its kept rows are b-1, b-1+dp, ... (Eq. 1), which a descriptor
   // with the pitch dp x ldw follows.  The producer warp fits the two box shapes it will use to the pattern.
@@ -660,26 +690,20 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
     if (tid == 0) MP_GT(0);
 #endif
     // ---- the products of this stage (set up by thread 0 before the barrier that opened the stage) ----
-    const int njobs = *s_njobs;
-    // first tile of this CTA: tiles are dealt round-robin over the stage's numbering (a loop instead of a
-    // remainder: the operands are a few multiples of G apart at most, and a division costs a microsecond of every
-    // role's start-up)
-    auto first_item = [&](const GemmJob& j) {
-      int r = cta - j.base;
-      while (r < 0) r += G;
-      return j.base + r;
-    };
-
-    if (warp == 0) {
+    const int njobs = s_njobs[st];
+    const GemmJob* job = jobs + 2 * st;
+    if (st == 0 && warp < MP_CC_W0 && job[0].mine == 0) {
+      // no tile in the first stage: these warps help to pack the weights
+      const int T = min(G, job[0].items);
+      mp_forward_jobs(p, rt, H, cta, G, -1, G * MP_CC_THREADS + (cta - T) * (MP_CC_W0 * 32) + tid,
+                      G * MP_CC_THREADS + (G - T) * (MP_CC_W0 * 32));
+    } else if (warp == 0) {
       // ===================== producer =====================
       // Lane s owns ring stage s: it waits for the stage, announces the bytes and issues the two or three boxes
       // of every block that falls on its stage, so up to MP_STAGES blocks are requested at once (one thread
       // issuing box after box, with a barrier hand-off each, paces at ~400 cycles per box).
       int stage_blocks = 0;  // contraction blocks of this CTA in this stage
-      for (int q = 0; q < njobs; ++q) {
-        const int f = first_item(job[q]);
-        for (int i = f; i < job[q].base + job[q].items; i += G) stage_blocks += job[q].nkb;
-      }
+      for (int q = 0; q < njobs; ++q) stage_blocks += job[q].mine * job[q].nkb;
       if (lane < MP_STAGES) {
         int d = (lane - gblk % MP_STAGES + MP_STAGES) % MP_STAGES;  // this lane's first block among the stage's blocks
         int seq0 = 0;
@@ -702,8 +726,8 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
           }
           const uint32_t bytes = (uint32_t)(MP_A_BYTES + (j.type == JT_F ? j.nt * 128 : MP_B_BYTES));
 #pragma unroll 1
-          for (int i = first_item(j); i < j.base + j.items && ok; i += G, seq0 += j.nkb) {
-            const int t = i - j.base;
+          for (int ti = 0; ti < j.mine && ok; ++ti, seq0 += j.nkb) {
+            const int t = j.tile[ti];
 #pragma unroll 1
             for (; d < seq0 + j.nkb; d += MP_STAGES) {
               const int kb = d - seq0;
@@ -745,7 +769,7 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
           const uint32_t idesc = make_idesc(j.nt, a_mn, b_mn, 128);
           const uint32_t d_tmem = tmem_base + (uint32_t)(w * MP_ACC_COLS);
 #pragma unroll 1
-          for (int i = first_item(j); i < j.base + j.items && ok; i += G, ++git, gblk += j.nkb) {
+          for (int ti = 0; ti < j.mine && ok; ++ti, ++git, gblk += j.nkb) {
             // the epilogue warps have taken the previous tile's sums out of the accumulators
             if (!mp_wait(tempty_bar, ((uint32_t)git & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
@@ -796,8 +820,8 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
         const int nin = l == 0 ? y.K : rt[l - 1].n;
         const uint32_t magic = (uint32_t)(0x100000000ull / (unsigned)dpi) + 1u;  // exact x / dpi for x < 2^16
 #pragma unroll 1
-        for (int i = first_item(j); i < j.base + j.items && ok; i += G, ++git) {
-          const int t = i - j.base;
+        for (int ti = 0; ti < j.mine && ok; ++ti, ++git) {
+          const int t = j.tile[ti];
           // ---- what does not depend on the accumulators is fetched while the products run ----
           float dO[MP_SMALL_N];
           __syncwarp();
@@ -1027,7 +1051,10 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
       // ===================== CUDA-core warps: the rest of the stage, beside the tiles =====================
       const int ct = tid - MP_CC_W0 * 32;
       MP_MARKC(0);
-      if (st == 0) mp_forward_jobs(p, rt, H, st, cta, G, ct);
+      if (st == 0) {
+        const int T = min(G, job[0].items);  // CTAs 0 .. T-1 have a tile; the others lend their idle warps
+        mp_forward_jobs(p, rt, H, cta, G, ct, cta * MP_CC_THREADS + ct, G * MP_CC_THREADS + (G - T) * (MP_CC_W0 * 32));
+      }
       if (st >= H) {
         const float* sdO = reinterpret_cast<const float*>(smem + MP_SDO_OFF);
         MP_MARKC(1);
@@ -1056,7 +1083,6 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
         *stop_flag = *abort_flag;
         // the draw of this iteration has been read by every CTA: the next launch draws the next one
         if (st == 0 && cta == 0 && p.any_sampled && p.counter != nullptr && !*abort_flag) *p.counter = *s_count + 1ull;
-        *s_njobs = mp_make_jobs(p, rt, H, G, st + 1, job);
       }
       block_sync();
       // what other CTAs stored with ordinary stores is read by TMA from here on
@@ -1117,6 +1143,10 @@ ard_status launch_mlp_persistent(ard_ctx* ctx, const ard_mlp_layer* layers, int 
     if (y.K % 8 != 0 || y.ldw % 8 != 0 || y.ldw < y.K || !aligned16(y.W) || !aligned16(y.dW)) return ARD_ERR_UNSUPPORTED;
     if (l > 0 && (!y.Wk || !aligned16(y.Wk))) return ARD_ERR_UNSUPPORTED;
     if (l < H) {
+      // no CTA may be dealt more tiles of a product than its list holds (half of the SMs is the fewest the weight
+      // gradient is spread over)
+      const int bw_tiles = ((y.N + 127) / 128) * ((y.K + 63) / 64), half = ctx->sm_count / 2 > 0 ? ctx->sm_count / 2 : 1;
+      if ((bw_tiles + half - 1) / half + 5 > MP_MAX_MINE || y.N > 32767 || y.K > 32767) return ARD_ERR_UNSUPPORTED;
       if (!y.compact_out || y.N % 64 != 0 || !y.dZ || !aligned16(y.A) || !aligned16(y.dZ)) return ARD_ERR_UNSUPPORTED;
       if (y.sample) any_sampled = true;
     } else {
