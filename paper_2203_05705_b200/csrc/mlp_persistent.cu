@@ -24,29 +24,12 @@
 // all SMs: what bounds a tile is its 128-row operand streaming through one SM.
 // The patterns are drawn by every CTA for itself (a few hundred instructions).  Every wait is bounded; a CTA that
 // gives up records the status, which the others poll at the grid barrier.
-#ifdef MP_TIMING
-#include <cstdio>
-#endif
 #include "ard_internal.h"
 #include "philox.h"
 #include "sm100_ptx.h"
 
 namespace {
 
-#ifdef MP_TIMING
-__device__ long long g_mark[4][8][8];  // [cta slot][stage][event]
-#ifndef MP_MARK_CTA
-#define MP_MARK_CTA 0
-#endif
-#define MP_MARK(ev) do { if (cta == MP_MARK_CTA && g_mark[0][st][ev] == 0) g_mark[0][st][ev] = clock64() - t_start; } while (0)
-__device__ unsigned long long g_gt[160][8][4];
-#define MP_GT(slot) do { g_gt[cta][st][slot] = global_ns(); } while (0)
-#define MP_MARKC(ev) do { __syncwarp(); if (cta == 147 && ct == 0) g_mark[1][st][ev] = clock64() - t_start; } while (0)
-#else
-#define MP_MARK(ev)
-#define MP_MARKC(ev)
-#define MP_GT(slot)
-#endif
 
 constexpr int MP_MAX_LAYERS = 4;                    // hidden layers + the output layer
 constexpr int MP_NI = 2;                            // issuing warps = accumulators per tile
@@ -322,14 +305,39 @@ __device__ __forceinline__ void mp_forward_jobs(const MpParams& p, const LayerRt
           if (dpi == 1) {
             *reinterpret_cast<uint4*>(dst + c0[k]) = v[k];
           } else {
+            // the kept ones among these 8 columns are consecutive in the packed row: gather them (at most 4) and
+            // store them with as few instructions as their alignment allows (a store instruction costs a warp
+            // ~150 cycles whatever its width)
             const uint32_t w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
+            int rel0 = c0[k] - bi;                       // position of column c0 relative to the first kept one
+            int e0 = 0;                                  // first kept column of this piece
+            if (rel0 < 0) { e0 = -rel0; rel0 = 0; }
+            else {
+              const int jq0 = (int)__umulhi((uint32_t)(rel0 + dpi - 1), magic);
+              e0 = jq0 * dpi - rel0;
+              rel0 = jq0 * dpi;
+            }
+            const int j0 = (int)__umulhi((uint32_t)rel0, magic);   // packed column of that one (rel0 is a multiple of dpi)
+            unsigned long long pk = 0ull;
+            int cnt = 0, nk = e0;                        // nk: the next kept column of the piece
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-              const int rel = c0[k] + e - bi;
-              if (rel < 0) continue;
-              const int jq = (int)__umulhi((uint32_t)rel, magic);
-              if (jq * dpi == rel && jq < nin)
-                dst[jq] = __ushort_as_bfloat16((unsigned short)((w[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu));
+              if (e == nk) {
+                nk += dpi;
+                if (j0 + cnt < nin) {
+                  pk |= (unsigned long long)((w[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu) << (16 * cnt);
+                  ++cnt;
+                }
+              }
+            }
+            __nv_bfloat16* d = dst + j0;
+            if (cnt == 4 && (j0 & 3) == 0) {
+              *reinterpret_cast<unsigned long long*>(d) = pk;
+            } else {
+              int done = 0;
+              if (cnt >= 1 && (j0 & 1)) { d[0] = __ushort_as_bfloat16((unsigned short)(pk & 0xFFFFu)); done = 1; }
+              for (; done + 2 <= cnt; done += 2) *reinterpret_cast<uint32_t*>(d + done) = (uint32_t)(pk >> (16 * done));
+              if (done < cnt) d[done] = __ushort_as_bfloat16((unsigned short)((pk >> (16 * done)) & 0xFFFFu));
             }
           }
         }
@@ -676,19 +684,37 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
     if (lane == 1) asm volatile("prefetch.tensormap [%0];" ::"l"(mapW0b) : "memory");
   }
 
-#ifdef MP_TIMING
-  long long tlog[8][3];
-  __shared__ long long s_t0;
-  if (tid == 0) s_t0 = clock64();
-  if (cta == MP_MARK_CTA && tid < 64) g_mark[0][tid >> 3][tid & 7] = 0;
-  block_sync();
-  const long long t_start = s_t0;
-#endif
+  // The output weights of a tile's neurons of the last hidden layer (columns bb + j dp of the output layer's
+  // weight), [chunk][output][16], into an epilogue warp's own staging block: no other warp is waited for.  All
+  // loads of a round are issued before the first one is used: rolled up, each would wait for the one before it.
+  auto stage_out_weights = [&](float* stg, int t, int nt, int lane_) {
+    const MpLayer& yo = p.layer[H];
+    const int l = H - 1;
+    const int total = (nt / 16) * 256;
+#pragma unroll 1
+    for (int e0 = 0; e0 < total; e0 += 512) {
+      float wv[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int e = e0 + lane_ + 32 * k;
+        const int o = (e >> 4) & 15;
+        const int col = t * nt + (e >> 8) * 16 + (e & 15);
+        wv[k] = 0.f;
+        if (e < total && o < yo.N && col < rt[l].n)
+          wv[k] = __bfloat162float(yo.W[(size_t)o * yo.ldw + rt[l].bb + (size_t)col * rt[l].dp]);
+      }
+#pragma unroll
+      for (int k = 0; k < 16; ++k)
+        if (e0 + lane_ + 32 * k < total) stg[e0 + lane_ + 32 * k] = wv[k];
+    }
+  };
+  // With more than one hidden layer the last one's product is stages away: its first tile's output weights are
+  // fetched now, off that stage's critical path (the stages before it leave this part of the staging block alone).
+  if (H > 1 && warp >= MP_EPI_W0 && warp < MP_CC_W0 && jobs[2 * (H - 1)].mine > 0)
+    stage_out_weights(reinterpret_cast<float*>(smem + MP_STG_OFF) + (warp - MP_EPI_W0) * MP_STG_WORDS,
+                      jobs[2 * (H - 1)].tile[0], jobs[2 * (H - 1)].nt, lane);
+
   for (int st = 0; st < n_stages; ++st) {
-#ifdef MP_TIMING
-    tlog[st][0] = clock64() - t_start;
-    if (tid == 0) MP_GT(0);
-#endif
     // ---- the products of this stage (set up by thread 0 before the barrier that opened the stage) ----
     const int njobs = s_njobs[st];
     const GemmJob* job = jobs + 2 * st;
@@ -736,7 +762,6 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
               const uint32_t sA = base + lane * MP_STAGE_BYTES;
               const uint32_t sB = sA + MP_A_BYTES;
               mbar_arrive_expect_tx(full_bar(lane), bytes);
-              if (d == 0) MP_MARK(0);
               const int kx = kb * MP_BK;
               if (j.type == JT_F) {
                 tma_load_2d(sA, ma, full_bar(lane), kx, 0);
@@ -780,7 +805,6 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
               const uint32_t phase = (uint32_t)(g / MP_STAGES) & 1u;
               if (!mp_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
               tc_fence_after();
-              if (w == 0 && kb == 0) MP_MARK(1);
               const uint32_t sA = base + stage * MP_STAGE_BYTES;
               const uint64_t ad0 = desc_a_hi | (uint64_t)((sA & 0x3FFFFu) >> 4);
               const uint64_t bd0 = desc_b_hi | (uint64_t)(((sA + MP_A_BYTES) & 0x3FFFFu) >> 4);
@@ -795,7 +819,6 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
             if (!ok) break;
             if (w < j.nkb) tc_commit(tfull_bar(w));
             else mbar_arrive(tfull_bar(w));  // no block of this tile was this warp's
-            if (w == 0 ) MP_MARK(2);
           }
         }
       }
@@ -825,7 +848,6 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
           // ---- what does not depend on the accumulators is fetched while the products run ----
           float dO[MP_SMALL_N];
           __syncwarp();
-          if (warp == MP_EPI_W0 && lane == 0 ) MP_MARK(5);
           if (j.type == JT_F) {
             // biases of the tile's neurons behind the (at most) 1024 staged output weights
 #pragma unroll
@@ -834,28 +856,8 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
               stg[1024 + jj] = (y.bias != nullptr && jj < j.nt && jc < rt[l].n) ? __ldg(y.bias + rt[l].bb + (size_t)jc * rt[l].dp) : 0.f;
             }
             if (fused_dz) {
-              // The output weights of the tile's neurons (columns bb + j dp of the output layer's weight),
-              // [chunk][output][16], in the warp's own staging block: no other warp is waited for.  All loads of a
-              // round are issued before the first one is used: rolled up, each would wait for the one before it.
-#pragma unroll 1
-              for (int e0 = 0; e0 < nch * 256; e0 += 512) {
-                float wv[16];
-#pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                  const int e = e0 + lane + 32 * k;
-                  const int o = (e >> 4) & 15;
-                  const int col = t * j.nt + (e >> 8) * 16 + (e & 15);
-                  wv[k] = 0.f;
-                  if (e < nch * 256 && o < yo.N && col < rt[l].n) {
-                    // stage H-1 >= 1: the packed copy of stage 0 (contiguous); a single hidden layer: the weight itself
-                    wv[k] = __bfloat162float(H > 1 ? __ldcg(yo.Wk + (size_t)o * yo.ldw + col)
-                                                   : yo.W[(size_t)o * yo.ldw + rt[l].bb + (size_t)col * rt[l].dp]);
-                  }
-                }
-#pragma unroll
-                for (int k = 0; k < 16; ++k)
-                  if (e0 + lane + 32 * k < nch * 256) stg[e0 + lane + 32 * k] = wv[k];
-              }
+              // the first tile's output weights were staged before the first stage (see below)
+              if (ti > 0 || H == 1) stage_out_weights(stg, t, j.nt, lane);
               const float* sdOe = reinterpret_cast<const float*>(smem + MP_SDO_OFF);
 #pragma unroll
               for (int o = 0; o < MP_SMALL_N; ++o) dO[o] = sdOe[o * 128 + row];
@@ -874,13 +876,11 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
             for (int k = 0; k < 8; ++k) reinterpret_cast<uint4*>(stg + lane * 36)[k] = a[k];
           }
           __syncwarp();
-          if (warp == MP_EPI_W0 && lane == 0 ) MP_MARK(6);
           bool all = true;
 #pragma unroll
           for (int w = 0; w < MP_NI; ++w) all = all && mp_wait(tfull_bar(w), (uint32_t)git & 1u, abort_flag, p.status);
           if (!all) { ok = false; break; }
           tc_fence_after();
-          if (warp == MP_EPI_W0 && lane == 0 ) MP_MARK(3);
           if (j.type == JT_BW) {
             // Weight gradient: accumulator row = kept neuron mt*128 + row, columns = kept fan-in ni*64 ...  The whole
             // 32 x 64 block of the warp leaves tensor memory first; then the warp stores one neuron's 64 values after
@@ -893,13 +893,15 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
               float acc[16];
 #pragma unroll
               for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-#pragma unroll 1
-              for (int w = 0; w < nacc; ++w) {
-                uint32_t r[16];
-                tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(w * MP_ACC_COLS + ch * 16), r);
+              {
+                static_assert(MP_NI == 2, "two accumulators are read side by side");
+                uint32_t r0[16], r1[16];
+                const uint32_t ta = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ch * 16);
+                tmem_ld16(ta, r0);
+                if (nacc > 1) tmem_ld16(ta + MP_ACC_COLS, r1);
                 tmem_ld_wait();
 #pragma unroll
-                for (int e = 0; e < 16; ++e) acc[e] += __uint_as_float(r[e]);
+                for (int e = 0; e < 16; ++e) acc[e] = __uint_as_float(r0[e]) + (nacc > 1 ? __uint_as_float(r1[e]) : 0.f);
               }
 #pragma unroll
               for (int e = 0; e < 16; ++e) stg[lane * MP_STG_LD + ch * 16 + e] = acc[e];
@@ -961,13 +963,14 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
             float acc[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e) acc[e] = 0.f;
-#pragma unroll 1
-            for (int w = 0; w < nacc; ++w) {
-              uint32_t r[16];
-              tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(w * MP_ACC_COLS + ch * 16), r);
+            {
+              uint32_t r0[16], r1[16];
+              const uint32_t ta = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ch * 16);
+              tmem_ld16(ta, r0);
+              if (nacc > 1) tmem_ld16(ta + MP_ACC_COLS, r1);
               tmem_ld_wait();
 #pragma unroll
-              for (int e = 0; e < 16; ++e) acc[e] += __uint_as_float(r[e]);
+              for (int e = 0; e < 16; ++e) acc[e] = __uint_as_float(r0[e]) + (nacc > 1 ? __uint_as_float(r1[e]) : 0.f);
             }
             if (ch == nch - 1) {  // the accumulators may be overwritten from here on
               tc_fence_before();
@@ -989,13 +992,26 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
               }
               if (fused_dz) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                  float s = 0.f;
+                for (int e = 0; e < 16; ++e) dz[e] = 0.f;
 #pragma unroll
-                  for (int o = 0; o < MP_SMALL_N; ++o) s += dO[o] * stg[(ch * MP_SMALL_N + o) * 16 + e];
+                for (int o = 0; o < MP_SMALL_N; ++o) {
+                  if (o < yo.N) {
+                    const float4* wq = reinterpret_cast<const float4*>(stg + (ch * MP_SMALL_N + o) * 16);
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                      const float4 w4 = wq[q4];
+                      dz[4 * q4] += dO[o] * w4.x;
+                      dz[4 * q4 + 1] += dO[o] * w4.y;
+                      dz[4 * q4 + 2] += dO[o] * w4.z;
+                      dz[4 * q4 + 3] += dO[o] * w4.w;
+                    }
+                  }
+                }
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
                   const uint32_t bits = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(acc[e]));
                   const bool pass = !y.relu || bf16_bits_positive(bits);
-                  dz[e] = (j0 + e < rt[l].n && pass) ? y.alpha * s : 0.f;
+                  dz[e] = (j0 + e < rt[l].n && pass) ? y.alpha * dz[e] : 0.f;
                 }
               }
               if (row_ok) {
@@ -1044,38 +1060,26 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
               }
             }
           }
-          if (warp == MP_EPI_W0 && lane == 0 ) MP_MARK(4);
         }
       }
     } else {
       // ===================== CUDA-core warps: the rest of the stage, beside the tiles =====================
       const int ct = tid - MP_CC_W0 * 32;
-      MP_MARKC(0);
       if (st == 0) {
         const int T = min(G, job[0].items);  // CTAs 0 .. T-1 have a tile; the others lend their idle warps
         mp_forward_jobs(p, rt, H, cta, G, ct, cta * MP_CC_THREADS + ct, G * MP_CC_THREADS + (G - T) * (MP_CC_W0 * 32));
       }
       if (st >= H) {
         const float* sdO = reinterpret_cast<const float*>(smem + MP_SDO_OFF);
-        MP_MARKC(1);
         mp_backward_jobs(p, rt, H, st, sdO, cta, G, ct);
       }
-      MP_MARKC(2);
       if (st < H) mp_zero_fill(p, rt, H, st, cta, G, ct);
-      MP_MARKC(3);
     }
-#ifdef MP_TIMING
-    tlog[st][1] = clock64() - t_start;  // this thread's own work of the stage is done
-    __syncwarp();
-    if (warp == MP_EPI_W0 && lane == 0) MP_GT(1);
-    if (warp == MP_CC_W0 && lane == 0) MP_GT(2);
-#endif
 
     // ---- grid-wide barrier (none behind the last stage) ----
     if (st + 1 < n_stages) {
       block_sync();
       if (tid == 0) {
-        MP_GT(3);
         __threadfence();
         atomicAdd(p.bar, 1u);
         ++barrier_no;
@@ -1089,31 +1093,8 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
       asm volatile("fence.proxy.async.global;" ::: "memory");
       if (*stop_flag) break;
     }
-#ifdef MP_TIMING
-    tlog[st][2] = clock64() - t_start;
-#endif
   }
 
-#ifdef MP_TIMING
-  if (tid == 0) {
-    const int st = n_stages - 1;
-    MP_GT(3);
-    for (int k = 0; k < n_stages; ++k)
-      printf("GT %d %d %llu %llu %llu %llu\n", cta, k, g_gt[cta][k][0], g_gt[cta][k][1], g_gt[cta][k][2], g_gt[cta][k][3]);
-  }
-  if (tid == 0 && cta == MP_MARK_CTA)
-    for (int st = 0; st < n_stages; ++st)
-      printf("  marks stage %d: epi_enter %lld first_issue %lld epi_prefetched %lld first_full %lld last_commit %lld tfull %lld epi_done %lld\n", st, g_mark[0][st][5],
-             g_mark[0][st][0], g_mark[0][st][6], g_mark[0][st][1], g_mark[0][st][2], g_mark[0][st][3], g_mark[0][st][4]);
-  if (tid == 0 && cta == 147)
-    for (int st = 0; st < n_stages; ++st)
-      printf("  cc marks stage %d: enter %lld sdO %lld jobs %lld zero %lld\n", st, g_mark[1][st][0], g_mark[1][st][1], g_mark[1][st][2], g_mark[1][st][3]);
-  if (lane == 0 && (cta == 0 || cta == 20 || cta == 100 || cta == G - 1) && (warp == 0 || warp == MP_EPI_W0 || warp == MP_CC_W0)) {
-    for (int st = 0; st < n_stages; ++st)
-      printf("cta %d warp %d stage %d: start %lld own_work_done %lld next %lld | dp %d/%d\n", cta, warp, st, tlog[st][0], tlog[st][1],
-             tlog[st][2], rt[0].dp, rt[1].dp);
-  }
-#endif
   // ---- teardown ----
   tc_fence_before();
   block_sync();
