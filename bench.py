@@ -671,6 +671,14 @@ def run_mlp_step(args, wl):
         detail["ms_per_step"]["graph_compact_warm_l2"] = ms / steps
         del flush
         detail["ms_per_step"]["eager_compact"] = timed(lambda: eager(compact), n2, warm)[0] / n2
+        # the same iterations call by call (one launch per product, three streams) instead of the one-kernel form
+        if launches_per_step == 1:
+            ard.ard_set_option(ctx, ard.ARD_OPT_MLP_PERSISTENT, 0)
+            gr_c = graphed(compact)
+            detail["ms_per_step"]["graph_compact_call_by_call"] = timed(gr_c.replay, n2, warm)[0] / n2
+            detail["ms_per_step"]["eager_compact_call_by_call"] = timed(lambda: eager(compact), n2, warm)[0] / n2
+            ard.ard_set_option(ctx, ard.ARD_OPT_MLP_PERSISTENT, 1)
+            del gr_c
         fullw = make_stack(0)
         gr_f = graphed(fullw)
         detail["ms_per_step"]["graph_full_width"] = timed(gr_f.replay, n2, warm)[0] / n2

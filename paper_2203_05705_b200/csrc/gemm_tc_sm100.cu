@@ -1379,6 +1379,7 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
 
   // ---- teardown ----
   tc_fence_before();
+  __syncwarp();  // lanes that left their role's loop one by one arrive at the block-wide barrier together
   if (CTAS == 2) cluster_sync_all();  // neither CTA may leave while its peer can still touch its memory
   else __syncthreads();
   if (warp == 1) {

@@ -340,6 +340,7 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
 
   // ---- teardown ----
   tc_fence_before();
+  __syncwarp();  // lanes that left their role's loop one by one arrive at the block-wide barrier together
   __syncthreads();
   if (warp == 15) {
     __syncwarp();
@@ -674,6 +675,7 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
 
   // ---- teardown ----
   tc_fence_before();
+  __syncwarp();  // lanes that left their role's loop one by one arrive at the block-wide barrier together
   __syncthreads();
   if (warp == 15) {
     __syncwarp();

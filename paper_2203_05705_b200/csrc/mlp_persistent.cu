@@ -271,7 +271,7 @@ __device__ __forceinline__ void mp_forward_jobs(const MpParams& p, const LayerRt
     }
     // (b) packed weights of the layers behind a dropped layer: Wk[i][j] = W[bb + i dp][bi + j dpi], zeros up to the
     //     next multiples of 64 both ways.  A thread reads 16 bytes of a kept row (8 fan-in columns) and stores those
-    //     that are kept, so the kept rows are read once, in whole lines; eight pieces are in flight per thread.
+    //     that are kept, so the kept rows are read once, in whole lines; four pieces are in flight per thread.
 #pragma unroll 1
     for (int l2 = 1; l2 <= H; ++l2) {
       const MpLayer& y = p.layer[l2];
@@ -283,11 +283,11 @@ __device__ __forceinline__ void mp_forward_jobs(const MpParams& p, const LayerRt
       const int vecs = y.K / 8;                 // 16-byte pieces of a weight row
       const int units = nkeep * vecs;
 #pragma unroll 1
-      for (int u0 = gtid; u0 < units; u0 += 8 * gthreads) {
-        uint4 v[8];
-        int ik[8], c0[8];
+      for (int u0 = gtid; u0 < units; u0 += 4 * gthreads) {
+        uint4 v[4];
+        int ik[4], c0[4];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int k = 0; k < 4; ++k) {
           const int u = u0 + k * gthreads;
           ik[k] = -1;
           c0[k] = 0;
@@ -299,45 +299,25 @@ __device__ __forceinline__ void mp_forward_jobs(const MpParams& p, const LayerRt
           }
         }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int k = 0; k < 4; ++k) {
           if (ik[k] < 0) continue;
           __nv_bfloat16* dst = y.Wk + (size_t)ik[k] * y.ldw;
           if (dpi == 1) {
             *reinterpret_cast<uint4*>(dst + c0[k]) = v[k];
           } else {
-            // the kept ones among these 8 columns are consecutive in the packed row: gather them (at most 4) and
-            // store them with as few instructions as their alignment allows (a store instruction costs a warp
-            // ~150 cycles whatever its width)
-            const uint32_t w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
-            int rel0 = c0[k] - bi;                       // position of column c0 relative to the first kept one
-            int e0 = 0;                                  // first kept column of this piece
-            if (rel0 < 0) { e0 = -rel0; rel0 = 0; }
+            // the kept ones among these 8 columns (Eq. 1), one short store each
+            int rel = c0[k] - bi, e0 = 0;
+            if (rel < 0) { e0 = -rel; rel = 0; }
             else {
-              const int jq0 = (int)__umulhi((uint32_t)(rel0 + dpi - 1), magic);
-              e0 = jq0 * dpi - rel0;
-              rel0 = jq0 * dpi;
+              const int jq0 = (int)__umulhi((uint32_t)(rel + dpi - 1), magic);
+              e0 = jq0 * dpi - rel;
+              rel = jq0 * dpi;
             }
-            const int j0 = (int)__umulhi((uint32_t)rel0, magic);   // packed column of that one (rel0 is a multiple of dpi)
-            unsigned long long pk = 0ull;
-            int cnt = 0, nk = e0;                        // nk: the next kept column of the piece
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              if (e == nk) {
-                nk += dpi;
-                if (j0 + cnt < nin) {
-                  pk |= (unsigned long long)((w[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu) << (16 * cnt);
-                  ++cnt;
-                }
-              }
-            }
-            __nv_bfloat16* d = dst + j0;
-            if (cnt == 4 && (j0 & 3) == 0) {
-              *reinterpret_cast<unsigned long long*>(d) = pk;
-            } else {
-              int done = 0;
-              if (cnt >= 1 && (j0 & 1)) { d[0] = __ushort_as_bfloat16((unsigned short)(pk & 0xFFFFu)); done = 1; }
-              for (; done + 2 <= cnt; done += 2) *reinterpret_cast<uint32_t*>(d + done) = (uint32_t)(pk >> (16 * done));
-              if (done < cnt) d[done] = __ushort_as_bfloat16((unsigned short)((pk >> (16 * done)) & 0xFFFFu));
+            int jq = (int)__umulhi((uint32_t)rel, magic);  // packed column of the first kept one
+#pragma unroll 1
+            for (int e = e0; e < 8 && jq < nin; e += dpi, ++jq) {
+              const uint32_t w = e < 2 ? v[k].x : (e < 4 ? v[k].y : (e < 6 ? v[k].z : v[k].w));
+              dst[jq] = __ushort_as_bfloat16((unsigned short)((w >> ((e & 1) * 16)) & 0xFFFFu));
             }
           }
         }
@@ -445,29 +425,29 @@ __device__ __forceinline__ void mp_backward_jobs(const MpParams& p, const LayerR
         if (sl == 0 && col_ok) y.db[rt[l].bb + (size_t)jc * rt[l].dp] = s;
       }
       if (first) {
-        // the outputs' sums first, then their reductions side by side (one after the other, each would wait for
-        // its own four shuffles)
+        // two outputs per round, their reductions side by side
         const size_t c = (size_t)bi + (size_t)jc * dpi;
-        float so[MP_SMALL_N];
+#pragma unroll 1
+        for (int o = 0; o < yo.N; o += 2) {
+          const bool two = o + 1 < yo.N;
+          float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-        for (int o = 0; o < MP_SMALL_N; ++o) {
-          so[o] = 0.f;
-          if (o < yo.N) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) so[o] += sdO[o * 128 + sl * 8 + k] * a[k];
+          for (int k = 0; k < 8; ++k) {
+            s0 += sdO[o * 128 + sl * 8 + k] * a[k];
+            s1 += sdO[(two ? o + 1 : o) * 128 + sl * 8 + k] * a[k];
           }
-        }
 #pragma unroll
-        for (int off = 2; off < 32; off <<= 1) {
-#pragma unroll
-          for (int o = 0; o < MP_SMALL_N; ++o) so[o] += __shfl_xor_sync(0xffffffffu, so[o], off);
-        }
-        if (sl == 0 && col_ok) {
-#pragma unroll
-          for (int o = 0; o < MP_SMALL_N; ++o) {
-            if (o < yo.N) {
-              if (yo.dW_is_f32) reinterpret_cast<float*>(yo.dW)[(size_t)o * yo.ldw + c] = so[o];
-              else reinterpret_cast<__nv_bfloat16*>(yo.dW)[(size_t)o * yo.ldw + c] = __float2bfloat16_rn(so[o]);
+          for (int off = 2; off < 32; off <<= 1) {
+            s0 += __shfl_xor_sync(0xffffffffu, s0, off);
+            s1 += __shfl_xor_sync(0xffffffffu, s1, off);
+          }
+          if (sl == 0 && col_ok) {
+            if (yo.dW_is_f32) {
+              reinterpret_cast<float*>(yo.dW)[(size_t)o * yo.ldw + c] = s0;
+              if (two) reinterpret_cast<float*>(yo.dW)[(size_t)(o + 1) * yo.ldw + c] = s1;
+            } else {
+              reinterpret_cast<__nv_bfloat16*>(yo.dW)[(size_t)o * yo.ldw + c] = __float2bfloat16_rn(s0);
+              if (two) reinterpret_cast<__nv_bfloat16*>(yo.dW)[(size_t)(o + 1) * yo.ldw + c] = __float2bfloat16_rn(s1);
             }
           }
         }
@@ -718,11 +698,10 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
     // ---- the products of this stage (set up by thread 0 before the barrier that opened the stage) ----
     const int njobs = s_njobs[st];
     const GemmJob* job = jobs + 2 * st;
-    if (st == 0 && warp < MP_CC_W0 && job[0].mine == 0) {
-      // no tile in the first stage: these warps help to pack the weights
-      const int T = min(G, job[0].items);
-      mp_forward_jobs(p, rt, H, cta, G, -1, G * MP_CC_THREADS + (cta - T) * (MP_CC_W0 * 32) + tid,
-                      G * MP_CC_THREADS + (G - T) * (MP_CC_W0 * 32));
+    // no tile in the first stage: the warps of the tile pipeline help to pack the weights
+    const bool helper = st == 0 && warp < MP_CC_W0 && job[0].mine == 0;
+    if (helper) {
+      // (their work is below, with the CUDA-core warps')
     } else if (warp == 0) {
       // ===================== producer =====================
       // Lane s owns ring stage s: it waits for the stage, announces the bytes and issues the two or three boxes
@@ -846,7 +825,6 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
         for (int ti = 0; ti < j.mine && ok; ++ti, ++git) {
           const int t = j.tile[ti];
           // ---- what does not depend on the accumulators is fetched while the products run ----
-          float dO[MP_SMALL_N];
           __syncwarp();
           if (j.type == JT_F) {
             // biases of the tile's neurons behind the (at most) 1024 staged output weights
@@ -858,9 +836,6 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
             if (fused_dz) {
               // the first tile's output weights were staged before the first stage (see below)
               if (ti > 0 || H == 1) stage_out_weights(stg, t, j.nt, lane);
-              const float* sdOe = reinterpret_cast<const float*>(smem + MP_SDO_OFF);
-#pragma unroll
-              for (int o = 0; o < MP_SMALL_N; ++o) dO[o] = sdOe[o * 128 + row];
             }
           } else if (j.type == JT_BD && l > 0) {
             // the bf16 outputs of the layer below, this thread's 64 columns (ReLU adjoint): 8 x 16 bytes at
@@ -993,18 +968,18 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
               if (fused_dz) {
 #pragma unroll
                 for (int e = 0; e < 16; ++e) dz[e] = 0.f;
+                const float* sdOe = reinterpret_cast<const float*>(smem + MP_SDO_OFF) + row;
+#pragma unroll 1
+                for (int o = 0; o < yo.N; ++o) {
+                  const float g = sdOe[o * 128];
+                  const float4* wq = reinterpret_cast<const float4*>(stg + (ch * MP_SMALL_N + o) * 16);
 #pragma unroll
-                for (int o = 0; o < MP_SMALL_N; ++o) {
-                  if (o < yo.N) {
-                    const float4* wq = reinterpret_cast<const float4*>(stg + (ch * MP_SMALL_N + o) * 16);
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                      const float4 w4 = wq[q4];
-                      dz[4 * q4] += dO[o] * w4.x;
-                      dz[4 * q4 + 1] += dO[o] * w4.y;
-                      dz[4 * q4 + 2] += dO[o] * w4.z;
-                      dz[4 * q4 + 3] += dO[o] * w4.w;
-                    }
+                  for (int q4 = 0; q4 < 4; ++q4) {
+                    const float4 w4 = wq[q4];
+                    dz[4 * q4] += g * w4.x;
+                    dz[4 * q4 + 1] += g * w4.y;
+                    dz[4 * q4 + 2] += g * w4.z;
+                    dz[4 * q4 + 3] += g * w4.w;
                   }
                 }
 #pragma unroll
@@ -1065,15 +1040,19 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
     } else {
       // ===================== CUDA-core warps: the rest of the stage, beside the tiles =====================
       const int ct = tid - MP_CC_W0 * 32;
-      if (st == 0) {
-        const int T = min(G, job[0].items);  // CTAs 0 .. T-1 have a tile; the others lend their idle warps
-        mp_forward_jobs(p, rt, H, cta, G, ct, cta * MP_CC_THREADS + ct, G * MP_CC_THREADS + (G - T) * (MP_CC_W0 * 32));
-      }
       if (st >= H) {
         const float* sdO = reinterpret_cast<const float*>(smem + MP_SDO_OFF);
         mp_backward_jobs(p, rt, H, st, sdO, cta, G, ct);
       }
       if (st < H) mp_zero_fill(p, rt, H, st, cta, G, ct);
+    }
+
+    if (st == 0 && (warp >= MP_CC_W0 || helper)) {
+      // kept lists and packed weights: the CUDA-core warps of every CTA and the idle warps of the CTAs without a tile
+      const int T = min(G, job[0].items);  // CTAs 0 .. T-1 have a tile
+      const int gthreads = G * MP_CC_THREADS + (G - T) * (MP_CC_W0 * 32);
+      const int gtid = helper ? G * MP_CC_THREADS + (cta - T) * (MP_CC_W0 * 32) + tid : cta * MP_CC_THREADS + (tid - MP_CC_W0 * 32);
+      mp_forward_jobs(p, rt, H, cta, G, helper ? -1 : tid - MP_CC_W0 * 32, gtid, gthreads);
     }
 
     // ---- grid-wide barrier (none behind the last stage) ----
