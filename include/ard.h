@@ -338,7 +338,16 @@ ard_status ard_sample_pattern_counter(ard_ctx* ctx, ard_pattern* pat, int dist_i
  * gradients are enqueued on two streams owned by the context, forked from `cuda_stream` after the patterns
  * are drawn and joined back into it before the call returns: to the caller (and to a capture) all work of
  * the call is ordered on `cuda_stream`, but the buffers of `layers` must not be touched by other streams
- * while the iteration runs. */
+ * while the iteration runs.
+ * A small stack runs as ONE cooperative kernel instead (a memset of 4 bytes and one launch per iteration;
+ * same results up to the order of fp32 additions, same patterns, same counter, the same bits from launch to
+ * launch): 2 to 4 layers, 1 <= B <= 128, every hidden layer a row pattern with compact_out != 0, N a multiple
+ * of 64 and K, ldw multiples of 8, the last layer at most 16 neurons wide, dense and not sampled, all
+ * pointers 16-byte aligned, ldx and lddx multiples of 8, a distribution of at most 64 periods, and a device
+ * that can hold one block per SM at once.  Anything else, ARD_PATH_CUDA_CORE, or
+ * ard_set_option(ctx, ARD_OPT_MLP_PERSISTENT, 0) takes the call-by-call path above.  In the one-kernel form
+ * Wk holds the packed weights as before, dWk is not used, and the kernel shares the context's grid-barrier
+ * counter and descriptor scratch with the whole-sequence LSTM kernels: one such kernel at a time per context. */
 typedef struct ard_mlp_layer {
   int K, N;          /* fan-in and neurons; K of layer l+1 == N of layer l                                  */
   ard_pattern* pat;  /* row pattern over the N neurons (created with K_dim = K, N_dim = N)                  */
