@@ -60,7 +60,7 @@ constexpr int MP_BAR_OFF = MP_SDO_OFF + 128 * MP_SMALL_N * 4;
 constexpr int MP_NBARS = 2 * MP_STAGES + MP_NI + 1;
 constexpr int MP_CDF_OFF = (MP_BAR_OFF + 8 * MP_NBARS + 15) / 16 * 16;
 constexpr int MP_MISC_OFF = MP_CDF_OFF + 64 * 8;
-constexpr int MP_SMEM = MP_MISC_OFF + 128 + 2 * (MP_MAX_LAYERS - 1) * 2 * 80 + 64 + 1024;   // + slack for the 1024-byte alignment of the ring
+constexpr int MP_SMEM = MP_MISC_OFF + 128 + 2 * (MP_MAX_LAYERS - 1) * 2 * 112 + 64 + 1024;   // + slack for the 1024-byte alignment of the ring
 static_assert(MP_SMEM <= 227 * 1024, "shared memory of the iteration kernel");
 
 enum { JT_F = 0, JT_BD = 1, JT_BW = 2 };
@@ -111,14 +111,14 @@ struct MpParams {
 
 struct LayerRt { int dp, bb, n, npad; };  // period, offset - 1, kept neurons, the latter rounded up to 64
 
-constexpr int MP_MAX_MINE = 24;  // most tiles of one product a CTA can be dealt (checked on the host)
+constexpr int MP_MAX_MINE = 40;  // most tiles of one product a CTA can be dealt (checked on the host)
 struct GemmJob {
   int type, l;
   int items, nkb, nt, ntn;
   int mine;                  // tiles of this CTA
   short tile[MP_MAX_MINE];   // their numbers
 };
-static_assert(sizeof(GemmJob) <= 80, "room per product in shared memory");
+static_assert(sizeof(GemmJob) <= 112, "room per product in shared memory");
 
 __device__ __forceinline__ unsigned int mp_ld_acquire(const unsigned int* p) {
   unsigned int v;

@@ -102,6 +102,9 @@ CASES = [
     ([328, 1024, 512, 256, 10], 64, [(2, 1), (1, 1), (4, 4)], True, True, True, True),   # three hidden layers
     ([328, 1024, 512, 256, 10], 9, [(5, 5), (3, 1), (2, 2)], False, False, True, False),
     ([784, 4096, 1024, 10], 128, [(1, 1), (2, 1)], True, True, True, True),   # 32-wide forward tiles
+    ([64, 64, 2], 1, [(1, 1)], True, True, True, True),                       # the smallest stack, one batch row
+    ([72, 128, 64, 16], 128, [(16, 7), (13, 13)], False, True, True, True),   # a handful of kept neurons per layer
+    ([1024, 4096, 4096, 8], 31, [(3, 3), (2, 2)], True, True, True, False),   # the widest layers the tile lists take
 ]
 
 
