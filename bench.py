@@ -720,6 +720,39 @@ def run_mlp_step(args, wl):
             sys.stderr.write("torch graph baseline skipped: %r\n" % (ex,))
         best_dense = min(v for k, v in detail["ms_per_step"].items() if k.startswith("torch") or k.endswith("dp1"))
         detail["speedup_vs_dense"] = {str(p): best_dense / (ms / steps)}
+        # the paper's sweep over the dropout rate on this network (Sec. 7, Table 1 reports conventional dropout /
+        # ARD): graph replays of the iteration at p = 0.3, 0.5, 0.7 (maximum-entropy K for each rate, rescale 1/(1-p))
+        # against torch's conventional dropout in a graph (whose time does not depend on p) and the own kernels
+        # with nothing dropped
+        sweep = {}
+        for di, rate in enumerate(RATES):
+            ard.ard_set_distribution(ctx, 1 + di, max_entropy_K(rate, n_dp))
+            for d in compact[0][:-1]:
+                d["sample"] = 1
+                d["alpha"] = 1.0 / (1.0 - rate)
+            st_r = (compact[0], ard.mlp_layers(compact[0]))
+
+            def eager_r():
+                ard.ard_mlp_step(ctx, st_r[1], L, B, X, dims[0], dOut, dims[-1], dX, dims[0], 1 + di, inputs.BASE_SEED,
+                                 base, counter)
+
+            sr = torch.cuda.Stream()
+            with torch.cuda.stream(sr):
+                eager_r()
+            torch.cuda.synchronize()
+            gr_r = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr_r):
+                eager_r()
+            t_r = timed(gr_r.replay, max(20, steps), warm)[0] / max(20, steps)
+            sweep[str(rate)] = {"ms_per_step": t_r, "ideal_speedup": 1.0 / (1.0 - rate),
+                                "speedup_vs_own_kernels_dp1": detail["ms_per_step"]["graph_own_kernels_dp1"] / t_r}
+            if "torch_graph_dropout" in detail["ms_per_step"]:
+                sweep[str(rate)]["speedup_vs_torch_graph_dropout"] = detail["ms_per_step"]["torch_graph_dropout"] / t_r
+            sweep[str(rate)]["speedup_vs_torch_eager_dropout"] = detail["ms_per_step"]["torch_eager_dropout"] / t_r
+            del gr_r
+        detail["rate_sweep"] = sweep
+        for d in compact[0][:-1]:
+            d["alpha"] = alpha
         # end to end: the input batch and the loss gradient come from pinned host memory and the network's
         # output goes back every iteration
         for d in compact[0][:-1]:
