@@ -53,6 +53,10 @@ WORKLOADS = {
     # stack of large layers where the second hidden layer multiplies two compact matrices
     "mlp2048_step": dict(config=2, dims=[784, 2048, 2048, 10], B=128, kind="mlp_step", p=0.5, n_dp=16),
     "mlp8192_step": dict(config=5, dims=[8192, 8192, 8192, 1024], B=4096, kind="mlp_step", p=0.5, n_dp=16),
+    # the other hidden sizes of the paper's MLP table (Sec. 7, Table 1: 1024 x 64, 1024 x 1024, 4096 x 4096; batch 128)
+    "mlp1024x64_step": dict(config=2, dims=[784, 1024, 64, 10], B=128, kind="mlp_step", p=0.5, n_dp=16),
+    "mlp1024_step": dict(config=2, dims=[784, 1024, 1024, 10], B=128, kind="mlp_step", p=0.5, n_dp=16),
+    "mlp4096_step": dict(config=2, dims=[784, 4096, 4096, 10], B=128, kind="mlp_step", p=0.5, n_dp=16),
     # a convolution layer as the product of its im2col input matrix with the filters, rows of the input matrix
     # dropped by predicted sensitivity (Sec. 5.1, 5.2.1): 3x3 filters, 256 -> 512 channels, 32768 output positions
     # run_len = 32: the sampled values of the sensitivity prediction are taken in runs of 32 neighbours, a departure
