@@ -820,7 +820,6 @@ __global__ void __launch_bounds__(MP_THREADS, 1) ard_mlp_persistent_kernel(const
         // weight gradient: where the kept fan-in columns go (Eq. 1)
         const int dpi = (j.type == JT_BW && l > 0) ? rt[l - 1].dp : 1, bi = (j.type == JT_BW && l > 0) ? rt[l - 1].bb : 0;
         const int nin = l == 0 ? y.K : rt[l - 1].n;
-        const uint32_t magic = (uint32_t)(0x100000000ull / (unsigned)dpi) + 1u;  // exact x / dpi for x < 2^16
 #pragma unroll 1
         for (int ti = 0; ti < j.mine && ok; ++ti, ++git) {
           const int t = j.tile[ti];
