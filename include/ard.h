@@ -95,9 +95,12 @@ ard_status ard_set_path(ard_ctx* ctx, ard_path path);
  *   ARD_OPT_BAND_ROWS [16]        raster band of the tensor-core tile order, in 128-row tiles (0: one band)
  *   ARD_OPT_MLP_PERSISTENT [1]    ard_mlp_step runs the whole iteration in one cooperative kernel when the stack
  *                                 fits it (see ard_mlp_step); 0: always call by call
+ *   ARD_OPT_LSTM_COMPACT_H [1]    the whole-sequence forward kernel of ard_lstm_forward contracts over the kept
+ *                                 units of h alone when the pattern drops any (0: over all H columns, the dropped
+ *                                 ones being zero); same results up to the order of fp32 additions
  * Errors: ARD_ERR_INVALID_ARG (unknown option, negative value). */
 typedef enum { ARD_OPT_PDL = 0, ARD_OPT_PDL_IN_CAPTURE = 1, ARD_OPT_SIDE_STREAMS = 2, ARD_OPT_CTA_PAIRS = 3,
-               ARD_OPT_BAND_ROWS = 4, ARD_OPT_MLP_PERSISTENT = 5 } ard_option;
+               ARD_OPT_BAND_ROWS = 4, ARD_OPT_MLP_PERSISTENT = 5, ARD_OPT_LSTM_COMPACT_H = 6 } ard_option;
 ard_status ard_set_option(ard_ctx* ctx, ard_option option, int value);
 /* Opt-in for training loops.  The tensor-core backward GEMMs of a row pattern read a compacted copy
  * of a full-width dY (kept columns only) that the library makes in the context workspace.  With

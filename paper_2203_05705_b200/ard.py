@@ -25,7 +25,7 @@ ARD_OUT_COMPACT, ARD_OUT_SCATTER_ZEROFILL = 0, 1
 ARD_FLAG_OUT_F32, ARD_FLAG_ACCUMULATE, ARD_FLAG_RELU = 0x10, 0x20, 0x40
 ARD_PATH_AUTO, ARD_PATH_CUDA_CORE, ARD_PATH_TENSOR_CORE = 0, 1, 2
 (ARD_OPT_PDL, ARD_OPT_PDL_IN_CAPTURE, ARD_OPT_SIDE_STREAMS, ARD_OPT_CTA_PAIRS, ARD_OPT_BAND_ROWS,
- ARD_OPT_MLP_PERSISTENT) = range(6)
+ ARD_OPT_MLP_PERSISTENT, ARD_OPT_LSTM_COMPACT_H) = range(7)
 ARD_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = [

@@ -179,6 +179,8 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
   ctx->lstm_persistent = 1;
   ctx->d_grid_bar = nullptr;
   ctx->d_lstm_partial = nullptr;
+  ctx->d_lstm_hc = nullptr;
+  ctx->lstm_compact_h = 1;
   ctx->pdl_in_capture = 1;
   ctx->mlp_two_streams = 1;
   ctx->mlp_persistent = 1;
@@ -222,7 +224,10 @@ ard_status ard_create(ard_ctx** out, int device, size_t workspace_bytes) {
         cudaMemset(ctx->d_sk_cnt, 0, cnt_bytes) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->d_tm_slots), tm_slots_bytes()) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->d_grid_bar), 256) != cudaSuccess ||
-        cudaMalloc(reinterpret_cast<void**>(&ctx->d_lstm_partial), lstm_bwd_partial_bytes(ctx->sm_count)) != cudaSuccess) {
+        cudaMalloc(reinterpret_cast<void**>(&ctx->d_lstm_partial), lstm_bwd_partial_bytes(ctx->sm_count)) != cudaSuccess ||
+        cudaMalloc(&ctx->d_lstm_hc, lstm_hc_bytes()) != cudaSuccess ||
+        cudaMemset(ctx->d_lstm_hc, 0, lstm_hc_bytes()) != cudaSuccess) {
+      if (ctx->d_lstm_hc) cudaFree(ctx->d_lstm_hc);
       if (ctx->d_lstm_partial) cudaFree(ctx->d_lstm_partial);
       if (ctx->d_grid_bar) cudaFree(ctx->d_grid_bar);
       if (ctx->d_tm_slots) cudaFree(ctx->d_tm_slots);
@@ -250,6 +255,7 @@ ard_status ard_destroy(ard_ctx* ctx) {
   if (ctx->d_sk_cnt) cudaFree(ctx->d_sk_cnt);
   if (ctx->d_grid_bar) cudaFree(ctx->d_grid_bar);
   if (ctx->d_lstm_partial) cudaFree(ctx->d_lstm_partial);
+  if (ctx->d_lstm_hc) cudaFree(ctx->d_lstm_hc);
   if (ctx->d_status) cudaFree(ctx->d_status);
   for (int i = 0; i < ctx->n_ev; ++i) cudaEventDestroy(ctx->ev[i]);
   if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
@@ -273,6 +279,7 @@ ard_status ard_set_option(ard_ctx* ctx, ard_option option, int value) {
     case ARD_OPT_CTA_PAIRS: ctx->use_pairs = value ? 1 : 0; return ARD_OK;
     case ARD_OPT_BAND_ROWS: ctx->band_m = value; return ARD_OK;
     case ARD_OPT_MLP_PERSISTENT: ctx->mlp_persistent = value ? 1 : 0; return ARD_OK;
+    case ARD_OPT_LSTM_COMPACT_H: ctx->lstm_compact_h = value ? 1 : 0; return ARD_OK;
   }
   return ARD_ERR_INVALID_ARG;
 }
@@ -1083,8 +1090,16 @@ static ard_status lstm_forward_impl(ard_ctx* ctx, const ard_pattern* pat, int T,
                       &mapW[gate]);
         if (st != ARD_OK) return st;
       }
-      st = launch_lstm_forward_persistent(ctx, pat, T, B, I, H, I, H, I > 0 ? 1 : 0, alpha, mapXH, mapW, XH, bias, C,
-                                          G, s);
+      // 2b. Under a pattern the recurrence contracts over the kept units of h_{t-1} alone: its operand is a compact
+      // copy of h in context scratch (two buffers, the kernel fills them).
+      TcMap mapHc;
+      const bool compact_h = ctx->lstm_compact_h && pat->dp_bound > 1 && ctx->d_lstm_hc != nullptr && H <= ARD_LSTM_HC_LD;
+      if (compact_h) {
+        st = get_maps(ctx, ctx->d_lstm_hc, 2 * B, ARD_LSTM_HC_LD, ARD_LSTM_HC_LD, 0, MAP_PLAIN, 0, 64, 64, &mapHc);
+        if (st != ARD_OK) return st;
+      }
+      st = launch_lstm_forward_persistent(ctx, pat, T, B, I, H, I, H, I > 0 ? 1 : 0, alpha, mapXH, mapW,
+                                          compact_h ? &mapHc : nullptr, W, ldw, XH, bias, C, G, s);
       if (st != ARD_ERR_UNSUPPORTED) return st;
       // not launchable as one kernel right now: the per-step path below recomputes everything
     }

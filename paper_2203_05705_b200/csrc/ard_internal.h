@@ -87,6 +87,9 @@ constexpr int ARD_TM_SM_MAX = 256;
 constexpr int ARD_TM_SLOTS = 16;
 constexpr int ARD_TM_LSTM_BLOCKS = 512;
 constexpr int ARD_TM_LSTM_SLOTS = 8;
+// Two buffers of 128 batch rows by (8 units per block x ARD_TM_LSTM_BLOCKS) bf16 columns.
+constexpr int ARD_LSTM_HC_LD = 8 * ARD_TM_LSTM_BLOCKS;
+static inline size_t lstm_hc_bytes() { return (size_t)2 * 128 * ARD_LSTM_HC_LD * 2; }
 static inline size_t tm_slots_bytes() {
   return ((size_t)ARD_TM_SM_MAX * ARD_TM_SLOTS + (size_t)ARD_TM_LSTM_BLOCKS * ARD_TM_LSTM_SLOTS) * sizeof(CUtensorMap);
 }
@@ -104,6 +107,8 @@ struct ard_ctx {
   int lstm_persistent; // ard_lstm_forward: one cooperative kernel for the whole sequence when the layer fits
   unsigned int* d_grid_bar;  // arrival counter of that kernel's grid-wide barrier
   float* d_lstm_partial;     // partial sums of the whole-sequence BPTT kernel, lstm_bwd_partial_bytes(sm_count)
+  void* d_lstm_hc;           // compact copies of h_{t-1} and h_t of the whole-sequence forward kernel, lstm_hc_bytes()
+  int lstm_compact_h;        // ... which contracts over the kept units of h alone under a pattern
   int use_pdl;        // launch kernels with programmatic stream serialization (see ard_launch)
   int pdl_in_capture; // ... also while the stream is being captured into a CUDA graph
   int stream_k;       // tensor-core row kernels: share the last, partial wave of tiles along the contraction
@@ -240,6 +245,7 @@ ard_status launch_lstm_backward_persistent(ard_ctx* ctx, const ard_pattern* pat,
 bool lstm_persistent_fits(ard_ctx* ctx, int B, int klen, int H);
 ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H,
                                           int kx0, int klen, int add_zx, float alpha, const TcMap& mapXH, const TcMap mapW[4],
+                                          const TcMap* mapHc, const void* W, int ldw,
                                           void* XH, const float* bias, float* C, float* G, cudaStream_t s);
 
 ard_status launch_gather_cols(ard_ctx* ctx, const int32_t* hdr, const int32_t* idx, const void* src, int ld_src,

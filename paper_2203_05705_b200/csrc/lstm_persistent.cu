@@ -48,10 +48,15 @@ constexpr int LP_PAIRS_MAX = (128 * LP_UNITS + LP_MATH - 1) / LP_MATH;  // (row,
 struct LstmFwdParams {
   TcMap mapXH;    // [(T+1)*B][I+H], boxes of 64 rows x 64 columns (used as encoded)
   TcMap mapW[4];  // per gate: [H rows][I+H], boxes of 8 rows x 64 columns; specialised to the kept rows by the kernel
+  TcMap mapHc;    // [2*B][ldhc]: the compact copies of h_{t-1} and h_t, boxes of 64 rows x 64 columns
   CUtensorMap* tm_slots;  // this launch's descriptor scratch: ARD_TM_LSTM_SLOTS slots per block
   const int32_t* hdr;
   int T, B, I, H;
   int kx0, klen;      // contraction columns [kx0, kx0 + klen) of [x | h] this kernel multiplies
+  const __nv_bfloat16* W;  // the weight itself, [4H][ldw]: its kept recurrent columns are gathered by the kernel
+  int ldw;
+  __nv_bfloat16* Hc;  // two buffers [B][ldhc]: column j = the j-th kept unit (nullptr: no compact recurrence)
+  int ldhc;
   int add_zx;         // the products of the other columns are waiting in G[t] (same layout as the gates)
   float alpha;
   __nv_bfloat16* XH;
@@ -97,7 +102,7 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
   uint8_t* smem = smem_raw + (base - raw_addr);
 
   const int KH = p.I + p.H;
-  const int nkb = (p.klen + LP_BK - 1) / LP_BK;
+  int nkb = (p.klen + LP_BK - 1) / LP_BK;
   // The activation row buffer comes first and the weight slice right after it: a block holds one or two
   // 64-row boxes, the MMA always reads 128 rows, and for a batch of at most 64 rows the upper half of
   // what it reads is the next block (or the start of the weight slice); those accumulator rows are
@@ -116,7 +121,7 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
   uint8_t* misc = smem + (bar_base - base) + 8 * (LP_GROUPS + 6);
   volatile uint32_t* tmem_ptr_smem = reinterpret_cast<volatile uint32_t*>(misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
-  const int gsz = (nkb + LP_GROUPS - 1) / LP_GROUPS;          // blocks per arrival group
+  int gsz = (nkb + LP_GROUPS - 1) / LP_GROUPS;                // blocks per arrival group
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -146,6 +151,39 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
   const int j0 = (int)blockIdx.x * LP_UNITS;                // first kept unit (compact index) of this CTA
   const bool active = (int)blockIdx.x < n_active;
   const int xblocks = p.I > p.kx0 ? (p.I - p.kx0) / LP_BK : 0;  // contraction blocks that hold only x columns
+  // Under a pattern the dropped units of h_{t-1} are exact zeros (Sec. 3.1), so the recurrent contraction runs over
+  // the kept units alone: the operand of a step is the compact copy of h_{t-1} (column j = j-th kept unit) that the
+  // cell update writes beside the full-width one, and the weight slice holds the kept fan-in columns only.  Those
+  // stride the weight's contiguous dimension, which no TMA box can follow, so the CTA gathers its slice itself,
+  // once per sequence, straight into the swizzled layout the MMA reads.
+  const bool compact = dp > 1 && p.Hc != nullptr && p.kx0 == p.I;
+  const int hs = compact ? 1 : 0;  // the compact h_0 is made by the kernel: one more grid-wide hand-over, before step 0
+  if (compact) {
+    nkb = (n_keep + LP_BK - 1) / LP_BK;
+    gsz = (nkb + LP_GROUPS - 1) / LP_GROUPS;
+    if (active) {
+      const int nchunks = nkb * 8;  // 16-byte pieces of a slice row
+      for (int task = threadIdx.x; task < LP_N * nchunks; task += LP_THREADS) {
+        const int r = task / nchunks, ch = task - r * nchunks;
+        const int g = r >> 3, k = r & 7, j = j0 + k;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        if (j < n_keep) {
+          const __nv_bfloat16* src = p.W + ((size_t)g * p.H + bb + (size_t)j * dp) * p.ldw + p.I + bb + (size_t)ch * 8 * dp;
+          uint32_t e[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            e[q] = (ch * 8 + q < n_keep) ? (uint32_t)__ldg(reinterpret_cast<const unsigned short*>(src) + (size_t)q * dp) : 0u;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) w[q] = e[2 * q] | (e[2 * q + 1] << 16);
+        }
+        // 128-byte swizzle: the 16-byte piece c of row k of an 8-row group sits at piece c ^ k
+        uint8_t* dst = smem + (sW - base) + (size_t)(ch >> 3) * LP_W_BLOCK + g * (LP_UNITS * LP_BK * 2) + k * 128 + (((ch & 7) ^ k) << 4);
+        *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      fence_proxy_async_smem();  // generic-proxy stores -> the tensor core's reads
+    }
+    __syncthreads();
+  }
 
   if (active) {
     if (warp == 11) {
@@ -153,28 +191,33 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
       // Loads the weight slice (lane = contraction block), then relays the grid barrier of every step to
       // the warps of this CTA through a shared-memory barrier.
       // The gates' weight descriptors become those of the kept rows (the weight area, still empty, is the work area).
-      CUtensorMap* slots = p.tm_slots + (size_t)blockIdx.x * ARD_TM_LSTM_SLOTS;
-      const CUtensorMap* mapW[4];
-#pragma unroll
-      for (int g = 0; g < 4; ++g)
-        mapW[g] = tensormap_specialise(&p.mapW[g], dp, bb + 1, n_keep, smem + (sW - base) + 128 * g, slots + g, lane);
-      fence_proxy_async_smem();
-      const int kb = lane;
-      if (kb < nkb && dp > 1) {
-#pragma unroll
-        for (int g = 0; g < 4; ++g) tensormap_acquire(mapW[g]);
-      }
-      if (lane == 0) mbar_arrive_expect_tx(wfull_bar, (uint32_t)nkb * LP_W_BLOCK);
-      __syncwarp();
-      if (kb < nkb) {
+      if (compact) {
+        // the slice is in place already (gathered by the whole CTA above)
+        if (lane == 0) mbar_arrive(wfull_bar);
+      } else {
+        CUtensorMap* slots = p.tm_slots + (size_t)blockIdx.x * ARD_TM_LSTM_SLOTS;
+        const CUtensorMap* mapW[4];
 #pragma unroll
         for (int g = 0; g < 4; ++g)
-          tma_load_2d(sW + kb * LP_W_BLOCK + g * (LP_UNITS * LP_BK * 2), mapW[g], wfull_bar, p.kx0 + kb * LP_BK, j0);
+          mapW[g] = tensormap_specialise(&p.mapW[g], dp, bb + 1, n_keep, smem + (sW - base) + 128 * g, slots + g, lane);
+        fence_proxy_async_smem();
+        const int kb = lane;
+        if (kb < nkb && dp > 1) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) tensormap_acquire(mapW[g]);
+        }
+        if (lane == 0) mbar_arrive_expect_tx(wfull_bar, (uint32_t)nkb * LP_W_BLOCK);
+        __syncwarp();
+        if (kb < nkb) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            tma_load_2d(sW + kb * LP_W_BLOCK + g * (LP_UNITS * LP_BK * 2), mapW[g], wfull_bar, p.kx0 + kb * LP_BK, j0);
+        }
       }
       if (lane == 0) {
-        for (int t = 1; t < p.T; ++t) {
-          // h_{t-1} is complete when every CTA with units has arrived t times
-          if (!grid_wait(p.bar, (unsigned)t * (unsigned)n_active, abort_flag, p.status)) break;
+        for (int t = 1 - hs; t < p.T; ++t) {
+          // h_{t-1} is complete when every CTA with units has arrived t times (once more with a compact h_0)
+          if (!grid_wait(p.bar, (unsigned)(t + hs) * (unsigned)n_active, abort_flag, p.status)) break;
           mbar_arrive(hready_bar);
         }
       }
@@ -190,7 +233,7 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
       const int kb0 = g * gsz, kb1 = min(nkb, kb0 + gsz);
       const int kb = kb0 + lane;
       const bool mine = kb < kb1;
-      const CUtensorMap* mapXH = &p.mapXH.tm;  // a kernel parameter, used as encoded
+      const CUtensorMap* mapXH = compact ? &p.mapHc.tm : &p.mapXH.tm;  // kernel parameters, used as encoded
       const uint32_t idesc = make_idesc(LP_N, false, false, 128);
       bool ok = (lane != 0) || mbar_wait(wfull_bar, 0u, abort_flag, p.status);
       for (int t = 0; t < p.T; ++t) {
@@ -201,14 +244,15 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
         if (lane == 0 && kb0 < kb1) mbar_arrive_expect_tx(gfull_bar(g), (uint32_t)(kb1 - kb0) * a_block);
         __syncwarp();
         auto issue = [&]() {
+          // full width: columns of [x_t | h_{t-1}], rows of step t; compact: the buffer that holds h_{t-1}
+          const int x = compact ? kb * LP_BK : p.kx0 + kb * LP_BK, y = compact ? (t & 1) * p.B : t * p.B;
           for (int rb = 0; rb < row_boxes; ++rb)
-            tma_load_2d(sA + kb * a_block + rb * LP_ROW_BOX, mapXH, gfull_bar(g), p.kx0 + kb * LP_BK,
-                        t * p.B + rb * 64);
+            tma_load_2d(sA + kb * a_block + rb * LP_ROW_BOX, mapXH, gfull_bar(g), x, y + rb * 64);
         };
         if (mine && kb < xblocks) issue();  // columns of x do not depend on the recurrence
-        if (t > 0 && kb1 > xblocks) {
+        if (t + hs > 0 && kb1 > xblocks) {
           // the other columns are h_{t-1}
-          if (!mbar_wait(hready_bar, (uint32_t)(t - 1) & 1u, abort_flag, p.status)) ok = false;
+          if (!mbar_wait(hready_bar, (uint32_t)(t - 1 + hs) & 1u, abort_flag, p.status)) ok = false;
           if (!__all_sync(0xffffffffu, ok)) break;
           asm volatile("fence.proxy.async.global;" ::: "memory");  // generic-proxy stores of other CTAs -> TMA reads
         }
@@ -245,6 +289,23 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
         const int q = tid + i * LP_MATH;
         const int row = q >> 3, k = q & 7;
         creg[i] = (q < npairs && k < nvalid) ? p.C[(size_t)row * p.H + j0 + k] : 0.f;
+      }
+      if (compact) {
+        // the compact copy of h_0 (buffer 0): this CTA's units of every row; the last CTA with units also clears
+        // the columns up to the next multiple of 64 in both buffers (they meet the zeros of the weight slice)
+        for (int q = tid; q < npairs; q += LP_MATH) {
+          const int row = q >> 3, k = q & 7;
+          if (k < nvalid) p.Hc[(size_t)row * p.ldhc + j0 + k] = p.XH[(size_t)row * ldxh + p.I + bb + (size_t)(j0 + k) * dp];
+        }
+        if ((int)blockIdx.x == n_active - 1) {
+          const int npad = nkb * LP_BK - n_keep;
+          for (int q = tid; q < 2 * p.B * npad; q += LP_MATH) {
+            const int row = q / npad, c = q - row * npad;
+            p.Hc[(size_t)row * p.ldhc + n_keep + c] = __float2bfloat16_rn(0.f);
+          }
+        }
+        asm volatile("bar.sync 1, 352;" ::: "memory");
+        if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
       }
       bool ok = true;
       for (int t = 0; t < p.T && ok; ++t) {
@@ -315,7 +376,9 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
             gg[i] = tanh_fast(zg);
             go[i] = sigmoid_fast(zo);
             creg[i] = gf[i] * creg[i] + gi[i] * gg[i];
-            p.XH[((size_t)(t + 1) * p.B + row) * ldxh + p.I + u] = __float2bfloat16_rn(p.alpha * go[i] * tanh_fast(creg[i]));
+            const __nv_bfloat16 h = __float2bfloat16_rn(p.alpha * go[i] * tanh_fast(creg[i]));
+            p.XH[((size_t)(t + 1) * p.B + row) * ldxh + p.I + u] = h;
+            if (compact) p.Hc[((size_t)((t + 1) & 1) * p.B + row) * p.ldhc + j0 + k] = h;
           }
         }
         // publish h_t: all stores of the CTA, then one release-add for the CTA
@@ -718,7 +781,7 @@ bool lstm_persistent_fits(ard_ctx* ctx, int B, int klen, int H) {
 
 ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H,
                                           int kx0, int klen, int add_zx, float alpha, const TcMap& mapXH, const TcMap mapW[4],
-                                          void* XH, const float* bias, float* C, float* G, cudaStream_t s) {
+                                          const TcMap* mapHc, const void* W, int ldw, void* XH, const float* bias, float* C, float* G, cudaStream_t s) {
   if ((H + LP_UNITS - 1) / LP_UNITS > ARD_TM_LSTM_BLOCKS) return ARD_ERR_UNSUPPORTED;
   LstmFwdParams p;
   p.mapXH = mapXH;
@@ -727,6 +790,11 @@ ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, 
   p.hdr = pat->d_hdr;
   p.T = T; p.B = B; p.I = I; p.H = H;
   p.kx0 = kx0; p.klen = klen; p.add_zx = add_zx;
+  p.mapHc = mapHc ? *mapHc : mapXH;
+  p.W = reinterpret_cast<const __nv_bfloat16*>(W);
+  p.ldw = ldw;
+  p.Hc = mapHc ? reinterpret_cast<__nv_bfloat16*>(ctx->d_lstm_hc) : nullptr;
+  p.ldhc = ARD_LSTM_HC_LD;
   p.alpha = alpha;
   p.XH = reinterpret_cast<__nv_bfloat16*>(XH);
   p.bias = bias;

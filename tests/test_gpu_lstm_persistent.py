@@ -77,6 +77,46 @@ def test_persistent_forward_matches_the_oracle_and_the_per_step_path(T, B, I, H)
         ctx.close()
 
 
+def test_compact_recurrence_and_full_width_recurrence_agree():
+    """Under a pattern the one-kernel forward contracts over the kept units of h alone (a compact copy of h in
+    context scratch, the weight's kept fan-in columns gathered by the kernel); with the option off it contracts over
+    all H columns, the dropped ones being zero.  Both against the oracle, at kept counts that leave a ragged last
+    block and a ragged last CTA, with a batch of more than one row box, a larger kept set run first (its values stay
+    in the scratch beyond the smaller set's columns) and h_0 non-zero."""
+    T, B, I, H = 5, 97, 64, 520
+    rng = np.random.default_rng(99)
+    W = inputs.bf16_round(rng.uniform(-0.08, 0.08, size=(I + H, 4 * H)).astype(np.float32))
+    X = inputs.bf16_round(rng.standard_normal((T, B, I)).astype(np.float32))
+    bias = rng.uniform(-0.5, 0.5, size=4 * H).astype(np.float32)
+    Wnm = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+    ctx = Ctx(1 << 20)
+    try:
+        pat = ctx.pattern(ard.ARD_ROW, I + H, H)
+        for dp, b in [(2, 1), (7, 3), (3, 3), (13, 13)]:
+            ard.ard_pattern_set(ctx.h, pat, dp, b)
+            m = OP.row_mask(H, dp, b)
+            keep = OP.row_keep(H, dp, b)
+            n = len(keep)
+            h0 = inputs.bf16_round((rng.uniform(-1, 1, size=(B, H)) * m[None, :]).astype(np.float32))
+            c0 = (rng.uniform(-1, 1, size=(B, H)) * m[None, :]).astype(np.float32)
+            fw = OL.fwd(X, W, bias, m, 1.3, h0=h0, c0=c0)
+            out = {}
+            for compact in (1, 0):
+                ard.ard_set_option(ctx.h, ard.ARD_OPT_LSTM_COMPACT_H, compact)
+                Hg, Cg, Gg, launches = _run(ctx, pat, T, B, I, H, Wnm, X, bias, h0, c0, keep, 1.3, 1)
+                assert launches == 2
+                assert OG.rel_fro(host(Hg), fw["Hs"]) <= TOL[ard.ARD_BF16], (compact, dp, b)
+                assert OG.rel_fro(host(Cg[T])[:, :n], fw["cT"][:, keep]) <= TOL[ard.ARD_BF16], (compact, dp, b)
+                assert bool(torch.all(Hg[:, :, torch.from_numpy(m == 0).cuda()] == 0)), (compact, dp, b)
+                out[compact] = (Hg, Cg[1:, :, :n].clone())
+            # the same products in another order of fp32 additions
+            assert float((out[1][0] - out[0][0]).abs().max()) <= 0.02, (dp, b)
+            assert float((out[1][1] - out[0][1]).abs().max()) <= 0.02, (dp, b)
+        ard.ard_set_option(ctx.h, ard.ARD_OPT_LSTM_COMPACT_H, 1)
+    finally:
+        ctx.close()
+
+
 def test_layers_that_do_not_fit_use_the_per_step_path():
     """Batch above 128 rows: the same call enqueues the per-step kernels."""
     T, B, I, H = 2, 130, 64, 64
