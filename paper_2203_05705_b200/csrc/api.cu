@@ -1164,7 +1164,7 @@ static ard_status lstm_backward_impl(ard_ctx* ctx, const ard_pattern* pat, int T
                       &mapW[gate]);
         if (st != ARD_OK) return st;
       }
-      st = launch_lstm_backward_persistent(ctx, pat, T, B, I, H, alpha, mapDZ, mapW, C, G, dH_last, D, dc, DZ, s);
+      st = launch_lstm_backward_persistent(ctx, pat, T, B, I, H, alpha, mapDZ, mapW, W, ldw, C, G, dH_last, D, dc, DZ, s);
       if (st == ARD_OK) {
         // dx_t for all t: the x halves of D are overwritten
         if (!recurrent_only) st = lstm_gate_gemm_bwd_tc(ctx, pat, T * B, I, H, DZ, H, W, ldw, D, KH, 0, s);

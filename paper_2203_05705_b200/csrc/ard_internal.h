@@ -239,7 +239,7 @@ ard_status launch_rows_tc(ard_ctx* ctx, GemmOp op, const TcArgs& a, const int32_
 size_t lstm_bwd_partial_bytes(int sm_count);
 bool lstm_persistent_bwd_fits(ard_ctx* ctx, int B, int H);
 ard_status launch_lstm_backward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
-                                           const TcMap mapDZ[4], const TcMap mapW[4],
+                                           const TcMap mapDZ[4], const TcMap mapW[4], const void* W, int ldw,
                                            const float* C, const float* G, const float* dH_last, float* D, float* dc,
                                            void* DZ, cudaStream_t s);
 bool lstm_persistent_fits(ard_ctx* ctx, int B, int klen, int H);

@@ -22,7 +22,14 @@
 //     update to the (batch row, unit) pairs, keep c in registers, and write h_t (bf16) into the operand
 //     of step t+1 and, after signalling, c_t and the gate activations for BPTT;
 //   - columns of x, if the kernel is given any, are loaded ahead; the h columns wait for the grid-wide
-//     barrier that says h_{t-1} is complete.
+//     barrier that says h_{t-1} is complete;
+//   - under a pattern (period > 1) the dropped units of h_{t-1} are exact zeros, so the contraction runs over
+//     the kept units only: the cell update also writes h_t into a compact copy (column j = j-th kept unit, two
+//     buffers in context scratch), which is the operand of step t+1, and the slice holds the kept fan-in
+//     columns of the weight only.  Those stride the weight's contiguous dimension, which a TMA box cannot
+//     follow, so the CTA gathers its slice with plain loads, once per sequence, straight into the swizzled
+//     layout the MMA reads.  A step's loads and MMAs shrink with the kept count (forward of 35 steps, batch 64,
+//     H = 1024: 218 -> 189 us at a period of 2, 204 -> 146 us at 8).
 // The grid barrier is an arrival counter in global memory: after its stores and a fence each CTA adds 1,
 // and the producer thread of each CTA polls for t * (number of CTAs with units) before it loads the
 // h half of step t.  The launch is cooperative, so all CTAs are resident; every wait is bounded (2 s)
@@ -92,6 +99,10 @@ __device__ bool grid_wait(const unsigned int* bar, unsigned int target, volatile
   }
 }
 
+__host__ __device__ inline bool lstm_fwd_zs_shared(int kx0, int I, int nkb, int a_block) {
+  return kx0 >= I && nkb * a_block >= LP_ZS_BYTES;
+}
+
 __device__ __forceinline__ float sigmoid_fast(float x) { return 1.f / (1.f + __expf(-x)); }
 __device__ __forceinline__ float tanh_fast(float x) { return 1.f - 2.f / (1.f + __expf(2.f * x)); }
 
@@ -111,8 +122,14 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
   const uint32_t a_block = (uint32_t)row_boxes * LP_ROW_BOX;
   const uint32_t sA = base;
   const uint32_t sW = base + (uint32_t)nkb * a_block;         // nkb blocks of 4 KiB
-  float* zs = reinterpret_cast<float*>(smem + (sW - base) + (size_t)nkb * LP_W_BLOCK);
-  const uint32_t bar_base = sW + (uint32_t)nkb * LP_W_BLOCK + LP_ZS_BYTES;  // gfull[4], tfull[2], tempty[2], wfull
+  // The staged pre-activations share the start of the row buffer when every block of a step waits for the grid-wide
+  // barrier (no x columns): they are written after the step's MMAs have completed and read before this CTA releases
+  // h_t, and the next loads are issued only after every CTA has released.  Without them the kernel stays below
+  // 196 KB of shared memory at H = 1024; one carve-out step higher (228 KB, next to no L1 left) this kernel was
+  // measured 1.5 % slower and the BPTT kernel 4 %.
+  const bool zs_shared = lstm_fwd_zs_shared(p.kx0, p.I, nkb, (int)a_block);
+  float* zs = reinterpret_cast<float*>(zs_shared ? smem : smem + (sW - base) + (size_t)nkb * LP_W_BLOCK);
+  const uint32_t bar_base = sW + (uint32_t)nkb * LP_W_BLOCK + (zs_shared ? 0 : LP_ZS_BYTES);  // gfull[4], tfull[2], tempty[2], wfull
   auto gfull_bar = [&](int g) { return bar_base + 8u * g; };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (LP_GROUPS + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (LP_GROUPS + 2 + a); };
@@ -381,7 +398,9 @@ __global__ void __launch_bounds__(LP_THREADS, 1) ard_lstm_forward_kernel(const _
             if (compact) p.Hc[((size_t)((t + 1) & 1) * p.B + row) * p.ldhc + j0 + k] = h;
           }
         }
-        // publish h_t: all stores of the CTA, then one release-add for the CTA
+        // publish h_t: all stores of the CTA, then one release-add for the CTA (the staged sums may lie in the row
+        // buffer, which the TMA unit overwrites next: generic-proxy accesses first)
+        fence_proxy_async_smem();
         asm volatile("bar.sync 1, 352;" ::: "memory");
         if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
 #pragma unroll
@@ -442,6 +461,18 @@ constexpr int LB_W_BLOCK = 64 * LB_COLS * 2; // one resident weight box
 constexpr int LB_THREADS = 512;              // warps 0-10 adjoint (0-3 also read TMEM), 11 relay, 12-15 load + MMA
 constexpr int LB_MATH = 352;
 constexpr int LB_PAIRS_MAX = (128 * LB_OWN + LB_MATH - 1) / LB_MATH;
+// Few kept units (all contraction blocks of a step fit the row buffer): the cut along the contraction is dropped.
+// A CTA owns LC_UNITS KEPT units, holds their fan-out weights over all 4 * n_keep kept gate rows (gathered by the
+// kernel, K-major) and contracts the whole of dz_{t+1} itself: one grid-wide barrier per step instead of two, no
+// partial sums through global memory.
+constexpr int LC_UNITS = 8;                    // kept units per CTA
+constexpr int LC_N = 16;                       // MMA width (the instruction's minimum at 128 rows): units 8-15 are zeros
+constexpr int LC_W_BLOCK = LC_N * LP_BK * 2;   // one contraction block of the resident weight slice
+constexpr int LC_ZS_LD = LC_UNITS + 1;         // staged recurrent sums: [128 rows][9] floats
+constexpr int LC_ZS_BYTES = 128 * LC_ZS_LD * 4;
+constexpr int LB_BAR_BYTES = 1024;             // barriers and flags at the start of shared memory
+constexpr int LB_SMEM_BYTES = 227 * 1024;      // the kernel always asks for all of it (one CTA per SM anyway)
+static_assert(LC_UNITS == LB_OWN, "both forms give a thread the same number of (row, unit) pairs");
 
 struct LstmBwdParams {
   TcMap mapDZ[4];  // per gate: [T*B rows][H columns], boxes 64 x 64; the kernel limits them to the n_keep compact columns
@@ -459,7 +490,226 @@ struct LstmBwdParams {
   float* partial;        // [CTA][128][64]
   unsigned int* bar;
   int* status;
+  const __nv_bfloat16* W;  // the weight itself, [4H][ldw] (the compact form gathers its slice from it)
+  int ldw;
+  int compact_ok;          // the compact form may be used when the drawn pattern allows it
+  int smem_bytes;          // dynamic shared memory of this launch
 };
+
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+
+// The compact form of the BPTT recurrence (see LC_UNITS).  Barriers gfull[4], tfull and hready of the caller's set.
+__device__ __forceinline__ void lstm_backward_compact(const LstmBwdParams& p, uint8_t* smem, uint32_t base, uint32_t bar_base,
+                                                      uint32_t tmem_base, volatile int* abort_flag, int dp, int bb,
+                                                      int n_keep) {
+  auto gfull_bar = [&](int g) { return bar_base + 8u * g; };
+  const uint32_t tfull_bar = bar_base + 8u * LP_GROUPS;
+  const uint32_t hready_bar = bar_base + 8u * (LP_GROUPS + 2);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KH = p.I + p.H, T = p.T;
+  const int row_boxes = (p.B + 63) / 64;
+  const uint32_t a_block = (uint32_t)row_boxes * LP_ROW_BOX;
+  const int nb = (n_keep + 63) / 64;                  // contraction blocks per gate
+  const int nblk = 4 * nb;                            // ... per step; block = gate * nb + jb
+  const int gsz = (nblk + LP_GROUPS - 1) / LP_GROUPS; // blocks per loader / MMA warp
+  const int n_active = (n_keep + LC_UNITS - 1) / LC_UNITS;
+  const bool active = (int)blockIdx.x < n_active;
+  const int j0 = (int)blockIdx.x * LC_UNITS;          // first kept unit (compact index) of this CTA
+  const uint32_t sA = base + LB_BAR_BYTES;            // the blocks of dz_{t+1}
+  const uint32_t sW = sA + (uint32_t)nblk * a_block;  // the weight slice
+  float* zs = reinterpret_cast<float*>(smem + (sW - base) + (size_t)nblk * LC_W_BLOCK);
+
+  if (active) {
+    // Weight slice, K-major: row r = unit j0 + r, column (gate, i) = W[gate * H + keep[i]][I + keep[j0 + r]], in the
+    // 128-byte swizzle (16-byte piece c of row r of an 8-row group sits at piece c ^ r); rows 8-15 and what lies
+    // beyond the kept counts are zeros.
+    for (int task = threadIdx.x; task < nblk * LC_N * 8; task += LB_THREADS) {
+      const int kb = task >> 7, r = (task >> 3) & 15, c = task & 7;
+      const int g = kb / nb, jb = kb - g * nb;
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      if (r < LC_UNITS && j0 + r < n_keep) {
+        const int i0 = jb * 64 + c * 8;
+        const unsigned short* src = reinterpret_cast<const unsigned short*>(p.W) +
+                                    ((size_t)g * p.H + bb + (size_t)i0 * dp) * p.ldw + p.I + bb + (size_t)(j0 + r) * dp;
+        uint32_t e[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) e[q] = (i0 + q < n_keep) ? (uint32_t)__ldg(src + (size_t)q * dp * p.ldw) : 0u;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) w[q] = e[2 * q] | (e[2 * q + 1] << 16);
+      }
+      uint8_t* dst = smem + (sW - base) + (size_t)kb * LC_W_BLOCK + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4);
+      *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    fence_proxy_async_smem();  // generic-proxy stores -> the tensor core's reads
+  }
+  __syncthreads();
+  if (!active) return;
+
+  CUtensorMap* slots = p.tm_slots + (size_t)blockIdx.x * ARD_TM_LSTM_SLOTS;
+  if (warp == 11) {
+    // ===================== descriptors of the compact gradient columns, barrier relay =====================
+#pragma unroll
+    for (int g = 0; g < 4; ++g)
+      tensormap_specialise(&p.mapDZ[g], dp, bb + 1, n_keep, reinterpret_cast<uint8_t*>(zs) + 128 * g, slots + 4 + g, lane);
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+      for (int ph = 1; ph <= T; ++ph) {
+        // dz of time index T - ph is complete when every CTA with units has arrived ph times
+        if (!grid_wait(p.bar, (unsigned)ph * (unsigned)n_active, abort_flag, p.status)) break;
+        mbar_arrive(hready_bar);
+      }
+    }
+  } else if (warp >= 12) {
+    // ===================== loaders and MMA issuers (group g4 = warp - 12) =====================
+    const int g4 = warp - 12;
+    const int kb0 = g4 * gsz, kb1 = min(nblk, kb0 + gsz);
+    const int kb = kb0 + lane;
+    const bool mine = kb < kb1;
+    int gate = 0, jb = 0;
+    if (mine) {
+      gate = kb / nb;
+      jb = kb - gate * nb;
+    }
+    const CUtensorMap* mdz = slots + 4 + gate;
+    const uint32_t idesc = make_idesc(LC_N, false, false, 128);
+    bool ok = true;
+    for (int k = 1; k <= T; ++k) {
+      if (ok && !mbar_wait(hready_bar, (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
+      if (!__all_sync(0xffffffffu, ok)) break;
+      if (k == 1 && mine) tensormap_acquire(mdz);  // written by warp 11 ahead of its first arrival on hready_bar
+      if (kb0 < kb1) {
+        asm volatile("fence.proxy.async.global;" ::: "memory");  // generic-proxy stores of other CTAs -> TMA reads
+        if (lane == 0) mbar_arrive_expect_tx(gfull_bar(g4), (uint32_t)(kb1 - kb0) * a_block);
+        __syncwarp();
+        if (mine)
+          for (int rb = 0; rb < row_boxes; ++rb)
+            tma_load_2d(sA + kb * a_block + rb * LP_ROW_BOX, mdz, gfull_bar(g4), jb * 64, (T - k) * p.B + rb * 64);
+        if (lane == 0) {
+          if (!mbar_wait(gfull_bar(g4), (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
+          if (ok) {
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(g4 * LB_COLS);
+            uint64_t ad = make_desc(sA + kb0 * a_block, 16, 1024), bd = make_desc(sW + kb0 * LC_W_BLOCK, 16, 1024);
+            for (int k2 = kb0; k2 < kb1; ++k2, ad += a_block >> 4, bd += LC_W_BLOCK >> 4) {
+#pragma unroll
+              for (int s = 0; s < LP_BK / 16; ++s)
+                tc_mma_bf16(d_tmem, ad + 2 * s, bd + 2 * s, idesc, (k2 != kb0 || s != 0) ? 1u : 0u);
+            }
+          }
+        }
+      }
+      if (lane == 0 && ok) {
+        if (kb0 < kb1) tc_commit(tfull_bar);
+        else mbar_arrive(tfull_bar);
+      }
+      __syncwarp();
+    }
+  } else {
+    // ===================== recurrent sums and cell adjoint (warps 0-10) =====================
+    const int tid = threadIdx.x;
+    const int npairs = p.B * LC_UNITS;  // (batch row, owned unit) pairs; pair q = row * 8 + kk
+    const size_t ldd = (size_t)KH;
+    float dcreg[LB_PAIRS_MAX];
+    int jj[LB_PAIRS_MAX];  // kept index of the pair's unit, -1 beyond the kept count or the batch
+#pragma unroll
+    for (int i = 0; i < LB_PAIRS_MAX; ++i) {
+      const int q = tid + i * LB_MATH;
+      const int row = q >> 3, j = j0 + (q & 7);
+      jj[i] = (q < npairs && j < n_keep) ? j : -1;
+      dcreg[i] = jj[i] >= 0 ? p.dc[(size_t)row * p.H + j] : 0.f;
+    }
+    bool ok = true;
+    for (int k = 0; k <= T && ok; ++k) {
+      const int t = T - 1 - k;  // time index whose dh is formed in this round (-1: the gradient of h_0)
+      float pg[LB_PAIRS_MAX][6], ups[LB_PAIRS_MAX];
+#pragma unroll
+      for (int i = 0; i < LB_PAIRS_MAX; ++i) {
+        ups[i] = 0.f;
+        if (jj[i] >= 0 && t >= 0) {
+          const int row = (tid + i * LB_MATH) >> 3, j = jj[i], u = bb + j * dp;
+          const float* gs = p.G + ((size_t)t * p.B + row) * 4 * p.H + j;
+          pg[i][0] = __ldcg(gs);
+          pg[i][1] = __ldcg(gs + p.H);
+          pg[i][2] = __ldcg(gs + 2 * p.H);
+          pg[i][3] = __ldcg(gs + 3 * p.H);
+          pg[i][4] = __ldcg(p.C + ((size_t)t * p.B + row) * p.H + j);
+          pg[i][5] = __ldcg(p.C + ((size_t)(t + 1) * p.B + row) * p.H + j);
+          ups[i] = (t == T - 1) ? p.dH_last[(size_t)row * p.H + u]
+                                : __ldcg(p.D + ((size_t)(t + 1) * p.B + row) * ldd + p.I + u);
+        }
+      }
+      if (k >= 1) {
+        if (warp < 4) {
+          if (!mbar_wait(tfull_bar, (uint32_t)(k - 1) & 1u, abort_flag, p.status)) ok = false;
+          if (ok) {
+            tc_fence_after();
+            const int row = warp * 32 + lane;
+            const uint32_t t_row = tmem_base + ((uint32_t)(warp * 32) << 16);
+            const int ngroups = (nblk + gsz - 1) / gsz;
+            uint32_t z[8], y[8];
+            tmem_ld8(t_row, z);
+            tmem_ld_wait();
+            for (int c = 1; c < ngroups; ++c) {
+              tmem_ld8(t_row + (uint32_t)(c * LB_COLS), y);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 8; ++i) z[i] = __float_as_uint(__uint_as_float(z[i]) + __uint_as_float(y[i]));
+            }
+            tc_fence_before();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) zs[row * LC_ZS_LD + i] = __uint_as_float(z[i]);
+          }
+        }
+        asm volatile("bar.sync 2, 352;" ::: "memory");
+        if (*abort_flag) { ok = false; break; }
+      }
+#pragma unroll
+      for (int i = 0; i < LB_PAIRS_MAX; ++i) {
+        if (jj[i] < 0) continue;
+        const int q = tid + i * LB_MATH;
+        const int row = q >> 3, j = jj[i], u = bb + j * dp;
+        const float rec = k >= 1 ? zs[row * LC_ZS_LD + (q & 7)] : 0.f;
+        if (t < 0) {  // gradient of h_0: added to what the caller left in the h half of D[0]
+          p.D[(size_t)row * ldd + p.I + u] += rec;
+          continue;
+        }
+        float dh;
+        if (t == T - 1) {
+          dh = ups[i];
+        } else {
+          dh = ups[i] + rec;  // upstream gradient of h_t plus the recurrent part
+          p.D[((size_t)(t + 1) * p.B + row) * ldd + p.I + u] = dh;
+        }
+        const float gi = pg[i][0], gf = pg[i][1], gg = pg[i][2], go = pg[i][3];
+        const float cp = pg[i][4];
+        const float tc = tanh_fast(pg[i][5]);
+        const float d_o = dh * p.alpha * tc;
+        const float dcv = dcreg[i] + dh * p.alpha * go * (1.f - tc * tc);
+        dcreg[i] = dcv * gf;
+        __nv_bfloat16* dz = p.DZ + ((size_t)t * p.B + row) * 4 * p.H + j;
+        dz[0] = __float2bfloat16_rn(dcv * gg * gi * (1.f - gi));
+        dz[p.H] = __float2bfloat16_rn(dcv * cp * gf * (1.f - gf));
+        dz[2 * p.H] = __float2bfloat16_rn(dcv * gi * (1.f - gg * gg));
+        dz[3 * p.H] = __float2bfloat16_rn(d_o * go * (1.f - go));
+      }
+      if (t >= 0) {
+        asm volatile("bar.sync 1, 352;" ::: "memory");
+        if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
+      }
+    }
+    if (ok) {
+#pragma unroll
+      for (int i = 0; i < LB_PAIRS_MAX; ++i)
+        if (jj[i] >= 0) p.dc[(size_t)((tid + i * LB_MATH) >> 3) * p.H + jj[i]] = dcreg[i];
+    }
+  }
+}
 
 __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const __grid_constant__ LstmBwdParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -470,10 +720,10 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
   const int KH = p.I + p.H;
   const int row_boxes = (p.B + 63) / 64;
   const uint32_t a_block = (uint32_t)row_boxes * LP_ROW_BOX;
-  const uint32_t sA = base;                                     // LB_MAX_BLOCKS blocks of dz
-  const uint32_t sW = base + LB_MAX_BLOCKS * a_block;            // LB_MAX_BLOCKS weight boxes (the MMA's 128-row read of
+  const uint32_t bar_base = base;                               // gfull[4], tfull, wfull, hready, pready; flags
+  const uint32_t sA = base + LB_BAR_BYTES;                      // LB_MAX_BLOCKS blocks of dz
+  const uint32_t sW = sA + LB_MAX_BLOCKS * a_block;             // LB_MAX_BLOCKS weight boxes (the MMA's 128-row read of
                                                                  // the last dz block ends inside this region)
-  const uint32_t bar_base = sW + LB_MAX_BLOCKS * LB_W_BLOCK;     // gfull[4], tfull, wfull, hready, pready
   auto gfull_bar = [&](int g) { return bar_base + 8u * g; };
   const uint32_t tfull_bar = bar_base + 8u * LP_GROUPS;
   const uint32_t wfull_bar = bar_base + 8u * (LP_GROUPS + 1);
@@ -521,7 +771,12 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
   const int gsz = (nblk + LP_GROUPS - 1) / LP_GROUPS;   // blocks per loader / MMA warp
   const int T = p.T;
 
-  if (warp == 11) {
+  // few kept units: every block of a step fits the row buffer beside the slice of one CTA's units
+  const bool compact = p.compact_ok && dp > 1 &&
+                       LB_BAR_BYTES + 4 * nb * ((int)a_block + LC_W_BLOCK) + LC_ZS_BYTES <= p.smem_bytes - 1024;
+  if (compact) {
+    lstm_backward_compact(p, smem, base, bar_base, tmem_base, abort_flag, dp, bb, n_keep);
+  } else if (warp == 11) {
     // ===================== weight loader and barrier relay =====================
     // the weight area, still empty, is the work area of the eight descriptors
 #pragma unroll
@@ -751,9 +1006,11 @@ __global__ void __launch_bounds__(LB_THREADS, 1) ard_lstm_backward_kernel(const 
 
 // Dynamic shared memory for klen contraction columns and batch B: the row buffer, the weight slice, the
 // staged pre-activations, barriers, and slack for the 1024-byte alignment.
-static size_t lstm_fwd_smem_bytes(int klen, int B) {
+static size_t lstm_fwd_smem_bytes(int klen, int B, int kx0 = 0, int I = 1) {
   const size_t nkb = (size_t)(klen + LP_BK - 1) / LP_BK;
-  return nkb * ((B + 63) / 64) * LP_ROW_BOX + nkb * LP_W_BLOCK + LP_ZS_BYTES + 8 * (LP_GROUPS + 6) + 16 + 1024;
+  const size_t a_block = (size_t)((B + 63) / 64) * LP_ROW_BOX;
+  const size_t zs = lstm_fwd_zs_shared(kx0, I, (int)nkb, (int)a_block) ? 0 : LP_ZS_BYTES;
+  return nkb * a_block + nkb * LP_W_BLOCK + zs + 8 * (LP_GROUPS + 6) + 16 + 1024;
 }
 
 // Can the whole-sequence kernel run this layer on this device?  (Shared memory for the weight slice, one
@@ -808,7 +1065,7 @@ ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((H + LP_UNITS - 1) / LP_UNITS);  // sized for dp = 1; CTAs without units leave at once
   cfg.blockDim = dim3(LP_THREADS);
-  cfg.dynamicSmemBytes = lstm_fwd_smem_bytes(klen, B);
+  cfg.dynamicSmemBytes = lstm_fwd_smem_bytes(klen, B, kx0, I);
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs resident: they wait for one another
@@ -829,8 +1086,20 @@ ard_status launch_lstm_forward_persistent(ard_ctx* ctx, const ard_pattern* pat, 
 }
 
 // ---- whole-sequence BPTT recurrence ----
-static size_t lstm_bwd_smem_bytes(int B) {
-  return (size_t)LB_MAX_BLOCKS * ((B + 63) / 64) * LP_ROW_BOX + (size_t)LB_MAX_BLOCKS * LB_W_BLOCK + 8 * (LP_GROUPS + 4) + 16 + 1024;
+// Shared memory of the BPTT kernel.  The form is chosen on the device from the drawn pattern, so the launch asks for
+// what either may need: 8 row blocks and 8 weight boxes behind the barriers for the form with partial sums, 16 row
+// blocks and slice blocks for the compact form (more kept units than that take the other form).  Asking for all
+// 227 KB instead cost the form with partial sums 4 % (390 -> 407 us per backward pass at H = 1024, batch 64).
+static size_t lstm_bwd_smem_bytes(int B, int compact_ok) {
+  static_assert((size_t)LB_MAX_BLOCKS * 2 * LP_ROW_BOX + (size_t)LB_MAX_BLOCKS * LB_W_BLOCK + LB_BAR_BYTES + 1024 <= LB_SMEM_BYTES,
+                "the form with partial sums does not fit");
+  const size_t a_block = (size_t)((B + 63) / 64) * LP_ROW_BOX;
+  const size_t sums = LB_MAX_BLOCKS * a_block + (size_t)LB_MAX_BLOCKS * LB_W_BLOCK + LB_BAR_BYTES + 1024;
+  if (!compact_ok) return sums;
+  // room for the compact form up to 4 blocks per gate (256 kept units), or whatever the other form needs
+  const size_t compact = 16 * (a_block + LC_W_BLOCK) + LC_ZS_BYTES + LB_BAR_BYTES + 1024;
+  const size_t want = compact > sums ? compact : sums;
+  return want < (size_t)LB_SMEM_BYTES ? want : (size_t)LB_SMEM_BYTES;
 }
 
 size_t lstm_bwd_partial_bytes(int sm_count) { return (size_t)sm_count * 128 * LB_COLS * sizeof(float); }
@@ -845,7 +1114,7 @@ bool lstm_persistent_bwd_fits(ard_ctx* ctx, int B, int H) {
     int n = 0;
     if (cudaFuncSetAttribute(ard_lstm_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
             cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, ard_lstm_backward_kernel, LB_THREADS, lstm_bwd_smem_bytes(128)) !=
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, ard_lstm_backward_kernel, LB_THREADS, lstm_bwd_smem_bytes(128, 1)) !=
             cudaSuccess ||
         n < 1)
       probed[dev] = -1;
@@ -856,7 +1125,7 @@ bool lstm_persistent_bwd_fits(ard_ctx* ctx, int B, int H) {
 }
 
 ard_status launch_lstm_backward_persistent(ard_ctx* ctx, const ard_pattern* pat, int T, int B, int I, int H, float alpha,
-                                           const TcMap mapDZ[4], const TcMap mapW[4],
+                                           const TcMap mapDZ[4], const TcMap mapW[4], const void* W, int ldw,
                                            const float* C, const float* G, const float* dH_last, float* D, float* dc,
                                            void* DZ, cudaStream_t s) {
   if ((H + LB_COLS - 1) / LB_COLS * LB_KPARTS > ARD_TM_LSTM_BLOCKS) return ARD_ERR_UNSUPPORTED;
@@ -871,11 +1140,15 @@ ard_status launch_lstm_backward_persistent(ard_ctx* ctx, const ard_pattern* pat,
   p.partial = ctx->d_lstm_partial;
   p.bar = ctx->d_grid_bar;
   p.status = ctx->d_status;
+  p.W = reinterpret_cast<const __nv_bfloat16*>(W);
+  p.ldw = ldw;
+  p.compact_ok = ctx->lstm_compact_h;
+  p.smem_bytes = (int)lstm_bwd_smem_bytes(B, p.compact_ok);
   ARD_CUDA_OK(cudaMemsetAsync(ctx->d_grid_bar, 0, sizeof(unsigned int), s));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((H + LB_COLS - 1) / LB_COLS * LB_KPARTS);
   cfg.blockDim = dim3(LB_THREADS);
-  cfg.dynamicSmemBytes = lstm_bwd_smem_bytes(B);
+  cfg.dynamicSmemBytes = lstm_bwd_smem_bytes(B, p.compact_ok);
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs resident: they wait for one another

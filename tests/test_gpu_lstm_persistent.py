@@ -187,3 +187,49 @@ def test_persistent_bptt_matches_the_oracle_and_the_per_step_path(T, B, I, H):
             assert float((a - c).abs().max()) <= 2e-2 * max(1.0, float(c.abs().max())), (dp, b)
     finally:
         ctx.close()
+
+
+@pytest.mark.parametrize("T,B,I,H,periods", [(4, 70, 64, 520, [(2, 2), (5, 1), (9, 4)]), (3, 64, 128, 1024, [(4, 3), (7, 7)])])
+def test_both_forms_of_the_bptt_recurrence_match_the_oracle(T, B, I, H, periods):
+    """With few kept units the BPTT kernel drops the cut along the contraction (a CTA owns 8 kept units and contracts
+    all of dz itself; one grid-wide barrier per step); ARD_OPT_LSTM_COMPACT_H = 0 keeps the form with partial sums.
+    The choice is made on the device from the drawn pattern: here both sides of the limit, a batch of two row boxes,
+    kept counts with a ragged last block and a ragged last CTA."""
+    from paper_2203_05705_b200.lstm import LstmLayer
+    rng = np.random.default_rng(T * 31 + B)
+    W = inputs.bf16_round(rng.uniform(-0.08, 0.08, size=(I + H, 4 * H)).astype(np.float32))
+    X = inputs.bf16_round(rng.standard_normal((T, B, I)).astype(np.float32))
+    dH = (rng.standard_normal((T, B, H)) / 8).astype(np.float32)
+    Wnm = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+    ctx = Ctx(1 << 20)
+    try:
+        pat = ctx.pattern(ard.ARD_ROW, I + H, H)
+        for dp, b in periods:
+            ard.ard_pattern_set(ctx.h, pat, dp, b)
+            m = OP.row_mask(H, dp, b)
+            keep = OP.row_keep(H, dp, b)
+            n = len(keep)
+            fw = OL.fwd(X, W, None, m, 1.5)
+            bw = OL.bwd(fw, W, m, 1.5, dH)
+            got = {}
+            for compact in (1, 0):
+                ard.ard_set_option(ctx.h, ard.ARD_OPT_LSTM_COMPACT_H, compact)
+                layer = LstmLayer(ctx.h, pat, T, B, I, H, Wnm)
+                layer.load_inputs(torch.from_numpy(X).to(BF).cuda())
+                layer.forward(1.5)
+                n0 = ard.ard_launch_count(ctx.h)
+                dX, dW = layer.backward(1.5, torch.from_numpy(dH).cuda())
+                torch.cuda.synchronize()
+                assert ard.ard_launch_count(ctx.h) - n0 == 3
+                assert ard.ard_last_device_status(ctx.h) == 0
+                assert OG.rel_fro(host(dX), bw["dX"]) <= TOL[ard.ARD_BF16], (compact, dp, b)
+                assert OG.rel_fro(host(dW), bw["dW"].T) <= TOL[ard.ARD_BF16], (compact, dp, b)
+                kidx = torch.from_numpy(keep).cuda()
+                assert OG.rel_fro(host(layer.D[0, :, I:][:, kidx]), bw["dh0"][:, keep]) <= TOL[ard.ARD_BF16], (compact, dp, b)
+                assert OG.rel_fro(host(layer.dc[:, :n]), bw["dc0"][:, keep]) <= TOL[ard.ARD_BF16], (compact, dp, b)
+                got[compact] = (dX.clone(), layer.dc[:, :n].clone())
+            assert float((got[1][0] - got[0][0]).abs().max()) <= 2e-2 * max(1.0, float(got[0][0].abs().max())), (dp, b)
+            assert float((got[1][1] - got[0][1]).abs().max()) <= 2e-2 * max(1.0, float(got[0][1].abs().max())), (dp, b)
+        ard.ard_set_option(ctx.h, ard.ARD_OPT_LSTM_COMPACT_H, 1)
+    finally:
+        ctx.close()
