@@ -271,22 +271,25 @@ def run_lstm(args, wl):
     X, dH = hX.cuda(), hdH.cuda()
     hH = torch.empty((T, B, H), dtype=bf).pin_memory()
     ctx = ard.ard_create(0, 2 * T * B * 4 * H + 4096)
+    apply_options(ctx, args)
     ard.ard_set_distribution(ctx, 0, max_entropy_K(p, n_dp))
     pat = ard.ard_pattern_create(ctx, ard.ARD_ROW, I + H, H, 0)
     layer = LstmLayer(ctx, pat, T, B, I, H, W)
     alpha = 1.0 / (1.0 - p)
 
-    def seq(it, dense=False, host=False):
+    def seq(it, dense=False, host=False, dist=0, scale=None, forced=None):
         if dense:
             ard.ard_pattern_set(ctx, pat, 1, 1)
+        elif forced is not None:
+            ard.ard_pattern_set(ctx, pat, forced, 1)
         else:
-            ard.ard_sample_pattern(ctx, pat, 0, inputs.BASE_SEED, it, 4)
+            ard.ard_sample_pattern(ctx, pat, dist, inputs.BASE_SEED, it, 4)
         if host:
             X.copy_(hX, non_blocking=True)
             dH.copy_(hdH, non_blocking=True)
         layer.load_inputs(X)
-        Hs = layer.forward(alpha)
-        layer.backward(alpha, dH)
+        Hs = layer.forward(alpha if scale is None else scale)
+        layer.backward(alpha if scale is None else scale, dH)
         if host:
             hH.copy_(Hs, non_blocking=True)
 
@@ -323,6 +326,17 @@ def run_lstm(args, wl):
     for i in range(ne):
         ard.ard_sample_pattern(ctx, pat, 0, inputs.BASE_SEED, 200000 + args.warmup + i, 4)
         nks_e.append(ard.ard_pattern_to_host(pat, 0)[2])
+    # the other rates of the paper's LSTM experiment (Sec. 7), each with its own distribution over the periods, and
+    # the sequence at a fixed period
+    nsw = max(5, steps // 4)
+    sweep, per_dp = {}, {}
+    for di, rate in enumerate(() if args.quick else RATES):
+        ard.ard_set_distribution(ctx, 1 + di, max_entropy_K(rate, n_dp))
+        ms_r, _, _ = timed(nsw, 300000 + 1000 * di, dist=1 + di, scale=1.0 / (1.0 - rate))
+        sweep["%.1f" % rate] = {"ms_per_step": ms_r / nsw}
+    for dpf in () if args.quick else (1, 2, 3, 4, 6, 8, 12, 16):
+        ms_f, _, _ = timed(nsw, 0, forced=dpf)
+        per_dp[str(dpf)] = {"ms_per_step": ms_f / nsw}
     # dense library baseline for context: the same layer without dropout in torch.nn.LSTM (cuDNN), bf16
     ms_lib = None
     try:
@@ -368,6 +382,13 @@ def run_lstm(args, wl):
             threads = os.cpu_count() or 1
         cpu = {"value": per_unit * (H // 2) / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": "one full sequence, dp=2", "seconds": dt}
+    ms_own_dense = ms_dense / max(5, steps // 4)
+    for v in list(sweep.values()) + list(per_dp.values()):
+        v["speedup_vs_own_kernels_dp1"] = ms_own_dense / v["ms_per_step"]
+        if ms_lib:
+            v["speedup_vs_torch_nn_lstm"] = ms_lib / v["ms_per_step"]
+    for k, v in sweep.items():
+        v["ideal_speedup"] = 1.0 / (1.0 - float(k))
     line = {
         "metric": "LSTM layer fwd+BPTT kept TFLOP/s (row pattern on hidden units, p=0.5)", "value": value,
         "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": args.warmup, "ms_per_step": ms / steps,
@@ -385,7 +406,8 @@ def run_lstm(args, wl):
         "cpu_baseline": cpu,
         "detail": {"dense_ms_per_step": {"own_kernels_dp1": ms_dense / max(5, steps // 4), "torch_nn_lstm": ms_lib},
                    "speedup_vs_dense": {str(p): min(ms_dense / max(5, steps // 4), ms_lib or 1e30) / (ms / steps)},
-                   "kept_fraction": {str(p): float(np.mean(nks)) / H}},
+                   "kept_fraction": {str(p): float(np.mean(nks)) / H},
+                   "rate_sweep": sweep, "per_dp": per_dp},
         "device_status": int(status),
     }
     print(json.dumps(line))

@@ -95,9 +95,12 @@ ard_status ard_set_path(ard_ctx* ctx, ard_path path);
  *   ARD_OPT_BAND_ROWS [16]        raster band of the tensor-core tile order, in 128-row tiles (0: one band)
  *   ARD_OPT_MLP_PERSISTENT [1]    ard_mlp_step runs the whole iteration in one cooperative kernel when the stack
  *                                 fits it (see ard_mlp_step); 0: always call by call
- *   ARD_OPT_LSTM_COMPACT_H [1]    the whole-sequence forward kernel of ard_lstm_forward contracts over the kept
- *                                 units of h alone when the pattern drops any (0: over all H columns, the dropped
- *                                 ones being zero); same results up to the order of fp32 additions
+ *   ARD_OPT_LSTM_COMPACT_H [1]    the whole-sequence kernels of ard_lstm_forward / ard_lstm_backward contract over
+ *                                 the kept units alone when the pattern drops any: forward over a compact copy of
+ *                                 h_{t-1} in context scratch, BPTT (at most 256 kept units) with every block of
+ *                                 dz_{t+1} in one CTA and one grid-wide barrier per step (0: forward over all H
+ *                                 columns, the dropped ones being zero, BPTT always cut along the contraction
+ *                                 with partial sums); same results up to the order of fp32 additions
  * Errors: ARD_ERR_INVALID_ARG (unknown option, negative value). */
 typedef enum { ARD_OPT_PDL = 0, ARD_OPT_PDL_IN_CAPTURE = 1, ARD_OPT_SIDE_STREAMS = 2, ARD_OPT_CTA_PAIRS = 3,
                ARD_OPT_BAND_ROWS = 4, ARD_OPT_MLP_PERSISTENT = 5, ARD_OPT_LSTM_COMPACT_H = 6 } ard_option;
@@ -594,7 +597,8 @@ ard_status ard_lstm_forward(ard_ctx* ctx, const ard_pattern* pat, int T, int B, 
  * When the layer fits (B <= 128, H <= 1024, 8*ceil(H/64) <= number of SMs, operands aligned) and
  * ard_set_lstm_persistent is on, the recurrence dh_{t-1} = upstream + dz_t W_h with the cell adjoint is ONE
  * cooperative kernel (weight slices resident in shared memory, dc in registers, two bounded grid-wide
- * synchronisations per step) and the x halves come from one product over all T*B rows; otherwise a loop
+ * synchronisations per step; one, and no partial sums, when the drawn pattern keeps at most 256 units, see
+ * ARD_OPT_LSTM_COMPACT_H) and the x halves come from one product over all T*B rows; otherwise a loop
  * in native code enqueues ard_lstm_gates_bwd and ard_lstm_gate_gemm_bwd per step.  In both cases the h
  * halves of D[1..T-1] are overwritten (kept units: the total gradient of h_{t-1}; dropped units:
  * unspecified), and the h half of D[0] is meaningful at kept units only. */
