@@ -581,7 +581,9 @@ ard_status ard_lstm_gate_gemm_bwd(ard_ctx* ctx, const ard_pattern* pat, int B, i
  * whole sequence and synchronises the SMs once per step (every wait bounded, see ARD_ERR_TIMEOUT); Z is
  * then not used.  Otherwise, or after ard_set_lstm_persistent(ctx, 0), it is a loop in native code that
  * enqueues ard_lstm_gate_gemm and ard_lstm_gates per step.  Both give the same C, G and XH up to
- * summation order.
+ * summation order.  Under a pattern that drops units the kernel contracts over the kept units of h_{t-1} only
+ * (ARD_OPT_LSTM_COMPACT_H): it keeps a compact copy of h in scratch of the context, next to the grid-barrier
+ * counter the whole-sequence kernels share, so one whole-sequence call at a time per context.
  *   XH [T+1][B][I+H] bf16: the caller fills the x halves of XH[0..T-1] and the h half of XH[0] (h_0, zeros at
  *   dropped units); C [T+1][B][H] fp32 compact cell states, C[0] = c_0; G [T][B][4H] fp32 saved gates;
  *   Z [B][4H] fp32 scratch; W [4H][I+H] bf16 (ldw); bias [4][H] or NULL. */
