@@ -233,3 +233,73 @@ def test_both_forms_of_the_bptt_recurrence_match_the_oracle(T, B, I, H, periods)
         ard.ard_set_option(ctx.h, ard.ARD_OPT_LSTM_COMPACT_H, 1)
     finally:
         ctx.close()
+
+
+def test_a_sequence_replays_from_a_cuda_graph_with_a_new_pattern_each_time():
+    """Sampler (device-resident iteration counter), whole-sequence forward and whole-sequence BPTT captured once into
+    a CUDA graph: every replay draws the next pattern, and the kernels choose their form on the device from it
+    (full contraction at a period of 1, compact h and partial sums at 2 - 3, compact h and one barrier per step
+    from 4 on at this size).  Outputs against the oracle for the oracle's draw of the same iteration."""
+    from distributions import max_entropy_K
+    T, B, I, H = 3, 8, 64, 1024
+    KH = I + H
+    rng = np.random.default_rng(2024)
+    W = inputs.bf16_round(rng.uniform(-0.05, 0.05, size=(KH, 4 * H)).astype(np.float32))
+    X = inputs.bf16_round(rng.standard_normal((T, B, I)).astype(np.float32))
+    dH = (rng.standard_normal((T, B, H)) / 8).astype(np.float32)
+    ctx = Ctx(1 << 20)
+    try:
+        Kd = max_entropy_K(0.6, 8)
+        cdf = ard.ard_quantise_distribution(Kd)
+        ard.ard_set_distribution(ctx.h, 0, Kd)
+        pat = ctx.pattern(ard.ARD_ROW, KH, H)
+        counter = torch.zeros(1, dtype=torch.int64, device="cuda")
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            Wnm = torch.from_numpy(np.ascontiguousarray(W.T)).to(BF).cuda()
+            XH = torch.zeros((T + 1, B, KH), dtype=BF, device="cuda")
+            XH[:T, :, :I] = torch.from_numpy(X).to(BF).cuda()
+            C = torch.zeros((T + 1, B, H), dtype=torch.float32, device="cuda")
+            G = torch.zeros((T, B, 4 * H), dtype=torch.float32, device="cuda")
+            Z = torch.zeros((B, 4 * H), dtype=torch.float32, device="cuda")
+            DZ = torch.zeros((T, B, 4 * H), dtype=BF, device="cuda")
+            D = torch.zeros((T, B, KH), dtype=torch.float32, device="cuda")
+            D0 = torch.zeros((T, B, KH), dtype=torch.float32, device="cuda")
+            D0[1:, :, I:] = torch.from_numpy(dH[:-1]).cuda()
+            dc = torch.zeros((B, H), dtype=torch.float32, device="cuda")
+            dW = torch.zeros((4 * H, KH), dtype=torch.float32, device="cuda")
+            dh_last = torch.from_numpy(dH[T - 1]).cuda().contiguous()
+            alpha = 1.0 / (1.0 - 0.6)
+
+            def seq(cs):
+                ard.ard_sample_pattern_counter(ctx.h, pat, 0, 31, 900, counter, 1, 5, cs)
+                C[1:].zero_()
+                D.copy_(D0)
+                dc.zero_()
+                ard.ard_lstm_forward(ctx.h, pat, T, B, I, H, alpha, XH, Wnm, KH, None, C, G, Z, cs)
+                ard.ard_lstm_backward(ctx.h, pat, T, B, I, H, alpha, XH, Wnm, KH, C, G, dh_last, D, dc, DZ, dW, cs)
+
+            seq(s.cuda_stream)  # one ordinary call first (iteration 900)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                seq(s.cuda_stream)
+            seen = set()
+            for it in range(1, 9):
+                g.replay()
+                torch.cuda.synchronize()
+                assert int(counter.item()) == it + 1
+                dp, b = OP.draw(cdf, 31, 900 + it, 5)
+                seen.add(1 if dp == 1 else (2 if dp <= 3 else 3))
+                m = OP.row_mask(H, dp, b)
+                keep = OP.row_keep(H, dp, b)
+                fw = OL.fwd(X, W, None, m, alpha)
+                bw = OL.bwd(fw, W, m, alpha, dH)
+                assert OG.rel_fro(host(XH[1:, :, I:].float()), fw["Hs"]) <= TOL[ard.ARD_BF16], (it, dp, b)
+                assert OG.rel_fro(host(D[:, :, :I]), bw["dX"]) <= TOL[ard.ARD_BF16], (it, dp, b)
+                assert OG.rel_fro(host(dW), bw["dW"].T) <= TOL[ard.ARD_BF16], (it, dp, b)
+                assert OG.rel_fro(host(dc[:, :len(keep)]), bw["dc0"][:, keep]) <= TOL[ard.ARD_BF16], (it, dp, b)
+            assert len(seen) >= 2, seen
+        assert ard.ard_last_device_status(ctx.h) == 0
+    finally:
+        ctx.close()
