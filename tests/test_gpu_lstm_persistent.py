@@ -39,7 +39,7 @@ def _run(ctx, pat, T, B, I, H, Wnm, X, bias, h0, c0, keep, alpha, persistent):
     return XH[1:, :, I:].float(), C, G, launches
 
 
-@pytest.mark.parametrize("T,B,I,H", [(6, 33, 128, 264), (4, 128, 192, 64), (3, 1, 64, 1024)])
+@pytest.mark.parametrize("T,B,I,H", [(6, 33, 128, 264), (4, 128, 192, 64), (3, 1, 64, 1024), (1, 5, 64, 128)])
 def test_persistent_forward_matches_the_oracle_and_the_per_step_path(T, B, I, H):
     rng = np.random.default_rng(T * 1000 + B)
     W = inputs.bf16_round(rng.uniform(-0.08, 0.08, size=(I + H, 4 * H)).astype(np.float32))
@@ -138,7 +138,7 @@ def test_layers_that_do_not_fit_use_the_per_step_path():
         ctx.close()
 
 
-@pytest.mark.parametrize("T,B,I,H", [(5, 33, 128, 264), (3, 128, 64, 128), (4, 7, 192, 1024)])
+@pytest.mark.parametrize("T,B,I,H", [(5, 33, 128, 264), (3, 128, 64, 128), (4, 7, 192, 1024), (1, 5, 64, 128)])
 def test_persistent_bptt_matches_the_oracle_and_the_per_step_path(T, B, I, H):
     """Whole-sequence BPTT kernel: dX, dW, dh_0, dc_0 against the oracle and against the per-step path."""
     from paper_2203_05705_b200.lstm import LstmLayer
