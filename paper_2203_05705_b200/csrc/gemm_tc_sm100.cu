@@ -29,6 +29,7 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;  // 64 bf16 = 128 bytes = one swizzle row
 constexpr int TC_THREADS = 320;  // warp 0 producer, warp 1 MMA, warps 2..9 epilogue
+constexpr int TC_THREADS_CLASS = TC_THREADS + 32;  // class form of the tile pattern: warp 10 is a second producer
 constexpr int ROWS_GATHER_WARPS = 4;  // row-list products: warp 0 and warps 10..12 gather (one warp cannot issue enough copies)
 constexpr int TC_THREADS_ROWS = TC_THREADS + 32 * (ROWS_GATHER_WARPS - 1);
 constexpr int EPI_WARPS = 8;
@@ -67,8 +68,10 @@ __host__ __device__ constexpr bool b_is_mn(int mode) {
   return mode != M_ROW_FWD && mode != M_TILE_FWD && mode != M_TILEC_FWD && mode != M_LSTM_FWD && mode != M_ROWS_FWD;
 }
 __host__ __device__ constexpr bool is_rows_mode(int mode) { return mode >= M_ROWS_FWD && mode <= M_ROWS_BWD_WEIGHT; }
-__host__ __device__ constexpr int tc_threads(int mode) { return is_rows_mode(mode) ? TC_THREADS_ROWS : TC_THREADS; }
 __host__ __device__ constexpr bool is_class_mode(int mode) { return mode >= M_TILEC_FWD && mode <= M_TILEC_BWD_WEIGHT; }
+__host__ __device__ constexpr int tc_threads(int mode) {
+  return is_rows_mode(mode) ? TC_THREADS_ROWS : (is_class_mode(mode) ? TC_THREADS_CLASS : TC_THREADS);
+}
 __host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 4 : (bn == 128 ? 6 : 8); }
 __host__ __device__ constexpr int tmem_cols_for(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }
 
@@ -713,7 +716,7 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
     const bool fits = n_list * 4 <= CLASS_LIST_BYTES - 1024;
     if (threadIdx.x == 0) sch.build_class_table(p, tab, total_smem);
     if (fits)
-      for (int i = threadIdx.x; i < n_list; i += TC_THREADS) slist[i] = sch.list[i];
+      for (int i = threadIdx.x; i < n_list; i += (int)blockDim.x) slist[i] = sch.list[i];
     __syncthreads();
     sch.ctab = tab;
     sch.total = total_smem[0];
@@ -830,16 +833,26 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
-  } else if (warp == 0) {
-    // ===================== TMA producer =====================
-    // The whole warp first turns the descriptors it was given into those of the sampled pattern (the first
-    // operand stage is free until the first load and serves as the 128-byte work area of each).
+  } else if (warp == 0 || (is_class_mode(MODE) && warp == 10)) {
+    // ===================== TMA producers =====================
+    // In the class form of the tile pattern two threads issue the copies, lane 0 of warp 0 the even contraction
+    // blocks (counted over all tiles of the CTA) and lane 0 of warp 10 the odd ones: there a thread spends ~160
+    // cycles in each copy instruction, three or four per block, and one thread alone paced the product (0.44 us per
+    // block where the MMAs need 0.34; -10 to -25 % per product with two).  Everywhere else one thread keeps up, and a
+    // second one gains nothing (the row form's weight gradient was 4 % slower with the eleventh warp merely present):
+    // only the class-form kernels have warp 10, and it stays idle in their dense draws.
+    constexpr bool TWO = is_class_mode(MODE) && !PLAIN;
+    // Warp 0 first turns the descriptors it was given into those of the sampled pattern (the first
+    // operand stage is free until the first load and serves as the 128-byte work area of each); warp 10 works out
+    // the same addresses and waits for it.
+    const int me = warp == 0 ? 0 : 1;
     const int32_t* hin = (FUSED && p.hdr_in != nullptr) ? p.hdr_in : p.hdr;
     const uint32_t smid = sm_id();
     CUtensorMap* slots = p.tm_slots + (size_t)(smid < (uint32_t)ARD_TM_SM_MAX ? smid : 0u) * ARD_TM_SLOTS;
     auto special = [&](int mi, int indexed, int slot) -> const CUtensorMap* {
       const int32_t* h = indexed == 2 ? hin : p.hdr;
       if (indexed == 0) return &p.maps[mi].tm;
+      if (me == 1) return tensormap_specialised_address(&p.maps[mi], h[HDR_DP], slots + slot);
       return tensormap_specialise(&p.maps[mi], h[HDR_DP], h[HDR_B], h[HDR_NKEEP], smem + 128 * slot, slots + slot, lane);
     };
     const CUtensorMap* mapA = special(0, p.mapA_indexed, 0);
@@ -853,7 +866,8 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
         if (MODE == M_LSTM_FWD || MODE == M_LSTM_BWD_DATA) mapB4[g] = special(6 + g, 1, 6 + g);
       }
     }
-    fence_proxy_async_smem();  // the work area is about to be overwritten by asynchronous copies
+    if (me == 0) fence_proxy_async_smem();  // the work area is about to be overwritten by asynchronous copies
+    if (is_class_mode(MODE)) asm volatile("bar.sync 3, 64;" ::: "memory");  // the rewritten descriptors are in global memory
     if (smid >= (uint32_t)ARD_TM_SM_MAX) {  // more SMs than the scratch was laid out for: refuse rather than share a slot
       if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (int)ARD_ERR_UNSUPPORTED); }
     } else if (lane == 0) {
@@ -873,6 +887,7 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
       }
       int stage = 0;
       uint32_t phase = 0;
+      int turn = 0;  // whose block this is: blocks alternate between the two producers over all tiles
       bool ok = true;
       Unit un;
       for (int i = 0; ok && sch.unit(w0, i, un); ++i) {
@@ -882,7 +897,18 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
         // walk of the kept-block list: entry li, 64-wide piece `sub` of that pattern tile
         int li = 0, sub = 0;
         int kbase = (ti.klist != nullptr && ti.nkb > 0) ? ti.klist[0] * p.ts : 0;
-        for (int kb = kb_begin; kb < kb_end; ++kb) {
+        if (!TWO && me == 1) break;  // one producer only
+        for (int kb = kb_begin; kb < kb_end; ++kb, turn ^= TWO ? 1 : 0) {
+          if (turn != me) {
+            // the other producer's block: only the walk moves on
+            if (ti.klist != nullptr && ++sub == ti.kper) {
+              sub = 0;
+              ++li;
+              if (kb + 1 < ti.nkb) kbase = ti.klist[li] * p.ts;
+            }
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            continue;
+          }
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sA = base + stage * L::STAGE_BYTES;
           const uint32_t sB = sA + L::A_BYTES;

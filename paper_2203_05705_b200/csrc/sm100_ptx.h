@@ -140,6 +140,15 @@ __device__ __forceinline__ const CUtensorMap* tensormap_specialise(const TcMap* 
   return slot;
 }
 
+// Where tensormap_specialise leaves (or finds) the descriptor, without doing anything: for a second thread that
+// issues copies through the same descriptors.
+__device__ __forceinline__ const CUtensorMap* tensormap_specialised_address(const TcMap* m, int dp, const CUtensorMap* slot) {
+  const int variant = m->variant;
+  const bool dense_elsewhere = variant == MAP_COMPACT_COLS && dp == 1 && m->dense_base != nullptr;
+  if (variant == MAP_PLAIN || (dp == 1 && !dense_elsewhere)) return &m->tm;
+  return slot;
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols)
                : "memory");
