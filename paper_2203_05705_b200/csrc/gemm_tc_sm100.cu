@@ -69,8 +69,11 @@ __host__ __device__ constexpr bool b_is_mn(int mode) {
 }
 __host__ __device__ constexpr bool is_rows_mode(int mode) { return mode >= M_ROWS_FWD && mode <= M_ROWS_BWD_WEIGHT; }
 __host__ __device__ constexpr bool is_class_mode(int mode) { return mode >= M_TILEC_FWD && mode <= M_TILEC_BWD_WEIGHT; }
+__host__ __device__ constexpr bool has_second_producer(int mode) {
+  return is_class_mode(mode) || mode == M_TILE_FWD || mode == M_TILE_BWD_DATA || mode == M_TILE_BWD_WEIGHT;
+}
 __host__ __device__ constexpr int tc_threads(int mode) {
-  return is_rows_mode(mode) ? TC_THREADS_ROWS : (is_class_mode(mode) ? TC_THREADS_CLASS : TC_THREADS);
+  return is_rows_mode(mode) ? TC_THREADS_ROWS : (has_second_producer(mode) ? TC_THREADS_CLASS : TC_THREADS);
 }
 __host__ __device__ constexpr int stages_for(int bn) { return bn == 256 ? 4 : (bn == 128 ? 6 : 8); }
 __host__ __device__ constexpr int tmem_cols_for(int bn) { return 2 * bn < 32 ? 32 : 2 * bn; }
@@ -833,15 +836,16 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
     }
-  } else if (warp == 0 || (is_class_mode(MODE) && warp == 10)) {
+  } else if (warp == 0 || (has_second_producer(MODE) && warp == 10)) {
     // ===================== TMA producers =====================
-    // In the class form of the tile pattern two threads issue the copies, lane 0 of warp 0 the even contraction
+    // In the class form of the tile pattern (and in the tile-list kernels) two threads issue the copies, lane 0 of warp 0 the even contraction
     // blocks (counted over all tiles of the CTA) and lane 0 of warp 10 the odd ones: there a thread spends ~160
     // cycles in each copy instruction, three or four per block, and one thread alone paced the product (0.44 us per
     // block where the MMAs need 0.34; -10 to -25 % per product with two).  Everywhere else one thread keeps up, and a
     // second one gains nothing (the row form's weight gradient was 4 % slower with the eleventh warp merely present):
-    // only the class-form kernels have warp 10, and it stays idle in their dense draws.
-    constexpr bool TWO = is_class_mode(MODE) && !PLAIN;
+    // only the class-form kernels and the tile-list kernels have warp 10, and it stays idle in the class form's
+    // dense draws.
+    constexpr bool TWO = has_second_producer(MODE) && !(is_class_mode(MODE) && PLAIN);
     // Warp 0 first turns the descriptors it was given into those of the sampled pattern (the first
     // operand stage is free until the first load and serves as the 128-byte work area of each); warp 10 works out
     // the same addresses and waits for it.
@@ -867,7 +871,7 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
       }
     }
     if (me == 0) fence_proxy_async_smem();  // the work area is about to be overwritten by asynchronous copies
-    if (is_class_mode(MODE)) asm volatile("bar.sync 3, 64;" ::: "memory");  // the rewritten descriptors are in global memory
+    if (has_second_producer(MODE)) asm volatile("bar.sync 3, 64;" ::: "memory");  // the rewritten descriptors are in global memory
     if (smid >= (uint32_t)ARD_TM_SM_MAX) {  // more SMs than the scratch was laid out for: refuse rather than share a slot
       if (lane == 0) { *abort_flag = 1; atomicMax(p.status, (int)ARD_ERR_UNSUPPORTED); }
     } else if (lane == 0) {
