@@ -411,31 +411,69 @@ struct Sched {
     if (MODE == M_TILEC_BWD_WEIGHT) return ((cnt + qm - 1) / qm) * ((len + qn - 1) / qn);
     return Mt * ((cnt + qn - 1) / qn);
   }
-  // One thread fills the per-class table in shared memory (at most 64 classes); callers synchronise.
-  // Classes that keep something come first, the empty ones (whose items only write zeros) after them; an entry
-  // is {first item, list offset, list length, members | class << 16}.  out[0] = number of items, out[1] = items
-  // of the non-empty classes, out[2] = how many zero items cost about as much as one of the others.
-  __device__ void build_class_table(const TcParams& p, int4* tab, int* out) const {
-    const int32_t* ptr = (MODE == M_TILEC_BWD_DATA) ? p.row_ptr : p.col_ptr;
-    int run = 0, slot = 0, heavy = 0;
-    long long blocks = 0;
-    for (int pass = 0; pass < 2; ++pass) {
-      for (int c = 0; c < nclass; ++c) {
-        const int off = ptr[c], len = ptr[c + 1] - off;
-        if ((len == 0) != (pass == 1)) continue;
-        const int cnt = class_members(c);
-        const int items = class_items(cnt, len);
-        tab[slot++] = make_int4(run, off, len, cnt | (c << 16));
-        run += items;
-        blocks += (long long)items * len * (p.ts >> 6);
-      }
-      if (pass == 0) heavy = run;
+  // One warp fills the per-class table in shared memory (at most 64 classes: two per lane, so the list pointers of
+  // all classes come back in one round trip; a single thread walking them took ~2.5 us of every launch); callers
+  // synchronise.
+  // Classes that keep something come first, the empty ones (whose items only write zeros) after them, each group
+  // by class number; an entry is {first item, list offset, list length, members | class << 16}.  out[0] = number of
+  // items, out[1] = items of the non-empty classes, out[2] = how many zero items cost about as much as one of the
+  // others.
+  __device__ static int warp_excl_scan(int v, int lane, int& total) {
+    int x = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, d);
+      if (lane >= d) x += y;
     }
-    out[0] = run;
-    out[1] = heavy;
-    // an item that only writes zeros takes about as long as 14 contraction blocks
-    const int avg = heavy > 0 ? (int)(blocks / heavy) : 0;
-    out[2] = min(64, max(1, (avg + 14) / 14));
+    total = __shfl_sync(0xffffffffu, x, 31);
+    return x - v;
+  }
+  __device__ void build_class_table(const TcParams& p, int4* tab, int* out, int lane) const {
+    const int32_t* ptr = (MODE == M_TILEC_BWD_DATA) ? p.row_ptr : p.col_ptr;
+    int off[2], len[2], cnt[2], items[2];
+    bool valid[2], full[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int c = lane + 32 * h;
+      valid[h] = c < nclass;
+      off[h] = valid[h] ? ptr[c] : 0;
+      len[h] = valid[h] ? ptr[c + 1] - off[h] : 0;
+      cnt[h] = valid[h] ? class_members(c) : 0;
+      items[h] = valid[h] ? class_items(cnt[h], len[h]) : 0;
+      full[h] = valid[h] && len[h] != 0;
+    }
+    const unsigned lt = (1u << lane) - 1u;
+    const unsigned mf0 = __ballot_sync(0xffffffffu, full[0]), mf1 = __ballot_sync(0xffffffffu, full[1]);
+    const unsigned me0 = __ballot_sync(0xffffffffu, valid[0] && !full[0]), me1 = __ballot_sync(0xffffffffu, valid[1] && !full[1]);
+    const int n_full = __popc(mf0) + __popc(mf1);
+    int tA, tB, tC, tD;
+    const int sA = warp_excl_scan(full[0] ? items[0] : 0, lane, tA);
+    const int sB = warp_excl_scan(full[1] ? items[1] : 0, lane, tB);
+    const int sC = warp_excl_scan(valid[0] && !full[0] ? items[0] : 0, lane, tC);
+    const int sD = warp_excl_scan(valid[1] && !full[1] ? items[1] : 0, lane, tD);
+    if (valid[0]) {
+      const int slot = full[0] ? __popc(mf0 & lt) : n_full + __popc(me0 & lt);
+      const int run = full[0] ? sA : tA + tB + sC;
+      tab[slot] = make_int4(run, off[0], len[0], cnt[0] | (lane << 16));
+    }
+    if (valid[1]) {
+      const int slot = full[1] ? __popc(mf0) + __popc(mf1 & lt) : n_full + __popc(me0) + __popc(me1 & lt);
+      const int run = full[1] ? tA + sB : tA + tB + tC + sD;
+      tab[slot] = make_int4(run, off[1], len[1], cnt[1] | ((lane + 32) << 16));
+    }
+    // contraction blocks of the non-empty classes' items
+    long long blocks = (full[0] ? (long long)items[0] * len[0] : 0) + (full[1] ? (long long)items[1] * len[1] : 0);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) blocks += __shfl_xor_sync(0xffffffffu, blocks, d);
+    blocks *= (p.ts >> 6);
+    if (lane == 0) {
+      const int heavy = tA + tB;
+      out[0] = heavy + tC + tD;
+      out[1] = heavy;
+      // an item that only writes zeros takes about as long as 14 contraction blocks
+      const int avg = heavy > 0 ? (int)(blocks / heavy) : 0;
+      out[2] = min(64, max(1, (avg + 14) / 14));
+    }
   }
   __device__ TileInfo class_tile(const TcParams& p, int t) const {
     TileInfo ti;
@@ -717,7 +755,7 @@ ard_gemm_tc_kernel(const __grid_constant__ TcParamsT<nmaps(MODE)> p) {
     int* total_smem = reinterpret_cast<int*>(smem + L::MISC_OFF + 8);  // [3]: items, items of non-empty classes, light_q
     int32_t* slist = reinterpret_cast<int32_t*>(smem + L::STG_OFF);
     const bool fits = n_list * 4 <= CLASS_LIST_BYTES - 1024;
-    if (threadIdx.x == 0) sch.build_class_table(p, tab, total_smem);
+    if (warp == 0) sch.build_class_table(p, tab, total_smem, lane);
     if (fits)
       for (int i = threadIdx.x; i < n_list; i += (int)blockDim.x) slist[i] = sch.list[i];
     __syncthreads();
