@@ -4,6 +4,7 @@
 """
 from __future__ import annotations
 
+import hashlib
 import os
 import subprocess
 import sys
@@ -32,6 +33,29 @@ def _stale(target, deps):
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def _sha(paths, extra=""):
+    h = hashlib.sha256(extra.encode())
+    for p in paths:
+        with open(p, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def _object_is_current(obj, deps, flags):
+    """An object counts only if it was made by this script from the sources as they are now: its side file holds
+    the hash of the sources (and flags) it was compiled from and the hash of the object itself, so an object written
+    by anything else (an experiment's build, an older checkout with newer time stamps) is compiled again."""
+    key = obj + ".key"
+    if not (os.path.exists(obj) and os.path.exists(key)):
+        return False
+    try:
+        with open(key) as f:
+            src_hash, obj_hash = f.read().split()
+    except ValueError:
+        return False
+    return src_hash == _sha(deps, " ".join(flags)) and obj_hash == _sha([obj])
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".h")]
@@ -42,9 +66,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
         s = os.path.join(CSRC, src)
         o = os.path.join(OBJ, src[:-3] + ".o")
         objs.append(o)
-        if force or _stale(o, [s] + headers):
+        deps = [s] + sorted(headers)
+        if force or not _object_is_current(o, deps, FLAGS):
             cmd = [NVCC] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
-            jobs.append(cmd)
+            jobs.append((cmd, o, deps))
 
     def run(cmd):
         r = subprocess.run(cmd, capture_output=True, text=True)
@@ -52,8 +77,15 @@ def build(force: bool = False, verbose: bool = False) -> str:
             raise RuntimeError("nvcc failed:\n" + " ".join(cmd) + "\n" + r.stdout + r.stderr)
         return r.stderr
 
+    def compile_one(job):
+        cmd, o, deps = job
+        out = run(cmd)
+        with open(o + ".key", "w") as f:
+            f.write(_sha(deps, " ".join(FLAGS)) + " " + _sha([o]))
+        return out
+
     with ThreadPoolExecutor(max_workers=max(1, min(6, len(jobs)))) as ex:
-        for out in ex.map(run, jobs):
+        for out in ex.map(compile_one, jobs):
             if verbose and out:
                 print(out)
     if jobs or force or _stale(LIB, objs):
